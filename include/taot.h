@@ -1,0 +1,204 @@
+/*
+ * taot.h -- C ABI of the TAOT replica-placement planner for one NVIDIA B200 (sm_100a).
+ *
+ * The planner turns one micro-batch of MoE router decisions into an executable guest-replica
+ * schedule.  Per problem (one MoE layer x one micro-batch; L problems per call, all
+ * independent) it runs, on the GPU and without ever returning to the host:
+ *
+ *   taot_histogram      token loads n[r][e], per-expert and per-rank loads   (Appendix A.1)
+ *   taot_excess_spare   overload / spare capacity against the integer mean   (Appendix A.1)
+ *   taot_sinkhorn       Phase 1: entropic OT by Sinkhorn-Knopp over the rank-by-rank topology
+ *                       cost, giving the flow hint T                         (Appendix A.2)
+ *   taot_match          Phase 2: column-priority integer replica matching    (Appendix A.3, Alg. 2)
+ *                       Phase 3: Lagrangian auction, rank -> slot counts X   (Appendix A.4, Alg. 3)
+ *   taot_assign         deterministic token -> replica rewrite of the routing table
+ *   taot_plan           all of the above chained on one stream
+ *   taot_plan_host      taot_plan with host buffers (copies in and out on the same stream)
+ *
+ * Conventions
+ *   - Shapes: L problems, R ranks, E experts, K guest slots per rank, S = R*K slots
+ *     (slot s = r*K + kappa lives on rank s / K), router top-k = k, T tokens per problem,
+ *     T % R == 0; source rank of token t is t / (T/R).  All arrays are dense, row-major,
+ *     in the index order written next to them.
+ *   - Every pointer named d_* is DEVICE memory owned by the caller; h_* is HOST memory owned by
+ *     the caller.  The library allocates device memory only inside taot_create (a few copies of
+ *     the topology) and frees it in taot_destroy; scratch space is the caller's `ws`
+ *     (taot_workspace_bytes bytes, 256-byte aligned).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
+ *     enqueue work and return; they never synchronise (except taot_create / taot_destroy).
+ *   - Return value: TAOT_OK, or a negative taot_status found on the host before anything was
+ *     launched.  Data-dependent conditions never fault or trap: they are OR-ed into d_info[l]
+ *     (TAOT_INFO_* bits).  The caller zeroes d_info before the first stage it runs; taot_plan
+ *     and taot_plan_host zero it themselves.
+ *   - Same inputs give the same output bits on every call.
+ */
+#ifndef TAOT_H
+#define TAOT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct taot_handle_s* taot_handle_t;
+
+typedef enum {
+    TAOT_OK = 0,
+    TAOT_ERR_NULL = -1,         /* a required pointer is NULL */
+    TAOT_ERR_PARAM = -2,        /* a parameter is out of its documented range */
+    TAOT_ERR_UNSUPPORTED = -3,  /* a size is valid but beyond what this build supports */
+    TAOT_ERR_CUDA = -4,         /* a CUDA runtime call failed (see cudaGetLastError) */
+    TAOT_ERR_ALIGN = -5         /* a device pointer is not aligned as required */
+} taot_status;
+
+/* bits of d_info[l] */
+enum {
+    TAOT_INFO_BAD_INDEX = 1,        /* topk_idx held a value outside [0, E): skipped / copied through */
+    TAOT_INFO_SINKHORN_CAP = 2,     /* tolerance mode reached max_iters above tol */
+    TAOT_INFO_NONFINITE = 4,        /* a non-finite value appeared in the Sinkhorn solve */
+    TAOT_INFO_AUCTION_RESIDUAL = 8, /* the auction stopped at auction_max_rounds with tokens unplaced */
+    TAOT_INFO_SUPPLY_SCALED = 16,   /* sum(s) > sum(d): supply was scaled by gamma < 1 */
+    TAOT_INFO_SINKHORN_SIZE = 32    /* |hot| * |cold| exceeds the on-chip capacity: plan left at zero */
+};
+
+/*
+ * Problem description.  Set struct_size = sizeof(taot_params).
+ * Supported ranges: 1 <= R <= 256, 1 <= E <= 1024, 1 <= K <= 8, 1 <= k <= 64, L >= 1,
+ * T >= R, T % R == 0, T*k < 2^31.
+ */
+typedef struct {
+    int32_t struct_size;
+    int32_t L;                  /* problems per call */
+    int32_t R;                  /* expert-parallel ranks */
+    int32_t E;                  /* experts */
+    int32_t K;                  /* guest slots per rank */
+    int32_t k;                  /* router top-k */
+    int64_t T;                  /* tokens per problem */
+    float   eps;                /* entropic regulariser (absolute, same unit as C), > 0 */
+    int32_t max_iters;          /* Sinkhorn iterations if tol <= 0, iteration cap otherwise; >= 1 */
+    float   tol;                /* stop once sum_i |rowsum_i - s~_i| <= tol * sum(s~); <= 0: fixed count */
+    int32_t check_every;        /* test the tolerance every this many iterations (>= 1) */
+    float   eps0;               /* the paper's epsilon_0 safeguard constant, e.g. 1e-8f */
+    float   price_step;         /* Phase-3 price increment, e.g. 0.1f */
+    int32_t auction_max_rounds; /* <= 0: run the auction to completion */
+} taot_params;
+
+/* Outputs of taot_plan / taot_plan_host: device pointers (host pointers for the _host call).
+ * Optional members may be NULL and are then kept in workspace only. */
+typedef struct {
+    int32_t* n;             /* [L,R,E]   tokens rank r sends to expert e */
+    int32_t* expert_load;   /* [L,E] */
+    int32_t* rank_load;     /* [L,R] */
+    int32_t* excess;        /* [L,R]     optional */
+    int32_t* spare;         /* [L,R]     optional */
+    float*   plan;          /* [L,R,R]   Phase-1 flow hint T, in tokens */
+    int32_t* sinkhorn_iters;/* [L] */
+    float*   row_err;       /* [L]       relative row-marginal violation at the returned iterate */
+    int32_t* slot_expert;   /* [L,R,K]   expert placed in slot (r, kappa), -1 = empty */
+    int32_t* slot_tokens;   /* [L,R,K]   tokens planned for that slot (the paper's A_es) */
+    int32_t* X;             /* [L,R,S]   tokens source rank r sends to slot s */
+    int32_t* rounds;        /* [L,2]     optional: Phase-2 inner rounds, Phase-3 rounds */
+    int32_t* new_idx;       /* [L,T,k]   rewritten routing table: e, or E + s for a guest slot */
+    int32_t* info;          /* [L]       TAOT_INFO_* bits */
+} taot_outputs;
+
+/*
+ * Create a planner for a fixed topology.  (Problem Formulation: R, E, home ranks r_e, cost W.)
+ *   h_e2r [E]   home rank of each expert, each in [0, R)
+ *   h_C  [R,R]  communication cost from row rank to column rank, finite, >= 0
+ *   h_B  [R,R]  topology preference (Appendix A.3: 1 intra-node, w_inter < 1 inter-node, 0 home),
+ *               or NULL to derive it from C: B_ii = 0, B_ij = min(1, c_min / C_ij) with c_min the
+ *               smallest positive off-diagonal cost (1 where C_ij <= 0).
+ * All three are HOST arrays, copied during the call (which synchronises the device).
+ * Errors: TAOT_ERR_NULL, TAOT_ERR_PARAM (ranges above, bad e2r entry, non-finite cost, eps <= 0),
+ * TAOT_ERR_UNSUPPORTED, TAOT_ERR_CUDA.  On error *out is NULL.
+ */
+int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_e2r,
+                const float* h_C, const float* h_B);
+
+/* Frees the handle's device copies.  Synchronises the device.  NULL is accepted. */
+int taot_destroy(taot_handle_t h);
+
+/* Scratch bytes taot_* calls need in `ws` for this handle (device memory, 256-byte aligned). */
+int taot_workspace_bytes(taot_handle_t h, size_t* bytes);
+
+/* Device scratch bytes taot_plan_host needs (staging of inputs/outputs plus the workspace). */
+int taot_host_workspace_bytes(taot_handle_t h, size_t* bytes);
+
+/*
+ * Load collection (Appendix A.1: n_re, and l_r = sum over r's experts of sum_r' n_r'e).
+ *   d_topk [L,T,k] int32, 4-byte aligned (16-byte alignment enables the vector path).
+ *   d_n [L,R,E], d_expert_load [L,E], d_rank_load [L,R]: fully overwritten.
+ * Side effect: per-chunk counts stay in `ws` for a later taot_assign(..., reuse_counts = 1).
+ * An index outside [0, E) is skipped and sets TAOT_INFO_BAD_INDEX.
+ */
+int taot_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_n, int32_t* d_expert_load,
+                   int32_t* d_rank_load, int32_t* d_info, void* ws, void* stream);
+
+/*
+ * Excess / spare (Appendix A.1) against the integer mean m = floor(sum_r l_r / R), for B rows:
+ *   excess = max(l - m, 0), spare = max(m - l, 0); d_s / d_d receive the same as fp32
+ *   (the supply and demand vectors of Phase 1).  Any output pointer may be NULL.
+ */
+int taot_excess_spare(taot_handle_t h, const int32_t* d_rank_load, int32_t B, int32_t* d_excess,
+                      int32_t* d_spare, float* d_s, float* d_d, void* stream);
+
+/*
+ * Phase 1 (Appendix A.2).  For each of B problems: supply d_s[b,:], demand d_d[b,:] (fp32, >= 0),
+ * cost C and eps from the handle.  gamma = min(1, sum d / max(sum s, eps0)), s~ = gamma s;
+ * iterate u = s~/(M v), v = d/(M^T u) from v = 1, M = exp(-C/eps), for max_iters iterations or
+ * until the row-marginal test passes; T = diag(u) M diag(v) followed by the column cap
+ * T_ij *= min(1, d_j / (sum_i T_ij + eps0)).
+ *   d_plan [B,R,R] fp32 (fully overwritten), d_iters [B], d_row_err [B], d_info [B].
+ * The iterates are carried so that neither M nor u, v can under- or overflow for any C/eps.
+ */
+int taot_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
+                  int32_t* d_iters, float* d_row_err, int32_t* d_info, void* ws, void* stream);
+
+/*
+ * Phases 2 and 3 (Appendix A.3 / Algorithm 2, Appendix A.4 / Algorithm 3) for L problems.
+ * Spill comes from d_expert_load by cumulative-excess differencing within each rank; the score
+ * min(spill, spare) + alpha B + 0.1 alpha T_norm (alpha = m R / E) is evaluated in fp32 with one
+ * rounding per operation; both argmax ties go to the lowest index.
+ *   in : d_n [L,R,E], d_expert_load [L,E], d_rank_load [L,R], d_plan [L,R,R]
+ *   out: d_slot_expert [L,R,K], d_slot_tokens [L,R,K], d_X [L,R,S], d_rounds [L,2] (or NULL)
+ */
+int taot_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load,
+               const int32_t* d_rank_load, const float* d_plan, int32_t* d_slot_expert,
+               int32_t* d_slot_tokens, int32_t* d_X, int32_t* d_rounds, int32_t* d_info, void* ws,
+               void* stream);
+
+/*
+ * Token reassignment ("token routing is adjusted accordingly", Problem Formulation).  Within each
+ * (source rank, expert) group, in flat order t*k + j, the slots holding that expert take, lowest
+ * slot first, the first X[r][s] entries; an entry so taken is rewritten to E + s, the rest keep e.
+ *   d_new_idx [L,T,k] must not alias d_topk.
+ *   reuse_counts != 0: trust the per-chunk counts left in `ws` by taot_histogram on the same
+ *   d_topk; 0: recount (one more read of d_topk).
+ */
+int taot_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_slot_expert,
+                const int32_t* d_X, int32_t* d_new_idx, int32_t* d_info, void* ws,
+                int32_t reuse_counts, void* stream);
+
+/* The whole path on one stream; `out` holds DEVICE pointers. */
+int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* out, void* ws, void* stream);
+
+/*
+ * The whole path with HOST buffers: h_topk [L,T,k] is copied to the device, the path runs, and
+ * every non-NULL member of `out` (HOST pointers) is copied back, all enqueued on `stream`.
+ * Pinned host memory makes the copies asynchronous.  d_ws: taot_host_workspace_bytes bytes.
+ */
+int taot_plan_host(taot_handle_t h, const int32_t* h_topk, const taot_outputs* out, void* d_ws,
+                   void* stream);
+
+/* Kernels launched by the last call on this handle (for launch accounting). */
+int taot_last_launch_count(taot_handle_t h, int32_t* count);
+
+const char* taot_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TAOT_H */

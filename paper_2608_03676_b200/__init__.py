@@ -1,0 +1,20 @@
+"""B200-native TAOT replica-placement planner: thin Python binding over libtaot.so.
+
+Every step of the path runs in the CUDA library; this package only marshals torch device
+tensors into the C ABI declared in include/taot.h.  There is no CPU fallback: importing the
+binding without the compiled library raises.
+"""
+from .binding import (  # noqa: F401
+    Planner,
+    TaotError,
+    TaotParams,
+    INFO_BAD_INDEX,
+    INFO_SINKHORN_CAP,
+    INFO_NONFINITE,
+    INFO_AUCTION_RESIDUAL,
+    INFO_SUPPLY_SCALED,
+    INFO_SINKHORN_SIZE,
+    library_path,
+    load_library,
+    exported_symbols,
+)

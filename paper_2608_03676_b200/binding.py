@@ -1,0 +1,254 @@
+"""ctypes binding of include/taot.h.  Argument marshalling only."""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Dict, Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libtaot.so")
+_lib = None
+
+INFO_BAD_INDEX = 1
+INFO_SINKHORN_CAP = 2
+INFO_NONFINITE = 4
+INFO_AUCTION_RESIDUAL = 8
+INFO_SUPPLY_SCALED = 16
+INFO_SINKHORN_SIZE = 32
+
+_SYMBOLS = [
+    "taot_create", "taot_destroy", "taot_workspace_bytes", "taot_host_workspace_bytes",
+    "taot_histogram", "taot_excess_spare", "taot_sinkhorn", "taot_match", "taot_assign",
+    "taot_plan", "taot_plan_host", "taot_last_launch_count", "taot_status_string",
+]
+
+
+class TaotError(RuntimeError):
+    pass
+
+
+class TaotParams(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_int32), ("L", ctypes.c_int32), ("R", ctypes.c_int32),
+        ("E", ctypes.c_int32), ("K", ctypes.c_int32), ("k", ctypes.c_int32), ("T", ctypes.c_int64),
+        ("eps", ctypes.c_float), ("max_iters", ctypes.c_int32), ("tol", ctypes.c_float),
+        ("check_every", ctypes.c_int32), ("eps0", ctypes.c_float), ("price_step", ctypes.c_float),
+        ("auction_max_rounds", ctypes.c_int32),
+    ]
+
+
+class _Outputs(ctypes.Structure):
+    _fields_ = [(name, ctypes.c_void_p) for name in (
+        "n", "expert_load", "rank_load", "excess", "spare", "plan", "sinkhorn_iters", "row_err",
+        "slot_expert", "slot_tokens", "X", "rounds", "new_idx", "info")]
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def exported_symbols():
+    return list(_SYMBOLS)
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libtaot.so; raise if it has not been built (there is no other code path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise TaotError(f"{_LIB_PATH} is missing: build it with `python -m paper_2608_03676_b200.build`")
+        lib = ctypes.CDLL(_LIB_PATH)
+        for name in _SYMBOLS:
+            getattr(lib, name)                      # raises AttributeError if a symbol is absent
+        lib.taot_status_string.restype = ctypes.c_char_p
+        for name in _SYMBOLS:
+            if name != "taot_status_string":
+                getattr(lib, name).restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        msg = load_library().taot_status_string(rc).decode()
+        raise TaotError(f"{what}: {msg} ({rc})")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TaotError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+    return t
+
+
+@dataclass
+class PlanResult:
+    tensors: Dict[str, torch.Tensor]
+
+    def __getitem__(self, key):
+        return self.tensors[key]
+
+
+class Planner:
+    """One planner handle for a fixed topology (e2r, C, optional B) and problem shape."""
+
+    def __init__(self, L: int, R: int, E: int, K: int, k: int, T: int, e2r, C, eps: float,
+                 max_iters: int, tol: float = 0.0, check_every: int = 1, B=None, eps0: float = 1e-8,
+                 price_step: float = 0.1, auction_max_rounds: int = 0, device: Optional[torch.device] = None):
+        if not torch.cuda.is_available():
+            raise TaotError("the TAOT planner needs a CUDA device; there is no CPU path")
+        self.lib = load_library()
+        self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+        self.L, self.R, self.E, self.K, self.k, self.T = L, R, E, K, k, T
+        self.S = R * K
+        p = TaotParams(ctypes.sizeof(TaotParams), L, R, E, K, k, T, eps, max_iters, tol, check_every, eps0,
+                       price_step, auction_max_rounds)
+        self.params = p
+        e2r_h = torch.as_tensor(e2r, dtype=torch.int32).contiguous().cpu()
+        C_h = torch.as_tensor(C, dtype=torch.float32).contiguous().cpu()
+        B_h = None if B is None else torch.as_tensor(B, dtype=torch.float32).contiguous().cpu()
+        if e2r_h.numel() != E or C_h.numel() != R * R or (B_h is not None and B_h.numel() != R * R):
+            raise TaotError("e2r / C / B have the wrong number of elements")
+        self.handle = ctypes.c_void_p()
+        with torch.cuda.device(self.device):
+            _check(self.lib.taot_create(ctypes.byref(self.handle), ctypes.byref(p), _ptr(e2r_h), _ptr(C_h),
+                                        _ptr(B_h)), "taot_create")
+            n = ctypes.c_size_t()
+            _check(self.lib.taot_workspace_bytes(self.handle, ctypes.byref(n)), "taot_workspace_bytes")
+            self.ws_bytes = n.value
+            _check(self.lib.taot_host_workspace_bytes(self.handle, ctypes.byref(n)), "taot_host_workspace_bytes")
+            self.host_ws_bytes = n.value
+            self.ws = torch.empty(max(self.ws_bytes, 256), dtype=torch.uint8, device=self.device)
+        self._host_ws = None
+
+    def close(self):
+        if getattr(self, "handle", None) is not None and self.handle.value:
+            self.lib.taot_destroy(self.handle)
+            self.handle = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ------------------------------------------------------------------ allocation helpers
+    def _empty(self, shape, dtype):
+        return torch.empty(shape, dtype=dtype, device=self.device)
+
+    def alloc_outputs(self) -> Dict[str, torch.Tensor]:
+        L, R, E, K, S, T, k = self.L, self.R, self.E, self.K, self.S, self.T, self.k
+        i32, f32 = torch.int32, torch.float32
+        return dict(
+            n=self._empty((L, R, E), i32), expert_load=self._empty((L, E), i32), rank_load=self._empty((L, R), i32),
+            excess=self._empty((L, R), i32), spare=self._empty((L, R), i32), plan=self._empty((L, R, R), f32),
+            sinkhorn_iters=self._empty((L,), i32), row_err=self._empty((L,), f32),
+            slot_expert=self._empty((L, R, K), i32), slot_tokens=self._empty((L, R, K), i32),
+            X=self._empty((L, R, S), i32), rounds=self._empty((L, 2), i32), new_idx=self._empty((L, T, k), i32),
+            info=torch.zeros((L,), dtype=i32, device=self.device))
+
+    def last_launch_count(self) -> int:
+        c = ctypes.c_int32()
+        _check(self.lib.taot_last_launch_count(self.handle, ctypes.byref(c)), "taot_last_launch_count")
+        return c.value
+
+    # ------------------------------------------------------------------ stages
+    def histogram(self, topk: torch.Tensor, info: Optional[torch.Tensor] = None):
+        _dev(topk, torch.int32, "topk")
+        L, R, E = self.L, self.R, self.E
+        n = self._empty((L, R, E), torch.int32)
+        el = self._empty((L, E), torch.int32)
+        rl = self._empty((L, R), torch.int32)
+        info = torch.zeros((L,), dtype=torch.int32, device=self.device) if info is None else info
+        _check(self.lib.taot_histogram(self.handle, _ptr(topk), _ptr(n), _ptr(el), _ptr(rl), _ptr(info),
+                                       _ptr(self.ws), _stream()), "taot_histogram")
+        return n, el, rl, info
+
+    def excess_spare(self, rank_load: torch.Tensor):
+        _dev(rank_load, torch.int32, "rank_load")
+        Bn, R = rank_load.shape
+        ex = self._empty((Bn, R), torch.int32); sp = self._empty((Bn, R), torch.int32)
+        s = self._empty((Bn, R), torch.float32); d = self._empty((Bn, R), torch.float32)
+        _check(self.lib.taot_excess_spare(self.handle, _ptr(rank_load), ctypes.c_int32(Bn), _ptr(ex), _ptr(sp),
+                                          _ptr(s), _ptr(d), _stream()), "taot_excess_spare")
+        return ex, sp, s, d
+
+    def sinkhorn(self, s: torch.Tensor, d: torch.Tensor, out: Optional[Dict[str, torch.Tensor]] = None):
+        _dev(s, torch.float32, "s"); _dev(d, torch.float32, "d")
+        Bn, R = s.shape
+        if out is None:
+            out = dict(plan=self._empty((Bn, R, R), torch.float32), iters=self._empty((Bn,), torch.int32),
+                       row_err=self._empty((Bn,), torch.float32),
+                       info=torch.zeros((Bn,), dtype=torch.int32, device=self.device))
+        _check(self.lib.taot_sinkhorn(self.handle, _ptr(s), _ptr(d), ctypes.c_int32(Bn), _ptr(out["plan"]),
+                                      _ptr(out["iters"]), _ptr(out["row_err"]), _ptr(out["info"]), _ptr(self.ws),
+                                      _stream()), "taot_sinkhorn")
+        return out
+
+    def match(self, n, expert_load, rank_load, plan, info: Optional[torch.Tensor] = None):
+        L, R, K, S = self.L, self.R, self.K, self.S
+        se = self._empty((L, R, K), torch.int32); stk = self._empty((L, R, K), torch.int32)
+        X = self._empty((L, R, S), torch.int32); rounds = self._empty((L, 2), torch.int32)
+        info = torch.zeros((L,), dtype=torch.int32, device=self.device) if info is None else info
+        _check(self.lib.taot_match(self.handle, _ptr(_dev(n, torch.int32, "n")),
+                                   _ptr(_dev(expert_load, torch.int32, "expert_load")),
+                                   _ptr(_dev(rank_load, torch.int32, "rank_load")),
+                                   _ptr(_dev(plan, torch.float32, "plan")), _ptr(se), _ptr(stk), _ptr(X),
+                                   _ptr(rounds), _ptr(info), _ptr(self.ws), _stream()), "taot_match")
+        return dict(slot_expert=se, slot_tokens=stk, X=X, rounds=rounds, info=info)
+
+    def assign(self, topk, slot_expert, X, reuse_counts: bool = False, info: Optional[torch.Tensor] = None,
+               out: Optional[torch.Tensor] = None):
+        _dev(topk, torch.int32, "topk")
+        new = torch.empty_like(topk) if out is None else out
+        info = torch.zeros((self.L,), dtype=torch.int32, device=self.device) if info is None else info
+        _check(self.lib.taot_assign(self.handle, _ptr(topk), _ptr(_dev(slot_expert, torch.int32, "slot_expert")),
+                                    _ptr(_dev(X, torch.int32, "X")), _ptr(new), _ptr(info), _ptr(self.ws),
+                                    ctypes.c_int32(1 if reuse_counts else 0), _stream()), "taot_assign")
+        return new, info
+
+    # ------------------------------------------------------------------ whole path
+    def _outputs_struct(self, out: Dict[str, torch.Tensor]) -> _Outputs:
+        o = _Outputs()
+        for name, _ in _Outputs._fields_:
+            t = out.get(name)
+            setattr(o, name, None if t is None else t.data_ptr())
+        return o
+
+    def plan(self, topk: torch.Tensor, out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+        _dev(topk, torch.int32, "topk")
+        out = self.alloc_outputs() if out is None else out
+        o = self._outputs_struct(out)
+        _check(self.lib.taot_plan(self.handle, _ptr(topk), ctypes.byref(o), _ptr(self.ws), _stream()), "taot_plan")
+        return out
+
+    def alloc_host_outputs(self, names=("plan", "slot_expert", "slot_tokens", "X", "new_idx", "info")):
+        L, R, E, K, S, T, k = self.L, self.R, self.E, self.K, self.S, self.T, self.k
+        shapes = dict(n=((L, R, E), torch.int32), expert_load=((L, E), torch.int32), rank_load=((L, R), torch.int32),
+                      excess=((L, R), torch.int32), spare=((L, R), torch.int32), plan=((L, R, R), torch.float32),
+                      sinkhorn_iters=((L,), torch.int32), row_err=((L,), torch.float32),
+                      slot_expert=((L, R, K), torch.int32), slot_tokens=((L, R, K), torch.int32),
+                      X=((L, R, S), torch.int32), rounds=((L, 2), torch.int32), new_idx=((L, T, k), torch.int32),
+                      info=((L,), torch.int32))
+        return {nm: torch.empty(shapes[nm][0], dtype=shapes[nm][1]).pin_memory() for nm in names}
+
+    def plan_host(self, topk_host: torch.Tensor, out_host: Dict[str, torch.Tensor]) -> Dict[str, torch.Tensor]:
+        """Whole path from a HOST routing table to HOST results; copies ride the current stream."""
+        if topk_host.is_cuda or topk_host.dtype != torch.int32 or not topk_host.is_contiguous():
+            raise TaotError("topk_host: expected a contiguous CPU int32 tensor")
+        if self._host_ws is None:
+            self._host_ws = torch.empty(self.host_ws_bytes, dtype=torch.uint8, device=self.device)
+        o = self._outputs_struct(out_host)
+        _check(self.lib.taot_plan_host(self.handle, _ptr(topk_host), ctypes.byref(o), _ptr(self._host_ws),
+                                       _stream()), "taot_plan_host")
+        return out_host

@@ -1,0 +1,376 @@
+// C ABI of libtaot: handle management, argument validation, workspace carve-up and the
+// stage chaining of taot_plan / taot_plan_host.  No arithmetic of the method lives here except
+// the two topology tables derived once per handle (the preference matrix B when the caller
+// gives none, and the first-iteration row normaliser of the Sinkhorn solve).
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "taot_internal.cuh"
+
+namespace {
+
+bool valid_params(const taot_params* p)
+{
+    if (p->struct_size != (int32_t)sizeof(taot_params)) return false;
+    if (p->L < 1 || p->R < 1 || p->E < 1 || p->K < 1 || p->k < 1) return false;
+    if (p->T < p->R || p->T % p->R != 0) return false;
+    if (p->T * (int64_t)p->k >= ((int64_t)1 << 31)) return false;
+    if (!(p->eps > 0.0f) || !std::isfinite(p->eps)) return false;
+    if (p->max_iters < 1) return false;
+    if (!(p->eps0 >= 0.0f) || !std::isfinite(p->eps0)) return false;
+    if (!std::isfinite(p->price_step) || !std::isfinite(p->tol)) return false;
+    return true;
+}
+
+bool supported_params(const taot_params* p)
+{
+    return p->R <= 256 && p->E <= 1024 && p->K <= 8 && p->k <= 64 &&
+           (int64_t)p->L * p->R * ((p->T / p->R * p->k + TAOT_CHUNK - 1) / TAOT_CHUNK) < ((int64_t)1 << 31);
+}
+
+template <typename T>
+int upload(T** dst, const T* src, size_t count)
+{
+    if (cudaMalloc(reinterpret_cast<void**>(dst), sizeof(T) * count) != cudaSuccess) return TAOT_ERR_CUDA;
+    if (cudaMemcpy(*dst, src, sizeof(T) * count, cudaMemcpyHostToDevice) != cudaSuccess) return TAOT_ERR_CUDA;
+    return TAOT_OK;
+}
+
+void layout(taot_handle_t h)
+{
+    const taot_params& p = h->p;
+    h->seg = p.T / p.R * p.k;
+    h->nc = (int32_t)((h->seg + TAOT_CHUNK - 1) / TAOT_CHUNK);
+    const int64_t r2 = (int64_t)p.R * p.R;
+    int64_t cap = r2 / 4 > 12288 ? r2 / 4 : 12288;
+    h->kcap = (int32_t)(cap < r2 ? cap : r2);
+    const size_t LR = (size_t)p.L * p.R;
+    const int dmax = p.E < p.R * p.K ? p.E : p.R * p.K;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { const size_t o = off; off = taot_align_up(off + bytes, 256); return o; };
+    h->off_cc = take(sizeof(int32_t) * LR * h->nc * p.E);
+    h->off_excess = take(sizeof(int32_t) * LR);
+    h->off_spare = take(sizeof(int32_t) * LR);
+    h->off_s = take(sizeof(float) * LR);
+    h->off_d = take(sizeof(float) * LR);
+    h->off_nrem = take(sizeof(int32_t) * (size_t)p.L * dmax * p.R);
+    h->ws_bytes = off;
+
+    const size_t S = (size_t)p.R * p.K;
+    off = 0;
+    h->hoff_topk = take(sizeof(int32_t) * (size_t)p.L * p.T * p.k);
+    h->hoff_new = take(sizeof(int32_t) * (size_t)p.L * p.T * p.k);
+    h->hoff_n = take(sizeof(int32_t) * LR * p.E);
+    h->hoff_el = take(sizeof(int32_t) * (size_t)p.L * p.E);
+    h->hoff_rl = take(sizeof(int32_t) * LR);
+    h->hoff_ex = take(sizeof(int32_t) * LR);
+    h->hoff_sp = take(sizeof(int32_t) * LR);
+    h->hoff_plan = take(sizeof(float) * LR * p.R);
+    h->hoff_it = take(sizeof(int32_t) * p.L);
+    h->hoff_err = take(sizeof(float) * p.L);
+    h->hoff_se = take(sizeof(int32_t) * p.L * S);
+    h->hoff_st = take(sizeof(int32_t) * p.L * S);
+    h->hoff_X = take(sizeof(int32_t) * LR * S);
+    h->hoff_rounds = take(sizeof(int32_t) * p.L * 2);
+    h->hoff_info = take(sizeof(int32_t) * p.L);
+    h->hoff_ws = take(h->ws_bytes);
+    h->host_ws_bytes = off;
+}
+
+inline char* at(void* base, size_t off) { return static_cast<char*>(base) + off; }
+
+}  // namespace
+
+extern "C" {
+
+const char* taot_status_string(int status)
+{
+    switch (status) {
+        case TAOT_OK: return "ok";
+        case TAOT_ERR_NULL: return "a required pointer is NULL";
+        case TAOT_ERR_PARAM: return "a parameter is out of range";
+        case TAOT_ERR_UNSUPPORTED: return "size not supported by this build";
+        case TAOT_ERR_CUDA: return "a CUDA runtime call failed";
+        case TAOT_ERR_ALIGN: return "a device pointer is misaligned";
+        default: return "unknown status";
+    }
+}
+
+int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_e2r, const float* h_C,
+                const float* h_B)
+{
+    if (out) *out = nullptr;
+    if (!out || !params || !h_e2r || !h_C) return TAOT_ERR_NULL;
+    if (!valid_params(params)) return TAOT_ERR_PARAM;
+    if (!supported_params(params)) return TAOT_ERR_UNSUPPORTED;
+    const int R = params->R, E = params->E;
+    for (int e = 0; e < E; ++e)
+        if (h_e2r[e] < 0 || h_e2r[e] >= R) return TAOT_ERR_PARAM;
+    for (int64_t q = 0; q < (int64_t)R * R; ++q)
+        if (!std::isfinite(h_C[q]) || h_C[q] < 0.0f) return TAOT_ERR_PARAM;
+    if (h_B)
+        for (int64_t q = 0; q < (int64_t)R * R; ++q)
+            if (!std::isfinite(h_B[q])) return TAOT_ERR_PARAM;
+
+    taot_handle_s* h = new (std::nothrow) taot_handle_s();
+    if (!h) return TAOT_ERR_CUDA;
+    std::memset(h, 0, sizeof(*h));
+    h->p = *params;
+    if (h->p.check_every < 1) h->p.check_every = 1;
+    if (cudaGetDevice(&h->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess) {
+        delete h;
+        return TAOT_ERR_CUDA;
+    }
+    layout(h);
+
+    // topology preference: given, or derived from the cost tiers (1 at the cheapest off-diagonal
+    // cost, c_min / C elsewhere, 0 on the diagonal)
+    std::vector<float> B((size_t)R * R);
+    if (h_B) {
+        std::memcpy(B.data(), h_B, sizeof(float) * (size_t)R * R);
+    } else {
+        float cmin = INFINITY;
+        for (int i = 0; i < R; ++i)
+            for (int j = 0; j < R; ++j) {
+                const float c = h_C[(size_t)i * R + j];
+                if (i != j && c > 0.0f && c < cmin) cmin = c;
+            }
+        for (int i = 0; i < R; ++i)
+            for (int j = 0; j < R; ++j) {
+                const float c = h_C[(size_t)i * R + j];
+                float b = 1.0f;
+                if (i == j) b = 0.0f;
+                else if (c > 0.0f && std::isfinite(cmin)) { b = cmin / c; if (b > 1.0f) b = 1.0f; }
+                B[(size_t)i * R + j] = b;
+            }
+    }
+    // first Sinkhorn row update with v = 1 on every rank: log-sum-exp of -C_ij/eps over all j
+    std::vector<double> lse0(R);
+    for (int i = 0; i < R; ++i) {
+        double mx = -INFINITY;
+        for (int j = 0; j < R; ++j) {
+            const double x = -(double)h_C[(size_t)i * R + j] / (double)params->eps;
+            if (x > mx) mx = x;
+        }
+        double acc = 0.0;
+        for (int j = 0; j < R; ++j) acc += std::exp(-(double)h_C[(size_t)i * R + j] / (double)params->eps - mx);
+        lse0[i] = mx + std::log(acc);
+    }
+    // experts by home rank (CSR), ascending expert index inside a rank
+    std::vector<int32_t> off(R + 1, 0), list(E);
+    for (int e = 0; e < E; ++e) off[h_e2r[e] + 1]++;
+    for (int r = 0; r < R; ++r) off[r + 1] += off[r];
+    {
+        std::vector<int32_t> cur(off.begin(), off.end() - 1);
+        for (int e = 0; e < E; ++e) list[cur[h_e2r[e]]++] = e;
+    }
+    int rc = TAOT_OK;
+    if (rc == TAOT_OK) rc = upload(&h->d_e2r, h_e2r, (size_t)E);
+    if (rc == TAOT_OK) rc = upload(&h->d_C, h_C, (size_t)R * R);
+    if (rc == TAOT_OK) rc = upload(&h->d_B, B.data(), (size_t)R * R);
+    if (rc == TAOT_OK) rc = upload(&h->d_rowlse0, lse0.data(), (size_t)R);
+    if (rc == TAOT_OK) rc = upload(&h->d_rank_off, off.data(), (size_t)R + 1);
+    if (rc == TAOT_OK) rc = upload(&h->d_rank_list, list.data(), (size_t)E);
+    if (rc == TAOT_OK && cudaDeviceSynchronize() != cudaSuccess) rc = TAOT_ERR_CUDA;
+    if (rc != TAOT_OK) {
+        taot_destroy(h);
+        return rc;
+    }
+    *out = h;
+    return TAOT_OK;
+}
+
+int taot_destroy(taot_handle_t h)
+{
+    if (!h) return TAOT_OK;
+    cudaDeviceSynchronize();
+    cudaFree(h->d_e2r); cudaFree(h->d_C); cudaFree(h->d_B); cudaFree(h->d_rowlse0);
+    cudaFree(h->d_rank_off); cudaFree(h->d_rank_list);
+    delete h;
+    return TAOT_OK;
+}
+
+int taot_workspace_bytes(taot_handle_t h, size_t* bytes)
+{
+    if (!h || !bytes) return TAOT_ERR_NULL;
+    *bytes = h->ws_bytes;
+    return TAOT_OK;
+}
+
+int taot_host_workspace_bytes(taot_handle_t h, size_t* bytes)
+{
+    if (!h || !bytes) return TAOT_ERR_NULL;
+    *bytes = h->host_ws_bytes;
+    return TAOT_OK;
+}
+
+int taot_last_launch_count(taot_handle_t h, int32_t* count)
+{
+    if (!h || !count) return TAOT_ERR_NULL;
+    *count = h->last_launches;
+    return TAOT_OK;
+}
+
+int taot_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_n, int32_t* d_expert_load,
+                   int32_t* d_rank_load, int32_t* d_info, void* ws, void* stream)
+{
+    if (!h || !d_topk || !d_n || !d_expert_load || !d_rank_load || !d_info || !ws) return TAOT_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(d_topk) & 3) || (reinterpret_cast<uintptr_t>(ws) & 255)) return TAOT_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t* cc = reinterpret_cast<int32_t*>(at(ws, h->off_cc));
+    int a = taot_launch_histogram(h, d_topk, cc, d_info, st);
+    if (a < 0) return a;
+    int b = taot_launch_merge(h, cc, d_n, d_expert_load, d_rank_load, nullptr, nullptr, nullptr, nullptr, st);
+    if (b < 0) return b;
+    h->last_launches = a + b;
+    return TAOT_OK;
+}
+
+int taot_excess_spare(taot_handle_t h, const int32_t* d_rank_load, int32_t B, int32_t* d_excess,
+                      int32_t* d_spare, float* d_s, float* d_d, void* stream)
+{
+    if (!h || !d_rank_load) return TAOT_ERR_NULL;
+    if (B < 1) return TAOT_ERR_PARAM;
+    int a = taot_launch_excess_spare(h, d_rank_load, B, d_excess, d_spare, d_s, d_d, static_cast<cudaStream_t>(stream));
+    if (a < 0) return a;
+    h->last_launches = a;
+    return TAOT_OK;
+}
+
+int taot_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
+                  int32_t* d_iters, float* d_row_err, int32_t* d_info, void* ws, void* stream)
+{
+    (void)ws;
+    if (!h || !d_s || !d_d || !d_plan || !d_iters || !d_row_err || !d_info) return TAOT_ERR_NULL;
+    if (B < 1) return TAOT_ERR_PARAM;
+    int a = taot_launch_sinkhorn(h, d_s, d_d, B, d_plan, d_iters, d_row_err, d_info, static_cast<cudaStream_t>(stream));
+    if (a < 0) return a;
+    h->last_launches = a;
+    return TAOT_OK;
+}
+
+int taot_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load, const int32_t* d_rank_load,
+               const float* d_plan, int32_t* d_slot_expert, int32_t* d_slot_tokens, int32_t* d_X,
+               int32_t* d_rounds, int32_t* d_info, void* ws, void* stream)
+{
+    if (!h || !d_n || !d_expert_load || !d_rank_load || !d_plan || !d_slot_expert || !d_slot_tokens || !d_X ||
+        !d_info || !ws)
+        return TAOT_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(ws) & 255) return TAOT_ERR_ALIGN;
+    int a = taot_launch_match(h, d_n, d_expert_load, d_rank_load, d_plan, d_slot_expert, d_slot_tokens, d_X,
+                              d_rounds, d_info, reinterpret_cast<int32_t*>(at(ws, h->off_nrem)),
+                              static_cast<cudaStream_t>(stream));
+    if (a < 0) return a;
+    h->last_launches = a;
+    return TAOT_OK;
+}
+
+int taot_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_slot_expert, const int32_t* d_X,
+                int32_t* d_new_idx, int32_t* d_info, void* ws, int32_t reuse_counts, void* stream)
+{
+    if (!h || !d_topk || !d_slot_expert || !d_X || !d_new_idx || !d_info || !ws) return TAOT_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(d_topk) & 3) || (reinterpret_cast<uintptr_t>(d_new_idx) & 3) ||
+        (reinterpret_cast<uintptr_t>(ws) & 255))
+        return TAOT_ERR_ALIGN;
+    if (d_topk == d_new_idx) return TAOT_ERR_PARAM;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t* cc = reinterpret_cast<int32_t*>(at(ws, h->off_cc));
+    int launches = 0;
+    if (!reuse_counts) {
+        int a = taot_launch_histogram(h, d_topk, cc, d_info, st);
+        if (a < 0) return a;
+        launches += a;
+    }
+    int b = taot_launch_assign(h, d_topk, cc, d_slot_expert, d_X, d_new_idx, d_info, st);
+    if (b < 0) return b;
+    h->last_launches = launches + b;
+    return TAOT_OK;
+}
+
+int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, void* ws, void* stream)
+{
+    if (!h || !d_topk || !o || !ws) return TAOT_ERR_NULL;
+    if (!o->n || !o->expert_load || !o->rank_load || !o->plan || !o->sinkhorn_iters || !o->row_err ||
+        !o->slot_expert || !o->slot_tokens || !o->X || !o->new_idx || !o->info)
+        return TAOT_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(d_topk) & 3) || (reinterpret_cast<uintptr_t>(o->new_idx) & 3) ||
+        (reinterpret_cast<uintptr_t>(ws) & 255))
+        return TAOT_ERR_ALIGN;
+    if (d_topk == o->new_idx) return TAOT_ERR_PARAM;
+    const taot_params& p = h->p;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t* cc = reinterpret_cast<int32_t*>(at(ws, h->off_cc));
+    int32_t* excess = o->excess ? o->excess : reinterpret_cast<int32_t*>(at(ws, h->off_excess));
+    int32_t* spare = o->spare ? o->spare : reinterpret_cast<int32_t*>(at(ws, h->off_spare));
+    float* fs = reinterpret_cast<float*>(at(ws, h->off_s));
+    float* fd = reinterpret_cast<float*>(at(ws, h->off_d));
+    TAOT_CUDA_OK(cudaMemsetAsync(o->info, 0, sizeof(int32_t) * p.L, st));
+    int total = 0, a;
+    if ((a = taot_launch_histogram(h, d_topk, cc, o->info, st)) < 0) return a;
+    total += a;
+    if ((a = taot_launch_merge(h, cc, o->n, o->expert_load, o->rank_load, excess, spare, fs, fd, st)) < 0) return a;
+    total += a;
+    if ((a = taot_launch_sinkhorn(h, fs, fd, p.L, o->plan, o->sinkhorn_iters, o->row_err, o->info, st)) < 0) return a;
+    total += a;
+    if ((a = taot_launch_match(h, o->n, o->expert_load, o->rank_load, o->plan, o->slot_expert, o->slot_tokens,
+                               o->X, o->rounds, o->info, reinterpret_cast<int32_t*>(at(ws, h->off_nrem)), st)) < 0)
+        return a;
+    total += a;
+    if ((a = taot_launch_assign(h, d_topk, cc, o->slot_expert, o->X, o->new_idx, o->info, st)) < 0) return a;
+    total += a;
+    h->last_launches = total;
+    return TAOT_OK;
+}
+
+int taot_plan_host(taot_handle_t h, const int32_t* h_topk, const taot_outputs* o, void* d_ws, void* stream)
+{
+    if (!h || !h_topk || !o || !d_ws) return TAOT_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(d_ws) & 255) return TAOT_ERR_ALIGN;
+    const taot_params& p = h->p;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t LR = (size_t)p.L * p.R, S = (size_t)p.R * p.K, NE = (size_t)p.L * p.T * p.k;
+    taot_outputs d;
+    d.n = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_n));
+    d.expert_load = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_el));
+    d.rank_load = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_rl));
+    d.excess = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_ex));
+    d.spare = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_sp));
+    d.plan = reinterpret_cast<float*>(at(d_ws, h->hoff_plan));
+    d.sinkhorn_iters = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_it));
+    d.row_err = reinterpret_cast<float*>(at(d_ws, h->hoff_err));
+    d.slot_expert = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_se));
+    d.slot_tokens = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_st));
+    d.X = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_X));
+    d.rounds = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_rounds));
+    d.new_idx = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_new));
+    d.info = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_info));
+    int32_t* d_topk = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_topk));
+    TAOT_CUDA_OK(cudaMemcpyAsync(d_topk, h_topk, sizeof(int32_t) * NE, cudaMemcpyHostToDevice, st));
+    const int rc = taot_plan(h, d_topk, &d, at(d_ws, h->hoff_ws), stream);
+    if (rc != TAOT_OK) return rc;
+#define TAOT_BACK(member, count, type)                                                                       \
+    if (o->member)                                                                                           \
+        TAOT_CUDA_OK(cudaMemcpyAsync(o->member, d.member, sizeof(type) * (count), cudaMemcpyDeviceToHost, st))
+    TAOT_BACK(n, LR * p.E, int32_t);
+    TAOT_BACK(expert_load, (size_t)p.L * p.E, int32_t);
+    TAOT_BACK(rank_load, LR, int32_t);
+    TAOT_BACK(excess, LR, int32_t);
+    TAOT_BACK(spare, LR, int32_t);
+    TAOT_BACK(plan, LR * p.R, float);
+    TAOT_BACK(sinkhorn_iters, (size_t)p.L, int32_t);
+    TAOT_BACK(row_err, (size_t)p.L, float);
+    TAOT_BACK(slot_expert, p.L * S, int32_t);
+    TAOT_BACK(slot_tokens, p.L * S, int32_t);
+    TAOT_BACK(X, LR * S, int32_t);
+    TAOT_BACK(rounds, (size_t)p.L * 2, int32_t);
+    TAOT_BACK(new_idx, NE, int32_t);
+    TAOT_BACK(info, (size_t)p.L, int32_t);
+#undef TAOT_BACK
+    return TAOT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,191 @@
+// Load collection (Appendix A.1): per-chunk expert histograms of the routing table, then one
+// merge per layer into n[r][e], expert_load, rank_load and the excess / spare vectors.
+//
+// The routing table of one layer is R contiguous segments (one per source rank) of SEG = (T/R)*k
+// int32 each, so n[l][r][:] is simply the E-bin histogram of segment (l, r).  Each CTA owns one
+// chunk of at most TAOT_CHUNK elements of one segment: it streams the chunk with 16-byte loads,
+// counts into per-warp private shared-memory histograms, and stores its E counts with plain
+// stores -- no global atomics, no zero-fill of the outputs.  The per-chunk counts are kept: the
+// reassignment kernel turns them into each chunk's starting ordinals.
+#include "taot_internal.cuh"
+
+namespace {
+
+constexpr int kThreads = TAOT_STREAM_THREADS;
+constexpr int kWarps = kThreads / 32;
+
+__device__ __forceinline__ int4 ld_stream(const int4* p)
+{
+    int4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void count_one(int32_t* hist, int32_t e, int32_t E, int& bad)
+{
+    if ((uint32_t)e < (uint32_t)E) atomicAdd(hist + e, 1);
+    else bad = 1;
+}
+
+__global__ void __launch_bounds__(kThreads)
+hist_chunk_kernel(const int32_t* __restrict__ topk, int32_t* __restrict__ cc, int32_t* __restrict__ info,
+                  int64_t layer_elems, int64_t seg, int32_t nc, int32_t R, int32_t E, int vec_ok)
+{
+    extern __shared__ int32_t sh_hist[];                 // [kWarps][E]
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int64_t id = blockIdx.x;
+    const int32_t c = (int32_t)(id % nc);
+    const int64_t lr = id / nc;
+    const int32_t l = (int32_t)(lr / R);
+    const int32_t r = (int32_t)(lr % R);
+    const int64_t start = (int64_t)c * TAOT_CHUNK;
+    const int32_t len = (int32_t)((seg - start) < (int64_t)TAOT_CHUNK ? (seg - start) : (int64_t)TAOT_CHUNK);
+    const int32_t* src = topk + (int64_t)l * layer_elems + (int64_t)r * seg + start;
+
+    for (int i = tid; i < kWarps * E; i += kThreads) sh_hist[i] = 0;
+    __syncthreads();
+    int32_t* hist = sh_hist + warp * E;
+    int bad = 0;
+
+    if (vec_ok) {
+        const int4* src4 = reinterpret_cast<const int4*>(src);
+        const int32_t nvec = len >> 2;
+        int32_t v = tid;
+        // full rounds of 8 loads in flight per thread
+        for (; v + 7 * kThreads < nvec; v += 8 * kThreads) {
+            int4 x[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) x[u] = ld_stream(src4 + v + u * kThreads);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                count_one(hist, x[u].x, E, bad); count_one(hist, x[u].y, E, bad);
+                count_one(hist, x[u].z, E, bad); count_one(hist, x[u].w, E, bad);
+            }
+        }
+        for (; v < nvec; v += kThreads) {
+            const int4 x = ld_stream(src4 + v);
+            count_one(hist, x.x, E, bad); count_one(hist, x.y, E, bad);
+            count_one(hist, x.z, E, bad); count_one(hist, x.w, E, bad);
+        }
+        for (int32_t i = (nvec << 2) + tid; i < len; i += kThreads) count_one(hist, src[i], E, bad);
+    } else {
+        for (int32_t i = tid; i < len; i += kThreads) count_one(hist, src[i], E, bad);
+    }
+    const int any_bad = __syncthreads_or(bad);
+    int32_t* out = cc + id * E;
+    for (int e = tid; e < E; e += kThreads) {
+        int32_t tot = 0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) tot += sh_hist[w * E + e];
+        out[e] = tot;
+    }
+    if (any_bad && tid == 0) atomicOr(info + l, TAOT_INFO_BAD_INDEX);
+}
+
+// excess / spare of one row of rank loads held in shared memory (Appendix A.1, integer mean)
+__device__ void excess_spare_row(const int32_t* s_rl, int32_t R, long long* s_tot, int32_t* excess,
+                                 int32_t* spare, float* fs, float* fd)
+{
+    const int tid = threadIdx.x;
+    if (tid == 0) *s_tot = 0;
+    __syncthreads();
+    long long part = 0;
+    for (int r = tid; r < R; r += blockDim.x) part += s_rl[r];
+    if (part) atomicAdd(reinterpret_cast<unsigned long long*>(s_tot), (unsigned long long)part);
+    __syncthreads();
+    const long long m = *s_tot / R;
+    for (int r = tid; r < R; r += blockDim.x) {
+        const long long lr = s_rl[r];
+        const int32_t ex = (int32_t)(lr > m ? lr - m : 0);
+        const int32_t sp = (int32_t)(m > lr ? m - lr : 0);
+        if (excess) excess[r] = ex;
+        if (spare) spare[r] = sp;
+        if (fs) fs[r] = (float)ex;
+        if (fd) fd[r] = (float)sp;
+    }
+}
+
+// one CTA per layer: n = sum over chunks, expert_load = sum over ranks, rank_load by home rank
+__global__ void __launch_bounds__(1024)
+merge_kernel(const int32_t* __restrict__ cc, const int32_t* __restrict__ e2r, int32_t* __restrict__ n,
+             int32_t* __restrict__ expert_load, int32_t* __restrict__ rank_load, int32_t* excess,
+             int32_t* spare, float* fs, float* fd, int32_t R, int32_t E, int32_t nc)
+{
+    extern __shared__ int32_t sh[];                      // el[E], rl[R]
+    __shared__ long long s_tot;
+    int32_t* s_el = sh;
+    int32_t* s_rl = sh + E;
+    const int l = blockIdx.x, tid = threadIdx.x;
+    for (int i = tid; i < E + R; i += blockDim.x) sh[i] = 0;
+    __syncthreads();
+    const int64_t RE = (int64_t)R * E;
+    for (int64_t idx = tid; idx < RE; idx += blockDim.x) {
+        const int32_t r = (int32_t)(idx / E), e = (int32_t)(idx % E);
+        const int32_t* p = cc + (((int64_t)l * R + r) * nc) * E + e;
+        int32_t v = 0;
+        for (int c = 0; c < nc; ++c) v += p[(int64_t)c * E];
+        n[(int64_t)l * RE + idx] = v;
+        if (v) atomicAdd(s_el + e, v);
+    }
+    __syncthreads();
+    for (int e = tid; e < E; e += blockDim.x) {
+        const int32_t v = s_el[e];
+        expert_load[(int64_t)l * E + e] = v;
+        if (v) atomicAdd(s_rl + e2r[e], v);
+    }
+    __syncthreads();
+    for (int r = tid; r < R; r += blockDim.x) rank_load[(int64_t)l * R + r] = s_rl[r];
+    excess_spare_row(s_rl, R, &s_tot, excess ? excess + (int64_t)l * R : nullptr,
+                     spare ? spare + (int64_t)l * R : nullptr, fs ? fs + (int64_t)l * R : nullptr,
+                     fd ? fd + (int64_t)l * R : nullptr);
+}
+
+__global__ void __launch_bounds__(256)
+excess_spare_kernel(const int32_t* __restrict__ rank_load, int32_t* excess, int32_t* spare, float* fs,
+                    float* fd, int32_t R)
+{
+    extern __shared__ int32_t sh[];                      // rl[R]
+    __shared__ long long s_tot;
+    const int64_t b = blockIdx.x;
+    for (int r = threadIdx.x; r < R; r += blockDim.x) sh[r] = rank_load[b * R + r];
+    __syncthreads();
+    excess_spare_row(sh, R, &s_tot, excess ? excess + b * R : nullptr, spare ? spare + b * R : nullptr,
+                     fs ? fs + b * R : nullptr, fd ? fd + b * R : nullptr);
+}
+
+}  // namespace
+
+int taot_launch_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_cc, int32_t* d_info, cudaStream_t st)
+{
+    const taot_params& p = h->p;
+    const int64_t layer_elems = p.T * p.k;
+    const int64_t blocks = (int64_t)p.L * p.R * h->nc;
+    const int vec_ok = ((reinterpret_cast<uintptr_t>(d_topk) & 15) == 0) && (h->seg % 4 == 0);
+    const size_t smem = sizeof(int32_t) * kWarps * p.E;
+    hist_chunk_kernel<<<(unsigned)blocks, kThreads, smem, st>>>(d_topk, d_cc, d_info, layer_elems, h->seg,
+                                                                 h->nc, p.R, p.E, vec_ok);
+    TAOT_CUDA_OK(cudaGetLastError());
+    return 1;
+}
+
+int taot_launch_merge(taot_handle_t h, const int32_t* d_cc, int32_t* d_n, int32_t* d_expert_load,
+                      int32_t* d_rank_load, int32_t* d_excess, int32_t* d_spare, float* d_s, float* d_d,
+                      cudaStream_t st)
+{
+    const taot_params& p = h->p;
+    const size_t smem = sizeof(int32_t) * (p.E + p.R);
+    merge_kernel<<<p.L, 1024, smem, st>>>(d_cc, h->d_e2r, d_n, d_expert_load, d_rank_load, d_excess, d_spare,
+                                          d_s, d_d, p.R, p.E, h->nc);
+    TAOT_CUDA_OK(cudaGetLastError());
+    return 1;
+}
+
+int taot_launch_excess_spare(taot_handle_t h, const int32_t* d_rank_load, int32_t B, int32_t* d_excess,
+                             int32_t* d_spare, float* d_s, float* d_d, cudaStream_t st)
+{
+    const taot_params& p = h->p;
+    excess_spare_kernel<<<B, 256, sizeof(int32_t) * p.R, st>>>(d_rank_load, d_excess, d_spare, d_s, d_d, p.R);
+    TAOT_CUDA_OK(cudaGetLastError());
+    return 1;
+}

@@ -1,0 +1,64 @@
+// Internal definitions shared by the translation units of libtaot (never installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "taot.h"
+
+// Elements of topk_idx one CTA of the histogram / reassignment kernels owns.  A chunk never
+// crosses a (layer, source rank) segment, so a segment of SEG = (T/R)*k elements has
+// NC = ceil(SEG / TAOT_CHUNK) chunks, the last one possibly short.
+#define TAOT_CHUNK 16384
+#define TAOT_STREAM_THREADS 256            // threads of the streaming kernels: 64 elements each
+
+struct taot_handle_s {
+    taot_params p;
+    int device;
+    int sm_count;
+    // topology, device copies
+    int32_t* d_e2r;          // [E]
+    float* d_C;              // [R,R]
+    float* d_B;              // [R,R] topology preference (given or derived)
+    double* d_rowlse0;       // [R]  LSE_j(-C_ij/eps) over all ranks j: the first u-update with v = 1
+    int32_t* d_rank_off;     // [R+1] CSR of experts by home rank
+    int32_t* d_rank_list;    // [E]
+    // derived sizes
+    int64_t seg;             // elements per (layer, rank) segment
+    int32_t nc;              // chunks per segment
+    int32_t kcap;            // Sinkhorn kernel-matrix capacity in floats per problem
+    // workspace layout (byte offsets)
+    size_t off_cc, off_excess, off_spare, off_s, off_d, off_nrem, off_plan_info;
+    size_t ws_bytes;
+    // host-call staging layout (byte offsets into d_ws of taot_plan_host)
+    size_t hoff_topk, hoff_new, hoff_n, hoff_el, hoff_rl, hoff_ex, hoff_sp, hoff_plan, hoff_it, hoff_err,
+           hoff_se, hoff_st, hoff_X, hoff_rounds, hoff_info, hoff_ws;
+    size_t host_ws_bytes;
+    int32_t last_launches;
+};
+
+static inline size_t taot_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// kernel launchers (each returns the number of kernels it enqueued, or a negative taot_status)
+int taot_launch_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_cc, int32_t* d_info, cudaStream_t st);
+int taot_launch_merge(taot_handle_t h, const int32_t* d_cc, int32_t* d_n, int32_t* d_expert_load,
+                      int32_t* d_rank_load, int32_t* d_excess, int32_t* d_spare, float* d_s, float* d_d,
+                      cudaStream_t st);
+int taot_launch_excess_spare(taot_handle_t h, const int32_t* d_rank_load, int32_t B, int32_t* d_excess,
+                             int32_t* d_spare, float* d_s, float* d_d, cudaStream_t st);
+int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
+                         int32_t* d_iters, float* d_row_err, int32_t* d_info, cudaStream_t st);
+int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load,
+                      const int32_t* d_rank_load, const float* d_plan, int32_t* d_slot_expert,
+                      int32_t* d_slot_tokens, int32_t* d_X, int32_t* d_rounds, int32_t* d_info,
+                      int32_t* d_nrem, cudaStream_t st);
+int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_cc,
+                       const int32_t* d_slot_expert, const int32_t* d_X, int32_t* d_new_idx,
+                       int32_t* d_info, cudaStream_t st);
+
+#define TAOT_CUDA_OK(expr)                              \
+    do {                                                \
+        cudaError_t _e = (expr);                        \
+        if (_e != cudaSuccess) return TAOT_ERR_CUDA;    \
+    } while (0)

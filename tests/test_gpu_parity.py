@@ -1,0 +1,128 @@
+"""GPU parity: every stage of the CUDA path, called through the C ABI, against the CPU oracle on
+the same seeded inputs.  Integer stages bit-exact; Sinkhorn within the stated tolerances."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import workloads as W
+from helpers import (check_sinkhorn_problem, cpu, make_planner, oracle_schedule_layer, topology)
+
+pytestmark = pytest.mark.gpu
+
+CASES = {
+    # name: (config, overrides) -- sized so the oracle finishes in seconds, still several chunks + a ragged tail
+    "cfg1": (W.get_config("cfg1"), {}),
+    "cfg2": (W.get_config("cfg2"), {}),
+    "cfg3_small": (W.get_config("cfg3").replace(L=3, T=64 * 2560), {}),      # SEG = 20480: 2 chunks, ragged
+    "cfg4_small": (W.get_config("cfg4").replace(L=2, T=256 * 2304), {}),     # SEG = 18432: 2 chunks, ragged
+}
+
+
+def _routing(cfg):
+    return W.routing_topk(cfg, device="cuda")
+
+
+@pytest.fixture(scope="module", params=list(CASES))
+def case(request):
+    cfg, over = CASES[request.param]
+    topk = _routing(cfg)
+    pl = make_planner(cfg, **over)
+    out = pl.plan(topk)
+    torch.cuda.synchronize()
+    yield cfg, topk, pl, {k: cpu(v) for k, v in out.items()}
+    pl.close()
+
+
+def test_histogram_bit_exact(case):
+    cfg, topk, pl, out = case
+    e2r, _ = topology(cfg)
+    n, el, rl, bad = O.histogram(cpu(topk), cfg.R, cfg.E, e2r.numpy())
+    assert (out["n"] == n).all() and (out["expert_load"] == el).all() and (out["rank_load"] == rl).all()
+    assert (bad == 0).all() and ((out["info"] & 1) == 0).all()
+    # the standalone entry point gives the same
+    n2, el2, rl2, info2 = pl.histogram(topk)
+    assert (cpu(n2) == n).all() and (cpu(el2) == el).all() and (cpu(rl2) == rl).all() and (cpu(info2) == 0).all()
+
+
+def test_excess_spare_bit_exact(case):
+    cfg, topk, pl, out = case
+    mean, ex, sp = O.excess_spare(out["rank_load"])
+    assert (out["excess"] == ex).all() and (out["spare"] == sp).all()
+    ex2, sp2, s2, d2 = pl.excess_spare(torch.from_numpy(out["rank_load"]).cuda())
+    assert (cpu(ex2) == ex).all() and (cpu(sp2) == sp).all()
+    assert (cpu(s2) == ex.astype(np.float32)).all() and (cpu(d2) == sp.astype(np.float32)).all()
+
+
+def test_sinkhorn_within_tolerance(case):
+    cfg, topk, pl, out = case
+    _, C = topology(cfg)
+    worst = 0.0
+    for l in range(cfg.L):
+        s = out["excess"][l].astype(np.float32); d = out["spare"][l].astype(np.float32)
+        r = check_sinkhorn_problem(s, d, C.numpy(), cfg.eps, out["plan"][l], out["sinkhorn_iters"][l],
+                                   out["row_err"][l], cfg.max_iters, cfg.tol)
+        worst = max(worst, r["max_rel"])
+        capped = bool(out["info"][l] & 2)
+        assert capped == (cfg.tol > 0 and out["sinkhorn_iters"][l] == cfg.max_iters and out["row_err"][l] > cfg.tol)
+    print(f"{cfg.name}: worst plan rel err {worst:.2e}, iters {out['sinkhorn_iters'].tolist()}")
+
+
+def test_schedule_bit_exact_given_the_gpu_plan(case):
+    cfg, topk, pl, out = case
+    e2r, C = topology(cfg)
+    B = O.default_preference(C.numpy())
+    for l in range(cfg.L):
+        m, a = oracle_schedule_layer(cfg, e2r.numpy(), B, out["n"][l], out["expert_load"][l], out["rank_load"][l],
+                                     out["plan"][l])
+        assert (out["slot_expert"][l].ravel() == m["slot_expert"]).all()
+        assert (out["slot_tokens"][l].ravel() == m["slot_tokens"]).all()
+        assert (out["X"][l] == a["X"]).all()
+        assert out["rounds"][l].tolist() == [m["inner_rounds"], a["rounds"]]
+        assert a["residual"] == 0 and not (out["info"][l] & 8)
+    print(f"{cfg.name}: rounds {out['rounds'].tolist()}")
+
+
+def test_assign_bit_exact(case):
+    cfg, topk, pl, out = case
+    tk = cpu(topk)
+    for l in range(cfg.L):
+        want = O.assign(tk[l], cfg.R, cfg.E, cfg.K, out["slot_expert"][l].ravel(), out["X"][l])
+        assert (out["new_idx"][l] == want).all()
+    # standalone call, recounting the chunks itself, and reusing the histogram's counts
+    se = torch.from_numpy(out["slot_expert"]).cuda(); X = torch.from_numpy(out["X"]).cuda()
+    new, info = pl.assign(topk, se, X, reuse_counts=False)
+    assert (cpu(new) == out["new_idx"]).all() and (cpu(info) == 0).all()
+    pl.histogram(topk)
+    new, info = pl.assign(topk, se, X, reuse_counts=True)
+    assert (cpu(new) == out["new_idx"]).all()
+
+
+def test_stage_calls_equal_the_chained_plan(case):
+    cfg, topk, pl, out = case
+    n, el, rl, _ = pl.histogram(topk)
+    ex, sp, s, d = pl.excess_spare(rl)
+    sk = pl.sinkhorn(s, d)
+    assert (cpu(sk["plan"]) == out["plan"]).all() and (cpu(sk["iters"]) == out["sinkhorn_iters"]).all()
+    m = pl.match(n, el, rl, sk["plan"])
+    assert (cpu(m["slot_expert"]) == out["slot_expert"]).all() and (cpu(m["X"]) == out["X"]).all()
+    assert pl.last_launch_count() == 1
+
+
+def test_plan_is_deterministic(case):
+    cfg, topk, pl, out = case
+    again = pl.plan(topk)
+    torch.cuda.synchronize()
+    for key, val in again.items():
+        assert (cpu(val) == out[key]).all(), key
+    assert pl.last_launch_count() == 5
+
+
+def test_plan_host_round_trip(case):
+    cfg, topk, pl, out = case
+    host_in = topk.cpu().pin_memory()
+    host_out = pl.alloc_host_outputs(("n", "plan", "slot_expert", "slot_tokens", "X", "new_idx", "info", "rounds"))
+    pl.plan_host(host_in, host_out)
+    torch.cuda.synchronize()
+    for key, val in host_out.items():
+        assert (val.numpy() == out[key]).all(), key
