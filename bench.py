@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the TAOT planner hot path on B200.
+
+One step = one pass of the whole path (histogram -> excess/spare -> Sinkhorn -> matching +
+auction -> token reassignment) over one batch of L synthetic routing problems, through
+`taot_plan`.  Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl ours|reference]
+
+N > 1 is launched with torch.distributed.run; every rank plans its own L problems (independent
+replicas, no data-path collective), the timed region is bracketed by barriers and the slowest
+rank's device time is reported.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as W  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+FLUSH_BYTES = 256 * 1024 * 1024
+FP32_LANES_PER_SM = 128
+STAGES = ["histogram", "merge", "sinkhorn", "match_auction", "assign"]
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default="cfg2", choices=sorted(W.CONFIGS))
+    ap.add_argument("--cpu-seconds", type=float, default=20.0, help="budget of the CPU-baseline sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-streams", action="store_true", help="skip the HBM-sized streaming report")
+    return ap.parse_args()
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+# ---------------------------------------------------------------------------------------------
+# helpers
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), sm_max_mhz=float(d.get("sm_max_mhz", 1965.0)), source="measured")
+    return dict(hbm_gbs=6650.0, sm_max_mhz=1965.0, source="fallback")
+
+
+def build_planner(cfg):
+    import paper_2608_03676_b200 as P
+    e2r = W.expert_to_rank(cfg.E, cfg.R, cfg.e2r_mode)
+    C = W.cost_matrix(cfg.R, cfg.gpus_per_node, cfg.tiers, cfg.nodes_per_group)
+    return P.Planner(L=cfg.L, R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k, T=cfg.T, e2r=e2r, C=C, eps=cfg.eps,
+                     max_iters=cfg.max_iters, tol=cfg.tol)
+
+
+def timed_steps(fn, steps, flush):
+    """Device time of `steps` calls of fn, each bracketed by its own event pair; L2 flushed before each."""
+    pairs = []
+    for _ in range(steps):
+        if flush is not None:
+            flush.zero_()
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        a.record(); fn(); b.record()
+        pairs.append((a, b))
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in pairs]
+
+
+def oracle_sample(cfg, topk_cpu, seconds):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload: whole layers, as many
+    as fit in about `seconds` (at least one)."""
+    import oracle as O
+    e2r = W.expert_to_rank(cfg.E, cfg.R, cfg.e2r_mode).numpy()
+    C = W.cost_matrix(cfg.R, cfg.gpus_per_node, cfg.tiers, cfg.nodes_per_group).numpy()
+    O.build()
+    done, t_total = 0, 0.0
+    while done < cfg.L:
+        t0 = time.perf_counter()
+        O.plan_layers(topk_cpu[done:done + 1], cfg.R, cfg.E, cfg.K, e2r, C, cfg.eps, cfg.max_iters, cfg.tol)
+        t_total += time.perf_counter() - t0
+        done += 1
+        if t_total + t_total / done > seconds:
+            break
+    return done, t_total
+
+
+def sinkhorn_work(out, cfg):
+    """FMA count the Sinkhorn kernel executed: 2 mat-vecs over the |hot| x |cold| block per iteration."""
+    ex = out["excess"].cpu().numpy(); sp = out["spare"].cpu().numpy(); it = out["sinkhorn_iters"].cpu().numpy()
+    hn = (ex > 0).sum(1).astype(np.int64); cn = (sp > 0).sum(1).astype(np.int64)
+    return int((2 * hn * cn * np.maximum(it - 1, 0)).sum()), it
+
+
+def roofline_for(stage, ms, cfg, out, peaks, sm_count):
+    topk_bytes = cfg.L * cfg.T * cfg.k * 4
+    hbm = peaks["hbm_gbs"]
+    if stage == "histogram":
+        a = topk_bytes / (ms * 1e-3) / 1e9
+        return dict(kernel="hist_chunk_kernel", bound="hbm", achieved=a, peak=hbm, unit="GB/s", frac=a / hbm,
+                    traffic=None, peak_source=peaks["source"], bytes_per_launch=topk_bytes)
+    if stage == "assign":
+        a = 2 * topk_bytes / (ms * 1e-3) / 1e9
+        return dict(kernel="assign_kernel", bound="hbm", achieved=a, peak=hbm, unit="GB/s", frac=a / hbm,
+                    traffic=None, peak_source=peaks["source"], bytes_per_launch=2 * topk_bytes)
+    if stage == "merge":
+        b = cfg.L * cfg.R * cfg.E * 4 * (2 + max(1, (cfg.T // cfg.R * cfg.k + 16383) // 16384))
+        a = b / (ms * 1e-3) / 1e9
+        return dict(kernel="merge_kernel", bound="hbm", achieved=a, peak=hbm, unit="GB/s", frac=a / hbm,
+                    traffic=None, peak_source=peaks["source"], bytes_per_launch=b)
+    fp32_peak = sm_count * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+    if stage == "sinkhorn":
+        fma, _ = sinkhorn_work(out, cfg)
+        a = 2 * fma / (ms * 1e-3) / 1e12
+        return dict(kernel="sinkhorn_kernel", bound="alu", achieved=a, peak=fp32_peak, unit="TFLOP/s",
+                    frac=a / fp32_peak, traffic=None,
+                    peak_source=f"derived: {sm_count} SMs x 128 fp32 lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz",
+                    flops_per_launch=2 * fma,
+                    note="latency-bound chains of dependent mat-vecs over L small problems; fraction of the "
+                         "fp32 FMA peak is reported, not claimed as the binding limit")
+    rounds = out["rounds"].cpu().numpy().astype(np.int64)
+    ops = int((rounds[:, 0] * cfg.R * cfg.E + rounds[:, 1] * cfg.R * cfg.S).sum())
+    a = ops / (ms * 1e-3) / 1e12
+    return dict(kernel="match_kernel", bound="alu", achieved=a, peak=fp32_peak / 2, unit="Tscore/s",
+                frac=a / (fp32_peak / 2), traffic=None,
+                peak_source="derived: one fp32 score evaluation per lane per clock",
+                note="dependent rounds of masked arg-max; dense score count of the paper's formulation "
+                     "(rounds x R x E and rounds x R x S), latency-bound by construction")
+
+
+def stream_report(name, peaks, steps=5):
+    """Histogram and reassignment on an HBM-sized routing table (larger than L2): GB/s of each."""
+    cfg = W.get_config(name)
+    topk = W.routing_topk(cfg, device="cuda")
+    pl = build_planner(cfg)
+    out = pl.alloc_outputs()
+    for _ in range(3):
+        pl.plan(topk, out)
+    pl.set_profiling(True)
+    acc = np.zeros(5)
+    for _ in range(steps):
+        pl.plan(topk, out)
+        acc += np.array(pl.stage_ms())
+    acc /= steps
+    b = topk.numel() * 4
+    rep = dict(workload=name, topk_bytes=b, stages_ms=dict(zip(STAGES, [float(x) for x in acc])),
+               histogram_gbs=b / (acc[0] * 1e-3) / 1e9, assign_gbs=2 * b / (acc[4] * 1e-3) / 1e9,
+               peak_gbs=peaks["hbm_gbs"], peak_source=peaks["source"],
+               remapped_tokens_per_s=cfg.L * cfg.T / (acc[4] * 1e-3),
+               plans_per_s=cfg.L / (acc.sum() * 1e-3))
+    rep["histogram_frac"] = rep["histogram_gbs"] / peaks["hbm_gbs"]
+    rep["assign_frac"] = rep["assign_gbs"] / peaks["hbm_gbs"]
+    pl.close()
+    del topk, out
+    torch.cuda.empty_cache()
+    return rep
+
+
+# ---------------------------------------------------------------------------------------------
+# arms
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = W.get_config(args.workload)
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    topk = W.routing_topk(cfg, device=dev).cpu().numpy()
+    per_step = max(2.0, min(args.cpu_seconds, 60.0 / max(1, args.steps + args.warmup)))
+    layers, secs = 0, 0.0
+    for i in range(args.warmup + args.steps):
+        n, t = oracle_sample(cfg, topk, per_step)
+        if i >= args.warmup:
+            layers += n; secs += t
+    value = layers / secs
+    line = dict(metric="placement plans/s (whole planner path)", value=value, unit="plans/s", n_gpus=args.gpus,
+                steps=args.steps, warmup=args.warmup, ms_per_step=1e3 * secs / max(1, args.steps),
+                higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                impl="reference", config=dict(workload=args.workload, L=cfg.L, R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k,
+                                              T=cfg.T),
+                cpu_baseline=dict(value=value, unit="plans/s", cores=1, kind="oracle",
+                                  sample=f"{layers // max(1, args.steps)} whole layer(s) per step of {cfg.L}"),
+                e2e=dict(value=value, unit="plans/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the planner has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    cfg = W.get_config(args.workload)
+    cfg = cfg.replace(seed=cfg.seed + 7919 * rank)            # every rank plans its own batch
+    peaks = measured_peaks()
+    props = torch.cuda.get_device_properties(local)
+    topk = W.routing_topk(cfg, device="cuda")
+    pl = build_planner(cfg)
+    out = pl.alloc_outputs()
+    topk_bytes = topk.numel() * 4
+    need_flush = 2 * topk_bytes < 4 * L2_BYTES
+    flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda") if need_flush else None
+
+    step = lambda: pl.plan(topk, out)
+    timed_steps(step, max(3, args.warmup), flush)
+    barrier(); torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ms = timed_steps(step, args.steps, flush)
+    torch.cuda.synchronize(); barrier()
+    launches = pl.last_launch_count() * args.steps
+    # per-kernel durations inside the same step, from events the library records between its kernels
+    pl.set_profiling(True)
+    stage_ms = np.zeros(5)
+    for _ in range(args.steps):
+        if flush is not None:
+            flush.zero_()
+        pl.plan(topk, out)
+        stage_ms += np.array(pl.stage_ms())
+    pl.set_profiling(False)
+    stage_ms /= args.steps
+    clocks = sampler.stop() if rank == 0 else None
+
+    total_ms = torch.tensor([float(sum(ms))], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(total_ms, op=dist.ReduceOp.MAX)
+    total_s = float(total_ms.item()) * 1e-3
+    value = world * cfg.L * args.steps / total_s
+
+    # end to end through the host-buffer entry point
+    host_in = topk.cpu().pin_memory()
+    host_out = pl.alloc_host_outputs(("plan", "slot_expert", "slot_tokens", "X", "new_idx", "info"))
+    d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+    e2e_step = lambda: pl.plan_host(host_in, host_out)
+    timed_steps(e2e_step, 3, flush)
+    barrier(); torch.cuda.synchronize()
+    e2e_ms = timed_steps(e2e_step, args.steps, flush)
+    e2e_total = torch.tensor([float(sum(e2e_ms))], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(e2e_total, op=dist.ReduceOp.MAX)
+    e2e_value = world * cfg.L * args.steps / (float(e2e_total.item()) * 1e-3)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    dominant = int(np.argmax(stage_ms))
+    roof = roofline_for(STAGES[dominant], float(stage_ms[dominant]), cfg, out, peaks, props.multi_processor_count)
+    fma, iters = sinkhorn_work(out, cfg)
+    rounds = out["rounds"].cpu().numpy()
+    info = out["info"].cpu().numpy()
+    line = dict(
+        metric="placement plans/s (whole planner path: histogram, excess/spare, Sinkhorn, matching+auction, token remap)",
+        value=value, unit="plans/s", n_gpus=world, steps=args.steps, warmup=max(3, args.warmup),
+        ms_per_step=float(np.mean(ms)), higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
+        data="synthetic",
+        config=dict(workload=args.workload, L=cfg.L, R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k, T=cfg.T,
+                    eps=cfg.eps, max_iters=cfg.max_iters, tol=cfg.tol,
+                    l2="flushed between steps (256 MiB write)" if need_flush else "inputs larger than L2",
+                    parallelism=f"{world} independent replica(s)"),
+        remapped_tokens_per_s=world * cfg.L * cfg.T * args.steps / total_s,
+        stages_ms=dict(zip(STAGES, [float(x) for x in stage_ms])),
+        sinkhorn=dict(iters_mean=float(iters.mean()), iters_max=int(iters.max()),
+                      converged_frac=float(((info & 2) == 0).mean()),
+                      plans_per_s=cfg.L / (float(stage_ms[2]) * 1e-3)),
+        rounds=dict(phase2_max=int(rounds[:, 0].max()), phase3_max=int(rounds[:, 1].max())),
+        roofline=roof, clocks=clocks,
+        e2e=dict(value=e2e_value, unit="plans/s", h2d_bytes_per_step=topk_bytes, d2h_bytes_per_step=d2h,
+                 ms_per_step=float(np.mean(e2e_ms))),
+        gpu_launches=launches,
+    )
+    line["rooflines"] = {s: roofline_for(s, float(stage_ms[i]), cfg, out, peaks, props.multi_processor_count)
+                         for i, s in enumerate(STAGES)}
+
+    if world == 1 and not args.no_streams:
+        line["hbm_streams"] = [stream_report(nm, peaks) for nm in ("cfg3", "cfg4") if nm != args.workload]
+    if world == 1 and not args.no_cpu_baseline:
+        n_layers, secs = oracle_sample(cfg, topk.cpu().numpy(), args.cpu_seconds)
+        line["cpu_baseline"] = dict(value=n_layers / secs, unit="plans/s", cores=1, kind="oracle",
+                                    sample=f"{n_layers} whole layer(s) of {cfg.L}, {secs:.2f} s")
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

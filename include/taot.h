@@ -193,6 +193,16 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* out, v
 int taot_plan_host(taot_handle_t h, const int32_t* h_topk, const taot_outputs* out, void* d_ws,
                    void* stream);
 
+/*
+ * Stage timing for benchmarks.  With profiling on, taot_plan (and taot_plan_host) records one CUDA
+ * event on `stream` before the first kernel and one after each of its five kernels (chunk
+ * histogram, merge, Sinkhorn, matching+auction, reassignment).  taot_get_stage_ms waits for the
+ * last of them and returns the five durations of the most recent call in milliseconds.
+ * The events are created by taot_create and owned by the handle.
+ */
+int taot_set_profiling(taot_handle_t h, int32_t on);
+int taot_get_stage_ms(taot_handle_t h, float* h_ms /* [5] */);
+
 /* Kernels launched by the last call on this handle (for launch accounting). */
 int taot_last_launch_count(taot_handle_t h, int32_t* count);
 

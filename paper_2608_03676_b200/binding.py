@@ -22,7 +22,8 @@ INFO_SINKHORN_SIZE = 32
 _SYMBOLS = [
     "taot_create", "taot_destroy", "taot_workspace_bytes", "taot_host_workspace_bytes",
     "taot_histogram", "taot_excess_spare", "taot_sinkhorn", "taot_match", "taot_assign",
-    "taot_plan", "taot_plan_host", "taot_last_launch_count", "taot_status_string",
+    "taot_plan", "taot_plan_host", "taot_set_profiling", "taot_get_stage_ms", "taot_last_launch_count",
+    "taot_status_string",
 ]
 
 
@@ -161,6 +162,16 @@ class Planner:
         c = ctypes.c_int32()
         _check(self.lib.taot_last_launch_count(self.handle, ctypes.byref(c)), "taot_last_launch_count")
         return c.value
+
+    def set_profiling(self, on: bool):
+        _check(self.lib.taot_set_profiling(self.handle, ctypes.c_int32(1 if on else 0)), "taot_set_profiling")
+
+    def stage_ms(self):
+        """Durations (ms) of the five kernels of the last profiled plan call:
+        chunk histogram, merge, Sinkhorn, matching+auction, reassignment.  Waits for them."""
+        ms = (ctypes.c_float * 5)()
+        _check(self.lib.taot_get_stage_ms(self.handle, ms), "taot_get_stage_ms")
+        return [float(x) for x in ms]
 
     # ------------------------------------------------------------------ stages
     def histogram(self, topk: torch.Tensor, info: Optional[torch.Tensor] = None):

@@ -175,6 +175,8 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
     if (rc == TAOT_OK) rc = upload(&h->d_rowlse0, lse0.data(), (size_t)R);
     if (rc == TAOT_OK) rc = upload(&h->d_rank_off, off.data(), (size_t)R + 1);
     if (rc == TAOT_OK) rc = upload(&h->d_rank_list, list.data(), (size_t)E);
+    for (int i = 0; i < 6 && rc == TAOT_OK; ++i)
+        if (cudaEventCreate(&h->ev[i]) != cudaSuccess) rc = TAOT_ERR_CUDA;
     if (rc == TAOT_OK && cudaDeviceSynchronize() != cudaSuccess) rc = TAOT_ERR_CUDA;
     if (rc != TAOT_OK) {
         taot_destroy(h);
@@ -190,6 +192,8 @@ int taot_destroy(taot_handle_t h)
     cudaDeviceSynchronize();
     cudaFree(h->d_e2r); cudaFree(h->d_C); cudaFree(h->d_B); cudaFree(h->d_rowlse0);
     cudaFree(h->d_rank_off); cudaFree(h->d_rank_list);
+    for (int i = 0; i < 6; ++i)
+        if (h->ev[i]) cudaEventDestroy(h->ev[i]);
     delete h;
     return TAOT_OK;
 }
@@ -205,6 +209,21 @@ int taot_host_workspace_bytes(taot_handle_t h, size_t* bytes)
 {
     if (!h || !bytes) return TAOT_ERR_NULL;
     *bytes = h->host_ws_bytes;
+    return TAOT_OK;
+}
+
+int taot_set_profiling(taot_handle_t h, int32_t on)
+{
+    if (!h) return TAOT_ERR_NULL;
+    h->profiling = on ? 1 : 0;
+    return TAOT_OK;
+}
+
+int taot_get_stage_ms(taot_handle_t h, float* h_ms)
+{
+    if (!h || !h_ms) return TAOT_ERR_NULL;
+    TAOT_CUDA_OK(cudaEventSynchronize(h->ev[5]));
+    for (int i = 0; i < 5; ++i) TAOT_CUDA_OK(cudaEventElapsedTime(h_ms + i, h->ev[i], h->ev[i + 1]));
     return TAOT_OK;
 }
 
@@ -310,18 +329,26 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, voi
     float* fd = reinterpret_cast<float*>(at(ws, h->off_d));
     TAOT_CUDA_OK(cudaMemsetAsync(o->info, 0, sizeof(int32_t) * p.L, st));
     int total = 0, a;
+#define TAOT_MARK(i) if (h->profiling) TAOT_CUDA_OK(cudaEventRecord(h->ev[i], st))
+    TAOT_MARK(0);
     if ((a = taot_launch_histogram(h, d_topk, cc, o->info, st)) < 0) return a;
     total += a;
+    TAOT_MARK(1);
     if ((a = taot_launch_merge(h, cc, o->n, o->expert_load, o->rank_load, excess, spare, fs, fd, st)) < 0) return a;
     total += a;
+    TAOT_MARK(2);
     if ((a = taot_launch_sinkhorn(h, fs, fd, p.L, o->plan, o->sinkhorn_iters, o->row_err, o->info, st)) < 0) return a;
     total += a;
+    TAOT_MARK(3);
     if ((a = taot_launch_match(h, o->n, o->expert_load, o->rank_load, o->plan, o->slot_expert, o->slot_tokens,
                                o->X, o->rounds, o->info, reinterpret_cast<int32_t*>(at(ws, h->off_nrem)), st)) < 0)
         return a;
     total += a;
+    TAOT_MARK(4);
     if ((a = taot_launch_assign(h, d_topk, cc, o->slot_expert, o->X, o->new_idx, o->info, st)) < 0) return a;
     total += a;
+    TAOT_MARK(5);
+#undef TAOT_MARK
     h->last_launches = total;
     return TAOT_OK;
 }

@@ -36,6 +36,8 @@ struct taot_handle_s {
            hoff_se, hoff_st, hoff_X, hoff_rounds, hoff_info, hoff_ws;
     size_t host_ws_bytes;
     int32_t last_launches;
+    int32_t profiling;
+    cudaEvent_t ev[6];
 };
 
 static inline size_t taot_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
