@@ -199,6 +199,24 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count):
                      "(rounds x R x E and rounds x R x S), latency-bound by construction")
 
 
+def rank_config(cfg, rank: int):
+    """Every rank plans its own batch: same shape, seed offset by rank (independent replicas)."""
+    return cfg.replace(seed=cfg.seed + 7919 * rank)
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Slowest rank's device time (the step time of a synchronous job)."""
+    import torch.distributed as dist
+    t = torch.tensor([float(ms)], device=device, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank_per_step: int, steps: int, world: int, slowest_ms: float) -> float:
+    return world * units_per_rank_per_step * steps / (slowest_ms * 1e-3)
+
+
 def stream_report(name, peaks, steps=5):
     """Histogram and reassignment on an HBM-sized routing table (larger than L2): GB/s of each."""
     cfg = W.get_config(name)
@@ -272,7 +290,7 @@ def run_ours(args):
             dist.barrier()
 
     cfg = W.get_config(args.workload)
-    cfg = cfg.replace(seed=cfg.seed + 7919 * rank)            # every rank plans its own batch
+    cfg = rank_config(cfg, rank)
     peaks = measured_peaks()
     props = torch.cuda.get_device_properties(local)
     topk = W.routing_topk(cfg, device="cuda")
@@ -303,11 +321,8 @@ def run_ours(args):
     stage_ms /= args.steps
     clocks = sampler.stop() if rank == 0 else None
 
-    total_ms = torch.tensor([float(sum(ms))], device="cuda", dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(total_ms, op=dist.ReduceOp.MAX)
-    total_s = float(total_ms.item()) * 1e-3
-    value = world * cfg.L * args.steps / total_s
+    total_s = max_over_ranks(sum(ms), world, "cuda") * 1e-3
+    value = whole_job_rate(cfg.L, args.steps, world, total_s * 1e3)
 
     # end to end through the host-buffer entry point
     host_in = topk.cpu().pin_memory()
@@ -317,10 +332,7 @@ def run_ours(args):
     timed_steps(e2e_step, 3, flush)
     barrier(); torch.cuda.synchronize()
     e2e_ms = timed_steps(e2e_step, args.steps, flush)
-    e2e_total = torch.tensor([float(sum(e2e_ms))], device="cuda", dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(e2e_total, op=dist.ReduceOp.MAX)
-    e2e_value = world * cfg.L * args.steps / (float(e2e_total.item()) * 1e-3)
+    e2e_value = whole_job_rate(cfg.L, args.steps, world, max_over_ranks(sum(e2e_ms), world, "cuda"))
 
     if rank != 0:
         if world > 1:
