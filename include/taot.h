@@ -50,7 +50,8 @@ typedef enum {
     TAOT_ERR_PARAM = -2,        /* a parameter is out of its documented range */
     TAOT_ERR_UNSUPPORTED = -3,  /* a size is valid but beyond what this build supports */
     TAOT_ERR_CUDA = -4,         /* a CUDA runtime call failed (see cudaGetLastError) */
-    TAOT_ERR_ALIGN = -5         /* a device pointer is not aligned as required */
+    TAOT_ERR_ALIGN = -5,        /* a device pointer is not aligned as required */
+    TAOT_ERR_STATIC_CAPACITY = -6 /* the problem needs more than the built-in scratch of taot_histogram_static */
 } taot_status;
 
 /* bits of d_info[l] */
@@ -136,6 +137,39 @@ int taot_host_workspace_bytes(taot_handle_t h, size_t* bytes);
  */
 int taot_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_n, int32_t* d_expert_load,
                    int32_t* d_rank_load, int32_t* d_info, void* ws, void* stream);
+
+/*
+ * taot_histogram for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this is a packaging variant of the load collection above, not a step of the method.)
+ *
+ * Who needs it: code that runs inside a memory plan it does not own -- a plug-in of a serving or
+ * training runtime that has pre-carved all device memory, a stage called while its stream is being
+ * captured, a process whose pool is exhausted.  Such a caller cannot cudaMalloc a workspace (the
+ * call may fail, it synchronises the device, and it is not allowed during capture) and may not
+ * have one to spare.  This entry point needs no handle and no workspace and calls no allocating
+ * routine: the per-chunk counts it needs live in a fixed 256-byte-aligned device array of
+ * TAOT_STATIC_SCRATCH_BYTES that is part of the library image.  Every GPU on which the library is
+ * loaded holds that array until the process exits.
+ *
+ *   d_topk [L,T,k], d_e2r [E] (home rank of each expert, values in [0,R) -- not checked here),
+ *   d_n [L,R,E], d_expert_load [L,E], d_rank_load [L,R], d_info [L]: device memory of the caller,
+ *   same meaning, layout and overwrite rules as taot_histogram; d_info is OR-ed into.
+ *
+ * Limits and rules:
+ *   - L * R * ceil((T/R)*k / 16384) * E * 4 bytes must fit in TAOT_STATIC_SCRATCH_BYTES, otherwise
+ *     nothing is launched and TAOT_ERR_STATIC_CAPACITY is returned.  Other errors as taot_histogram.
+ *   - The first call on each device looks up the array's device address (with that device current).
+ *     Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents.  Each
+ *     call overwrites every count it later reads, so nothing needs clearing; but two calls whose
+ *     kernels overlap on the GPU (different streams, no dependency between them) race on it and
+ *     give wrong loads.  Serialise them.
+ *   - The per-chunk counts are not available to taot_assign afterwards (use reuse_counts = 0).
+ */
+#define TAOT_STATIC_SCRATCH_BYTES (4u << 20)
+int taot_histogram_static(const int32_t* d_topk, int32_t L, int64_t T, int32_t k, int32_t R, int32_t E,
+                          const int32_t* d_e2r, int32_t* d_n, int32_t* d_expert_load,
+                          int32_t* d_rank_load, int32_t* d_info, void* stream);
 
 /*
  * Excess / spare (Appendix A.1) against the integer mean m = floor(sum_r l_r / R), for B rows:

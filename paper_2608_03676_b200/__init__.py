@@ -17,4 +17,6 @@ from .binding import (  # noqa: F401
     library_path,
     load_library,
     exported_symbols,
+    histogram_static,
+    STATIC_SCRATCH_BYTES,
 )

@@ -21,7 +21,7 @@ INFO_SINKHORN_SIZE = 32
 
 _SYMBOLS = [
     "taot_create", "taot_destroy", "taot_workspace_bytes", "taot_host_workspace_bytes",
-    "taot_histogram", "taot_excess_spare", "taot_sinkhorn", "taot_match", "taot_assign",
+    "taot_histogram", "taot_histogram_static", "taot_excess_spare", "taot_sinkhorn", "taot_match", "taot_assign",
     "taot_plan", "taot_plan_host", "taot_set_profiling", "taot_get_stage_ms", "taot_last_launch_count",
     "taot_status_string",
 ]
@@ -90,6 +90,28 @@ def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
     if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
         raise TaotError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
     return t
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def histogram_static(topk: torch.Tensor, R: int, E: int, e2r_dev: torch.Tensor, n: torch.Tensor,
+                     expert_load: torch.Tensor, rank_load: torch.Tensor, info: torch.Tensor) -> int:
+    """Load collection through `taot_histogram_static`, the entry point for callers that cannot
+    allocate device memory: no handle, no workspace; the caller passes every input and output
+    (CUDA tensors it already owns) and gets the status code back instead of an exception, so that
+    a caller in a no-allocation region can decide what to do.  Problems whose per-chunk counts
+    exceed STATIC_SCRATCH_BYTES return the capacity error (-6) and launch nothing.  Calls share one
+    built-in scratch array per GPU: do not let two of them overlap on the device."""
+    lib = load_library()
+    L, T, k = topk.shape
+    for t, dt, nm in ((topk, torch.int32, "topk"), (e2r_dev, torch.int32, "e2r"), (n, torch.int32, "n"),
+                      (expert_load, torch.int32, "expert_load"), (rank_load, torch.int32, "rank_load"),
+                      (info, torch.int32, "info")):
+        _dev(t, dt, nm)
+    return int(lib.taot_histogram_static(_ptr(topk), ctypes.c_int32(L), ctypes.c_int64(T), ctypes.c_int32(k),
+                                         ctypes.c_int32(R), ctypes.c_int32(E), _ptr(e2r_dev), _ptr(n),
+                                         _ptr(expert_load), _ptr(rank_load), _ptr(info), _stream()))
 
 
 @dataclass

@@ -95,6 +95,9 @@ const char* taot_status_string(int status)
         case TAOT_ERR_UNSUPPORTED: return "size not supported by this build";
         case TAOT_ERR_CUDA: return "a CUDA runtime call failed";
         case TAOT_ERR_ALIGN: return "a device pointer is misaligned";
+        case TAOT_ERR_STATIC_CAPACITY:
+            return "taot_histogram_static: L*R*chunks*E*4 bytes of per-chunk counts exceed the built-in "
+                   "scratch (TAOT_STATIC_SCRATCH_BYTES); use taot_histogram with a workspace";
         default: return "unknown status";
     }
 }

@@ -7,6 +7,9 @@
 // counts into per-warp private shared-memory histograms, and stores its E counts with plain
 // stores -- no global atomics, no zero-fill of the outputs.  The per-chunk counts are kept: the
 // reassignment kernel turns them into each chunk's starting ordinals.
+#include <cstring>
+#include <mutex>
+
 #include "taot_internal.cuh"
 
 namespace {
@@ -188,4 +191,72 @@ int taot_launch_excess_spare(taot_handle_t h, const int32_t* d_rank_load, int32_
     excess_spare_kernel<<<B, 256, sizeof(int32_t) * p.R, st>>>(d_rank_load, d_excess, d_spare, d_s, d_d, p.R);
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Load collection for callers that cannot allocate device memory.
+//
+// taot_histogram needs a caller-supplied workspace for its per-chunk counts.  A caller that sits
+// inside someone else's memory plan -- a plug-in of a serving runtime whose device memory is fully
+// pre-carved, code running between the stages of a captured step, a process whose memory pool is
+// already exhausted -- may have no way of getting one: cudaMalloc is off limits there (it can
+// fail, it synchronises the device, and it is illegal during stream capture).  For those callers
+// the per-chunk counts live in the fixed array below, which is part of the library image: every GPU
+// that loads libtaot.so carries these 4 MiB until the process exits, whether or not the entry point
+// is ever called.
+namespace {
+
+static __device__ __align__(256) unsigned char g_static_counts[TAOT_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+int32_t* g_static_counts_addr[kMaxDevices] = {nullptr};   // device address of g_static_counts, per device
+
+}  // namespace
+
+extern "C" int taot_histogram_static(const int32_t* d_topk, int32_t L, int64_t T, int32_t k, int32_t R,
+                                     int32_t E, const int32_t* d_e2r, int32_t* d_n, int32_t* d_expert_load,
+                                     int32_t* d_rank_load, int32_t* d_info, void* stream)
+{
+    if (!d_topk || !d_e2r || !d_n || !d_expert_load || !d_rank_load || !d_info) return TAOT_ERR_NULL;
+    if (L < 1 || R < 1 || E < 1 || k < 1 || T < R || T % R != 0 || T * (int64_t)k >= ((int64_t)1 << 31))
+        return TAOT_ERR_PARAM;
+    if (R > 256 || E > 1024 || k > 64) return TAOT_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(d_topk) & 3) return TAOT_ERR_ALIGN;
+    const int64_t seg = T / R * k;
+    const int64_t nc = (seg + TAOT_CHUNK - 1) / TAOT_CHUNK;
+    const int64_t need = (int64_t)L * R * nc * E * (int64_t)sizeof(int32_t);
+    if (need > (int64_t)TAOT_STATIC_SCRATCH_BYTES) return TAOT_ERR_STATIC_CAPACITY;
+
+    // Set-up, once per device, with that device current: in host code `g_static_counts` is only a
+    // stand-in for the symbol, so the address a kernel can use has to be asked for.
+    int dev = -1;
+    TAOT_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return TAOT_ERR_UNSUPPORTED;
+    int32_t* counts = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_counts_addr[dev]) {
+            void* addr = nullptr;
+            if (cudaGetSymbolAddress(&addr, g_static_counts) != cudaSuccess || !addr) return TAOT_ERR_CUDA;
+            g_static_counts_addr[dev] = static_cast<int32_t*>(addr);
+        }
+        counts = g_static_counts_addr[dev];
+    }
+
+    // The kernels are the ones taot_histogram runs; they read only these fields of a handle.
+    taot_handle_s view;
+    std::memset(&view, 0, sizeof(view));
+    view.p.L = L; view.p.R = R; view.p.E = E; view.p.k = k; view.p.T = T;
+    view.seg = seg;
+    view.nc = (int32_t)nc;
+    view.d_e2r = const_cast<int32_t*>(d_e2r);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // Nothing in the array has to start at zero: every chunk's CTA overwrites all E of its counts
+    // with plain stores before the merge kernel reads them.
+    int a = taot_launch_histogram(&view, d_topk, counts, d_info, st);
+    if (a < 0) return a;
+    int b = taot_launch_merge(&view, counts, d_n, d_expert_load, d_rank_load, nullptr, nullptr, nullptr, nullptr, st);
+    if (b < 0) return b;
+    return TAOT_OK;
 }
