@@ -43,6 +43,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="cfg2", choices=sorted(W.CONFIGS))
+    ap.add_argument("--layers", type=int, default=0, help="override L (smaller batch, e.g. for a profiler capture)")
     ap.add_argument("--cpu-seconds", type=float, default=20.0, help="budget of the CPU-baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-streams", action="store_true", help="skip the HBM-sized streaming report")
@@ -254,6 +255,8 @@ def run_reference(args):
     if rank != 0:
         return
     cfg = W.get_config(args.workload)
+    if args.layers > 0:
+        cfg = cfg.replace(L=args.layers)
     dev = "cuda" if torch.cuda.is_available() else "cpu"
     topk = W.routing_topk(cfg, device=dev).cpu().numpy()
     per_step = max(2.0, min(args.cpu_seconds, 60.0 / max(1, args.steps + args.warmup)))
@@ -290,6 +293,8 @@ def run_ours(args):
             dist.barrier()
 
     cfg = W.get_config(args.workload)
+    if args.layers > 0:
+        cfg = cfg.replace(L=args.layers)
     cfg = rank_config(cfg, rank)
     peaks = measured_peaks()
     props = torch.cuda.get_device_properties(local)

@@ -4,13 +4,14 @@
 // Formulation; the paper fixes the counts X, this rule fixes which entries.)
 //
 // One CTA per chunk of at most TAOT_CHUNK entries, the same chunks the histogram kernel counted.
-// The chunk is loaded once into registers (64 entries per thread, all loads issued up front).
-// From the per-chunk counts the CTA knows, for every expert, the ordinal range its entries
-// occupy inside the (rank, expert) group; if that range falls inside one slot's quota (or
-// outside all of them) the whole chunk maps that expert to one target and a shared-memory table
-// lookup suffices.  Only experts whose range straddles a quota boundary need per-entry ordinals,
-// which come from warp ballots over the register-resident chunk.  8 bytes of HBM traffic per
-// entry: one read, one write.
+// The chunk is loaded once into registers (64 entries per thread, all loads issued up front);
+// each warp owns 2048 contiguous entries.  The chunk counts of the histogram pass give the ordinal
+// at which each expert's entries start in this chunk; a per-warp shared-memory histogram refines
+// that to the start inside each warp's span.  If a warp's ordinal range for an expert falls inside
+// one slot's quota (or outside all of them) every such entry of the warp has the same target and a
+// per-warp lookup table suffices; only a (warp, expert) pair whose range straddles a quota boundary
+// -- a handful per layer -- gets exact per-entry ordinals from warp ballots.  8 bytes of HBM traffic
+// per entry: one read, one write.
 #include "taot_internal.cuh"
 
 namespace {
@@ -44,21 +45,20 @@ __device__ __forceinline__ void st_stream(int4* p, const int4& v)
     asm volatile("st.global.cs.v4.s32 [%0], {%1,%2,%3,%4};" :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
+template <bool VEC>
 __global__ void __launch_bounds__(kThreads)
 assign_kernel(AssignArgs a)
 {
     extern __shared__ int32_t sh[];
     const int E = a.E, S = a.R * a.K;
-    int32_t* tab = sh;                  // [E]  >= 0: target for the whole chunk; -(1+b): boundary expert b
-    int32_t* base = tab + E;            // [E]  ordinal of the chunk's first entry of e within (rank, e)
-    int32_t* blist = base + E;          // [E]  boundary experts
-    int32_t* cntw = blist + E;          // [E * kWarps] per-warp counts of each boundary expert
-    int32_t* ent_s = cntw + E * kWarps; // [S]  slots this source rank feeds, ascending
+    int32_t* hw = sh;                   // [kWarps][E] per-warp histogram of the warp's 2048 entries
+    int32_t* tabw = hw + kWarps * E;    // [kWarps][E] per-warp target table (-1: straddles a quota boundary)
+    int32_t* base = tabw + kWarps * E;  // [E]  ordinal of the chunk's first entry of e within (rank, e)
+    int32_t* ent_s = base + E;          // [S]  slots this source rank feeds, ascending
     int32_t* ent_e = ent_s + S;         // [S]  their expert
     int32_t* ent_lo = ent_e + S;        // [S]  first ordinal the slot takes
     int32_t* ent_hi = ent_lo + S;       // [S]  one past the last
     __shared__ int s_wcnt[kWarps];
-    __shared__ int s_nb;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int64_t id = blockIdx.x;
@@ -74,22 +74,11 @@ assign_kernel(AssignArgs a)
     // ---- the chunk, in registers; warp w owns entries [w*2048, w*2048+2048), 128 per iteration
     int4 x[kIters];
     const int32_t wbase_elem = warp * kWarpSpan + lane * 4;
-    if (a.vec_ok) {
 #pragma unroll
-        for (int it = 0; it < kIters; ++it) {
-            const int32_t pos = wbase_elem + it * 128;
-            if (pos + 3 < len) x[it] = ld_stream(reinterpret_cast<const int4*>(src + pos));
-            else {
-                x[it].x = pos < len ? src[pos] : -1;
-                x[it].y = pos + 1 < len ? src[pos + 1] : -1;
-                x[it].z = pos + 2 < len ? src[pos + 2] : -1;
-                x[it].w = -1;
-            }
-        }
-    } else {
-#pragma unroll
-        for (int it = 0; it < kIters; ++it) {
-            const int32_t pos = wbase_elem + it * 128;
+    for (int it = 0; it < kIters; ++it) {
+        const int32_t pos = wbase_elem + it * 128;
+        if (VEC && pos + 3 < len) x[it] = ld_stream(reinterpret_cast<const int4*>(src + pos));
+        else {
             x[it].x = pos < len ? src[pos] : -1;
             x[it].y = pos + 1 < len ? src[pos + 1] : -1;
             x[it].z = pos + 2 < len ? src[pos + 2] : -1;
@@ -97,7 +86,14 @@ assign_kernel(AssignArgs a)
         }
     }
 
-    // ---- slots fed by this source rank (X > 0), ascending slot order
+    // ---- while the loads fly: zero the histograms, chunk-start ordinals, the slots this rank feeds
+    for (int i = tid; i < kWarps * E; i += kThreads) hw[i] = 0;
+    const int32_t* ccseg = a.cc + lr * a.nc * (int64_t)E;
+    for (int e = tid; e < E; e += kThreads) {
+        int32_t b = 0;
+        for (int cp = 0; cp < c; ++cp) b += ccseg[(int64_t)cp * E + e];
+        base[e] = b;
+    }
     const int32_t* Xrow = a.X + lr * S;
     const int32_t* se = a.slot_expert + (int64_t)l * S;
     int m = 0;
@@ -118,15 +114,6 @@ assign_kernel(AssignArgs a)
         for (int w = 0; w < kWarps; ++w) m += s_wcnt[w];
         __syncthreads();
     }
-    // ---- chunk-start ordinal and default target per expert
-    const int32_t* ccseg = a.cc + lr * a.nc * (int64_t)E;
-    for (int e = tid; e < E; e += kThreads) {
-        int32_t b = 0;
-        for (int cp = 0; cp < c; ++cp) b += ccseg[(int64_t)cp * E + e];
-        base[e] = b;
-        tab[e] = e;
-    }
-    if (tid == 0) s_nb = 0;
     // ordinal interval [lo, hi) each entry takes within its (rank, expert) group
     for (int q = tid; q < m; q += kThreads) {
         const int e = ent_e[q];
@@ -136,45 +123,54 @@ assign_kernel(AssignArgs a)
     }
     __syncthreads();
     for (int q = tid; q < m; q += kThreads) ent_hi[q] += ent_lo[q];
-    __syncthreads();
-    // classify: whole chunk range inside one interval -> table; straddling -> boundary expert
-    for (int q = tid; q < m; q += kThreads) {
-        const int e = ent_e[q];
-        const int32_t cnt = ccseg[(int64_t)c * E + e];
-        const int32_t b = base[e];
-        if (cnt == 0 || ent_hi[q] <= b || ent_lo[q] >= b + cnt) continue;
-        if (ent_lo[q] <= b && ent_hi[q] >= b + cnt) tab[e] = E + ent_s[q];
-        else tab[e] = -1;
-    }
-    __syncthreads();
-    for (int e = tid; e < E; e += kThreads)
-        if (tab[e] == -1) {
-            const int bi = atomicAdd(&s_nb, 1);
-            blist[bi] = e;
-            tab[e] = -(1 + bi);
-        }
-    __syncthreads();
-    const int nb = s_nb;
 
-    // ---- boundary experts: exact ordinals from ballots over the register-resident chunk
-    unsigned long long done = 0ull;
-    if (nb > 0) {
-        for (int bi = 0; bi < nb; ++bi) {
-            const int eb = blist[bi];
-            int cnt = 0;
+    // ---- per-warp histogram of the register-resident entries
+    int32_t* myh = hw + warp * E;
+    int bad = 0;
 #pragma unroll
-            for (int it = 0; it < kIters; ++it)
-                cnt += (x[it].x == eb) + (x[it].y == eb) + (x[it].z == eb) + (x[it].w == eb);
-            for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-            if (lane == 0) cntw[bi * kWarps + warp] = cnt;
+    for (int it = 0; it < kIters; ++it) {
+        const int32_t* xv = reinterpret_cast<const int32_t*>(&x[it]);
+        const int32_t pos = wbase_elem + it * 128;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int32_t e = xv[j];
+            if ((uint32_t)e < (uint32_t)E) atomicAdd(myh + e, 1);
+            else if (pos + j < len) bad = 1;
         }
-        __syncthreads();
-        const unsigned lt = (1u << lane) - 1u;
-        for (int bi = 0; bi < nb; ++bi) {
-            const int eb = blist[bi];
+    }
+    bad = __syncthreads_or(bad);          // also: every warp's histogram and ent_hi are complete
+
+    // ---- this warp's table: default e; entries of this source rank override where they apply
+    int32_t* myt = tabw + warp * E;
+    for (int e = lane; e < E; e += 32) myt[e] = e;
+    __syncwarp();
+    for (int q = lane; q < m; q += 32) {
+        const int e = ent_e[q];
+        const int32_t cnt = myh[e];
+        if (cnt == 0) continue;
+        int32_t st = base[e];
+        for (int w = 0; w < warp; ++w) st += hw[w * E + e];
+        if (ent_hi[q] <= st || ent_lo[q] >= st + cnt) continue;
+        myt[e] = (ent_lo[q] <= st && ent_hi[q] >= st + cnt) ? E + ent_s[q] : -1;   // at most one full cover
+    }
+    __syncwarp();
+
+    // ---- (warp, expert) pairs that straddle a quota boundary: exact ordinals from ballots
+    for (int eb0 = 0; eb0 < E; eb0 += 32) {
+        const int ecand = eb0 + lane;
+        unsigned todo = __ballot_sync(0xffffffffu, ecand < E && myt[ecand] == -1);
+        while (todo) {
+            const int eb = eb0 + __ffs(todo) - 1;
+            todo &= todo - 1;
             int32_t running = base[eb];
-            for (int w = 0; w < warp; ++w) running += cntw[bi * kWarps + w];
-            if (cntw[bi * kWarps + warp] == 0) continue;
+            for (int w = 0; w < warp; ++w) running += hw[w * E + eb];
+            const int32_t mine = myh[eb];
+            int q0 = m, q1 = m;                  // entries of eb whose interval can touch [running, running+mine)
+            for (int q = 0; q < m; ++q)
+                if (ent_e[q] == eb && ent_hi[q] > running) { q0 = q; break; }
+            for (int q = q0; q < m; ++q)
+                if (ent_e[q] == eb && ent_lo[q] >= running + mine) { q1 = q; break; }
+            const unsigned lt = (1u << lane) - 1u;
 #pragma unroll
             for (int it = 0; it < kIters; ++it) {
                 int32_t* xv = reinterpret_cast<int32_t*>(&x[it]);
@@ -187,57 +183,37 @@ assign_kernel(AssignArgs a)
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     if (mm[j]) {
-                        int32_t target = eb;
-                        for (int q = 0; q < m; ++q)
-                            if (ent_e[q] == eb && ord >= ent_lo[q] && ord < ent_hi[q]) { target = E + ent_s[q]; break; }
-                        xv[j] = target;
-                        done |= 1ull << (it * 4 + j);
+                        for (int q = q0; q < q1; ++q)
+                            if (ent_e[q] == eb && ord >= ent_lo[q] && ord < ent_hi[q]) { xv[j] = E + ent_s[q]; break; }
                         ++ord;
                     }
                 }
                 running += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
             }
+            // what is still eb in the registers stays eb; moved entries are now >= E and pass through
+            if (lane == 0) myt[eb] = eb;
         }
+        __syncwarp();
     }
 
-    // ---- everything else: one table lookup per entry
-    int bad = 0;
+    // ---- one table lookup per entry (values >= E or < 0 pass through unchanged), then store
 #pragma unroll
     for (int it = 0; it < kIters; ++it) {
         int32_t* xv = reinterpret_cast<int32_t*>(&x[it]);
-        const int32_t pos = wbase_elem + it * 128;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            if ((done >> (it * 4 + j)) & 1ull) continue;
             const int32_t e = xv[j];
-            if ((uint32_t)e < (uint32_t)E) xv[j] = tab[e];
-            else if (pos + j < len) bad = 1;
+            if ((uint32_t)e < (uint32_t)E) xv[j] = myt[e];
         }
-    }
-
-    // ---- store
-    if (a.vec_ok) {
-#pragma unroll
-        for (int it = 0; it < kIters; ++it) {
-            const int32_t pos = wbase_elem + it * 128;
-            if (pos + 3 < len) st_stream(reinterpret_cast<int4*>(dst + pos), x[it]);
-            else {
-                if (pos < len) dst[pos] = x[it].x;
-                if (pos + 1 < len) dst[pos + 1] = x[it].y;
-                if (pos + 2 < len) dst[pos + 2] = x[it].z;
-            }
-        }
-    } else {
-#pragma unroll
-        for (int it = 0; it < kIters; ++it) {
-            const int32_t pos = wbase_elem + it * 128;
+        const int32_t pos = wbase_elem + it * 128;
+        if (VEC && pos + 3 < len) st_stream(reinterpret_cast<int4*>(dst + pos), x[it]);
+        else {
             if (pos < len) dst[pos] = x[it].x;
             if (pos + 1 < len) dst[pos + 1] = x[it].y;
             if (pos + 2 < len) dst[pos + 2] = x[it].z;
             if (pos + 3 < len) dst[pos + 3] = x[it].w;
         }
     }
-    bad = __syncthreads_or(bad);
     if (bad && tid == 0) atomicOr(a.info + l, TAOT_INFO_BAD_INDEX);
 }
 
@@ -254,10 +230,15 @@ int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_
     a.vec_ok = ((reinterpret_cast<uintptr_t>(d_topk) & 15) == 0) &&
                ((reinterpret_cast<uintptr_t>(d_new_idx) & 15) == 0) && (h->seg % 4 == 0);
     const int S = p.R * p.K;
-    const size_t smem = sizeof(int32_t) * ((size_t)p.E * (3 + kWarps) + 4 * (size_t)S);
-    TAOT_CUDA_OK(cudaFuncSetAttribute(assign_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const size_t smem = sizeof(int32_t) * ((size_t)p.E * (2 * kWarps + 1) + 4 * (size_t)S);
     const int64_t blocks = (int64_t)p.L * p.R * h->nc;
-    assign_kernel<<<(unsigned)blocks, kThreads, smem, st>>>(a);
+    if (a.vec_ok) {
+        TAOT_CUDA_OK(cudaFuncSetAttribute(assign_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        assign_kernel<true><<<(unsigned)blocks, kThreads, smem, st>>>(a);
+    } else {
+        TAOT_CUDA_OK(cudaFuncSetAttribute(assign_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        assign_kernel<false><<<(unsigned)blocks, kThreads, smem, st>>>(a);
+    }
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
 }
