@@ -229,9 +229,10 @@ int taot_plan_host(taot_handle_t h, const int32_t* h_topk, const taot_outputs* o
 
 /*
  * Stage timing for benchmarks.  With profiling on, taot_plan (and taot_plan_host) records one CUDA
- * event on `stream` before the first kernel and one after each of its five kernels (chunk
- * histogram, merge, Sinkhorn, matching+auction, reassignment).  taot_get_stage_ms waits for the
- * last of them and returns the five durations of the most recent call in milliseconds.
+ * event on `stream` before the first kernel and one after each of its five stages (chunk
+ * histogram; merge; Sinkhorn; matching + auction; reassignment = table build + rewrite kernels).
+ * taot_get_stage_ms waits for the last of them and returns the five durations of the most recent
+ * call in milliseconds.
  * The events are created by taot_create and owned by the handle.
  */
 int taot_set_profiling(taot_handle_t h, int32_t on);

@@ -5,13 +5,17 @@
 //
 // One CTA per chunk of at most TAOT_CHUNK entries, the same chunks the histogram kernel counted.
 // The chunk is loaded once into registers (64 entries per thread, all loads issued up front);
-// each warp owns 2048 contiguous entries.  The chunk counts of the histogram pass give the ordinal
-// at which each expert's entries start in this chunk; a per-warp shared-memory histogram refines
-// that to the start inside each warp's span.  If a warp's ordinal range for an expert falls inside
-// one slot's quota (or outside all of them) every such entry of the warp has the same target and a
-// per-warp lookup table suffices; only a (warp, expert) pair whose range straddles a quota boundary
-// -- a handful per layer -- gets exact per-entry ordinals from warp ballots.  8 bytes of HBM traffic
-// per entry: one read, one write.
+// each warp owns 2048 contiguous entries.  The chunk counts of the histogram pass give, for every
+// expert, the ordinal range its entries occupy in this chunk.  If that range falls inside one
+// slot's quota (or outside all of them) every such entry of the chunk has the same target: one
+// shared-memory table lookup per entry, and that is all most chunks need.  An expert whose range
+// straddles a quota boundary (about one chunk in five has one) is counted per warp from the
+// registers; warps that do not contain the boundary still get a single target for it, and only the
+// one warp that does computes exact per-entry ordinals from ballots.  The per-chunk tables are built
+// by a small kernel with one CTA per (layer, source rank) segment, so that the streaming kernel's
+// common path is: 16 loads in flight, one table row from L2, 64 lookups, 16 stores.  8 bytes of HBM
+// traffic per entry: one read, one write.  Out-of-range indices are copied through (the histogram pass, whose
+// counts this kernel consumes, is the one that flags them).
 #include "taot_internal.cuh"
 
 namespace {
@@ -24,6 +28,8 @@ constexpr int kWarpSpan = TAOT_CHUNK / kWarps;           // entries one warp own
 struct AssignArgs {
     const int32_t* topk;
     const int32_t* cc;
+    int32_t* tabg;          // [L,R,NC,E] per-chunk target tables written by the prep kernel
+    int32_t* nbg;           // [L,R,NC]   number of boundary experts of each chunk
     const int32_t* slot_expert;
     const int32_t* X;
     int32_t* out;
@@ -45,57 +51,13 @@ __device__ __forceinline__ void st_stream(int4* p, const int4& v)
     asm volatile("st.global.cs.v4.s32 [%0], {%1,%2,%3,%4};" :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
-template <bool VEC>
-__global__ void __launch_bounds__(kThreads)
-assign_kernel(AssignArgs a)
+// Shared by both kernels: the slots this source rank feeds (X > 0), ascending, with the ordinal
+// interval [lo, hi) each takes inside its (rank, expert) group.  Returns the number of entries.
+// On return ent_hi holds COUNTS (hi - lo); the caller adds ent_lo after its last use of the counts.
+__device__ int build_entries(const int32_t* Xrow, const int32_t* se, int S, int E, int32_t* ent_s,
+                             int32_t* ent_e, int32_t* ent_lo, int32_t* ent_hi, int* s_wcnt)
 {
-    extern __shared__ int32_t sh[];
-    const int E = a.E, S = a.R * a.K;
-    int32_t* hw = sh;                   // [kWarps][E] per-warp histogram of the warp's 2048 entries
-    int32_t* tabw = hw + kWarps * E;    // [kWarps][E] per-warp target table (-1: straddles a quota boundary)
-    int32_t* base = tabw + kWarps * E;  // [E]  ordinal of the chunk's first entry of e within (rank, e)
-    int32_t* ent_s = base + E;          // [S]  slots this source rank feeds, ascending
-    int32_t* ent_e = ent_s + S;         // [S]  their expert
-    int32_t* ent_lo = ent_e + S;        // [S]  first ordinal the slot takes
-    int32_t* ent_hi = ent_lo + S;       // [S]  one past the last
-    __shared__ int s_wcnt[kWarps];
-
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t id = blockIdx.x;
-    const int32_t c = (int32_t)(id % a.nc);
-    const int64_t lr = id / a.nc;
-    const int32_t l = (int32_t)(lr / a.R);
-    const int64_t start = (int64_t)c * TAOT_CHUNK;
-    const int32_t len = (int32_t)((a.seg - start) < (int64_t)TAOT_CHUNK ? (a.seg - start) : (int64_t)TAOT_CHUNK);
-    const int64_t goff = (int64_t)l * a.layer_elems + (lr % a.R) * a.seg + start;
-    const int32_t* src = a.topk + goff;
-    int32_t* dst = a.out + goff;
-
-    // ---- the chunk, in registers; warp w owns entries [w*2048, w*2048+2048), 128 per iteration
-    int4 x[kIters];
-    const int32_t wbase_elem = warp * kWarpSpan + lane * 4;
-#pragma unroll
-    for (int it = 0; it < kIters; ++it) {
-        const int32_t pos = wbase_elem + it * 128;
-        if (VEC && pos + 3 < len) x[it] = ld_stream(reinterpret_cast<const int4*>(src + pos));
-        else {
-            x[it].x = pos < len ? src[pos] : -1;
-            x[it].y = pos + 1 < len ? src[pos + 1] : -1;
-            x[it].z = pos + 2 < len ? src[pos + 2] : -1;
-            x[it].w = pos + 3 < len ? src[pos + 3] : -1;
-        }
-    }
-
-    // ---- while the loads fly: zero the histograms, chunk-start ordinals, the slots this rank feeds
-    for (int i = tid; i < kWarps * E; i += kThreads) hw[i] = 0;
-    const int32_t* ccseg = a.cc + lr * a.nc * (int64_t)E;
-    for (int e = tid; e < E; e += kThreads) {
-        int32_t b = 0;
-        for (int cp = 0; cp < c; ++cp) b += ccseg[(int64_t)cp * E + e];
-        base[e] = b;
-    }
-    const int32_t* Xrow = a.X + lr * S;
-    const int32_t* se = a.slot_expert + (int64_t)l * S;
     int m = 0;
     for (int sb = 0; sb < S; sb += kThreads) {
         const int s = sb + tid;
@@ -109,12 +71,11 @@ assign_kernel(AssignArgs a)
         for (int w = 0; w < warp; ++w) off += s_wcnt[w];
         if (p) {
             const int q = off + __popc(bal & ((1u << lane) - 1u));
-            ent_s[q] = s; ent_e[q] = ev; ent_hi[q] = xv;     // hi holds the count until the prefix below
+            ent_s[q] = s; ent_e[q] = ev; ent_hi[q] = xv;
         }
         for (int w = 0; w < kWarps; ++w) m += s_wcnt[w];
         __syncthreads();
     }
-    // ordinal interval [lo, hi) each entry takes within its (rank, expert) group
     for (int q = tid; q < m; q += kThreads) {
         const int e = ent_e[q];
         int32_t lo = 0;
@@ -122,55 +83,162 @@ assign_kernel(AssignArgs a)
         ent_lo[q] = lo;
     }
     __syncthreads();
-    for (int q = tid; q < m; q += kThreads) ent_hi[q] += ent_lo[q];
+    return m;
+}
 
-    // ---- per-warp histogram of the register-resident entries
-    int32_t* myh = hw + warp * E;
-    int bad = 0;
+// One CTA per (layer, source rank): the target table of every chunk of the segment.
+// tab[e] = e (stays), E + s (the chunk's whole ordinal range of e lies in slot s's quota) or -1
+// (the range straddles a quota boundary: a boundary expert of that chunk).
+__global__ void __launch_bounds__(kThreads)
+assign_prep_kernel(AssignArgs a)
+{
+    extern __shared__ int32_t sh[];
+    const int E = a.E, S = a.R * a.K;
+    int32_t* tab = sh;                  // [E]
+    int32_t* base = tab + E;            // [E] running ordinal at the start of the current chunk
+    int32_t* ent_s = base + E;          // [S]
+    int32_t* ent_e = ent_s + S;
+    int32_t* ent_lo = ent_e + S;
+    int32_t* ent_hi = ent_lo + S;
+    __shared__ int s_wcnt[kWarps];
+    __shared__ int s_nb;
+    const int tid = threadIdx.x;
+    const int64_t lr = blockIdx.x;
+    const int32_t l = (int32_t)(lr / a.R);
+    const int m = build_entries(a.X + lr * S, a.slot_expert + (int64_t)l * S, S, E, ent_s, ent_e, ent_lo, ent_hi, s_wcnt);
+    for (int e = tid; e < E; e += kThreads) base[e] = 0;
+    const int32_t* ccseg = a.cc + lr * a.nc * (int64_t)E;
+    for (int c = 0; c < a.nc; ++c) {
+        for (int e = tid; e < E; e += kThreads) tab[e] = e;
+        if (tid == 0) s_nb = 0;
+        __syncthreads();
+        for (int q = tid; q < m; q += kThreads) {
+            const int e = ent_e[q];
+            const int32_t lo = ent_lo[q], hi = lo + ent_hi[q];
+            const int32_t cnt = ccseg[(int64_t)c * E + e];
+            const int32_t b = base[e];
+            if (!(cnt == 0 || hi <= b || lo >= b + cnt))
+                tab[e] = (lo <= b && hi >= b + cnt) ? E + ent_s[q] : -1;      // at most one full cover per expert
+        }
+        __syncthreads();
+        int32_t* out = a.tabg + (lr * a.nc + c) * (int64_t)E;
+        for (int e = tid; e < E; e += kThreads) {
+            const int32_t t = tab[e];
+            out[e] = t;
+            if (t == -1) atomicAdd(&s_nb, 1);
+            base[e] += ccseg[(int64_t)c * E + e];
+        }
+        __syncthreads();
+        if (tid == 0) a.nbg[lr * a.nc + c] = s_nb;
+        __syncthreads();
+    }
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(kThreads, 2)
+assign_kernel(AssignArgs a)
+{
+    extern __shared__ int32_t sh[];
+    const int E = a.E, S = a.R * a.K;
+    int32_t* tab = sh;                  // [E]  >= 0: target for the whole chunk; -(1+b): boundary expert b
+    int32_t* base = tab + E;            // [E]  ordinal of the chunk's first entry of e within (rank, e)
+    int32_t* blist = base + E;          // [E]  boundary experts of this chunk
+    int32_t* cntw = blist + E;          // [E * kWarps] per-warp counts of each boundary expert
+    int32_t* wtab = cntw + E * kWarps;  // [kWarps][E] per-warp tables, used only if the chunk has a boundary expert
+    int32_t* ent_s = wtab + E * kWarps; // [S]  slots this source rank feeds, ascending
+    int32_t* ent_e = ent_s + S;         // [S]  their expert
+    int32_t* ent_lo = ent_e + S;        // [S]  first ordinal the slot takes
+    int32_t* ent_hi = ent_lo + S;       // [S]  one past the last
+    __shared__ int s_wcnt[kWarps];
+    __shared__ int s_nb;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t id = blockIdx.x;
+    const int nb = a.nbg[id];
+    const int32_t c = (int32_t)(id % a.nc);
+    const int64_t lr = id / a.nc;
+    const int32_t l = (int32_t)(lr / a.R);
+    const int64_t start = (int64_t)c * TAOT_CHUNK;
+    const int32_t len = (int32_t)((a.seg - start) < (int64_t)TAOT_CHUNK ? (a.seg - start) : (int64_t)TAOT_CHUNK);
+    const int64_t goff = (int64_t)l * a.layer_elems + (lr % a.R) * a.seg + start;
+    const int32_t* src = a.topk + goff;
+    int32_t* dst = a.out + goff;
+    const bool full = VEC && (len == TAOT_CHUNK);
+
+    // ---- the chunk, in registers; warp w owns entries [w*2048, w*2048+2048), 128 per iteration
+    int4 x[kIters];
+    const int32_t wbase_elem = warp * kWarpSpan + lane * 4;
+    if (full) {
 #pragma unroll
-    for (int it = 0; it < kIters; ++it) {
-        const int32_t* xv = reinterpret_cast<const int32_t*>(&x[it]);
-        const int32_t pos = wbase_elem + it * 128;
+        for (int it = 0; it < kIters; ++it)
+            x[it] = ld_stream(reinterpret_cast<const int4*>(src + wbase_elem + it * 128));
+    } else {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int32_t e = xv[j];
-            if ((uint32_t)e < (uint32_t)E) atomicAdd(myh + e, 1);
-            else if (pos + j < len) bad = 1;
+        for (int it = 0; it < kIters; ++it) {
+            const int32_t pos = wbase_elem + it * 128;
+            x[it].x = pos < len ? src[pos] : -1;
+            x[it].y = pos + 1 < len ? src[pos + 1] : -1;
+            x[it].z = pos + 2 < len ? src[pos + 2] : -1;
+            x[it].w = pos + 3 < len ? src[pos + 3] : -1;
         }
     }
-    bad = __syncthreads_or(bad);          // also: every warp's histogram and ent_hi are complete
 
-    // ---- this warp's table: default e; entries of this source rank override where they apply
-    int32_t* myt = tabw + warp * E;
-    for (int e = lane; e < E; e += 32) myt[e] = e;
-    __syncwarp();
-    for (int q = lane; q < m; q += 32) {
-        const int e = ent_e[q];
-        const int32_t cnt = myh[e];
-        if (cnt == 0) continue;
-        int32_t st = base[e];
-        for (int w = 0; w < warp; ++w) st += hw[w * E + e];
-        if (ent_hi[q] <= st || ent_lo[q] >= st + cnt) continue;
-        myt[e] = (ent_lo[q] <= st && ent_hi[q] >= st + cnt) ? E + ent_s[q] : -1;   // at most one full cover
-    }
-    __syncwarp();
+    // ---- this chunk's table row (built by the prep kernel) and its boundary count
+    const int32_t* trow = a.tabg + id * (int64_t)E;
+    for (int e = tid; e < E; e += kThreads) tab[e] = trow[e];
+    __syncthreads();
+    const int32_t* lut = tab;
 
-    // ---- (warp, expert) pairs that straddle a quota boundary: exact ordinals from ballots
-    for (int eb0 = 0; eb0 < E; eb0 += 32) {
-        const int ecand = eb0 + lane;
-        unsigned todo = __ballot_sync(0xffffffffu, ecand < E && myt[ecand] == -1);
-        while (todo) {
-            const int eb = eb0 + __ffs(todo) - 1;
-            todo &= todo - 1;
-            int32_t running = base[eb];
-            for (int w = 0; w < warp; ++w) running += hw[w * E + eb];
-            const int32_t mine = myh[eb];
-            int q0 = m, q1 = m;                  // entries of eb whose interval can touch [running, running+mine)
-            for (int q = 0; q < m; ++q)
-                if (ent_e[q] == eb && ent_hi[q] > running) { q0 = q; break; }
-            for (int q = q0; q < m; ++q)
-                if (ent_e[q] == eb && ent_lo[q] >= running + mine) { q1 = q; break; }
-            const unsigned lt = (1u << lane) - 1u;
+    if (nb > 0) {
+        // ---- rare path: rebuild this rank's quota intervals, refine the boundary experts per warp
+        const int m = build_entries(a.X + lr * S, a.slot_expert + (int64_t)l * S, S, E, ent_s, ent_e, ent_lo, ent_hi, s_wcnt);
+        for (int q = tid; q < m; q += kThreads) ent_hi[q] += ent_lo[q];
+        const int32_t* ccseg = a.cc + lr * a.nc * (int64_t)E;
+        if (tid == 0) s_nb = 0;
+        __syncthreads();
+        for (int e = tid; e < E; e += kThreads)
+            if (tab[e] == -1) {
+                int32_t b = 0;
+                for (int cp = 0; cp < c; ++cp) b += ccseg[(int64_t)cp * E + e];
+                const int bi = atomicAdd(&s_nb, 1);
+                blist[bi] = e;
+                base[bi] = b;
+                tab[e] = e;                              // refined per warp below
+            }
+        __syncthreads();
+        // per-warp counts of the boundary experts, from the registers
+        for (int bi = 0; bi < nb; ++bi) {
+            const int eb = blist[bi];
+            int cnt = 0;
+#pragma unroll
+            for (int it = 0; it < kIters; ++it)
+                cnt += (x[it].x == eb) + (x[it].y == eb) + (x[it].z == eb) + (x[it].w == eb);
+            for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+            if (lane == 0) cntw[bi * kWarps + warp] = cnt;
+        }
+        int32_t* myt = wtab + warp * E;
+        for (int e = lane; e < E; e += 32) myt[e] = tab[e];
+        __syncthreads();
+        const unsigned lt = (1u << lane) - 1u;
+        for (int bi = 0; bi < nb; ++bi) {
+            const int eb = blist[bi];
+            const int32_t mine = cntw[bi * kWarps + warp];
+            int32_t running = base[bi];
+            for (int w = 0; w < warp; ++w) running += cntw[bi * kWarps + w];
+            // this warp's ordinals of eb are [running, running + mine): inside one interval, outside all, or straddling
+            int32_t target = eb;
+            bool straddle = false;
+            int q0 = m, q1 = m;
+            for (int q = 0; q < m; ++q) {
+                if (ent_e[q] != eb || mine == 0) continue;
+                if (ent_hi[q] <= running || ent_lo[q] >= running + mine) continue;
+                if (ent_lo[q] <= running && ent_hi[q] >= running + mine) target = E + ent_s[q];
+                else { straddle = true; if (q0 == m) q0 = q; q1 = q + 1; }
+            }
+            if (!straddle) {
+                if (lane == 0) myt[eb] = target;
+                continue;
+            }
 #pragma unroll
             for (int it = 0; it < kIters; ++it) {
                 int32_t* xv = reinterpret_cast<int32_t*>(&x[it]);
@@ -191,54 +259,67 @@ assign_kernel(AssignArgs a)
                 running += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
             }
             // what is still eb in the registers stays eb; moved entries are now >= E and pass through
-            if (lane == 0) myt[eb] = eb;
         }
         __syncwarp();
+        lut = myt;
     }
 
     // ---- one table lookup per entry (values >= E or < 0 pass through unchanged), then store
+    if (full) {
 #pragma unroll
-    for (int it = 0; it < kIters; ++it) {
-        int32_t* xv = reinterpret_cast<int32_t*>(&x[it]);
+        for (int it = 0; it < kIters; ++it) {
+            int32_t* xv = reinterpret_cast<int32_t*>(&x[it]);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int32_t e = xv[j];
-            if ((uint32_t)e < (uint32_t)E) xv[j] = myt[e];
+            for (int j = 0; j < 4; ++j) {
+                const int32_t e = xv[j];
+                if ((uint32_t)e < (uint32_t)E) xv[j] = lut[e];
+            }
+            st_stream(reinterpret_cast<int4*>(dst + wbase_elem + it * 128), x[it]);
         }
-        const int32_t pos = wbase_elem + it * 128;
-        if (VEC && pos + 3 < len) st_stream(reinterpret_cast<int4*>(dst + pos), x[it]);
-        else {
+    } else {
+#pragma unroll
+        for (int it = 0; it < kIters; ++it) {
+            int32_t* xv = reinterpret_cast<int32_t*>(&x[it]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int32_t e = xv[j];
+                if ((uint32_t)e < (uint32_t)E) xv[j] = lut[e];
+            }
+            const int32_t pos = wbase_elem + it * 128;
             if (pos < len) dst[pos] = x[it].x;
             if (pos + 1 < len) dst[pos + 1] = x[it].y;
             if (pos + 2 < len) dst[pos + 2] = x[it].z;
             if (pos + 3 < len) dst[pos + 3] = x[it].w;
         }
     }
-    if (bad && tid == 0) atomicOr(a.info + l, TAOT_INFO_BAD_INDEX);
 }
 
 }  // namespace
 
-int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_cc,
-                       const int32_t* d_slot_expert, const int32_t* d_X, int32_t* d_new_idx,
+int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_cc, int32_t* d_tabg,
+                       int32_t* d_nbg, const int32_t* d_slot_expert, const int32_t* d_X, int32_t* d_new_idx,
                        int32_t* d_info, cudaStream_t st)
 {
     const taot_params& p = h->p;
     AssignArgs a;
-    a.topk = d_topk; a.cc = d_cc; a.slot_expert = d_slot_expert; a.X = d_X; a.out = d_new_idx; a.info = d_info;
+    a.topk = d_topk; a.cc = d_cc; a.tabg = d_tabg; a.nbg = d_nbg;
+    a.slot_expert = d_slot_expert; a.X = d_X; a.out = d_new_idx; a.info = d_info;
     a.layer_elems = p.T * p.k; a.seg = h->seg; a.nc = h->nc; a.R = p.R; a.E = p.E; a.K = p.K;
     a.vec_ok = ((reinterpret_cast<uintptr_t>(d_topk) & 15) == 0) &&
                ((reinterpret_cast<uintptr_t>(d_new_idx) & 15) == 0) && (h->seg % 4 == 0);
     const int S = p.R * p.K;
-    const size_t smem = sizeof(int32_t) * ((size_t)p.E * (2 * kWarps + 1) + 4 * (size_t)S);
-    const int64_t blocks = (int64_t)p.L * p.R * h->nc;
+    const size_t smem_prep = sizeof(int32_t) * (2 * (size_t)p.E + 4 * (size_t)S);
+    assign_prep_kernel<<<(unsigned)((int64_t)p.L * p.R), kThreads, smem_prep, st>>>(a);
+    TAOT_CUDA_OK(cudaGetLastError());
+    const size_t smem = sizeof(int32_t) * ((size_t)p.E * (3 + 2 * kWarps) + 4 * (size_t)S);
+    const unsigned blocks = (unsigned)((int64_t)p.L * p.R * h->nc);
     if (a.vec_ok) {
         TAOT_CUDA_OK(cudaFuncSetAttribute(assign_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        assign_kernel<true><<<(unsigned)blocks, kThreads, smem, st>>>(a);
+        assign_kernel<true><<<blocks, kThreads, smem, st>>>(a);
     } else {
         TAOT_CUDA_OK(cudaFuncSetAttribute(assign_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        assign_kernel<false><<<(unsigned)blocks, kThreads, smem, st>>>(a);
+        assign_kernel<false><<<blocks, kThreads, smem, st>>>(a);
     }
     TAOT_CUDA_OK(cudaGetLastError());
-    return 1;
+    return 2;
 }

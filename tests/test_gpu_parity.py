@@ -115,7 +115,7 @@ def test_plan_is_deterministic(case):
     torch.cuda.synchronize()
     for key, val in again.items():
         assert (cpu(val) == out[key]).all(), key
-    assert pl.last_launch_count() == 5
+    assert pl.last_launch_count() == 6
 
 
 def test_plan_host_round_trip(case):
