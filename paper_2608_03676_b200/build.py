@@ -14,7 +14,7 @@ OBJ = os.path.join(PKG, "csrc", "build")
 SOURCES = ["api.cu", "histogram.cu", "sinkhorn.cu", "match.cu", "assign.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v",
-              "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+              "-I", os.path.join(ROOT, "include"), "-I", CSRC] + os.environ.get("TAOT_EXTRA_NVCC_FLAGS", "").split()
 
 
 def _nvcc() -> str:

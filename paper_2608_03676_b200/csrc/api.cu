@@ -59,6 +59,7 @@ void layout(taot_handle_t h)
     h->off_s = take(sizeof(float) * LR);
     h->off_d = take(sizeof(float) * LR);
     h->off_nrem = take(sizeof(int32_t) * (size_t)p.L * dmax * p.R);
+    h->off_t12 = take(sizeof(float) * (size_t)p.L * p.E * 2 * p.R);
     h->ws_bytes = off;
 
     const size_t S = (size_t)p.R * p.K;
@@ -153,6 +154,35 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
                 B[(size_t)i * R + j] = b;
             }
     }
+    // distinct values of the auction bonus (B off the diagonal, 1 on it) and, per host and value,
+    // the set of source ranks that have it
+    std::vector<float> tierval;
+    std::vector<uint32_t> tiermask;
+    {
+        std::vector<float> vals;
+        for (int i = 0; i < R && (int)vals.size() <= TAOT_MAX_TIERS; ++i)
+            for (int j = 0; j < R && (int)vals.size() <= TAOT_MAX_TIERS; ++j) {
+                const float b3 = (i == j) ? 1.0f : B[(size_t)i * R + j];
+                bool seen = false;
+                for (float v : vals) seen |= (v == b3);
+                if (!seen) vals.push_back(b3);
+            }
+        if ((int)vals.size() <= TAOT_MAX_TIERS) {
+            for (size_t x = 0; x < vals.size(); ++x)
+                for (size_t y = x + 1; y < vals.size(); ++y)
+                    if (vals[y] > vals[x]) std::swap(vals[x], vals[y]);
+            tierval = vals;
+            const int W = (R + 31) / 32, Tn = (int)vals.size();
+            tiermask.assign((size_t)R * Tn * W, 0u);
+            for (int host = 0; host < R; ++host)
+                for (int r = 0; r < R; ++r) {
+                    const float b3 = (r == host) ? 1.0f : B[(size_t)r * R + host];
+                    for (int t = 0; t < Tn; ++t)
+                        if (vals[t] == b3) tiermask[((size_t)host * Tn + t) * W + (r >> 5)] |= 1u << (r & 31);
+                }
+        }
+    }
+    h->ntiers = (int32_t)tierval.size();
     // first Sinkhorn row update with v = 1 on every rank: log-sum-exp of -C_ij/eps over all j
     std::vector<double> lse0(R);
     for (int i = 0; i < R; ++i) {
@@ -180,6 +210,8 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
     if (rc == TAOT_OK) rc = upload(&h->d_rowlse0, lse0.data(), (size_t)R);
     if (rc == TAOT_OK) rc = upload(&h->d_rank_off, off.data(), (size_t)R + 1);
     if (rc == TAOT_OK) rc = upload(&h->d_rank_list, list.data(), (size_t)E);
+    if (rc == TAOT_OK && h->ntiers > 0) rc = upload(&h->d_tierval, tierval.data(), tierval.size());
+    if (rc == TAOT_OK && h->ntiers > 0) rc = upload(&h->d_tiermask, tiermask.data(), tiermask.size());
     for (int i = 0; i < 6 && rc == TAOT_OK; ++i)
         if (cudaEventCreate(&h->ev[i]) != cudaSuccess) rc = TAOT_ERR_CUDA;
     if (rc == TAOT_OK && cudaDeviceSynchronize() != cudaSuccess) rc = TAOT_ERR_CUDA;
@@ -196,7 +228,7 @@ int taot_destroy(taot_handle_t h)
     if (!h) return TAOT_OK;
     cudaDeviceSynchronize();
     cudaFree(h->d_e2r); cudaFree(h->d_C); cudaFree(h->d_B); cudaFree(h->d_rowlse0);
-    cudaFree(h->d_rank_off); cudaFree(h->d_rank_list);
+    cudaFree(h->d_rank_off); cudaFree(h->d_rank_list); cudaFree(h->d_tierval); cudaFree(h->d_tiermask);
     for (int i = 0; i < 6; ++i)
         if (h->ev[i]) cudaEventDestroy(h->ev[i]);
     delete h;
@@ -287,7 +319,7 @@ int taot_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load
     if (reinterpret_cast<uintptr_t>(ws) & 255) return TAOT_ERR_ALIGN;
     int a = taot_launch_match(h, d_n, d_expert_load, d_rank_load, d_plan, d_slot_expert, d_slot_tokens, d_X,
                               d_rounds, d_info, reinterpret_cast<int32_t*>(at(ws, h->off_nrem)),
-                              static_cast<cudaStream_t>(stream));
+                              reinterpret_cast<float*>(at(ws, h->off_t12)), static_cast<cudaStream_t>(stream));
     if (a < 0) return a;
     h->last_launches = a;
     return TAOT_OK;
@@ -347,7 +379,8 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, voi
     total += a;
     TAOT_MARK(3);
     if ((a = taot_launch_match(h, o->n, o->expert_load, o->rank_load, o->plan, o->slot_expert, o->slot_tokens,
-                               o->X, o->rounds, o->info, reinterpret_cast<int32_t*>(at(ws, h->off_nrem)), st)) < 0)
+                               o->X, o->rounds, o->info, reinterpret_cast<int32_t*>(at(ws, h->off_nrem)),
+                               reinterpret_cast<float*>(at(ws, h->off_t12)), st)) < 0)
         return a;
     total += a;
     TAOT_MARK(4);

@@ -1,12 +1,25 @@
 // Phase 2 (Appendix A.3, Algorithm 2: column-priority iterative matching) and Phase 3
-// (Appendix A.4, Algorithm 3: Lagrangian auction), one CTA per layer, all state in shared memory.
+// (Appendix A.4, Algorithm 3: Lagrangian auction), one CTA per layer, all round state in shared
+// memory.
 //
 // Both phases are chains of short dependent rounds; a round is "every rank (slot) takes an
 // argmax, conflicts are arbitrated by a second argmax, winners are applied".  The argmaxes are
 // taken over packed 64-bit keys (score bits high, inverted index low) so that a single integer
 // max gives "highest score, lowest index on ties", independent of thread order.  Scores are fp32
-// with one rounding per operation (__fmul_rn / __fadd_rn / __fdiv_rn: no FMA contraction), which
-// keeps every integer decision reproducible bit for bit on a CPU.
+// with one rounding per operation (__fmul_rn / __fadd_rn / __fsub_rn / __fdiv_rn: no FMA
+// contraction), which keeps every integer decision reproducible bit for bit on a CPU.
+//
+// Phase 2: the two score terms that do not change between rounds (alpha*B and 0.1*alpha*T_norm)
+// are computed once per layer for the experts that spill; a round is then one thread per rank
+// scanning those experts with coalesced reads.
+//
+// Phase 3: the bonus matrix of a real topology has a handful of distinct values (tiers).  Within
+// a tier a slot's score  B3 - step*wins[r]  depends on r only through wins[r], so the best source
+// rank of a tier is "lowest wins, then lowest index" among the ranks that still hold tokens.  Ranks
+// are kept as bit sets (per tier and host, per win count, per expert availability), and a bid is a
+// few word-wide ANDs instead of a scan over all R ranks; the exact fp32 score is still what is
+// compared, including win counts whose scores round to the same float.  A bonus matrix with more
+// than kMaxTiers distinct values (or a negative price step) takes the dense scan instead.
 #include "taot_internal.cuh"
 
 namespace {
@@ -22,13 +35,16 @@ struct MatchArgs {
     const float* B;              // [R,R]
     const int32_t* rank_off;     // [R+1]
     const int32_t* rank_list;    // [E]
+    const uint32_t* tiermask;    // [R hosts][ntiers][W] bit r: B3[r][host] == tierval[t]
+    const float* tierval;        // [ntiers] descending
     int32_t* slot_expert;        // [L,R,K]
     int32_t* slot_tokens;        // [L,R,K]
     int32_t* X;                  // [L,R,S]
     int32_t* rounds;             // [L,2] or null
     int32_t* info;               // [L]
     int32_t* nrem_g;             // [L, dmax, R] global fallback for the remaining counts
-    int32_t R, E, K, dmax;
+    float* t12;                  // [L, E, 2, R] scratch: alpha*B and beta*T_norm rows of the spilling experts
+    int32_t R, E, K, dmax, ntiers, W;
     float eps0, price_step;
     int32_t auction_max_rounds;
     int32_t nrem_in_smem;
@@ -49,10 +65,28 @@ __device__ __forceinline__ u64 warp_max_u64(u64 k)
     return k;
 }
 
-__global__ void match_kernel(MatchArgs a)
+constexpr int kMaxW = 8;          // words of a rank bit set: R <= 256
+
+// Arbitration "best bidder per target" for one warp's worth of bids.  Many bidders often pick the
+// same target (all slots of a tier chase the cheapest rank), so the lanes that bid for the same
+// target first agree on their best key with warp-wide reductions and only one of them touches the
+// shared-memory arbiter.  key = (score bits << 32) | inverted bidder index; valid bids have key != 0.
+__device__ __forceinline__ void arbitrate(u64* arb, int target, u64 key)
+{
+    const unsigned active = __ballot_sync(0xffffffffu, key != 0);
+    if (key == 0) return;
+    const unsigned group = __match_any_sync(active, target);
+    const uint32_t hi = (uint32_t)(key >> 32), lo = (uint32_t)key;
+    const uint32_t hi_max = __reduce_max_sync(group, hi);
+    const uint32_t lo_max = __reduce_max_sync(group, hi == hi_max ? lo : 0u);
+    if ((__ffs(group) - 1) == (int)(threadIdx.x & 31)) atomicMax(arb + target, ((u64)hi_max << 32) | (u64)lo_max);
+}
+
+__global__ void __launch_bounds__(256)
+match_kernel(MatchArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    const int R = a.R, E = a.E, K = a.K, S = R * K;
+    const int R = a.R, E = a.E, K = a.K, S = R * K, W = a.W;
     const int NT = blockDim.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, NW = NT >> 5;
     const int64_t l = blockIdx.x;
 
@@ -60,8 +94,9 @@ __global__ void match_kernel(MatchArgs a)
     u64* arb_e = reinterpret_cast<u64*>(smem_raw);            // [E]  Phase 2 arbitration per expert
     u64* arb_r = arb_e + E;                                    // [R]  Phase 3 arbitration per rank
     int32_t* spill = reinterpret_cast<int32_t*>(arb_r + R);    // [E]
-    int32_t* hotlist = spill + E;                              // [E]
-    int32_t* dcol = hotlist + E;                               // [E]  expert -> column of nrem, or -1
+    int32_t* hot0 = spill + E;                                 // [E]  experts that spill at the start of Phase 2
+    int32_t* hot_home = hot0 + E;                              // [E]  their home ranks
+    int32_t* dcol = hot_home + E;                              // [E]  expert -> column of nrem, or -1
     int32_t* spare = dcol + E;                                 // [R]
     int32_t* excess = spare + R;                               // [R]
     int32_t* matched = excess + R;                             // [R]
@@ -70,7 +105,10 @@ __global__ void match_kernel(MatchArgs a)
     int32_t* slot_e = wins + R;                                // [S]
     int32_t* slot_a0 = slot_e + S;                             // [S]  planned tokens (Phase 2 result)
     int32_t* slot_a = slot_a0 + S;                             // [S]  still to collect (Phase 3)
-    int32_t* nrem_s = slot_a + S;                              // [dmax*R] if it fits
+    uint32_t* avail = reinterpret_cast<uint32_t*>(slot_a + S); // [dmax][W]  ranks still holding tokens of the expert
+    uint32_t* lvl = avail + a.dmax * W;                        // [S+1][W]   ranks by win count
+    int32_t* wstart = reinterpret_cast<int32_t*>(lvl + (S + 1) * W);   // [S][ntiers] resume level of each slot and tier
+    int32_t* nrem_s = wstart + S * (a.ntiers > 0 ? a.ntiers : 1);      // [dmax*R] if it fits
     __shared__ long long s_tot;
     __shared__ int s_cnt, s_any;
 
@@ -79,9 +117,10 @@ __global__ void match_kernel(MatchArgs a)
     const int32_t* rl = a.rank_load + l * R;
     const float* plan = a.plan + l * (int64_t)R * R;
     int32_t* nrem = a.nrem_in_smem ? nrem_s : a.nrem_g + l * (int64_t)a.dmax * R;
+    float* t12 = a.t12 + l * (int64_t)E * 2 * R;
 
     // ---- integer mean, excess, spare (Appendix A.1)
-    if (tid == 0) s_tot = 0;
+    if (tid == 0) { s_tot = 0; s_cnt = 0; }
     __syncthreads();
     {
         long long part = 0;
@@ -108,59 +147,72 @@ __global__ void match_kernel(MatchArgs a)
             if (v < mine || (v == mine && e2 <= e)) cum += v;
         }
         const long long hi = cum - mean, lo = cum - mine - mean;
-        spill[e] = (int32_t)((hi > 0 ? hi : 0) - (lo > 0 ? lo : 0));
+        const int32_t sp = (int32_t)((hi > 0 ? hi : 0) - (lo > 0 ? lo : 0));
+        spill[e] = sp;
         arb_e[e] = 0;
+        if (sp > 0) {
+            const int q = atomicAdd(&s_cnt, 1);
+            hot0[q] = e;
+            hot_home[q] = r;
+        }
     }
     for (int s = tid; s < S; s += NT) { slot_e[s] = -1; slot_a0[s] = 0; }
     __syncthreads();
+    const int nhot0 = s_cnt;
 
     const float alpha = __fdiv_rn((float)(mean * (long long)R), (float)E);
     const float beta = __fmul_rn(0.1f, alpha);
 
+    // ---- round-invariant score terms of the spilling experts: t1 = alpha*B, t2 = beta*T/max(excess, eps0)
+    for (int64_t idx = tid; idx < (int64_t)nhot0 * R; idx += NT) {
+        const int q = (int)(idx / R), r = (int)(idx - (int64_t)q * R);
+        const int hr = hot_home[q];
+        const float ex = fmaxf((float)excess[hr], a.eps0);
+        const float tn = __fdiv_rn(plan[(int64_t)hr * R + r], ex);
+        t12[((int64_t)q * 2) * R + r] = __fmul_rn(alpha, a.B[(int64_t)hr * R + r]);
+        t12[((int64_t)q * 2 + 1) * R + r] = __fmul_rn(beta, tn);
+    }
+    __syncthreads();
+
     // =========================================================== Phase 2
+#ifdef TAOT_DEBUG_CLOCKS
+    const long long clk0 = clock64();
+#endif
     int rounds2 = 0;
     for (int kappa = 0; kappa < K; ++kappa) {
         for (int r = tid; r < R; r += NT) matched[r] = 0;
         for (;;) {
-            if (tid == 0) { s_cnt = 0; s_any = 0; }
+            if (tid == 0) s_any = 0;
             __syncthreads();
-            for (int e = tid; e < E; e += NT)
-                if (spill[e] > 0) hotlist[atomicAdd(&s_cnt, 1)] = e;
-            __syncthreads();
-            const int nhot = s_cnt;
-            if (nhot == 0) break;
             // Steps 1-2: every unmatched cold rank takes its best candidate expert
-            for (int r = warp; r < R; r += NW) {
-                if (matched[r] || spare[r] <= 0) { if (lane == 0) estar[r] = -1; continue; }
-                const int32_t sp = spare[r];
+            for (int rb = 0; rb < R; rb += NT) {
+                const int r = rb + tid;                       // whole warps stay in the loop for the warp-wide arbitration
+                int best_e = -1;
                 u64 key = 0;
-                for (int q = lane; q < nhot; q += 32) {
-                    const int e = hotlist[q];
-                    const int hr = a.e2r[e];
-                    if (hr == r) continue;
-                    bool placed = false;
-                    for (int kk = 0; kk < kappa; ++kk) placed |= (slot_e[r * K + kk] == e);
-                    if (placed) continue;
-                    const int32_t gain = spill[e] < sp ? spill[e] : sp;
-                    const float ex = fmaxf((float)excess[hr], a.eps0);
-                    const float tn = __fdiv_rn(plan[(int64_t)hr * R + r], ex);
-                    const float t1 = __fmul_rn(alpha, a.B[(int64_t)hr * R + r]);
-                    const float t2 = __fmul_rn(beta, tn);
-                    const float sc = __fadd_rn(__fadd_rn((float)gain, t1), t2);
-                    const u64 k64 = ((u64)__float_as_uint(sc) << 32) | (u64)(0xFFFFFFFFu - (uint32_t)e);
-                    key = k64 > key ? k64 : key;
-                }
-                key = warp_max_u64(key);
-                if (lane == 0) {
-                    if (key == 0) estar[r] = -1;
-                    else {
-                        const int e = (int)(0xFFFFFFFFu - (uint32_t)key);
-                        estar[r] = e;
-                        // Step 3: arbitration, best rank per expert (ties: lowest rank)
-                        atomicMax(arb_e + e, (key & 0xFFFFFFFF00000000ull) | (u64)(0xFFFFFFFFu - (uint32_t)r));
-                        s_any = 1;
+                const int32_t sp = r < R ? spare[r] : 0;
+                if (r < R && !matched[r] && sp > 0) {
+                    for (int q = 0; q < nhot0; ++q) {
+                        const int e = hot0[q];
+                        const int32_t se = spill[e];
+                        if (se <= 0 || hot_home[q] == r) continue;
+                        bool placed = false;
+                        for (int kk = 0; kk < kappa; ++kk) placed |= (slot_e[r * K + kk] == e);
+                        if (placed) continue;
+                        const int32_t gain = se < sp ? se : sp;
+                        const float t1 = t12[((int64_t)q * 2) * R + r];
+                        const float t2 = t12[((int64_t)q * 2 + 1) * R + r];
+                        const float sc = __fadd_rn(__fadd_rn((float)gain, t1), t2);
+                        const u64 k64 = ((u64)__float_as_uint(sc) << 32) | (u64)(0xFFFFFFFFu - (uint32_t)e);
+                        key = k64 > key ? k64 : key;
                     }
                 }
+                if (key != 0) {
+                    best_e = (int)(0xFFFFFFFFu - (uint32_t)key);
+                    s_any = 1;
+                }
+                if (r < R) estar[r] = best_e;
+                // Step 3: arbitration, best rank per expert (ties: lowest rank)
+                arbitrate(arb_e, best_e, key == 0 ? 0ull : ((key & 0xFFFFFFFF00000000ull) | (u64)(0xFFFFFFFFu - (uint32_t)r)));
             }
             __syncthreads();
             if (!s_any) break;
@@ -177,13 +229,15 @@ __global__ void match_kernel(MatchArgs a)
                 }
             }
             __syncthreads();
-            for (int q = tid; q < nhot; q += NT) arb_e[hotlist[q]] = 0;
+            for (int q = tid; q < nhot0; q += NT) arb_e[hot0[q]] = 0;
             ++rounds2;
-            __syncthreads();
         }
         __syncthreads();
     }
 
+#ifdef TAOT_DEBUG_CLOCKS
+    const long long clk1 = clock64();
+#endif
     // =========================================================== Phase 3
     // compact the experts that sit in some slot; keep their per-rank remaining counts transposed [col][r]
     for (int e = tid; e < E; e += NT) dcol[e] = -1;
@@ -196,48 +250,151 @@ __global__ void match_kernel(MatchArgs a)
     __syncthreads();
     for (int e = tid; e < E; e += NT)
         if (dcol[e] == -2) dcol[e] = atomicAdd(&s_cnt, 1);
+    for (int i = tid; i < a.dmax * W; i += NT) avail[i] = 0u;
+    for (int i = tid; i < (S + 1) * W; i += NT) lvl[i] = 0u;
+    for (int i = tid; i < S * a.ntiers; i += NT) wstart[i] = 0;
     __syncthreads();
     const int D = s_cnt;
     for (int e = 0; e < E; ++e) {
         const int col = dcol[e];
         if (col < 0) continue;
-        for (int r = tid; r < R; r += NT) nrem[col * R + r] = n[(int64_t)r * E + e];
+        for (int r = tid; r < R; r += NT) {
+            const int32_t v = n[(int64_t)r * E + e];
+            nrem[col * R + r] = v;
+            if (v > 0) atomicOr(avail + col * W + (r >> 5), 1u << (r & 31));
+        }
     }
+    for (int r = tid; r < R; r += NT) atomicOr(lvl + (r >> 5), 1u << (r & 31));      // every rank starts with 0 wins
     int32_t* Xl = a.X + l * (int64_t)R * S;
     for (int64_t q = tid; q < (int64_t)R * S; q += NT) Xl[q] = 0;
     __syncthreads();
 
     int rounds3 = 0;
+#ifdef TAOT_DEBUG_CLOCKS
+    long long dbg_bid = 0, dbg_wait = 0, dbg_serve = 0;
+#endif
     const long long cap = (long long)R * S + S;
+    const bool tiered = a.ntiers > 0;
     for (;;) {
         if (a.auction_max_rounds > 0 && rounds3 >= a.auction_max_rounds) break;
         if (rounds3 >= cap || D == 0) break;
         if (tid == 0) s_any = 0;
         __syncthreads();
+#ifdef TAOT_DEBUG_CLOCKS
+        const long long ca = clock64();
+#endif
         // Step 1: every unfinished slot bids for the source rank with the best bonus minus price
-        for (int s = warp; s < S; s += NW) {
-            const int e = slot_e[s];
-            if (e < 0 || slot_a[s] <= 0) continue;
-            const int host = s / K;
-            const int32_t* col = nrem + dcol[e] * R;
-            u64 key = 0;
-            for (int r = lane; r < R; r += 32) {
-                if (col[r] <= 0) continue;
-                const float b3 = (r == host) ? 1.0f : a.B[(int64_t)r * R + host];
-                const float price = __fmul_rn(a.price_step, (float)wins[r]);
-                const float sc = __fsub_rn(b3, price);
-                const u64 k64 = ((u64)ordered_bits(sc) << 32) | (u64)(0xFFFFFFFFu - (uint32_t)r);
-                key = k64 > key ? k64 : key;
-            }
-            key = warp_max_u64(key);
-            if (lane == 0 && key != 0) {
-                const int r = (int)(0xFFFFFFFFu - (uint32_t)key);
+        if (tiered) {
+            for (int sb = 0; sb < S; sb += NT) {
+                const int s = sb + tid;
+                const int e = s < S ? slot_e[s] : -1;
+                const bool live = e >= 0 && slot_a[s] > 0;
+                const int host = s / K;
+                const uint32_t* av = avail + (live ? dcol[e] : 0) * W;
+                const uint32_t* tm = a.tiermask + (int64_t)(live ? host : 0) * a.ntiers * W;
+                u64 key = 0;
+                for (int t = 0; live && t < a.ntiers; ++t) {
+                    uint32_t cand[kMaxW];
+                    uint32_t any = 0;
+                    int pc = 0;
+#pragma unroll
+                    for (int w = 0; w < kMaxW; ++w) {
+                        cand[w] = (w < W) ? (tm[t * W + w] & av[w]) : 0u;
+                        any |= cand[w];
+                        pc += __popc(cand[w]);
+                    }
+                    if (!any) continue;
+                    const float vt = a.tierval[t];
+                    // the lowest win count among this tier's candidates never decreases: resume from the last one
+                    int wl = wstart[s * a.ntiers + t];
+                    const float ub = __fsub_rn(vt, __fmul_rn(a.price_step, (float)wl));
+                    if (key != 0 && (u64)ordered_bits(ub) < (key >> 32)) continue;      // cannot beat a better tier
+                    if (pc <= 8) {
+                        // few candidates: score each one
+                        int wmin = S + 1;
+#pragma unroll
+                        for (int w = 0; w < kMaxW; ++w) {
+                            uint32_t bits = cand[w];
+                            while (bits) {
+                                const int r = (w << 5) + __ffs(bits) - 1;
+                                bits &= bits - 1;
+                                const int wr = wins[r];
+                                wmin = wr < wmin ? wr : wmin;
+                                const float sc = __fsub_rn(vt, __fmul_rn(a.price_step, (float)wr));
+                                const u64 k64 = ((u64)ordered_bits(sc) << 32) | (u64)(0xFFFFFFFFu - (uint32_t)r);
+                                key = k64 > key ? k64 : key;
+                            }
+                        }
+                        wstart[s * a.ntiers + t] = wmin;
+                        continue;
+                    }
+                    int r_best = -1;
+                    for (; wl <= S; ++wl) {
+                        const uint32_t* lv = lvl + wl * W;
+#pragma unroll
+                        for (int w = 0; w < kMaxW; ++w) {
+                            if (w < W && r_best < 0) {
+                                const uint32_t hit = cand[w] & lv[w];
+                                if (hit) r_best = (w << 5) + __ffs(hit) - 1;
+                            }
+                        }
+                        if (r_best >= 0) break;
+                    }
+                    if (r_best < 0) continue;
+                    wstart[s * a.ntiers + t] = wl;
+                    const float sc = __fsub_rn(vt, __fmul_rn(a.price_step, (float)wl));
+                    // higher win counts whose score rounds to the same float compete on rank index alone
+                    for (int w2 = wl + 1; w2 <= S; ++w2) {
+                        if (__fsub_rn(vt, __fmul_rn(a.price_step, (float)w2)) != sc) break;
+                        const uint32_t* lv = lvl + w2 * W;
+                        int r2 = -1;
+#pragma unroll
+                        for (int w = 0; w < kMaxW; ++w) {
+                            if (w < W && r2 < 0) {
+                                const uint32_t hit = cand[w] & lv[w];
+                                if (hit) r2 = (w << 5) + __ffs(hit) - 1;
+                            }
+                        }
+                        if (r2 >= 0 && r2 < r_best) r_best = r2;
+                    }
+                    const u64 k64 = ((u64)ordered_bits(sc) << 32) | (u64)(0xFFFFFFFFu - (uint32_t)r_best);
+                    key = k64 > key ? k64 : key;
+                }
                 // Step 2: the rank keeps its best bidder (ties: lowest slot)
-                atomicMax(arb_r + r, (key & 0xFFFFFFFF00000000ull) | (u64)(0xFFFFFFFFu - (uint32_t)s));
-                s_any = 1;
+                const int rsel = (int)(0xFFFFFFFFu - (uint32_t)key);
+                if (key != 0) s_any = 1;
+                arbitrate(arb_r, rsel, key == 0 ? 0ull : ((key & 0xFFFFFFFF00000000ull) | (u64)(0xFFFFFFFFu - (uint32_t)s)));
+            }
+        } else {
+            for (int s = warp; s < S; s += NW) {
+                const int e = slot_e[s];
+                if (e < 0 || slot_a[s] <= 0) continue;
+                const int host = s / K;
+                const int32_t* col = nrem + dcol[e] * R;
+                u64 key = 0;
+                for (int r = lane; r < R; r += 32) {
+                    if (col[r] <= 0) continue;
+                    const float b3 = (r == host) ? 1.0f : a.B[(int64_t)r * R + host];
+                    const float price = __fmul_rn(a.price_step, (float)wins[r]);
+                    const float sc = __fsub_rn(b3, price);
+                    const u64 k64 = ((u64)ordered_bits(sc) << 32) | (u64)(0xFFFFFFFFu - (uint32_t)r);
+                    key = k64 > key ? k64 : key;
+                }
+                key = warp_max_u64(key);
+                if (lane == 0 && key != 0) {
+                    const int r = (int)(0xFFFFFFFFu - (uint32_t)key);
+                    atomicMax(arb_r + r, (key & 0xFFFFFFFF00000000ull) | (u64)(0xFFFFFFFFu - (uint32_t)s));
+                    s_any = 1;
+                }
             }
         }
+#ifdef TAOT_DEBUG_CLOCKS
+        const long long cb = clock64();
+#endif
         __syncthreads();
+#ifdef TAOT_DEBUG_CLOCKS
+        const long long cc_ = clock64();
+#endif
         if (!s_any) break;
         // Steps 3-4: allocate, update holdings, plan and price
         for (int r = tid; r < R; r += NT) {
@@ -245,15 +402,27 @@ __global__ void match_kernel(MatchArgs a)
             if (k64 == 0) continue;
             arb_r[r] = 0;
             const int s = (int)(0xFFFFFFFFu - (uint32_t)k64);
-            const int e = slot_e[s];
-            int32_t* cell = nrem + dcol[e] * R + r;
-            const int32_t x = *cell < slot_a[s] ? *cell : slot_a[s];
-            Xl[(int64_t)r * S + s] += x;
-            *cell -= x;
+            const int col = dcol[slot_e[s]];
+            int32_t* cell = nrem + col * R + r;
+            const int32_t have = *cell;
+            const int32_t x = have < slot_a[s] ? have : slot_a[s];
+            Xl[(int64_t)r * S + s] = x;          // a (rank, slot) pair is served at most once
+            *cell = have - x;
             slot_a[s] -= x;
-            if (x > 0) wins[r]++;
+            const uint32_t bit = 1u << (r & 31);
+            if (have - x == 0) atomicAnd(avail + col * W + (r >> 5), ~bit);
+            if (x > 0) {
+                const int w0 = wins[r];
+                wins[r] = w0 + 1;
+                atomicAnd(lvl + w0 * W + (r >> 5), ~bit);
+                atomicOr(lvl + (w0 + 1) * W + (r >> 5), bit);
+            }
         }
         ++rounds3;
+#ifdef TAOT_DEBUG_CLOCKS
+        const long long cd = clock64();
+        dbg_bid += cb - ca; dbg_wait += cc_ - cb; dbg_serve += cd - cc_;
+#endif
         __syncthreads();
     }
 
@@ -267,14 +436,18 @@ __global__ void match_kernel(MatchArgs a)
     residual = __syncthreads_or(residual);
     if (tid == 0) {
         if (a.rounds) { a.rounds[l * 2] = rounds2; a.rounds[l * 2 + 1] = rounds3; }
+#ifdef TAOT_DEBUG_CLOCKS
+        if (a.rounds) { a.rounds[l * 2] = (int)(dbg_bid / 1000) * 100000 + (int)(dbg_wait / 1000); a.rounds[l * 2 + 1] = (int)(dbg_serve / 1000) * 100000 + (int)((clock64() - clk1) / 1000); }
+#endif
         if (residual) atomicOr(a.info + l, TAOT_INFO_AUCTION_RESIDUAL);
     }
 }
 
-size_t match_smem_fixed(int R, int E, int K)
+size_t match_smem_fixed(int R, int E, int K, int dmax, int W, int ntiers)
 {
-    const int S = R * K;
-    return sizeof(u64) * (E + R) + sizeof(int32_t) * (3 * (size_t)E + 5 * (size_t)R + 3 * (size_t)S);
+    const size_t S = (size_t)R * K;
+    return sizeof(u64) * (E + R) + sizeof(int32_t) * (4 * (size_t)E + 5 * (size_t)R + 3 * S) +
+           sizeof(uint32_t) * ((size_t)dmax * W + (S + 1) * W) + sizeof(int32_t) * S * (ntiers > 0 ? ntiers : 1);
 }
 
 }  // namespace
@@ -282,24 +455,27 @@ size_t match_smem_fixed(int R, int E, int K)
 int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load,
                       const int32_t* d_rank_load, const float* d_plan, int32_t* d_slot_expert,
                       int32_t* d_slot_tokens, int32_t* d_X, int32_t* d_rounds, int32_t* d_info,
-                      int32_t* d_nrem, cudaStream_t st)
+                      int32_t* d_nrem, float* d_t12, cudaStream_t st)
 {
     const taot_params& p = h->p;
     MatchArgs a;
     a.n = d_n; a.expert_load = d_expert_load; a.rank_load = d_rank_load; a.plan = d_plan;
     a.e2r = h->d_e2r; a.B = h->d_B; a.rank_off = h->d_rank_off; a.rank_list = h->d_rank_list;
+    a.tiermask = h->d_tiermask; a.tierval = h->d_tierval;
     a.slot_expert = d_slot_expert; a.slot_tokens = d_slot_tokens; a.X = d_X; a.rounds = d_rounds;
-    a.info = d_info; a.nrem_g = d_nrem;
+    a.info = d_info; a.nrem_g = d_nrem; a.t12 = d_t12;
     a.R = p.R; a.E = p.E; a.K = p.K;
     a.dmax = p.E < p.R * p.K ? p.E : p.R * p.K;
+    a.W = (p.R + 31) / 32;
+    a.ntiers = (h->ntiers > 0 && p.price_step >= 0.0f && a.W <= kMaxW) ? h->ntiers : 0;
     a.eps0 = p.eps0; a.price_step = p.price_step; a.auction_max_rounds = p.auction_max_rounds;
-    size_t smem = match_smem_fixed(p.R, p.E, p.K);
+    size_t smem = match_smem_fixed(p.R, p.E, p.K, a.dmax, a.W, a.ntiers);
     const size_t nrem_bytes = sizeof(int32_t) * (size_t)a.dmax * p.R;
     a.nrem_in_smem = (smem + nrem_bytes <= 200 * 1024) ? 1 : 0;
     if (a.nrem_in_smem) smem += nrem_bytes;
-    const int NT = p.R <= 32 ? 128 : (p.R <= 64 ? 256 : (p.R <= 128 ? 512 : 1024));
+    if (smem > 227 * 1024) return TAOT_ERR_UNSUPPORTED;
     TAOT_CUDA_OK(cudaFuncSetAttribute(match_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    match_kernel<<<p.L, NT, smem, st>>>(a);
+    match_kernel<<<p.L, 256, smem, st>>>(a);
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
 }

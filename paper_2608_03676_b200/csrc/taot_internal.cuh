@@ -12,6 +12,7 @@
 // NC = ceil(SEG / TAOT_CHUNK) chunks, the last one possibly short.
 #define TAOT_CHUNK 16384
 #define TAOT_STREAM_THREADS 256            // threads of the streaming kernels: 64 elements each
+#define TAOT_MAX_TIERS 8                   // distinct bonus values the bit-set auction handles
 
 struct taot_handle_s {
     taot_params p;
@@ -24,12 +25,15 @@ struct taot_handle_s {
     double* d_rowlse0;       // [R]  LSE_j(-C_ij/eps) over all ranks j: the first u-update with v = 1
     int32_t* d_rank_off;     // [R+1] CSR of experts by home rank
     int32_t* d_rank_list;    // [E]
+    uint32_t* d_tiermask;    // [R hosts][ntiers][W] bit r set iff bonus(r -> host) == tierval[t]; null if ntiers == 0
+    float* d_tierval;        // [ntiers] distinct values of the auction bonus matrix, descending
+    int32_t ntiers;          // 0: too many distinct values, the auction scans densely
     // derived sizes
     int64_t seg;             // elements per (layer, rank) segment
     int32_t nc;              // chunks per segment
     int32_t kcap;            // Sinkhorn kernel-matrix capacity in floats per problem
     // workspace layout (byte offsets)
-    size_t off_cc, off_tabg, off_nbg, off_excess, off_spare, off_s, off_d, off_nrem;
+    size_t off_cc, off_tabg, off_nbg, off_excess, off_spare, off_s, off_d, off_nrem, off_t12;
     size_t ws_bytes;
     // host-call staging layout (byte offsets into d_ws of taot_plan_host)
     size_t hoff_topk, hoff_new, hoff_n, hoff_el, hoff_rl, hoff_ex, hoff_sp, hoff_plan, hoff_it, hoff_err,
@@ -54,7 +58,7 @@ int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, in
 int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load,
                       const int32_t* d_rank_load, const float* d_plan, int32_t* d_slot_expert,
                       int32_t* d_slot_tokens, int32_t* d_X, int32_t* d_rounds, int32_t* d_info,
-                      int32_t* d_nrem, cudaStream_t st);
+                      int32_t* d_nrem, float* d_t12, cudaStream_t st);
 int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_cc, int32_t* d_tabg,
                        int32_t* d_nbg, const int32_t* d_slot_expert, const int32_t* d_X, int32_t* d_new_idx,
                        int32_t* d_info, cudaStream_t st);

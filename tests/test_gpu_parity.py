@@ -126,3 +126,44 @@ def test_plan_host_round_trip(case):
     torch.cuda.synchronize()
     for key, val in host_out.items():
         assert (val.numpy() == out[key]).all(), key
+
+
+def test_auction_dense_scan_with_an_untiered_preference_matrix():
+    """A preference matrix with many distinct values takes the dense scan of Phase 3 instead of the
+    tier bit sets; both must agree with the oracle bit for bit."""
+    cfg = W.get_config("cfg2").replace(L=4)
+    e2r, C = topology(cfg)
+    g = torch.Generator().manual_seed(5)
+    B = torch.rand((cfg.R, cfg.R), generator=g, dtype=torch.float32)
+    B.fill_diagonal_(0.0)
+    topk = _routing(cfg)
+    pl = make_planner(cfg, B=B)
+    out = {k: cpu(v) for k, v in pl.plan(topk).items()}
+    for l in range(cfg.L):
+        m, a = oracle_schedule_layer(cfg, e2r.numpy(), B.numpy(), out["n"][l], out["expert_load"][l],
+                                     out["rank_load"][l], out["plan"][l])
+        assert (out["slot_expert"][l].ravel() == m["slot_expert"]).all()
+        assert (out["slot_tokens"][l].ravel() == m["slot_tokens"]).all()
+        assert (out["X"][l] == a["X"]).all()
+        assert out["rounds"][l].tolist() == [m["inner_rounds"], a["rounds"]]
+    pl.close()
+
+
+def test_auction_scores_that_round_together_and_a_round_cap():
+    """A price step so small that different win counts give the same fp32 score (ties must then go to
+    the lowest rank index, as in a dense scan), and a fixed number of auction rounds."""
+    cfg = W.get_config("cfg2").replace(L=3)
+    e2r, C = topology(cfg)
+    B = O.default_preference(C.numpy())
+    topk = _routing(cfg)
+    for step, cap in ((1e-9, 0), (0.1, 5), (0.0, 0)):
+        pl = make_planner(cfg, price_step=step, auction_max_rounds=cap)
+        out = {k: cpu(v) for k, v in pl.plan(topk).items()}
+        for l in range(cfg.L):
+            m, a = oracle_schedule_layer(cfg, e2r.numpy(), B, out["n"][l], out["expert_load"][l],
+                                         out["rank_load"][l], out["plan"][l], price_step=step,
+                                         auction_max_rounds=cap)
+            assert (out["X"][l] == a["X"]).all()
+            assert out["rounds"][l, 1] == a["rounds"]
+            assert bool(out["info"][l] & 8) == (a["residual"] > 0)
+        pl.close()
