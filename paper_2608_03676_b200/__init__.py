@@ -19,4 +19,5 @@ from .binding import (  # noqa: F401
     exported_symbols,
     histogram_static,
     STATIC_SCRATCH_BYTES,
+    PLAN_LAUNCHES,
 )

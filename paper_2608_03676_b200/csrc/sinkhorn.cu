@@ -13,32 +13,11 @@
 //
 // Stopping: half-step 1 of iteration t+1 produces the row sums of iterate t for free
 // (rowsum_i = u~_i * (K~ v~)_i), so the tolerance test costs nothing extra.
-#include "taot_internal.cuh"
+#include "sinkhorn_common.cuh"
+
+using namespace taot_sk;
 
 namespace {
-
-struct SinkArgs {
-    const float* s;
-    const float* d;
-    const float* C;
-    const double* rowlse0;
-    float* plan;
-    int32_t* iters;
-    float* row_err;
-    int32_t* info;
-    int32_t R;
-    int32_t kcap;
-    double inv_eps;
-    float eps0;
-    int32_t max_iters;
-    float tol;
-    int32_t check_every;
-};
-
-constexpr float kDriftLo = 2.0611536e-9f;   // e^-20
-constexpr float kDriftHi = 4.8516520e8f;    // e^+20
-constexpr float kSumLo = 1e-30f;
-constexpr float kSumHi = 1e30f;
 
 struct Smem {
     double* alpha;   // [R] by compact hot index
@@ -92,31 +71,6 @@ size_t smem_bytes(int R, int NT, int kcap)
 {
     return sizeof(double) * (3 * R + 32) + sizeof(float) * (6 * R + (NT > R ? NT : R)) +
            sizeof(int32_t) * (4 * R + 36) + sizeof(float) * (size_t)kcap;
-}
-
-// ordered compaction of {i < R : val[i] > 0} into list[], positions into pos[]; returns the count
-__device__ int compact_positive(const float* val, int R, int32_t* list, int32_t* pos, int32_t* wcnt)
-{
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, NW = blockDim.x >> 5;
-    int total = 0;
-    for (int base = 0; base < R; base += blockDim.x) {
-        const int i = base + tid;
-        const bool p = (i < R) && (val[i] > 0.0f);
-        const unsigned m = __ballot_sync(0xffffffffu, p);
-        if (lane == 0) wcnt[warp] = __popc(m);
-        __syncthreads();
-        int off = total;
-        for (int w = 0; w < warp; ++w) off += wcnt[w];
-        if (i < R) pos[i] = -1;
-        if (p) {
-            const int q = off + __popc(m & ((1u << lane) - 1u));
-            list[q] = i;
-            pos[i] = q;
-        }
-        for (int w = 0; w < NW; ++w) total += wcnt[w];
-        __syncthreads();
-    }
-    return total;
 }
 
 // K~_ij = exp(alpha_i + beta_j - C_ij/eps), fp64 exponent and exp, rounded once to fp32
@@ -188,6 +142,7 @@ __global__ void sinkhorn_kernel(SinkArgs a)
     const Smem m = carve(smem_raw, R, NT);
     const int64_t b = blockIdx.x;
     __shared__ double s_sum[2];
+    if (a.only_marked && a.iters[b] != kHandBack) return;
 
     // ---- supply scaling gamma = min(1, sum d / max(sum s, eps0)), compaction
     if (tid == 0) { s_sum[0] = 0.0; s_sum[1] = 0.0; }
@@ -374,6 +329,8 @@ __global__ void sinkhorn_kernel(SinkArgs a)
 
 }  // namespace
 
+int taot_launch_sinkhorn_tile(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st);
+
 int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
                          int32_t* d_iters, float* d_row_err, int32_t* d_info, cudaStream_t st)
 {
@@ -385,10 +342,15 @@ int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, in
     a.inv_eps = 1.0 / (double)p.eps;
     a.eps0 = p.eps0; a.max_iters = p.max_iters; a.tol = p.tol;
     a.check_every = p.check_every < 1 ? 1 : p.check_every;
+    // fast path: kernel matrix in registers; problems it cannot hold (or whose fp32 sums leave the
+    // safe range) come back marked and are solved by the shared-memory kernel below
+    a.only_marked = 1;
+    const int launched = taot_launch_sinkhorn_tile(h, a, B, st);
+    if (launched < 0) return launched;
     const int NT = p.R <= 32 ? 32 : (p.R <= 64 ? 128 : (p.R <= 128 ? 256 : 512));
     const size_t smem = smem_bytes(p.R, NT, h->kcap);
     TAOT_CUDA_OK(cudaFuncSetAttribute(sinkhorn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     sinkhorn_kernel<<<B, NT, smem, st>>>(a);
     TAOT_CUDA_OK(cudaGetLastError());
-    return 1;
+    return launched + 1;
 }
