@@ -66,8 +66,9 @@ enum {
 
 /*
  * Problem description.  Set struct_size = sizeof(taot_params).
- * Supported ranges: 1 <= R <= 256, 1 <= E <= 1024, 1 <= K <= 8, 1 <= k <= 64, L >= 1,
- * T >= R, T % R == 0, T*k < 2^31.
+ * Supported ranges: 1 <= R <= 256 for the whole path (taot_excess_spare and taot_sinkhorn alone accept
+ * R up to 1024; the other calls then return TAOT_ERR_UNSUPPORTED), 1 <= E <= 1024, 1 <= K <= 8,
+ * 1 <= k <= 64, L >= 1, T >= R, T % R == 0, T*k < 2^31.
  */
 typedef struct {
     int32_t struct_size;
@@ -187,6 +188,10 @@ int taot_excess_spare(taot_handle_t h, const int32_t* d_rank_load, int32_t B, in
  * T_ij *= min(1, d_j / (sum_i T_ij + eps0)).
  *   d_plan [B,R,R] fp32 (fully overwritten), d_iters [B], d_row_err [B], d_info [B].
  * The iterates are carried so that neither M nor u, v can under- or overflow for any C/eps.
+ * `ws` is needed only for R > 256 (the kernel matrix then lives in workspace; batches larger than
+ * the handle's L are solved in slices of L).  Problems with |{s>0}| * |{d>0}| beyond the capacity
+ * (R*R/4 for R > 128, which disjoint supply/demand ranks never exceed) get TAOT_INFO_SINKHORN_SIZE
+ * and a zero plan.
  */
 int taot_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
                   int32_t* d_iters, float* d_row_err, int32_t* d_info, void* ws, void* stream);

@@ -27,7 +27,7 @@ bool valid_params(const taot_params* p)
 
 bool supported_params(const taot_params* p)
 {
-    return p->R <= 256 && p->E <= 1024 && p->K <= 8 && p->k <= 64 &&
+    return p->R <= 1024 && p->E <= 1024 && p->K <= 8 && p->k <= 64 &&
            (int64_t)p->L * p->R * ((p->T / p->R * p->k + TAOT_CHUNK - 1) / TAOT_CHUNK) < ((int64_t)1 << 31);
 }
 
@@ -47,6 +47,11 @@ void layout(taot_handle_t h)
     const int64_t r2 = (int64_t)p.R * p.R;
     int64_t cap = r2 / 4 > 12288 ? r2 / 4 : 12288;
     h->kcap = (int32_t)(cap < r2 ? cap : r2);
+    h->kcap_global = 0;
+    if (p.R > 256) {                      // beyond shared memory: the kernel matrix lives in workspace
+        h->kcap = 0;
+        h->kcap_global = r2 / 4;          // |hot| * |cold| <= R^2/4 whenever supply and demand ranks are disjoint
+    }
     const size_t LR = (size_t)p.L * p.R;
     const int dmax = p.E < p.R * p.K ? p.E : p.R * p.K;
     size_t off = 0;
@@ -60,6 +65,7 @@ void layout(taot_handle_t h)
     h->off_d = take(sizeof(float) * LR);
     h->off_nrem = take(sizeof(int32_t) * (size_t)p.L * dmax * p.R);
     h->off_t12 = take(sizeof(float) * (size_t)p.L * p.E * 2 * p.R);
+    h->off_kt = take(sizeof(float) * (size_t)p.L * (size_t)h->kcap_global);
     h->ws_bytes = off;
 
     const size_t S = (size_t)p.R * p.K;
@@ -274,6 +280,7 @@ int taot_last_launch_count(taot_handle_t h, int32_t* count)
 int taot_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_n, int32_t* d_expert_load,
                    int32_t* d_rank_load, int32_t* d_info, void* ws, void* stream)
 {
+    if (h && h->p.R > 256) return TAOT_ERR_UNSUPPORTED;      // beyond 256 ranks only Phase 1 is built
     if (!h || !d_topk || !d_n || !d_expert_load || !d_rank_load || !d_info || !ws) return TAOT_ERR_NULL;
     if ((reinterpret_cast<uintptr_t>(d_topk) & 3) || (reinterpret_cast<uintptr_t>(ws) & 255)) return TAOT_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -300,10 +307,12 @@ int taot_excess_spare(taot_handle_t h, const int32_t* d_rank_load, int32_t B, in
 int taot_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
                   int32_t* d_iters, float* d_row_err, int32_t* d_info, void* ws, void* stream)
 {
-    (void)ws;
     if (!h || !d_s || !d_d || !d_plan || !d_iters || !d_row_err || !d_info) return TAOT_ERR_NULL;
     if (B < 1) return TAOT_ERR_PARAM;
-    int a = taot_launch_sinkhorn(h, d_s, d_d, B, d_plan, d_iters, d_row_err, d_info, static_cast<cudaStream_t>(stream));
+    if (h->kcap_global > 0 && (!ws || (reinterpret_cast<uintptr_t>(ws) & 255))) return ws ? TAOT_ERR_ALIGN : TAOT_ERR_NULL;
+    int a = taot_launch_sinkhorn(h, d_s, d_d, B, d_plan, d_iters, d_row_err, d_info,
+                                 ws ? reinterpret_cast<float*>(at(ws, h->off_kt)) : nullptr,
+                                 static_cast<cudaStream_t>(stream));
     if (a < 0) return a;
     h->last_launches = a;
     return TAOT_OK;
@@ -313,6 +322,7 @@ int taot_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load
                const float* d_plan, int32_t* d_slot_expert, int32_t* d_slot_tokens, int32_t* d_X,
                int32_t* d_rounds, int32_t* d_info, void* ws, void* stream)
 {
+    if (h && h->p.R > 256) return TAOT_ERR_UNSUPPORTED;      // beyond 256 ranks only Phase 1 is built
     if (!h || !d_n || !d_expert_load || !d_rank_load || !d_plan || !d_slot_expert || !d_slot_tokens || !d_X ||
         !d_info || !ws)
         return TAOT_ERR_NULL;
@@ -328,6 +338,7 @@ int taot_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load
 int taot_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_slot_expert, const int32_t* d_X,
                 int32_t* d_new_idx, int32_t* d_info, void* ws, int32_t reuse_counts, void* stream)
 {
+    if (h && h->p.R > 256) return TAOT_ERR_UNSUPPORTED;      // beyond 256 ranks only Phase 1 is built
     if (!h || !d_topk || !d_slot_expert || !d_X || !d_new_idx || !d_info || !ws) return TAOT_ERR_NULL;
     if ((reinterpret_cast<uintptr_t>(d_topk) & 3) || (reinterpret_cast<uintptr_t>(d_new_idx) & 3) ||
         (reinterpret_cast<uintptr_t>(ws) & 255))
@@ -350,6 +361,7 @@ int taot_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_slot_ex
 
 int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, void* ws, void* stream)
 {
+    if (h && h->p.R > 256) return TAOT_ERR_UNSUPPORTED;      // beyond 256 ranks only Phase 1 is built
     if (!h || !d_topk || !o || !ws) return TAOT_ERR_NULL;
     if (!o->n || !o->expert_load || !o->rank_load || !o->plan || !o->sinkhorn_iters || !o->row_err ||
         !o->slot_expert || !o->slot_tokens || !o->X || !o->new_idx || !o->info)
@@ -375,7 +387,9 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, voi
     if ((a = taot_launch_merge(h, cc, o->n, o->expert_load, o->rank_load, excess, spare, fs, fd, st)) < 0) return a;
     total += a;
     TAOT_MARK(2);
-    if ((a = taot_launch_sinkhorn(h, fs, fd, p.L, o->plan, o->sinkhorn_iters, o->row_err, o->info, st)) < 0) return a;
+    if ((a = taot_launch_sinkhorn(h, fs, fd, p.L, o->plan, o->sinkhorn_iters, o->row_err, o->info,
+                                  reinterpret_cast<float*>(at(ws, h->off_kt)), st)) < 0)
+        return a;
     total += a;
     TAOT_MARK(3);
     if ((a = taot_launch_match(h, o->n, o->expert_load, o->rank_load, o->plan, o->slot_expert, o->slot_tokens,

@@ -135,11 +135,11 @@ __device__ void slow_half2(const Smem& m, const SinkArgs& a, int Hn, int Cn)
     __syncthreads();
 }
 
-__global__ void sinkhorn_kernel(SinkArgs a)
+__global__ void __launch_bounds__(1024) sinkhorn_kernel(SinkArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int R = a.R, NT = blockDim.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, NW = NT >> 5;
-    const Smem m = carve(smem_raw, R, NT);
+    Smem m = carve(smem_raw, R, NT);
     const int64_t b = blockIdx.x;
     __shared__ double s_sum[2];
     if (a.only_marked && a.iters[b] != kHandBack) return;
@@ -185,7 +185,11 @@ __global__ void sinkhorn_kernel(SinkArgs a)
     int info = 0;
     if (sum_s > sum_d) info |= TAOT_INFO_SUPPLY_SCALED;
     const bool empty = (Hn == 0) || (Cn == 0);
-    const bool too_big = (int64_t)Hn * Cn > (int64_t)a.kcap;
+    bool too_big = (int64_t)Hn * Cn > (int64_t)a.kcap;
+    if (too_big && a.kt_global != nullptr && (int64_t)Hn * Cn <= a.kcap_global) {
+        m.Kt = a.kt_global + b * a.kcap_global;           // kernel matrix in global memory (L2 when the batch is small)
+        too_big = false;
+    }
     if (too_big) info |= TAOT_INFO_SINKHORN_SIZE;
 
     int t = 0;
@@ -332,25 +336,41 @@ __global__ void sinkhorn_kernel(SinkArgs a)
 int taot_launch_sinkhorn_tile(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st);
 
 int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
-                         int32_t* d_iters, float* d_row_err, int32_t* d_info, cudaStream_t st)
+                         int32_t* d_iters, float* d_row_err, int32_t* d_info, float* d_kt, cudaStream_t st)
 {
     const taot_params& p = h->p;
     SinkArgs a;
-    a.s = d_s; a.d = d_d; a.C = h->d_C; a.rowlse0 = h->d_rowlse0;
-    a.plan = d_plan; a.iters = d_iters; a.row_err = d_row_err; a.info = d_info;
+    a.C = h->d_C; a.rowlse0 = h->d_rowlse0;
     a.R = p.R; a.kcap = h->kcap;
     a.inv_eps = 1.0 / (double)p.eps;
     a.eps0 = p.eps0; a.max_iters = p.max_iters; a.tol = p.tol;
     a.check_every = p.check_every < 1 ? 1 : p.check_every;
-    // fast path: kernel matrix in registers; problems it cannot hold (or whose fp32 sums leave the
-    // safe range) come back marked and are solved by the shared-memory kernel below
-    a.only_marked = 1;
-    const int launched = taot_launch_sinkhorn_tile(h, a, B, st);
-    if (launched < 0) return launched;
-    const int NT = p.R <= 32 ? 32 : (p.R <= 64 ? 128 : (p.R <= 128 ? 256 : 512));
+    a.kt_global = h->kcap_global > 0 ? d_kt : nullptr;
+    a.kcap_global = h->kcap_global;
+    const int NT = p.R <= 32 ? 32 : (p.R <= 64 ? 128 : (p.R <= 128 ? 256 : (p.R <= 256 ? 512 : 1024)));
     const size_t smem = smem_bytes(p.R, NT, h->kcap);
     TAOT_CUDA_OK(cudaFuncSetAttribute(sinkhorn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    sinkhorn_kernel<<<B, NT, smem, st>>>(a);
-    TAOT_CUDA_OK(cudaGetLastError());
-    return launched + 1;
+    int launched = 0;
+    // the global scratch (if any) holds p.L problems: larger batches go through in slices
+    const int32_t slice = a.kt_global ? p.L : B;
+    for (int32_t b0 = 0; b0 < B; b0 += slice) {
+        const int32_t nb = (B - b0) < slice ? (B - b0) : slice;
+        a.s = d_s + (int64_t)b0 * p.R; a.d = d_d + (int64_t)b0 * p.R;
+        a.plan = d_plan + (int64_t)b0 * p.R * p.R; a.iters = d_iters + b0; a.row_err = d_row_err + b0;
+        a.info = d_info + b0;
+        if (p.R <= 256) {
+            // fast path: kernel matrix in registers; problems it cannot hold (or whose fp32 sums leave the
+            // safe range) come back marked and are solved by the shared-memory kernel below
+            a.only_marked = 1;
+            const int n = taot_launch_sinkhorn_tile(h, a, nb, st);
+            if (n < 0) return n;
+            launched += n;
+        } else {
+            a.only_marked = 0;
+        }
+        sinkhorn_kernel<<<nb, NT, smem, st>>>(a);
+        TAOT_CUDA_OK(cudaGetLastError());
+        launched += 1;
+    }
+    return launched;
 }

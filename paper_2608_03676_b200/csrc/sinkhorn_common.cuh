@@ -22,6 +22,8 @@ struct SinkArgs {
     float tol;
     int32_t check_every;
     int32_t only_marked;     // generic kernel: solve only the problems the register-tile kernel handed back
+    float* kt_global;        // [B][kcap_global] kernel-matrix scratch in global memory for problems too big for
+    int64_t kcap_global;     // shared memory (floats per problem); null / 0 if the handle has none
 };
 
 constexpr float kDriftLo = 2.0611536e-9f;   // e^-20

@@ -31,9 +31,10 @@ struct taot_handle_s {
     // derived sizes
     int64_t seg;             // elements per (layer, rank) segment
     int32_t nc;              // chunks per segment
-    int32_t kcap;            // Sinkhorn kernel-matrix capacity in floats per problem
+    int32_t kcap;            // Sinkhorn kernel-matrix capacity in floats per problem (shared memory)
+    int64_t kcap_global;     // same, global-memory scratch per problem (R > 256 only), else 0
     // workspace layout (byte offsets)
-    size_t off_cc, off_tabg, off_nbg, off_excess, off_spare, off_s, off_d, off_nrem, off_t12;
+    size_t off_cc, off_tabg, off_nbg, off_excess, off_spare, off_s, off_d, off_nrem, off_t12, off_kt;
     size_t ws_bytes;
     // host-call staging layout (byte offsets into d_ws of taot_plan_host)
     size_t hoff_topk, hoff_new, hoff_n, hoff_el, hoff_rl, hoff_ex, hoff_sp, hoff_plan, hoff_it, hoff_err,
@@ -54,7 +55,7 @@ int taot_launch_merge(taot_handle_t h, const int32_t* d_cc, int32_t* d_n, int32_
 int taot_launch_excess_spare(taot_handle_t h, const int32_t* d_rank_load, int32_t B, int32_t* d_excess,
                              int32_t* d_spare, float* d_s, float* d_d, cudaStream_t st);
 int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
-                         int32_t* d_iters, float* d_row_err, int32_t* d_info, cudaStream_t st);
+                         int32_t* d_iters, float* d_row_err, int32_t* d_info, float* d_kt, cudaStream_t st);
 int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load,
                       const int32_t* d_rank_load, const float* d_plan, int32_t* d_slot_expert,
                       int32_t* d_slot_tokens, int32_t* d_X, int32_t* d_rounds, int32_t* d_info,

@@ -1,0 +1,64 @@
+"""Config 5 (Sinkhorn-only scaling sweep): sampled cells against the oracle.  Rank loads come from
+the sweep generator, supply/demand from `taot_excess_spare`, 500 fixed iterations, 3-tier cost."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import workloads as W
+from workloads.configs import SWEEP_ITERS, SWEEP_TIERS
+from helpers import check_sinkhorn_problem, cpu
+
+pytestmark = pytest.mark.gpu
+
+
+def _planner(B, R, eps_frac, iters=SWEEP_ITERS, tol=0.0):
+    import paper_2608_03676_b200 as P
+    C = W.cost_matrix(R, 8, SWEEP_TIERS, 4)
+    e2r = torch.arange(R, dtype=torch.int32)
+    pl = P.Planner(L=B, R=R, E=R, K=1, k=1, T=R, e2r=e2r, C=C, eps=eps_frac * max(SWEEP_TIERS),
+                   max_iters=iters, tol=tol)
+    return pl, C
+
+
+@pytest.mark.parametrize("R,B,check", [(8, 64, 64), (16, 64, 64), (64, 64, 16), (256, 64, 4), (1024, 3, 1)])
+@pytest.mark.parametrize("eps_frac", [0.1, 0.01])
+def test_sweep_cell(R, B, check, eps_frac):
+    pl, C = _planner(B, R, eps_frac)
+    loads = W.sweep_rank_loads(B, R, seed=1000 + R, device="cuda")
+    ex, sp, s, d = pl.excess_spare(loads)
+    mean, ex_ref, sp_ref = O.excess_spare(cpu(loads))
+    assert (cpu(ex) == ex_ref).all() and (cpu(sp) == sp_ref).all()
+    out = pl.sinkhorn(s, d)
+    torch.cuda.synchronize()
+    plan, iters, err, info = cpu(out["plan"]), cpu(out["iters"]), cpu(out["row_err"]), cpu(out["info"])
+    assert (iters == SWEEP_ITERS).all() and (info == 0).all()
+    worst = 0.0
+    for b in range(check):
+        r = check_sinkhorn_problem(cpu(s)[b], cpu(d)[b], C.numpy(), eps_frac * max(SWEEP_TIERS), plan[b], iters[b],
+                                   err[b], SWEEP_ITERS, 0.0)
+        worst = max(worst, r["max_rel"])
+    # properties that hold for every problem of the cell, checked on the GPU
+    tot = s.double().sum(1)
+    col_viol = (out["plan"].double().sum(1) - d.double()).abs().sum(1)
+    assert bool((col_viol <= 1e-5 * tot).all())
+    assert bool((out["plan"] >= 0).all())
+    print(f"R={R} eps={eps_frac}: worst rel err {worst:.2e} over {check} problems")
+    pl.close()
+
+
+def test_batches_larger_than_the_handle_and_unsupported_calls_beyond_256_ranks():
+    import paper_2608_03676_b200 as P
+    R = 512
+    pl, C = _planner(2, R, 0.1, iters=20)
+    loads = W.sweep_rank_loads(5, R, seed=7, device="cuda")        # 5 problems through a handle built for 2
+    ex, sp, s, d = pl.excess_spare(loads)
+    out = pl.sinkhorn(s, d)
+    torch.cuda.synchronize()
+    for b in (0, 2, 4):
+        check_sinkhorn_problem(cpu(s)[b], cpu(d)[b], C.numpy(), 0.1 * max(SWEEP_TIERS), cpu(out["plan"])[b],
+                               cpu(out["iters"])[b], cpu(out["row_err"])[b], 20, 0.0)
+    topk = torch.zeros((2, R, 1), dtype=torch.int32, device="cuda")
+    with pytest.raises(P.TaotError):
+        pl.histogram(topk)
+    pl.close()
