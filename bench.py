@@ -47,6 +47,10 @@ def parse_args():
     ap.add_argument("--cpu-seconds", type=float, default=20.0, help="budget of the CPU-baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-streams", action="store_true", help="skip the HBM-sized streaming report")
+    ap.add_argument("--sweep", action="store_true",
+                    help="config 5: time taot_sinkhorn alone over the (B, R, eps) grid and print one JSON object")
+    ap.add_argument("--sweep-max-elems", type=float, default=6e9,
+                    help="skip sweep cells whose plan tensor would exceed this many floats")
     return ap.parse_args()
 
 
@@ -383,8 +387,46 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Config 5: Sinkhorn only.  Per cell: plans/s and the executed-FMA fraction of the fp32 peak."""
+    import paper_2608_03676_b200 as P
+    from workloads.configs import SWEEP_ITERS, SWEEP_TIERS
+    torch.cuda.set_device(0)
+    peaks = measured_peaks()
+    props = torch.cuda.get_device_properties(0)
+    fp32_peak = props.multi_processor_count * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+    cells = []
+    for (B, R, eps_frac) in W.sweep_cells():
+        if B * R * R > args.sweep_max_elems:
+            cells.append(dict(B=B, R=R, eps_frac=eps_frac, skipped="plan tensor larger than --sweep-max-elems"))
+            continue
+        C = W.cost_matrix(R, 8, SWEEP_TIERS, 4)
+        pl = P.Planner(L=B, R=R, E=R, K=1, k=1, T=R, e2r=torch.arange(R, dtype=torch.int32), C=C,
+                       eps=eps_frac * max(SWEEP_TIERS), max_iters=SWEEP_ITERS, tol=0.0)
+        loads = W.sweep_rank_loads(B, R, seed=5000 + R, device="cuda")
+        ex, sp, s, d = pl.excess_spare(loads)
+        out = pl.sinkhorn(s, d)
+        reps = 3 if B * R * R < 5e8 else 1
+        ms = timed_steps(lambda: pl.sinkhorn(s, d, out), reps + 1, None)[1:]
+        hn = (ex > 0).sum(1).double(); cn = (sp > 0).sum(1).double()
+        fma = float((2 * hn * cn * (SWEEP_ITERS - 1)).sum())
+        t = float(np.median(ms)) * 1e-3
+        cells.append(dict(B=B, R=R, eps_frac=eps_frac, ms=t * 1e3, plans_per_s=B / t,
+                          tflops=2 * fma / t / 1e12, frac_fp32_peak=2 * fma / t / 1e12 / fp32_peak,
+                          hot_mean=float(hn.mean()), cold_mean=float(cn.mean()),
+                          info_or=int(out["info"].max())))
+        pl.close()
+        del out, loads, s, d, ex, sp
+        torch.cuda.empty_cache()
+    print(json.dumps(dict(metric="Sinkhorn placement plans/s per (B, R, eps) cell, 500 fixed iterations",
+                          unit="plans/s", fp32_peak_tflops=fp32_peak, cells=cells)))
+
+
 def main():
     args = parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

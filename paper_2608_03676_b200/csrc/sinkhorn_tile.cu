@@ -43,102 +43,33 @@ __device__ __forceinline__ float transpose_reduce(float (&p)[N], int lane)
     return v;
 }
 
+// Shared-memory state of one problem (arrays sized for RMAX = 32*CG ranks).
+template <int NW, int CG>
+struct TileSmem {
+    static constexpr int RMAX = 32 * CG;
+    double alpha[RMAX], beta[RMAX], phin[RMAX], red[64];
+    float st[RMAX], dd[RMAX], sv[RMAX], dv[RMAX], vs[RMAX];
+    float part[NW > 1 ? NW * RMAX : 1];
+    float errw[32];
+    int32_t hot[RMAX], cold[RMAX], hpos[RMAX], cpos[RMAX], wcnt[32];
+    int flags[4];                    // [parity]: some u~, v~ of this iteration left [e^-20, e^20]
+    double sum[2];
+};
+
+// The iteration proper, for a tile of RPW rows per warp.  Returns false if the problem must be handed back.
 template <int NW, int RPW, int CG>
-__global__ void __launch_bounds__(NW * 32)
-sinkhorn_tile_kernel(SinkArgs a)
+__device__ __forceinline__ bool tile_solve(const SinkArgs& a, TileSmem<NW, CG>& sm, int Hn, int Cn, double sum_st,
+                                           int info, float* out, int64_t b)
 {
     constexpr int RMAX = 32 * CG, NT = NW * 32;
-    __shared__ double sh_alpha[RMAX], sh_beta[RMAX], sh_phin[RMAX], sh_red[64];
-    __shared__ float sh_st[RMAX], sh_dd[RMAX], sh_sv[RMAX], sh_dv[RMAX], sh_vs[RMAX];
-    __shared__ float sh_part[NW > 1 ? NW * RMAX : 1];
-    __shared__ float sh_errw[32];
-    __shared__ int32_t sh_hot[RMAX], sh_cold[RMAX], sh_hpos[RMAX], sh_cpos[RMAX], sh_wcnt[32];
-    __shared__ int sh_flags[4];             // [parity*2 + 0] bad sum, [parity*2 + 1] drift
-    __shared__ double s_sum[2];
-
     const int R = a.R, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t b = blockIdx.x;
-
-    // ---- supply scaling gamma = min(1, sum d / max(sum s, eps0)), compaction of supply / demand ranks
-    {
-        double ps = 0.0, pd = 0.0;
-        for (int i = tid; i < R; i += NT) {
-            const float sv = a.s[b * R + i], dv = a.d[b * R + i];
-            ps += sv > 0.0f ? (double)sv : 0.0;
-            pd += dv > 0.0f ? (double)dv : 0.0;
-        }
-        for (int o = 16; o > 0; o >>= 1) {
-            ps += __shfl_xor_sync(kFull, ps, o);
-            pd += __shfl_xor_sync(kFull, pd, o);
-        }
-        if (lane == 0) { sh_red[warp] = ps; sh_red[32 + warp] = pd; }
-        if (tid < 4) sh_flags[tid] = 0;
-        __syncthreads();
-        if (tid == 0) {
-            double S = 0.0, D = 0.0;
-            for (int w = 0; w < NW; ++w) { S += sh_red[w]; D += sh_red[32 + w]; }
-            s_sum[0] = S; s_sum[1] = D;
-        }
-        __syncthreads();
-    }
-    const double sum_s = s_sum[0], sum_d = s_sum[1];
-    const double gamma = fmin(1.0, sum_d / fmax(sum_s, (double)a.eps0));
-    for (int i = tid; i < R; i += NT) {
-        const float sv = a.s[b * R + i], dv = a.d[b * R + i];
-        sh_sv[i] = sv > 0.0f ? (float)(gamma * (double)sv) : 0.0f;
-        sh_dv[i] = dv > 0.0f ? dv : 0.0f;
-    }
-    __syncthreads();
-    const int Hn = compact_positive(sh_sv, R, sh_hot, sh_hpos, sh_wcnt);
-    const int Cn = compact_positive(sh_dv, R, sh_cold, sh_cpos, sh_wcnt);
-    if (Hn > NW * RPW) {                     // does not fit this tile: the other kernel takes it
-        if (tid == 0) a.iters[b] = kHandBack;
-        return;
-    }
-    for (int i = tid; i < Hn; i += NT) sh_st[i] = sh_sv[sh_hot[i]];
-    for (int j = tid; j < Cn; j += NT) sh_dd[j] = sh_dv[sh_cold[j]];
-    __syncthreads();
-
-    int info = 0;
-    if (sum_s > sum_d) info |= TAOT_INFO_SUPPLY_SCALED;
-    float* out = a.plan + b * (int64_t)R * R;
-    if (Hn == 0 || Cn == 0) {
-        for (int q = tid; q < R * R; q += NT) out[q] = 0.0f;
-        if (tid == 0) {
-            a.iters[b] = 0;
-            a.row_err[b] = 0.0f;
-            if (info) atomicOr(a.info + b, info);
-        }
-        return;
-    }
-    double sum_st = 0.0;
-    for (int i = 0; i < Hn; ++i) sum_st += (double)sh_st[i];          // same order in every thread
     const double tol_abs = (double)a.tol * sum_st;
 
-    // ---- iteration 1 in the log domain (v = 1 on every rank): phi = log s~ - LSE_j(-C_ij/eps) over all j,
-    //      psi_j = log d_j - LSE_i(phi_i - C_ij/eps)
-    for (int i = tid; i < Hn; i += NT) sh_phin[i] = log((double)sh_st[i]) - a.rowlse0[sh_hot[i]];
-    __syncthreads();
-    for (int j = tid; j < Cn; j += NT) {
-        const int cj = sh_cold[j];
-        double mx = -INFINITY;
-        for (int i = 0; i < Hn; ++i) {
-            const double x = sh_phin[i] - (double)a.C[(int64_t)sh_hot[i] * R + cj] * a.inv_eps;
-            mx = x > mx ? x : mx;
-        }
-        double acc = 0.0;
-        for (int i = 0; i < Hn; ++i)
-            acc += exp(sh_phin[i] - (double)a.C[(int64_t)sh_hot[i] * R + cj] * a.inv_eps - mx);
-        sh_beta[j] = log((double)sh_dd[j]) - (mx + log(acc));
-    }
-    for (int i = tid; i < Hn; i += NT) sh_alpha[i] = sh_phin[i];
-    __syncthreads();
-
-    // ---- this thread's tile and the scalars it owns
     const int row0 = warp * RPW;
     const int rowl = row0 + (lane & (RPW - 1));       // the row whose sum this lane ends up holding
     const bool row_ok = rowl < Hn;
-    const float st_l = row_ok ? sh_st[rowl] : 1.0f;
+    const bool row_owner = row_ok && lane < RPW;
+    const float st_l = row_ok ? sm.st[rowl] : 1.0f;
     float K[RPW][CG];
     float ddg[CG], vreg[CG];
     bool col_ok[CG];
@@ -146,7 +77,7 @@ sinkhorn_tile_kernel(SinkArgs a)
     for (int g = 0; g < CG; ++g) {
         const int col = lane + 32 * g;
         col_ok[g] = col < Cn;
-        ddg[g] = col_ok[g] ? sh_dd[col] : 1.0f;
+        ddg[g] = col_ok[g] ? sm.dd[col] : 1.0f;
         vreg[g] = 1.0f;
     }
     auto build_tile = [&]() {
@@ -158,8 +89,8 @@ sinkhorn_tile_kernel(SinkArgs a)
                 const int col = lane + 32 * g;
                 float v = 0.0f;
                 if (row < Hn && col < Cn) {
-                    const double c = (double)a.C[(int64_t)sh_hot[row] * R + sh_cold[col]] * a.inv_eps;
-                    v = (float)exp(sh_alpha[row] + sh_beta[col] - c);
+                    const double c = (double)a.C[(int64_t)sm.hot[row] * R + sm.cold[col]] * a.inv_eps;
+                    v = (float)exp(sm.alpha[row] + sm.beta[col] - c);
                 }
                 K[aa][g] = v;
             }
@@ -168,27 +99,28 @@ sinkhorn_tile_kernel(SinkArgs a)
     build_tile();
     float uo = 1.0f;                 // committed u~ of row `rowl`
     int t = 1;
+    int until_check = a.check_every; // iterations until the next tolerance test (tested when it reaches 1)
     float err_out = 0.0f;
-    bool hand_back = false;
+    const float tol_abs_f = (float)tol_abs;
+    // u~ and v~ must stay inside [e^-20, e^20]; for positive floats that is one unsigned compare on the bits
+    // (negative, NaN and infinite values fall outside too)
+    const uint32_t lo_bits = __float_as_uint(kDriftLo), span_bits = __float_as_uint(kDriftHi) - lo_bits;
 
     for (;;) {
-        const int par = (t & 1) * 2;
+        const int par = t & 1;
         // ================= half-step 1: r = K~ v~ (row sums of iterate t), u' = s~ / r
         float p[RPW];
 #pragma unroll
         for (int aa = 0; aa < RPW; ++aa) {
-            float acc = 0.0f;
+            float acc = K[aa][0] * vreg[0];
 #pragma unroll
-            for (int g = 0; g < CG; ++g) acc = fmaf(K[aa][g], vreg[g], acc);
+            for (int g = 1; g < CG; ++g) acc = fmaf(K[aa][g], vreg[g], acc);
             p[aa] = acc;
         }
         const float r = transpose_reduce<RPW>(p, lane);
-        const float un = row_ok ? st_l / r : 1.0f;
-        float e = (row_ok && lane < RPW) ? fabsf(fmaf(uo, r, -st_l)) : 0.0f;
-        bool bad = row_ok && !(r > kSumLo && r < kSumHi);
-        bool drift = row_ok && !(un > kDriftLo && un < kDriftHi);
-        for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(kFull, e, o);
-        // column partials over this warp's rows, with the proposed u'
+        const float un = row_ok ? st_l * __frcp_rn(r) : 1.0f;
+        bool odd = (__float_as_uint(un) - lo_bits) > span_bits;       // out of range: fold, or hand back
+        // ================= half-step 2 (speculative until the stop test): c = K~^T u', v' = d / c
         float cp[CG];
 #pragma unroll
         for (int g = 0; g < CG; ++g) cp[g] = 0.0f;
@@ -198,73 +130,94 @@ sinkhorn_tile_kernel(SinkArgs a)
 #pragma unroll
             for (int g = 0; g < CG; ++g) cp[g] = fmaf(K[aa][g], ua, cp[g]);
         }
-        double err;
-        if (NW == 1) {
-            err = (double)e;
-        } else {
-#pragma unroll
-            for (int g = 0; g < CG; ++g) sh_part[warp * RMAX + lane + 32 * g] = cp[g];
-            if (lane == 0) sh_errw[warp] = e;
-            if (bad) sh_flags[par] = 1;
-            if (drift) sh_flags[par + 1] = 1;
-            __syncthreads();
-            err = 0.0;
-            for (int w = 0; w < NW; ++w) err += (double)sh_errw[w];
-            if (tid == 0) { sh_flags[(par ^ 2)] = 0; sh_flags[(par ^ 2) + 1] = 0; }
+        // ---- the row sums belong to iterate t: is this where the solve stops?
+        const bool last = t >= a.max_iters;
+        const bool check = a.tol > 0.0f && until_check == 1;
+        float err = 0.0f;
+        if (last || check) {                                             // uniform over the block
+            float e = row_owner ? fabsf(fmaf(uo, r, -st_l)) : 0.0f;
+            for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(kFull, e, o);
+            err = e;
         }
-        // ---- the row sums just computed belong to iterate t: stop here?
-        const bool check = a.tol > 0.0f && (t % a.check_every == 0);
-        if (NW == 1) bad = __any_sync(kFull, bad);
-        else bad = sh_flags[par] != 0;
-        if (bad) { hand_back = true; break; }
-        if (t >= a.max_iters || (check && err <= tol_abs)) {
-            err_out = (float)(err / sum_st);
-            if (a.tol > 0.0f && !(err <= tol_abs)) info |= TAOT_INFO_SINKHORN_CAP;
-            break;
-        }
-        // ================= half-step 2: c = K~^T u', v' = d / c
+        float vnew[CG];
         if (NW == 1) {
-            bool bad2 = false;
 #pragma unroll
             for (int g = 0; g < CG; ++g) {
-                const float c = cp[g];
-                if (col_ok[g]) {
-                    bad2 |= !(c > kSumLo && c < kSumHi);
-                    const float vn = ddg[g] / c;
-                    drift |= !(vn > kDriftLo && vn < kDriftHi);
-                    vreg[g] = vn;
-                }
+                const float vn = col_ok[g] ? ddg[g] * __frcp_rn(cp[g]) : 1.0f;
+                odd |= (__float_as_uint(vn) - lo_bits) > span_bits;
+                vnew[g] = vn;
             }
-            if (__any_sync(kFull, bad2)) { hand_back = true; break; }
-            drift = __any_sync(kFull, drift);
+            odd = __any_sync(kFull, odd);
         } else {
+#pragma unroll
+            for (int g = 0; g < CG; ++g) sm.part[warp * RMAX + lane + 32 * g] = cp[g];
+            if ((last || check) && lane == 0) sm.errw[warp] = err;
+            if (odd) sm.flags[par] = 1;
+            __syncthreads();
+            if (last || check) {
+                err = 0.0f;
+#pragma unroll
+                for (int w = 0; w < NW; ++w) err += sm.errw[w];
+            }
+            if (tid == 0) sm.flags[par ^ 1] = 0;
+        }
+        if (last || (check && err <= tol_abs_f)) {
+            // a row sum outside the safe range makes this row error meaningless: let the other kernel redo it
+            const bool bad_r = row_ok && !(r > kSumLo && r < kSumHi);
+            if (NW == 1 ? __any_sync(kFull, bad_r) : __syncthreads_or(bad_r)) return false;
+            err_out = (float)((double)err / sum_st);
+            if (a.tol > 0.0f && !(err <= tol_abs_f)) info |= TAOT_INFO_SINKHORN_CAP;
+            break;
+        }
+        if (NW > 1) {
             for (int j = tid; j < Cn; j += NT) {
                 float c = 0.0f;
 #pragma unroll
-                for (int w = 0; w < NW; ++w) c += sh_part[w * RMAX + j];
-                if (!(c > kSumLo && c < kSumHi)) sh_flags[par] = 1;
-                const float vn = sh_dd[j] / c;
-                if (!(vn > kDriftLo && vn < kDriftHi)) sh_flags[par + 1] = 1;
-                sh_vs[j] = vn;
+                for (int w = 0; w < NW; ++w) c += sm.part[w * RMAX + j];
+                const float vn = sm.dd[j] * __frcp_rn(c);
+                if ((__float_as_uint(vn) - lo_bits) > span_bits) sm.flags[par] = 1;
+                sm.vs[j] = vn;
             }
             __syncthreads();
-            if (sh_flags[par]) { hand_back = true; break; }
-            drift = sh_flags[par + 1] != 0;
+            odd = sm.flags[par] != 0;
 #pragma unroll
-            for (int g = 0; g < CG; ++g) vreg[g] = col_ok[g] ? sh_vs[lane + 32 * g] : 1.0f;
+            for (int g = 0; g < CG; ++g) vnew[g] = col_ok[g] ? sm.vs[lane + 32 * g] : 1.0f;
         }
+        if (odd) {
+            // rare: either u~, v~ merely drifted (fold them into the potentials) or a sum left the range in which
+            // fp32 products are trustworthy (hand the problem back).  Decide from the sums themselves.
+            bool bad = row_ok && !(r > kSumLo && r < kSumHi);
+            if (NW == 1) {
+#pragma unroll
+                for (int g = 0; g < CG; ++g) bad |= col_ok[g] && !(cp[g] > kSumLo && cp[g] < kSumHi);
+                bad = __any_sync(kFull, bad);
+            } else {
+                for (int j = tid; j < Cn; j += NT) {
+                    float c = 0.0f;
+#pragma unroll
+                    for (int w = 0; w < NW; ++w) c += sm.part[w * RMAX + j];
+                    bad |= !(c > kSumLo && c < kSumHi);
+                }
+                bad = __syncthreads_or(bad);
+            }
+            if (bad) return false;
+        }
+        // ---- commit iteration t+1
         uo = un;
+#pragma unroll
+        for (int g = 0; g < CG; ++g) vreg[g] = vnew[g];
         ++t;
-        if (drift) {
+        until_check = until_check == 1 ? a.check_every : until_check - 1;
+        if (odd) {
             // fold u~, v~ into the fp64 potentials and rebuild the tile around them
-            if (row_ok && lane < RPW) sh_alpha[rowl] += log((double)uo);
+            if (row_owner) sm.alpha[rowl] += log((double)uo);
             if (NW == 1) {
 #pragma unroll
                 for (int g = 0; g < CG; ++g)
-                    if (col_ok[g]) sh_beta[lane + 32 * g] += log((double)vreg[g]);
+                    if (col_ok[g]) sm.beta[lane + 32 * g] += log((double)vreg[g]);
                 __syncwarp();
             } else {
-                for (int j = tid; j < Cn; j += NT) sh_beta[j] += log((double)sh_vs[j]);
+                for (int j = tid; j < Cn; j += NT) sm.beta[j] += log((double)sm.vs[j]);
                 __syncthreads();
             }
             uo = 1.0f;
@@ -275,18 +228,13 @@ sinkhorn_tile_kernel(SinkArgs a)
         }
     }
 
-    if (hand_back) {
-        if (tid == 0) a.iters[b] = kHandBack;
-        return;
-    }
-
     // ---- T = diag(u) M diag(v) from the total potentials, then the column cap
     if (NW > 1) __syncthreads();
-    if (row_ok && lane < RPW) sh_alpha[rowl] += log((double)uo);
-    if (warp == 0 || NW == 1) {
+    if (row_owner) sm.alpha[rowl] += log((double)uo);
+    if (warp == 0) {
 #pragma unroll
         for (int g = 0; g < CG; ++g)
-            if (col_ok[g]) sh_beta[lane + 32 * g] += log((double)vreg[g]);     // every warp holds the same v~
+            if (col_ok[g]) sm.beta[lane + 32 * g] += log((double)vreg[g]);     // every warp holds the same v~
     }
     __syncthreads();
     build_tile();
@@ -305,17 +253,17 @@ sinkhorn_tile_kernel(SinkArgs a)
             fg[g] = col_ok[g] ? (float)fmin(1.0, (double)ddg[g] / ((double)cs[g] + (double)a.eps0)) : 0.0f;
     } else {
 #pragma unroll
-        for (int g = 0; g < CG; ++g) sh_part[warp * RMAX + lane + 32 * g] = cs[g];
+        for (int g = 0; g < CG; ++g) sm.part[warp * RMAX + lane + 32 * g] = cs[g];
         __syncthreads();
         for (int j = tid; j < Cn; j += NT) {
             double c = 0.0;
 #pragma unroll
-            for (int w = 0; w < NW; ++w) c += (double)sh_part[w * RMAX + j];
-            sh_vs[j] = (float)fmin(1.0, (double)sh_dd[j] / (c + (double)a.eps0));
+            for (int w = 0; w < NW; ++w) c += (double)sm.part[w * RMAX + j];
+            sm.vs[j] = (float)fmin(1.0, (double)sm.dd[j] / (c + (double)a.eps0));
         }
         __syncthreads();
 #pragma unroll
-        for (int g = 0; g < CG; ++g) fg[g] = col_ok[g] ? sh_vs[lane + 32 * g] : 0.0f;
+        for (int g = 0; g < CG; ++g) fg[g] = col_ok[g] ? sm.vs[lane + 32 * g] : 0.0f;
     }
     // zero the R x R block, then scatter the hot x cold entries
     for (int q = tid; q < R * R; q += NT) out[q] = 0.0f;
@@ -325,13 +273,13 @@ sinkhorn_tile_kernel(SinkArgs a)
     for (int aa = 0; aa < RPW; ++aa) {
         const int row = row0 + aa;
         if (row >= Hn) continue;
-        float* orow = out + (int64_t)sh_hot[row] * R;
+        float* orow = out + (int64_t)sm.hot[row] * R;
 #pragma unroll
         for (int g = 0; g < CG; ++g) {
             if (!col_ok[g]) continue;
             const float val = K[aa][g] * fg[g];
             if (!isfinite(val)) nonfinite = 1;
-            orow[sh_cold[lane + 32 * g]] = val;
+            orow[sm.cold[lane + 32 * g]] = val;
         }
     }
     nonfinite = __syncthreads_or(nonfinite);
@@ -341,6 +289,98 @@ sinkhorn_tile_kernel(SinkArgs a)
         a.row_err[b] = err_out;
         if (info) atomicOr(a.info + b, info);
     }
+    return true;
+}
+
+// RP0 < RP1 < RP2: rows-per-warp variants; the smallest that holds the problem's supply ranks runs.
+template <int NW, int CG, int RP0, int RP1, int RP2>
+__global__ void __launch_bounds__(NW * 32)
+sinkhorn_tile_kernel(SinkArgs a)
+{
+    constexpr int NT = NW * 32;
+    __shared__ TileSmem<NW, CG> sm;
+    const int R = a.R, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t b = blockIdx.x;
+
+    // ---- supply scaling gamma = min(1, sum d / max(sum s, eps0)), compaction of supply / demand ranks
+    {
+        double ps = 0.0, pd = 0.0;
+        for (int i = tid; i < R; i += NT) {
+            const float sv = a.s[b * R + i], dv = a.d[b * R + i];
+            ps += sv > 0.0f ? (double)sv : 0.0;
+            pd += dv > 0.0f ? (double)dv : 0.0;
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            ps += __shfl_xor_sync(kFull, ps, o);
+            pd += __shfl_xor_sync(kFull, pd, o);
+        }
+        if (lane == 0) { sm.red[warp] = ps; sm.red[32 + warp] = pd; }
+        if (tid < 4) sm.flags[tid] = 0;
+        __syncthreads();
+        if (tid == 0) {
+            double S = 0.0, D = 0.0;
+            for (int w = 0; w < NW; ++w) { S += sm.red[w]; D += sm.red[32 + w]; }
+            sm.sum[0] = S; sm.sum[1] = D;
+        }
+        __syncthreads();
+    }
+    const double sum_s = sm.sum[0], sum_d = sm.sum[1];
+    const double gamma = fmin(1.0, sum_d / fmax(sum_s, (double)a.eps0));
+    for (int i = tid; i < R; i += NT) {
+        const float sv = a.s[b * R + i], dv = a.d[b * R + i];
+        sm.sv[i] = sv > 0.0f ? (float)(gamma * (double)sv) : 0.0f;
+        sm.dv[i] = dv > 0.0f ? dv : 0.0f;
+    }
+    __syncthreads();
+    const int Hn = compact_positive(sm.sv, R, sm.hot, sm.hpos, sm.wcnt);
+    const int Cn = compact_positive(sm.dv, R, sm.cold, sm.cpos, sm.wcnt);
+    if (Hn > NW * RP2) {                     // does not fit any tile: the other kernel takes it
+        if (tid == 0) a.iters[b] = kHandBack;
+        return;
+    }
+    for (int i = tid; i < Hn; i += NT) sm.st[i] = sm.sv[sm.hot[i]];
+    for (int j = tid; j < Cn; j += NT) sm.dd[j] = sm.dv[sm.cold[j]];
+    __syncthreads();
+
+    int info = 0;
+    if (sum_s > sum_d) info |= TAOT_INFO_SUPPLY_SCALED;
+    float* out = a.plan + b * (int64_t)R * R;
+    if (Hn == 0 || Cn == 0) {
+        for (int q = tid; q < R * R; q += NT) out[q] = 0.0f;
+        if (tid == 0) {
+            a.iters[b] = 0;
+            a.row_err[b] = 0.0f;
+            if (info) atomicOr(a.info + b, info);
+        }
+        return;
+    }
+    double sum_st = 0.0;
+    for (int i = 0; i < Hn; ++i) sum_st += (double)sm.st[i];          // same order in every thread
+
+    // ---- iteration 1 in the log domain (v = 1 on every rank): phi = log s~ - LSE_j(-C_ij/eps) over all j,
+    //      psi_j = log d_j - LSE_i(phi_i - C_ij/eps)
+    for (int i = tid; i < Hn; i += NT) sm.phin[i] = log((double)sm.st[i]) - a.rowlse0[sm.hot[i]];
+    __syncthreads();
+    for (int j = tid; j < Cn; j += NT) {
+        const int cj = sm.cold[j];
+        double mx = -INFINITY;
+        for (int i = 0; i < Hn; ++i) {
+            const double x = sm.phin[i] - (double)a.C[(int64_t)sm.hot[i] * R + cj] * a.inv_eps;
+            mx = x > mx ? x : mx;
+        }
+        double acc = 0.0;
+        for (int i = 0; i < Hn; ++i)
+            acc += exp(sm.phin[i] - (double)a.C[(int64_t)sm.hot[i] * R + cj] * a.inv_eps - mx);
+        sm.beta[j] = log((double)sm.dd[j]) - (mx + log(acc));
+    }
+    for (int i = tid; i < Hn; i += NT) sm.alpha[i] = sm.phin[i];
+    __syncthreads();
+
+    bool done;
+    if (Hn <= NW * RP0) done = tile_solve<NW, RP0, CG>(a, sm, Hn, Cn, sum_st, info, out, b);
+    else if (Hn <= NW * RP1) done = tile_solve<NW, RP1, CG>(a, sm, Hn, Cn, sum_st, info, out, b);
+    else done = tile_solve<NW, RP2, CG>(a, sm, Hn, Cn, sum_st, info, out, b);
+    if (!done && tid == 0) a.iters[b] = kHandBack;
 }
 
 }  // namespace
@@ -348,10 +388,10 @@ sinkhorn_tile_kernel(SinkArgs a)
 int taot_launch_sinkhorn_tile(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st)
 {
     const int R = h->p.R;
-    if (R <= 32) sinkhorn_tile_kernel<1, 16, 1><<<B, 32, 0, st>>>(a);
-    else if (R <= 64) sinkhorn_tile_kernel<1, 32, 2><<<B, 32, 0, st>>>(a);
-    else if (R <= 128) sinkhorn_tile_kernel<4, 16, 4><<<B, 128, 0, st>>>(a);
-    else sinkhorn_tile_kernel<16, 8, 8><<<B, 512, 0, st>>>(a);
+    if (R <= 32) sinkhorn_tile_kernel<1, 1, 4, 8, 16><<<B, 32, 0, st>>>(a);
+    else if (R <= 64) sinkhorn_tile_kernel<1, 2, 8, 16, 32><<<B, 32, 0, st>>>(a);
+    else if (R <= 128) sinkhorn_tile_kernel<4, 4, 4, 8, 16><<<B, 128, 0, st>>>(a);
+    else sinkhorn_tile_kernel<16, 8, 2, 4, 8><<<B, 512, 0, st>>>(a);
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
 }
