@@ -184,7 +184,7 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
                 for (int r = 0; r < R; ++r) {
                     const float b3 = (r == host) ? 1.0f : B[(size_t)r * R + host];
                     for (int t = 0; t < Tn; ++t)
-                        if (vals[t] == b3) tiermask[((size_t)host * Tn + t) * W + (r >> 5)] |= 1u << (r & 31);
+                        if (vals[t] == b3) tiermask[((size_t)t * W + (r >> 5)) * R + host] |= 1u << (r & 31);
                 }
         }
     }

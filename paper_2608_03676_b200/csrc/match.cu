@@ -35,7 +35,7 @@ struct MatchArgs {
     const float* B;              // [R,R]
     const int32_t* rank_off;     // [R+1]
     const int32_t* rank_list;    // [E]
-    const uint32_t* tiermask;    // [R hosts][ntiers][W] bit r: B3[r][host] == tierval[t]
+    const uint32_t* tiermask;    // [ntiers][W][R hosts] bit r of word w: B3[32w + r][host] == tierval[t]
     const float* tierval;        // [ntiers] descending
     int32_t* slot_expert;        // [L,R,K]
     int32_t* slot_tokens;        // [L,R,K]
@@ -48,6 +48,7 @@ struct MatchArgs {
     float eps0, price_step;
     int32_t auction_max_rounds;
     int32_t nrem_in_smem;
+    int32_t tm_in_smem;
 };
 
 __device__ __forceinline__ uint32_t ordered_bits(float f)
@@ -67,22 +68,46 @@ __device__ __forceinline__ u64 warp_max_u64(u64 k)
 
 constexpr int kMaxW = 8;          // words of a rank bit set: R <= 256
 
+// Lowest set bit over kMaxW words (bit index = 32*w + bit), or -1: independent ANDs and a select tree
+// instead of a word-by-word scan, so that a lone warp is not held up by a long dependency chain.
+__device__ __forceinline__ int first_hit(const uint32_t (&cand)[8], const uint32_t* lv, int stride, int W)
+{
+    uint32_t h[8];
+#pragma unroll
+    for (int w = 0; w < 8; ++w) h[w] = (w < W) ? (cand[w] & lv[w * stride]) : 0u;
+    // pairwise: keep the lower word if it is nonzero
+    const uint32_t a0 = h[0] ? h[0] : h[1]; const int i0 = h[0] ? 0 : 1;
+    const uint32_t a1 = h[2] ? h[2] : h[3]; const int i1 = h[2] ? 2 : 3;
+    const uint32_t a2 = h[4] ? h[4] : h[5]; const int i2 = h[4] ? 4 : 5;
+    const uint32_t a3 = h[6] ? h[6] : h[7]; const int i3 = h[6] ? 6 : 7;
+    const uint32_t b0 = a0 ? a0 : a1; const int j0 = a0 ? i0 : i1;
+    const uint32_t b1 = a2 ? a2 : a3; const int j1 = a2 ? i2 : i3;
+    const uint32_t c = b0 ? b0 : b1; const int k = b0 ? j0 : j1;
+    return c ? (k << 5) + __ffs(c) - 1 : -1;
+}
+
 // Arbitration "best bidder per target" for one warp's worth of bids.  Many bidders often pick the
 // same target (all slots of a tier chase the cheapest rank), so the lanes that bid for the same
 // target first agree on their best key with warp-wide reductions and only one of them touches the
 // shared-memory arbiter.  key = (score bits << 32) | inverted bidder index; valid bids have key != 0.
 __device__ __forceinline__ void arbitrate(u64* arb, int target, u64 key)
 {
-    const unsigned active = __ballot_sync(0xffffffffu, key != 0);
-    if (key == 0) return;
-    const unsigned group = __match_any_sync(active, target);
+    unsigned todo = __ballot_sync(0xffffffffu, key != 0);
     const uint32_t hi = (uint32_t)(key >> 32), lo = (uint32_t)key;
-    const uint32_t hi_max = __reduce_max_sync(group, hi);
-    const uint32_t lo_max = __reduce_max_sync(group, hi == hi_max ? lo : 0u);
-    if ((__ffs(group) - 1) == (int)(threadIdx.x & 31)) atomicMax(arb + target, ((u64)hi_max << 32) | (u64)lo_max);
+    const int lane = threadIdx.x & 31;
+    while (todo) {                                   // one pass per distinct target among this warp's bids
+        const int leader = __ffs(todo) - 1;
+        const int tgt = __shfl_sync(0xffffffffu, target, leader);
+        const bool mine = key != 0 && target == tgt;
+        const unsigned group = __ballot_sync(0xffffffffu, mine);
+        const uint32_t hi_max = __reduce_max_sync(0xffffffffu, mine ? hi : 0u);
+        const uint32_t lo_max = __reduce_max_sync(0xffffffffu, (mine && hi == hi_max) ? lo : 0u);
+        if (lane == leader) atomicMax(arb + tgt, ((u64)hi_max << 32) | (u64)lo_max);
+        todo &= ~group;
+    }
 }
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 match_kernel(MatchArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -92,8 +117,8 @@ match_kernel(MatchArgs a)
 
     // ---- carve shared memory
     u64* arb_e = reinterpret_cast<u64*>(smem_raw);            // [E]  Phase 2 arbitration per expert
-    u64* arb_r = arb_e + E;                                    // [R]  Phase 3 arbitration per rank
-    int32_t* spill = reinterpret_cast<int32_t*>(arb_r + R);    // [E]
+    u64* arb_r = arb_e + E;                                    // [2][R]  Phase 3 arbitration per rank, ping-pong by round
+    int32_t* spill = reinterpret_cast<int32_t*>(arb_r + 2 * R); // [E]
     int32_t* hot0 = spill + E;                                 // [E]  experts that spill at the start of Phase 2
     int32_t* hot_home = hot0 + E;                              // [E]  their home ranks
     int32_t* dcol = hot_home + E;                              // [E]  expert -> column of nrem, or -1
@@ -105,12 +130,16 @@ match_kernel(MatchArgs a)
     int32_t* slot_e = wins + R;                                // [S]
     int32_t* slot_a0 = slot_e + S;                             // [S]  planned tokens (Phase 2 result)
     int32_t* slot_a = slot_a0 + S;                             // [S]  still to collect (Phase 3)
-    uint32_t* avail = reinterpret_cast<uint32_t*>(slot_a + S); // [dmax][W]  ranks still holding tokens of the expert
-    uint32_t* lvl = avail + a.dmax * W;                        // [S+1][W]   ranks by win count
-    int32_t* wstart = reinterpret_cast<int32_t*>(lvl + (S + 1) * W);   // [S][ntiers] resume level of each slot and tier
-    int32_t* nrem_s = wstart + S * (a.ntiers > 0 ? a.ntiers : 1);      // [dmax*R] if it fits
+    uint32_t* avail = reinterpret_cast<uint32_t*>(slot_a + S); // [W][dmax]  ranks still holding tokens of the expert (word-major: no bank conflicts across slots)
+    uint32_t* lvl = avail + a.dmax * W;                        // [W][S+1]   ranks by win count (word-major)
+    uint32_t* tm_s = lvl + (S + 1) * W;                                // [ntiers][W][S] tier masks by slot, if they fit
+    int32_t* nrem_s = reinterpret_cast<int32_t*>(tm_s + (a.tm_in_smem ? a.ntiers * W * S : 0));   // [dmax*R] if it fits
     __shared__ long long s_tot;
     __shared__ int s_cnt, s_any;
+#ifdef TAOT_DEBUG_CLOCKS
+    __shared__ long long s_dbg[5];
+    if (threadIdx.x < 5) s_dbg[threadIdx.x] = 0;
+#endif
 
     const int32_t* n = a.n + l * (int64_t)R * E;
     const int32_t* el = a.expert_load + l * E;
@@ -135,6 +164,7 @@ match_kernel(MatchArgs a)
         spare[r] = (int32_t)(mean > lr ? mean - lr : 0);
         wins[r] = 0;
         arb_r[r] = 0;
+        arb_r[R + r] = 0;
     }
     // ---- spill by cumulative-excess differencing: position of e in its rank's (load, index) order
     for (int e = tid; e < E; e += NT) {
@@ -175,9 +205,6 @@ match_kernel(MatchArgs a)
     __syncthreads();
 
     // =========================================================== Phase 2
-#ifdef TAOT_DEBUG_CLOCKS
-    const long long clk0 = clock64();
-#endif
     int rounds2 = 0;
     for (int kappa = 0; kappa < K; ++kappa) {
         for (int r = tid; r < R; r += NT) matched[r] = 0;
@@ -235,9 +262,6 @@ match_kernel(MatchArgs a)
         __syncthreads();
     }
 
-#ifdef TAOT_DEBUG_CLOCKS
-    const long long clk1 = clock64();
-#endif
     // =========================================================== Phase 3
     // compact the experts that sit in some slot; keep their per-rank remaining counts transposed [col][r]
     for (int e = tid; e < E; e += NT) dcol[e] = -1;
@@ -252,7 +276,6 @@ match_kernel(MatchArgs a)
         if (dcol[e] == -2) dcol[e] = atomicAdd(&s_cnt, 1);
     for (int i = tid; i < a.dmax * W; i += NT) avail[i] = 0u;
     for (int i = tid; i < (S + 1) * W; i += NT) lvl[i] = 0u;
-    for (int i = tid; i < S * a.ntiers; i += NT) wstart[i] = 0;
     __syncthreads();
     const int D = s_cnt;
     for (int e = 0; e < E; ++e) {
@@ -261,111 +284,190 @@ match_kernel(MatchArgs a)
         for (int r = tid; r < R; r += NT) {
             const int32_t v = n[(int64_t)r * E + e];
             nrem[col * R + r] = v;
-            if (v > 0) atomicOr(avail + col * W + (r >> 5), 1u << (r & 31));
+            if (v > 0) atomicOr(avail + (r >> 5) * a.dmax + col, 1u << (r & 31));
         }
     }
-    for (int r = tid; r < R; r += NT) atomicOr(lvl + (r >> 5), 1u << (r & 31));      // every rank starts with 0 wins
+    for (int r = tid; r < R; r += NT) atomicOr(lvl + (r >> 5) * (S + 1), 1u << (r & 31));      // every rank starts with 0 wins
     int32_t* Xl = a.X + l * (int64_t)R * S;
     for (int64_t q = tid; q < (int64_t)R * S; q += NT) Xl[q] = 0;
     __syncthreads();
 
     int rounds3 = 0;
-#ifdef TAOT_DEBUG_CLOCKS
-    long long dbg_bid = 0, dbg_wait = 0, dbg_serve = 0;
-#endif
     const long long cap = (long long)R * S + S;
-    const bool tiered = a.ntiers > 0;
-    for (;;) {
-        if (a.auction_max_rounds > 0 && rounds3 >= a.auction_max_rounds) break;
-        if (rounds3 >= cap || D == 0) break;
-        if (tid == 0) s_any = 0;
-        __syncthreads();
+    const bool tiered = a.ntiers > 0 && S <= NT;
+    if (tiered && D > 0) {
+        // ---- bit-set auction: thread s is slot s for the whole auction and keeps the slot's state in registers
+        const int s = tid;
+        bool live = s < S && slot_e[s] >= 0 && slot_a[s] > 0;
+        const int e = live ? slot_e[s] : 0;
+        const int col = live ? dcol[e] : 0;
+        const int host = s < S ? s / K : 0;
+        int32_t A = live ? slot_a[s] : 0;
+        int32_t wst[TAOT_MAX_TIERS];             // per tier: lowest win count seen among its candidates (never decreases)
+#pragma unroll
+        for (int t = 0; t < TAOT_MAX_TIERS; ++t) wst[t] = 0;
+        float tval[TAOT_MAX_TIERS];
+#pragma unroll
+        for (int t = 0; t < TAOT_MAX_TIERS; ++t) tval[t] = t < a.ntiers ? a.tierval[t] : 0.0f;
+        const uint32_t* av = avail + col;                          // word w at av[w * dmax]
+        // this slot's tier masks: tier t, word w at tm[(t * W + w) * tms]; a shared-memory copy when it fits
+        const uint32_t* tm = a.tiermask + host;
+        int tms = R;
+        if (a.tm_in_smem) {
+            for (int q = tid; q < a.ntiers * W * S; q += NT) {
+                const int ss = q % S, tw = q / S;
+                tm_s[q] = a.tiermask[(int64_t)tw * R + ss / K];
+            }
+            __syncthreads();
+            tm = tm_s + (s < S ? s : 0);
+            tms = S;
+        }
+        const int LS = S + 1;                                      // lvl: word w of level wl at lvl[w * LS + wl]
+        // a tier whose ranks (for this slot's host) all sit in one 32-bit word is handled with that word alone
+        int twrd[TAOT_MAX_TIERS];
+        uint32_t tmw[TAOT_MAX_TIERS];
+#pragma unroll
+        for (int t = 0; t < TAOT_MAX_TIERS; ++t) {
+            twrd[t] = -1; tmw[t] = 0u;
+            if (t < a.ntiers) {
+                int nz = 0, wd = 0;
+                uint32_t val = 0u;
+                for (int w = 0; w < W; ++w) {
+                    const uint32_t mk = tm[(t * W + w) * tms];
+                    if (mk) { ++nz; wd = w; val = mk; }
+                }
+                if (nz <= 1) { twrd[t] = wd; tmw[t] = val; }
+            }
+        }
+        int prev_r = -1;                         // rank whose arbiter entry this slot won last round
 #ifdef TAOT_DEBUG_CLOCKS
-        const long long ca = clock64();
+        long long dbg[5] = {0, 0, 0, 0, 0};
+        int dbg_levels = 0, dbg_bits = 0, dbg_tiers = 0; (void)dbg_levels; (void)dbg_bits; (void)dbg_tiers;
 #endif
-        // Step 1: every unfinished slot bids for the source rank with the best bonus minus price
-        if (tiered) {
-            for (int sb = 0; sb < S; sb += NT) {
-                const int s = sb + tid;
-                const int e = s < S ? slot_e[s] : -1;
-                const bool live = e >= 0 && slot_a[s] > 0;
-                const int host = s / K;
-                const uint32_t* av = avail + (live ? dcol[e] : 0) * W;
-                const uint32_t* tm = a.tiermask + (int64_t)(live ? host : 0) * a.ntiers * W;
-                u64 key = 0;
-                for (int t = 0; live && t < a.ntiers; ++t) {
-                    uint32_t cand[kMaxW];
-                    uint32_t any = 0;
-                    int pc = 0;
+        for (;;) {
+            if (a.auction_max_rounds > 0 && rounds3 >= a.auction_max_rounds) break;
+            if (rounds3 >= cap) break;
+            u64* arb = arb_r + (rounds3 & 1) * R;
+            // Step 1: bid for the source rank with the best bonus minus price
+#ifdef TAOT_DEBUG_CLOCKS
+            const long long c0 = clock64();
+#endif
+            u64 key = 0;
+            if (live) {
 #pragma unroll
-                    for (int w = 0; w < kMaxW; ++w) {
-                        cand[w] = (w < W) ? (tm[t * W + w] & av[w]) : 0u;
-                        any |= cand[w];
-                        pc += __popc(cand[w]);
-                    }
-                    if (!any) continue;
-                    const float vt = a.tierval[t];
-                    // the lowest win count among this tier's candidates never decreases: resume from the last one
-                    int wl = wstart[s * a.ntiers + t];
+                for (int t = 0; t < TAOT_MAX_TIERS; ++t) {
+                    if (t >= a.ntiers) break;
+                    const float vt = tval[t];
+                    int wl = wst[t];
+                    // best score this tier can still offer: skip it if a better tier already beats that
                     const float ub = __fsub_rn(vt, __fmul_rn(a.price_step, (float)wl));
-                    if (key != 0 && (u64)ordered_bits(ub) < (key >> 32)) continue;      // cannot beat a better tier
-                    if (pc <= 8) {
-                        // few candidates: score each one
-                        int wmin = S + 1;
-#pragma unroll
-                        for (int w = 0; w < kMaxW; ++w) {
-                            uint32_t bits = cand[w];
-                            while (bits) {
-                                const int r = (w << 5) + __ffs(bits) - 1;
-                                bits &= bits - 1;
-                                const int wr = wins[r];
-                                wmin = wr < wmin ? wr : wmin;
-                                const float sc = __fsub_rn(vt, __fmul_rn(a.price_step, (float)wr));
-                                const u64 k64 = ((u64)ordered_bits(sc) << 32) | (u64)(0xFFFFFFFFu - (uint32_t)r);
-                                key = k64 > key ? k64 : key;
-                            }
-                        }
-                        wstart[s * a.ntiers + t] = wmin;
-                        continue;
-                    }
+                    if (key != 0 && (u64)ordered_bits(ub) < (key >> 32)) continue;
                     int r_best = -1;
-                    for (; wl <= S; ++wl) {
-                        const uint32_t* lv = lvl + wl * W;
+                    float sc;
+                    if (twrd[t] >= 0) {
+                        // the tier's ranks (for this host) sit in one 32-bit word: node or rail-group tiers
+                        const int wd = twrd[t];
+                        const uint32_t c1 = tmw[t] & av[wd * a.dmax];
+                        if (!c1) continue;
+                        const uint32_t* lv = lvl + wd * LS;
+                        for (; wl <= S; ++wl) {
+                            const uint32_t hit = c1 & lv[wl];
+                            if (hit) { r_best = (wd << 5) + __ffs(hit) - 1; break; }
+                        }
+                        if (r_best < 0) continue;
+                        sc = __fsub_rn(vt, __fmul_rn(a.price_step, (float)wl));
+                        // higher win counts whose score rounds to the same float compete on rank index alone
+                        for (int w2 = wl + 1; w2 <= S; ++w2) {
+                            if (__fsub_rn(vt, __fmul_rn(a.price_step, (float)w2)) != sc) break;
+                            const uint32_t hit = c1 & lv[w2];
+                            if (hit) { const int r2 = (wd << 5) + __ffs(hit) - 1; r_best = r2 < r_best ? r2 : r_best; }
+                        }
+                    } else {
+                        uint32_t cand[kMaxW];
+                        uint32_t any = 0;
 #pragma unroll
                         for (int w = 0; w < kMaxW; ++w) {
-                            if (w < W && r_best < 0) {
-                                const uint32_t hit = cand[w] & lv[w];
-                                if (hit) r_best = (w << 5) + __ffs(hit) - 1;
-                            }
+                            cand[w] = (w < W) ? (tm[(t * W + w) * tms] & av[w * a.dmax]) : 0u;
+                            any |= cand[w];
                         }
-                        if (r_best >= 0) break;
-                    }
-                    if (r_best < 0) continue;
-                    wstart[s * a.ntiers + t] = wl;
-                    const float sc = __fsub_rn(vt, __fmul_rn(a.price_step, (float)wl));
-                    // higher win counts whose score rounds to the same float compete on rank index alone
-                    for (int w2 = wl + 1; w2 <= S; ++w2) {
-                        if (__fsub_rn(vt, __fmul_rn(a.price_step, (float)w2)) != sc) break;
-                        const uint32_t* lv = lvl + w2 * W;
-                        int r2 = -1;
-#pragma unroll
-                        for (int w = 0; w < kMaxW; ++w) {
-                            if (w < W && r2 < 0) {
-                                const uint32_t hit = cand[w] & lv[w];
-                                if (hit) r2 = (w << 5) + __ffs(hit) - 1;
-                            }
+                        if (!any) continue;
+                        for (; wl <= S; ++wl) {
+                            r_best = first_hit(cand, lvl + wl, LS, W);
+                            if (r_best >= 0) break;
                         }
-                        if (r2 >= 0 && r2 < r_best) r_best = r2;
+                        if (r_best < 0) continue;
+                        sc = __fsub_rn(vt, __fmul_rn(a.price_step, (float)wl));
+                        for (int w2 = wl + 1; w2 <= S; ++w2) {
+                            if (__fsub_rn(vt, __fmul_rn(a.price_step, (float)w2)) != sc) break;
+                            const int r2 = first_hit(cand, lvl + w2, LS, W);
+                            if (r2 >= 0 && r2 < r_best) r_best = r2;
+                        }
                     }
+                    wst[t] = wl;
                     const u64 k64 = ((u64)ordered_bits(sc) << 32) | (u64)(0xFFFFFFFFu - (uint32_t)r_best);
                     key = k64 > key ? k64 : key;
                 }
-                // Step 2: the rank keeps its best bidder (ties: lowest slot)
-                const int rsel = (int)(0xFFFFFFFFu - (uint32_t)key);
-                if (key != 0) s_any = 1;
-                arbitrate(arb_r, rsel, key == 0 ? 0ull : ((key & 0xFFFFFFFF00000000ull) | (u64)(0xFFFFFFFFu - (uint32_t)s)));
             }
-        } else {
+            // Step 2: the rank keeps its best bidder (ties: lowest slot)
+#ifdef TAOT_DEBUG_CLOCKS
+            const long long c1 = clock64();
+#endif
+            const int rsel = (int)(0xFFFFFFFFu - (uint32_t)key);
+            arbitrate(arb, rsel, key == 0 ? 0ull : ((key & 0xFFFFFFFF00000000ull) | (u64)(0xFFFFFFFFu - (uint32_t)s)));
+#ifdef TAOT_DEBUG_CLOCKS
+            const long long c2 = clock64();
+#endif
+            if (!__syncthreads_or(key != 0)) break;
+#ifdef TAOT_DEBUG_CLOCKS
+            const long long c3 = clock64();
+#endif
+            if (prev_r >= 0) { arb_r[((rounds3 & 1) ^ 1) * R + prev_r] = 0; prev_r = -1; }
+            // Steps 3-4: the winning slot of each rank collects x = min(n, A); holdings, plan and price follow
+            if (key != 0 && (uint32_t)arb[rsel] == 0xFFFFFFFFu - (uint32_t)s) {
+                int32_t* cell = nrem + col * R + rsel;
+                const int32_t have = *cell;
+                const int32_t x = have < A ? have : A;
+                Xl[(int64_t)rsel * S + s] = x;             // a (rank, slot) pair is served at most once
+                *cell = have - x;
+                A -= x;
+                const uint32_t bit = 1u << (rsel & 31);
+                if (have - x == 0) atomicAnd(avail + (rsel >> 5) * a.dmax + col, ~bit);
+                if (x > 0) {
+                    const int w0 = wins[rsel];
+                    wins[rsel] = w0 + 1;
+                    atomicAnd(lvl + (rsel >> 5) * LS + w0, ~bit);
+                    atomicOr(lvl + (rsel >> 5) * LS + w0 + 1, bit);
+                }
+                prev_r = rsel;
+                if (A <= 0) live = false;
+            }
+            ++rounds3;
+#ifdef TAOT_DEBUG_CLOCKS
+            const long long c4 = clock64();
+#endif
+            __syncthreads();
+#ifdef TAOT_DEBUG_CLOCKS
+            const long long c5 = clock64();
+            dbg[0] += c1 - c0; dbg[1] += c2 - c1; dbg[2] += c3 - c2; dbg[3] += c4 - c3;
+#endif
+        }
+#ifdef TAOT_DEBUG_CLOCKS
+        for (int i = 0; i < 5; ++i) atomicMax(reinterpret_cast<u64*>(&s_dbg[i]), (u64)dbg[i]);
+        __syncthreads();
+        if (l == 0 && a.rounds) {   // per-thread totals into the tail of X of the LAST layer (debug only)
+            int32_t* dump = a.X + (int64_t)(gridDim.x - 1) * R * S;
+            dump[tid] = (int)(dbg[0] / 1000); dump[NT + tid] = dbg_levels; dump[2 * NT + tid] = dbg_bits; dump[3*NT + tid] = dbg_tiers;
+        }
+#endif
+        if (s < S) slot_a[s] = A;
+        __syncthreads();
+    } else {
+        for (;;) {
+            if (a.auction_max_rounds > 0 && rounds3 >= a.auction_max_rounds) break;
+            if (rounds3 >= cap || D == 0) break;
+            if (tid == 0) s_any = 0;
+            __syncthreads();
+            // Step 1: every unfinished slot bids for the source rank with the best bonus minus price (dense scan)
             for (int s = warp; s < S; s += NW) {
                 const int e = slot_e[s];
                 if (e < 0 || slot_a[s] <= 0) continue;
@@ -383,47 +485,31 @@ match_kernel(MatchArgs a)
                 key = warp_max_u64(key);
                 if (lane == 0 && key != 0) {
                     const int r = (int)(0xFFFFFFFFu - (uint32_t)key);
+                    // Step 2: the rank keeps its best bidder (ties: lowest slot)
                     atomicMax(arb_r + r, (key & 0xFFFFFFFF00000000ull) | (u64)(0xFFFFFFFFu - (uint32_t)s));
                     s_any = 1;
                 }
             }
-        }
-#ifdef TAOT_DEBUG_CLOCKS
-        const long long cb = clock64();
-#endif
-        __syncthreads();
-#ifdef TAOT_DEBUG_CLOCKS
-        const long long cc_ = clock64();
-#endif
-        if (!s_any) break;
-        // Steps 3-4: allocate, update holdings, plan and price
-        for (int r = tid; r < R; r += NT) {
-            const u64 k64 = arb_r[r];
-            if (k64 == 0) continue;
-            arb_r[r] = 0;
-            const int s = (int)(0xFFFFFFFFu - (uint32_t)k64);
-            const int col = dcol[slot_e[s]];
-            int32_t* cell = nrem + col * R + r;
-            const int32_t have = *cell;
-            const int32_t x = have < slot_a[s] ? have : slot_a[s];
-            Xl[(int64_t)r * S + s] = x;          // a (rank, slot) pair is served at most once
-            *cell = have - x;
-            slot_a[s] -= x;
-            const uint32_t bit = 1u << (r & 31);
-            if (have - x == 0) atomicAnd(avail + col * W + (r >> 5), ~bit);
-            if (x > 0) {
-                const int w0 = wins[r];
-                wins[r] = w0 + 1;
-                atomicAnd(lvl + w0 * W + (r >> 5), ~bit);
-                atomicOr(lvl + (w0 + 1) * W + (r >> 5), bit);
+            __syncthreads();
+            if (!s_any) break;
+            // Steps 3-4: allocate, update holdings, plan and price
+            for (int r = tid; r < R; r += NT) {
+                const u64 k64 = arb_r[r];
+                if (k64 == 0) continue;
+                arb_r[r] = 0;
+                const int s = (int)(0xFFFFFFFFu - (uint32_t)k64);
+                const int col = dcol[slot_e[s]];
+                int32_t* cell = nrem + col * R + r;
+                const int32_t have = *cell;
+                const int32_t x = have < slot_a[s] ? have : slot_a[s];
+                Xl[(int64_t)r * S + s] = x;          // a (rank, slot) pair is served at most once
+                *cell = have - x;
+                slot_a[s] -= x;
+                if (x > 0) wins[r]++;
             }
+            ++rounds3;
+            __syncthreads();
         }
-        ++rounds3;
-#ifdef TAOT_DEBUG_CLOCKS
-        const long long cd = clock64();
-        dbg_bid += cb - ca; dbg_wait += cc_ - cb; dbg_serve += cd - cc_;
-#endif
-        __syncthreads();
     }
 
     // ---- outputs
@@ -437,7 +523,7 @@ match_kernel(MatchArgs a)
     if (tid == 0) {
         if (a.rounds) { a.rounds[l * 2] = rounds2; a.rounds[l * 2 + 1] = rounds3; }
 #ifdef TAOT_DEBUG_CLOCKS
-        if (a.rounds) { a.rounds[l * 2] = (int)(dbg_bid / 1000) * 100000 + (int)(dbg_wait / 1000); a.rounds[l * 2 + 1] = (int)(dbg_serve / 1000) * 100000 + (int)((clock64() - clk1) / 1000); }
+        if (a.rounds && l < 5) { a.rounds[l * 2] = (int)(s_dbg[l] / 1000); a.rounds[l * 2 + 1] = rounds3; }
 #endif
         if (residual) atomicOr(a.info + l, TAOT_INFO_AUCTION_RESIDUAL);
     }
@@ -446,8 +532,8 @@ match_kernel(MatchArgs a)
 size_t match_smem_fixed(int R, int E, int K, int dmax, int W, int ntiers)
 {
     const size_t S = (size_t)R * K;
-    return sizeof(u64) * (E + R) + sizeof(int32_t) * (4 * (size_t)E + 5 * (size_t)R + 3 * S) +
-           sizeof(uint32_t) * ((size_t)dmax * W + (S + 1) * W) + sizeof(int32_t) * S * (ntiers > 0 ? ntiers : 1);
+    return sizeof(u64) * (E + 2 * (size_t)R) + sizeof(int32_t) * (4 * (size_t)E + 5 * (size_t)R + 3 * S) +
+           sizeof(uint32_t) * ((size_t)dmax * W + (S + 1) * W);
 }
 
 }  // namespace
@@ -471,11 +557,17 @@ int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expe
     a.eps0 = p.eps0; a.price_step = p.price_step; a.auction_max_rounds = p.auction_max_rounds;
     size_t smem = match_smem_fixed(p.R, p.E, p.K, a.dmax, a.W, a.ntiers);
     const size_t nrem_bytes = sizeof(int32_t) * (size_t)a.dmax * p.R;
+    const size_t tm_bytes = sizeof(uint32_t) * (size_t)a.ntiers * a.W * p.R * p.K;
+    a.tm_in_smem = (a.ntiers > 0 && smem + tm_bytes <= 96 * 1024) ? 1 : 0;
+    if (a.tm_in_smem) smem += tm_bytes;
     a.nrem_in_smem = (smem + nrem_bytes <= 200 * 1024) ? 1 : 0;
     if (a.nrem_in_smem) smem += nrem_bytes;
     if (smem > 227 * 1024) return TAOT_ERR_UNSUPPORTED;
     TAOT_CUDA_OK(cudaFuncSetAttribute(match_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    match_kernel<<<p.L, 256, smem, st>>>(a);
+    int need = p.R * p.K > p.R ? p.R * p.K : p.R;
+    int NT = ((need + 31) / 32) * 32;
+    NT = NT < 128 ? 128 : (NT > 1024 ? 1024 : NT);
+    match_kernel<<<p.L, NT, smem, st>>>(a);
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
 }

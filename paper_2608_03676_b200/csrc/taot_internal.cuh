@@ -25,7 +25,7 @@ struct taot_handle_s {
     double* d_rowlse0;       // [R]  LSE_j(-C_ij/eps) over all ranks j: the first u-update with v = 1
     int32_t* d_rank_off;     // [R+1] CSR of experts by home rank
     int32_t* d_rank_list;    // [E]
-    uint32_t* d_tiermask;    // [R hosts][ntiers][W] bit r set iff bonus(r -> host) == tierval[t]; null if ntiers == 0
+    uint32_t* d_tiermask;    // [ntiers][W][R hosts] bit r of word w set iff bonus(32w + r -> host) == tierval[t]; null if ntiers == 0
     float* d_tierval;        // [ntiers] distinct values of the auction bonus matrix, descending
     int32_t ntiers;          // 0: too many distinct values, the auction scans densely
     // derived sizes
