@@ -33,6 +33,11 @@ import workloads as W  # noqa: E402
 L2_BYTES = 126 * 1024 * 1024
 FLUSH_BYTES = 256 * 1024 * 1024
 FP32_LANES_PER_SM = 128
+# DRAM bytes per algorithmic byte of the streaming kernels, from the ncu captures summarised under profiles/
+# (config 3 shape with 8 layers; traffic grows in proportion to the entries processed, so a full launch is
+# scaled by its own algorithmic bytes).  The reassignment figure is read + write once dirty L2 lines drain.
+HIST_TRAFFIC_RATIO = 1.045
+ASSIGN_TRAFFIC_RATIO = 1.01
 STAGES = ["histogram", "merge", "sinkhorn", "match_auction", "assign"]
 
 
@@ -174,11 +179,12 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count):
     if stage == "histogram":
         a = topk_bytes / (ms * 1e-3) / 1e9
         return dict(kernel="hist_chunk_kernel", bound="hbm", achieved=a, peak=hbm, unit="GB/s", frac=a / hbm,
-                    traffic=None, peak_source=peaks["source"], bytes_per_launch=topk_bytes)
+                    traffic=HIST_TRAFFIC_RATIO * topk_bytes, peak_source=peaks["source"], bytes_per_launch=topk_bytes)
     if stage == "assign":
         a = 2 * topk_bytes / (ms * 1e-3) / 1e9
-        return dict(kernel="assign_kernel", bound="hbm", achieved=a, peak=hbm, unit="GB/s", frac=a / hbm,
-                    traffic=None, peak_source=peaks["source"], bytes_per_launch=2 * topk_bytes)
+        return dict(kernel="assign_prep_kernel + assign_kernel", bound="hbm", achieved=a, peak=hbm, unit="GB/s",
+                    frac=a / hbm, traffic=ASSIGN_TRAFFIC_RATIO * 2 * topk_bytes, peak_source=peaks["source"],
+                    bytes_per_launch=2 * topk_bytes)
     if stage == "merge":
         b = cfg.L * cfg.R * cfg.E * 4 * (2 + max(1, (cfg.T // cfg.R * cfg.k + 16383) // 16384))
         a = b / (ms * 1e-3) / 1e9
@@ -188,12 +194,14 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count):
     if stage == "sinkhorn":
         fma, _ = sinkhorn_work(out, cfg)
         a = 2 * fma / (ms * 1e-3) / 1e12
-        return dict(kernel="sinkhorn_kernel", bound="alu", achieved=a, peak=fp32_peak, unit="TFLOP/s",
+        return dict(kernel="sinkhorn_tile_kernel", bound="alu", achieved=a, peak=fp32_peak, unit="TFLOP/s",
                     frac=a / fp32_peak, traffic=None,
                     peak_source=f"derived: {sm_count} SMs x 128 fp32 lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz",
                     flops_per_launch=2 * fma,
-                    note="latency-bound chains of dependent mat-vecs over L small problems; fraction of the "
-                         "fp32 FMA peak is reported, not claimed as the binding limit")
+                    note="one dependent chain of small mat-vecs per problem and only L problems per call: "
+                         "latency-bound; DRAM traffic is ~0.1 MB per launch (ncu); the fp32-FMA fraction is "
+                         "reported, not claimed as the binding limit (see profiles/sweep_config5.md for batches "
+                         "that fill the GPU)")
     rounds = out["rounds"].cpu().numpy().astype(np.int64)
     ops = int((rounds[:, 0] * cfg.R * cfg.E + rounds[:, 1] * cfg.R * cfg.S).sum())
     a = ops / (ms * 1e-3) / 1e12

@@ -350,7 +350,7 @@ match_kernel(MatchArgs a)
             u64* arb = arb_r + (rounds3 & 1) * R;
             // Step 1: bid for the source rank with the best bonus minus price
 #ifdef TAOT_DEBUG_CLOCKS
-            const long long c0 = clock64();
+            __syncwarp(); const long long c0 = clock64();
 #endif
             u64 key = 0;
             if (live) {
@@ -410,16 +410,16 @@ match_kernel(MatchArgs a)
             }
             // Step 2: the rank keeps its best bidder (ties: lowest slot)
 #ifdef TAOT_DEBUG_CLOCKS
-            const long long c1 = clock64();
+            __syncwarp(); const long long c1 = clock64();
 #endif
             const int rsel = (int)(0xFFFFFFFFu - (uint32_t)key);
             arbitrate(arb, rsel, key == 0 ? 0ull : ((key & 0xFFFFFFFF00000000ull) | (u64)(0xFFFFFFFFu - (uint32_t)s)));
 #ifdef TAOT_DEBUG_CLOCKS
-            const long long c2 = clock64();
+            __syncwarp(); const long long c2 = clock64();
 #endif
             if (!__syncthreads_or(key != 0)) break;
 #ifdef TAOT_DEBUG_CLOCKS
-            const long long c3 = clock64();
+            __syncwarp(); const long long c3 = clock64();
 #endif
             if (prev_r >= 0) { arb_r[((rounds3 & 1) ^ 1) * R + prev_r] = 0; prev_r = -1; }
             // Steps 3-4: the winning slot of each rank collects x = min(n, A); holdings, plan and price follow
@@ -443,12 +443,12 @@ match_kernel(MatchArgs a)
             }
             ++rounds3;
 #ifdef TAOT_DEBUG_CLOCKS
-            const long long c4 = clock64();
+            __syncwarp(); const long long c4 = clock64();
 #endif
             __syncthreads();
 #ifdef TAOT_DEBUG_CLOCKS
             const long long c5 = clock64();
-            dbg[0] += c1 - c0; dbg[1] += c2 - c1; dbg[2] += c3 - c2; dbg[3] += c4 - c3;
+            dbg[0] += c1 - c0; dbg[1] += c2 - c1; dbg[2] += c3 - c2; dbg[3] += c4 - c3; dbg[4] += c5 - c4;
 #endif
         }
 #ifdef TAOT_DEBUG_CLOCKS
@@ -456,7 +456,7 @@ match_kernel(MatchArgs a)
         __syncthreads();
         if (l == 0 && a.rounds) {   // per-thread totals into the tail of X of the LAST layer (debug only)
             int32_t* dump = a.X + (int64_t)(gridDim.x - 1) * R * S;
-            dump[tid] = (int)(dbg[0] / 1000); dump[NT + tid] = dbg_levels; dump[2 * NT + tid] = dbg_bits; dump[3*NT + tid] = dbg_tiers;
+            dump[tid] = (int)(dbg[0] / 1000); dump[NT + tid] = (int)(dbg[1] / 1000); dump[2 * NT + tid] = (int)(dbg[2] / 1000); dump[3*NT + tid] = (int)(dbg[3] / 1000); dump[4*NT + tid] = (int)(dbg[4] / 1000);
         }
 #endif
         if (s < S) slot_a[s] = A;
