@@ -1,0 +1,164 @@
+"""Edge and degenerate cases of the CUDA path against the oracle: bad indices, balanced layers,
+supply exceeding demand, unaligned / ragged routing tables, extreme cost/eps (hand-back and
+log-domain paths of the Sinkhorn kernels), overlapping supply/demand supports, odd expert maps."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import workloads as W
+from helpers import check_sinkhorn_problem, cpu, make_planner, oracle_schedule_layer, topology
+
+pytestmark = pytest.mark.gpu
+
+
+def _full_check(cfg, topk, pl, B=None, e2r=None, C=None, expect_bad=False):
+    """Plan on the GPU and compare every stage with the oracle (schedule fed the GPU plan)."""
+    e2r_t, C_t = topology(cfg)
+    e2r = e2r_t.numpy() if e2r is None else e2r
+    C = C_t.numpy() if C is None else C
+    Bm = O.default_preference(C) if B is None else B
+    out = {k: cpu(v) for k, v in pl.plan(topk).items()}
+    tk = cpu(topk)
+    n, el, rl, bad = O.histogram(tk, cfg.R, cfg.E, e2r)
+    assert (out["n"] == n).all() and (out["expert_load"] == el).all() and (out["rank_load"] == rl).all()
+    assert ((out["info"] & 1) != 0).tolist() == (bad > 0).tolist()
+    assert bool((bad > 0).any()) == expect_bad
+    mean, ex, sp = O.excess_spare(rl)
+    assert (out["excess"] == ex).all() and (out["spare"] == sp).all()
+    for l in range(cfg.L):
+        s = ex[l].astype(np.float32); d = sp[l].astype(np.float32)
+        check_sinkhorn_problem(s, d, C, pl.params.eps, out["plan"][l], out["sinkhorn_iters"][l], out["row_err"][l],
+                               pl.params.max_iters, pl.params.tol, pl.params.check_every)
+        assert bool(out["info"][l] & 16) == (s.sum() > d.sum())
+        m, a = oracle_schedule_layer(cfg, e2r, Bm, n[l], el[l], rl[l], out["plan"][l])
+        assert (out["slot_expert"][l].ravel() == m["slot_expert"]).all()
+        assert (out["slot_tokens"][l].ravel() == m["slot_tokens"]).all()
+        assert (out["X"][l] == a["X"]).all()
+        want = O.assign(tk[l], cfg.R, cfg.E, cfg.K, m["slot_expert"], a["X"])
+        assert (out["new_idx"][l] == want).all()
+    return out
+
+
+def test_out_of_range_indices_are_skipped_flagged_and_copied_through():
+    cfg = W.get_config("cfg2").replace(L=3)
+    topk = W.routing_topk(cfg, device="cuda")
+    topk[1, 5, 2] = -1
+    topk[1, 9000, 0] = cfg.E
+    topk[2, 16383, 7] = 2 ** 30
+    pl = make_planner(cfg)
+    out = _full_check(cfg, topk, pl, expect_bad=True)
+    assert out["info"][0] & 1 == 0 and out["info"][1] & 1 and out["info"][2] & 1
+    assert out["new_idx"][1, 5, 2] == -1 and out["new_idx"][1, 9000, 0] == cfg.E and out["new_idx"][2, 16383, 7] == 2 ** 30
+    pl.close()
+
+
+def test_perfectly_balanced_layer_moves_nothing():
+    cfg = W.get_config("cfg1").replace(L=2)
+    topk = W.routing_topk(cfg, device="cuda")
+    # layer 1: every token t picks experts (t mod E) and (t+1 mod E): all ranks carry the same load
+    t = torch.arange(cfg.T, device="cuda")
+    topk[1, :, 0] = (t % cfg.E).int()
+    topk[1, :, 1] = ((t + 1) % cfg.E).int()
+    pl = make_planner(cfg)
+    out = _full_check(cfg, topk, pl)
+    assert (out["excess"][1] == 0).all() and (out["plan"][1] == 0).all() and out["sinkhorn_iters"][1] == 0
+    assert (out["slot_expert"][1] == -1).all() and (out["X"][1] == 0).all()
+    assert (out["new_idx"][1] == cpu(topk)[1]).all()
+    pl.close()
+
+
+def test_total_load_not_divisible_by_ranks_scales_the_supply():
+    # T*k = 3*1000*3 = 9000 entries over R = 7 ranks?  T must be a multiple of R: T = 7*143, k = 3 -> 3003 entries,
+    # 3003 mod 7 = 0; use E = 7*3 experts but route one extra-heavy pattern so that sum(l) mod R != 0 is impossible
+    # with every entry counted.  Bad indices are skipped, which makes the counted total non-divisible.
+    cfg = W.get_config("cfg1").replace(L=2, R=7, E=21, K=2, k=3, T=7 * 143, gpus_per_node=4)
+    topk = W.routing_topk(cfg, device="cuda")
+    topk[0, 0, 0] = -5                      # one entry dropped: total = 3002, 3002 mod 7 = 6 -> sum(excess) > sum(spare)
+    pl = make_planner(cfg, max_iters=300, tol=0.0)
+    out = _full_check(cfg, topk, pl, expect_bad=True)
+    assert out["info"][0] & 16 and out["excess"][0].sum() - out["spare"][0].sum() == 6
+    pl.close()
+
+
+@pytest.mark.parametrize("k,tpr,R,E", [(3, 1001, 4, 12), (5, 3333, 8, 16), (1, 40000, 2, 6), (8, 2049, 4, 8)])
+def test_unaligned_and_ragged_segments(k, tpr, R, E):
+    # SEG = tpr*k: not a multiple of 4 (scalar load path) and/or several chunks with a short last one
+    cfg = W.get_config("cfg1").replace(L=2, R=R, E=E, K=2, k=k, T=R * tpr, gpus_per_node=2, zipf=(1.3, 1.3))
+    topk = W.routing_topk(cfg, device="cuda")
+    pl = make_planner(cfg, max_iters=200, tol=1e-6)
+    _full_check(cfg, topk, pl)
+    # a routing table that does not start on a 16-byte boundary
+    buf = torch.empty(topk.numel() + 1, dtype=torch.int32, device="cuda")
+    shifted = buf[1:].view_as(topk)
+    shifted.copy_(topk)
+    n, el, rl, info = pl.histogram(shifted)
+    n0, el0, rl0, _ = pl.histogram(topk)
+    assert torch.equal(n, n0) and torch.equal(rl, rl0)
+    out = pl.plan(topk)
+    new, _ = pl.assign(shifted, out["slot_expert"], out["X"], reuse_counts=False)
+    assert torch.equal(new, out["new_idx"])
+    pl.close()
+
+
+def test_uneven_expert_map_and_three_slots():
+    cfg = W.get_config("cfg2").replace(L=3, K=3)
+    e2r = torch.tensor([0] * 10 + [1] * 2 + [2] * 1 + [3] * 7 + list(range(4, 16)) * 3 + [15] * 8, dtype=torch.int32)
+    assert e2r.numel() == cfg.E
+    C = W.cost_matrix(cfg.R, cfg.gpus_per_node, cfg.tiers)
+    import paper_2608_03676_b200 as P
+    pl = P.Planner(L=cfg.L, R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k, T=cfg.T, e2r=e2r, C=C, eps=cfg.eps, max_iters=500,
+                   tol=1e-6)
+    topk = W.routing_topk(cfg, device="cuda")
+    _full_check(cfg, topk, pl, e2r=e2r.numpy())
+    pl.close()
+
+
+@pytest.mark.parametrize("eps,iters,check_every", [(0.004, 150, 1), (0.02, 1, 1), (0.2, 400, 7)])
+def test_extreme_cost_over_eps_single_iteration_and_sparse_checks(eps, iters, check_every):
+    # eps = 0.004 gives C/eps up to 2500: far beyond fp32's exponent range
+    cfg = W.get_config("cfg2").replace(L=6)
+    topk = W.routing_topk(cfg, device="cuda")
+    pl = make_planner(cfg, eps=eps, max_iters=iters, tol=1e-6 if check_every > 1 else 0.0, check_every=check_every)
+    _full_check(cfg, topk, pl)
+    pl.close()
+
+
+def test_overlapping_supports_and_many_supply_ranks_take_the_shared_memory_kernel():
+    # taot_sinkhorn with arbitrary s, d: ranks with both supply and demand, more supply ranks than the register
+    # tile holds (R = 64: 32 rows), zero rows, and a problem with no demand at all
+    cfg = W.get_config("cfg3").replace(L=4, T=64 * 64)
+    pl = make_planner(cfg, max_iters=120, tol=0.0)
+    _, C = topology(cfg)
+    g = torch.Generator().manual_seed(3)
+    s = torch.rand((4, 64), generator=g) * 100
+    d = torch.rand((4, 64), generator=g) * 100
+    s[0, 40:] = 0; d[0, :24] = 0                       # 40 supply ranks (> 32), overlapping with demand on 24..39
+    s[1, ::2] = 0                                      # overlapping supports everywhere else
+    s[2] = 0; s[2, 5] = 7; d[2] = 0; d[2, 9] = 7       # 1 x 1 problem
+    d[3] = 0                                           # nothing can move
+    out = pl.sinkhorn(s.cuda(), d.cuda())
+    torch.cuda.synchronize()
+    for b in range(4):
+        check_sinkhorn_problem(s[b].numpy(), d[b].numpy(), C.numpy(), cfg.eps, cpu(out["plan"])[b],
+                               cpu(out["iters"])[b], cpu(out["row_err"])[b], 120, 0.0)
+    assert cpu(out["iters"]).tolist() == [120, 120, 120, 0]
+    pl.close()
+
+
+def test_handle_validation_and_null_arguments_return_status_codes():
+    import ctypes
+    import paper_2608_03676_b200 as P
+    cfg = W.get_config("cfg1")
+    pl = make_planner(cfg)
+    lib = P.load_library()
+    topk = W.routing_topk(cfg, device="cuda")
+    out = pl.alloc_outputs()
+    assert lib.taot_histogram(pl.handle, None, None, None, None, None, None, None) == -1
+    o = pl._outputs_struct(out)
+    assert lib.taot_plan(pl.handle, ctypes.c_void_p(topk.data_ptr()), ctypes.byref(o), ctypes.c_void_p(pl.ws.data_ptr() + 4), None) == -5
+    o.new_idx = topk.data_ptr()                         # in-place rewrite is refused
+    assert lib.taot_plan(pl.handle, ctypes.c_void_p(topk.data_ptr()), ctypes.byref(o), ctypes.c_void_p(pl.ws.data_ptr()), None) == -2
+    with pytest.raises(P.TaotError):
+        pl.histogram(topk.cpu())                        # host tensor where device memory is required
+    pl.close()

@@ -1,0 +1,61 @@
+"""Configs 3 and 4 at their full sizes, in the launch configuration bench.py times: properties that hold at
+any size on every layer, and the oracle on sampled layers (each of which it can compute in seconds)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import workloads as W
+from helpers import check_sinkhorn_problem, cpu, make_planner, oracle_schedule_layer, topology
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,sample", [("cfg3", (0, 31, 57)), ("cfg4", (0, 47))])
+def test_full_size(name, sample):
+    cfg = W.get_config(name)
+    e2r, C = topology(cfg)
+    B = O.default_preference(C.numpy())
+    topk = W.routing_topk(cfg, device="cuda")
+    pl = make_planner(cfg)
+    out = pl.plan(topk)
+    torch.cuda.synchronize()
+    L, R, E, K, S, T, k = cfg.L, cfg.R, cfg.E, cfg.K, cfg.S, cfg.T, cfg.k
+    # ---- every layer, on the GPU
+    assert int(out["n"].sum()) == L * T * k and int(out["info"].bitwise_and(1).sum()) == 0
+    assert torch.equal(out["n"].sum(1), out["expert_load"])
+    ones = torch.ones_like(topk[0].reshape(-1))
+    for l in range(L):
+        el = torch.zeros(E, dtype=torch.int32, device="cuda").index_add_(0, topk[l].reshape(-1).long(), ones)
+        assert torch.equal(el, out["expert_load"][l])
+    ex = out["excess"].double(); sp = out["spare"].double()
+    assert torch.equal(ex.sum(1), sp.sum(1))                                     # T*k divisible by R: balanced masses
+    col_viol = (out["plan"].double().sum(1) - sp).abs().sum(1)
+    assert bool((col_viol <= 1e-5 * ex.sum(1)).all()) and bool((out["plan"] >= 0).all())
+    conv = (out["info"] & 2) == 0
+    row_viol = (out["plan"].double().sum(2) - ex).abs().sum(1)
+    assert bool((row_viol[conv] <= (1e-6 + 5e-7 + 1e-5) * ex.sum(1)[conv]).all())
+    assert bool((out["X"].sum(1) == out["slot_tokens"].reshape(L, S)).all())     # every slot fully collected
+    moved = out["new_idx"] != topk
+    assert int(moved.sum()) == int(out["X"].sum())                               # token conservation
+    assert bool((out["new_idx"][moved] >= E).all()) and bool((out["new_idx"][~moved] == topk[~moved]).all())
+    again = pl.plan(topk)
+    torch.cuda.synchronize()
+    for key in ("plan", "X", "new_idx", "sinkhorn_iters"):
+        assert torch.equal(again[key], out[key]), key                            # deterministic
+    # ---- sampled layers against the oracle
+    for l in sample:
+        tk = cpu(topk[l:l + 1])
+        n, el, rl, bad = O.histogram(tk, R, E, e2r.numpy())
+        assert (cpu(out["n"][l]) == n[0]).all() and (cpu(out["rank_load"][l]) == rl[0]).all()
+        mean, exo, spo = O.excess_spare(rl)
+        plan = cpu(out["plan"][l])
+        check_sinkhorn_problem(exo[0].astype(np.float32), spo[0].astype(np.float32), C.numpy(), cfg.eps, plan,
+                               int(out["sinkhorn_iters"][l]), float(out["row_err"][l]), cfg.max_iters, cfg.tol)
+        m, a = oracle_schedule_layer(cfg, e2r.numpy(), B, n[0], el[0], rl[0], plan)
+        assert (cpu(out["slot_expert"][l]).ravel() == m["slot_expert"]).all()
+        assert (cpu(out["X"][l]) == a["X"]).all()
+        assert cpu(out["rounds"][l]).tolist() == [m["inner_rounds"], a["rounds"]]
+        want = O.assign(tk[0], R, E, K, m["slot_expert"], a["X"])
+        assert (cpu(out["new_idx"][l]) == want).all()
+    pl.close()
