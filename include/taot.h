@@ -61,7 +61,9 @@ enum {
     TAOT_INFO_NONFINITE = 4,        /* a non-finite value appeared in the Sinkhorn solve */
     TAOT_INFO_AUCTION_RESIDUAL = 8, /* the auction stopped at auction_max_rounds with tokens unplaced */
     TAOT_INFO_SUPPLY_SCALED = 16,   /* sum(s) > sum(d): supply was scaled by gamma < 1 */
-    TAOT_INFO_SINKHORN_SIZE = 32    /* |hot| * |cold| exceeds the on-chip capacity: plan left at zero */
+    TAOT_INFO_SINKHORN_SIZE = 32,   /* |hot| * |cold| exceeds the on-chip capacity: plan left at zero */
+    TAOT_INFO_INTERNAL = 64         /* a bounded wait inside a kernel ran out (asynchronous copy never landed):
+                                       the outputs of that call are incomplete */
 };
 
 /*

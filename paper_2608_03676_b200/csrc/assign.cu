@@ -16,6 +16,8 @@
 // common path is: 16 loads in flight, one table row from L2, 64 lookups, 16 stores.  8 bytes of HBM
 // traffic per entry: one read, one write.  Out-of-range indices are copied through (the histogram pass, whose
 // counts this kernel consumes, is the one that flags them).
+#include <cstdio>
+
 #include "taot_internal.cuh"
 
 namespace {
@@ -58,8 +60,9 @@ __device__ int build_entries(const int32_t* Xrow, const int32_t* se, int S, int 
                              int32_t* ent_e, int32_t* ent_lo, int32_t* ent_hi, int* s_wcnt)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int NT = blockDim.x, NWB = NT >> 5;
     int m = 0;
-    for (int sb = 0; sb < S; sb += kThreads) {
+    for (int sb = 0; sb < S; sb += NT) {
         const int s = sb + tid;
         const int32_t xv = s < S ? Xrow[s] : 0;
         const int32_t ev = s < S ? se[s] : -1;
@@ -73,10 +76,10 @@ __device__ int build_entries(const int32_t* Xrow, const int32_t* se, int S, int 
             const int q = off + __popc(bal & ((1u << lane) - 1u));
             ent_s[q] = s; ent_e[q] = ev; ent_hi[q] = xv;
         }
-        for (int w = 0; w < kWarps; ++w) m += s_wcnt[w];
+        for (int w = 0; w < NWB; ++w) m += s_wcnt[w];
         __syncthreads();
     }
-    for (int q = tid; q < m; q += kThreads) {
+    for (int q = tid; q < m; q += NT) {
         const int e = ent_e[q];
         int32_t lo = 0;
         for (int p = 0; p < q; ++p) lo += (ent_e[p] == e) ? ent_hi[p] : 0;
@@ -294,6 +297,266 @@ assign_kernel(AssignArgs a)
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Persistent, bulk-copy-pipelined version of the rewrite (used when the routing table is 16-byte
+// aligned and E is a multiple of 4).  One CTA per SM walks chunks blockIdx.x, +gridDim.x, ...; a
+// single thread keeps kStages-1 chunks in flight with cp.async.bulk (global -> shared, completion
+// counted on an mbarrier per stage, no multicast), so the loads of the next chunks overlap the
+// lookups and stores of the current one.  Each stage carries the chunk (<= 64 KB) and its table row.
+// Arithmetic and rare path are those of assign_kernel; the chunk is read from shared memory
+// instead of registers.
+
+constexpr int kSThreads = 256;
+constexpr int kSWarps = kSThreads / 32;
+constexpr int kSWarpSpan = TAOT_CHUNK / kSWarps;        // 2048 entries per warp, contiguous
+constexpr int kSIters = kSWarpSpan / 128;               // 16 x 16-byte accesses per lane
+constexpr uint32_t kBulkPiece = 8192;                   // bytes per bulk copy: several pieces in flight per chunk
+constexpr uint32_t kWaitSpins = 1u << 20;               // bound on mbarrier polling (each poll can itself block for a while)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// Poll until the phase with the given parity completes; false if the spin bound ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
+{
+    const uint32_t addr = smem_u32(bar);
+    for (uint32_t spin = 0; spin < kWaitSpins; ++spin) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+struct StreamLayout {
+    int stages;
+    size_t off_tab, off_scratch, bytes;       // chunk buffers start at 0
+};
+
+StreamLayout stream_layout(int E, int S)
+{
+    const size_t scratch = sizeof(int32_t) * ((size_t)E * (2 + 2 * kSWarps) + 4 * (size_t)S);   // base, blist, cntw, wtab, ent_*
+    StreamLayout L;
+    const size_t per_stage = (size_t)TAOT_CHUNK * 4 + (size_t)E * 4;
+    const size_t budget = 220 * 1024;
+    int st = (int)((budget - scratch - 256) / per_stage);
+    L.stages = st > 4 ? 4 : st;
+    L.off_tab = (size_t)L.stages * TAOT_CHUNK * 4;
+    L.off_scratch = L.off_tab + (size_t)L.stages * E * 4;
+    L.bytes = L.off_scratch + scratch;
+    return L;
+}
+
+__global__ void __launch_bounds__(kSThreads, 1)
+assign_stream_kernel(AssignArgs a, int stages, uint32_t off_tab, uint32_t off_scratch, int64_t nchunks)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(8) uint64_t bars[4];
+    __shared__ int s_wcnt[32];
+    __shared__ int s_nb;
+    const int E = a.E, S = a.R * a.K;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int32_t* scratch = reinterpret_cast<int32_t*>(smem + off_scratch);
+    int32_t* base = scratch;                    // [E]  start ordinal of each boundary expert (indexed by its list position)
+    int32_t* blist = base + E;                  // [E]
+    int32_t* cntw = blist + E;                  // [E * kSWarps]
+    int32_t* wtab = cntw + E * kSWarps;         // [kSWarps][E]
+    int32_t* ent_s = wtab + E * kSWarps;        // [S] ...
+    int32_t* ent_e = ent_s + S;
+    int32_t* ent_lo = ent_e + S;
+    int32_t* ent_hi = ent_lo + S;
+
+    if (tid == 0) {
+        for (int st = 0; st < stages; ++st) mbar_init(&bars[st], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    auto chunk_geometry = [&](int64_t id, int64_t& goff, int32_t& len) {
+        const int32_t c = (int32_t)(id % a.nc);
+        const int64_t lr = id / a.nc;
+        const int64_t start = (int64_t)c * TAOT_CHUNK;
+        len = (int32_t)((a.seg - start) < (int64_t)TAOT_CHUNK ? (a.seg - start) : (int64_t)TAOT_CHUNK);
+        goff = (lr / a.R) * a.layer_elems + (lr % a.R) * a.seg + start;
+    };
+    auto issue = [&](int64_t id, int st) {      // one thread: arm the stage and start its two copies
+        int64_t goff; int32_t len;
+        chunk_geometry(id, goff, len);
+        const uint32_t bytes = (uint32_t)len * 4u;
+        mbar_expect_tx(&bars[st], bytes + (uint32_t)E * 4u);
+        unsigned char* dstb = smem + (size_t)st * TAOT_CHUNK * 4;
+        const unsigned char* srcb = reinterpret_cast<const unsigned char*>(a.topk + goff);
+        for (uint32_t o = 0; o < bytes; o += kBulkPiece)
+            bulk_load(dstb + o, srcb + o, (bytes - o) < kBulkPiece ? (bytes - o) : kBulkPiece, &bars[st]);
+        bulk_load(smem + off_tab + (size_t)st * E * 4, a.tabg + id * (int64_t)E, (uint32_t)E * 4u, &bars[st]);
+    };
+
+    const int64_t first = blockIdx.x, stride = gridDim.x;
+    if (tid == 0)
+        for (int st = 0; st < stages; ++st)
+            if (first + st * stride < nchunks) issue(first + st * stride, st);
+
+    int64_t it_global = 0;
+    for (int64_t id = first; id < nchunks; id += stride, ++it_global) {
+        const int st = (int)(it_global % stages);
+        const uint32_t parity = (uint32_t)((it_global / stages) & 1);
+        const int nb = a.nbg[id];
+        int64_t goff; int32_t len;
+        chunk_geometry(id, goff, len);
+        const int64_t lr = id / a.nc;
+        const int32_t c = (int32_t)(id % a.nc);
+        const int32_t l = (int32_t)(lr / a.R);
+        int32_t* buf = reinterpret_cast<int32_t*>(smem + (size_t)st * TAOT_CHUNK * 4);
+        const int32_t* tab = reinterpret_cast<const int32_t*>(smem + off_tab + (size_t)st * E * 4);
+        int32_t* dst = a.out + goff;
+
+        const bool ok = mbar_wait(&bars[st], parity);
+        if (__syncthreads_or(!ok)) {
+            // the copy never completed: report, give the copies still in flight one more bounded chance to land
+            // (their destination is this CTA's shared memory), and leave
+            if (tid == 0) {
+                atomicOr(a.info + l, TAOT_INFO_INTERNAL);
+                for (int s2 = 0; s2 < stages; ++s2) {
+                    const int64_t use = (it_global + ((s2 - st + stages) % stages)) / stages;
+                    (void)mbar_wait(&bars[s2], (uint32_t)(use & 1));
+                }
+            }
+            __syncthreads();
+            return;
+        }
+        const int32_t wbase = warp * kSWarpSpan + lane * 4;
+        const int32_t* lut = tab;
+        if (nb > 0) {
+            // ---- rare path: this rank's quota intervals, per-warp refinement of the boundary experts
+            const int m = build_entries(a.X + lr * S, a.slot_expert + (int64_t)l * S, S, E, ent_s, ent_e, ent_lo, ent_hi, s_wcnt);
+            for (int q = tid; q < m; q += kSThreads) ent_hi[q] += ent_lo[q];
+            const int32_t* ccseg = a.cc + lr * a.nc * (int64_t)E;
+            if (tid == 0) s_nb = 0;
+            __syncthreads();
+            for (int e = tid; e < E; e += kSThreads)
+                if (tab[e] == -1) {
+                    int32_t b = 0;
+                    for (int cp = 0; cp < c; ++cp) b += ccseg[(int64_t)cp * E + e];
+                    const int bi = atomicAdd(&s_nb, 1);
+                    blist[bi] = e;
+                    base[bi] = b;
+                }
+            __syncthreads();
+#pragma unroll 1
+            for (int bi = 0; bi < nb; ++bi) {
+                const int eb = blist[bi];
+                int cnt = 0;
+#pragma unroll 4
+                for (int it = 0; it < kSIters; ++it) {
+                    const int32_t pos = wbase + it * 128;
+                    if (pos < len) {
+                        const int4 v = *reinterpret_cast<const int4*>(buf + pos);
+                        cnt += (v.x == eb) + (v.y == eb) + (v.z == eb) + (v.w == eb);
+                    }
+                }
+                for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+                if (lane == 0) cntw[bi * kSWarps + warp] = cnt;
+            }
+            int32_t* myt = wtab + warp * E;
+            for (int e = lane; e < E; e += 32) { const int32_t t = tab[e]; myt[e] = t == -1 ? e : t; }
+            __syncthreads();
+            const unsigned lt = (1u << lane) - 1u;
+#pragma unroll 1
+            for (int bi = 0; bi < nb; ++bi) {
+                const int eb = blist[bi];
+                const int32_t mine = cntw[bi * kSWarps + warp];
+                int32_t running = base[bi];
+                for (int w = 0; w < warp; ++w) running += cntw[bi * kSWarps + w];
+                // this warp's ordinals of eb are [running, running + mine): inside one interval, outside all, or
+                // straddling; the (at most two, else a list walk) intervals it straddles are kept in registers
+                int32_t target = eb;
+                int nstr = 0, q0 = m, q1 = m;
+                int32_t lo0 = 0, hi0 = 0, t0 = eb, lo1 = 0, hi1 = 0, t1 = eb;
+                for (int q = 0; q < m; ++q) {
+                    if (ent_e[q] != eb || mine == 0) continue;
+                    if (ent_hi[q] <= running || ent_lo[q] >= running + mine) continue;
+                    if (ent_lo[q] <= running && ent_hi[q] >= running + mine) { target = E + ent_s[q]; continue; }
+                    if (nstr == 0) { lo0 = ent_lo[q]; hi0 = ent_hi[q]; t0 = E + ent_s[q]; q0 = q; }
+                    else if (nstr == 1) { lo1 = ent_lo[q]; hi1 = ent_hi[q]; t1 = E + ent_s[q]; }
+                    ++nstr;
+                    q1 = q + 1;
+                }
+                if (nstr == 0) {
+                    if (lane == 0) myt[eb] = target;
+                    continue;
+                }
+#pragma unroll 1
+                for (int it = 0; it < kSIters; ++it) {           // kept rolled: this code runs rarely and must stay small
+                    const int32_t pos = wbase + it * 128;
+                    int4 v = make_int4(-1, -1, -1, -1);
+                    if (pos < len) v = *reinterpret_cast<const int4*>(buf + pos);
+                    int32_t* xv = reinterpret_cast<int32_t*>(&v);
+                    const bool m0 = xv[0] == eb, m1 = xv[1] == eb, m2 = xv[2] == eb, m3 = xv[3] == eb;
+                    const unsigned b0 = __ballot_sync(0xffffffffu, m0), b1 = __ballot_sync(0xffffffffu, m1);
+                    const unsigned b2 = __ballot_sync(0xffffffffu, m2), b3 = __ballot_sync(0xffffffffu, m3);
+                    if ((b0 | b1 | b2 | b3) == 0) continue;
+                    int32_t ord = running + __popc(b0 & lt) + __popc(b1 & lt) + __popc(b2 & lt) + __popc(b3 & lt);
+                    const bool mm[4] = {m0, m1, m2, m3};
+                    bool changed = false;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (mm[j]) {
+                            if (nstr <= 2) {
+                                if (ord >= lo0 && ord < hi0) { xv[j] = t0; changed = true; }
+                                else if (nstr == 2 && ord >= lo1 && ord < hi1) { xv[j] = t1; changed = true; }
+                            } else {
+                                for (int q = q0; q < q1; ++q)
+                                    if (ent_e[q] == eb && ord >= ent_lo[q] && ord < ent_hi[q]) { xv[j] = E + ent_s[q]; changed = true; break; }
+                            }
+                            ++ord;
+                        }
+                    }
+                    if (changed) *reinterpret_cast<int4*>(buf + pos) = v;        // moved entries are now >= E and pass through
+                    running += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
+                }
+            }
+            __syncwarp();
+            lut = myt;
+        }
+        // ---- one table lookup per entry (values >= E or < 0 pass through unchanged), then store
+#pragma unroll 4
+        for (int it = 0; it < kSIters; ++it) {
+            const int32_t pos = wbase + it * 128;
+            if (pos < len) {
+                int4 v = *reinterpret_cast<const int4*>(buf + pos);
+#ifndef TAOT_DBG_NOLOOKUP
+                if ((uint32_t)v.x < (uint32_t)E) v.x = lut[v.x];
+                if ((uint32_t)v.y < (uint32_t)E) v.y = lut[v.y];
+                if ((uint32_t)v.z < (uint32_t)E) v.z = lut[v.z];
+                if ((uint32_t)v.w < (uint32_t)E) v.w = lut[v.w];
+#endif
+#ifdef TAOT_DBG_NOSTORE
+                if (v.x == 0x7fffffff)
+#endif
+                st_stream(reinterpret_cast<int4*>(dst + pos), v);
+            }
+        }
+        __syncthreads();                         // everyone is done with this stage's buffers
+        if (tid == 0 && id + (int64_t)stages * stride < nchunks) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            issue(id + (int64_t)stages * stride, st);
+        }
+    }
+}
+
 }  // namespace
 
 int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_cc, int32_t* d_tabg,
@@ -313,7 +576,13 @@ int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_
     TAOT_CUDA_OK(cudaGetLastError());
     const size_t smem = sizeof(int32_t) * ((size_t)p.E * (3 + 2 * kWarps) + 4 * (size_t)S);
     const unsigned blocks = (unsigned)((int64_t)p.L * p.R * h->nc);
-    if (a.vec_ok) {
+    const StreamLayout sl = stream_layout(p.E, S);
+    if (a.vec_ok && p.E % 4 == 0 && sl.stages >= 2) {
+        TAOT_CUDA_OK(cudaFuncSetAttribute(assign_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sl.bytes));
+        const unsigned grid = blocks < (unsigned)h->sm_count ? blocks : (unsigned)h->sm_count;
+        assign_stream_kernel<<<grid, kSThreads, sl.bytes, st>>>(a, sl.stages, (uint32_t)sl.off_tab, (uint32_t)sl.off_scratch,
+                                                              (int64_t)blocks);
+    } else if (a.vec_ok) {
         TAOT_CUDA_OK(cudaFuncSetAttribute(assign_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         assign_kernel<true><<<blocks, kThreads, smem, st>>>(a);
     } else {
