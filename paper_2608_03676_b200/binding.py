@@ -94,8 +94,9 @@ def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
 
 STATIC_SCRATCH_BYTES = 4 << 20
 # kernels one taot_plan call enqueues: chunk histogram, merge, Sinkhorn (register tile + shared-memory
-# kernel for handed-back problems), matching+auction, reassignment (table build + rewrite)
-PLAN_LAUNCHES = 7
+# kernel for handed-back problems), matching+auction, reassignment (tables, pipelined rewrite of the chunks
+# without a split, rewrite of the chunks with one) -- for a 16-byte aligned routing table with E % 4 == 0
+PLAN_LAUNCHES = 8
 
 
 def histogram_static(topk: torch.Tensor, R: int, E: int, e2r_dev: torch.Tensor, n: torch.Tensor,

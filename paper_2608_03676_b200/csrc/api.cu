@@ -57,8 +57,10 @@ void layout(taot_handle_t h)
     size_t off = 0;
     auto take = [&](size_t bytes) { const size_t o = off; off = taot_align_up(off + bytes, 256); return o; };
     h->off_cc = take(sizeof(int32_t) * LR * h->nc * p.E);
-    h->off_tabg = take(sizeof(int32_t) * LR * h->nc * p.E);
+    h->off_tabg = take(sizeof(int32_t) * LR * h->nc * (p.E + 20));   // E targets + row tail (assign.cu: kRowTail)
     h->off_nbg = take(sizeof(int32_t) * LR * h->nc);
+    h->off_soff = take(sizeof(int32_t) * LR * h->nc);
+    h->off_splits = take(16 * LR * (size_t)p.R * p.K);
     h->off_excess = take(sizeof(int32_t) * LR);
     h->off_spare = take(sizeof(int32_t) * LR);
     h->off_s = take(sizeof(float) * LR);
@@ -352,8 +354,7 @@ int taot_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_slot_ex
         if (a < 0) return a;
         launches += a;
     }
-    int b = taot_launch_assign(h, d_topk, cc, reinterpret_cast<int32_t*>(at(ws, h->off_tabg)),
-                               reinterpret_cast<int32_t*>(at(ws, h->off_nbg)), d_slot_expert, d_X, d_new_idx, d_info, st);
+    int b = taot_launch_assign(h, d_topk, ws, d_slot_expert, d_X, d_new_idx, d_info, st);
     if (b < 0) return b;
     h->last_launches = launches + b;
     return TAOT_OK;
@@ -398,10 +399,7 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, voi
         return a;
     total += a;
     TAOT_MARK(4);
-    if ((a = taot_launch_assign(h, d_topk, cc, reinterpret_cast<int32_t*>(at(ws, h->off_tabg)),
-                                reinterpret_cast<int32_t*>(at(ws, h->off_nbg)), o->slot_expert, o->X, o->new_idx,
-                                o->info, st)) < 0)
-        return a;
+    if ((a = taot_launch_assign(h, d_topk, ws, o->slot_expert, o->X, o->new_idx, o->info, st)) < 0) return a;
     total += a;
     TAOT_MARK(5);
 #undef TAOT_MARK

@@ -3,59 +3,69 @@
 // X[r][s] entries each) and the rest stay.  ("Token routing is adjusted accordingly", Problem
 // Formulation; the paper fixes the counts X, this rule fixes which entries.)
 //
-// One CTA per chunk of at most TAOT_CHUNK entries, the same chunks the histogram kernel counted.
-// The chunk is loaded once into registers (64 entries per thread, all loads issued up front);
-// each warp owns 2048 contiguous entries.  The chunk counts of the histogram pass give, for every
-// expert, the ordinal range its entries occupy in this chunk.  If that range falls inside one
-// slot's quota (or outside all of them) every such entry of the chunk has the same target: one
-// shared-memory table lookup per entry, and that is all most chunks need.  An expert whose range
-// straddles a quota boundary (about one chunk in five has one) is counted per warp from the
-// registers; warps that do not contain the boundary still get a single target for it, and only the
-// one warp that does computes exact per-entry ordinals from ballots.  The per-chunk tables are built
-// by a small kernel with one CTA per (layer, source rank) segment, so that the streaming kernel's
-// common path is: 16 loads in flight, one table row from L2, 64 lookups, 16 stores.  8 bytes of HBM
-// traffic per entry: one read, one write.  Out-of-range indices are copied through (the histogram pass, whose
-// counts this kernel consumes, is the one that flags them).
-#include <cstdio>
-
+// Within a (rank, expert) group the slots take consecutive ordinal intervals [0,x1), [x1,x1+x2), ...
+// The chunk counts of the histogram pass say which ordinals of each expert fall into each chunk of
+// at most TAOT_CHUNK entries, so for most (chunk, expert) pairs every entry has the same target and
+// the rewrite is a table lookup.  Where an interval ends strictly inside a chunk's ordinal range
+// (a "split": at most one per slot this rank feeds, about one chunk in five has one), the entries
+// before the split position go to that slot and the later ones follow the next interval.  Kernels:
+//   assign_prep_kernel   one CTA per (layer, source rank): per chunk, the table expert -> target of
+//                        the chunk's LAST entry of that expert, and the splits (expert, in-chunk
+//                        ordinal, slot before); up to four of them ride in the tail of the table row;
+//   assign_stream_kernel persistent, one CTA per SM: chunks staged in shared memory by bulk
+//                        asynchronous copies (cp.async.bulk + mbarrier, no multicast), several in
+//                        flight; per entry one table lookup; in a chunk with splits the CTA first finds
+//                        each split's flat position (per-warp counts, then ballots in the one warp that
+//                        holds it) and applies "expert e before position P -> slot" as predicated
+//                        overrides; 16-byte streaming stores.  The compute hides under the copies.
+//   assign_chunk_kernel  one CTA per chunk: the chunks that do hold a split (staged in shared memory the same
+//                        way, since they are read three times), and, with ordinary loads, every chunk of a
+//                        routing table that is not 16-byte aligned or whose segments are not multiples of 4.
+// 8 bytes of HBM traffic per entry (one read, one write).  Out-of-range indices are copied through (the histogram pass, whose counts this path
+// consumes, is the one that flags them).
 #include "taot_internal.cuh"
 
 namespace {
 
 constexpr int kThreads = TAOT_STREAM_THREADS;
 constexpr int kWarps = kThreads / 32;
-constexpr int kIters = TAOT_CHUNK / (kThreads * 4);      // int4 loads per thread: 16
 constexpr int kWarpSpan = TAOT_CHUNK / kWarps;           // entries one warp owns, contiguous: 2048
+constexpr int kIters = kWarpSpan / 128;                  // 16-byte accesses per lane: 16
+constexpr int kRowSplits = 4;                            // split records that ride in the tail of a table row
+constexpr int kRowTail = 4 + 4 * kRowSplits;             // {ns, soff, 0, 0} + records {expert, rel / -, target before, position}
 
 struct AssignArgs {
     const int32_t* topk;
-    const int32_t* cc;
-    int32_t* tabg;          // [L,R,NC,E] per-chunk target tables written by the prep kernel
-    int32_t* nbg;           // [L,R,NC]   number of boundary experts of each chunk
+    const int32_t* cc;          // [L,R,NC,E] chunk counts (histogram pass)
+    int32_t* tabg;              // [L,R,NC,E+kRowTail] target of the chunk's last entry of each expert, then the row tail
+    int32_t* nsg;               // [L,R,NC]   number of splits in the chunk
+    int32_t* soff;              // [L,R,NC]   index of the chunk's first split record in its segment's list
+    int4* splits;               // [L,R,S]    {expert, ordinal of the split relative to the chunk, target before, position}
     const int32_t* slot_expert;
     const int32_t* X;
     int32_t* out;
     int32_t* info;
     int64_t layer_elems, seg;
-    int32_t nc, R, E, K, vec_ok;
+    int32_t nc, R, E, K;
 };
 
-__device__ __forceinline__ int4 ld_stream(const int4* p)
-{
-    int4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
-}
 
 __device__ __forceinline__ void st_stream(int4* p, const int4& v)
 {
     asm volatile("st.global.cs.v4.s32 [%0], {%1,%2,%3,%4};" :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
-// Shared by both kernels: the slots this source rank feeds (X > 0), ascending, with the ordinal
-// interval [lo, hi) each takes inside its (rank, expert) group.  Returns the number of entries.
-// On return ent_hi holds COUNTS (hi - lo); the caller adds ent_lo after its last use of the counts.
+__device__ __forceinline__ void chunk_geometry(const AssignArgs& a, int64_t id, int64_t& goff, int32_t& len)
+{
+    const int32_t c = (int32_t)(id % a.nc);
+    const int64_t lr = id / a.nc;
+    const int64_t start = (int64_t)c * TAOT_CHUNK;
+    len = (int32_t)((a.seg - start) < (int64_t)TAOT_CHUNK ? (a.seg - start) : (int64_t)TAOT_CHUNK);
+    goff = (lr / a.R) * a.layer_elems + (lr % a.R) * a.seg + start;
+}
+
+// The slots this source rank feeds (X > 0), ascending, with the ordinal interval [lo, hi) each takes
+// inside its (rank, expert) group.  Returns the number of entries.
 __device__ int build_entries(const int32_t* Xrow, const int32_t* se, int S, int E, int32_t* ent_s,
                              int32_t* ent_e, int32_t* ent_lo, int32_t* ent_hi, int* s_wcnt)
 {
@@ -74,7 +84,7 @@ __device__ int build_entries(const int32_t* Xrow, const int32_t* se, int S, int 
         for (int w = 0; w < warp; ++w) off += s_wcnt[w];
         if (p) {
             const int q = off + __popc(bal & ((1u << lane) - 1u));
-            ent_s[q] = s; ent_e[q] = ev; ent_hi[q] = xv;
+            ent_s[q] = s; ent_e[q] = ev; ent_hi[q] = xv;         // count for now
         }
         for (int w = 0; w < NWB; ++w) m += s_wcnt[w];
         __syncthreads();
@@ -86,232 +96,290 @@ __device__ int build_entries(const int32_t* Xrow, const int32_t* se, int S, int 
         ent_lo[q] = lo;
     }
     __syncthreads();
+    for (int q = tid; q < m; q += NT) ent_hi[q] += ent_lo[q];
+    __syncthreads();
     return m;
 }
 
-// One CTA per (layer, source rank): the target table of every chunk of the segment.
-// tab[e] = e (stays), E + s (the chunk's whole ordinal range of e lies in slot s's quota) or -1
-// (the range straddles a quota boundary: a boundary expert of that chunk).
+// chunks of a segment handled per pass of the prep kernel (bounds its shared memory)
+__host__ __device__ inline int prep_tile(int E) { const int t = 6144 / E; return t < 1 ? 1 : (t > 32 ? 32 : t); }
+
 __global__ void __launch_bounds__(kThreads)
 assign_prep_kernel(AssignArgs a)
 {
     extern __shared__ int32_t sh[];
-    const int E = a.E, S = a.R * a.K;
-    int32_t* tab = sh;                  // [E]
-    int32_t* base = tab + E;            // [E] running ordinal at the start of the current chunk
-    int32_t* ent_s = base + E;          // [S]
+    const int E = a.E, S = a.R * a.K, NC = a.nc, NCT = prep_tile(E) < NC ? prep_tile(E) : NC;
+    int32_t* ent_s = sh;                // [S]
     int32_t* ent_e = ent_s + S;
     int32_t* ent_lo = ent_e + S;
     int32_t* ent_hi = ent_lo + S;
-    __shared__ int s_wcnt[kWarps];
-    __shared__ int s_nb;
+    int32_t* carry = ent_hi + S;        // [E] ordinal at the start of the current tile of chunks
+    int32_t* cnts = carry + E;          // [NCT][E] counts of the tile's chunks
+    int32_t* base = cnts + NCT * E;     // [NCT][E] ordinal at the start of each chunk
+    int32_t* tab = base + NCT * E;      // [NCT][E] targets
+    int32_t* nsc = tab + NCT * E;       // [NCT] splits per chunk
+    __shared__ int s_wcnt[32];
+    __shared__ int s_over;
     const int tid = threadIdx.x;
     const int64_t lr = blockIdx.x;
     const int32_t l = (int32_t)(lr / a.R);
+    const int32_t* ccseg = a.cc + lr * NC * (int64_t)E;
+    int32_t* rows = a.tabg + lr * NC * (int64_t)(E + kRowTail);
+    int4* over = a.splits + lr * S;
+    for (int e = tid; e < E; e += kThreads) carry[e] = 0;
+    if (tid == 0) s_over = 0;
     const int m = build_entries(a.X + lr * S, a.slot_expert + (int64_t)l * S, S, E, ent_s, ent_e, ent_lo, ent_hi, s_wcnt);
-    for (int e = tid; e < E; e += kThreads) base[e] = 0;
-    const int32_t* ccseg = a.cc + lr * a.nc * (int64_t)E;
-    for (int c = 0; c < a.nc; ++c) {
-        for (int e = tid; e < E; e += kThreads) tab[e] = e;
-        if (tid == 0) s_nb = 0;
+    for (int c0 = 0; c0 < NC; c0 += NCT) {
+        const int nct = (NC - c0) < NCT ? (NC - c0) : NCT;
+        for (int i = tid; i < nct * E; i += kThreads) { cnts[i] = ccseg[(int64_t)c0 * E + i]; tab[i] = i % E; }
+        for (int c = tid; c < nct; c += kThreads) nsc[c] = 0;
         __syncthreads();
-        for (int q = tid; q < m; q += kThreads) {
-            const int e = ent_e[q];
-            const int32_t lo = ent_lo[q], hi = lo + ent_hi[q];
-            const int32_t cnt = ccseg[(int64_t)c * E + e];
-            const int32_t b = base[e];
-            if (!(cnt == 0 || hi <= b || lo >= b + cnt))
-                tab[e] = (lo <= b && hi >= b + cnt) ? E + ent_s[q] : -1;      // at most one full cover per expert
-        }
-        __syncthreads();
-        int32_t* out = a.tabg + (lr * a.nc + c) * (int64_t)E;
         for (int e = tid; e < E; e += kThreads) {
-            const int32_t t = tab[e];
-            out[e] = t;
-            if (t == -1) atomicAdd(&s_nb, 1);
-            base[e] += ccseg[(int64_t)c * E + e];
+            int32_t b = carry[e];
+            for (int c = 0; c < nct; ++c) { base[c * E + e] = b; b += cnts[c * E + e]; }
+            carry[e] = b;
         }
         __syncthreads();
-        if (tid == 0) a.nbg[lr * a.nc + c] = s_nb;
+        for (int i = tid; i < nct * m; i += kThreads) {
+            const int c = i / m, q = i - c * m;
+            const int e = ent_e[q];
+            const int32_t cnt = cnts[c * E + e];
+            if (cnt == 0) continue;
+            const int32_t b = base[c * E + e], lo = ent_lo[q], hi = ent_hi[q];
+            const int32_t last = b + cnt - 1;
+            if (lo <= last && last < hi) tab[c * E + e] = E + ent_s[q];    // the slot that takes the chunk's last entry of e
+            if (hi > b && hi < b + cnt) {                                  // this slot's quota ends inside the chunk
+                const int k = atomicAdd(&nsc[c], 1);
+                if (k < kRowSplits) {
+                    int32_t* tail = rows + (int64_t)(c0 + c) * (E + kRowTail) + E + 4 + 4 * k;
+                    tail[0] = e; tail[1] = hi - b; tail[2] = E + ent_s[q]; tail[3] = -1;
+                } else {
+                    over[atomicAdd(&s_over, 1)] = make_int4(e, hi - b, E + ent_s[q], c0 + c);   // the segment's overflow list
+                }
+            }
+        }
         __syncthreads();
+        for (int i = tid; i < nct * E; i += kThreads) {
+            const int c = i / E, e = i - c * E;
+            rows[(int64_t)(c0 + c) * (E + kRowTail) + e] = tab[i];
+        }
+        for (int c = tid; c < nct; c += kThreads) {
+            rows[(int64_t)(c0 + c) * (E + kRowTail) + E] = nsc[c];
+            a.nsg[lr * NC + c0 + c] = nsc[c];
+        }
+        __syncthreads();
+    }
+    // the overflow count is final only now: every row of the segment gets it
+    for (int c = tid; c < NC; c += kThreads) {
+        int32_t* tail = rows + (int64_t)c * (E + kRowTail) + E;
+        tail[1] = s_over; tail[2] = 0; tail[3] = 0;
     }
 }
 
+// Flat position, inside the chunk held at `buf`, of the entry of expert eb whose in-chunk ordinal is rel
+// (entries of eb before it belong to the slot whose quota ends there).  Block-wide: warp w owns entries
+// [w*2048, (w+1)*2048); per-warp counts, then ballots in the one warp that holds the entry.
 template <bool VEC>
-__global__ void __launch_bounds__(kThreads, 2)
-assign_kernel(AssignArgs a)
+__device__ int32_t locate_split(const int32_t* buf, int32_t len, int eb, int rel, int* s_cntw, int* s_pos)
 {
-    extern __shared__ int32_t sh[];
-    const int E = a.E, S = a.R * a.K;
-    int32_t* tab = sh;                  // [E]  >= 0: target for the whole chunk; -(1+b): boundary expert b
-    int32_t* base = tab + E;            // [E]  ordinal of the chunk's first entry of e within (rank, e)
-    int32_t* blist = base + E;          // [E]  boundary experts of this chunk
-    int32_t* cntw = blist + E;          // [E * kWarps] per-warp counts of each boundary expert
-    int32_t* wtab = cntw + E * kWarps;  // [kWarps][E] per-warp tables, used only if the chunk has a boundary expert
-    int32_t* ent_s = wtab + E * kWarps; // [S]  slots this source rank feeds, ascending
-    int32_t* ent_e = ent_s + S;         // [S]  their expert
-    int32_t* ent_lo = ent_e + S;        // [S]  first ordinal the slot takes
-    int32_t* ent_hi = ent_lo + S;       // [S]  one past the last
-    __shared__ int s_wcnt[kWarps];
-    __shared__ int s_nb;
-
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t id = blockIdx.x;
-    const int nb = a.nbg[id];
-    const int32_t c = (int32_t)(id % a.nc);
-    const int64_t lr = id / a.nc;
-    const int32_t l = (int32_t)(lr / a.R);
-    const int64_t start = (int64_t)c * TAOT_CHUNK;
-    const int32_t len = (int32_t)((a.seg - start) < (int64_t)TAOT_CHUNK ? (a.seg - start) : (int64_t)TAOT_CHUNK);
-    const int64_t goff = (int64_t)l * a.layer_elems + (lr % a.R) * a.seg + start;
-    const int32_t* src = a.topk + goff;
-    int32_t* dst = a.out + goff;
-    const bool full = VEC && (len == TAOT_CHUNK);
-
-    // ---- the chunk, in registers; warp w owns entries [w*2048, w*2048+2048), 128 per iteration
-    int4 x[kIters];
-    const int32_t wbase_elem = warp * kWarpSpan + lane * 4;
-    if (full) {
-#pragma unroll
-        for (int it = 0; it < kIters; ++it)
-            x[it] = ld_stream(reinterpret_cast<const int4*>(src + wbase_elem + it * 128));
-    } else {
-#pragma unroll
+    const int32_t wbase = warp * kWarpSpan + lane * 4;
+    const unsigned lt = (1u << lane) - 1u;
+    auto load4 = [&](int32_t pos) {
+        int4 v = make_int4(-1, -1, -1, -1);
+        if (VEC && pos + 3 < len) v = *reinterpret_cast<const int4*>(buf + pos);
+        else {
+            if (pos < len) v.x = buf[pos];
+            if (pos + 1 < len) v.y = buf[pos + 1];
+            if (pos + 2 < len) v.z = buf[pos + 2];
+            if (pos + 3 < len) v.w = buf[pos + 3];
+        }
+        return v;
+    };
+    int cnt = 0;
+#pragma unroll 4
+    for (int it = 0; it < kIters; ++it) {
+        const int4 v = load4(wbase + it * 128);
+        cnt += (v.x == eb) + (v.y == eb) + (v.z == eb) + (v.w == eb);
+    }
+    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    if (lane == 0) s_cntw[warp] = cnt;
+    if (tid == 0) *s_pos = 0x7fffffff;
+    __syncthreads();
+    int running = 0;
+    for (int w = 0; w < warp; ++w) running += s_cntw[w];
+    if (running <= rel && rel < running + s_cntw[warp]) {
+#pragma unroll 1
         for (int it = 0; it < kIters; ++it) {
-            const int32_t pos = wbase_elem + it * 128;
-            x[it].x = pos < len ? src[pos] : -1;
-            x[it].y = pos + 1 < len ? src[pos + 1] : -1;
-            x[it].z = pos + 2 < len ? src[pos + 2] : -1;
-            x[it].w = pos + 3 < len ? src[pos + 3] : -1;
+            const int32_t pos = wbase + it * 128;
+            const int4 v = load4(pos);
+            const bool m0 = v.x == eb, m1 = v.y == eb, m2 = v.z == eb, m3 = v.w == eb;
+            const unsigned b0 = __ballot_sync(0xffffffffu, m0), b1 = __ballot_sync(0xffffffffu, m1);
+            const unsigned b2 = __ballot_sync(0xffffffffu, m2), b3 = __ballot_sync(0xffffffffu, m3);
+            const int tot = __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
+            if (running + tot > rel) {
+                int ord = running + __popc(b0 & lt) + __popc(b1 & lt) + __popc(b2 & lt) + __popc(b3 & lt);
+                if (m0) { if (ord == rel) *s_pos = pos; ++ord; }
+                if (m1) { if (ord == rel) *s_pos = pos + 1; ++ord; }
+                if (m2) { if (ord == rel) *s_pos = pos + 2; ++ord; }
+                if (m3) { if (ord == rel) *s_pos = pos + 3; ++ord; }
+                break;
+            }
+            running += tot;
         }
     }
-
-    // ---- this chunk's table row (built by the prep kernel) and its boundary count
-    const int32_t* trow = a.tabg + id * (int64_t)E;
-    for (int e = tid; e < E; e += kThreads) tab[e] = trow[e];
     __syncthreads();
-    const int32_t* lut = tab;
+    return *s_pos;
+}
 
-    if (nb > 0) {
-        // ---- rare path: rebuild this rank's quota intervals, refine the boundary experts per warp
-        const int m = build_entries(a.X + lr * S, a.slot_expert + (int64_t)l * S, S, E, ent_s, ent_e, ent_lo, ent_hi, s_wcnt);
-        for (int q = tid; q < m; q += kThreads) ent_hi[q] += ent_lo[q];
-        const int32_t* ccseg = a.cc + lr * a.nc * (int64_t)E;
-        if (tid == 0) s_nb = 0;
-        __syncthreads();
-        for (int e = tid; e < E; e += kThreads)
-            if (tab[e] == -1) {
-                int32_t b = 0;
-                for (int cp = 0; cp < c; ++cp) b += ccseg[(int64_t)cp * E + e];
-                const int bi = atomicAdd(&s_nb, 1);
-                blist[bi] = e;
-                base[bi] = b;
-                tab[e] = e;                              // refined per warp below
-            }
-        __syncthreads();
-        // per-warp counts of the boundary experts, from the registers
-        for (int bi = 0; bi < nb; ++bi) {
-            const int eb = blist[bi];
-            int cnt = 0;
-#pragma unroll
-            for (int it = 0; it < kIters; ++it)
-                cnt += (x[it].x == eb) + (x[it].y == eb) + (x[it].z == eb) + (x[it].w == eb);
-            for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-            if (lane == 0) cntw[bi * kWarps + warp] = cnt;
+// Rewrite one chunk: `buf` holds its entries (shared memory in the pipelined kernel, global memory in the
+// plain one), `tab` its table row with tail in shared memory, `recs` is scratch for S records.  Block-wide.
+template <bool VEC>
+__device__ void rewrite_chunk(const AssignArgs& a, int64_t id, const int32_t* buf, int32_t* tab, int32_t* dst,
+                              int32_t len, int4* recs, int* s_cntw, int* s_pos)
+{
+    const int E = a.E;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t wbase = warp * kWarpSpan + lane * 4;
+    const int ns = tab[E];
+    auto emit = [&](int32_t pos, const int4& v) {
+        if (VEC) st_stream(reinterpret_cast<int4*>(dst + pos), v);
+        else {
+            if (pos < len) dst[pos] = v.x;
+            if (pos + 1 < len) dst[pos + 1] = v.y;
+            if (pos + 2 < len) dst[pos + 2] = v.z;
+            if (pos + 3 < len) dst[pos + 3] = v.w;
         }
-        int32_t* myt = wtab + warp * E;
-        for (int e = lane; e < E; e += 32) myt[e] = tab[e];
-        __syncthreads();
-        const unsigned lt = (1u << lane) - 1u;
-        for (int bi = 0; bi < nb; ++bi) {
-            const int eb = blist[bi];
-            const int32_t mine = cntw[bi * kWarps + warp];
-            int32_t running = base[bi];
-            for (int w = 0; w < warp; ++w) running += cntw[bi * kWarps + w];
-            // this warp's ordinals of eb are [running, running + mine): inside one interval, outside all, or straddling
-            int32_t target = eb;
-            bool straddle = false;
-            int q0 = m, q1 = m;
-            for (int q = 0; q < m; ++q) {
-                if (ent_e[q] != eb || mine == 0) continue;
-                if (ent_hi[q] <= running || ent_lo[q] >= running + mine) continue;
-                if (ent_lo[q] <= running && ent_hi[q] >= running + mine) target = E + ent_s[q];
-                else { straddle = true; if (q0 == m) q0 = q; q1 = q + 1; }
+    };
+    auto fetch = [&](int32_t pos) {
+        int4 v = make_int4(-1, -1, -1, -1);
+        if (VEC) v = *reinterpret_cast<const int4*>(buf + pos);
+        else {
+            if (pos < len) v.x = buf[pos];
+            if (pos + 1 < len) v.y = buf[pos + 1];
+            if (pos + 2 < len) v.z = buf[pos + 2];
+            if (pos + 3 < len) v.w = buf[pos + 3];
+        }
+        return v;
+    };
+    if (ns == 0) {
+        // ---- the common case: one table lookup per entry (values >= E or < 0 pass through unchanged)
+#pragma unroll 4
+        for (int it = 0; it < kIters; ++it) {
+            const int32_t pos = wbase + it * 128;
+            if (pos < len) {
+                int4 v = fetch(pos);
+                if ((uint32_t)v.x < (uint32_t)E) v.x = tab[v.x];
+                if ((uint32_t)v.y < (uint32_t)E) v.y = tab[v.y];
+                if ((uint32_t)v.z < (uint32_t)E) v.z = tab[v.z];
+                if ((uint32_t)v.w < (uint32_t)E) v.w = tab[v.w];
+                emit(pos, v);
             }
-            if (!straddle) {
-                if (lane == 0) myt[eb] = target;
-                continue;
-            }
+        }
+        return;
+    }
+    if (ns <= kRowSplits) {
+        // ---- a few splits: locate each, then apply them latest position first as predicated overrides
+        int32_t re[kRowSplits], rp[kRowSplits], rt[kRowSplits];
 #pragma unroll
-            for (int it = 0; it < kIters; ++it) {
-                int32_t* xv = reinterpret_cast<int32_t*>(&x[it]);
-                const bool m0 = xv[0] == eb, m1 = xv[1] == eb, m2 = xv[2] == eb, m3 = xv[3] == eb;
-                const unsigned b0 = __ballot_sync(0xffffffffu, m0), b1 = __ballot_sync(0xffffffffu, m1);
-                const unsigned b2 = __ballot_sync(0xffffffffu, m2), b3 = __ballot_sync(0xffffffffu, m3);
-                if ((b0 | b1 | b2 | b3) == 0) continue;
-                int32_t ord = running + __popc(b0 & lt) + __popc(b1 & lt) + __popc(b2 & lt) + __popc(b3 & lt);
-                const bool mm[4] = {m0, m1, m2, m3};
+        for (int k = 0; k < kRowSplits; ++k) {
+            re[k] = -1; rp[k] = -1; rt[k] = 0;            // -1 never equals a valid expert
+            if (k < ns) {                                  // uniform over the block
+                re[k] = tab[E + 4 + 4 * k];
+                rt[k] = tab[E + 4 + 4 * k + 2];
+                rp[k] = locate_split<VEC>(buf, len, re[k], tab[E + 4 + 4 * k + 1], s_cntw, s_pos);
+            }
+        }
+#pragma unroll
+        for (int x = 1; x < kRowSplits; ++x)               // sort by position, descending (unused records sink)
+#pragma unroll
+            for (int y = x; y > 0; --y)
+                if (rp[y] > rp[y - 1]) {
+                    int32_t t;
+                    t = rp[y]; rp[y] = rp[y - 1]; rp[y - 1] = t;
+                    t = re[y]; re[y] = re[y - 1]; re[y - 1] = t;
+                    t = rt[y]; rt[y] = rt[y - 1]; rt[y - 1] = t;
+                }
+#pragma unroll 2
+        for (int it = 0; it < kIters; ++it) {
+            const int32_t pos = wbase + it * 128;
+            if (pos < len) {
+                int4 v = fetch(pos);
+                int32_t* xv = reinterpret_cast<int32_t*>(&v);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    if (mm[j]) {
-                        for (int q = q0; q < q1; ++q)
-                            if (ent_e[q] == eb && ord >= ent_lo[q] && ord < ent_hi[q]) { xv[j] = E + ent_s[q]; break; }
-                        ++ord;
+                    const int32_t e = xv[j];
+                    if ((uint32_t)e < (uint32_t)E) {
+                        int32_t t = tab[e];
+#pragma unroll
+                        for (int k = 0; k < kRowSplits; ++k)
+                            if (e == re[k] && pos + j < rp[k]) t = rt[k];
+                        xv[j] = t;
                     }
                 }
-                running += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
+                emit(pos, v);
             }
-            // what is still eb in the registers stays eb; moved entries are now >= E and pass through
         }
-        __syncwarp();
-        lut = myt;
+        return;
     }
-
-    // ---- one table lookup per entry (values >= E or < 0 pass through unchanged), then store
-    if (full) {
-#pragma unroll
-        for (int it = 0; it < kIters; ++it) {
-            int32_t* xv = reinterpret_cast<int32_t*>(&x[it]);
+    // ---- many splits in one chunk (rare): all records into shared memory, located one by one, then a list walk
+    const int c = (int)(id % a.nc);
+    const int4* over = a.splits + (id / a.nc) * (int64_t)(a.R * a.K);
+    const int nover = tab[E + 1];
+    __shared__ int s_n;
+    if (tid == 0) s_n = 0;
+    __syncthreads();
+    for (int k = tid; k < kRowSplits; k += blockDim.x)
+        recs[atomicAdd(&s_n, 1)] = make_int4(tab[E + 4 + 4 * k], tab[E + 4 + 4 * k + 1], tab[E + 4 + 4 * k + 2], -1);
+    for (int q = tid; q < nover; q += blockDim.x) {
+        const int4 r = over[q];
+        if (r.w == c) recs[atomicAdd(&s_n, 1)] = make_int4(r.x, r.y, r.z, -1);
+    }
+    __syncthreads();
+    const int nrec = s_n;
+    for (int k = 0; k < nrec; ++k) {
+        const int32_t P = locate_split<VEC>(buf, len, recs[k].x, recs[k].y, s_cntw, s_pos);
+        if (tid == 0) recs[k].w = P;
+    }
+    __syncthreads();
+    for (int k = tid; k < nrec; k += blockDim.x) {      // mark the experts that have a split: -1 - target
+        const int32_t e = recs[k].x;
+        const int32_t t = tab[e];
+        if (t >= 0) tab[e] = -1 - t;
+    }
+    __syncthreads();
+#pragma unroll 1
+    for (int it = 0; it < kIters; ++it) {
+        const int32_t pos = wbase + it * 128;
+        if (pos < len) {
+            int4 v = fetch(pos);
+            int32_t* xv = reinterpret_cast<int32_t*>(&v);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int32_t e = xv[j];
-                if ((uint32_t)e < (uint32_t)E) xv[j] = lut[e];
+                if ((uint32_t)e >= (uint32_t)E) continue;
+                int32_t t = tab[e];
+                if (t < 0) {                               // nearest split after this position, else the final target
+                    int32_t best = 0x7fffffff;
+                    t = -1 - t;
+                    for (int k = 0; k < nrec; ++k) {
+                        const int4 r = recs[k];
+                        if (r.x == e && pos + j < r.w && r.w < best) { best = r.w; t = r.z; }
+                    }
+                }
+                xv[j] = t;
             }
-            st_stream(reinterpret_cast<int4*>(dst + wbase_elem + it * 128), x[it]);
-        }
-    } else {
-#pragma unroll
-        for (int it = 0; it < kIters; ++it) {
-            int32_t* xv = reinterpret_cast<int32_t*>(&x[it]);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int32_t e = xv[j];
-                if ((uint32_t)e < (uint32_t)E) xv[j] = lut[e];
-            }
-            const int32_t pos = wbase_elem + it * 128;
-            if (pos < len) dst[pos] = x[it].x;
-            if (pos + 1 < len) dst[pos + 1] = x[it].y;
-            if (pos + 2 < len) dst[pos + 2] = x[it].z;
-            if (pos + 3 < len) dst[pos + 3] = x[it].w;
+            emit(pos, v);
         }
     }
 }
 
 // ---------------------------------------------------------------------------------------------
-// Persistent, bulk-copy-pipelined version of the rewrite (used when the routing table is 16-byte
-// aligned and E is a multiple of 4).  One CTA per SM walks chunks blockIdx.x, +gridDim.x, ...; a
-// single thread keeps kStages-1 chunks in flight with cp.async.bulk (global -> shared, completion
-// counted on an mbarrier per stage, no multicast), so the loads of the next chunks overlap the
-// lookups and stores of the current one.  Each stage carries the chunk (<= 64 KB) and its table row.
-// Arithmetic and rare path are those of assign_kernel; the chunk is read from shared memory
-// instead of registers.
+// persistent bulk-copy pipeline
 
-constexpr int kSThreads = 256;
-constexpr int kSWarps = kSThreads / 32;
-constexpr int kSWarpSpan = TAOT_CHUNK / kSWarps;        // 2048 entries per warp, contiguous
-constexpr int kSIters = kSWarpSpan / 128;               // 16 x 16-byte accesses per lane
-constexpr uint32_t kBulkPiece = 8192;                   // bytes per bulk copy: several pieces in flight per chunk
 constexpr uint32_t kWaitSpins = 1u << 20;               // bound on mbarrier polling (each poll can itself block for a while)
+constexpr uint32_t kBulkPiece = 8192;                   // bytes per bulk copy: several pieces in flight per chunk
+constexpr int kMaxStages = 4;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -341,43 +409,81 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
     return false;
 }
 
+// One CTA per chunk.  STAGE: the chunk is first copied to shared memory with bulk asynchronous copies (used for
+// the chunks that hold a split, whose entries are read three times: count, locate, rewrite); otherwise it is read
+// from global memory (any alignment).
+template <bool VEC, bool STAGE>
+__global__ void __launch_bounds__(kThreads)
+assign_chunk_kernel(AssignArgs a, int only_split)
+{
+    extern __shared__ __align__(128) unsigned char shc[];
+    const int E = a.E;
+    int32_t* stage = reinterpret_cast<int32_t*>(shc);                      // [TAOT_CHUNK] if STAGE
+    int32_t* tab = reinterpret_cast<int32_t*>(shc + (STAGE ? (size_t)TAOT_CHUNK * 4 : 0));   // [E + kRowTail]
+    int4* recs = reinterpret_cast<int4*>(tab + ((E + kRowTail + 3) & ~3));
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int s_cntw[kWarps];
+    __shared__ int s_pos;
+    const int tid = threadIdx.x;
+    const int64_t id = blockIdx.x;
+    if (only_split && a.nsg[id] == 0) return;            // the pipelined kernel rewrites the chunks without splits
+    int64_t goff; int32_t len;
+    chunk_geometry(a, id, goff, len);
+    const int32_t* buf = a.topk + goff;
+    if (STAGE) {
+        if (tid == 0) {
+            mbar_init(&bar, 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            const uint32_t bytes = (uint32_t)len * 4u;
+            mbar_expect_tx(&bar, bytes);
+            for (uint32_t o = 0; o < bytes; o += kBulkPiece)
+                bulk_load(reinterpret_cast<unsigned char*>(stage) + o, reinterpret_cast<const unsigned char*>(buf) + o,
+                          (bytes - o) < kBulkPiece ? (bytes - o) : kBulkPiece, &bar);
+        }
+        buf = stage;
+    }
+    const int32_t* trow = a.tabg + id * (int64_t)(E + kRowTail);
+    for (int e = tid; e < E + kRowTail; e += kThreads) tab[e] = trow[e];
+    __syncthreads();                                     // table row in place; the barrier is initialised
+    if (STAGE) {
+        const bool ok = mbar_wait(&bar, 0);
+        if (__syncthreads_or(!ok)) {                     // the copy never landed: report and leave (bounded wait already spent)
+            if (tid == 0) atomicOr(a.info + (int32_t)((id / a.nc) / a.R), TAOT_INFO_INTERNAL);
+            return;
+        }
+    }
+    rewrite_chunk<VEC>(a, id, buf, tab, a.out + goff, len, recs, s_cntw, &s_pos);
+}
+
 struct StreamLayout {
     int stages;
-    size_t off_tab, off_scratch, bytes;       // chunk buffers start at 0
+    size_t off_tab, off_recs, bytes;          // chunk buffers start at 0
 };
 
 StreamLayout stream_layout(int E, int S)
 {
-    const size_t scratch = sizeof(int32_t) * ((size_t)E * (2 + 2 * kSWarps) + 4 * (size_t)S);   // base, blist, cntw, wtab, ent_*
+    const size_t recs = sizeof(int4) * (size_t)(S + kRowSplits);
+    const size_t per_stage = (size_t)TAOT_CHUNK * 4 + (size_t)(E + kRowTail) * 4;
+    const size_t budget = 224 * 1024;
     StreamLayout L;
-    const size_t per_stage = (size_t)TAOT_CHUNK * 4 + (size_t)E * 4;
-    const size_t budget = 220 * 1024;
-    int st = (int)((budget - scratch - 256) / per_stage);
-    L.stages = st > 4 ? 4 : st;
+    int st = (int)((budget - recs - 256) / per_stage);
+    L.stages = st > kMaxStages ? kMaxStages : st;
     L.off_tab = (size_t)L.stages * TAOT_CHUNK * 4;
-    L.off_scratch = L.off_tab + (size_t)L.stages * E * 4;
-    L.bytes = L.off_scratch + scratch;
+    L.off_recs = taot_align_up(L.off_tab + (size_t)L.stages * (E + kRowTail) * 4, 16);
+    L.bytes = L.off_recs + recs;
     return L;
 }
 
-__global__ void __launch_bounds__(kSThreads, 1)
-assign_stream_kernel(AssignArgs a, int stages, uint32_t off_tab, uint32_t off_scratch, int64_t nchunks)
+__global__ void __launch_bounds__(kThreads, 1)
+assign_stream_kernel(AssignArgs a, int stages, uint32_t off_tab, uint32_t off_recs, int64_t nchunks)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ __align__(8) uint64_t bars[4];
-    __shared__ int s_wcnt[32];
-    __shared__ int s_nb;
-    const int E = a.E, S = a.R * a.K;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    int32_t* scratch = reinterpret_cast<int32_t*>(smem + off_scratch);
-    int32_t* base = scratch;                    // [E]  start ordinal of each boundary expert (indexed by its list position)
-    int32_t* blist = base + E;                  // [E]
-    int32_t* cntw = blist + E;                  // [E * kSWarps]
-    int32_t* wtab = cntw + E * kSWarps;         // [kSWarps][E]
-    int32_t* ent_s = wtab + E * kSWarps;        // [S] ...
-    int32_t* ent_e = ent_s + S;
-    int32_t* ent_lo = ent_e + S;
-    int32_t* ent_hi = ent_lo + S;
+    __shared__ __align__(8) uint64_t bars[kMaxStages];
+    __shared__ int s_cntw[kWarps];
+    __shared__ int s_pos;
+    const int E = a.E;
+    const int tid = threadIdx.x;
+    int4* recs = reinterpret_cast<int4*>(smem + off_recs);
 
     if (tid == 0) {
         for (int st = 0; st < stages; ++st) mbar_init(&bars[st], 1);
@@ -385,42 +491,41 @@ assign_stream_kernel(AssignArgs a, int stages, uint32_t off_tab, uint32_t off_sc
     }
     __syncthreads();
 
-    auto chunk_geometry = [&](int64_t id, int64_t& goff, int32_t& len) {
-        const int32_t c = (int32_t)(id % a.nc);
-        const int64_t lr = id / a.nc;
-        const int64_t start = (int64_t)c * TAOT_CHUNK;
-        len = (int32_t)((a.seg - start) < (int64_t)TAOT_CHUNK ? (a.seg - start) : (int64_t)TAOT_CHUNK);
-        goff = (lr / a.R) * a.layer_elems + (lr % a.R) * a.seg + start;
-    };
-    auto issue = [&](int64_t id, int st) {      // one thread: arm the stage and start its two copies
+    auto issue = [&](int64_t id, int st) {      // one thread: arm the stage and start the copies of chunk and table row
         int64_t goff; int32_t len;
-        chunk_geometry(id, goff, len);
+        chunk_geometry(a, id, goff, len);
         const uint32_t bytes = (uint32_t)len * 4u;
-        mbar_expect_tx(&bars[st], bytes + (uint32_t)E * 4u);
+        mbar_expect_tx(&bars[st], bytes + (uint32_t)(E + kRowTail) * 4u);
         unsigned char* dstb = smem + (size_t)st * TAOT_CHUNK * 4;
         const unsigned char* srcb = reinterpret_cast<const unsigned char*>(a.topk + goff);
         for (uint32_t o = 0; o < bytes; o += kBulkPiece)
             bulk_load(dstb + o, srcb + o, (bytes - o) < kBulkPiece ? (bytes - o) : kBulkPiece, &bars[st]);
-        bulk_load(smem + off_tab + (size_t)st * E * 4, a.tabg + id * (int64_t)E, (uint32_t)E * 4u, &bars[st]);
+        bulk_load(smem + off_tab + (size_t)st * (E + kRowTail) * 4, a.tabg + id * (int64_t)(E + kRowTail), (uint32_t)(E + kRowTail) * 4u, &bars[st]);
     };
 
-    const int64_t first = blockIdx.x, stride = gridDim.x;
-    if (tid == 0)
+    // this CTA's chunks: blockIdx.x, +gridDim.x, ... without the ones that hold a split (those need block-wide
+    // counting with barriers, which would stall the pipeline; a second kernel rewrites them)
+    const int64_t stride = gridDim.x;
+    auto advance = [&](int64_t id) {
+        while (id < nchunks && a.nsg[id] != 0) id += stride;
+        return id;
+    };
+    int64_t iss_id = 0;                          // thread 0: next chunk to start copying
+    int64_t id = advance(blockIdx.x);
+    if (tid == 0) {
+        iss_id = id;
         for (int st = 0; st < stages; ++st)
-            if (first + st * stride < nchunks) issue(first + st * stride, st);
+            if (iss_id < nchunks) { issue(iss_id, st); iss_id = advance(iss_id + stride); }
+    }
 
-    int64_t it_global = 0;
-    for (int64_t id = first; id < nchunks; id += stride, ++it_global) {
-        const int st = (int)(it_global % stages);
-        const uint32_t parity = (uint32_t)((it_global / stages) & 1);
-        const int nb = a.nbg[id];
+    int64_t use = 0;
+    for (; id < nchunks; id = advance(id + stride), ++use) {
+        const int st = (int)(use % stages);
+        const uint32_t parity = (uint32_t)((use / stages) & 1);
         int64_t goff; int32_t len;
-        chunk_geometry(id, goff, len);
-        const int64_t lr = id / a.nc;
-        const int32_t c = (int32_t)(id % a.nc);
-        const int32_t l = (int32_t)(lr / a.R);
-        int32_t* buf = reinterpret_cast<int32_t*>(smem + (size_t)st * TAOT_CHUNK * 4);
-        const int32_t* tab = reinterpret_cast<const int32_t*>(smem + off_tab + (size_t)st * E * 4);
+        chunk_geometry(a, id, goff, len);
+        const int32_t* buf = reinterpret_cast<const int32_t*>(smem + (size_t)st * TAOT_CHUNK * 4);
+        int32_t* tab = reinterpret_cast<int32_t*>(smem + off_tab + (size_t)st * (E + kRowTail) * 4);
         int32_t* dst = a.out + goff;
 
         const bool ok = mbar_wait(&bars[st], parity);
@@ -428,167 +533,73 @@ assign_stream_kernel(AssignArgs a, int stages, uint32_t off_tab, uint32_t off_sc
             // the copy never completed: report, give the copies still in flight one more bounded chance to land
             // (their destination is this CTA's shared memory), and leave
             if (tid == 0) {
-                atomicOr(a.info + l, TAOT_INFO_INTERNAL);
+                atomicOr(a.info + (int32_t)((id / a.nc) / a.R), TAOT_INFO_INTERNAL);
                 for (int s2 = 0; s2 < stages; ++s2) {
-                    const int64_t use = (it_global + ((s2 - st + stages) % stages)) / stages;
-                    (void)mbar_wait(&bars[s2], (uint32_t)(use & 1));
+                    const int64_t u2 = (use + ((s2 - st + stages) % stages)) / stages;
+                    (void)mbar_wait(&bars[s2], (uint32_t)(u2 & 1));
                 }
             }
             __syncthreads();
             return;
         }
-        const int32_t wbase = warp * kSWarpSpan + lane * 4;
-        const int32_t* lut = tab;
-        if (nb > 0) {
-            // ---- rare path: this rank's quota intervals, per-warp refinement of the boundary experts
-            const int m = build_entries(a.X + lr * S, a.slot_expert + (int64_t)l * S, S, E, ent_s, ent_e, ent_lo, ent_hi, s_wcnt);
-            for (int q = tid; q < m; q += kSThreads) ent_hi[q] += ent_lo[q];
-            const int32_t* ccseg = a.cc + lr * a.nc * (int64_t)E;
-            if (tid == 0) s_nb = 0;
-            __syncthreads();
-            for (int e = tid; e < E; e += kSThreads)
-                if (tab[e] == -1) {
-                    int32_t b = 0;
-                    for (int cp = 0; cp < c; ++cp) b += ccseg[(int64_t)cp * E + e];
-                    const int bi = atomicAdd(&s_nb, 1);
-                    blist[bi] = e;
-                    base[bi] = b;
-                }
-            __syncthreads();
-#pragma unroll 1
-            for (int bi = 0; bi < nb; ++bi) {
-                const int eb = blist[bi];
-                int cnt = 0;
-#pragma unroll 4
-                for (int it = 0; it < kSIters; ++it) {
-                    const int32_t pos = wbase + it * 128;
-                    if (pos < len) {
-                        const int4 v = *reinterpret_cast<const int4*>(buf + pos);
-                        cnt += (v.x == eb) + (v.y == eb) + (v.z == eb) + (v.w == eb);
-                    }
-                }
-                for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-                if (lane == 0) cntw[bi * kSWarps + warp] = cnt;
-            }
-            int32_t* myt = wtab + warp * E;
-            for (int e = lane; e < E; e += 32) { const int32_t t = tab[e]; myt[e] = t == -1 ? e : t; }
-            __syncthreads();
-            const unsigned lt = (1u << lane) - 1u;
-#pragma unroll 1
-            for (int bi = 0; bi < nb; ++bi) {
-                const int eb = blist[bi];
-                const int32_t mine = cntw[bi * kSWarps + warp];
-                int32_t running = base[bi];
-                for (int w = 0; w < warp; ++w) running += cntw[bi * kSWarps + w];
-                // this warp's ordinals of eb are [running, running + mine): inside one interval, outside all, or
-                // straddling; the (at most two, else a list walk) intervals it straddles are kept in registers
-                int32_t target = eb;
-                int nstr = 0, q0 = m, q1 = m;
-                int32_t lo0 = 0, hi0 = 0, t0 = eb, lo1 = 0, hi1 = 0, t1 = eb;
-                for (int q = 0; q < m; ++q) {
-                    if (ent_e[q] != eb || mine == 0) continue;
-                    if (ent_hi[q] <= running || ent_lo[q] >= running + mine) continue;
-                    if (ent_lo[q] <= running && ent_hi[q] >= running + mine) { target = E + ent_s[q]; continue; }
-                    if (nstr == 0) { lo0 = ent_lo[q]; hi0 = ent_hi[q]; t0 = E + ent_s[q]; q0 = q; }
-                    else if (nstr == 1) { lo1 = ent_lo[q]; hi1 = ent_hi[q]; t1 = E + ent_s[q]; }
-                    ++nstr;
-                    q1 = q + 1;
-                }
-                if (nstr == 0) {
-                    if (lane == 0) myt[eb] = target;
-                    continue;
-                }
-#pragma unroll 1
-                for (int it = 0; it < kSIters; ++it) {           // kept rolled: this code runs rarely and must stay small
-                    const int32_t pos = wbase + it * 128;
-                    int4 v = make_int4(-1, -1, -1, -1);
-                    if (pos < len) v = *reinterpret_cast<const int4*>(buf + pos);
-                    int32_t* xv = reinterpret_cast<int32_t*>(&v);
-                    const bool m0 = xv[0] == eb, m1 = xv[1] == eb, m2 = xv[2] == eb, m3 = xv[3] == eb;
-                    const unsigned b0 = __ballot_sync(0xffffffffu, m0), b1 = __ballot_sync(0xffffffffu, m1);
-                    const unsigned b2 = __ballot_sync(0xffffffffu, m2), b3 = __ballot_sync(0xffffffffu, m3);
-                    if ((b0 | b1 | b2 | b3) == 0) continue;
-                    int32_t ord = running + __popc(b0 & lt) + __popc(b1 & lt) + __popc(b2 & lt) + __popc(b3 & lt);
-                    const bool mm[4] = {m0, m1, m2, m3};
-                    bool changed = false;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        if (mm[j]) {
-                            if (nstr <= 2) {
-                                if (ord >= lo0 && ord < hi0) { xv[j] = t0; changed = true; }
-                                else if (nstr == 2 && ord >= lo1 && ord < hi1) { xv[j] = t1; changed = true; }
-                            } else {
-                                for (int q = q0; q < q1; ++q)
-                                    if (ent_e[q] == eb && ord >= ent_lo[q] && ord < ent_hi[q]) { xv[j] = E + ent_s[q]; changed = true; break; }
-                            }
-                            ++ord;
-                        }
-                    }
-                    if (changed) *reinterpret_cast<int4*>(buf + pos) = v;        // moved entries are now >= E and pass through
-                    running += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
-                }
-            }
-            __syncwarp();
-            lut = myt;
-        }
-        // ---- one table lookup per entry (values >= E or < 0 pass through unchanged), then store
-#pragma unroll 4
-        for (int it = 0; it < kSIters; ++it) {
-            const int32_t pos = wbase + it * 128;
-            if (pos < len) {
-                int4 v = *reinterpret_cast<const int4*>(buf + pos);
-#ifndef TAOT_DBG_NOLOOKUP
-                if ((uint32_t)v.x < (uint32_t)E) v.x = lut[v.x];
-                if ((uint32_t)v.y < (uint32_t)E) v.y = lut[v.y];
-                if ((uint32_t)v.z < (uint32_t)E) v.z = lut[v.z];
-                if ((uint32_t)v.w < (uint32_t)E) v.w = lut[v.w];
-#endif
-#ifdef TAOT_DBG_NOSTORE
-                if (v.x == 0x7fffffff)
-#endif
-                st_stream(reinterpret_cast<int4*>(dst + pos), v);
-            }
-        }
+        rewrite_chunk<true>(a, id, buf, tab, dst, len, recs, s_cntw, &s_pos);
         __syncthreads();                         // everyone is done with this stage's buffers
-        if (tid == 0 && id + (int64_t)stages * stride < nchunks) {
+        if (tid == 0 && iss_id < nchunks) {
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            issue(id + (int64_t)stages * stride, st);
+            issue(iss_id, st);
+            iss_id = advance(iss_id + stride);
         }
     }
 }
 
 }  // namespace
 
-int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_cc, int32_t* d_tabg,
-                       int32_t* d_nbg, const int32_t* d_slot_expert, const int32_t* d_X, int32_t* d_new_idx,
-                       int32_t* d_info, cudaStream_t st)
+int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, void* ws, const int32_t* d_slot_expert,
+                       const int32_t* d_X, int32_t* d_new_idx, int32_t* d_info, cudaStream_t st)
 {
     const taot_params& p = h->p;
+    char* w = static_cast<char*>(ws);
     AssignArgs a;
-    a.topk = d_topk; a.cc = d_cc; a.tabg = d_tabg; a.nbg = d_nbg;
+    a.topk = d_topk;
+    a.cc = reinterpret_cast<const int32_t*>(w + h->off_cc);
+    a.tabg = reinterpret_cast<int32_t*>(w + h->off_tabg);
+    a.nsg = reinterpret_cast<int32_t*>(w + h->off_nbg);
+    a.soff = reinterpret_cast<int32_t*>(w + h->off_soff);
+    a.splits = reinterpret_cast<int4*>(w + h->off_splits);
     a.slot_expert = d_slot_expert; a.X = d_X; a.out = d_new_idx; a.info = d_info;
     a.layer_elems = p.T * p.k; a.seg = h->seg; a.nc = h->nc; a.R = p.R; a.E = p.E; a.K = p.K;
-    a.vec_ok = ((reinterpret_cast<uintptr_t>(d_topk) & 15) == 0) &&
-               ((reinterpret_cast<uintptr_t>(d_new_idx) & 15) == 0) && (h->seg % 4 == 0);
+    const int vec_ok = ((reinterpret_cast<uintptr_t>(d_topk) & 15) == 0) &&
+                       ((reinterpret_cast<uintptr_t>(d_new_idx) & 15) == 0) && (h->seg % 4 == 0);
     const int S = p.R * p.K;
-    const size_t smem_prep = sizeof(int32_t) * (2 * (size_t)p.E + 4 * (size_t)S);
+    const unsigned blocks = (unsigned)((int64_t)p.L * p.R * h->nc);
+    const int nct = prep_tile(p.E) < h->nc ? prep_tile(p.E) : h->nc;
+    const size_t smem_prep = sizeof(int32_t) * (4 * (size_t)S + (size_t)p.E + 3 * (size_t)nct * p.E + nct);
+    TAOT_CUDA_OK(cudaFuncSetAttribute(assign_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_prep));
     assign_prep_kernel<<<(unsigned)((int64_t)p.L * p.R), kThreads, smem_prep, st>>>(a);
     TAOT_CUDA_OK(cudaGetLastError());
-    const size_t smem = sizeof(int32_t) * ((size_t)p.E * (3 + 2 * kWarps) + 4 * (size_t)S);
-    const unsigned blocks = (unsigned)((int64_t)p.L * p.R * h->nc);
     const StreamLayout sl = stream_layout(p.E, S);
-    if (a.vec_ok && p.E % 4 == 0 && sl.stages >= 2) {
+    int launches = 2;
+    if (vec_ok && p.E % 4 == 0 && sl.stages >= 2) {
         TAOT_CUDA_OK(cudaFuncSetAttribute(assign_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sl.bytes));
         const unsigned grid = blocks < (unsigned)h->sm_count ? blocks : (unsigned)h->sm_count;
-        assign_stream_kernel<<<grid, kSThreads, sl.bytes, st>>>(a, sl.stages, (uint32_t)sl.off_tab, (uint32_t)sl.off_scratch,
-                                                              (int64_t)blocks);
-    } else if (a.vec_ok) {
-        TAOT_CUDA_OK(cudaFuncSetAttribute(assign_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        assign_kernel<true><<<blocks, kThreads, smem, st>>>(a);
+        assign_stream_kernel<<<grid, kThreads, sl.bytes, st>>>(a, sl.stages, (uint32_t)sl.off_tab, (uint32_t)sl.off_recs,
+                                                             (int64_t)blocks);
+        TAOT_CUDA_OK(cudaGetLastError());
+        const size_t smem = (size_t)TAOT_CHUNK * 4 + sizeof(int32_t) * (((size_t)p.E + kRowTail + 3) & ~(size_t)3) +
+                            sizeof(int4) * (size_t)(S + kRowSplits);
+        TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        assign_chunk_kernel<true, true><<<blocks, kThreads, smem, st>>>(a, 1);      // the chunks that hold a split
+        launches = 3;
     } else {
-        TAOT_CUDA_OK(cudaFuncSetAttribute(assign_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        assign_kernel<false><<<blocks, kThreads, smem, st>>>(a);
+        const size_t smem = sizeof(int32_t) * (((size_t)p.E + kRowTail + 3) & ~(size_t)3) + sizeof(int4) * (size_t)(S + kRowSplits);
+        if (vec_ok) {
+            TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            assign_chunk_kernel<true, false><<<blocks, kThreads, smem, st>>>(a, 0);
+        } else {
+            TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            assign_chunk_kernel<false, false><<<blocks, kThreads, smem, st>>>(a, 0);
+        }
     }
     TAOT_CUDA_OK(cudaGetLastError());
-    return 2;
+    return launches;
 }

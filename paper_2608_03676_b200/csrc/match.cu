@@ -136,10 +136,6 @@ match_kernel(MatchArgs a)
     int32_t* nrem_s = reinterpret_cast<int32_t*>(tm_s + (a.tm_in_smem ? a.ntiers * W * S : 0));   // [dmax*R] if it fits
     __shared__ long long s_tot;
     __shared__ int s_cnt, s_any;
-#ifdef TAOT_DEBUG_CLOCKS
-    __shared__ long long s_dbg[5];
-    if (threadIdx.x < 5) s_dbg[threadIdx.x] = 0;
-#endif
 
     const int32_t* n = a.n + l * (int64_t)R * E;
     const int32_t* el = a.expert_load + l * E;
@@ -340,18 +336,11 @@ match_kernel(MatchArgs a)
             }
         }
         int prev_r = -1;                         // rank whose arbiter entry this slot won last round
-#ifdef TAOT_DEBUG_CLOCKS
-        long long dbg[5] = {0, 0, 0, 0, 0};
-        int dbg_levels = 0, dbg_bits = 0, dbg_tiers = 0; (void)dbg_levels; (void)dbg_bits; (void)dbg_tiers;
-#endif
         for (;;) {
             if (a.auction_max_rounds > 0 && rounds3 >= a.auction_max_rounds) break;
             if (rounds3 >= cap) break;
             u64* arb = arb_r + (rounds3 & 1) * R;
             // Step 1: bid for the source rank with the best bonus minus price
-#ifdef TAOT_DEBUG_CLOCKS
-            __syncwarp(); const long long c0 = clock64();
-#endif
             u64 key = 0;
             if (live) {
 #pragma unroll
@@ -409,18 +398,9 @@ match_kernel(MatchArgs a)
                 }
             }
             // Step 2: the rank keeps its best bidder (ties: lowest slot)
-#ifdef TAOT_DEBUG_CLOCKS
-            __syncwarp(); const long long c1 = clock64();
-#endif
             const int rsel = (int)(0xFFFFFFFFu - (uint32_t)key);
             arbitrate(arb, rsel, key == 0 ? 0ull : ((key & 0xFFFFFFFF00000000ull) | (u64)(0xFFFFFFFFu - (uint32_t)s)));
-#ifdef TAOT_DEBUG_CLOCKS
-            __syncwarp(); const long long c2 = clock64();
-#endif
             if (!__syncthreads_or(key != 0)) break;
-#ifdef TAOT_DEBUG_CLOCKS
-            __syncwarp(); const long long c3 = clock64();
-#endif
             if (prev_r >= 0) { arb_r[((rounds3 & 1) ^ 1) * R + prev_r] = 0; prev_r = -1; }
             // Steps 3-4: the winning slot of each rank collects x = min(n, A); holdings, plan and price follow
             if (key != 0 && (uint32_t)arb[rsel] == 0xFFFFFFFFu - (uint32_t)s) {
@@ -442,23 +422,8 @@ match_kernel(MatchArgs a)
                 if (A <= 0) live = false;
             }
             ++rounds3;
-#ifdef TAOT_DEBUG_CLOCKS
-            __syncwarp(); const long long c4 = clock64();
-#endif
             __syncthreads();
-#ifdef TAOT_DEBUG_CLOCKS
-            const long long c5 = clock64();
-            dbg[0] += c1 - c0; dbg[1] += c2 - c1; dbg[2] += c3 - c2; dbg[3] += c4 - c3; dbg[4] += c5 - c4;
-#endif
         }
-#ifdef TAOT_DEBUG_CLOCKS
-        for (int i = 0; i < 5; ++i) atomicMax(reinterpret_cast<u64*>(&s_dbg[i]), (u64)dbg[i]);
-        __syncthreads();
-        if (l == 0 && a.rounds) {   // per-thread totals into the tail of X of the LAST layer (debug only)
-            int32_t* dump = a.X + (int64_t)(gridDim.x - 1) * R * S;
-            dump[tid] = (int)(dbg[0] / 1000); dump[NT + tid] = (int)(dbg[1] / 1000); dump[2 * NT + tid] = (int)(dbg[2] / 1000); dump[3*NT + tid] = (int)(dbg[3] / 1000); dump[4*NT + tid] = (int)(dbg[4] / 1000);
-        }
-#endif
         if (s < S) slot_a[s] = A;
         __syncthreads();
     } else {
@@ -522,9 +487,6 @@ match_kernel(MatchArgs a)
     residual = __syncthreads_or(residual);
     if (tid == 0) {
         if (a.rounds) { a.rounds[l * 2] = rounds2; a.rounds[l * 2 + 1] = rounds3; }
-#ifdef TAOT_DEBUG_CLOCKS
-        if (a.rounds && l < 5) { a.rounds[l * 2] = (int)(s_dbg[l] / 1000); a.rounds[l * 2 + 1] = rounds3; }
-#endif
         if (residual) atomicOr(a.info + l, TAOT_INFO_AUCTION_RESIDUAL);
     }
 }
