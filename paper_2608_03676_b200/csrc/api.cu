@@ -60,6 +60,7 @@ void layout(taot_handle_t h)
     h->off_tabg = take(sizeof(int32_t) * LR * h->nc * (p.E + 20));   // E targets + row tail (assign.cu: kRowTail)
     h->off_nbg = take(sizeof(int32_t) * LR * h->nc);
     h->off_soff = take(sizeof(int32_t) * LR * h->nc);
+    h->off_work = take(16);
     h->off_splits = take(16 * LR * (size_t)p.R * p.K);
     h->off_excess = take(sizeof(int32_t) * LR);
     h->off_spare = take(sizeof(int32_t) * LR);

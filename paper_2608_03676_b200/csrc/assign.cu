@@ -45,6 +45,7 @@ struct AssignArgs {
     const int32_t* X;
     int32_t* out;
     int32_t* info;
+    unsigned long long* work;   // chunk counter of the pipelined kernel (zeroed by the prep kernel)
     int64_t layer_elems, seg;
     int32_t nc, R, E, K;
 };
@@ -128,6 +129,7 @@ assign_prep_kernel(AssignArgs a)
     int4* over = a.splits + lr * S;
     for (int e = tid; e < E; e += kThreads) carry[e] = 0;
     if (tid == 0) s_over = 0;
+    if (tid == 0 && blockIdx.x == 0) *a.work = 0ull;
     const int m = build_entries(a.X + lr * S, a.slot_expert + (int64_t)l * S, S, E, ent_s, ent_e, ent_lo, ent_hi, s_wcnt);
     for (int c0 = 0; c0 < NC; c0 += NCT) {
         const int nct = (NC - c0) < NCT ? (NC - c0) : NCT;
@@ -455,100 +457,135 @@ assign_chunk_kernel(AssignArgs a, int only_split)
     rewrite_chunk<VEC>(a, id, buf, tab, a.out + goff, len, recs, s_cntw, &s_pos);
 }
 
+// ---- the pipelined kernel ----
+constexpr int kStreamConsumers = 512;                    // threads that rewrite; one more warp only starts copies
+constexpr int kStreamThreads = kStreamConsumers + 32;
+constexpr int kStreamUnroll = 4;
+
 struct StreamLayout {
     int stages;
-    size_t off_tab, off_recs, bytes;          // chunk buffers start at 0
+    size_t off_tab, bytes;                    // chunk buffers start at 0
 };
 
-StreamLayout stream_layout(int E, int S)
+StreamLayout stream_layout(int E)
 {
-    const size_t recs = sizeof(int4) * (size_t)(S + kRowSplits);
-    const size_t per_stage = (size_t)TAOT_CHUNK * 4 + (size_t)(E + kRowTail) * 4;
+    const size_t per_stage = (size_t)TAOT_CHUNK * 4 + (size_t)E * 4;
     const size_t budget = 224 * 1024;
     StreamLayout L;
-    int st = (int)((budget - recs - 256) / per_stage);
+    int st = (int)((budget - 256) / per_stage);
     L.stages = st > kMaxStages ? kMaxStages : st;
     L.off_tab = (size_t)L.stages * TAOT_CHUNK * 4;
-    L.off_recs = taot_align_up(L.off_tab + (size_t)L.stages * (E + kRowTail) * 4, 16);
-    L.bytes = L.off_recs + recs;
+    L.bytes = L.off_tab + (size_t)L.stages * E * 4;
     return L;
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
-assign_stream_kernel(AssignArgs a, int stages, uint32_t off_tab, uint32_t off_recs, int64_t nchunks)
+// Persistent, one CTA per SM.  Warp 0 is the producer: one lane claims the next chunk without a split from a
+// global counter, arms the stage's "full" barrier and starts the bulk copies of the chunk and of its table row.
+// The other warps are consumers: wait for "full", rewrite the chunk (one table lookup per entry, 16-byte
+// streaming stores), and arrive on the stage's "empty" barrier, which the producer waits on before it reuses
+// the stage.  No CTA-wide barrier inside the loop.  Every wait is bounded; a wait that runs out sets
+// TAOT_INFO_INTERNAL, stops the CTA's loop, and the CTA leaves after one more bounded wait per armed stage.
+__global__ void __launch_bounds__(kStreamThreads, 1)
+assign_stream_kernel(AssignArgs a, int stages, uint32_t off_tab, int64_t nchunks, unsigned long long* work)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ __align__(8) uint64_t bars[kMaxStages];
-    __shared__ int s_cntw[kWarps];
-    __shared__ int s_pos;
+    __shared__ __align__(8) uint64_t full[kMaxStages];
+    __shared__ __align__(8) uint64_t empty[kMaxStages];
+    __shared__ long long s_id[kMaxStages];               // chunk staged in each stage, -1 = no more work
+    __shared__ int s_abort;
     const int E = a.E;
     const int tid = threadIdx.x;
-    int4* recs = reinterpret_cast<int4*>(smem + off_recs);
+    const int warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
-        for (int st = 0; st < stages; ++st) mbar_init(&bars[st], 1);
+        for (int st = 0; st < stages; ++st) { mbar_init(&full[st], 1); mbar_init(&empty[st], kStreamConsumers / 32); }
+        s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
 
-    auto issue = [&](int64_t id, int st) {      // one thread: arm the stage and start the copies of chunk and table row
-        int64_t goff; int32_t len;
-        chunk_geometry(a, id, goff, len);
-        const uint32_t bytes = (uint32_t)len * 4u;
-        mbar_expect_tx(&bars[st], bytes + (uint32_t)(E + kRowTail) * 4u);
-        unsigned char* dstb = smem + (size_t)st * TAOT_CHUNK * 4;
-        const unsigned char* srcb = reinterpret_cast<const unsigned char*>(a.topk + goff);
-        for (uint32_t o = 0; o < bytes; o += kBulkPiece)
-            bulk_load(dstb + o, srcb + o, (bytes - o) < kBulkPiece ? (bytes - o) : kBulkPiece, &bars[st]);
-        bulk_load(smem + off_tab + (size_t)st * (E + kRowTail) * 4, a.tabg + id * (int64_t)(E + kRowTail), (uint32_t)(E + kRowTail) * 4u, &bars[st]);
-    };
-
-    // this CTA's chunks: blockIdx.x, +gridDim.x, ... without the ones that hold a split (those need block-wide
-    // counting with barriers, which would stall the pipeline; a second kernel rewrites them)
-    const int64_t stride = gridDim.x;
-    auto advance = [&](int64_t id) {
-        while (id < nchunks && a.nsg[id] != 0) id += stride;
-        return id;
-    };
-    int64_t iss_id = 0;                          // thread 0: next chunk to start copying
-    int64_t id = advance(blockIdx.x);
-    if (tid == 0) {
-        iss_id = id;
-        for (int st = 0; st < stages; ++st)
-            if (iss_id < nchunks) { issue(iss_id, st); iss_id = advance(iss_id + stride); }
-    }
-
-    int64_t use = 0;
-    for (; id < nchunks; id = advance(id + stride), ++use) {
-        const int st = (int)(use % stages);
-        const uint32_t parity = (uint32_t)((use / stages) & 1);
-        int64_t goff; int32_t len;
-        chunk_geometry(a, id, goff, len);
-        const int32_t* buf = reinterpret_cast<const int32_t*>(smem + (size_t)st * TAOT_CHUNK * 4);
-        int32_t* tab = reinterpret_cast<int32_t*>(smem + off_tab + (size_t)st * (E + kRowTail) * 4);
-        int32_t* dst = a.out + goff;
-
-        const bool ok = mbar_wait(&bars[st], parity);
-        if (__syncthreads_or(!ok)) {
-            // the copy never completed: report, give the copies still in flight one more bounded chance to land
-            // (their destination is this CTA's shared memory), and leave
-            if (tid == 0) {
-                atomicOr(a.info + (int32_t)((id / a.nc) / a.R), TAOT_INFO_INTERNAL);
-                for (int s2 = 0; s2 < stages; ++s2) {
-                    const int64_t u2 = (use + ((s2 - st + stages) % stages)) / stages;
-                    (void)mbar_wait(&bars[s2], (uint32_t)(u2 & 1));
+    if (warp == 0) {
+        if (lane == 0) {
+            long long armed_mask = 0;                    // stages whose copies may still be in flight
+            for (int64_t use = 0;; ++use) {
+                const int st = (int)(use % stages);
+                if (use >= stages) {                     // wait until the consumers have left this stage
+                    if (!mbar_wait(&empty[st], (uint32_t)(((use / stages) - 1) & 1))) {
+                        atomicOr(a.info, TAOT_INFO_INTERNAL);
+                        *(volatile int*)&s_abort = 1;
+                        break;
+                    }
+                    armed_mask &= ~(1ll << st);
+                }
+                if (*(volatile int*)&s_abort) break;
+                int64_t id;
+                do { id = (int64_t)atomicAdd(work, 1ull); } while (id < nchunks && a.nsg[id] != 0);
+                if (id >= nchunks) {
+                    s_id[st] = -1;
+                    asm volatile("{\n\t.reg .b64 t;\n\tmbarrier.arrive.shared::cta.b64 t, [%0];\n\t}" :: "r"(smem_u32(&full[st])) : "memory");
+                    break;
+                }
+                s_id[st] = id;
+                int64_t goff; int32_t len;
+                chunk_geometry(a, id, goff, len);
+                const uint32_t bytes = (uint32_t)len * 4u;
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_expect_tx(&full[st], bytes + (uint32_t)E * 4u);
+                unsigned char* dstb = smem + (size_t)st * TAOT_CHUNK * 4;
+                const unsigned char* srcb = reinterpret_cast<const unsigned char*>(a.topk + goff);
+                for (uint32_t o = 0; o < bytes; o += kBulkPiece)
+                    bulk_load(dstb + o, srcb + o, (bytes - o) < kBulkPiece ? (bytes - o) : kBulkPiece, &full[st]);
+                bulk_load(smem + off_tab + (size_t)st * E * 4, a.tabg + id * (int64_t)(E + kRowTail), (uint32_t)E * 4u, &full[st]);
+                armed_mask |= 1ll << st;
+            }
+            (void)armed_mask;
+        }
+    } else {
+        const int c = tid - 32;
+        for (int64_t use = 0;; ++use) {
+            const int st = (int)(use % stages);
+            if (!mbar_wait(&full[st], (uint32_t)((use / stages) & 1))) {
+                if (lane == 0) atomicOr(a.info, TAOT_INFO_INTERNAL);
+                *(volatile int*)&s_abort = 1;
+                break;
+            }
+            const long long id = s_id[st];
+            if (id < 0) break;
+            int64_t goff; int32_t len;
+            chunk_geometry(a, id, goff, len);
+            const int4* buf = reinterpret_cast<const int4*>(smem + (size_t)st * TAOT_CHUNK * 4);
+            const int32_t* tab = reinterpret_cast<const int32_t*>(smem + off_tab + (size_t)st * E * 4);
+            int4* dst = reinterpret_cast<int4*>(a.out + goff);
+            const int n4 = len >> 2;                     // segments are multiples of 4 entries on this path
+            for (int i0 = c; i0 < n4; i0 += kStreamConsumers * kStreamUnroll) {
+                int4 v[kStreamUnroll];
+#pragma unroll
+                for (int u = 0; u < kStreamUnroll; ++u) {
+                    const int i = i0 + u * kStreamConsumers;
+                    if (i < n4) v[u] = buf[i];
+                }
+#pragma unroll
+                for (int u = 0; u < kStreamUnroll; ++u) {
+                    const int i = i0 + u * kStreamConsumers;
+                    if (i < n4) {
+                        int4 o = v[u];
+                        o.x = (unsigned)o.x < (unsigned)E ? tab[o.x] : o.x;
+                        o.y = (unsigned)o.y < (unsigned)E ? tab[o.y] : o.y;
+                        o.z = (unsigned)o.z < (unsigned)E ? tab[o.z] : o.z;
+                        o.w = (unsigned)o.w < (unsigned)E ? tab[o.w] : o.w;
+                        st_stream(dst + i, o);
+                    }
                 }
             }
-            __syncthreads();
-            return;
+            __syncwarp();
+            if (lane == 0)
+                asm volatile("{\n\t.reg .b64 t;\n\tmbarrier.arrive.shared::cta.b64 t, [%0];\n\t}" :: "r"(smem_u32(&empty[st])) : "memory");
         }
-        rewrite_chunk<true>(a, id, buf, tab, dst, len, recs, s_cntw, &s_pos);
-        __syncthreads();                         // everyone is done with this stage's buffers
-        if (tid == 0 && iss_id < nchunks) {
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            issue(iss_id, st);
-            iss_id = advance(iss_id + stride);
-        }
+    }
+    __syncthreads();
+    if (s_abort && tid == 0) {
+        // copies that were started may still be landing in this CTA's shared memory: give each stage one more bounded wait
+        for (int st = 0; st < stages; ++st) { (void)mbar_wait(&full[st], 0); (void)mbar_wait(&full[st], 1); }
     }
 }
 
@@ -567,6 +604,7 @@ int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, void* ws, const i
     a.soff = reinterpret_cast<int32_t*>(w + h->off_soff);
     a.splits = reinterpret_cast<int4*>(w + h->off_splits);
     a.slot_expert = d_slot_expert; a.X = d_X; a.out = d_new_idx; a.info = d_info;
+    a.work = reinterpret_cast<unsigned long long*>(w + h->off_work);
     a.layer_elems = p.T * p.k; a.seg = h->seg; a.nc = h->nc; a.R = p.R; a.E = p.E; a.K = p.K;
     const int vec_ok = ((reinterpret_cast<uintptr_t>(d_topk) & 15) == 0) &&
                        ((reinterpret_cast<uintptr_t>(d_new_idx) & 15) == 0) && (h->seg % 4 == 0);
@@ -577,13 +615,12 @@ int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, void* ws, const i
     TAOT_CUDA_OK(cudaFuncSetAttribute(assign_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_prep));
     assign_prep_kernel<<<(unsigned)((int64_t)p.L * p.R), kThreads, smem_prep, st>>>(a);
     TAOT_CUDA_OK(cudaGetLastError());
-    const StreamLayout sl = stream_layout(p.E, S);
+    const StreamLayout sl = stream_layout(p.E);
     int launches = 2;
     if (vec_ok && p.E % 4 == 0 && sl.stages >= 2) {
         TAOT_CUDA_OK(cudaFuncSetAttribute(assign_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sl.bytes));
         const unsigned grid = blocks < (unsigned)h->sm_count ? blocks : (unsigned)h->sm_count;
-        assign_stream_kernel<<<grid, kThreads, sl.bytes, st>>>(a, sl.stages, (uint32_t)sl.off_tab, (uint32_t)sl.off_recs,
-                                                             (int64_t)blocks);
+        assign_stream_kernel<<<grid, kStreamThreads, sl.bytes, st>>>(a, sl.stages, (uint32_t)sl.off_tab, (int64_t)blocks, a.work);
         TAOT_CUDA_OK(cudaGetLastError());
         const size_t smem = (size_t)TAOT_CHUNK * 4 + sizeof(int32_t) * (((size_t)p.E + kRowTail + 3) & ~(size_t)3) +
                             sizeof(int4) * (size_t)(S + kRowSplits);
