@@ -15,4 +15,7 @@ from .binding import (  # noqa: F401
     auction,
     assign,
     plan_layers,
+    report,
+    REPORT_INTS,
+    REPORT_REALS,
 )

@@ -150,12 +150,46 @@ def assign(topk_layer, R: int, E: int, K: int, slot_expert, X) -> np.ndarray:
     return out
 
 
+REPORT_INTS = ("total_load", "rerouted", "mean_load", "max_before", "min_before", "max_after", "min_after",
+               "hot_ranks", "cold_ranks", "hot_experts", "clones", "intra", "inter", "same_rank")
+REPORT_REALS = ("rho_before", "rho_after", "dev_before", "dev_after", "peak_reduction", "frac_rerouted",
+                "cost_ratio", "cost_C")
+
+
+def report(R: int, E: int, K: int, e2r, C, B, expert_load, rank_load, slot_expert, X, lam: float = 3.0):
+    """Dispatch report of one layer.  Returns a dict with the scalar fields named in REPORT_INTS /
+    REPORT_REALS and the arrays spill [E], load_after [R], slot_moved [S], slot_kind [S]."""
+    e2r = _i32(e2r); C = _f32(C); B = _f32(B)
+    el = _i32(expert_load); rl = _i32(rank_load); se = _i32(slot_expert).reshape(-1); X = _i32(X)
+    S = R * K
+    spill_out = np.empty((E,), np.int32)
+    la = np.empty((R,), np.int32)
+    moved = np.empty((S,), np.int32)
+    kind = np.empty((S,), np.int32)
+    ints = np.zeros((len(REPORT_INTS),), np.int64)
+    reals = np.zeros((len(REPORT_REALS),), np.float64)
+    _L().oracle_report(ctypes.c_int32(R), ctypes.c_int32(E), ctypes.c_int32(K), _p(e2r), _p(C), _p(B),
+                       _p(el), _p(rl), _p(se), _p(X), ctypes.c_double(lam), _p(spill_out), _p(la),
+                       _p(moved), _p(kind), _p(ints), _p(reals))
+    out = dict(spill=spill_out, load_after=la, slot_moved=moved, slot_kind=kind)
+    out.update({k: int(v) for k, v in zip(REPORT_INTS, ints)})
+    out.update({k: float(v) for k, v in zip(REPORT_REALS, reals)})
+    return out
+
+
 def plan_layers(topk, R: int, E: int, K: int, e2r, C, eps: float, max_iters: int, tol: float = 0.0,
                 check_every: int = 1, B=None, eps0: float = 1e-8, price_step: float = 0.1,
-                auction_max_rounds: int = 0, do_assign: bool = True):
+                auction_max_rounds: int = 0, do_assign: bool = True, hint: bool = True,
+                topology: bool = True):
     """The whole path on the CPU, layer by layer: histogram, excess/spare, Sinkhorn (the fp64 plan
     is rounded to fp32 before it is used as the Phase-2 hint, as the library's plan is fp32),
-    spill, matching, auction, reassignment."""
+    spill, matching, auction, reassignment.
+
+    The two switches of the paper's ablation (Ablation Study, Table 2): hint=False leaves the
+    Phase-1 term out of the Phase-2 score (Phase 1 is not run, the plan is zero); topology=False
+    leaves the topology-preference term out of the Phase-2 score.  A term left out is a term that
+    is exactly zero, so the matching is fed a zero plan / a zero preference matrix.  Phase 3 is not
+    ablated and always sees the real preference matrix."""
     topk = _i32(topk)
     L = topk.shape[0]
     C = _f32(C)
@@ -168,12 +202,14 @@ def plan_layers(topk, R: int, E: int, K: int, e2r, C, eps: float, max_iters: int
                slot_tokens=np.zeros((L, R, K), np.int32), X=np.zeros((L, R, R * K), np.int32),
                auction_rounds=np.zeros(L, np.int32), match_rounds=np.zeros(L, np.int32),
                new_idx=np.empty_like(topk) if do_assign else None)
+    B2 = Bm if topology else np.zeros_like(Bm)
     for l in range(L):
-        sk = sinkhorn(ex[l].astype(np.float32), sp[l].astype(np.float32), C, eps, max_iters, tol,
-                      check_every, eps0)
-        out["plan"][l] = sk["plan"]; out["n_iter"][l] = sk["n_iter"]; out["row_err"][l] = sk["row_err"]
+        if hint:
+            sk = sinkhorn(ex[l].astype(np.float32), sp[l].astype(np.float32), C, eps, max_iters, tol,
+                          check_every, eps0)
+            out["plan"][l] = sk["plan"]; out["n_iter"][l] = sk["n_iter"]; out["row_err"][l] = sk["row_err"]
         spl = spill(el[l], e2r, R, mean[l])
-        m = match(R, E, K, e2r, mean[l], ex[l], spl, sp[l], Bm, sk["plan"].astype(np.float32), eps0)
+        m = match(R, E, K, e2r, mean[l], ex[l], spl, sp[l], B2, out["plan"][l].astype(np.float32), eps0)
         out["slot_expert"][l] = m["slot_expert"].reshape(R, K)
         out["slot_tokens"][l] = m["slot_tokens"].reshape(R, K)
         out["match_rounds"][l] = m["inner_rounds"]

@@ -493,3 +493,101 @@ void oracle_assign(const int32_t* topk, int64_t T, int32_t k, int32_t R, int32_t
     }
     free(ord);
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Dispatch report of one layer (Appendix B.3, the four-part per-layer diagnostics; Evaluation,
+ * the metric definitions: imbalance, intra-/inter-node transfers, weighted cost at 1 : lambda).
+ *
+ *   part 1  loads before: rank_load, expert_load; hot ranks (l_r above the mean), hot experts
+ *           (positive spill, i.e. the experts Phase 2 may clone); spill is returned per expert
+ *   part 2  cloning plan: per slot the tokens rerouted to it (column sum of X) and the kind of
+ *           copy, from the home rank of its expert to the rank of the slot:
+ *             0 empty, 1 intra-node (B[home][host] >= 1), 2 inter-node, 3 home rank itself;
+ *           counts of each kind; weighted cost intra + lambda * inter, and sum of C[home][host]
+ *   part 3  projected load: l'_r = l_r - tokens leaving r's home experts + tokens entering r's slots
+ *   part 4  rho = (max_r l_r - mean) / mean with mean = total / R (Problem Formulation), before
+ *           and after; largest absolute deviation from the mean as a fraction, before and after;
+ *           peak-load reduction (max before - max after) / max before; fraction rerouted.
+ * Ratios are fp64, one IEEE operation each; a zero denominator gives 0.
+ *
+ * ints[14]: total, rerouted, floor mean, max before, min before, max after, min after, hot ranks,
+ *           cold ranks, hot experts, clones, intra, inter, same-rank
+ * reals[8]: rho before, rho after, deviation before, deviation after, peak reduction,
+ *           fraction rerouted, cost at 1:lambda, cost by C
+ */
+void oracle_report(int32_t R, int32_t E, int32_t K, const int32_t* e2r, const float* C, const float* B,
+                   const int32_t* expert_load, const int32_t* rank_load, const int32_t* slot_expert,
+                   const int32_t* X, double lambda, int32_t* spill, int32_t* load_after,
+                   int32_t* slot_moved, int32_t* slot_kind, int64_t* ints, double* reals)
+{
+    const int32_t S = R * K;
+    int64_t total = 0;
+    for (int32_t r = 0; r < R; ++r) total += rank_load[r];
+    const int64_t mfloor = total / R;
+    const double mean = (double)total / (double)R;
+
+    /* part 1 */
+    oracle_spill(expert_load, e2r, R, E, mfloor, spill);
+    int64_t hot_ranks = 0, cold_ranks = 0, hot_experts = 0;
+    int64_t max_b = rank_load[0], min_b = rank_load[0];
+    for (int32_t r = 0; r < R; ++r) {
+        if (rank_load[r] > mfloor) ++hot_ranks;
+        if (rank_load[r] < mfloor) ++cold_ranks;
+        if (rank_load[r] > max_b) max_b = rank_load[r];
+        if (rank_load[r] < min_b) min_b = rank_load[r];
+    }
+    for (int32_t e = 0; e < E; ++e) if (spill[e] > 0) ++hot_experts;
+
+    /* part 2 */
+    int64_t rerouted = 0, clones = 0, intra = 0, inter = 0, same = 0;
+    double cost_C = 0.0;
+    for (int32_t s = 0; s < S; ++s) {
+        int64_t moved = 0;
+        for (int32_t r = 0; r < R; ++r) moved += X[(int64_t)r * S + s];
+        slot_moved[s] = (int32_t)moved;
+        rerouted += moved;
+        const int32_t e = slot_expert[s];
+        if (e < 0) { slot_kind[s] = 0; continue; }
+        const int32_t home = e2r[e], host = s / K;
+        ++clones;
+        if (home == host) { slot_kind[s] = 3; ++same; }
+        else if (B[(int64_t)home * R + host] >= 1.0f) { slot_kind[s] = 1; ++intra; }
+        else { slot_kind[s] = 2; ++inter; }
+        cost_C = cost_C + (double)C[(int64_t)home * R + host];
+    }
+    const double linter = lambda * (double)inter;
+    const double cost_ratio = (double)intra + linter;
+
+    /* part 3 */
+    for (int32_t r = 0; r < R; ++r) load_after[r] = rank_load[r];
+    for (int32_t s = 0; s < S; ++s) {
+        const int32_t e = slot_expert[s];
+        if (e < 0) continue;
+        load_after[e2r[e]] -= slot_moved[s];
+        load_after[s / K] += slot_moved[s];
+    }
+    int64_t max_a = load_after[0], min_a = load_after[0];
+    for (int32_t r = 0; r < R; ++r) {
+        if (load_after[r] > max_a) max_a = load_after[r];
+        if (load_after[r] < min_a) min_a = load_after[r];
+    }
+
+    /* part 4 */
+    double rho_b = 0.0, rho_a = 0.0, dev_b = 0.0, dev_a = 0.0, peak = 0.0, frac = 0.0;
+    if (mean > 0.0) {
+        const double up_b = (double)max_b - mean, dn_b = mean - (double)min_b;
+        const double up_a = (double)max_a - mean, dn_a = mean - (double)min_a;
+        rho_b = up_b / mean;
+        rho_a = up_a / mean;
+        dev_b = (up_b > dn_b ? up_b : dn_b) / mean;
+        dev_a = (up_a > dn_a ? up_a : dn_a) / mean;
+    }
+    if (max_b > 0) peak = (double)(max_b - max_a) / (double)max_b;
+    if (total > 0) frac = (double)rerouted / (double)total;
+
+    ints[0] = total; ints[1] = rerouted; ints[2] = mfloor; ints[3] = max_b; ints[4] = min_b;
+    ints[5] = max_a; ints[6] = min_a; ints[7] = hot_ranks; ints[8] = cold_ranks; ints[9] = hot_experts;
+    ints[10] = clones; ints[11] = intra; ints[12] = inter; ints[13] = same;
+    reals[0] = rho_b; reals[1] = rho_a; reals[2] = dev_b; reals[3] = dev_a; reals[4] = peak;
+    reals[5] = frac; reals[6] = cost_ratio; reals[7] = cost_C;
+}

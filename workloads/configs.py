@@ -29,6 +29,8 @@ class PlannerConfig:
     e2r_mode: str = "contiguous"   # "contiguous": e // (E/R);  "stride2": e -> 2e (odd ranks host nothing)
     zipf: Tuple[float, float] = (1.0, 1.0)   # per-layer exponent ~ U[lo, hi]
     hot_frac: float = 0.0       # fraction of tokens forced onto one random expert per layer
+    rank_fracs: Tuple[float, ...] = ()   # if set: layer l sends fraction rank_fracs[l % len] of its tokens to
+                                         # the experts of one random rank and the rest to uniformly random experts
     eps_frac: float = 0.05      # eps = eps_frac * max(C)
     max_iters: int = 200
     tol: float = 0.0            # <= 0: exactly max_iters iterations
@@ -63,6 +65,19 @@ CONFIGS = {
     "cfg4": PlannerConfig("cfg4", L=48, R=256, E=128, K=1, k=8, T=1048576, gpus_per_node=8,
                           tiers=(0.0, 1.0, 6.0, 16.0), nodes_per_group=4, e2r_mode="stride2",
                           zipf=(0.6, 1.6), eps_frac=0.005, max_iters=1000, tol=1e-6),
+    # Imbalance built as in the paper's sensitivity study: 30/50/70/90 % of the tokens go to one rank, the
+    # rest at random; EP32, E=256, K=2, cost 1 intra-node / lambda=3 cross-node, eps = lambda.  3 seeds per level.
+    "llep32": PlannerConfig("llep32", L=12, R=32, E=256, K=2, k=8, T=65536, gpus_per_node=8,
+                            tiers=(0.0, 1.0, 3.0), eps_frac=1.0, max_iters=1000, tol=1e-6,
+                            rank_fracs=(0.3, 0.5, 0.7, 0.9)),
+    # The initial-imbalance ladder of the balance-quality study: rho_0 in {10,20,30,50,70} %, reached by sending
+    # the fraction rho_0/(R-1) of the tokens to one rank; EP16 and EP32, 3 seeds per level.
+    "ladder16": PlannerConfig("ladder16", L=15, R=16, E=256, K=2, k=8, T=32768, gpus_per_node=8,
+                              tiers=(0.0, 1.0, 3.0), eps_frac=1.0, max_iters=1000, tol=1e-6,
+                              rank_fracs=tuple(x / 15.0 for x in (0.1, 0.2, 0.3, 0.5, 0.7))),
+    "ladder32": PlannerConfig("ladder32", L=15, R=32, E=256, K=2, k=8, T=65536, gpus_per_node=8,
+                              tiers=(0.0, 1.0, 3.0), eps_frac=1.0, max_iters=1000, tol=1e-6,
+                              rank_fracs=tuple(x / 31.0 for x in (0.1, 0.2, 0.3, 0.5, 0.7))),
 }
 
 

@@ -129,6 +129,8 @@ def routing_topk(cfg: PlannerConfig, device="cpu", layers: Optional[Sequence[int
     out = torch.empty((len(layers), T, k), dtype=torch.int32, device=device)
     chunk = max(1, min(T, max_chunk_elems // E))
     e_ids = torch.arange(E, dtype=torch.int64, device=device)
+    if cfg.rank_fracs:
+        return _routing_one_hot_rank(cfg, device, layers, out, chunk, e_ids)
     for li, layer in enumerate(layers):
         logp = _layer_log_popularity(cfg, layer, device)
         if cfg.hot_frac > 0:
@@ -146,6 +148,30 @@ def routing_topk(cfg: PlannerConfig, device="cpu", layers: Optional[Sequence[int
                 force = (ut < cfg.hot_frac) & ~(idx == hot).any(dim=1)
                 idx[force, k - 1] = hot
             out[li, t0:t1] = idx.to(torch.int32)
+    return out
+
+
+def _routing_one_hot_rank(cfg, device, layers, out, chunk, e_ids):
+    """Routing with a fraction of the tokens sent to one rank: in layer l a token is "hot" with probability
+    rank_fracs[l % len]; a hot token's k choices are k distinct experts of the layer's hot rank (seeded), any
+    other token's are k distinct uniformly random experts.  Needs k <= experts per rank."""
+    T, E, k, R = cfg.T, cfg.E, cfg.k, cfg.R
+    home = expert_to_rank(E, R, cfg.e2r_mode, device=device).to(torch.int64)
+    for li, layer in enumerate(layers):
+        f = cfg.rank_fracs[layer % len(cfg.rank_fracs)]
+        uh = uniform01(cfg.seed, 7, torch.tensor([layer], dtype=torch.int64, device=device))
+        hot_rank = min(R - 1, int(float(uh[0]) * R))
+        on_hot = home == hot_rank
+        assert int(on_hot.sum()) >= k, "the hot rank must host at least k experts"
+        bar = torch.where(on_hot, 0.0, -float("inf")).to(torch.float64)
+        for t0 in range(0, T, chunk):
+            t1 = min(T, t0 + chunk)
+            tok = torch.arange(t0, t1, dtype=torch.int64, device=device)
+            ctr = ((layer * T + tok)[:, None]) * E + e_ids[None, :]
+            keys = -torch.log(-torch.log(uniform01(cfg.seed, 3, ctr)))
+            hot_tok = uniform01(cfg.seed, 8, layer * T + tok) < f
+            keys = torch.where(hot_tok[:, None], keys + bar[None, :], keys)
+            out[li, t0:t1] = torch.topk(keys, k, dim=1, largest=True, sorted=True).indices.to(torch.int32)
     return out
 
 
