@@ -14,6 +14,7 @@
  *   taot_assign         deterministic token -> replica rewrite of the routing table
  *   taot_plan           all of the above chained on one stream
  *   taot_plan_host      taot_plan with host buffers (copies in and out on the same stream)
+ *   taot_report         the per-layer dispatch diagnostics of a finished plan        (Appendix B.3)
  *
  * Conventions
  *   - Shapes: L problems, R ranks, E experts, K guest slots per rank, S = R*K slots
@@ -87,7 +88,19 @@ typedef struct {
     float   eps0;               /* the paper's epsilon_0 safeguard constant, e.g. 1e-8f */
     float   price_step;         /* Phase-3 price increment, e.g. 0.1f */
     int32_t auction_max_rounds; /* <= 0: run the auction to completion */
+    int32_t ablation;           /* TAOT_ABLATE_* bits, 0 = the full method */
 } taot_params;
+
+/*
+ * The two switches of the paper's algorithm-level ablation (Ablation Study, Table 2).  A term that is
+ * switched off is left out of the Phase-2 score (which is the same as the term being exactly zero).
+ * Phase 3 is never ablated: it only assigns tokens and always uses the real topology preference.
+ */
+enum {
+    TAOT_ABLATE_HINT = 1,       /* no Phase-1 flow hint: taot_match ignores d_plan (it may be NULL); taot_plan does
+                                   not run the Sinkhorn stage and returns a zero plan, zero iterations, zero row_err */
+    TAOT_ABLATE_TOPOLOGY = 2    /* no topology-preference term alpha*B in the Phase-2 score */
+};
 
 /* Outputs of taot_plan / taot_plan_host: device pointers (host pointers for the _host call).
  * Optional members may be NULL and are then kept in workspace only. */
@@ -233,6 +246,47 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* out, v
  */
 int taot_plan_host(taot_handle_t h, const int32_t* h_topk, const taot_outputs* out, void* d_ws,
                    void* stream);
+
+/*
+ * One layer's dispatch diagnostics (Appendix B.3; metric definitions of the Evaluation section).  128 bytes.
+ */
+typedef struct {
+    int64_t total_load;      /* sum_r l_r */
+    int64_t rerouted;        /* sum_{r,s} X[r][s]: tokens sent to guest replicas */
+    int32_t mean_load;       /* floor(total_load / R), the mean the planner balances against */
+    int32_t max_before, min_before;   /* extreme rank loads before rerouting */
+    int32_t max_after, min_after;     /* extreme projected rank loads after rerouting */
+    int32_t hot_ranks;       /* ranks with l_r above the mean */
+    int32_t cold_ranks;      /* ranks with l_r below the mean */
+    int32_t hot_experts;     /* experts with positive spill (the candidates of Phase 2) */
+    int32_t clones;          /* occupied guest slots = expert-weight transfers */
+    int32_t intra, inter;    /* of those: inside the home node (B[home][host] >= 1) / across nodes */
+    int32_t same_rank;       /* of those: hosted by the home rank itself (neither intra nor inter) */
+    double rho_before, rho_after;     /* (max_r l_r - mean) / mean with mean = total_load / R */
+    double dev_before, dev_after;     /* max_r |l_r - mean| / mean */
+    double peak_reduction;   /* (max_before - max_after) / max_before */
+    double frac_rerouted;    /* rerouted / total_load */
+    double cost_ratio;       /* intra + lambda * inter: the weighted cost at 1 : lambda */
+    double cost_C;           /* sum over occupied slots of C[home rank][host rank] */
+} taot_report_row;
+
+/*
+ * Dispatch report of L finished plans (Appendix B.3, parts 1-4), computed on the GPU.
+ *   in : d_expert_load [L,E], d_rank_load [L,R], d_slot_expert [L,R,K], d_X [L,R,S] as taot_plan wrote them;
+ *        lambda: the inter-node weight of cost_ratio (the paper uses 3).
+ *   out: d_rows [L] (device memory, 8-byte aligned); optional (NULL to skip) per-element arrays
+ *        d_spill [L,E]        spill of each expert before matching (part 1: the hot experts are spill > 0)
+ *        d_load_after [L,R]   projected rank loads (part 3)
+ *        d_slot_moved [L,S]   tokens rerouted to each slot (part 2)
+ *        d_slot_kind [L,S]    0 empty, 1 intra-node copy, 2 inter-node copy, 3 hosted by the home rank
+ * Integer fields are exact; each ratio is a single IEEE fp64 operation; a zero denominator gives 0.
+ * A zero ratio or an empty plan is not an error.  Errors: TAOT_ERR_NULL, TAOT_ERR_ALIGN,
+ * TAOT_ERR_UNSUPPORTED (R > 256), TAOT_ERR_PARAM (lambda not finite).
+ */
+int taot_report(taot_handle_t h, const int32_t* d_expert_load, const int32_t* d_rank_load,
+                const int32_t* d_slot_expert, const int32_t* d_X, double lambda, taot_report_row* d_rows,
+                int32_t* d_spill, int32_t* d_load_after, int32_t* d_slot_moved, int32_t* d_slot_kind,
+                void* stream);
 
 /*
  * Stage timing for benchmarks.  With profiling on, taot_plan (and taot_plan_host) records one CUDA

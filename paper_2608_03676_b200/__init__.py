@@ -20,4 +20,10 @@ from .binding import (  # noqa: F401
     histogram_static,
     STATIC_SCRATCH_BYTES,
     PLAN_LAUNCHES,
+    PLAN_LAUNCHES_NO_HINT,
+    ABLATE_HINT,
+    ABLATE_TOPOLOGY,
+    INFO_INTERNAL,
+    ReportRow,
 )
+from .report import format_layer  # noqa: F401

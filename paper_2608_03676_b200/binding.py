@@ -18,11 +18,15 @@ INFO_NONFINITE = 4
 INFO_AUCTION_RESIDUAL = 8
 INFO_SUPPLY_SCALED = 16
 INFO_SINKHORN_SIZE = 32
+INFO_INTERNAL = 64
+
+ABLATE_HINT = 1
+ABLATE_TOPOLOGY = 2
 
 _SYMBOLS = [
     "taot_create", "taot_destroy", "taot_workspace_bytes", "taot_host_workspace_bytes",
     "taot_histogram", "taot_histogram_static", "taot_excess_spare", "taot_sinkhorn", "taot_match", "taot_assign",
-    "taot_plan", "taot_plan_host", "taot_set_profiling", "taot_get_stage_ms", "taot_last_launch_count",
+    "taot_plan", "taot_plan_host", "taot_report", "taot_set_profiling", "taot_get_stage_ms", "taot_last_launch_count",
     "taot_status_string",
 ]
 
@@ -37,7 +41,21 @@ class TaotParams(ctypes.Structure):
         ("E", ctypes.c_int32), ("K", ctypes.c_int32), ("k", ctypes.c_int32), ("T", ctypes.c_int64),
         ("eps", ctypes.c_float), ("max_iters", ctypes.c_int32), ("tol", ctypes.c_float),
         ("check_every", ctypes.c_int32), ("eps0", ctypes.c_float), ("price_step", ctypes.c_float),
-        ("auction_max_rounds", ctypes.c_int32),
+        ("auction_max_rounds", ctypes.c_int32), ("ablation", ctypes.c_int32),
+    ]
+
+
+class ReportRow(ctypes.Structure):
+    """taot_report_row: one layer's dispatch diagnostics (128 bytes)."""
+    _fields_ = [
+        ("total_load", ctypes.c_int64), ("rerouted", ctypes.c_int64), ("mean_load", ctypes.c_int32),
+        ("max_before", ctypes.c_int32), ("min_before", ctypes.c_int32), ("max_after", ctypes.c_int32),
+        ("min_after", ctypes.c_int32), ("hot_ranks", ctypes.c_int32), ("cold_ranks", ctypes.c_int32),
+        ("hot_experts", ctypes.c_int32), ("clones", ctypes.c_int32), ("intra", ctypes.c_int32),
+        ("inter", ctypes.c_int32), ("same_rank", ctypes.c_int32),
+        ("rho_before", ctypes.c_double), ("rho_after", ctypes.c_double), ("dev_before", ctypes.c_double),
+        ("dev_after", ctypes.c_double), ("peak_reduction", ctypes.c_double), ("frac_rerouted", ctypes.c_double),
+        ("cost_ratio", ctypes.c_double), ("cost_C", ctypes.c_double),
     ]
 
 
@@ -97,6 +115,7 @@ STATIC_SCRATCH_BYTES = 4 << 20
 # kernel for handed-back problems), matching+auction, reassignment (tables, pipelined rewrite of the chunks
 # without a split, rewrite of the chunks with one) -- for a 16-byte aligned routing table with E % 4 == 0
 PLAN_LAUNCHES = 8
+PLAN_LAUNCHES_NO_HINT = 6       # with ABLATE_HINT the two Sinkhorn kernels are not launched
 
 
 def histogram_static(topk: torch.Tensor, R: int, E: int, e2r_dev: torch.Tensor, n: torch.Tensor,
@@ -131,7 +150,8 @@ class Planner:
 
     def __init__(self, L: int, R: int, E: int, K: int, k: int, T: int, e2r, C, eps: float,
                  max_iters: int, tol: float = 0.0, check_every: int = 1, B=None, eps0: float = 1e-8,
-                 price_step: float = 0.1, auction_max_rounds: int = 0, device: Optional[torch.device] = None):
+                 price_step: float = 0.1, auction_max_rounds: int = 0, ablation: int = 0,
+                 device: Optional[torch.device] = None):
         if not torch.cuda.is_available():
             raise TaotError("the TAOT planner needs a CUDA device; there is no CPU path")
         self.lib = load_library()
@@ -139,8 +159,9 @@ class Planner:
         self.L, self.R, self.E, self.K, self.k, self.T = L, R, E, K, k, T
         self.S = R * K
         p = TaotParams(ctypes.sizeof(TaotParams), L, R, E, K, k, T, eps, max_iters, tol, check_every, eps0,
-                       price_step, auction_max_rounds)
+                       price_step, auction_max_rounds, ablation)
         self.params = p
+        self.ablation = ablation
         e2r_h = torch.as_tensor(e2r, dtype=torch.int32).contiguous().cpu()
         C_h = torch.as_tensor(C, dtype=torch.float32).contiguous().cpu()
         B_h = None if B is None else torch.as_tensor(B, dtype=torch.float32).contiguous().cpu()
@@ -240,7 +261,8 @@ class Planner:
         _check(self.lib.taot_match(self.handle, _ptr(_dev(n, torch.int32, "n")),
                                    _ptr(_dev(expert_load, torch.int32, "expert_load")),
                                    _ptr(_dev(rank_load, torch.int32, "rank_load")),
-                                   _ptr(_dev(plan, torch.float32, "plan")), _ptr(se), _ptr(stk), _ptr(X),
+                                   _ptr(None if plan is None else _dev(plan, torch.float32, "plan")), _ptr(se),
+                                   _ptr(stk), _ptr(X),
                                    _ptr(rounds), _ptr(info), _ptr(self.ws), _stream()), "taot_match")
         return dict(slot_expert=se, slot_tokens=stk, X=X, rounds=rounds, info=info)
 
@@ -253,6 +275,26 @@ class Planner:
                                     _ptr(_dev(X, torch.int32, "X")), _ptr(new), _ptr(info), _ptr(self.ws),
                                     ctypes.c_int32(1 if reuse_counts else 0), _stream()), "taot_assign")
         return new, info
+
+    def report(self, expert_load, rank_load, slot_expert, X, lam: float = 3.0) -> Dict[str, object]:
+        """Dispatch diagnostics of L finished plans through `taot_report`.  Returns the row fields as numpy
+        arrays of length L (named as in `ReportRow`) plus the tensors spill [L,E], load_after [L,R],
+        slot_moved [L,S], slot_kind [L,S] (still on the device)."""
+        import numpy as np
+        L, R, E, S = self.L, self.R, self.E, self.S
+        rows = torch.zeros((L, ctypes.sizeof(ReportRow)), dtype=torch.uint8, device=self.device)
+        spill = self._empty((L, E), torch.int32); after = self._empty((L, R), torch.int32)
+        moved = self._empty((L, S), torch.int32); kind = self._empty((L, S), torch.int32)
+        _check(self.lib.taot_report(self.handle, _ptr(_dev(expert_load, torch.int32, "expert_load")),
+                                    _ptr(_dev(rank_load, torch.int32, "rank_load")),
+                                    _ptr(_dev(slot_expert, torch.int32, "slot_expert")),
+                                    _ptr(_dev(X, torch.int32, "X")), ctypes.c_double(lam), _ptr(rows), _ptr(spill),
+                                    _ptr(after), _ptr(moved), _ptr(kind), _stream()), "taot_report")
+        raw = rows.cpu().numpy().tobytes()
+        recs = (ReportRow * L).from_buffer_copy(raw)
+        out: Dict[str, object] = {name: np.array([getattr(r, name) for r in recs]) for name, _ in ReportRow._fields_}
+        out.update(spill=spill, load_after=after, slot_moved=moved, slot_kind=kind)
+        return out
 
     # ------------------------------------------------------------------ whole path
     def _outputs_struct(self, out: Dict[str, torch.Tensor]) -> _Outputs:

@@ -22,6 +22,7 @@ bool valid_params(const taot_params* p)
     if (p->max_iters < 1) return false;
     if (!(p->eps0 >= 0.0f) || !std::isfinite(p->eps0)) return false;
     if (!std::isfinite(p->price_step) || !std::isfinite(p->tol)) return false;
+    if (p->ablation & ~(TAOT_ABLATE_HINT | TAOT_ABLATE_TOPOLOGY)) return false;
     return true;
 }
 
@@ -326,13 +327,28 @@ int taot_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load
                int32_t* d_rounds, int32_t* d_info, void* ws, void* stream)
 {
     if (h && h->p.R > 256) return TAOT_ERR_UNSUPPORTED;      // beyond 256 ranks only Phase 1 is built
-    if (!h || !d_n || !d_expert_load || !d_rank_load || !d_plan || !d_slot_expert || !d_slot_tokens || !d_X ||
-        !d_info || !ws)
+    if (!h || !d_n || !d_expert_load || !d_rank_load || !d_slot_expert || !d_slot_tokens || !d_X || !d_info || !ws)
         return TAOT_ERR_NULL;
+    if (!d_plan && !(h->p.ablation & TAOT_ABLATE_HINT)) return TAOT_ERR_NULL;
     if (reinterpret_cast<uintptr_t>(ws) & 255) return TAOT_ERR_ALIGN;
     int a = taot_launch_match(h, d_n, d_expert_load, d_rank_load, d_plan, d_slot_expert, d_slot_tokens, d_X,
                               d_rounds, d_info, reinterpret_cast<int32_t*>(at(ws, h->off_nrem)),
                               reinterpret_cast<float*>(at(ws, h->off_t12)), static_cast<cudaStream_t>(stream));
+    if (a < 0) return a;
+    h->last_launches = a;
+    return TAOT_OK;
+}
+
+int taot_report(taot_handle_t h, const int32_t* d_expert_load, const int32_t* d_rank_load,
+                const int32_t* d_slot_expert, const int32_t* d_X, double lambda, taot_report_row* d_rows,
+                int32_t* d_spill, int32_t* d_load_after, int32_t* d_slot_moved, int32_t* d_slot_kind, void* stream)
+{
+    if (h && h->p.R > 256) return TAOT_ERR_UNSUPPORTED;
+    if (!h || !d_expert_load || !d_rank_load || !d_slot_expert || !d_X || !d_rows) return TAOT_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(d_rows) & 7) return TAOT_ERR_ALIGN;
+    if (!std::isfinite(lambda)) return TAOT_ERR_PARAM;
+    int a = taot_launch_report(h, d_expert_load, d_rank_load, d_slot_expert, d_X, lambda, d_rows, d_spill,
+                               d_load_after, d_slot_moved, d_slot_kind, static_cast<cudaStream_t>(stream));
     if (a < 0) return a;
     h->last_launches = a;
     return TAOT_OK;
@@ -389,8 +405,13 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, voi
     if ((a = taot_launch_merge(h, cc, o->n, o->expert_load, o->rank_load, excess, spare, fs, fd, st)) < 0) return a;
     total += a;
     TAOT_MARK(2);
-    if ((a = taot_launch_sinkhorn(h, fs, fd, p.L, o->plan, o->sinkhorn_iters, o->row_err, o->info,
-                                  reinterpret_cast<float*>(at(ws, h->off_kt)), st)) < 0)
+    if (p.ablation & TAOT_ABLATE_HINT) {       // Phase 1 switched off: no solve, a zero hint
+        TAOT_CUDA_OK(cudaMemsetAsync(o->plan, 0, sizeof(float) * (size_t)p.L * p.R * p.R, st));
+        TAOT_CUDA_OK(cudaMemsetAsync(o->sinkhorn_iters, 0, sizeof(int32_t) * p.L, st));
+        TAOT_CUDA_OK(cudaMemsetAsync(o->row_err, 0, sizeof(float) * p.L, st));
+        a = 0;
+    } else if ((a = taot_launch_sinkhorn(h, fs, fd, p.L, o->plan, o->sinkhorn_iters, o->row_err, o->info,
+                                         reinterpret_cast<float*>(at(ws, h->off_kt)), st)) < 0)
         return a;
     total += a;
     TAOT_MARK(3);

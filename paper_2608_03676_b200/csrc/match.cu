@@ -47,6 +47,7 @@ struct MatchArgs {
     int32_t R, E, K, dmax, ntiers, W;
     float eps0, price_step;
     int32_t auction_max_rounds;
+    int32_t ablation;            // TAOT_ABLATE_* bits: a term switched off is an exact zero in the score
     int32_t nrem_in_smem;
     int32_t tm_in_smem;
 };
@@ -194,8 +195,9 @@ match_kernel(MatchArgs a)
         const int q = (int)(idx / R), r = (int)(idx - (int64_t)q * R);
         const int hr = hot_home[q];
         const float ex = fmaxf((float)excess[hr], a.eps0);
-        const float tn = __fdiv_rn(plan[(int64_t)hr * R + r], ex);
-        t12[((int64_t)q * 2) * R + r] = __fmul_rn(alpha, a.B[(int64_t)hr * R + r]);
+        const float tn = (a.ablation & TAOT_ABLATE_HINT) ? 0.0f : __fdiv_rn(plan[(int64_t)hr * R + r], ex);
+        const float bp = (a.ablation & TAOT_ABLATE_TOPOLOGY) ? 0.0f : a.B[(int64_t)hr * R + r];
+        t12[((int64_t)q * 2) * R + r] = __fmul_rn(alpha, bp);
         t12[((int64_t)q * 2 + 1) * R + r] = __fmul_rn(beta, tn);
     }
     __syncthreads();
@@ -517,6 +519,7 @@ int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expe
     a.W = (p.R + 31) / 32;
     a.ntiers = (h->ntiers > 0 && p.price_step >= 0.0f && a.W <= kMaxW) ? h->ntiers : 0;
     a.eps0 = p.eps0; a.price_step = p.price_step; a.auction_max_rounds = p.auction_max_rounds;
+    a.ablation = p.ablation;
     size_t smem = match_smem_fixed(p.R, p.E, p.K, a.dmax, a.W, a.ntiers);
     const size_t nrem_bytes = sizeof(int32_t) * (size_t)a.dmax * p.R;
     const size_t tm_bytes = sizeof(uint32_t) * (size_t)a.ntiers * a.W * p.R * p.K;

@@ -63,6 +63,11 @@ int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expe
 int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, void* ws, const int32_t* d_slot_expert,
                        const int32_t* d_X, int32_t* d_new_idx, int32_t* d_info, cudaStream_t st);
 
+int taot_launch_report(taot_handle_t h, const int32_t* d_expert_load, const int32_t* d_rank_load,
+                       const int32_t* d_slot_expert, const int32_t* d_X, double lambda, taot_report_row* d_rows,
+                       int32_t* d_spill, int32_t* d_load_after, int32_t* d_slot_moved, int32_t* d_slot_kind,
+                       cudaStream_t st);
+
 #define TAOT_CUDA_OK(expr)                              \
     do {                                                \
         cudaError_t _e = (expr);                        \
