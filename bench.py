@@ -190,14 +190,17 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count):
         a = b / (ms * 1e-3) / 1e9
         return dict(kernel="merge_kernel", bound="hbm", achieved=a, peak=hbm, unit="GB/s", frac=a / hbm,
                     traffic=None, peak_source=peaks["source"], bytes_per_launch=b)
-    fp32_peak = sm_count * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+    derived = sm_count * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+    fp32_peak = peaks.get("fma_tflops") or derived
+    fp32_src = (f"measured: taot_measure_alu_peaks (FMA chain kernel; ex2 {peaks.get('ex2_tops', 0):.2f} T/s); "
+                f"derived figure {derived:.1f}") if peaks.get("fma_tflops") else \
+        f"derived: {sm_count} SMs x 128 fp32 lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz"
     if stage == "sinkhorn":
         fma, _ = sinkhorn_work(out, cfg)
         a = 2 * fma / (ms * 1e-3) / 1e12
         return dict(kernel="sinkhorn_tile_kernel", bound="alu", achieved=a, peak=fp32_peak, unit="TFLOP/s",
                     frac=a / fp32_peak, traffic=None,
-                    peak_source=f"derived: {sm_count} SMs x 128 fp32 lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz",
-                    flops_per_launch=2 * fma,
+                    peak_source=fp32_src, flops_per_launch=2 * fma,
                     note="one dependent chain of small mat-vecs per problem and only L problems per call: "
                          "latency-bound; DRAM traffic is ~0.1 MB per launch (ncu); the fp32-FMA fraction is "
                          "reported, not claimed as the binding limit (see profiles/sweep_config5.md for batches "
@@ -207,7 +210,7 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count):
     a = ops / (ms * 1e-3) / 1e12
     return dict(kernel="match_kernel", bound="alu", achieved=a, peak=fp32_peak / 2, unit="Tscore/s",
                 frac=a / (fp32_peak / 2), traffic=None,
-                peak_source="derived: one fp32 score evaluation per lane per clock",
+                peak_source="half the FP32 FMA peak: one fp32 score evaluation per lane per clock",
                 note="dependent rounds of masked arg-max; dense score count of the paper's formulation "
                      "(rounds x R x E and rounds x R x S), latency-bound by construction")
 
@@ -309,6 +312,8 @@ def run_ours(args):
         cfg = cfg.replace(L=args.layers)
     cfg = rank_config(cfg, rank)
     peaks = measured_peaks()
+    import paper_2608_03676_b200 as P
+    peaks.update(P.measure_alu_peaks())              # FP32-FMA and ex2 ceilings of this GPU, measured once, untimed
     props = torch.cuda.get_device_properties(local)
     topk = W.routing_topk(cfg, device="cuda")
     pl = build_planner(cfg)
@@ -402,7 +407,8 @@ def run_sweep(args):
     torch.cuda.set_device(0)
     peaks = measured_peaks()
     props = torch.cuda.get_device_properties(0)
-    fp32_peak = props.multi_processor_count * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+    alu = P.measure_alu_peaks()
+    fp32_peak = alu["fma_tflops"]                    # measured FMA-chain throughput of this GPU
     cells = []
     for (B, R, eps_frac) in W.sweep_cells():
         if B * R * R > args.sweep_max_elems:
@@ -427,7 +433,10 @@ def run_sweep(args):
         del out, loads, s, d, ex, sp
         torch.cuda.empty_cache()
     print(json.dumps(dict(metric="Sinkhorn placement plans/s per (B, R, eps) cell, 500 fixed iterations",
-                          unit="plans/s", fp32_peak_tflops=fp32_peak, cells=cells)))
+                          unit="plans/s", fp32_peak_tflops=fp32_peak, ex2_peak_tops=alu["ex2_tops"],
+                          fp32_peak_source="measured: taot_measure_alu_peaks",
+                          fp32_peak_derived=props.multi_processor_count * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12,
+                          cells=cells)))
 
 
 def main():

@@ -299,6 +299,16 @@ int taot_report(taot_handle_t h, const int32_t* d_expert_load, const int32_t* d_
 int taot_set_profiling(taot_handle_t h, int32_t on);
 int taot_get_stage_ms(taot_handle_t h, float* h_ms /* [5] */);
 
+/*
+ * Arithmetic ceilings of the current device, measured: FP32 fused multiply-add throughput (TFLOP/s, 2 flops per
+ * FMA) and ex2 special-function throughput (T op/s).  They are the denominators of the Sinkhorn stage's roofline
+ * (its inner loop is FP32 multiply-adds; its log-domain steps are ex2/lg2).  (The paper has no counterpart: a
+ * measurement aid, not a step of the method.)  Launches two register-only kernels five times each on `stream`,
+ * WAITS for them, and returns the best rate.  d_sink: device memory of at least 4 * 2048 * (number of SMs) bytes
+ * (practically never written).  h_*: host floats.  Errors: TAOT_ERR_NULL, TAOT_ERR_CUDA.
+ */
+int taot_measure_alu_peaks(float* h_fma_tflops, float* h_ex2_tops, void* d_sink, void* stream);
+
 /* Kernels launched by the last call on this handle (for launch accounting). */
 int taot_last_launch_count(taot_handle_t h, int32_t* count);
 

@@ -25,5 +25,6 @@ from .binding import (  # noqa: F401
     ABLATE_TOPOLOGY,
     INFO_INTERNAL,
     ReportRow,
+    measure_alu_peaks,
 )
 from .report import format_layer  # noqa: F401

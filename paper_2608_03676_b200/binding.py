@@ -26,7 +26,7 @@ ABLATE_TOPOLOGY = 2
 _SYMBOLS = [
     "taot_create", "taot_destroy", "taot_workspace_bytes", "taot_host_workspace_bytes",
     "taot_histogram", "taot_histogram_static", "taot_excess_spare", "taot_sinkhorn", "taot_match", "taot_assign",
-    "taot_plan", "taot_plan_host", "taot_report", "taot_set_profiling", "taot_get_stage_ms", "taot_last_launch_count",
+    "taot_plan", "taot_plan_host", "taot_report", "taot_measure_alu_peaks", "taot_set_profiling", "taot_get_stage_ms", "taot_last_launch_count",
     "taot_status_string",
 ]
 
@@ -135,6 +135,17 @@ def histogram_static(topk: torch.Tensor, R: int, E: int, e2r_dev: torch.Tensor, 
     return int(lib.taot_histogram_static(_ptr(topk), ctypes.c_int32(L), ctypes.c_int64(T), ctypes.c_int32(k),
                                          ctypes.c_int32(R), ctypes.c_int32(E), _ptr(e2r_dev), _ptr(n),
                                          _ptr(expert_load), _ptr(rank_load), _ptr(info), _stream()))
+
+
+def measure_alu_peaks() -> Dict[str, float]:
+    """FP32-FMA (TFLOP/s) and ex2 (T op/s) throughput of the current GPU, measured by `taot_measure_alu_peaks`."""
+    lib = load_library()
+    sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+    sink = torch.zeros(2048 * sms, dtype=torch.float32, device="cuda")
+    fma = ctypes.c_float(); ex2 = ctypes.c_float()
+    _check(lib.taot_measure_alu_peaks(ctypes.byref(fma), ctypes.byref(ex2), _ptr(sink), _stream()),
+           "taot_measure_alu_peaks")
+    return dict(fma_tflops=float(fma.value), ex2_tops=float(ex2.value))
 
 
 @dataclass

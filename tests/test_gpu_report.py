@@ -167,3 +167,17 @@ def test_one_hot_rank_workloads_full_path_parity():
             assert (out["slot_expert"][l].ravel() == m["slot_expert"]).all() and (out["X"][l] == a["X"]).all()
             assert (out["new_idx"][l] == O.assign(tk[l], cfg.R, cfg.E, cfg.K, m["slot_expert"], a["X"])).all()
         pl.close()
+
+
+def test_measured_alu_peaks_are_plausible():
+    """The FMA and ex2 ceilings used as roofline denominators: within a factor of the figures that the SM
+    count and clock imply (128 FMA lanes and 16 special-function lanes per SM per clock)."""
+    import paper_2608_03676_b200 as P
+    pk = P.measure_alu_peaks()
+    props = torch.cuda.get_device_properties(0)
+    clock_hz = 1.965e9
+    fma_nominal = props.multi_processor_count * 128 * 2 * clock_hz / 1e12
+    ex2_nominal = props.multi_processor_count * 16 * clock_hz / 1e12
+    assert 0.5 * fma_nominal < pk["fma_tflops"] < 1.1 * fma_nominal, pk
+    assert 0.5 * ex2_nominal < pk["ex2_tops"] < 1.1 * ex2_nominal, pk
+    print(pk, fma_nominal, ex2_nominal)
