@@ -43,6 +43,13 @@ __device__ __forceinline__ float transpose_reduce(float (&p)[N], int lane)
     return v;
 }
 
+__device__ __forceinline__ float rcp_fast(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 // Shared-memory state of one problem (arrays sized for RMAX = 32*CG ranks).
 template <int NW, int CG>
 struct TileSmem {
@@ -292,6 +299,230 @@ __device__ __forceinline__ bool tile_solve(const SinkArgs& a, TileSmem<NW, CG>& 
     return true;
 }
 
+// One-warp variant with a two-dimensional lane grid: lane = (lr, lc) with 4 row lanes x 8 column lanes; the lane
+// holds K~[ra][cg] for rows ra*4 + lr (ra < NRA) and columns cg*8 + lc (cg < NCG).  Row sums reduce over the 8
+// column lanes (3 butterfly shuffles per ra), column sums over the 4 row lanes (2 shuffles per cg); after a
+// butterfly every lane of the group holds the same bits, so u~ and v~ are computed redundantly where they are
+// needed and nothing is broadcast.  For the small problems of the planner (a few supply ranks, tens of demand
+// ranks) this is a much shorter dependent chain per iteration than one row set per lane.
+template <int NRA, int NCG, int CG>
+__device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& sm, int Hn, int Cn, double sum_st,
+                                           int info, float* out, int64_t b)
+{
+    constexpr int RL = 4, CL = 8;
+    const int R = a.R, lane = threadIdx.x & 31;
+    const int lr = lane >> 3, lc = lane & 7;
+    const double tol_abs = (double)a.tol * sum_st;
+
+    float K[NRA][NCG];
+    float stl[NRA], uo[NRA], ddg[NCG], vreg[NCG];
+    bool row_ok[NRA], col_ok[NCG];
+#pragma unroll
+    for (int ra = 0; ra < NRA; ++ra) {
+        const int row = ra * RL + lr;
+        row_ok[ra] = row < Hn;
+        stl[ra] = row_ok[ra] ? sm.st[row] : 1.0f;
+        uo[ra] = 1.0f;
+    }
+#pragma unroll
+    for (int cg = 0; cg < NCG; ++cg) {
+        const int col = cg * CL + lc;
+        col_ok[cg] = col < Cn;
+        ddg[cg] = col_ok[cg] ? sm.dd[col] : 1.0f;
+        vreg[cg] = 1.0f;
+    }
+    auto build_tile = [&]() {
+#pragma unroll
+        for (int ra = 0; ra < NRA; ++ra) {
+            const int row = ra * RL + lr;
+#pragma unroll
+            for (int cg = 0; cg < NCG; ++cg) {
+                const int col = cg * CL + lc;
+                float v = 0.0f;
+                if (row < Hn && col < Cn) {
+                    const double c = (double)a.C[(int64_t)sm.hot[row] * R + sm.cold[col]] * a.inv_eps;
+                    v = (float)exp(sm.alpha[row] + sm.beta[col] - c);
+                }
+                K[ra][cg] = v;
+            }
+        }
+    };
+    build_tile();
+    int t = 1;
+    int until_check = a.check_every;
+    float err_out = 0.0f;
+    const float tol_abs_f = (float)tol_abs;
+    const uint32_t lo_bits = __float_as_uint(kDriftLo), span_bits = __float_as_uint(kDriftHi) - lo_bits;
+
+    for (;;) {
+        // Drift test on the u~, v~ this iteration STARTS from; the vote is issued here and consumed at the end of
+        // the iteration, so neither it nor the branch it feeds sits on the dependent chain.  Acting one update
+        // late is safe: a value that left [e^-20, e^20] is still far inside the fp32 range, and should an update
+        // jump past that range after all, its sums leave (kSumLo, kSumHi) and the problem is handed back.
+        bool odd = false;
+#pragma unroll
+        for (int ra = 0; ra < NRA; ++ra) odd |= (__float_as_uint(uo[ra]) - lo_bits) > span_bits;
+#pragma unroll
+        for (int cg = 0; cg < NCG; ++cg) odd |= (__float_as_uint(vreg[cg]) - lo_bits) > span_bits;
+        odd = __any_sync(kFull, odd);
+        // ================= half-step 1: r = K~ v~, u' = s~ / r
+        float r[NRA], un[NRA];
+#pragma unroll
+        for (int ra = 0; ra < NRA; ++ra) {
+            float acc = K[ra][0] * vreg[0];
+#pragma unroll
+            for (int cg = 1; cg < NCG; ++cg) acc = fmaf(K[ra][cg], vreg[cg], acc);
+            r[ra] = acc;
+        }
+#pragma unroll
+        for (int off = 1; off < CL; off <<= 1) {
+#pragma unroll
+            for (int ra = 0; ra < NRA; ++ra) r[ra] += __shfl_xor_sync(kFull, r[ra], off);
+        }
+#pragma unroll
+        for (int ra = 0; ra < NRA; ++ra) un[ra] = row_ok[ra] ? stl[ra] * rcp_fast(r[ra]) : 1.0f;
+        // ================= half-step 2 (speculative until the stop test): c = K~^T u', v' = d / c
+        float cp[NCG], vnew[NCG];
+#pragma unroll
+        for (int cg = 0; cg < NCG; ++cg) {
+            float acc = K[0][cg] * un[0];
+#pragma unroll
+            for (int ra = 1; ra < NRA; ++ra) acc = fmaf(K[ra][cg], un[ra], acc);
+            cp[cg] = acc;
+        }
+#pragma unroll
+        for (int off = CL; off < 32; off <<= 1) {
+#pragma unroll
+            for (int cg = 0; cg < NCG; ++cg) cp[cg] += __shfl_xor_sync(kFull, cp[cg], off);
+        }
+        // ---- the row sums belong to iterate t: is this where the solve stops?
+        const bool last = t >= a.max_iters;
+        const bool check = a.tol > 0.0f && until_check == 1;
+        float err = 0.0f;
+        if (last || check) {                                             // uniform over the warp
+            float e = 0.0f;
+#pragma unroll
+            for (int ra = 0; ra < NRA; ++ra) e += row_ok[ra] ? fabsf(fmaf(uo[ra], r[ra], -stl[ra])) : 0.0f;
+#pragma unroll
+            for (int off = CL; off < 32; off <<= 1) e += __shfl_xor_sync(kFull, e, off);
+            err = e;                                                     // the same bits in every lane
+        }
+#pragma unroll
+        for (int cg = 0; cg < NCG; ++cg) vnew[cg] = col_ok[cg] ? ddg[cg] * rcp_fast(cp[cg]) : 1.0f;
+        if (last || (check && err <= tol_abs_f)) {
+            bool bad_r = false;
+#pragma unroll
+            for (int ra = 0; ra < NRA; ++ra) bad_r |= row_ok[ra] && !(r[ra] > kSumLo && r[ra] < kSumHi);
+            if (__any_sync(kFull, bad_r)) return false;
+            err_out = (float)((double)err / sum_st);
+            if (a.tol > 0.0f && !(err <= tol_abs_f)) info |= TAOT_INFO_SINKHORN_CAP;
+            break;
+        }
+        // ---- commit iteration t+1
+#pragma unroll
+        for (int ra = 0; ra < NRA; ++ra) uo[ra] = un[ra];
+#pragma unroll
+        for (int cg = 0; cg < NCG; ++cg) vreg[cg] = vnew[cg];
+        ++t;
+        until_check = until_check == 1 ? a.check_every : until_check - 1;
+        if (odd) {
+            // rare: either u~, v~ merely drifted (fold them into the potentials) or a sum of this update left the
+            // range in which fp32 products are trustworthy (hand the problem back)
+            bool bad = false;
+#pragma unroll
+            for (int ra = 0; ra < NRA; ++ra) bad |= row_ok[ra] && !(r[ra] > kSumLo && r[ra] < kSumHi);
+#pragma unroll
+            for (int cg = 0; cg < NCG; ++cg) bad |= col_ok[cg] && !(cp[cg] > kSumLo && cp[cg] < kSumHi);
+            if (__any_sync(kFull, bad)) return false;
+            // fold u~, v~ into the fp64 potentials (one lane per row / column) and rebuild the tile around them
+#pragma unroll
+            for (int ra = 0; ra < NRA; ++ra)
+                if (row_ok[ra] && lc == 0) sm.alpha[ra * RL + lr] += log((double)uo[ra]);
+#pragma unroll
+            for (int cg = 0; cg < NCG; ++cg)
+                if (col_ok[cg] && lr == 0) sm.beta[cg * CL + lc] += log((double)vreg[cg]);
+            __syncwarp();
+#pragma unroll
+            for (int ra = 0; ra < NRA; ++ra) uo[ra] = 1.0f;
+#pragma unroll
+            for (int cg = 0; cg < NCG; ++cg) vreg[cg] = 1.0f;
+            build_tile();
+        }
+    }
+
+    // ---- T = diag(u) M diag(v) from the total potentials, then the column cap
+#pragma unroll
+    for (int ra = 0; ra < NRA; ++ra)
+        if (row_ok[ra] && lc == 0) sm.alpha[ra * RL + lr] += log((double)uo[ra]);
+#pragma unroll
+    for (int cg = 0; cg < NCG; ++cg)
+        if (col_ok[cg] && lr == 0) sm.beta[cg * CL + lc] += log((double)vreg[cg]);
+    __syncwarp();
+    build_tile();
+    float fg[NCG];
+#pragma unroll
+    for (int cg = 0; cg < NCG; ++cg) {
+        float acc = 0.0f;
+#pragma unroll
+        for (int ra = 0; ra < NRA; ++ra) acc += K[ra][cg];
+#pragma unroll
+        for (int off = CL; off < 32; off <<= 1) acc += __shfl_xor_sync(kFull, acc, off);
+        fg[cg] = col_ok[cg] ? (float)fmin(1.0, (double)ddg[cg] / ((double)acc + (double)a.eps0)) : 0.0f;
+    }
+    for (int q = lane; q < R * R; q += 32) out[q] = 0.0f;
+    __syncwarp();
+    int nonfinite = 0;
+#pragma unroll
+    for (int ra = 0; ra < NRA; ++ra) {
+        if (!row_ok[ra]) continue;
+        float* orow = out + (int64_t)sm.hot[ra * RL + lr] * R;
+#pragma unroll
+        for (int cg = 0; cg < NCG; ++cg) {
+            if (!col_ok[cg]) continue;
+            const float val = K[ra][cg] * fg[cg];
+            if (!isfinite(val)) nonfinite = 1;
+            orow[sm.cold[cg * CL + lc]] = val;
+        }
+    }
+    if (__any_sync(kFull, nonfinite != 0)) info |= TAOT_INFO_NONFINITE;
+    if (lane == 0) {
+        a.iters[b] = t;
+        a.row_err[b] = err_out;
+        if (info) atomicOr(a.info + b, info);
+    }
+    return true;
+}
+
+// Picks the smallest lane-grid tile that holds the problem (one warp); false: hand the problem back.
+template <int CG>
+__device__ __forceinline__ bool grid_dispatch(const SinkArgs& a, TileSmem<1, CG>& sm, int Hn, int Cn, double sum_st,
+                                              int info, float* out, int64_t b)
+{
+#define TAOT_GRID(NRA, NCG) grid_solve<NRA, NCG, CG>(a, sm, Hn, Cn, sum_st, info, out, b)
+    if (CG == 1) {                     // up to 32 ranks
+        if (Cn <= 16) {
+            if (Hn <= 4) return TAOT_GRID(1, 2);
+            if (Hn <= 8) return TAOT_GRID(2, 2);
+            if (Hn <= 16) return TAOT_GRID(4, 2);
+            return TAOT_GRID(8, 2);
+        }
+        if (Hn <= 4) return TAOT_GRID(1, 4);
+        if (Hn <= 8) return TAOT_GRID(2, 4);
+        if (Hn <= 16) return TAOT_GRID(4, 4);
+        return TAOT_GRID(8, 4);
+    } else {                           // up to 64 ranks
+        if (Cn <= 32) {
+            if (Hn <= 8) return TAOT_GRID(2, 4);
+            if (Hn <= 16) return TAOT_GRID(4, 4);
+            return TAOT_GRID(8, 4);
+        }
+        if (Hn <= 8) return TAOT_GRID(2, 8);
+        if (Hn <= 16) return TAOT_GRID(4, 8);
+        return TAOT_GRID(8, 8);
+    }
+#undef TAOT_GRID
+}
+
 // RP0 < RP1 < RP2: rows-per-warp variants; the smallest that holds the problem's supply ranks runs.
 template <int NW, int CG, int RP0, int RP1, int RP2>
 __global__ void __launch_bounds__(NW * 32)
@@ -334,7 +565,7 @@ sinkhorn_tile_kernel(SinkArgs a)
     __syncthreads();
     const int Hn = compact_positive(sm.sv, R, sm.hot, sm.hpos, sm.wcnt);
     const int Cn = compact_positive(sm.dv, R, sm.cold, sm.cpos, sm.wcnt);
-    if (Hn > NW * RP2) {                     // does not fit any tile: the other kernel takes it
+    if (Hn > (NW == 1 ? 32 : NW * RP2)) {    // does not fit any tile: the other kernel takes it
         if (tid == 0) a.iters[b] = kHandBack;
         return;
     }
@@ -377,7 +608,8 @@ sinkhorn_tile_kernel(SinkArgs a)
     __syncthreads();
 
     bool done;
-    if (Hn <= NW * RP0) done = tile_solve<NW, RP0, CG>(a, sm, Hn, Cn, sum_st, info, out, b);
+    if constexpr (NW == 1) done = grid_dispatch<CG>(a, sm, Hn, Cn, sum_st, info, out, b);
+    else if (Hn <= NW * RP0) done = tile_solve<NW, RP0, CG>(a, sm, Hn, Cn, sum_st, info, out, b);
     else if (Hn <= NW * RP1) done = tile_solve<NW, RP1, CG>(a, sm, Hn, Cn, sum_st, info, out, b);
     else done = tile_solve<NW, RP2, CG>(a, sm, Hn, Cn, sum_st, info, out, b);
     if (!done && tid == 0) a.iters[b] = kHandBack;
