@@ -125,7 +125,7 @@ __device__ __forceinline__ bool tile_solve(const SinkArgs& a, TileSmem<NW, CG>& 
             p[aa] = acc;
         }
         const float r = transpose_reduce<RPW>(p, lane);
-        const float un = row_ok ? st_l * __frcp_rn(r) : 1.0f;
+        const float un = row_ok ? st_l * rcp_fast(r) : 1.0f;
         bool odd = (__float_as_uint(un) - lo_bits) > span_bits;       // out of range: fold, or hand back
         // ================= half-step 2 (speculative until the stop test): c = K~^T u', v' = d / c
         float cp[CG];
@@ -150,7 +150,7 @@ __device__ __forceinline__ bool tile_solve(const SinkArgs& a, TileSmem<NW, CG>& 
         if (NW == 1) {
 #pragma unroll
             for (int g = 0; g < CG; ++g) {
-                const float vn = col_ok[g] ? ddg[g] * __frcp_rn(cp[g]) : 1.0f;
+                const float vn = col_ok[g] ? ddg[g] * rcp_fast(cp[g]) : 1.0f;
                 odd |= (__float_as_uint(vn) - lo_bits) > span_bits;
                 vnew[g] = vn;
             }
@@ -181,7 +181,7 @@ __device__ __forceinline__ bool tile_solve(const SinkArgs& a, TileSmem<NW, CG>& 
                 float c = 0.0f;
 #pragma unroll
                 for (int w = 0; w < NW; ++w) c += sm.part[w * RMAX + j];
-                const float vn = sm.dd[j] * __frcp_rn(c);
+                const float vn = sm.dd[j] * rcp_fast(c);
                 if ((__float_as_uint(vn) - lo_bits) > span_bits) sm.flags[par] = 1;
                 sm.vs[j] = vn;
             }
