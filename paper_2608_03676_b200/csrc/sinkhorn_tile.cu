@@ -510,15 +510,18 @@ __device__ __forceinline__ bool grid_dispatch(const SinkArgs& a, TileSmem<1, CG>
         if (Hn <= 8) return TAOT_GRID(2, 4);
         if (Hn <= 16) return TAOT_GRID(4, 4);
         return TAOT_GRID(8, 4);
-    } else {                           // up to 64 ranks
-        if (Cn <= 32) {
-            if (Hn <= 8) return TAOT_GRID(2, 4);
-            if (Hn <= 16) return TAOT_GRID(4, 4);
-            return TAOT_GRID(8, 4);
-        }
-        if (Hn <= 8) return TAOT_GRID(2, 8);
-        if (Hn <= 16) return TAOT_GRID(4, 8);
-        return TAOT_GRID(8, 8);
+    } else {                           // up to 64 ranks: rows in steps of 4 (NRA), columns in steps of 16 (NCG = 4, 6, 8)
+#define TAOT_GRID_ROWS(NCG)                                  \
+        if (Hn <= 8) return TAOT_GRID(2, NCG);              \
+        if (Hn <= 12) return TAOT_GRID(3, NCG);             \
+        if (Hn <= 16) return TAOT_GRID(4, NCG);             \
+        if (Hn <= 20) return TAOT_GRID(5, NCG);             \
+        if (Hn <= 24) return TAOT_GRID(6, NCG);             \
+        return TAOT_GRID(8, NCG);
+        if (Cn <= 32) { TAOT_GRID_ROWS(4) }
+        if (Cn <= 48) { TAOT_GRID_ROWS(6) }
+        TAOT_GRID_ROWS(8)
+#undef TAOT_GRID_ROWS
     }
 #undef TAOT_GRID
 }
