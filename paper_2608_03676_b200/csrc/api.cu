@@ -57,18 +57,19 @@ void layout(taot_handle_t h)
     const int dmax = p.E < p.R * p.K ? p.E : p.R * p.K;
     size_t off = 0;
     auto take = [&](size_t bytes) { const size_t o = off; off = taot_align_up(off + bytes, 256); return o; };
-    h->off_cc = take(sizeof(int32_t) * LR * h->nc * p.E);
-    h->off_tabg = take(sizeof(int32_t) * LR * h->nc * (p.E + 20));   // E targets + row tail (assign.cu: kRowTail)
-    h->off_nbg = take(sizeof(int32_t) * LR * h->nc);
-    h->off_soff = take(sizeof(int32_t) * LR * h->nc);
+    const size_t path = p.R <= 256 ? 1 : 0;       // beyond 256 ranks only Phase 1 runs: no schedule buffers
+    h->off_cc = take(path * sizeof(int32_t) * LR * h->nc * p.E);
+    h->off_tabg = take(path * sizeof(int32_t) * LR * h->nc * (p.E + 20));   // E targets + row tail (assign.cu: kRowTail)
+    h->off_nbg = take(path * sizeof(int32_t) * LR * h->nc);
+    h->off_soff = take(path * sizeof(int32_t) * LR * h->nc);
     h->off_work = take(16);
-    h->off_splits = take(16 * LR * (size_t)p.R * p.K);
+    h->off_splits = take(path * 16 * LR * (size_t)p.R * p.K);
     h->off_excess = take(sizeof(int32_t) * LR);
     h->off_spare = take(sizeof(int32_t) * LR);
     h->off_s = take(sizeof(float) * LR);
     h->off_d = take(sizeof(float) * LR);
-    h->off_nrem = take(sizeof(int32_t) * (size_t)p.L * dmax * p.R);
-    h->off_t12 = take(sizeof(float) * (size_t)p.L * p.E * 2 * p.R);
+    h->off_nrem = take(path * sizeof(int32_t) * (size_t)p.L * dmax * p.R);
+    h->off_t12 = take(path * sizeof(float) * (size_t)p.L * p.E * 2 * p.R);
     h->off_kt = take(sizeof(float) * (size_t)p.L * (size_t)h->kcap_global);
     h->ws_bytes = off;
 
