@@ -51,6 +51,8 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=0, help="override L (smaller batch, e.g. for a profiler capture)")
     ap.add_argument("--cpu-seconds", type=float, default=20.0, help="budget of the CPU-baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-groups", type=int, default=4,
+                    help="layer groups (streams) the end-to-end host call is pipelined over")
     ap.add_argument("--no-streams", action="store_true", help="skip the HBM-sized streaming report")
     ap.add_argument("--sweep", action="store_true",
                     help="config 5: time taot_sinkhorn alone over the (B, R, eps) grid and print one JSON object")
@@ -346,11 +348,30 @@ def run_ours(args):
     total_s = max_over_ranks(sum(ms), world, "cuda") * 1e-3
     value = whole_job_rate(cfg.L, args.steps, world, total_s * 1e3)
 
+    # the same step replayed from a CUDA graph (captured once, untimed): launch gaps shrink, the kernels are the same
+    graph_ms = None
+    if world == 1:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            pl.plan(topk, out)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            pl.plan(topk, out)
+        timed_steps(g.replay, 3, flush)
+        graph_ms = timed_steps(g.replay, args.steps, flush)
+
     # end to end through the host-buffer entry point
     host_in = topk.cpu().pin_memory()
-    host_out = pl.alloc_host_outputs(("plan", "slot_expert", "slot_tokens", "X", "new_idx", "info"))
+    e2r_h = W.expert_to_rank(cfg.E, cfg.R, cfg.e2r_mode)
+    C_h = W.cost_matrix(cfg.R, cfg.gpus_per_node, cfg.tiers, cfg.nodes_per_group)
+    hp = P.PipelinedHostPlanner(L=cfg.L, groups=args.e2e_groups, R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k, T=cfg.T,
+                                e2r=e2r_h, C=C_h, eps=cfg.eps, max_iters=cfg.max_iters, tol=cfg.tol)
+    host_out = hp.alloc_host_outputs(("plan", "slot_expert", "slot_tokens", "X", "new_idx", "info"))
     d2h = sum(t.numel() * t.element_size() for t in host_out.values())
-    e2e_step = lambda: pl.plan_host(host_in, host_out)
+    e2e_step = lambda: hp.plan_host(host_in, host_out)
     timed_steps(e2e_step, 3, flush)
     barrier(); torch.cuda.synchronize()
     e2e_ms = timed_steps(e2e_step, args.steps, flush)
@@ -383,9 +404,13 @@ def run_ours(args):
         rounds=dict(phase2_max=int(rounds[:, 0].max()), phase3_max=int(rounds[:, 1].max())),
         roofline=roof, clocks=clocks,
         e2e=dict(value=e2e_value, unit="plans/s", h2d_bytes_per_step=topk_bytes, d2h_bytes_per_step=d2h,
-                 ms_per_step=float(np.mean(e2e_ms))),
+                 ms_per_step=float(np.mean(e2e_ms)),
+                 api=f"PipelinedHostPlanner.plan_host: taot_plan_host on {len(hp.planners)} groups of layers, one stream each"),
         gpu_launches=launches,
     )
+    if graph_ms is not None:
+        line["cuda_graph"] = dict(ms_per_step=float(np.mean(graph_ms)), value=cfg.L / (float(np.mean(graph_ms)) * 1e-3),
+                                  unit="plans/s", note="the same taot_plan call captured once and replayed")
     line["rooflines"] = {s: roofline_for(s, float(stage_ms[i]), cfg, out, peaks, props.multi_processor_count)
                          for i, s in enumerate(STAGES)}
 

@@ -26,5 +26,6 @@ from .binding import (  # noqa: F401
     INFO_INTERNAL,
     ReportRow,
     measure_alu_peaks,
+    PipelinedHostPlanner,
 )
 from .report import format_layer  # noqa: F401

@@ -342,3 +342,49 @@ class Planner:
         _check(self.lib.taot_plan_host(self.handle, _ptr(topk_host), ctypes.byref(o), _ptr(self._host_ws),
                                        _stream()), "taot_plan_host")
         return out_host
+
+
+class PipelinedHostPlanner:
+    """`taot_plan_host` over groups of layers on separate streams, so that the host-to-device copy of one group,
+    the kernels of another and the device-to-host copy of a third overlap (the L problems of a call are
+    independent, so splitting the batch changes no result).  Holds one `Planner` (handle, workspace, staging) per
+    group; `plan_host` enqueues every group and makes the caller's current stream wait for all of them."""
+
+    def __init__(self, L: int, groups: int = 4, **planner_kwargs):
+        groups = max(1, min(groups, L))
+        base, extra = divmod(L, groups)
+        self.bounds = []
+        lo = 0
+        for g in range(groups):
+            hi = lo + base + (1 if g < extra else 0)
+            self.bounds.append((lo, hi))
+            lo = hi
+        self.planners = [Planner(L=hi - lo, **planner_kwargs) for lo, hi in self.bounds]
+        self.streams = [torch.cuda.Stream() for _ in self.planners]
+        self.L = L
+
+    def alloc_host_outputs(self, names=("plan", "slot_expert", "slot_tokens", "X", "new_idx", "info")):
+        parts = [p.alloc_host_outputs(names) for p in self.planners]
+        # one pinned tensor per output, of which every group sees its slice
+        out = {}
+        for nm in names:
+            shape = (self.L,) + tuple(parts[0][nm].shape[1:])
+            out[nm] = torch.empty(shape, dtype=parts[0][nm].dtype).pin_memory()
+        return out
+
+    def plan_host(self, topk_host: torch.Tensor, out_host: Dict[str, torch.Tensor]) -> Dict[str, torch.Tensor]:
+        cur = torch.cuda.current_stream()
+        for (lo, hi), pl, st in zip(self.bounds, self.planners, self.streams):
+            st.wait_stream(cur)
+            with torch.cuda.stream(st):
+                pl.plan_host(topk_host[lo:hi], {k: v[lo:hi] for k, v in out_host.items()})
+        for st in self.streams:
+            cur.wait_stream(st)
+        return out_host
+
+    def launch_count(self) -> int:
+        return sum(p.last_launch_count() for p in self.planners)
+
+    def close(self):
+        for p in self.planners:
+            p.close()

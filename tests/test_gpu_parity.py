@@ -168,3 +168,65 @@ def test_auction_scores_that_round_together_and_a_round_cap():
             assert out["rounds"][l, 1] == a["rounds"]
             assert bool(out["info"][l] & 8) == (a["residual"] > 0)
         pl.close()
+
+
+def test_plan_is_capturable_in_a_cuda_graph():
+    """taot_plan neither allocates nor synchronises, so a stream capture of it replays to the same bits
+    (the paper stresses CUDA-graph compatibility of the planner, Appendix A.4)."""
+    cfg = W.get_config("cfg2").replace(L=4)
+    topk = _routing(cfg)
+    pl = make_planner(cfg)
+    out = pl.alloc_outputs()
+    pl.plan(topk, out)
+    torch.cuda.synchronize()
+    want = {k: cpu(v).copy() for k, v in out.items()}
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        pl.plan(topk, out)                       # warm-up on the capture stream
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        pl.plan(topk, out)
+    for _ in range(3):
+        for v in out.values():
+            v.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        for key, val in out.items():
+            assert (cpu(val) == want[key]).all(), key
+    # new routing written into the captured input buffer is planned by the next replay
+    cfg2 = cfg.replace(seed=cfg.seed + 1)
+    topk2 = _routing(cfg2)
+    fresh = {k: cpu(v).copy() for k, v in pl.plan(topk2).items()}
+    topk.copy_(topk2)
+    g.replay()
+    torch.cuda.synchronize()
+    for key, val in out.items():
+        assert (cpu(val) == fresh[key]).all(), key
+    pl.close()
+
+
+def test_pipelined_host_planner_equals_the_single_call():
+    import paper_2608_03676_b200 as P
+    cfg = W.get_config("cfg2").replace(L=7)            # 7 layers over 3 groups: uneven split
+    e2r, C = topology(cfg)
+    topk = _routing(cfg)
+    pl = make_planner(cfg)
+    want = {k: cpu(v) for k, v in pl.plan(topk).items()}
+    hp = P.PipelinedHostPlanner(L=cfg.L, groups=3, R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k, T=cfg.T, e2r=e2r, C=C,
+                                eps=cfg.eps, max_iters=cfg.max_iters, tol=cfg.tol)
+    assert [hi - lo for lo, hi in hp.bounds] == [3, 2, 2]
+    names = ("n", "plan", "sinkhorn_iters", "slot_expert", "slot_tokens", "X", "new_idx", "info", "rounds")
+    host_out = hp.alloc_host_outputs(names)
+    host_in = topk.cpu().pin_memory()
+    for _ in range(2):
+        for v in host_out.values():
+            v.zero_()
+        hp.plan_host(host_in, host_out)
+        torch.cuda.synchronize()
+        for key in names:
+            assert (host_out[key].numpy() == want[key]).all(), key
+    assert hp.launch_count() == 3 * P.PLAN_LAUNCHES
+    hp.close(); pl.close()
