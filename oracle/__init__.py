@@ -16,6 +16,7 @@ from .binding import (  # noqa: F401
     assign,
     plan_layers,
     report,
+    dispatch,
     REPORT_INTS,
     REPORT_REALS,
 )

@@ -150,6 +150,39 @@ def assign(topk_layer, R: int, E: int, K: int, slot_expert, X) -> np.ndarray:
     return out
 
 
+def dispatch(new_idx_layer, R: int, E: int, K: int, e2r):
+    """Dispatch metadata of one rewritten routing table (the step after the planner: what the token
+    all-to-all needs).  new_idx_layer int32 [T,k]: e in [0,E) = expert e on its home rank, E + s = guest slot
+    s on rank s // K.  Source rank r owns the R contiguous segments of T/R*k entries.
+
+    Definition, per source rank: order its entries by (destination rank, target index) keeping the original
+    flat order among equal keys (a stable sort); perm[i] is the position of entry i in that order, i.e. its
+    place in the rank's send buffer.  send_counts[r][q] = entries of source rank r that execute on rank q;
+    target_counts[r][t] = entries of source rank r with target t (t < E + S).  An index outside [0, E + S)
+    cannot be delivered: it is counted nowhere and sorts after every valid entry, in its original order.
+
+    Returns dict(perm int32 [T,k], send_counts int32 [R,R], target_counts int32 [R,E+S], bad int)."""
+    x = _i32(new_idx_layer)
+    T, k = x.shape
+    S = R * K
+    e2r = _i32(e2r).astype(np.int64)
+    seg = T // R * k
+    flat = x.reshape(R, seg).astype(np.int64)
+    valid = (flat >= 0) & (flat < E + S)
+    safe = np.where(valid, flat, 0)
+    dest = np.where(safe < E, e2r[np.minimum(safe, E - 1)], (safe - E) // K)
+    key = np.where(valid, dest * (E + S) + safe, R * (E + S))
+    perm = np.empty((R, seg), np.int32)
+    send = np.zeros((R, R), np.int32)
+    tc = np.zeros((R, E + S), np.int32)
+    for r in range(R):
+        order = np.argsort(key[r], kind="stable")
+        perm[r, order] = np.arange(seg, dtype=np.int32)
+        send[r] = np.bincount(dest[r][valid[r]], minlength=R)
+        tc[r] = np.bincount(flat[r][valid[r]], minlength=E + S)
+    return dict(perm=perm.reshape(T, k), send_counts=send, target_counts=tc, bad=int((~valid).sum()))
+
+
 REPORT_INTS = ("total_load", "rerouted", "mean_load", "max_before", "min_before", "max_after", "min_after",
                "hot_ranks", "cold_ranks", "hot_experts", "clones", "intra", "inter", "same_rank")
 REPORT_REALS = ("rho_before", "rho_after", "dev_before", "dev_after", "peak_reduction", "frac_rerouted",
