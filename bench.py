@@ -257,6 +257,13 @@ def stream_report(name, peaks, steps=5):
                plans_per_s=cfg.L / (acc.sum() * 1e-3))
     rep["histogram_frac"] = rep["histogram_gbs"] / peaks["hbm_gbs"]
     rep["assign_frac"] = rep["assign_gbs"] / peaks["hbm_gbs"]
+    # the step after the path: dispatch metadata (two reads of the rewritten table, one write of the positions)
+    dsp = pl.dispatch(out["new_idx"])
+    dms = timed_steps(lambda: pl.dispatch(out["new_idx"], out=dsp), steps, None)
+    rep["dispatch_ms"] = float(np.mean(dms))
+    rep["dispatch_gbs"] = 3 * b / (rep["dispatch_ms"] * 1e-3) / 1e9
+    rep["dispatch_frac"] = rep["dispatch_gbs"] / peaks["hbm_gbs"]
+    del dsp
     pl.close()
     del topk, out
     torch.cuda.empty_cache()

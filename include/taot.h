@@ -15,6 +15,7 @@
  *   taot_plan           all of the above chained on one stream
  *   taot_plan_host      taot_plan with host buffers (copies in and out on the same stream)
  *   taot_report         the per-layer dispatch diagnostics of a finished plan        (Appendix B.3)
+ *   taot_dispatch       send counts and send-buffer positions for the token all-to-all that follows
  *
  * Conventions
  *   - Shapes: L problems, R ranks, E experts, K guest slots per rank, S = R*K slots
@@ -246,6 +247,24 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* out, v
  */
 int taot_plan_host(taot_handle_t h, const int32_t* h_topk, const taot_outputs* out, void* d_ws,
                    void* stream);
+
+/*
+ * Dispatch metadata for the token all-to-all that follows the planner (Method: the rewritten routing is what the
+ * dispatcher executes; the paper does not spell the bookkeeping out, so the layout below is this library's).
+ * For each problem l and source rank r (the R contiguous segments of (T/R)*k entries of d_new_idx[l]):
+ *   d_send_counts [L,R,R]      [l][r][q] = entries of source rank r that execute on rank q
+ *                              (target e < E executes on its home rank, target E + s on rank s / K)
+ *   d_target_counts [L,R,E+S]  [l][r][t] = entries of source rank r with target t; optional (NULL to skip)
+ *   d_perm [L,T,k]             position of every entry in its source rank's send buffer when that buffer is ordered
+ *                              by (destination rank, target index, original flat order): a stable sort, so
+ *                              send_buffer[perm[i]] = entry i; positions run over [0, (T/R)*k) per source rank
+ * An index outside [0, E+S) cannot be delivered: it is counted nowhere, its positions follow all valid entries in
+ * original order, and TAOT_INFO_BAD_INDEX is set.  d_perm must not alias d_new_idx.  Uses `ws`.
+ * Errors: TAOT_ERR_NULL, TAOT_ERR_ALIGN (4-byte tables, 256-byte ws), TAOT_ERR_PARAM (aliasing),
+ * TAOT_ERR_UNSUPPORTED (R > 256).
+ */
+int taot_dispatch(taot_handle_t h, const int32_t* d_new_idx, int32_t* d_send_counts, int32_t* d_target_counts,
+                  int32_t* d_perm, int32_t* d_info, void* ws, void* stream);
 
 /*
  * One layer's dispatch diagnostics (Appendix B.3; metric definitions of the Evaluation section).  128 bytes.

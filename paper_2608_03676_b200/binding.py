@@ -26,7 +26,7 @@ ABLATE_TOPOLOGY = 2
 _SYMBOLS = [
     "taot_create", "taot_destroy", "taot_workspace_bytes", "taot_host_workspace_bytes",
     "taot_histogram", "taot_histogram_static", "taot_excess_spare", "taot_sinkhorn", "taot_match", "taot_assign",
-    "taot_plan", "taot_plan_host", "taot_report", "taot_measure_alu_peaks", "taot_set_profiling", "taot_get_stage_ms", "taot_last_launch_count",
+    "taot_plan", "taot_plan_host", "taot_report", "taot_dispatch", "taot_measure_alu_peaks", "taot_set_profiling", "taot_get_stage_ms", "taot_last_launch_count",
     "taot_status_string",
 ]
 
@@ -286,6 +286,24 @@ class Planner:
                                     _ptr(_dev(X, torch.int32, "X")), _ptr(new), _ptr(info), _ptr(self.ws),
                                     ctypes.c_int32(1 if reuse_counts else 0), _stream()), "taot_assign")
         return new, info
+
+    def dispatch(self, new_idx: torch.Tensor, info: Optional[torch.Tensor] = None, want_target_counts: bool = True,
+                 out: Optional[Dict[str, torch.Tensor]] = None):
+        """Send counts [L,R,R], target counts [L,R,E+S] and send-buffer positions [L,T,k] of a rewritten routing
+        table, through `taot_dispatch`.  `out`: a dict returned by an earlier call, to reuse its tensors."""
+        _dev(new_idx, torch.int32, "new_idx")
+        L, R, E, S = self.L, self.R, self.E, self.S
+        if out is not None:
+            send, tc, perm, info = out["send_counts"], out["target_counts"], out["perm"], out["info"]
+            info.zero_()
+        else:
+            send = self._empty((L, R, R), torch.int32)
+            tc = self._empty((L, R, E + S), torch.int32) if want_target_counts else None
+            perm = torch.empty_like(new_idx)
+            info = torch.zeros((L,), dtype=torch.int32, device=self.device) if info is None else info
+        _check(self.lib.taot_dispatch(self.handle, _ptr(new_idx), _ptr(send), _ptr(tc), _ptr(perm), _ptr(info),
+                                      _ptr(self.ws), _stream()), "taot_dispatch")
+        return dict(send_counts=send, target_counts=tc, perm=perm, info=info)
 
     def report(self, expert_load, rank_load, slot_expert, X, lam: float = 3.0) -> Dict[str, object]:
         """Dispatch diagnostics of L finished plans through `taot_report`.  Returns the row fields as numpy

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libtaot.so")
 OBJ = os.path.join(PKG, "csrc", "build")
-SOURCES = ["api.cu", "histogram.cu", "sinkhorn.cu", "sinkhorn_tile.cu", "match.cu", "assign.cu", "report.cu", "peaks.cu"]
+SOURCES = ["api.cu", "histogram.cu", "sinkhorn.cu", "sinkhorn_tile.cu", "match.cu", "assign.cu", "report.cu", "peaks.cu", "dispatch.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v",
               "-I", os.path.join(ROOT, "include"), "-I", CSRC] + os.environ.get("TAOT_EXTRA_NVCC_FLAGS", "").split()

@@ -71,6 +71,7 @@ void layout(taot_handle_t h)
     h->off_nrem = take(path * sizeof(int32_t) * (size_t)p.L * dmax * p.R);
     h->off_t12 = take(path * sizeof(float) * (size_t)p.L * p.E * 2 * p.R);
     h->off_kt = take(sizeof(float) * (size_t)p.L * (size_t)h->kcap_global);
+    h->off_dc = take(path * sizeof(int32_t) * LR * h->nc * ((size_t)p.E + (size_t)p.R * p.K + 1));
     h->ws_bytes = off;
 
     const size_t S = (size_t)p.R * p.K;
@@ -222,6 +223,20 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
     if (rc == TAOT_OK) rc = upload(&h->d_rank_off, off.data(), (size_t)R + 1);
     if (rc == TAOT_OK) rc = upload(&h->d_rank_list, list.data(), (size_t)E);
     if (rc == TAOT_OK && h->ntiers > 0) rc = upload(&h->d_tierval, tierval.data(), tierval.size());
+    if (rc == TAOT_OK && R <= 256) {
+        // targets (experts, then guest slots) in the order of the send buffer: by destination rank, then by index
+        const int K = params->K, NT = E + R * K;
+        std::vector<int32_t> tdest(NT + 1), torder(NT + 1), tpos(NT + 1), fill(R + 1, 0);
+        for (int t = 0; t < NT; ++t) tdest[t] = t < E ? h_e2r[t] : (t - E) / K;
+        tdest[NT] = R;
+        for (int t = 0; t <= NT; ++t) fill[tdest[t]]++;
+        int32_t run = 0;
+        for (int q = 0; q <= R; ++q) { const int32_t c = fill[q]; fill[q] = run; run += c; }
+        for (int t = 0; t <= NT; ++t) { tpos[t] = fill[tdest[t]]++; torder[tpos[t]] = t; }   // ascending t inside a rank
+        rc = upload(&h->d_tpos, tpos.data(), tpos.size());
+        if (rc == TAOT_OK) rc = upload(&h->d_torder, torder.data(), torder.size());
+        if (rc == TAOT_OK) rc = upload(&h->d_tdest, tdest.data(), tdest.size());
+    }
     if (rc == TAOT_OK && h->ntiers > 0) rc = upload(&h->d_tiermask, tiermask.data(), tiermask.size());
     for (int i = 0; i < 6 && rc == TAOT_OK; ++i)
         if (cudaEventCreate(&h->ev[i]) != cudaSuccess) rc = TAOT_ERR_CUDA;
@@ -240,6 +255,7 @@ int taot_destroy(taot_handle_t h)
     cudaDeviceSynchronize();
     cudaFree(h->d_e2r); cudaFree(h->d_C); cudaFree(h->d_B); cudaFree(h->d_rowlse0);
     cudaFree(h->d_rank_off); cudaFree(h->d_rank_list); cudaFree(h->d_tierval); cudaFree(h->d_tiermask);
+    cudaFree(h->d_tpos); cudaFree(h->d_torder); cudaFree(h->d_tdest);
     for (int i = 0; i < 6; ++i)
         if (h->ev[i]) cudaEventDestroy(h->ev[i]);
     delete h;
@@ -335,6 +351,22 @@ int taot_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load
     int a = taot_launch_match(h, d_n, d_expert_load, d_rank_load, d_plan, d_slot_expert, d_slot_tokens, d_X,
                               d_rounds, d_info, reinterpret_cast<int32_t*>(at(ws, h->off_nrem)),
                               reinterpret_cast<float*>(at(ws, h->off_t12)), static_cast<cudaStream_t>(stream));
+    if (a < 0) return a;
+    h->last_launches = a;
+    return TAOT_OK;
+}
+
+int taot_dispatch(taot_handle_t h, const int32_t* d_new_idx, int32_t* d_send_counts, int32_t* d_target_counts,
+                  int32_t* d_perm, int32_t* d_info, void* ws, void* stream)
+{
+    if (h && h->p.R > 256) return TAOT_ERR_UNSUPPORTED;
+    if (!h || !d_new_idx || !d_send_counts || !d_perm || !d_info || !ws) return TAOT_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(d_new_idx) & 3) || (reinterpret_cast<uintptr_t>(d_perm) & 3) ||
+        (reinterpret_cast<uintptr_t>(ws) & 255))
+        return TAOT_ERR_ALIGN;
+    if (d_new_idx == d_perm) return TAOT_ERR_PARAM;
+    int a = taot_launch_dispatch(h, d_new_idx, d_send_counts, d_target_counts, d_perm, d_info, ws,
+                                 static_cast<cudaStream_t>(stream));
     if (a < 0) return a;
     h->last_launches = a;
     return TAOT_OK;

@@ -25,17 +25,18 @@ __device__ __forceinline__ int4 ld_stream(const int4* p)
     return v;
 }
 
-__device__ __forceinline__ void count_one(int32_t* hist, int32_t e, int32_t E, int& bad)
+// nb == E: out-of-range values are only flagged; nb == E + 1: they are also counted, in bin E
+__device__ __forceinline__ void count_one(int32_t* hist, int32_t e, int32_t E, int32_t nb, int& bad)
 {
     if ((uint32_t)e < (uint32_t)E) atomicAdd(hist + e, 1);
-    else bad = 1;
+    else { bad = 1; if (nb > E) atomicAdd(hist + E, 1); }
 }
 
 __global__ void __launch_bounds__(kThreads)
 hist_chunk_kernel(const int32_t* __restrict__ topk, int32_t* __restrict__ cc, int32_t* __restrict__ info,
-                  int64_t layer_elems, int64_t seg, int32_t nc, int32_t R, int32_t E, int vec_ok)
+                  int64_t layer_elems, int64_t seg, int32_t nc, int32_t R, int32_t E, int32_t nb, int vec_ok)
 {
-    extern __shared__ int32_t sh_hist[];                 // [kWarps][E]
+    extern __shared__ int32_t sh_hist[];                 // [kWarps][nb]
     const int tid = threadIdx.x, warp = tid >> 5;
     const int64_t id = blockIdx.x;
     const int32_t c = (int32_t)(id % nc);
@@ -46,9 +47,9 @@ hist_chunk_kernel(const int32_t* __restrict__ topk, int32_t* __restrict__ cc, in
     const int32_t len = (int32_t)((seg - start) < (int64_t)TAOT_CHUNK ? (seg - start) : (int64_t)TAOT_CHUNK);
     const int32_t* src = topk + (int64_t)l * layer_elems + (int64_t)r * seg + start;
 
-    for (int i = tid; i < kWarps * E; i += kThreads) sh_hist[i] = 0;
+    for (int i = tid; i < kWarps * nb; i += kThreads) sh_hist[i] = 0;
     __syncthreads();
-    int32_t* hist = sh_hist + warp * E;
+    int32_t* hist = sh_hist + warp * nb;
     int bad = 0;
 
     if (vec_ok) {
@@ -62,25 +63,25 @@ hist_chunk_kernel(const int32_t* __restrict__ topk, int32_t* __restrict__ cc, in
             for (int u = 0; u < 8; ++u) x[u] = ld_stream(src4 + v + u * kThreads);
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                count_one(hist, x[u].x, E, bad); count_one(hist, x[u].y, E, bad);
-                count_one(hist, x[u].z, E, bad); count_one(hist, x[u].w, E, bad);
+                count_one(hist, x[u].x, E, nb, bad); count_one(hist, x[u].y, E, nb, bad);
+                count_one(hist, x[u].z, E, nb, bad); count_one(hist, x[u].w, E, nb, bad);
             }
         }
         for (; v < nvec; v += kThreads) {
             const int4 x = ld_stream(src4 + v);
-            count_one(hist, x.x, E, bad); count_one(hist, x.y, E, bad);
-            count_one(hist, x.z, E, bad); count_one(hist, x.w, E, bad);
+            count_one(hist, x.x, E, nb, bad); count_one(hist, x.y, E, nb, bad);
+            count_one(hist, x.z, E, nb, bad); count_one(hist, x.w, E, nb, bad);
         }
-        for (int32_t i = (nvec << 2) + tid; i < len; i += kThreads) count_one(hist, src[i], E, bad);
+        for (int32_t i = (nvec << 2) + tid; i < len; i += kThreads) count_one(hist, src[i], E, nb, bad);
     } else {
-        for (int32_t i = tid; i < len; i += kThreads) count_one(hist, src[i], E, bad);
+        for (int32_t i = tid; i < len; i += kThreads) count_one(hist, src[i], E, nb, bad);
     }
     const int any_bad = __syncthreads_or(bad);
-    int32_t* out = cc + id * E;
-    for (int e = tid; e < E; e += kThreads) {
+    int32_t* out = cc + id * nb;
+    for (int e = tid; e < nb; e += kThreads) {
         int32_t tot = 0;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) tot += sh_hist[w * E + e];
+        for (int w = 0; w < kWarps; ++w) tot += sh_hist[w * nb + e];
         out[e] = tot;
     }
     if (any_bad && tid == 0) atomicOr(info + l, TAOT_INFO_BAD_INDEX);
@@ -167,7 +168,25 @@ int taot_launch_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_cc,
     const int vec_ok = ((reinterpret_cast<uintptr_t>(d_topk) & 15) == 0) && (h->seg % 4 == 0);
     const size_t smem = sizeof(int32_t) * kWarps * p.E;
     hist_chunk_kernel<<<(unsigned)blocks, kThreads, smem, st>>>(d_topk, d_cc, d_info, layer_elems, h->seg,
-                                                                 h->nc, p.R, p.E, vec_ok);
+                                                                 h->nc, p.R, p.E, p.E, vec_ok);
+    TAOT_CUDA_OK(cudaGetLastError());
+    return 1;
+}
+
+// The same chunk histogram over `bins` values with one more bin for everything out of range (rows of bins + 1
+// counts): the counting pass of the dispatch metadata, where the table holds experts and guest slots.
+int taot_launch_chunk_counts(taot_handle_t h, const int32_t* d_idx, int32_t* d_counts, int32_t* d_info, int32_t bins,
+                             cudaStream_t st)
+{
+    const taot_params& p = h->p;
+    const int64_t blocks = (int64_t)p.L * p.R * h->nc;
+    const int vec_ok = ((reinterpret_cast<uintptr_t>(d_idx) & 15) == 0) && (h->seg % 4 == 0);
+    const size_t smem = sizeof(int32_t) * kWarps * (size_t)(bins + 1);
+    // only ever raise the limit: the load-collection launch above relies on the default 48 KB
+    if (smem > 48 * 1024)
+        TAOT_CUDA_OK(cudaFuncSetAttribute(hist_chunk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    hist_chunk_kernel<<<(unsigned)blocks, kThreads, smem, st>>>(d_idx, d_counts, d_info, p.T * p.k, h->seg, h->nc,
+                                                                 p.R, bins, bins + 1, vec_ok);
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
 }

@@ -26,6 +26,9 @@ struct taot_handle_s {
     int32_t* d_rank_off;     // [R+1] CSR of experts by home rank
     int32_t* d_rank_list;    // [E]
     uint32_t* d_tiermask;    // [ntiers][W][R hosts] bit r of word w set iff bonus(32w + r -> host) == tierval[t]; null if ntiers == 0
+    int32_t* d_tpos;         // [E+S+1] position of each target in (destination rank, target) order; last = undeliverable
+    int32_t* d_torder;       // [E+S+1] target at each position
+    int32_t* d_tdest;        // [E+S+1] destination rank of each target (R for the undeliverable bin)
     float* d_tierval;        // [ntiers] distinct values of the auction bonus matrix, descending
     int32_t ntiers;          // 0: too many distinct values, the auction scans densely
     // derived sizes
@@ -34,7 +37,7 @@ struct taot_handle_s {
     int32_t kcap;            // Sinkhorn kernel-matrix capacity in floats per problem (shared memory)
     int64_t kcap_global;     // same, global-memory scratch per problem (R > 256 only), else 0
     // workspace layout (byte offsets)
-    size_t off_cc, off_tabg, off_nbg, off_soff, off_work, off_splits, off_excess, off_spare, off_s, off_d, off_nrem, off_t12, off_kt;
+    size_t off_cc, off_tabg, off_nbg, off_soff, off_work, off_splits, off_excess, off_spare, off_s, off_d, off_nrem, off_t12, off_kt, off_dc;
     size_t ws_bytes;
     // host-call staging layout (byte offsets into d_ws of taot_plan_host)
     size_t hoff_topk, hoff_new, hoff_n, hoff_el, hoff_rl, hoff_ex, hoff_sp, hoff_plan, hoff_it, hoff_err,
@@ -67,6 +70,11 @@ int taot_launch_report(taot_handle_t h, const int32_t* d_expert_load, const int3
                        const int32_t* d_slot_expert, const int32_t* d_X, double lambda, taot_report_row* d_rows,
                        int32_t* d_spill, int32_t* d_load_after, int32_t* d_slot_moved, int32_t* d_slot_kind,
                        cudaStream_t st);
+
+int taot_launch_chunk_counts(taot_handle_t h, const int32_t* d_idx, int32_t* d_counts, int32_t* d_info, int32_t bins,
+                             cudaStream_t st);
+int taot_launch_dispatch(taot_handle_t h, const int32_t* d_new_idx, int32_t* d_send_counts, int32_t* d_target_counts,
+                         int32_t* d_perm, int32_t* d_info, void* ws, cudaStream_t st);
 
 #define TAOT_CUDA_OK(expr)                              \
     do {                                                \
