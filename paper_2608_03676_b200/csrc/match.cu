@@ -50,6 +50,7 @@ struct MatchArgs {
     int32_t ablation;            // TAOT_ABLATE_* bits: a term switched off is an exact zero in the score
     int32_t nrem_in_smem;
     int32_t tm_in_smem;
+    int32_t big_floats;          // 4-byte words of the shared block that holds the Phase-2 score rows, then nrem
 };
 
 __device__ __forceinline__ uint32_t ordered_bits(float f)
@@ -143,7 +144,7 @@ match_kernel(MatchArgs a)
     const int32_t* rl = a.rank_load + l * R;
     const float* plan = a.plan + l * (int64_t)R * R;
     int32_t* nrem = a.nrem_in_smem ? nrem_s : a.nrem_g + l * (int64_t)a.dmax * R;
-    float* t12 = a.t12 + l * (int64_t)E * 2 * R;
+    float* t12 = a.t12 + l * (int64_t)E * 2 * R;      // global scratch; replaced by shared memory below if the rows fit
 
     // ---- integer mean, excess, spare (Appendix A.1)
     if (tid == 0) { s_tot = 0; s_cnt = 0; }
@@ -189,8 +190,11 @@ match_kernel(MatchArgs a)
 
     const float alpha = __fdiv_rn((float)(mean * (long long)R), (float)E);
     const float beta = __fmul_rn(0.1f, alpha);
+    // the rows are only read in Phase 2 and the remaining counts only exist in Phase 3: they share one block
+    if ((int64_t)nhot0 * 2 * R <= (int64_t)a.big_floats) t12 = reinterpret_cast<float*>(nrem_s);
 
     // ---- round-invariant score terms of the spilling experts: t1 = alpha*B, t2 = beta*T/max(excess, eps0)
+#pragma unroll 4
     for (int64_t idx = tid; idx < (int64_t)nhot0 * R; idx += NT) {
         const int q = (int)(idx / R), r = (int)(idx - (int64_t)q * R);
         const int hr = hot_home[q];
@@ -276,14 +280,15 @@ match_kernel(MatchArgs a)
     for (int i = tid; i < (S + 1) * W; i += NT) lvl[i] = 0u;
     __syncthreads();
     const int D = s_cnt;
-    for (int e = 0; e < E; ++e) {
-        const int col = dcol[e];
-        if (col < 0) continue;
-        for (int r = tid; r < R; r += NT) {
-            const int32_t v = n[(int64_t)r * E + e];
-            nrem[col * R + r] = v;
-            if (v > 0) atomicOr(avail + (r >> 5) * a.dmax + col, 1u << (r & 31));
-        }
+    for (int e = tid; e < E; e += NT)
+        if (dcol[e] >= 0) hot0[dcol[e]] = e;                   // column -> expert (the Phase-2 list is no longer needed)
+    __syncthreads();
+#pragma unroll 4
+    for (int q = tid; q < D * R; q += NT) {
+        const int col = q / R, r = q - col * R;
+        const int32_t v = n[(int64_t)r * E + hot0[col]];
+        nrem[q] = v;
+        if (v > 0) atomicOr(avail + (r >> 5) * a.dmax + col, 1u << (r & 31));
     }
     for (int r = tid; r < R; r += NT) atomicOr(lvl + (r >> 5) * (S + 1), 1u << (r & 31));      // every rank starts with 0 wins
     int32_t* Xl = a.X + l * (int64_t)R * S;
@@ -338,10 +343,17 @@ match_kernel(MatchArgs a)
             }
         }
         int prev_r = -1;                         // rank whose arbiter entry this slot won last round
+        {
+            // the arbiter words of the tiered auction: two ping-pong sets of [R] score bits (0) and [R] slots (all ones)
+            uint32_t* w32 = reinterpret_cast<uint32_t*>(arb_r);
+            for (int q = tid; q < 4 * R; q += NT) w32[q] = ((q / R) & 1) ? 0xFFFFFFFFu : 0u;
+            __syncthreads();
+        }
         for (;;) {
             if (a.auction_max_rounds > 0 && rounds3 >= a.auction_max_rounds) break;
             if (rounds3 >= cap) break;
-            u64* arb = arb_r + (rounds3 & 1) * R;
+            uint32_t* ahi = reinterpret_cast<uint32_t*>(arb_r) + (rounds3 & 1) * 2 * R;   // [R] best score bits per rank
+            uint32_t* alo = ahi + R;                                                       // [R] lowest slot offering it
             // Step 1: bid for the source rank with the best bonus minus price
             u64 key = 0;
             if (live) {
@@ -399,13 +411,22 @@ match_kernel(MatchArgs a)
                     key = k64 > key ? k64 : key;
                 }
             }
-            // Step 2: the rank keeps its best bidder (ties: lowest slot)
+            // Step 2: the rank keeps its best bidder (ties: lowest slot), in two native 32-bit shared-memory atomics:
+            // the highest score first, then the lowest slot among the bidders that offered it
             const int rsel = (int)(0xFFFFFFFFu - (uint32_t)key);
-            arbitrate(arb, rsel, key == 0 ? 0ull : ((key & 0xFFFFFFFF00000000ull) | (u64)(0xFFFFFFFFu - (uint32_t)s)));
+            const uint32_t hi = (uint32_t)(key >> 32);
+            if (key != 0) atomicMax(ahi + rsel, hi);
             if (!__syncthreads_or(key != 0)) break;
-            if (prev_r >= 0) { arb_r[((rounds3 & 1) ^ 1) * R + prev_r] = 0; prev_r = -1; }
+            if (prev_r >= 0) {                      // last round's winner clears the entries that round used
+                uint32_t* ohi = reinterpret_cast<uint32_t*>(arb_r) + ((rounds3 & 1) ^ 1) * 2 * R;
+                ohi[prev_r] = 0u; ohi[R + prev_r] = 0xFFFFFFFFu;
+                prev_r = -1;
+            }
+            const bool top = key != 0 && ahi[rsel] == hi;
+            if (top) atomicMin(alo + rsel, (uint32_t)s);
+            __syncthreads();
             // Steps 3-4: the winning slot of each rank collects x = min(n, A); holdings, plan and price follow
-            if (key != 0 && (uint32_t)arb[rsel] == 0xFFFFFFFFu - (uint32_t)s) {
+            if (top && alo[rsel] == (uint32_t)s) {
                 int32_t* cell = nrem + col * R + rsel;
                 const int32_t have = *cell;
                 const int32_t x = have < A ? have : A;
@@ -526,7 +547,14 @@ int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expe
     a.tm_in_smem = (a.ntiers > 0 && smem + tm_bytes <= 96 * 1024) ? 1 : 0;
     if (a.tm_in_smem) smem += tm_bytes;
     a.nrem_in_smem = (smem + nrem_bytes <= 200 * 1024) ? 1 : 0;
-    if (a.nrem_in_smem) smem += nrem_bytes;
+    // one block for the Phase-2 score rows (2 * R floats per spilling expert) and then the remaining counts: as large
+    // as the counts need if those live in shared memory, and at least 64 KB when there is room
+    size_t big = a.nrem_in_smem ? nrem_bytes : 0;
+    const size_t want = sizeof(float) * 2 * (size_t)p.R * (size_t)p.E;
+    const size_t room = 200 * 1024 > smem ? 200 * 1024 - smem : 0;
+    if (big < want) big = want < room ? want : (room > big ? room : big);
+    a.big_floats = (int32_t)(big / 4);
+    smem += big;
     if (smem > 227 * 1024) return TAOT_ERR_UNSUPPORTED;
     TAOT_CUDA_OK(cudaFuncSetAttribute(match_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int need = p.R * p.K > p.R ? p.R * p.K : p.R;
