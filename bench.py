@@ -129,6 +129,9 @@ def measured_peaks():
     return dict(hbm_gbs=6650.0, sm_max_mhz=1965.0, source="fallback")
 
 
+METRIC = "placement plans/s (whole planner path: histogram, excess/spare, Sinkhorn, matching+auction, token remap)"
+
+
 def build_planner(cfg):
     import paper_2608_03676_b200 as P
     e2r = W.expert_to_rank(cfg.E, cfg.R, cfg.e2r_mode)
@@ -294,7 +297,7 @@ def run_reference(args):
         if i >= args.warmup:
             layers += n; secs += t
     value = layers / secs
-    line = dict(metric="placement plans/s (whole planner path)", value=value, unit="plans/s", n_gpus=args.gpus,
+    line = dict(metric=METRIC, value=value, unit="plans/s", n_gpus=args.gpus,
                 steps=args.steps, warmup=args.warmup, ms_per_step=1e3 * secs / max(1, args.steps),
                 higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
                 impl="reference", config=dict(workload=args.workload, L=cfg.L, R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k,
@@ -400,7 +403,7 @@ def run_ours(args):
     rounds = out["rounds"].cpu().numpy()
     info = out["info"].cpu().numpy()
     line = dict(
-        metric="placement plans/s (whole planner path: histogram, excess/spare, Sinkhorn, matching+auction, token remap)",
+        metric=METRIC,
         value=value, unit="plans/s", n_gpus=world, steps=args.steps, warmup=max(3, args.warmup),
         ms_per_step=float(np.mean(ms)), higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
         data="synthetic",
