@@ -2,6 +2,7 @@
 // stage chaining of taot_plan / taot_plan_host.  No arithmetic of the method lives here except
 // the two topology tables derived once per handle (the preference matrix B when the caller
 // gives none, and the first-iteration row normaliser of the Sinkhorn solve).
+#include <algorithm>
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
@@ -195,6 +196,30 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
         }
     }
     h->ntiers = (int32_t)tierval.size();
+    // Every score a bid of the tiered auction can take is  tierval[t] - price_step * w  for a tier t and a win count
+    // w in [0, S].  All (t, w) pairs are listed once, best score first (evaluated with the same two fp32 operations
+    // the kernel uses), so that a slot walks the list instead of comparing tiers; pairs with the same score form a
+    // group (bit 31 = "the next entry has the same score").  Entry: w << 8 | t.
+    std::vector<uint32_t> bidlist;
+    if (h->ntiers > 0 && params->price_step > 0.0f && R <= 256) {
+        const int S = R * params->K;
+        struct Pair { float sc; int t, w; };
+        std::vector<Pair> pairs;
+        pairs.reserve((size_t)h->ntiers * (S + 1));
+        for (int t = 0; t < h->ntiers; ++t)
+            for (int w = 0; w <= S; ++w) {
+                volatile float price = params->price_step * (float)w;     // one rounding per operation
+                volatile float sc = tierval[t] - price;
+                pairs.push_back(Pair{sc, t, w});
+            }
+        std::stable_sort(pairs.begin(), pairs.end(), [](const Pair& x, const Pair& y) { return x.sc > y.sc; });
+        bidlist.resize(pairs.size());
+        for (size_t i = 0; i < pairs.size(); ++i) {
+            const bool tie_next = i + 1 < pairs.size() && pairs[i + 1].sc == pairs[i].sc;
+            bidlist[i] = ((uint32_t)pairs[i].w << 8) | (uint32_t)pairs[i].t | (tie_next ? 0x80000000u : 0u);
+        }
+    }
+    h->nbid = (int32_t)bidlist.size();
     // first Sinkhorn row update with v = 1 on every rank: log-sum-exp of -C_ij/eps over all j
     std::vector<double> lse0(R);
     for (int i = 0; i < R; ++i) {
@@ -238,6 +263,7 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
         if (rc == TAOT_OK) rc = upload(&h->d_tdest, tdest.data(), tdest.size());
     }
     if (rc == TAOT_OK && h->ntiers > 0) rc = upload(&h->d_tiermask, tiermask.data(), tiermask.size());
+    if (rc == TAOT_OK && h->nbid > 0) rc = upload(&h->d_bidlist, bidlist.data(), bidlist.size());
     for (int i = 0; i < 6 && rc == TAOT_OK; ++i)
         if (cudaEventCreate(&h->ev[i]) != cudaSuccess) rc = TAOT_ERR_CUDA;
     if (rc == TAOT_OK && cudaDeviceSynchronize() != cudaSuccess) rc = TAOT_ERR_CUDA;
@@ -255,7 +281,7 @@ int taot_destroy(taot_handle_t h)
     cudaDeviceSynchronize();
     cudaFree(h->d_e2r); cudaFree(h->d_C); cudaFree(h->d_B); cudaFree(h->d_rowlse0);
     cudaFree(h->d_rank_off); cudaFree(h->d_rank_list); cudaFree(h->d_tierval); cudaFree(h->d_tiermask);
-    cudaFree(h->d_tpos); cudaFree(h->d_torder); cudaFree(h->d_tdest);
+    cudaFree(h->d_tpos); cudaFree(h->d_torder); cudaFree(h->d_tdest); cudaFree(h->d_bidlist);
     for (int i = 0; i < 6; ++i)
         if (h->ev[i]) cudaEventDestroy(h->ev[i]);
     delete h;

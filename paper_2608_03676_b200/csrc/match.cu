@@ -14,12 +14,14 @@
 // scanning those experts with coalesced reads.
 //
 // Phase 3: the bonus matrix of a real topology has a handful of distinct values (tiers).  Within
-// a tier a slot's score  B3 - step*wins[r]  depends on r only through wins[r], so the best source
-// rank of a tier is "lowest wins, then lowest index" among the ranks that still hold tokens.  Ranks
-// are kept as bit sets (per tier and host, per win count, per expert availability), and a bid is a
-// few word-wide ANDs instead of a scan over all R ranks; the exact fp32 score is still what is
-// compared, including win counts whose scores round to the same float.  A bonus matrix with more
-// than kMaxTiers distinct values (or a negative price step) takes the dense scan instead.
+// a tier a slot's score  B3 - step*wins[r]  depends on r only through wins[r], so every score a bid
+// can take is one of (tier, win count) pairs, and those are listed once per handle in order of
+// decreasing fp32 score (equal scores grouped).  Ranks are kept as bit sets (per tier and host, per
+// win count, per expert availability); a slot walks the list with a cursor that never moves back
+// and a probe is a few word-wide ANDs instead of a scan over all R ranks.  The exact fp32 score is
+// what orders the list, so win counts or tiers whose scores round to the same float compete on the
+// rank index alone, as in a dense scan.  A bonus matrix with more than kMaxTiers distinct values (or
+// a price step that is not positive) takes the dense scan instead.
 #include "taot_internal.cuh"
 
 namespace {
@@ -37,6 +39,7 @@ struct MatchArgs {
     const int32_t* rank_list;    // [E]
     const uint32_t* tiermask;    // [ntiers][W][R hosts] bit r of word w: B3[32w + r][host] == tierval[t]
     const float* tierval;        // [ntiers] descending
+    const uint32_t* bidlist;     // [nbid] (tier, win count) pairs by decreasing score: w << 8 | t, bit 31: next has the same score
     int32_t* slot_expert;        // [L,R,K]
     int32_t* slot_tokens;        // [L,R,K]
     int32_t* X;                  // [L,R,S]
@@ -44,7 +47,7 @@ struct MatchArgs {
     int32_t* info;               // [L]
     int32_t* nrem_g;             // [L, dmax, R] global fallback for the remaining counts
     float* t12;                  // [L, E, 2, R] scratch: alpha*B and beta*T_norm rows of the spilling experts
-    int32_t R, E, K, dmax, ntiers, W;
+    int32_t R, E, K, dmax, ntiers, W, nbid;
     float eps0, price_step;
     int32_t auction_max_rounds;
     int32_t ablation;            // TAOT_ABLATE_* bits: a term switched off is an exact zero in the score
@@ -135,7 +138,11 @@ match_kernel(MatchArgs a)
     uint32_t* avail = reinterpret_cast<uint32_t*>(slot_a + S); // [W][dmax]  ranks still holding tokens of the expert (word-major: no bank conflicts across slots)
     uint32_t* lvl = avail + a.dmax * W;                        // [W][S+1]   ranks by win count (word-major)
     uint32_t* tm_s = lvl + (S + 1) * W;                                // [ntiers][W][S] tier masks by slot, if they fit
-    int32_t* nrem_s = reinterpret_cast<int32_t*>(tm_s + (a.tm_in_smem ? a.ntiers * W * S : 0));   // [dmax*R] if it fits
+    uint32_t* bid_s = tm_s + (a.tm_in_smem ? a.ntiers * W * S : 0);    // [nbid] (tier, win count) pairs, best score first
+    float* tval_s = reinterpret_cast<float*>(bid_s + a.nbid);          // [ntiers]
+    int32_t* tw_word = reinterpret_cast<int32_t*>(tval_s + a.ntiers);  // [ntiers][S] word holding the whole tier for the slot's host, or -1
+    uint32_t* tw_mask = reinterpret_cast<uint32_t*>(tw_word + (a.nbid ? a.ntiers * S : 0));   // [ntiers][S] that word's mask
+    int32_t* nrem_s = reinterpret_cast<int32_t*>(tw_mask + (a.nbid ? a.ntiers * S : 0));      // [dmax*R] if it fits
     __shared__ long long s_tot;
     __shared__ int s_cnt, s_any;
 
@@ -297,21 +304,20 @@ match_kernel(MatchArgs a)
 
     int rounds3 = 0;
     const long long cap = (long long)R * S + S;
-    const bool tiered = a.ntiers > 0 && S <= NT;
+    const bool tiered = a.nbid > 0 && S <= NT;
     if (tiered && D > 0) {
-        // ---- bit-set auction: thread s is slot s for the whole auction and keeps the slot's state in registers
+        // ---- bit-set auction: thread s is slot s for the whole auction and keeps the slot's state in registers.
+        // A bid walks the list of all (tier, win count) pairs in order of decreasing score: the first pair that still
+        // has a candidate rank (in the tier for this slot's host, holding tokens of the slot's expert, with that win
+        // count) is the bid; pairs of equal score are scanned together and the lowest rank wins.  Win counts only grow
+        // and holdings only shrink, so no pair before the cursor can ever regain a candidate: the cursor never moves
+        // back and a round costs one or two probes per slot.
         const int s = tid;
         bool live = s < S && slot_e[s] >= 0 && slot_a[s] > 0;
         const int e = live ? slot_e[s] : 0;
         const int col = live ? dcol[e] : 0;
         const int host = s < S ? s / K : 0;
         int32_t A = live ? slot_a[s] : 0;
-        int32_t wst[TAOT_MAX_TIERS];             // per tier: lowest win count seen among its candidates (never decreases)
-#pragma unroll
-        for (int t = 0; t < TAOT_MAX_TIERS; ++t) wst[t] = 0;
-        float tval[TAOT_MAX_TIERS];
-#pragma unroll
-        for (int t = 0; t < TAOT_MAX_TIERS; ++t) tval[t] = t < a.ntiers ? a.tierval[t] : 0.0f;
         const uint32_t* av = avail + col;                          // word w at av[w * dmax]
         // this slot's tier masks: tier t, word w at tm[(t * W + w) * tms]; a shared-memory copy when it fits
         const uint32_t* tm = a.tiermask + host;
@@ -321,108 +327,78 @@ match_kernel(MatchArgs a)
                 const int ss = q % S, tw = q / S;
                 tm_s[q] = a.tiermask[(int64_t)tw * R + ss / K];
             }
-            __syncthreads();
             tm = tm_s + (s < S ? s : 0);
             tms = S;
         }
+        for (int q = tid; q < a.nbid; q += NT) bid_s[q] = a.bidlist[q];
+        for (int t = tid; t < a.ntiers; t += NT) tval_s[t] = a.tierval[t];
+        {
+            // the arbiter words: two ping-pong sets of [R] score bits (0) and [R] slots (all ones)
+            uint32_t* w32 = reinterpret_cast<uint32_t*>(arb_r);
+            for (int q = tid; q < 4 * R; q += NT) w32[q] = ((q / R) & 1) ? 0xFFFFFFFFu : 0u;
+        }
+        __syncthreads();
         const int LS = S + 1;                                      // lvl: word w of level wl at lvl[w * LS + wl]
-        // a tier whose ranks (for this slot's host) all sit in one 32-bit word is handled with that word alone
-        int twrd[TAOT_MAX_TIERS];
-        uint32_t tmw[TAOT_MAX_TIERS];
-#pragma unroll
-        for (int t = 0; t < TAOT_MAX_TIERS; ++t) {
-            twrd[t] = -1; tmw[t] = 0u;
-            if (t < a.ntiers) {
+        // a tier whose ranks (for this slot's host) all sit in one 32-bit word is probed with that word alone
+        if (s < S) {
+            for (int t = 0; t < a.ntiers; ++t) {
                 int nz = 0, wd = 0;
                 uint32_t val = 0u;
                 for (int w = 0; w < W; ++w) {
                     const uint32_t mk = tm[(t * W + w) * tms];
                     if (mk) { ++nz; wd = w; val = mk; }
                 }
-                if (nz <= 1) { twrd[t] = wd; tmw[t] = val; }
+                tw_word[t * S + s] = nz <= 1 ? wd : -1;
+                tw_mask[t * S + s] = nz <= 1 ? val : 0u;
             }
         }
+        int cur = 0;                             // first list entry (start of a group of equal scores) that may still hit
         int prev_r = -1;                         // rank whose arbiter entry this slot won last round
-        {
-            // the arbiter words of the tiered auction: two ping-pong sets of [R] score bits (0) and [R] slots (all ones)
-            uint32_t* w32 = reinterpret_cast<uint32_t*>(arb_r);
-            for (int q = tid; q < 4 * R; q += NT) w32[q] = ((q / R) & 1) ? 0xFFFFFFFFu : 0u;
-            __syncthreads();
-        }
         for (;;) {
             if (a.auction_max_rounds > 0 && rounds3 >= a.auction_max_rounds) break;
             if (rounds3 >= cap) break;
             uint32_t* ahi = reinterpret_cast<uint32_t*>(arb_r) + (rounds3 & 1) * 2 * R;   // [R] best score bits per rank
             uint32_t* alo = ahi + R;                                                       // [R] lowest slot offering it
             // Step 1: bid for the source rank with the best bonus minus price
-            u64 key = 0;
+            int r_best = -1, t_best = 0, w_best = 0;
             if (live) {
+                while (cur < a.nbid) {
+                    int g = cur;
+                    uint32_t pr;
+                    do {
+                        pr = bid_s[g++];
+                        const int t = (int)(pr & 0xFFu), wl = (int)((pr >> 8) & 0xFFFFu);
+                        const int wd = tw_word[t * S + s];
+                        int r;
+                        if (wd >= 0) {
+                            const uint32_t hit = tw_mask[t * S + s] & av[wd * a.dmax] & lvl[wd * LS + wl];
+                            r = hit ? (wd << 5) + __ffs(hit) - 1 : -1;
+                        } else {
+                            uint32_t cand[kMaxW];
 #pragma unroll
-                for (int t = 0; t < TAOT_MAX_TIERS; ++t) {
-                    if (t >= a.ntiers) break;
-                    const float vt = tval[t];
-                    int wl = wst[t];
-                    // best score this tier can still offer: skip it if a better tier already beats that
-                    const float ub = __fsub_rn(vt, __fmul_rn(a.price_step, (float)wl));
-                    if (key != 0 && (u64)ordered_bits(ub) < (key >> 32)) continue;
-                    int r_best = -1;
-                    float sc;
-                    if (twrd[t] >= 0) {
-                        // the tier's ranks (for this host) sit in one 32-bit word: node or rail-group tiers
-                        const int wd = twrd[t];
-                        const uint32_t c1 = tmw[t] & av[wd * a.dmax];
-                        if (!c1) continue;
-                        const uint32_t* lv = lvl + wd * LS;
-                        for (; wl <= S; ++wl) {
-                            const uint32_t hit = c1 & lv[wl];
-                            if (hit) { r_best = (wd << 5) + __ffs(hit) - 1; break; }
+                            for (int w = 0; w < kMaxW; ++w) cand[w] = (w < W) ? (tm[(t * W + w) * tms] & av[w * a.dmax]) : 0u;
+                            r = first_hit(cand, lvl + wl, LS, W);
                         }
-                        if (r_best < 0) continue;
-                        sc = __fsub_rn(vt, __fmul_rn(a.price_step, (float)wl));
-                        // higher win counts whose score rounds to the same float compete on rank index alone
-                        for (int w2 = wl + 1; w2 <= S; ++w2) {
-                            if (__fsub_rn(vt, __fmul_rn(a.price_step, (float)w2)) != sc) break;
-                            const uint32_t hit = c1 & lv[w2];
-                            if (hit) { const int r2 = (wd << 5) + __ffs(hit) - 1; r_best = r2 < r_best ? r2 : r_best; }
-                        }
-                    } else {
-                        uint32_t cand[kMaxW];
-                        uint32_t any = 0;
-#pragma unroll
-                        for (int w = 0; w < kMaxW; ++w) {
-                            cand[w] = (w < W) ? (tm[(t * W + w) * tms] & av[w * a.dmax]) : 0u;
-                            any |= cand[w];
-                        }
-                        if (!any) continue;
-                        for (; wl <= S; ++wl) {
-                            r_best = first_hit(cand, lvl + wl, LS, W);
-                            if (r_best >= 0) break;
-                        }
-                        if (r_best < 0) continue;
-                        sc = __fsub_rn(vt, __fmul_rn(a.price_step, (float)wl));
-                        for (int w2 = wl + 1; w2 <= S; ++w2) {
-                            if (__fsub_rn(vt, __fmul_rn(a.price_step, (float)w2)) != sc) break;
-                            const int r2 = first_hit(cand, lvl + w2, LS, W);
-                            if (r2 >= 0 && r2 < r_best) r_best = r2;
-                        }
-                    }
-                    wst[t] = wl;
-                    const u64 k64 = ((u64)ordered_bits(sc) << 32) | (u64)(0xFFFFFFFFu - (uint32_t)r_best);
-                    key = k64 > key ? k64 : key;
+                        if (r >= 0 && (r_best < 0 || r < r_best)) { r_best = r; t_best = t; w_best = wl; }
+                    } while (pr & 0x80000000u);
+                    if (r_best >= 0) break;
+                    cur = g;                     // the whole group is empty for good
                 }
             }
+            const float sc = __fsub_rn(tval_s[t_best], __fmul_rn(a.price_step, (float)w_best));
+            const bool bids = r_best >= 0;
+            const int rsel = r_best;
+            const uint32_t hi = ordered_bits(sc);
             // Step 2: the rank keeps its best bidder (ties: lowest slot), in two native 32-bit shared-memory atomics:
             // the highest score first, then the lowest slot among the bidders that offered it
-            const int rsel = (int)(0xFFFFFFFFu - (uint32_t)key);
-            const uint32_t hi = (uint32_t)(key >> 32);
-            if (key != 0) atomicMax(ahi + rsel, hi);
-            if (!__syncthreads_or(key != 0)) break;
+            if (bids) atomicMax(ahi + rsel, hi);
+            if (!__syncthreads_or(bids)) break;
             if (prev_r >= 0) {                      // last round's winner clears the entries that round used
                 uint32_t* ohi = reinterpret_cast<uint32_t*>(arb_r) + ((rounds3 & 1) ^ 1) * 2 * R;
                 ohi[prev_r] = 0u; ohi[R + prev_r] = 0xFFFFFFFFu;
                 prev_r = -1;
             }
-            const bool top = key != 0 && ahi[rsel] == hi;
+            const bool top = bids && ahi[rsel] == hi;
             if (top) atomicMin(alo + rsel, (uint32_t)s);
             __syncthreads();
             // Steps 3-4: the winning slot of each rank collects x = min(n, A); holdings, plan and price follow
@@ -532,16 +508,18 @@ int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expe
     MatchArgs a;
     a.n = d_n; a.expert_load = d_expert_load; a.rank_load = d_rank_load; a.plan = d_plan;
     a.e2r = h->d_e2r; a.B = h->d_B; a.rank_off = h->d_rank_off; a.rank_list = h->d_rank_list;
-    a.tiermask = h->d_tiermask; a.tierval = h->d_tierval;
+    a.tiermask = h->d_tiermask; a.tierval = h->d_tierval; a.bidlist = h->d_bidlist;
     a.slot_expert = d_slot_expert; a.slot_tokens = d_slot_tokens; a.X = d_X; a.rounds = d_rounds;
     a.info = d_info; a.nrem_g = d_nrem; a.t12 = d_t12;
     a.R = p.R; a.E = p.E; a.K = p.K;
     a.dmax = p.E < p.R * p.K ? p.E : p.R * p.K;
     a.W = (p.R + 31) / 32;
-    a.ntiers = (h->ntiers > 0 && p.price_step >= 0.0f && a.W <= kMaxW) ? h->ntiers : 0;
+    a.nbid = (h->ntiers > 0 && h->nbid > 0 && a.W <= kMaxW && p.R * p.K <= 1024) ? h->nbid : 0;
+    a.ntiers = a.nbid > 0 ? h->ntiers : 0;
     a.eps0 = p.eps0; a.price_step = p.price_step; a.auction_max_rounds = p.auction_max_rounds;
     a.ablation = p.ablation;
     size_t smem = match_smem_fixed(p.R, p.E, p.K, a.dmax, a.W, a.ntiers);
+    if (a.nbid > 0) smem += sizeof(uint32_t) * ((size_t)a.nbid + a.ntiers + 2 * (size_t)a.ntiers * p.R * p.K);
     const size_t nrem_bytes = sizeof(int32_t) * (size_t)a.dmax * p.R;
     const size_t tm_bytes = sizeof(uint32_t) * (size_t)a.ntiers * a.W * p.R * p.K;
     a.tm_in_smem = (a.ntiers > 0 && smem + tm_bytes <= 96 * 1024) ? 1 : 0;

@@ -31,6 +31,8 @@ struct taot_handle_s {
     int32_t* d_tdest;        // [E+S+1] destination rank of each target (R for the undeliverable bin)
     float* d_tierval;        // [ntiers] distinct values of the auction bonus matrix, descending
     int32_t ntiers;          // 0: too many distinct values, the auction scans densely
+    uint32_t* d_bidlist;     // [nbid] every (tier, win count) pair, best score first: w << 8 | t, bit 31 = next has the same score
+    int32_t nbid;            // 0: no list (no tiers, or price step <= 0): the auction scans densely
     // derived sizes
     int64_t seg;             // elements per (layer, rank) segment
     int32_t nc;              // chunks per segment
