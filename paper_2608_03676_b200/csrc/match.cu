@@ -139,8 +139,7 @@ match_kernel(MatchArgs a)
     uint32_t* lvl = avail + a.dmax * W;                        // [W][S+1]   ranks by win count (word-major)
     uint32_t* tm_s = lvl + (S + 1) * W;                                // [ntiers][W][S] tier masks by slot, if they fit
     uint32_t* bid_s = tm_s + (a.tm_in_smem ? a.ntiers * W * S : 0);    // [nbid] (tier, win count) pairs, best score first
-    float* tval_s = reinterpret_cast<float*>(bid_s + a.nbid);          // [ntiers]
-    int32_t* tw_word = reinterpret_cast<int32_t*>(tval_s + a.ntiers);  // [ntiers][S] word holding the whole tier for the slot's host, or -1
+    int32_t* tw_word = reinterpret_cast<int32_t*>(bid_s + a.nbid);     // [ntiers][S] word holding the whole tier for the slot's host, or -1
     uint32_t* tw_mask = reinterpret_cast<uint32_t*>(tw_word + (a.nbid ? a.ntiers * S : 0));   // [ntiers][S] that word's mask
     int32_t* nrem_s = reinterpret_cast<int32_t*>(tw_mask + (a.nbid ? a.ntiers * S : 0));      // [dmax*R] if it fits
     __shared__ long long s_tot;
@@ -331,12 +330,7 @@ match_kernel(MatchArgs a)
             tms = S;
         }
         for (int q = tid; q < a.nbid; q += NT) bid_s[q] = a.bidlist[q];
-        for (int t = tid; t < a.ntiers; t += NT) tval_s[t] = a.tierval[t];
-        {
-            // the arbiter words: two ping-pong sets of [R] score bits (0) and [R] slots (all ones)
-            uint32_t* w32 = reinterpret_cast<uint32_t*>(arb_r);
-            for (int q = tid; q < 4 * R; q += NT) w32[q] = ((q / R) & 1) ? 0xFFFFFFFFu : 0u;
-        }
+        for (int q = tid; q < 2 * R; q += NT) reinterpret_cast<uint32_t*>(arb_r)[q] = 0u;     // the two arbiter sets
         __syncthreads();
         const int LS = S + 1;                                      // lvl: word w of level wl at lvl[w * LS + wl]
         // a tier whose ranks (for this slot's host) all sit in one 32-bit word is probed with that word alone
@@ -357,10 +351,10 @@ match_kernel(MatchArgs a)
         for (;;) {
             if (a.auction_max_rounds > 0 && rounds3 >= a.auction_max_rounds) break;
             if (rounds3 >= cap) break;
-            uint32_t* ahi = reinterpret_cast<uint32_t*>(arb_r) + (rounds3 & 1) * 2 * R;   // [R] best score bits per rank
-            uint32_t* alo = ahi + R;                                                       // [R] lowest slot offering it
+            uint32_t* arb = reinterpret_cast<uint32_t*>(arb_r) + (rounds3 & 1) * R;       // [R] best bid per rank, ping-pong
+            uint32_t* arb_o = reinterpret_cast<uint32_t*>(arb_r) + ((rounds3 & 1) ^ 1) * R;
             // Step 1: bid for the source rank with the best bonus minus price
-            int r_best = -1, t_best = 0, w_best = 0;
+            int r_best = -1;
             if (live) {
                 while (cur < a.nbid) {
                     int g = cur;
@@ -379,30 +373,23 @@ match_kernel(MatchArgs a)
                             for (int w = 0; w < kMaxW; ++w) cand[w] = (w < W) ? (tm[(t * W + w) * tms] & av[w * a.dmax]) : 0u;
                             r = first_hit(cand, lvl + wl, LS, W);
                         }
-                        if (r >= 0 && (r_best < 0 || r < r_best)) { r_best = r; t_best = t; w_best = wl; }
+                        if (r >= 0 && (r_best < 0 || r < r_best)) r_best = r;
                     } while (pr & 0x80000000u);
                     if (r_best >= 0) break;
                     cur = g;                     // the whole group is empty for good
                 }
             }
-            const float sc = __fsub_rn(tval_s[t_best], __fmul_rn(a.price_step, (float)w_best));
+            // Step 2: the rank keeps its best bidder (ties: lowest slot).  The position of a score in the list orders
+            // scores exactly as their fp32 values do, so (list position, slot) packs into one 32-bit key and a single
+            // native shared-memory atomicMax arbitrates: smaller position = higher score, then the lower slot.
             const bool bids = r_best >= 0;
             const int rsel = r_best;
-            const uint32_t hi = ordered_bits(sc);
-            // Step 2: the rank keeps its best bidder (ties: lowest slot), in two native 32-bit shared-memory atomics:
-            // the highest score first, then the lowest slot among the bidders that offered it
-            if (bids) atomicMax(ahi + rsel, hi);
+            const uint32_t key = ((uint32_t)(a.nbid - cur) << 16) | (uint32_t)(0xFFFF - s);
+            if (bids) atomicMax(arb + rsel, key);
             if (!__syncthreads_or(bids)) break;
-            if (prev_r >= 0) {                      // last round's winner clears the entries that round used
-                uint32_t* ohi = reinterpret_cast<uint32_t*>(arb_r) + ((rounds3 & 1) ^ 1) * 2 * R;
-                ohi[prev_r] = 0u; ohi[R + prev_r] = 0xFFFFFFFFu;
-                prev_r = -1;
-            }
-            const bool top = bids && ahi[rsel] == hi;
-            if (top) atomicMin(alo + rsel, (uint32_t)s);
-            __syncthreads();
+            if (prev_r >= 0) { arb_o[prev_r] = 0u; prev_r = -1; }     // last round's winner clears the entry it used
             // Steps 3-4: the winning slot of each rank collects x = min(n, A); holdings, plan and price follow
-            if (top && alo[rsel] == (uint32_t)s) {
+            if (bids && arb[rsel] == key) {
                 int32_t* cell = nrem + col * R + rsel;
                 const int32_t have = *cell;
                 const int32_t x = have < A ? have : A;
@@ -519,7 +506,7 @@ int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expe
     a.eps0 = p.eps0; a.price_step = p.price_step; a.auction_max_rounds = p.auction_max_rounds;
     a.ablation = p.ablation;
     size_t smem = match_smem_fixed(p.R, p.E, p.K, a.dmax, a.W, a.ntiers);
-    if (a.nbid > 0) smem += sizeof(uint32_t) * ((size_t)a.nbid + a.ntiers + 2 * (size_t)a.ntiers * p.R * p.K);
+    if (a.nbid > 0) smem += sizeof(uint32_t) * ((size_t)a.nbid + 2 * (size_t)a.ntiers * p.R * p.K);
     const size_t nrem_bytes = sizeof(int32_t) * (size_t)a.dmax * p.R;
     const size_t tm_bytes = sizeof(uint32_t) * (size_t)a.ntiers * a.W * p.R * p.K;
     a.tm_in_smem = (a.ntiers > 0 && smem + tm_bytes <= 96 * 1024) ? 1 : 0;
