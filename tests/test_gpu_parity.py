@@ -170,6 +170,26 @@ def test_auction_scores_that_round_together_and_a_round_cap():
         pl.close()
 
 
+@pytest.mark.parametrize("step", [0.0625, 0.25, 1.0 / 3.0, -0.05])
+def test_auction_price_steps_with_ties_across_tiers(step):
+    """Price steps that make scores of different tiers coincide exactly (1 - 15/16 = 1/16 is both the intra-node
+    bonus after 15 wins and the far-tier bonus of the three-tier cost), a coarse and an inexact step, and a negative
+    one (dense scan): the auction must follow the oracle bit for bit in every case."""
+    for cfg in (W.get_config("cfg4").replace(L=2, T=256 * 2304), W.get_config("cfg2").replace(L=3)):
+        e2r, C = topology(cfg)
+        B = O.default_preference(C.numpy())
+        topk = _routing(cfg)
+        pl = make_planner(cfg, price_step=step)
+        out = {k: cpu(v) for k, v in pl.plan(topk).items()}
+        for l in range(cfg.L):
+            m, a = oracle_schedule_layer(cfg, e2r.numpy(), B, out["n"][l], out["expert_load"][l],
+                                         out["rank_load"][l], out["plan"][l], price_step=step)
+            assert (out["X"][l] == a["X"]).all()
+            assert out["rounds"][l, 1] == a["rounds"]
+            assert bool(out["info"][l] & 8) == (a["residual"] > 0)
+        pl.close()
+
+
 def test_plan_is_capturable_in_a_cuda_graph():
     """taot_plan neither allocates nor synchronises, so a stream capture of it replays to the same bits
     (the paper stresses CUDA-graph compatibility of the planner, Appendix A.4)."""
