@@ -305,7 +305,7 @@ __device__ __forceinline__ bool tile_solve(const SinkArgs& a, TileSmem<NW, CG>& 
 // butterfly every lane of the group holds the same bits, so u~ and v~ are computed redundantly where they are
 // needed and nothing is broadcast.  For the small problems of the planner (a few supply ranks, tens of demand
 // ranks) this is a much shorter dependent chain per iteration than one row set per lane.
-template <int NRA, int NCG, int CG>
+template <int NRA, int NCG, int CG, bool TOL>
 __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& sm, int Hn, int Cn, double sum_st,
                                            int info, float* out, int64_t b)
 {
@@ -395,37 +395,38 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
 #pragma unroll
             for (int cg = 0; cg < NCG; ++cg) cp[cg] += __shfl_xor_sync(kFull, cp[cg], off);
         }
-        // ---- the row sums belong to iterate t: is this where the solve stops?
-        const bool last = t >= a.max_iters;
-        const bool check = a.tol > 0.0f && until_check == 1;
-        float err = 0.0f;
-        if (last || check) {                                             // uniform over the warp
+        // ---- the row sums belong to iterate t: is this where the solve stops?  The loop body is kept free of
+        // branches (a lone warp pays dearly for each one): in tolerance mode the error is computed every iteration,
+        // and the stop test and the drift test share one rarely taken branch.
+        auto row_error = [&]() {
             float e = 0.0f;
 #pragma unroll
             for (int ra = 0; ra < NRA; ++ra) e += row_ok[ra] ? fabsf(fmaf(uo[ra], r[ra], -stl[ra])) : 0.0f;
 #pragma unroll
             for (int off = CL; off < 32; off <<= 1) e += __shfl_xor_sync(kFull, e, off);
-            err = e;                                                     // the same bits in every lane
-        }
+            return e;                                                    // the same bits in every lane
+        };
+        float err = 0.0f;
+        if (TOL) err = row_error();
 #pragma unroll
         for (int cg = 0; cg < NCG; ++cg) vnew[cg] = col_ok[cg] ? ddg[cg] * rcp_fast(cp[cg]) : 1.0f;
-        if (last || (check && err <= tol_abs_f)) {
-            bool bad_r = false;
-#pragma unroll
-            for (int ra = 0; ra < NRA; ++ra) bad_r |= row_ok[ra] && !(r[ra] > kSumLo && r[ra] < kSumHi);
-            if (__any_sync(kFull, bad_r)) return false;
-            err_out = (float)((double)err / sum_st);
-            if (a.tol > 0.0f && !(err <= tol_abs_f)) info |= TAOT_INFO_SINKHORN_CAP;
-            break;
+        bool stop = t >= a.max_iters;
+        if (TOL) {
+            const bool check = until_check == 1;
+            stop |= check && err <= tol_abs_f;
+            until_check = check ? a.check_every : until_check - 1;
         }
-        // ---- commit iteration t+1
+        if (stop | odd) {
+            if (stop) {
+                if (!TOL) err = row_error();
+                bool bad_r = false;
 #pragma unroll
-        for (int ra = 0; ra < NRA; ++ra) uo[ra] = un[ra];
-#pragma unroll
-        for (int cg = 0; cg < NCG; ++cg) vreg[cg] = vnew[cg];
-        ++t;
-        until_check = until_check == 1 ? a.check_every : until_check - 1;
-        if (odd) {
+                for (int ra = 0; ra < NRA; ++ra) bad_r |= row_ok[ra] && !(r[ra] > kSumLo && r[ra] < kSumHi);
+                if (__any_sync(kFull, bad_r)) return false;
+                err_out = (float)((double)err / sum_st);
+                if (TOL && !(err <= tol_abs_f)) info |= TAOT_INFO_SINKHORN_CAP;
+                break;
+            }
             // rare: either u~, v~ merely drifted (fold them into the potentials) or a sum of this update left the
             // range in which fp32 products are trustworthy (hand the problem back)
             bool bad = false;
@@ -434,20 +435,28 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
 #pragma unroll
             for (int cg = 0; cg < NCG; ++cg) bad |= col_ok[cg] && !(cp[cg] > kSumLo && cp[cg] < kSumHi);
             if (__any_sync(kFull, bad)) return false;
-            // fold u~, v~ into the fp64 potentials (one lane per row / column) and rebuild the tile around them
+            // commit iteration t+1, fold u~, v~ into the fp64 potentials (one lane per row / column), rebuild the tile
 #pragma unroll
             for (int ra = 0; ra < NRA; ++ra)
-                if (row_ok[ra] && lc == 0) sm.alpha[ra * RL + lr] += log((double)uo[ra]);
+                if (row_ok[ra] && lc == 0) sm.alpha[ra * RL + lr] += log((double)un[ra]);
 #pragma unroll
             for (int cg = 0; cg < NCG; ++cg)
-                if (col_ok[cg] && lr == 0) sm.beta[cg * CL + lc] += log((double)vreg[cg]);
+                if (col_ok[cg] && lr == 0) sm.beta[cg * CL + lc] += log((double)vnew[cg]);
             __syncwarp();
 #pragma unroll
             for (int ra = 0; ra < NRA; ++ra) uo[ra] = 1.0f;
 #pragma unroll
             for (int cg = 0; cg < NCG; ++cg) vreg[cg] = 1.0f;
             build_tile();
+            ++t;
+            continue;
         }
+        // ---- commit iteration t+1
+#pragma unroll
+        for (int ra = 0; ra < NRA; ++ra) uo[ra] = un[ra];
+#pragma unroll
+        for (int cg = 0; cg < NCG; ++cg) vreg[cg] = vnew[cg];
+        ++t;
     }
 
     // ---- T = diag(u) M diag(v) from the total potentials, then the column cap
@@ -494,11 +503,11 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
 }
 
 // Picks the smallest lane-grid tile that holds the problem (one warp); false: hand the problem back.
-template <int CG>
+template <int CG, bool TOL>
 __device__ __forceinline__ bool grid_dispatch(const SinkArgs& a, TileSmem<1, CG>& sm, int Hn, int Cn, double sum_st,
                                               int info, float* out, int64_t b)
 {
-#define TAOT_GRID(NRA, NCG) grid_solve<NRA, NCG, CG>(a, sm, Hn, Cn, sum_st, info, out, b)
+#define TAOT_GRID(NRA, NCG) grid_solve<NRA, NCG, CG, TOL>(a, sm, Hn, Cn, sum_st, info, out, b)
     if (CG == 1) {                     // up to 32 ranks
         if (Cn <= 16) {
             if (Hn <= 4) return TAOT_GRID(1, 2);
@@ -611,7 +620,10 @@ sinkhorn_tile_kernel(SinkArgs a)
     __syncthreads();
 
     bool done;
-    if constexpr (NW == 1) done = grid_dispatch<CG>(a, sm, Hn, Cn, sum_st, info, out, b);
+    if constexpr (NW == 1) {
+        done = a.tol > 0.0f ? grid_dispatch<CG, true>(a, sm, Hn, Cn, sum_st, info, out, b)
+                            : grid_dispatch<CG, false>(a, sm, Hn, Cn, sum_st, info, out, b);
+    }
     else if (Hn <= NW * RP0) done = tile_solve<NW, RP0, CG>(a, sm, Hn, Cn, sum_st, info, out, b);
     else if (Hn <= NW * RP1) done = tile_solve<NW, RP1, CG>(a, sm, Hn, Cn, sum_st, info, out, b);
     else done = tile_solve<NW, RP2, CG>(a, sm, Hn, Cn, sum_st, info, out, b);
