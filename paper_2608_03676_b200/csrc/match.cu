@@ -214,19 +214,24 @@ match_kernel(MatchArgs a)
 
     // =========================================================== Phase 2
     int rounds2 = 0;
+    int qsh = 0;                                  // lanes per rank in the scan: QS = 2^qsh, the largest power of two <= min(32, NT / R)
+    while ((2 << qsh) <= 32 && (2 << qsh) * R <= NT) ++qsh;
+    const int QS = 1 << qsh;
+    const int qs = tid & (QS - 1);
     for (int kappa = 0; kappa < K; ++kappa) {
         for (int r = tid; r < R; r += NT) matched[r] = 0;
         for (;;) {
             if (tid == 0) s_any = 0;
             __syncthreads();
-            // Steps 1-2: every unmatched cold rank takes its best candidate expert
-            for (int rb = 0; rb < R; rb += NT) {
-                const int r = rb + tid;                       // whole warps stay in the loop for the warp-wide arbitration
+            // Steps 1-2: every unmatched cold rank takes its best candidate expert.  QS adjacent lanes share one rank
+            // and split the list of spilling experts between them; their best keys meet by xor-shuffles.
+            for (int rb = 0; rb < R; rb += NT >> qsh) {
+                const int r = rb + (tid >> qsh);                  // whole warps stay in the loop for the warp-wide steps
                 int best_e = -1;
                 u64 key = 0;
                 const int32_t sp = r < R ? spare[r] : 0;
                 if (r < R && !matched[r] && sp > 0) {
-                    for (int q = 0; q < nhot0; ++q) {
+                    for (int q = qs; q < nhot0; q += QS) {
                         const int e = hot0[q];
                         const int32_t se = spill[e];
                         if (se <= 0 || hot_home[q] == r) continue;
@@ -241,13 +246,18 @@ match_kernel(MatchArgs a)
                         key = k64 > key ? k64 : key;
                     }
                 }
-                if (key != 0) {
-                    best_e = (int)(0xFFFFFFFFu - (uint32_t)key);
-                    s_any = 1;
+                for (int o = 1; o < QS; o <<= 1) {
+                    const u64 other = __shfl_xor_sync(0xffffffffu, key, o);
+                    key = other > key ? other : key;
                 }
-                if (r < R) estar[r] = best_e;
+                if (key != 0) best_e = (int)(0xFFFFFFFFu - (uint32_t)key);
+                const bool lead = qs == 0 && r < R;
+                if (lead) {
+                    estar[r] = best_e;
+                    if (key != 0) s_any = 1;
+                }
                 // Step 3: arbitration, best rank per expert (ties: lowest rank)
-                arbitrate(arb_e, best_e, key == 0 ? 0ull : ((key & 0xFFFFFFFF00000000ull) | (u64)(0xFFFFFFFFu - (uint32_t)r)));
+                arbitrate(arb_e, best_e, (key == 0 || !lead) ? 0ull : ((key & 0xFFFFFFFF00000000ull) | (u64)(0xFFFFFFFFu - (uint32_t)r)));
             }
             __syncthreads();
             if (!s_any) break;
