@@ -49,7 +49,7 @@ def parse_args():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="cfg2", choices=sorted(W.CONFIGS))
     ap.add_argument("--layers", type=int, default=0, help="override L (smaller batch, e.g. for a profiler capture)")
-    ap.add_argument("--cpu-seconds", type=float, default=20.0, help="budget of the CPU-baseline sample")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-groups", type=int, default=4,
                     help="layer groups (streams) the end-to-end host call is pipelined over")
@@ -153,22 +153,45 @@ def timed_steps(fn, steps, flush):
     return [a.elapsed_time(b) for a, b in pairs]
 
 
-def oracle_sample(cfg, topk_cpu, seconds):
-    """Time the CPU oracle, as it stands, on a bounded sample of the workload: whole layers, as many
-    as fit in about `seconds` (at least one)."""
+def oracle_sample(cfg, topk_cpu, seconds, threads=1):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload: whole layers, taken round-robin
+    (the workload is repeated if it is shorter than the budget) for about `seconds`.  threads > 1: that many
+    layers at a time, one per host thread (the C routines release the interpreter lock)."""
     import oracle as O
     e2r = W.expert_to_rank(cfg.E, cfg.R, cfg.e2r_mode).numpy()
     C = W.cost_matrix(cfg.R, cfg.gpus_per_node, cfg.tiers, cfg.nodes_per_group).numpy()
     O.build()
+    one = lambda l: O.plan_layers(topk_cpu[l:l + 1], cfg.R, cfg.E, cfg.K, e2r, C, cfg.eps, cfg.max_iters, cfg.tol)
     done, t_total = 0, 0.0
-    while done < cfg.L:
-        t0 = time.perf_counter()
-        O.plan_layers(topk_cpu[done:done + 1], cfg.R, cfg.E, cfg.K, e2r, C, cfg.eps, cfg.max_iters, cfg.tol)
-        t_total += time.perf_counter() - t0
-        done += 1
-        if t_total + t_total / done > seconds:
-            break
+    if threads <= 1:
+        while True:
+            t0 = time.perf_counter()
+            one(done % cfg.L)
+            t_total += time.perf_counter() - t0
+            done += 1
+            if t_total + t_total / done > seconds:
+                break
+        return done, t_total
+    from concurrent.futures import ThreadPoolExecutor
+    with ThreadPoolExecutor(max_workers=threads) as pool:
+        while True:
+            t0 = time.perf_counter()
+            list(pool.map(one, [(done + i) % cfg.L for i in range(threads)]))
+            t_total += time.perf_counter() - t0
+            done += threads
+            if t_total + t_total * threads / done > seconds:
+                break
     return done, t_total
+
+
+def cpu_model():
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.startswith("model name"):
+                return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
 
 
 def sinkhorn_work(out, cfg):
@@ -405,13 +428,16 @@ def run_ours(args):
     line = dict(
         metric=METRIC,
         value=value, unit="plans/s", n_gpus=world, steps=args.steps, warmup=max(3, args.warmup),
-        ms_per_step=float(np.mean(ms)), higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
+        ms_per_step=float(np.mean(ms)), ms_per_step_median=float(np.median(ms)), ms_per_step_min=float(np.min(ms)),
+        higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
         data="synthetic",
         config=dict(workload=args.workload, L=cfg.L, R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k, T=cfg.T,
                     eps=cfg.eps, max_iters=cfg.max_iters, tol=cfg.tol,
                     l2="flushed between steps (256 MiB write)" if need_flush else "inputs larger than L2",
                     parallelism=f"{world} independent replica(s)"),
-        remapped_tokens_per_s=world * cfg.L * cfg.T * args.steps / total_s,
+        remapped_tokens_per_s=cfg.L * cfg.T / (float(stage_ms[4]) * 1e-3),
+        histogram_tokens_per_s=cfg.L * cfg.T / (float(stage_ms[0]) * 1e-3),
+        planned_tokens_per_s=world * cfg.L * cfg.T * args.steps / total_s,
         stages_ms=dict(zip(STAGES, [float(x) for x in stage_ms])),
         sinkhorn=dict(iters_mean=float(iters.mean()), iters_max=int(iters.max()),
                       converged_frac=float(((info & 2) == 0).mean()),
@@ -436,7 +462,13 @@ def run_ours(args):
     if world == 1 and not args.no_cpu_baseline:
         n_layers, secs = oracle_sample(cfg, topk.cpu().numpy(), args.cpu_seconds)
         line["cpu_baseline"] = dict(value=n_layers / secs, unit="plans/s", cores=1, kind="oracle",
-                                    sample=f"{n_layers} whole layer(s) of {cfg.L}, {secs:.2f} s")
+                                    sample=f"{n_layers} whole layer(s) (the {cfg.L}-layer workload taken round-robin), "
+                                           f"{secs:.2f} s", cpu=cpu_model())
+        cores = max(1, min(len(os.sched_getaffinity(0)), cfg.L))
+        if cores > 1:
+            n_mt, secs_mt = oracle_sample(cfg, topk.cpu().numpy(), max(2.0, args.cpu_seconds / 4), threads=cores)
+            line["cpu_baseline_threads"] = dict(value=n_mt / secs_mt, unit="plans/s", cores=cores, kind="oracle",
+                                                sample=f"{n_mt} whole layer(s), one per host thread, {secs_mt:.2f} s")
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
