@@ -1,0 +1,9 @@
+// Register-tile Sinkhorn kernel, up to 64 ranks (one warp per problem, 4x8 lane grid).
+#include "sinkhorn_tile.cuh"
+
+int taot_launch_sinkhorn_tile_r64(const SinkArgs& a, int32_t B, int sm_count, cudaStream_t st)
+{
+    sinkhorn_tile_kernel<1, 2, 8, 16, 32, 1><<<B, 32, 0, st>>>(a, (int64_t)B);
+    TAOT_CUDA_OK(cudaGetLastError());
+    return 1;
+}
