@@ -345,6 +345,7 @@ int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, in
     a.inv_eps = 1.0 / (double)p.eps;
     a.eps0 = p.eps0; a.max_iters = p.max_iters; a.tol = p.tol;
     a.check_every = p.check_every < 1 ? 1 : p.check_every;
+    a.skip_solved = 0;
     a.kt_global = h->kcap_global > 0 ? d_kt : nullptr;
     a.kcap_global = h->kcap_global;
     const int NT = p.R <= 32 ? 32 : (p.R <= 64 ? 128 : (p.R <= 128 ? 256 : (p.R <= 256 ? 512 : 1024)));

@@ -22,9 +22,20 @@ struct SinkArgs {
     float tol;
     int32_t check_every;
     int32_t only_marked;     // generic kernel: solve only the problems the register-tile kernel handed back
+    int32_t skip_solved;     // tile kernels: solve only the problems an earlier kernel of the chain handed back
     float* kt_global;        // [B][kcap_global] kernel-matrix scratch in global memory for problems too big for
     int64_t kcap_global;     // shared memory (floats per problem); null / 0 if the handle has none
 };
+
+// exp(x) rounded to fp32 for an fp64 argument of either sign and any magnitude the solve meets: x = xh + xl with
+// xh = fl32(x), exp(x) = expf(xh) * (1 + xl).  Relative error ~3e-7 (expf is the accurate one, 2 ulp), at a small
+// fraction of the cost of an fp64 exponential on this GPU.
+__device__ __forceinline__ float exp_split(double x)
+{
+    const float xh = (float)x;
+    const float xl = (float)(x - (double)xh);
+    return expf(xh) * (1.0f + xl);
+}
 
 constexpr float kDriftLo = 2.0611536e-9f;   // e^-20
 constexpr float kDriftHi = 4.8516520e8f;    // e^+20

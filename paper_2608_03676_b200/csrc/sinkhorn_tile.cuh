@@ -98,7 +98,7 @@ __device__ __forceinline__ bool tile_solve(const SinkArgs& a, TileSmem<NW, CG>& 
                 float v = 0.0f;
                 if (row < Hn && col < Cn) {
                     const double c = (double)a.C[(int64_t)sm.hot[row] * R + sm.cold[col]] * a.inv_eps;
-                    v = (float)exp(sm.alpha[row] + sm.beta[col] - c);
+                    v = exp_split(sm.alpha[row] + sm.beta[col] - c);
                 }
                 K[aa][g] = v;
             }
@@ -342,7 +342,7 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
                 float v = 0.0f;
                 if (row < Hn && col < Cn) {
                     const double c = (double)a.C[(int64_t)sm.hot[row] * R + sm.cold[col]] * a.inv_eps;
-                    v = (float)exp(sm.alpha[row] + sm.beta[col] - c);
+                    v = exp_split(sm.alpha[row] + sm.beta[col] - c);
                 }
                 K[ra][cg] = v;
             }
@@ -544,6 +544,7 @@ __device__ __forceinline__ void tile_problem(const SinkArgs& a, TileSmem<NW, CG>
 {
     constexpr int NT = NW * 32;
     const int R = a.R, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (a.skip_solved && a.iters[b] != kHandBack) return;      // chained launch: only what an earlier kernel left
 
     // ---- supply scaling gamma = min(1, sum d / max(sum s, eps0)), compaction of supply / demand ranks
     {
@@ -577,7 +578,7 @@ __device__ __forceinline__ void tile_problem(const SinkArgs& a, TileSmem<NW, CG>
     __syncthreads();
     const int Hn = compact_positive(sm.sv, R, sm.hot, sm.hpos, sm.wcnt);
     const int Cn = compact_positive(sm.dv, R, sm.cold, sm.cpos, sm.wcnt);
-    if (Hn > (NW == 1 ? 32 : NW * RP2)) {    // does not fit any tile: the other kernel takes it
+    if (Hn > (NW == 1 ? 32 : NW * RP2)) {    // does not fit any tile: another kernel takes it
         if (tid == 0) a.iters[b] = kHandBack;
         return;
     }

@@ -21,7 +21,9 @@ def _planner(B, R, eps_frac, iters=SWEEP_ITERS, tol=0.0):
     return pl, C
 
 
-@pytest.mark.parametrize("R,B,check", [(8, 64, 64), (16, 64, 64), (64, 64, 16), (256, 64, 4), (1024, 3, 1)])
+@pytest.mark.parametrize("R,B,check", [(8, 64, 64), (16, 64, 64), (64, 64, 16), (256, 64, 4), (1024, 3, 1),
+                                       # batches of at least 4 x 148 problems take the batch builds of the kernels
+                                       (16, 1024, 8), (64, 1024, 6), (256, 640, 3)])
 @pytest.mark.parametrize("eps_frac", [0.1, 0.01])
 def test_sweep_cell(R, B, check, eps_frac):
     pl, C = _planner(B, R, eps_frac)
@@ -44,6 +46,31 @@ def test_sweep_cell(R, B, check, eps_frac):
     assert bool((col_viol <= 1e-5 * tot).all())
     assert bool((out["plan"] >= 0).all())
     print(f"R={R} eps={eps_frac}: worst rel err {worst:.2e} over {check} problems")
+    pl.close()
+
+
+def test_large_batch_with_mixed_problem_sizes_walks_the_kernel_chain():
+    """A batch that takes the 4-warp batch kernel, in which some problems have more supply ranks than that kernel
+    holds (they must come back marked and be solved by the 16-warp kernel), in tolerance mode."""
+    R, B = 256, 640
+    pl, C = _planner(B, R, 0.1, iters=300, tol=1e-6)
+    loads = W.sweep_rank_loads(B, R, seed=77, device="cuda")
+    g = torch.Generator(device="cuda").manual_seed(9)
+    wide = torch.randint(1000, 60000, (B // 2, R), generator=g, device="cuda", dtype=torch.int32)
+    loads[1::2] = wide                                   # every other problem: about half of the ranks above the mean
+    ex, sp, s, d = pl.excess_spare(loads)
+    hn = (ex > 0).sum(1)
+    assert int(hn[0::2].max()) <= 32 < int(hn[1::2].min())      # some of the wide ones exceed 128 too: third kernel
+    out = pl.sinkhorn(s, d)
+    torch.cuda.synchronize()
+    plan, iters, err, info = cpu(out["plan"]), cpu(out["iters"]), cpu(out["row_err"]), cpu(out["info"])
+    assert (iters >= 1).all() and (iters <= 300).all() and ((info & ~(2 | 16)) == 0).all()   # 16: supply scaled (the integer mean leaves a remainder)
+    for b in (0, 1, 2, 3, 638, 639):
+        check_sinkhorn_problem(cpu(s)[b], cpu(d)[b], C.numpy(), 0.1 * max(SWEEP_TIERS), plan[b], iters[b], err[b],
+                               300, 1e-6)
+    tot = s.double().sum(1)
+    col_viol = (out["plan"].double().sum(1) - d.double()).abs().sum(1)
+    assert bool((col_viol <= 1e-5 * tot).all()) and bool((out["plan"] >= 0).all())
     pl.close()
 
 
