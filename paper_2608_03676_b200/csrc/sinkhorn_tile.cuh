@@ -614,7 +614,7 @@ __device__ __forceinline__ void tile_problem(const SinkArgs& a, TileSmem<NW, CG>
         }
         double acc = 0.0;
         for (int i = 0; i < Hn; ++i)
-            acc += exp(sm.phin[i] - (double)a.C[(int64_t)sm.hot[i] * R + cj] * a.inv_eps - mx);
+            acc += (double)exp_split(sm.phin[i] - (double)a.C[(int64_t)sm.hot[i] * R + cj] * a.inv_eps - mx);
         sm.beta[j] = log((double)sm.dd[j]) - (mx + log(acc));
     }
     for (int i = tid; i < Hn; i += NT) sm.alpha[i] = sm.phin[i];
