@@ -354,6 +354,13 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
     float err_out = 0.0f;
     const float tol_abs_f = (float)tol_abs;
     const uint32_t lo_bits = __float_as_uint(kDriftLo), span_bits = __float_as_uint(kDriftHi) - lo_bits;
+    float usave[NRA], vsave[NCG];    // tolerance mode: the iterate whose error is still to be tested
+    bool pend = false;
+    float err_pend = 0.0f;
+#pragma unroll
+    for (int ra = 0; ra < NRA; ++ra) usave[ra] = 1.0f;
+#pragma unroll
+    for (int cg = 0; cg < NCG; ++cg) vsave[cg] = 1.0f;
 
     for (;;) {
         // Drift test on the u~, v~ this iteration STARTS from; the vote is issued here and consumed at the end of
@@ -368,18 +375,21 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
         odd = __any_sync(kFull, odd);
         // ================= half-step 1: r = K~ v~, u' = s~ / r
         float r[NRA], un[NRA];
+        auto row_sums = [&]() {
 #pragma unroll
-        for (int ra = 0; ra < NRA; ++ra) {
-            float acc = K[ra][0] * vreg[0];
+            for (int ra = 0; ra < NRA; ++ra) {
+                float acc = K[ra][0] * vreg[0];
 #pragma unroll
-            for (int cg = 1; cg < NCG; ++cg) acc = fmaf(K[ra][cg], vreg[cg], acc);
-            r[ra] = acc;
-        }
+                for (int cg = 1; cg < NCG; ++cg) acc = fmaf(K[ra][cg], vreg[cg], acc);
+                r[ra] = acc;
+            }
 #pragma unroll
-        for (int off = 1; off < CL; off <<= 1) {
+            for (int off = 1; off < CL; off <<= 1) {
 #pragma unroll
-            for (int ra = 0; ra < NRA; ++ra) r[ra] += __shfl_xor_sync(kFull, r[ra], off);
-        }
+                for (int ra = 0; ra < NRA; ++ra) r[ra] += __shfl_xor_sync(kFull, r[ra], off);
+            }
+        };
+        row_sums();
 #pragma unroll
         for (int ra = 0; ra < NRA; ++ra) un[ra] = row_ok[ra] ? stl[ra] * rcp_fast(r[ra]) : 1.0f;
         // ================= half-step 2 (speculative until the stop test): c = K~^T u', v' = d / c
@@ -397,8 +407,9 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
             for (int cg = 0; cg < NCG; ++cg) cp[cg] += __shfl_xor_sync(kFull, cp[cg], off);
         }
         // ---- the row sums belong to iterate t: is this where the solve stops?  The loop body is kept free of
-        // branches (a lone warp pays dearly for each one): in tolerance mode the error is computed every iteration,
-        // and the stop test and the drift test share one rarely taken branch.
+        // branches (a lone warp pays dearly for each one) and the one branch it has never waits for this iteration's
+        // error: in tolerance mode the error of iterate t is computed every iteration but TESTED one iteration later,
+        // when it has long arrived; the iterate it belongs to is kept in registers and restored if the test passes.
         auto row_error = [&]() {
             float e = 0.0f;
 #pragma unroll
@@ -407,23 +418,41 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
             for (int off = CL; off < 32; off <<= 1) e += __shfl_xor_sync(kFull, e, off);
             return e;                                                    // the same bits in every lane
         };
-        float err = 0.0f;
-        if (TOL) err = row_error();
+        auto rows_bad = [&]() {
+            bool bad_r = false;
+#pragma unroll
+            for (int ra = 0; ra < NRA; ++ra) bad_r |= row_ok[ra] && !(r[ra] > kSumLo && r[ra] < kSumHi);
+            return __any_sync(kFull, bad_r) != 0;
+        };
+        float err_now = 0.0f;
+        bool check_now = false;
+        if (TOL) {
+            err_now = row_error();
+            check_now = until_check == 1;
+            until_check = check_now ? a.check_every : until_check - 1;
+        }
 #pragma unroll
         for (int cg = 0; cg < NCG; ++cg) vnew[cg] = col_ok[cg] ? ddg[cg] * rcp_fast(cp[cg]) : 1.0f;
-        bool stop = t >= a.max_iters;
-        if (TOL) {
-            const bool check = until_check == 1;
-            stop |= check && err <= tol_abs_f;
-            until_check = check ? a.check_every : until_check - 1;
-        }
-        if (stop | odd) {
-            if (stop) {
-                if (!TOL) err = row_error();
-                bool bad_r = false;
+        const bool stop_prev = TOL && pend && err_pend <= tol_abs_f;
+        const bool last = t >= a.max_iters;
+        if (stop_prev | last | odd) {
+            if (stop_prev) {
+                // iterate t-1 met the tolerance: go back to it (its row sums are recomputed for the range check)
 #pragma unroll
-                for (int ra = 0; ra < NRA; ++ra) bad_r |= row_ok[ra] && !(r[ra] > kSumLo && r[ra] < kSumHi);
-                if (__any_sync(kFull, bad_r)) return false;
+                for (int ra = 0; ra < NRA; ++ra) uo[ra] = usave[ra];
+#pragma unroll
+                for (int cg = 0; cg < NCG; ++cg) vreg[cg] = vsave[cg];
+                --t;
+                row_sums();
+                const float err = row_error();
+                if (rows_bad()) return false;
+                err_out = (float)((double)err / sum_st);
+                break;
+            }
+            if (last || (check_now && err_now <= tol_abs_f)) {
+                // the iteration cap, or (only reached together with a drift event) a test that is due right now
+                const float err = TOL ? err_now : row_error();
+                if (rows_bad()) return false;
                 err_out = (float)((double)err / sum_st);
                 if (TOL && !(err <= tol_abs_f)) info |= TAOT_INFO_SINKHORN_CAP;
                 break;
@@ -449,10 +478,19 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
 #pragma unroll
             for (int cg = 0; cg < NCG; ++cg) vreg[cg] = 1.0f;
             build_tile();
+            pend = false;                        // the test of iterate t was settled above
             ++t;
             continue;
         }
-        // ---- commit iteration t+1
+        // ---- commit iteration t+1; iterate t stays behind until its error has been tested
+        if (TOL) {
+            pend = check_now;
+            err_pend = err_now;
+#pragma unroll
+            for (int ra = 0; ra < NRA; ++ra) usave[ra] = uo[ra];
+#pragma unroll
+            for (int cg = 0; cg < NCG; ++cg) vsave[cg] = vreg[cg];
+        }
 #pragma unroll
         for (int ra = 0; ra < NRA; ++ra) uo[ra] = un[ra];
 #pragma unroll
