@@ -12,17 +12,19 @@
 //   assign_prep_kernel   one CTA per (layer, source rank): per chunk, the table expert -> target of
 //                        the chunk's LAST entry of that expert, and the splits (expert, in-chunk
 //                        ordinal, slot before); up to four of them ride in the tail of the table row;
-//   assign_stream_kernel persistent, one CTA per SM: chunks staged in shared memory by bulk
-//                        asynchronous copies (cp.async.bulk + mbarrier, no multicast), several in
-//                        flight; per entry one table lookup; in a chunk with splits the CTA first finds
-//                        each split's flat position (per-warp counts, then ballots in the one warp that
-//                        holds it) and applies "expert e before position P -> slot" as predicated
-//                        overrides; 16-byte streaming stores.  The compute hides under the copies.
-//   assign_chunk_kernel  one CTA per chunk: the chunks that do hold a split (staged in shared memory the same
-//                        way, since they are read three times), and, with ordinary loads, every chunk of a
-//                        routing table that is not 16-byte aligned or whose segments are not multiples of 4.
-// 8 bytes of HBM traffic per entry (one read, one write).  Out-of-range indices are copied through (the histogram pass, whose counts this path
-// consumes, is the one that flags them).
+//   assign_stream_kernel persistent, one CTA per SM, for the chunks WITHOUT a split: a producer warp claims chunks
+//                        from a global counter and stages them (and their table rows) in shared memory with bulk
+//                        asynchronous copies (cp.async.bulk + mbarrier, no multicast), three stages in flight;
+//                        16 consumer warps do one table lookup per entry and 16-byte streaming stores; full /
+//                        empty mbarriers per stage, no CTA-wide barrier in the loop, every wait bounded;
+//   assign_chunk_kernel  one CTA per chunk: the chunks that do hold a split, staged in shared memory the same way
+//                        since they are read three times -- per-warp counts of the split experts, ballots in the
+//                        one warp that holds a split to find its flat position, then the rewrite with
+//                        "expert e before position P -> slot" as predicated overrides -- and, with ordinary loads,
+//                        every chunk of a routing table that is not 16-byte aligned or whose segments are not
+//                        multiples of 4 entries.
+// 8 bytes of HBM traffic per entry (one read, one write).  Out-of-range indices are copied through (the histogram
+// pass, whose counts this path consumes, is the one that flags them).
 #include "taot_internal.cuh"
 
 namespace {

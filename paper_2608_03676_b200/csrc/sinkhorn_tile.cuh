@@ -1,19 +1,26 @@
 // Phase 1 fast path: Sinkhorn-Knopp (Appendix A.2) with the absorbed kernel matrix K~ held in
 // REGISTERS.  Same arithmetic as the shared-memory kernel in sinkhorn.cu (absorbed potentials,
-// fp32 mat-vecs, fp64 folds), different data placement:
+// fp32 mat-vecs, fp64 folds), different data placement.  Two layouts:
 //
+// grid_solve (one warp per problem, up to 64 ranks): a 4 x 8 lane grid; lane (lr, lc) holds K~ for rows
+//   ra*4 + lr and columns cg*8 + lc.  Row sums reduce over the 8 column lanes and column sums over the 4 row
+//   lanes by xor-butterflies, after which every lane of a group holds the same bits, so u~ and v~ are computed
+//   where they are needed and nothing is broadcast.  No barrier, no shared memory and (besides one rarely taken
+//   exit) no branch in the loop.
+//
+// tile_solve (4 or 16 warps per problem, up to 128 / 256 ranks):
 //   warp w owns compact rows [w*RPW, (w+1)*RPW)  (rows = ranks with supply),
 //   lane l owns compact columns l + 32*g, g < CG (columns = ranks with demand),
 //   K[a][g] in registers; every warp keeps v~ for its lane's columns in registers.
+//   Half-step 1 (row sums) is warp-local: RPW partial sums per lane are reduced across the 32 lanes
+//   by a transposing butterfly (RPW-1 + log2(32/RPW) shuffles for all rows together), after which
+//   lane a holds row a's sum and computes u~_a = s~_a / r_a.  Half-step 2 (column sums) is
+//   lane-local over the warp's rows (u~_a broadcast by shuffle); the partials of the warps
+//   meet in shared memory (two block barriers per iteration).
 //
-// Half-step 1 (row sums) is warp-local: RPW partial sums per lane are reduced across the 32 lanes
-// by a transposing butterfly (RPW-1 + log2(32/RPW) shuffles for all rows together), after which
-// lane a holds row a's sum and computes u~_a = s~_a / r_a.  Half-step 2 (column sums) is
-// lane-local over the warp's rows (u~_a broadcast by shuffle); with several warps the partials
-// meet in shared memory (two block barriers per iteration, none with one warp).
-//
-// A problem that does not fit the tile (more than NW*RPW rows with supply), or whose fp32 sums
-// leave the safe range, is handed back (iters[b] = -1) and solved by the shared-memory kernel.
+// A problem that does not fit the tile (too many rows with supply), or whose fp32 sums leave the
+// safe range, is handed back (iters[b] = -1) and solved by the next kernel of the chain, in the end
+// by the shared-memory kernel, which holds any problem.
 #pragma once
 #include "sinkhorn_common.cuh"
 
