@@ -18,7 +18,8 @@ def _full_check(cfg, topk, pl, B=None, e2r=None, C=None, expect_bad=False):
     e2r = e2r_t.numpy() if e2r is None else e2r
     C = C_t.numpy() if C is None else C
     Bm = O.default_preference(C) if B is None else B
-    out = {k: cpu(v) for k, v in pl.plan(topk).items()}
+    dev = pl.plan(topk)
+    out = {k: cpu(v) for k, v in dev.items()}
     tk = cpu(topk)
     n, el, rl, bad = O.histogram(tk, cfg.R, cfg.E, e2r)
     assert (out["n"] == n).all() and (out["expert_load"] == el).all() and (out["rank_load"] == rl).all()
@@ -37,6 +38,23 @@ def _full_check(cfg, topk, pl, B=None, e2r=None, C=None, expect_bad=False):
         assert (out["X"][l] == a["X"]).all()
         want = O.assign(tk[l], cfg.R, cfg.E, cfg.K, m["slot_expert"], a["X"])
         assert (out["new_idx"][l] == want).all()
+    # the diagnostics and the dispatch metadata of the same plan
+    rep = pl.report(dev["expert_load"], dev["rank_load"], dev["slot_expert"], dev["X"], 3.0)
+    dsp = pl.dispatch(dev["new_idx"])
+    torch.cuda.synchronize()
+    for l in range(cfg.L):
+        wr = O.report(cfg.R, cfg.E, cfg.K, e2r, C, Bm, el[l], rl[l], out["slot_expert"][l], out["X"][l], 3.0)
+        for key in O.REPORT_INTS:
+            assert int(rep[key][l]) == wr[key], (l, key)
+        for key in O.REPORT_REALS:
+            assert float(rep[key][l]) == wr[key], (l, key)
+        for key in ("spill", "load_after", "slot_moved", "slot_kind"):
+            assert (cpu(rep[key])[l] == wr[key]).all(), (l, key)
+        wd = O.dispatch(out["new_idx"][l], cfg.R, cfg.E, cfg.K, e2r)
+        assert (cpu(dsp["perm"])[l] == wd["perm"]).all()
+        assert (cpu(dsp["send_counts"])[l] == wd["send_counts"]).all()
+        assert (cpu(dsp["target_counts"])[l] == wd["target_counts"]).all()
+        assert bool(cpu(dsp["info"])[l] & 1) == (wd["bad"] > 0)
     return out
 
 
