@@ -43,6 +43,26 @@ def test_full_size(name, sample):
     torch.cuda.synchronize()
     for key in ("plan", "X", "new_idx", "sinkhorn_iters"):
         assert torch.equal(again[key], out[key]), key                            # deterministic
+    # ---- report and dispatch metadata at full size: properties on every layer
+    rep = pl.report(out["expert_load"], out["rank_load"], out["slot_expert"], out["X"], 3.0)
+    dsp = pl.dispatch(out["new_idx"])
+    torch.cuda.synchronize()
+    assert (cpu(rep["load_after"]).sum(1) == L * 0 + T * k).all() and (rep["rerouted"] == cpu(out["X"].sum((1, 2)))).all()
+    assert torch.equal(dsp["send_counts"].sum(1), rep["load_after"])             # what a rank receives = its projected load
+    assert torch.equal(dsp["target_counts"][:, :, E:], out["X"])                 # guest-slot columns = the auction's X
+    seg = T // R * k
+    e2r_d = e2r.cuda().long()
+    for l in range(L):
+        new = out["new_idx"][l].reshape(R, seg).long()
+        dest = torch.where(new < E, e2r_d[new.clamp(max=E - 1)], (new - E) // K)
+        key = dest * (E + S) + new
+        perm = dsp["perm"][l].reshape(R, seg).long()
+        buf = torch.empty_like(key).scatter_(1, perm, key)                       # the send buffer, by position
+        assert bool((buf[:, 1:] >= buf[:, :-1]).all())                           # ordered by (destination, target)
+        order = torch.empty_like(perm).scatter_(1, perm, torch.arange(seg, device="cuda").expand(R, seg))
+        same = buf[:, 1:] == buf[:, :-1]
+        assert bool((order[:, 1:][same] > order[:, :-1][same]).all())            # stable among equal keys
+        assert bool((torch.sort(perm, dim=1).values == torch.arange(seg, device="cuda")).all())   # a permutation
     # ---- sampled layers against the oracle
     for l in sample:
         tk = cpu(topk[l:l + 1])
@@ -58,4 +78,9 @@ def test_full_size(name, sample):
         assert cpu(out["rounds"][l]).tolist() == [m["inner_rounds"], a["rounds"]]
         want = O.assign(tk[0], R, E, K, m["slot_expert"], a["X"])
         assert (cpu(out["new_idx"][l]) == want).all()
+        wd = O.dispatch(want, R, E, K, e2r.numpy())
+        assert (cpu(dsp["perm"][l]) == wd["perm"]).all() and (cpu(dsp["send_counts"][l]) == wd["send_counts"]).all()
+        wr = O.report(R, E, K, e2r.numpy(), C.numpy(), B, el[0], rl[0], m["slot_expert"], a["X"], 3.0)
+        assert all(int(rep[key][l]) == wr[key] for key in O.REPORT_INTS)
+        assert all(float(rep[key][l]) == wr[key] for key in O.REPORT_REALS)
     pl.close()
