@@ -334,6 +334,7 @@ __global__ void __launch_bounds__(1024) sinkhorn_kernel(SinkArgs a)
 }  // namespace
 
 int taot_launch_sinkhorn_tile(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st);
+int taot_launch_sinkhorn_cluster(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st);
 
 int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
                          int32_t* d_iters, float* d_row_err, int32_t* d_info, float* d_kt, cudaStream_t st)
@@ -367,7 +368,12 @@ int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, in
             if (n < 0) return n;
             launched += n;
         } else {
-            a.only_marked = 0;
+            // beyond 256 ranks: four-CTA clusters hold the kernel matrix in distributed shared memory; what they hand
+            // back (or everything, if no slice fits) goes to the kernel below with the matrix in workspace
+            const int n = taot_launch_sinkhorn_cluster(h, a, nb, st);
+            if (n < 0) return n;
+            launched += n;
+            a.only_marked = n > 0 ? 1 : 0;
         }
         sinkhorn_kernel<<<nb, NT, smem, st>>>(a);
         TAOT_CUDA_OK(cudaGetLastError());
