@@ -74,6 +74,28 @@ def test_large_batch_with_mixed_problem_sizes_walks_the_kernel_chain():
     pl.close()
 
 
+@pytest.mark.parametrize("R", [512, 1024])
+def test_cluster_kernel_and_its_fall_through_beyond_256_ranks(R):
+    """About half of the ranks with supply: at 512 ranks the four-CTA clusters hold the problem, at 1024 ranks a
+    slice of 128 rows x 512 columns does not fit and the problem falls through to the kernel with the matrix in
+    workspace; one narrow problem beside it stays on the clusters.  Both against the oracle."""
+    B = 3
+    pl, C = _planner(B, R, 0.1, iters=40, tol=0.0)
+    loads = W.sweep_rank_loads(B, R, seed=31, device="cuda")
+    g = torch.Generator(device="cuda").manual_seed(4)
+    loads[1] = torch.randint(1000, 60000, (R,), generator=g, device="cuda", dtype=torch.int32)
+    ex, sp, s, d = pl.excess_spare(loads)
+    hn = (ex > 0).sum(1).tolist()
+    assert hn[1] > R // 3 and hn[0] < R // 8
+    out = pl.sinkhorn(s, d)
+    torch.cuda.synchronize()
+    plan, iters, err, info = cpu(out["plan"]), cpu(out["iters"]), cpu(out["row_err"]), cpu(out["info"])
+    assert (iters == 40).all() and ((info & ~16) == 0).all()
+    for b in range(B):
+        check_sinkhorn_problem(cpu(s)[b], cpu(d)[b], C.numpy(), 0.1 * max(SWEEP_TIERS), plan[b], iters[b], err[b], 40, 0.0)
+    pl.close()
+
+
 def test_batches_larger_than_the_handle_and_unsupported_calls_beyond_256_ranks():
     import paper_2608_03676_b200 as P
     R = 512
