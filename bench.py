@@ -44,8 +44,8 @@ STAGES = ["histogram", "merge", "sinkhorn", "match_auction", "assign"]
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="cfg2", choices=sorted(W.CONFIGS))
     ap.add_argument("--layers", type=int, default=0, help="override L (smaller batch, e.g. for a profiler capture)")
