@@ -197,6 +197,7 @@ sinkhorn_cluster_kernel(SinkArgs a, int32_t kcap)
             acc += (double)exp_split(m.phin[i] - (double)a.C[(int64_t)m.hot[i] * R + cj] * a.inv_eps - mx);
         m.beta[j] = log((double)m.dd[j]) - (mx + log(acc));
         m.v[j] = 1.0f;
+        m.vn[j] = 1.0f;
     }
     for (int i = tid; i < Hn; i += kNT) m.alpha[i] = m.phin[i];
     __syncthreads();
@@ -206,27 +207,31 @@ sinkhorn_cluster_kernel(SinkArgs a, int32_t kcap)
     int t = 1;
     float err_out = 0.0f;
     bool handed_back = false;
+    // committed and candidate vectors swap roles on every commit, so an iteration needs no copy and only two block
+    // barriers besides the cluster barrier
+    float* ucur = m.u; float* unew = m.un;
+    float* vcur = m.v; float* vnew = m.vn;
+    if (tid < 4) m.flags[tid] = 0;
+    __syncthreads();
     for (;;) {
         float* xb = m.xbuf + (t & 1) * XS;
         // ================= half-step 1 (own rows): r = K~ v~, u' = s~ / r, row error of iterate t
-        if (tid < 4) m.flags[tid] = 0;
-        __syncthreads();
         {
             float e = 0.0f;
             for (int i = i0 + warp; i < i1; i += kNW) {
                 const float* krow = m.Ks + (i - i0) * Cn;
                 float pa = 0.0f, pb = 0.0f;
                 int j = lane;
-                for (; j + 32 < Cn; j += 64) { pa = fmaf(krow[j], m.v[j], pa); pb = fmaf(krow[j + 32], m.v[j + 32], pb); }
-                if (j < Cn) pa = fmaf(krow[j], m.v[j], pa);
+                for (; j + 32 < Cn; j += 64) { pa = fmaf(krow[j], vcur[j], pa); pb = fmaf(krow[j + 32], vcur[j + 32], pb); }
+                if (j < Cn) pa = fmaf(krow[j], vcur[j], pa);
                 float p = pa + pb;
                 for (int o = 16; o > 0; o >>= 1) p += __shfl_xor_sync(0xffffffffu, p, o);
                 if (lane == 0) {
                     if (!(p > kSumLo && p < kSumHi)) m.flags[0] = 1;
                     const float un = m.st[i] / p;
                     if (!(un > kDriftLo && un < kDriftHi)) m.flags[1] = 1;
-                    m.un[i] = un;
-                    e += fabsf(fmaf(m.u[i], p, -m.st[i]));
+                    unew[i] = un;
+                    e += fabsf(fmaf(ucur[i], p, -m.st[i]));
                 }
             }
             if (lane == 0) m.errw[warp] = e;
@@ -237,7 +242,7 @@ sinkhorn_cluster_kernel(SinkArgs a, int32_t kcap)
             // four independent accumulators over the rows (summed in a fixed order): the loop is latency-bound otherwise
             float p0 = 0.0f, p1 = 0.0f, p2 = 0.0f, p3 = 0.0f;
             const float* kc = m.Ks + j;
-            const float* ur = m.un + i0;
+            const float* ur = unew + i0;
             const int n = i1 - i0;
             int i = 0;
             for (; i + 3 < n; i += 4) {
@@ -254,6 +259,8 @@ sinkhorn_cluster_kernel(SinkArgs a, int32_t kcap)
             for (int w = 0; w < kNW; ++w) e += m.errw[w];
             xb[R] = e;
             xb[R + 1] = __int_as_float(m.flags[0] | (m.flags[1] << 1));
+            // every reader of the four flags is past the barrier above; the next writers come after the barriers below
+            m.flags[0] = 0; m.flags[1] = 0; m.flags[2] = 0; m.flags[3] = 0;
         }
         cluster.sync();
         // ================= gather: the same sums, in rank order, in every CTA
@@ -272,7 +279,7 @@ sinkhorn_cluster_kernel(SinkArgs a, int32_t kcap)
                 if (!(c > kSumLo && c < kSumHi)) m.flags[2] = 1;
                 const float vn = m.dd[j] / c;
                 if (!(vn > kDriftLo && vn < kDriftHi)) m.flags[3] = 1;
-                m.vn[j] = vn;
+                vnew[j] = vn;
             }
         }
         __syncthreads();
@@ -288,15 +295,16 @@ sinkhorn_cluster_kernel(SinkArgs a, int32_t kcap)
         // ---- commit (u', v'); fold them into (alpha, beta) if they drifted
         const bool drift = (fl & 2) != 0 || m.flags[3] != 0;
         if (drift) {
-            for (int i = i0 + tid; i < i1; i += kNT) { m.alpha[i] += log((double)m.un[i]); m.u[i] = 1.0f; }
-            for (int j = tid; j < Cn; j += kNT) { m.beta[j] += log((double)m.vn[j]); m.v[j] = 1.0f; }
+            __syncthreads();
+            for (int i = i0 + tid; i < i1; i += kNT) { m.alpha[i] += log((double)unew[i]); ucur[i] = 1.0f; unew[i] = 1.0f; }
+            for (int j = tid; j < Cn; j += kNT) { m.beta[j] += log((double)vnew[j]); vcur[j] = 1.0f; vnew[j] = 1.0f; }
             __syncthreads();
             rebuild();
+            __syncthreads();
         } else {
-            for (int i = i0 + tid; i < i1; i += kNT) m.u[i] = m.un[i];
-            for (int j = tid; j < Cn; j += kNT) m.v[j] = m.vn[j];
+            { float* x = ucur; ucur = unew; unew = x; }
+            { float* x = vcur; vcur = vnew; vnew = x; }
         }
-        __syncthreads();
         ++t;
     }
     if (handed_back) {
@@ -308,8 +316,8 @@ sinkhorn_cluster_kernel(SinkArgs a, int32_t kcap)
 
     // ---- T = diag(u) M diag(v) from the total potentials, then the column cap
     __syncthreads();
-    for (int i = i0 + tid; i < i1; i += kNT) m.alpha[i] += log((double)m.u[i]);
-    for (int j = tid; j < Cn; j += kNT) m.beta[j] += log((double)m.v[j]);
+    for (int i = i0 + tid; i < i1; i += kNT) m.alpha[i] += log((double)ucur[i]);
+    for (int j = tid; j < Cn; j += kNT) m.beta[j] += log((double)vcur[j]);
     __syncthreads();
     rebuild();
     __syncthreads();
