@@ -2,11 +2,12 @@
 // CTAs per problem.  The absorbed kernel matrix K~ (|hot| x |cold| fp32, 350 KB at 1024 ranks) is split by rows
 // over the four CTAs' shared memory, so an iteration never touches L2 or HBM:
 //   half-step 1  each CTA forms the row sums of its own rows (a warp per row) and u~ for them;
-//   half-step 2  each CTA forms the partial column sums over its rows; after one cluster barrier every CTA reads
-//                the four partials of every column through distributed shared memory, adds them in rank order
-//                (so all four get the same bits) and forms the whole v~; the row-error partials and the range
-//                flags of half-step 1 travel in the same block, double-buffered so that one barrier per iteration
-//                is enough.
+//   half-step 2  each CTA forms the partial column sums over its rows and stores them into ALL four CTAs' shared
+//                memory (remote stores through distributed shared memory: nobody waits for a round trip); after one
+//                cluster barrier every CTA adds the four partials of every column in rank order from its own
+//                copy (so all four get the same bits) and forms the whole v~; the row-error partials and the range
+//                flags of half-step 1 travel in the same blocks, double-buffered so that one barrier per
+//                iteration is enough.
 // Everything else (compaction, potentials, first iteration in the log domain) is computed redundantly and
 // identically by the four CTAs, which keeps every decision (stop, fold, hand back) uniform over the cluster.
 // A problem whose slice does not fit, or whose fp32 sums leave the safe range, is handed back (iters = -1) to the
@@ -36,7 +37,7 @@ struct CSmem {
     float* un;       // [R]
     float* v;        // [R]
     float* vn;       // [R]
-    float* xbuf;     // [2][R + kXTail] exchanged block: partial column sums, error partial, flags
+    float* xbuf;     // [2][kCluster][R + kXTail] exchange blocks, one per source CTA: partial column sums, error partial, flags
     float* errw;     // [32]
     int32_t* hot;    // [R]
     int32_t* cold;   // [R]
@@ -47,7 +48,7 @@ struct CSmem {
 
 __host__ __device__ inline size_t csmem_state_bytes(int R)
 {
-    return sizeof(double) * (3 * (size_t)R + 64) + sizeof(float) * (6 * (size_t)R + 2 * ((size_t)R + kXTail) + 32) +
+    return sizeof(double) * (3 * (size_t)R + 64) + sizeof(float) * (6 * (size_t)R + 2 * kCluster * ((size_t)R + kXTail) + 32) +
            sizeof(int32_t) * (2 * (size_t)R + 36);
 }
 
@@ -66,7 +67,7 @@ __device__ __forceinline__ CSmem ccarve(unsigned char* base, int R)
     m.un = fp; fp += R;
     m.v = fp; fp += R;
     m.vn = fp; fp += R;
-    m.xbuf = fp; fp += 2 * (R + kXTail);
+    m.xbuf = fp; fp += 2 * kCluster * (R + kXTail);
     m.errw = fp; fp += 32;
     int32_t* ip = reinterpret_cast<int32_t*>(fp);
     m.hot = ip; ip += R;
@@ -214,7 +215,10 @@ sinkhorn_cluster_kernel(SinkArgs a, int32_t kcap)
     if (tid < 4) m.flags[tid] = 0;
     __syncthreads();
     for (;;) {
-        float* xb = m.xbuf + (t & 1) * XS;
+        float* xb = m.xbuf + (t & 1) * kCluster * XS;      // this iteration's blocks: [source rank][XS], filled by the peers
+        float* xd[kCluster];                                // my block inside every CTA's copy (remote stores)
+#pragma unroll
+        for (int k = 0; k < kCluster; ++k) xd[k] = cluster.map_shared_rank(xb, k) + rank * XS;
         // ================= half-step 1 (own rows): r = K~ v~, u' = s~ / r, row error of iterate t
         {
             float e = 0.0f;
@@ -252,30 +256,32 @@ sinkhorn_cluster_kernel(SinkArgs a, int32_t kcap)
                 p3 = fmaf(kc[(i + 3) * Cn], ur[i + 3], p3);
             }
             for (; i < n; ++i) p0 = fmaf(kc[i * Cn], ur[i], p0);
-            xb[j] = (p0 + p1) + (p2 + p3);
+            const float p = (p0 + p1) + (p2 + p3);
+#pragma unroll
+            for (int k = 0; k < kCluster; ++k) xd[k][j] = p;             // pushed, so that the reads after the barrier are local
         }
-        if (tid == 0) {
-            float e = 0.0f;
-            for (int w = 0; w < kNW; ++w) e += m.errw[w];
-            xb[R] = e;
-            xb[R + 1] = __int_as_float(m.flags[0] | (m.flags[1] << 1));
-            // every reader of the four flags is past the barrier above; the next writers come after the barriers below
-            m.flags[0] = 0; m.flags[1] = 0; m.flags[2] = 0; m.flags[3] = 0;
+        if (warp == 0) {
+            float e = m.errw[lane];                                      // one partial per warp, reduced in a fixed tree
+            for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+            if (lane == 0) {
+                const float fl0 = __int_as_float(m.flags[0] | (m.flags[1] << 1));
+#pragma unroll
+                for (int k = 0; k < kCluster; ++k) { xd[k][R] = e; xd[k][R + 1] = fl0; }
+                // every reader of the four flags is past the barrier above; the next writers come after the barriers below
+                m.flags[0] = 0; m.flags[1] = 0; m.flags[2] = 0; m.flags[3] = 0;
+            }
         }
         cluster.sync();
         // ================= gather: the same sums, in rank order, in every CTA
         float err = 0.0f;
         int fl = 0;
         {
-            const float* xr[kCluster];
 #pragma unroll
-            for (int k = 0; k < kCluster; ++k) xr[k] = cluster.map_shared_rank(xb, k);
-#pragma unroll
-            for (int k = 0; k < kCluster; ++k) { err += xr[k][R]; fl |= __float_as_int(xr[k][R + 1]); }
+            for (int k = 0; k < kCluster; ++k) { err += xb[k * XS + R]; fl |= __float_as_int(xb[k * XS + R + 1]); }
             for (int j = tid; j < Cn; j += kNT) {
                 float c = 0.0f;
 #pragma unroll
-                for (int k = 0; k < kCluster; ++k) c += xr[k][j];
+                for (int k = 0; k < kCluster; ++k) c += xb[k * XS + j];
                 if (!(c > kSumLo && c < kSumHi)) m.flags[2] = 1;
                 const float vn = m.dd[j] / c;
                 if (!(vn > kDriftLo && vn < kDriftHi)) m.flags[3] = 1;
@@ -308,8 +314,7 @@ sinkhorn_cluster_kernel(SinkArgs a, int32_t kcap)
         ++t;
     }
     if (handed_back) {
-        // every CTA took this branch; none may leave while another could still read its exchange block
-        cluster.sync();
+        // every CTA took this branch in the same iteration, after the barrier that completed all remote stores
         if (rank == 0 && tid == 0) a.iters[b] = kHandBack;
         return;
     }
@@ -321,26 +326,27 @@ sinkhorn_cluster_kernel(SinkArgs a, int32_t kcap)
     __syncthreads();
     rebuild();
     __syncthreads();
-    float* xb = m.xbuf + ((t + 1) & 1) * XS;                             // the buffer the last iteration did not use
-    for (int j = tid; j < Cn; j += kNT) {
-        float cs = 0.0f;
-        for (int i = i0; i < i1; ++i) cs += m.Ks[(i - i0) * Cn + j];
-        xb[j] = cs;
+    float* xb = m.xbuf + ((t + 1) & 1) * kCluster * XS;                  // the blocks the last iteration did not use
+    {
+        float* xd[kCluster];
+#pragma unroll
+        for (int k = 0; k < kCluster; ++k) xd[k] = cluster.map_shared_rank(xb, k) + rank * XS;
+        for (int j = tid; j < Cn; j += kNT) {
+            float cs = 0.0f;
+            for (int i = i0; i < i1; ++i) cs += m.Ks[(i - i0) * Cn + j];
+#pragma unroll
+            for (int k = 0; k < kCluster; ++k) xd[k][j] = cs;
+        }
     }
     // zero the R x R block (shared between the CTAs) before anyone writes entries into it
     for (int64_t q = (int64_t)rank * kNT + tid; q < (int64_t)R * R; q += (int64_t)kCluster * kNT) out[q] = 0.0f;
     __threadfence();
     cluster.sync();
-    {
-        const float* xr[kCluster];
+    for (int j = tid; j < Cn; j += kNT) {
+        double cs = 0.0;
 #pragma unroll
-        for (int k = 0; k < kCluster; ++k) xr[k] = cluster.map_shared_rank(xb, k);
-        for (int j = tid; j < Cn; j += kNT) {
-            double cs = 0.0;
-#pragma unroll
-            for (int k = 0; k < kCluster; ++k) cs += (double)xr[k][j];
-            m.vn[j] = (float)fmin(1.0, (double)m.dd[j] / (cs + (double)a.eps0));
-        }
+        for (int k = 0; k < kCluster; ++k) cs += (double)xb[k * XS + j];
+        m.vn[j] = (float)fmin(1.0, (double)m.dd[j] / (cs + (double)a.eps0));
     }
     __syncthreads();
     int nonfinite = 0;
@@ -355,7 +361,6 @@ sinkhorn_cluster_kernel(SinkArgs a, int32_t kcap)
     }
     nonfinite = __syncthreads_or(nonfinite);
     if (nonfinite && tid == 0) atomicOr(a.info + b, TAOT_INFO_NONFINITE);
-    cluster.sync();                                                      // remote reads of xb are done before any CTA exits
     if (rank == 0 && tid == 0) {
         a.iters[b] = t;
         a.row_err[b] = err_out;
