@@ -27,5 +27,6 @@ from .binding import (  # noqa: F401
     ReportRow,
     measure_alu_peaks,
     PipelinedHostPlanner,
+    split_layers,
 )
 from .report import format_layer  # noqa: F401

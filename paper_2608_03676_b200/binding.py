@@ -362,6 +362,18 @@ class Planner:
         return out_host
 
 
+def split_layers(L: int, groups: int):
+    """Contiguous, near-equal split of L layers into at most `groups` non-empty groups: [(lo, hi), ...]."""
+    groups = max(1, min(groups, L))
+    base, extra = divmod(L, groups)
+    bounds, lo = [], 0
+    for g in range(groups):
+        hi = lo + base + (1 if g < extra else 0)
+        bounds.append((lo, hi))
+        lo = hi
+    return bounds
+
+
 class PipelinedHostPlanner:
     """`taot_plan_host` over groups of layers on separate streams, so that the host-to-device copy of one group,
     the kernels of another and the device-to-host copy of a third overlap (the L problems of a call are
@@ -369,14 +381,7 @@ class PipelinedHostPlanner:
     group; `plan_host` enqueues every group and makes the caller's current stream wait for all of them."""
 
     def __init__(self, L: int, groups: int = 4, **planner_kwargs):
-        groups = max(1, min(groups, L))
-        base, extra = divmod(L, groups)
-        self.bounds = []
-        lo = 0
-        for g in range(groups):
-            hi = lo + base + (1 if g < extra else 0)
-            self.bounds.append((lo, hi))
-            lo = hi
+        self.bounds = split_layers(L, groups)
         self.planners = [Planner(L=hi - lo, **planner_kwargs) for lo, hi in self.bounds]
         self.streams = [torch.cuda.Stream() for _ in self.planners]
         self.L = L
