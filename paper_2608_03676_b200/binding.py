@@ -385,6 +385,7 @@ class PipelinedHostPlanner:
         self.planners = [Planner(L=hi - lo, **planner_kwargs) for lo, hi in self.bounds]
         self.streams = [torch.cuda.Stream() for _ in self.planners]
         self.L = L
+        self._key, self._calls, self._held = None, [], None
 
     def alloc_host_outputs(self, names=("plan", "slot_expert", "slot_tokens", "X", "new_idx", "info")):
         parts = [p.alloc_host_outputs(names) for p in self.planners]
@@ -396,11 +397,23 @@ class PipelinedHostPlanner:
         return out
 
     def plan_host(self, topk_host: torch.Tensor, out_host: Dict[str, torch.Tensor]) -> Dict[str, torch.Tensor]:
+        if topk_host.is_cuda or topk_host.dtype != torch.int32 or not topk_host.is_contiguous():
+            raise TaotError("topk_host: expected a contiguous CPU int32 tensor")
+        # the per-group argument blocks depend only on the buffers' addresses: marshal them once per buffer set
+        key = (topk_host.data_ptr(),) + tuple((k, v.data_ptr()) for k, v in sorted(out_host.items()))
+        if key != self._key:
+            calls = []
+            for (lo, hi), pl in zip(self.bounds, self.planners):
+                if pl._host_ws is None:
+                    pl._host_ws = torch.empty(pl.host_ws_bytes, dtype=torch.uint8, device=pl.device)
+                o = pl._outputs_struct({k: v[lo:hi] for k, v in out_host.items()})
+                calls.append((pl, _ptr(topk_host[lo:hi]), o, _ptr(pl._host_ws)))
+            self._calls, self._key, self._held = calls, key, (topk_host, out_host)
         cur = torch.cuda.current_stream()
-        for (lo, hi), pl, st in zip(self.bounds, self.planners, self.streams):
+        fn = self.planners[0].lib.taot_plan_host
+        for (pl, tp, o, ws), st in zip(self._calls, self.streams):
             st.wait_stream(cur)
-            with torch.cuda.stream(st):
-                pl.plan_host(topk_host[lo:hi], {k: v[lo:hi] for k, v in out_host.items()})
+            _check(fn(pl.handle, tp, ctypes.byref(o), ws, ctypes.c_void_p(st.cuda_stream)), "taot_plan_host")
         for st in self.streams:
             cur.wait_stream(st)
         return out_host
