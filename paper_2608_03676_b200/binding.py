@@ -116,6 +116,8 @@ STATIC_SCRATCH_BYTES = 4 << 20
 # without a split, rewrite of the chunks with one) -- for a 16-byte aligned routing table with E % 4 == 0
 PLAN_LAUNCHES = 8
 PLAN_LAUNCHES_NO_HINT = 6       # with ABLATE_HINT the two Sinkhorn kernels are not launched
+# A routing table of at most 3 x (number of SMs) chunks is rewritten by the per-chunk kernel alone: one launch fewer
+# (`Planner.plan_launches()` gives the count for a handle).
 
 
 def histogram_static(topk: torch.Tensor, R: int, E: int, e2r_dev: torch.Tensor, n: torch.Tensor,
@@ -215,6 +217,14 @@ class Planner:
             slot_expert=self._empty((L, R, K), i32), slot_tokens=self._empty((L, R, K), i32),
             X=self._empty((L, R, S), i32), rounds=self._empty((L, 2), i32), new_idx=self._empty((L, T, k), i32),
             info=torch.zeros((L,), dtype=i32, device=self.device))
+
+    def plan_launches(self) -> int:
+        """Kernels one `plan` call of this handle enqueues (16-byte aligned routing table, E % 4 == 0)."""
+        sms = torch.cuda.get_device_properties(self.device).multi_processor_count
+        seg = self.T // self.R * self.k
+        chunks = self.L * self.R * ((seg + 16383) // 16384)
+        n = PLAN_LAUNCHES_NO_HINT if (self.ablation & ABLATE_HINT) else PLAN_LAUNCHES
+        return n - 1 if chunks <= 3 * sms else n
 
     def last_launch_count(self) -> int:
         c = ctypes.c_int32()
@@ -420,6 +430,9 @@ class PipelinedHostPlanner:
 
     def launch_count(self) -> int:
         return sum(p.last_launch_count() for p in self.planners)
+
+    def plan_launches(self) -> int:
+        return sum(p.plan_launches() for p in self.planners)
 
     def close(self):
         for p in self.planners:

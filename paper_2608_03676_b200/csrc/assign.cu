@@ -619,7 +619,15 @@ int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, void* ws, const i
     TAOT_CUDA_OK(cudaGetLastError());
     const StreamLayout sl = stream_layout(p.E);
     int launches = 2;
-    if (vec_ok && p.E % 4 == 0 && sl.stages >= 2) {
+    // A routing table whose chunks all fit one wave of the per-chunk kernel (three CTAs per SM) is latency-bound, not
+    // bandwidth-bound: the pipelined kernel would only add a launch, so the staged per-chunk kernel takes every chunk.
+    const bool one_wave = blocks <= 3u * (unsigned)h->sm_count;
+    if (vec_ok && one_wave) {
+        const size_t smem = (size_t)TAOT_CHUNK * 4 + sizeof(int32_t) * (((size_t)p.E + kRowTail + 3) & ~(size_t)3) +
+                            sizeof(int4) * (size_t)(S + kRowSplits);
+        TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        assign_chunk_kernel<true, true><<<blocks, kThreads, smem, st>>>(a, 0);
+    } else if (vec_ok && p.E % 4 == 0 && sl.stages >= 2) {
         TAOT_CUDA_OK(cudaFuncSetAttribute(assign_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sl.bytes));
         const unsigned grid = blocks < (unsigned)h->sm_count ? blocks : (unsigned)h->sm_count;
         assign_stream_kernel<<<grid, kStreamThreads, sl.bytes, st>>>(a, sl.stages, (uint32_t)sl.off_tab, (int64_t)blocks, a.work);
