@@ -180,3 +180,65 @@ def test_handle_validation_and_null_arguments_return_status_codes():
     with pytest.raises(P.TaotError):
         pl.histogram(topk.cpu())                        # host tensor where device memory is required
     pl.close()
+
+
+def test_many_quota_boundaries_inside_one_chunk():
+    """A hand-made schedule in which ten guest slots hold the same expert and every source rank feeds each of
+    them a few tokens: ten quota intervals end inside the single chunk of a segment, more than the four split
+    records a table row carries, so the rewrite walks the overflow list.  Checked through taot_assign alone."""
+    cfg = W.get_config("cfg1").replace(L=2, R=8, E=8, K=4, k=2, T=8 * 4096)
+    e2r, _ = topology(cfg)
+    topk = W.routing_topk(cfg, device="cuda")
+    pl = make_planner(cfg)
+    n, el, rl, _ = pl.histogram(topk)
+    n_h = cpu(n)
+    S = cfg.S
+    slot_expert = np.full((cfg.L, S), -1, np.int32)
+    X = np.zeros((cfg.L, cfg.R, S), np.int32)
+    for l in range(cfg.L):
+        e0 = int(np.argmax(n_h[l].sum(0)))                               # the busiest expert of the layer
+        slots = [s for s in range(S) if s // cfg.K != e2r[e0]][:10]
+        for q, s in enumerate(slots):
+            slot_expert[l, s] = e0
+            for r in range(cfg.R):
+                X[l, r, s] = min(3 + (q + r) % 5, max(0, int(n_h[l, r, e0]) // 12))
+        other = int(np.argsort(n_h[l].sum(0))[-2])                       # and one slot for the runner-up
+        s2 = [s for s in range(S) if slot_expert[l, s] < 0 and s // cfg.K != e2r[other]][0]
+        slot_expert[l, s2] = other
+        X[l, :, s2] = np.minimum(n_h[l, :, other] // 3, 50)
+    se_d = torch.from_numpy(slot_expert.reshape(cfg.L, cfg.R, cfg.K)).cuda()
+    X_d = torch.from_numpy(X).cuda()
+    for reuse in (True, False):
+        if reuse:
+            pl.histogram(topk)
+        new, info = pl.assign(topk, se_d, X_d, reuse_counts=reuse)
+        torch.cuda.synchronize()
+        assert (cpu(info) == 0).all()
+        for l in range(cfg.L):
+            want = O.assign(cpu(topk)[l], cfg.R, cfg.E, cfg.K, slot_expert[l], X[l])
+            assert (cpu(new)[l] == want).all()
+            assert int((want >= cfg.E).sum()) == int(X[l].sum())
+    pl.close()
+
+
+def test_largest_supported_dimensions():
+    """E = 1024 experts, K = 8 slots per rank, top-64 routing (the documented maxima) on 64 ranks: every stage,
+    the report and the dispatch metadata against the oracle."""
+    cfg = W.get_config("cfg1").replace(L=1, R=64, E=1024, K=8, k=64, T=64 * 96, gpus_per_node=8,
+                                       tiers=(0.0, 1.0, 4.0), zipf=(1.1, 1.1))
+    topk = W.routing_topk(cfg, device="cuda")
+    pl = make_planner(cfg, max_iters=300, tol=1e-6)
+    out = _full_check(cfg, topk, pl)
+    assert out["X"].sum() > 0
+    pl.close()
+
+
+def test_most_slots_256_ranks_by_8_slots():
+    """S = 2048 guest slots (256 ranks x 8): more slots than the one-thread-per-slot auction holds, so Phase 3 takes
+    the dense scan; the whole path, the report and the dispatch metadata against the oracle."""
+    cfg = W.get_config("cfg4").replace(L=1, E=512, K=8, k=8, T=256 * 64, e2r_mode="contiguous", zipf=(1.3, 1.3))
+    topk = W.routing_topk(cfg, device="cuda")
+    pl = make_planner(cfg, max_iters=200, tol=1e-6)
+    out = _full_check(cfg, topk, pl)
+    assert out["X"].sum() > 0
+    pl.close()
