@@ -242,3 +242,21 @@ def test_most_slots_256_ranks_by_8_slots():
     out = _full_check(cfg, topk, pl)
     assert out["X"].sum() > 0
     pl.close()
+
+
+def test_smallest_table_and_everything_on_one_expert():
+    """One token per rank with top-1 routing (the smallest table the API accepts), and a layer in which every
+    entry names the same expert (one rank holds the whole load, its other experts none)."""
+    cfg = W.get_config("cfg1").replace(L=2, R=8, E=32, K=2, k=1, T=8)
+    topk = W.routing_topk(cfg, device="cuda")
+    pl = make_planner(cfg, max_iters=100, tol=0.0)
+    _full_check(cfg, topk, pl)
+    pl.close()
+    cfg = W.get_config("cfg1").replace(L=2, k=2, T=8 * 640)
+    topk = W.routing_topk(cfg, device="cuda")
+    topk[0, :, 0] = 5                          # layer 0: first choice always expert 5 ...
+    topk[0, :, 1] = 5                          # ... and the second too (duplicates inside a token are legal input)
+    pl = make_planner(cfg, max_iters=200, tol=1e-6)
+    out = _full_check(cfg, topk, pl)
+    assert out["rank_load"][0].max() == cfg.T * cfg.k and (out["slot_expert"][0] >= 0).sum() > 0
+    pl.close()
