@@ -25,17 +25,20 @@ __device__ __forceinline__ int4 ld_stream(const int4* p)
     return v;
 }
 
-// nb == E: out-of-range values are only flagged; nb == E + 1: they are also counted, in bin E
-__device__ __forceinline__ void count_one(int32_t* hist, int32_t e, int32_t E, int32_t nb, int& bad)
+// EXTRA == false: out-of-range values are only flagged; true: they are also counted, in bin E (rows of E + 1 bins)
+template <bool EXTRA>
+__device__ __forceinline__ void count_one(int32_t* hist, int32_t e, int32_t E, int& bad)
 {
     if ((uint32_t)e < (uint32_t)E) atomicAdd(hist + e, 1);
-    else { bad = 1; if (nb > E) atomicAdd(hist + E, 1); }
+    else { bad = 1; if (EXTRA) atomicAdd(hist + E, 1); }
 }
 
+template <bool EXTRA>
 __global__ void __launch_bounds__(kThreads)
 hist_chunk_kernel(const int32_t* __restrict__ topk, int32_t* __restrict__ cc, int32_t* __restrict__ info,
-                  int64_t layer_elems, int64_t seg, int32_t nc, int32_t R, int32_t E, int32_t nb, int vec_ok)
+                  int64_t layer_elems, int64_t seg, int32_t nc, int32_t R, int32_t E, int vec_ok)
 {
+    const int32_t nb = EXTRA ? E + 1 : E;
     extern __shared__ int32_t sh_hist[];                 // [kWarps][nb]
     const int tid = threadIdx.x, warp = tid >> 5;
     const int64_t id = blockIdx.x;
@@ -63,18 +66,18 @@ hist_chunk_kernel(const int32_t* __restrict__ topk, int32_t* __restrict__ cc, in
             for (int u = 0; u < 8; ++u) x[u] = ld_stream(src4 + v + u * kThreads);
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-                count_one(hist, x[u].x, E, nb, bad); count_one(hist, x[u].y, E, nb, bad);
-                count_one(hist, x[u].z, E, nb, bad); count_one(hist, x[u].w, E, nb, bad);
+                count_one<EXTRA>(hist, x[u].x, E, bad); count_one<EXTRA>(hist, x[u].y, E, bad);
+                count_one<EXTRA>(hist, x[u].z, E, bad); count_one<EXTRA>(hist, x[u].w, E, bad);
             }
         }
         for (; v < nvec; v += kThreads) {
             const int4 x = ld_stream(src4 + v);
-            count_one(hist, x.x, E, nb, bad); count_one(hist, x.y, E, nb, bad);
-            count_one(hist, x.z, E, nb, bad); count_one(hist, x.w, E, nb, bad);
+            count_one<EXTRA>(hist, x.x, E, bad); count_one<EXTRA>(hist, x.y, E, bad);
+            count_one<EXTRA>(hist, x.z, E, bad); count_one<EXTRA>(hist, x.w, E, bad);
         }
-        for (int32_t i = (nvec << 2) + tid; i < len; i += kThreads) count_one(hist, src[i], E, nb, bad);
+        for (int32_t i = (nvec << 2) + tid; i < len; i += kThreads) count_one<EXTRA>(hist, src[i], E, bad);
     } else {
-        for (int32_t i = tid; i < len; i += kThreads) count_one(hist, src[i], E, nb, bad);
+        for (int32_t i = tid; i < len; i += kThreads) count_one<EXTRA>(hist, src[i], E, bad);
     }
     const int any_bad = __syncthreads_or(bad);
     int32_t* out = cc + id * nb;
@@ -167,8 +170,8 @@ int taot_launch_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_cc,
     const int64_t blocks = (int64_t)p.L * p.R * h->nc;
     const int vec_ok = ((reinterpret_cast<uintptr_t>(d_topk) & 15) == 0) && (h->seg % 4 == 0);
     const size_t smem = sizeof(int32_t) * kWarps * p.E;
-    hist_chunk_kernel<<<(unsigned)blocks, kThreads, smem, st>>>(d_topk, d_cc, d_info, layer_elems, h->seg,
-                                                                 h->nc, p.R, p.E, p.E, vec_ok);
+    hist_chunk_kernel<false><<<(unsigned)blocks, kThreads, smem, st>>>(d_topk, d_cc, d_info, layer_elems, h->seg,
+                                                                        h->nc, p.R, p.E, vec_ok);
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
 }
@@ -182,11 +185,11 @@ int taot_launch_chunk_counts(taot_handle_t h, const int32_t* d_idx, int32_t* d_c
     const int64_t blocks = (int64_t)p.L * p.R * h->nc;
     const int vec_ok = ((reinterpret_cast<uintptr_t>(d_idx) & 15) == 0) && (h->seg % 4 == 0);
     const size_t smem = sizeof(int32_t) * kWarps * (size_t)(bins + 1);
-    // only ever raise the limit: the load-collection launch above relies on the default 48 KB
+    // the default limit is 48 KB
     if (smem > 48 * 1024)
-        TAOT_CUDA_OK(cudaFuncSetAttribute(hist_chunk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    hist_chunk_kernel<<<(unsigned)blocks, kThreads, smem, st>>>(d_idx, d_counts, d_info, p.T * p.k, h->seg, h->nc,
-                                                                 p.R, bins, bins + 1, vec_ok);
+        TAOT_CUDA_OK(cudaFuncSetAttribute(hist_chunk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    hist_chunk_kernel<true><<<(unsigned)blocks, kThreads, smem, st>>>(d_idx, d_counts, d_info, p.T * p.k, h->seg, h->nc,
+                                                                       p.R, bins, vec_ok);
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
 }
