@@ -56,6 +56,9 @@ def parse_args():
     ap.add_argument("--no-streams", action="store_true", help="skip the HBM-sized streaming report")
     ap.add_argument("--sweep", action="store_true",
                     help="config 5: time taot_sinkhorn alone over the (B, R, eps) grid and print one JSON object")
+    ap.add_argument("--sweep-batches", type=int, nargs="+", default=[1, 64, 1024, 4096], help="batch sizes of --sweep")
+    ap.add_argument("--sweep-ranks", type=int, nargs="+", default=[8, 16, 64, 256, 1024], help="rank counts of --sweep")
+    ap.add_argument("--sweep-eps", type=float, nargs="+", default=[0.1, 0.01], help="eps / max(C) values of --sweep")
     ap.add_argument("--sweep-max-elems", type=float, default=6e9,
                     help="skip sweep cells whose plan tensor would exceed this many floats")
     return ap.parse_args()
@@ -484,7 +487,9 @@ def run_sweep(args):
     alu = P.measure_alu_peaks()
     fp32_peak = alu["fma_tflops"]                    # measured FMA-chain throughput of this GPU
     cells = []
-    for (B, R, eps_frac) in W.sweep_cells():
+    cells_todo = W.sweep_cells(batches=tuple(args.sweep_batches), ranks=tuple(args.sweep_ranks),
+                               eps_fracs=tuple(args.sweep_eps))
+    for (B, R, eps_frac) in cells_todo:
         if B * R * R > args.sweep_max_elems:
             cells.append(dict(B=B, R=R, eps_frac=eps_frac, skipped="plan tensor larger than --sweep-max-elems"))
             continue
