@@ -53,6 +53,10 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-groups", type=int, default=4,
                     help="layer groups (streams) the end-to-end host call is pipelined over")
+    ap.add_argument("--e2e-depth", type=int, default=3,
+                    help="host calls in flight in the end-to-end measurement")
+    ap.add_argument("--e2e-stream-groups", type=int, default=1,
+                    help="layer groups per call when several calls are in flight")
     ap.add_argument("--no-streams", action="store_true", help="skip the HBM-sized streaming report")
     ap.add_argument("--sweep", action="store_true",
                     help="config 5: time taot_sinkhorn alone over the (B, R, eps) grid and print one JSON object")
@@ -408,15 +412,44 @@ def run_ours(args):
     host_in = topk.cpu().pin_memory()
     e2r_h = W.expert_to_rank(cfg.E, cfg.R, cfg.e2r_mode)
     C_h = W.cost_matrix(cfg.R, cfg.gpus_per_node, cfg.tiers, cfg.nodes_per_group)
-    hp = P.PipelinedHostPlanner(L=cfg.L, groups=args.e2e_groups, R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k, T=cfg.T,
-                                e2r=e2r_h, C=C_h, eps=cfg.eps, max_iters=cfg.max_iters, tol=cfg.tol)
-    host_out = hp.alloc_host_outputs(("plan", "slot_expert", "slot_tokens", "X", "new_idx", "info"))
+    depth = max(1, args.e2e_depth)
+    kw = dict(R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k, T=cfg.T, e2r=e2r_h, C=C_h, eps=cfg.eps, max_iters=cfg.max_iters,
+              tol=cfg.tol)
+    names = ("plan", "slot_expert", "slot_tokens", "X", "new_idx", "info")
+    # (a) one call at a time, pipelined over groups of layers inside the call: every step waits for the previous one
+    hp = P.PipelinedHostPlanner(L=cfg.L, groups=args.e2e_groups, **kw)
+    host_out = hp.alloc_host_outputs(names)
     d2h = sum(t.numel() * t.element_size() for t in host_out.values())
     e2e_step = lambda: hp.plan_host(host_in, host_out)
     timed_steps(e2e_step, 3, flush)
     barrier(); torch.cuda.synchronize()
-    e2e_ms = timed_steps(e2e_step, args.steps, flush)
-    e2e_value = whole_job_rate(cfg.L, args.steps, world, max_over_ranks(sum(e2e_ms), world, "cuda"))
+    serial_ms = timed_steps(e2e_step, args.steps, flush)
+    serial_value = whole_job_rate(cfg.L, args.steps, world, max_over_ranks(sum(serial_ms), world, "cuda"))
+    n_groups = len(hp.planners)
+    hp.close(); del host_out
+    sp = P.StreamingHostPlanner(L=cfg.L, depth=depth, groups=args.e2e_stream_groups, **kw)
+    host_outs = sp.alloc_host_outputs(names)
+
+    # (b) `depth` calls in flight: step i starts once step i - depth has delivered its outputs (and L2 has been
+    # flushed after that), while the steps between them are still copying and computing
+    def streamed(steps):
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(steps):
+            sp.wait_lane(i % depth)
+            if flush is not None:
+                flush.zero_()
+            sp.submit(host_in, host_outs[i % depth])
+        sp.join()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b)
+
+    streamed(3 * depth)
+    barrier(); torch.cuda.synchronize()
+    e2e_total_ms = streamed(args.steps)
+    e2e_ms = [e2e_total_ms / args.steps]
+    e2e_value = whole_job_rate(cfg.L, args.steps, world, max_over_ranks(e2e_total_ms, world, "cuda"))
 
     if rank != 0:
         if world > 1:
@@ -448,8 +481,11 @@ def run_ours(args):
         rounds=dict(phase2_max=int(rounds[:, 0].max()), phase3_max=int(rounds[:, 1].max())),
         roofline=roof, clocks=clocks,
         e2e=dict(value=e2e_value, unit="plans/s", h2d_bytes_per_step=topk_bytes, d2h_bytes_per_step=d2h,
-                 ms_per_step=float(np.mean(e2e_ms)),
-                 api=f"PipelinedHostPlanner.plan_host: taot_plan_host on {len(hp.planners)} groups of layers, one stream each"),
+                 ms_per_step=float(np.mean(e2e_ms)), in_flight=depth,
+                 serial_value=serial_value, serial_ms_per_step=float(np.mean(serial_ms)),
+                 api=f"StreamingHostPlanner.submit: taot_plan_host, {depth} call(s) in flight, each on "
+                     f"{len(sp.lanes[0].planners)} group(s) of layers; serial_*: PipelinedHostPlanner.plan_host, one "
+                     f"call at a time on {n_groups} groups of layers (one stream each)"),
         gpu_launches=launches,
     )
     if dispatch is not None:

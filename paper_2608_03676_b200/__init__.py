@@ -27,6 +27,7 @@ from .binding import (  # noqa: F401
     ReportRow,
     measure_alu_peaks,
     PipelinedHostPlanner,
+    StreamingHostPlanner,
     split_layers,
 )
 from .report import format_layer  # noqa: F401

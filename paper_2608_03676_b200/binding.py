@@ -406,7 +406,7 @@ class PipelinedHostPlanner:
             out[nm] = torch.empty(shape, dtype=parts[0][nm].dtype).pin_memory()
         return out
 
-    def plan_host(self, topk_host: torch.Tensor, out_host: Dict[str, torch.Tensor]) -> Dict[str, torch.Tensor]:
+    def plan_host(self, topk_host: torch.Tensor, out_host: Dict[str, torch.Tensor], join: bool = True) -> Dict[str, torch.Tensor]:
         if topk_host.is_cuda or topk_host.dtype != torch.int32 or not topk_host.is_contiguous():
             raise TaotError("topk_host: expected a contiguous CPU int32 tensor")
         # the per-group argument blocks depend only on the buffers' addresses: marshal them once per buffer set
@@ -424,9 +424,15 @@ class PipelinedHostPlanner:
         for (pl, tp, o, ws), st in zip(self._calls, self.streams):
             st.wait_stream(cur)
             _check(fn(pl.handle, tp, ctypes.byref(o), ws, ctypes.c_void_p(st.cuda_stream)), "taot_plan_host")
+        if join:
+            self.join()
+        return out_host
+
+    def join(self):
+        """Make the caller's current stream wait for everything enqueued on the group streams."""
+        cur = torch.cuda.current_stream()
         for st in self.streams:
             cur.wait_stream(st)
-        return out_host
 
     def launch_count(self) -> int:
         return sum(p.last_launch_count() for p in self.planners)
@@ -437,3 +443,72 @@ class PipelinedHostPlanner:
     def close(self):
         for p in self.planners:
             p.close()
+
+
+class StreamingHostPlanner:
+    """Several `taot_plan_host` calls in flight: `depth` pipelined planners (each with its own handles, workspaces,
+    staging buffers and streams) take the submitted steps in turn, so that the copies of one step overlap the
+    kernels of the previous one.  `submit` only enqueues; `result` blocks the host until that step's outputs are in
+    host memory.  A lane is reused only after its previous step has finished (the submitting stream waits for it),
+    so a caller must read a step's outputs before it submits `depth` further steps into the same output buffers."""
+
+    def __init__(self, L: int, depth: int = 2, groups: int = 4, **planner_kwargs):
+        if depth < 1:
+            raise TaotError("depth must be at least 1")
+        self.lanes = [PipelinedHostPlanner(L=L, groups=groups, **planner_kwargs) for _ in range(depth)]
+        self.depth = depth
+        self.L = L
+        self._done = [torch.cuda.Event() for _ in range(depth)]
+        self._busy = [False] * depth
+        self._outs = [None] * depth
+        self._n = 0
+
+    def alloc_host_outputs(self, names=("plan", "slot_expert", "slot_tokens", "X", "new_idx", "info")):
+        """One pinned output set per lane."""
+        return [lane.alloc_host_outputs(names) for lane in self.lanes]
+
+    def submit(self, topk_host: torch.Tensor, out_host: Dict[str, torch.Tensor]) -> int:
+        """Enqueue one step; returns its ticket.  The current stream first waits for the lane's previous step."""
+        lane = self._n % self.depth
+        cur = torch.cuda.current_stream()
+        if self._busy[lane]:
+            cur.wait_event(self._done[lane])
+        pl = self.lanes[lane]
+        pl.plan_host(topk_host, out_host, join=False)
+        # the lane's completion: an event on its first stream after that stream has waited for the others
+        first = pl.streams[0]
+        for st in pl.streams[1:]:
+            first.wait_stream(st)
+        self._done[lane].record(first)
+        self._busy[lane] = True
+        self._outs[lane] = out_host
+        self._n += 1
+        return self._n - 1
+
+    def lane_of(self, ticket: int) -> int:
+        return ticket % self.depth
+
+    def wait_lane(self, lane: int):
+        """Make the current stream wait for the step last submitted to this lane."""
+        if self._busy[lane]:
+            torch.cuda.current_stream().wait_event(self._done[lane])
+
+    def result(self, ticket: int) -> Dict[str, torch.Tensor]:
+        """Block the host until the step is complete; its outputs (valid until the lane's next submit)."""
+        if ticket < self._n - self.depth or ticket >= self._n:
+            raise TaotError("ticket is not in flight")
+        lane = ticket % self.depth
+        self._done[lane].synchronize()
+        return self._outs[lane]
+
+    def join(self):
+        """Make the current stream wait for every step in flight."""
+        for lane in range(self.depth):
+            self.wait_lane(lane)
+
+    def launch_count(self) -> int:
+        return sum(l.launch_count() for l in self.lanes)
+
+    def close(self):
+        for l in self.lanes:
+            l.close()

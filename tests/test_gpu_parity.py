@@ -250,3 +250,35 @@ def test_pipelined_host_planner_equals_the_single_call():
             assert (host_out[key].numpy() == want[key]).all(), key
     assert hp.launch_count() == hp.plan_launches() == 3 * (P.PLAN_LAUNCHES - 1)
     hp.close(); pl.close()
+
+
+def test_streaming_host_planner_keeps_steps_apart():
+    """Two host calls in flight on alternating inputs: every step's outputs are those of a lone call on its input."""
+    import paper_2608_03676_b200 as P
+    cfg = W.get_config("cfg2").replace(L=5)
+    e2r, C = topology(cfg)
+    pl = make_planner(cfg)
+    inputs = [_routing(cfg.replace(seed=cfg.seed + i)) for i in range(3)]
+    names = ("n", "plan", "sinkhorn_iters", "slot_expert", "slot_tokens", "X", "new_idx", "info", "rounds")
+    want = [{k: cpu(v).copy() for k, v in pl.plan(t).items()} for t in inputs]
+    assert (want[0]["new_idx"] != want[1]["new_idx"]).any()
+    sp = P.StreamingHostPlanner(L=cfg.L, depth=2, groups=2, R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k, T=cfg.T, e2r=e2r,
+                                C=C, eps=cfg.eps, max_iters=cfg.max_iters, tol=cfg.tol)
+    outs = sp.alloc_host_outputs(names)
+    host_in = [t.cpu().pin_memory() for t in inputs]
+    tickets = []
+    for step in range(7):
+        which = step % 3
+        if step >= 2:                                   # read the step that used this lane before submitting into it
+            got = sp.result(tickets[step - 2][0])
+            ref = want[tickets[step - 2][1]]
+            for key in names:
+                assert (got[key].numpy() == ref[key]).all(), (step, key)
+        tickets.append((sp.submit(host_in[which], outs[step % 2]), which))
+    for t, which in tickets[-2:]:
+        got = sp.result(t)
+        for key in names:
+            assert (got[key].numpy() == want[which][key]).all(), (t, key)
+    with pytest.raises(P.TaotError):
+        sp.result(0)
+    sp.close(); pl.close()
