@@ -220,6 +220,23 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
         }
     }
     h->nbid = (int32_t)bidlist.size();
+    // a cost that depends only on "same node of 8 ranks / same rail group of 32 ranks / neither" lets the Sinkhorn
+    // sums be taken tier by tier (sinkhorn_tiered.cu)
+    h->tier_ok = 0;
+    if (R == 256 || R == 512 || R == 1024) {
+        const float c1 = h_C[1], c2 = h_C[8], c3 = h_C[32];
+        bool ok = std::isfinite(c1) && std::isfinite(c2) && std::isfinite(c3);
+        for (int i = 0; i < R && ok; ++i)
+            for (int j = 0; j < R && ok; ++j) {
+                if (i == j) continue;
+                const float want = (i / 8 == j / 8) ? c1 : ((i / 32 == j / 32) ? c2 : c3);
+                ok = h_C[(size_t)i * R + j] == want;
+            }
+        if (ok) {
+            h->tier_ok = 1;
+            h->tier_cost[0] = c1; h->tier_cost[1] = c2; h->tier_cost[2] = c3;
+        }
+    }
     // first Sinkhorn row update with v = 1 on every rank: log-sum-exp of -C_ij/eps over all j
     std::vector<double> lse0(R);
     for (int i = 0; i < R; ++i) {

@@ -335,6 +335,7 @@ __global__ void __launch_bounds__(1024) sinkhorn_kernel(SinkArgs a)
 
 int taot_launch_sinkhorn_tile(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st);
 int taot_launch_sinkhorn_cluster(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st);
+int taot_launch_sinkhorn_tiered(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st);
 
 int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
                          int32_t* d_iters, float* d_row_err, int32_t* d_info, float* d_kt, cudaStream_t st)
@@ -360,7 +361,13 @@ int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, in
         a.s = d_s + (int64_t)b0 * p.R; a.d = d_d + (int64_t)b0 * p.R;
         a.plan = d_plan + (int64_t)b0 * p.R * p.R; a.iters = d_iters + b0; a.row_err = d_row_err + b0;
         a.info = d_info + b0;
-        if (p.R <= 256) {
+        const int nt = taot_launch_sinkhorn_tiered(h, a, nb, st);
+        if (nt < 0) return nt;
+        if (nt > 0) {
+            // tiered cost: O(R) sums per half-step, one warp per problem; what it hands back goes to the kernel below
+            launched += nt;
+            a.only_marked = 1;
+        } else if (p.R <= 256) {
             // fast path: kernel matrix in registers; problems it cannot hold (or whose fp32 sums leave the
             // safe range) come back marked and are solved by the shared-memory kernel below
             a.only_marked = 1;

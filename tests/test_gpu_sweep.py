@@ -12,21 +12,33 @@ from helpers import check_sinkhorn_problem, cpu
 pytestmark = pytest.mark.gpu
 
 
-def _planner(B, R, eps_frac, iters=SWEEP_ITERS, tol=0.0):
+def _planner(B, R, eps_frac, iters=SWEEP_ITERS, tol=0.0, general=False):
+    """general: a few entries of the tiered cost are raised, so that it no longer depends on the tier alone and the
+    solve takes the kernels that hold the kernel matrix itself (register tiles, clusters, workspace) instead of the
+    tier-by-tier sums."""
     import paper_2608_03676_b200 as P
     C = W.cost_matrix(R, 8, SWEEP_TIERS, 4)
+    if general:
+        i = torch.arange(R)
+        bump = ((i[:, None] * 5 + i[None, :] * 3) % 11 == 0) & (i[:, None] != i[None, :])
+        C = C + 0.25 * bump.to(C.dtype)
     e2r = torch.arange(R, dtype=torch.int32)
     pl = P.Planner(L=B, R=R, E=R, K=1, k=1, T=R, e2r=e2r, C=C, eps=eps_frac * max(SWEEP_TIERS),
                    max_iters=iters, tol=tol)
     return pl, C
 
 
-@pytest.mark.parametrize("R,B,check", [(8, 64, 64), (16, 64, 64), (64, 64, 16), (256, 64, 4), (1024, 3, 1),
-                                       # batches of at least 4 x 148 problems take the batch builds of the kernels
-                                       (16, 1024, 8), (64, 1024, 6), (256, 640, 3)])
+@pytest.mark.parametrize("R,B,check,general", [
+    (8, 64, 64, False), (16, 64, 64, False), (64, 64, 16, False), (256, 64, 4, False), (1024, 3, 1, False),
+    # batches of at least 4 x 148 problems take the batch builds of the kernels
+    (16, 1024, 8, False), (64, 1024, 6, False), (256, 640, 3, False),
+    # 8 or more problems beyond 256 ranks: tier-by-tier sums with 16 and 32 ranks per lane
+    (512, 8, 2, False), (1024, 8, 1, False),
+    # a cost that is not tiered: 16-warp register tile, 4-warp batch tile, clusters
+    (256, 64, 3, True), (256, 640, 2, True), (1024, 3, 1, True)])
 @pytest.mark.parametrize("eps_frac", [0.1, 0.01])
-def test_sweep_cell(R, B, check, eps_frac):
-    pl, C = _planner(B, R, eps_frac)
+def test_sweep_cell(R, B, check, eps_frac, general):
+    pl, C = _planner(B, R, eps_frac, general=general)
     loads = W.sweep_rank_loads(B, R, seed=1000 + R, device="cuda")
     ex, sp, s, d = pl.excess_spare(loads)
     mean, ex_ref, sp_ref = O.excess_spare(cpu(loads))
@@ -49,11 +61,13 @@ def test_sweep_cell(R, B, check, eps_frac):
     pl.close()
 
 
-def test_large_batch_with_mixed_problem_sizes_walks_the_kernel_chain():
+@pytest.mark.parametrize("general", [True, False])
+def test_large_batch_with_mixed_problem_sizes_walks_the_kernel_chain(general):
     """A batch that takes the 4-warp batch kernel, in which some problems have more supply ranks than that kernel
-    holds (they must come back marked and be solved by the 16-warp kernel), in tolerance mode."""
+    holds (they must come back marked and be solved by the 16-warp kernel), in tolerance mode.  With the tiered
+    cost the same batch goes through the tier-by-tier kernel, which has no such limit."""
     R, B = 256, 640
-    pl, C = _planner(B, R, 0.1, iters=300, tol=1e-6)
+    pl, C = _planner(B, R, 0.1, iters=300, tol=1e-6, general=general)
     loads = W.sweep_rank_loads(B, R, seed=77, device="cuda")
     g = torch.Generator(device="cuda").manual_seed(9)
     wide = torch.randint(1000, 60000, (B // 2, R), generator=g, device="cuda", dtype=torch.int32)
@@ -80,7 +94,7 @@ def test_cluster_kernel_and_its_fall_through_beyond_256_ranks(R):
     slice of 128 rows x 512 columns does not fit and the problem falls through to the kernel with the matrix in
     workspace; one narrow problem beside it stays on the clusters.  Both against the oracle."""
     B = 3
-    pl, C = _planner(B, R, 0.1, iters=40, tol=0.0)
+    pl, C = _planner(B, R, 0.1, iters=40, tol=0.0, general=True)
     loads = W.sweep_rank_loads(B, R, seed=31, device="cuda")
     g = torch.Generator(device="cuda").manual_seed(4)
     loads[1] = torch.randint(1000, 60000, (R,), generator=g, device="cuda", dtype=torch.int32)
@@ -110,4 +124,24 @@ def test_batches_larger_than_the_handle_and_unsupported_calls_beyond_256_ranks()
     topk = torch.zeros((2, R, 1), dtype=torch.int32, device="cuda")
     with pytest.raises(P.TaotError):
         pl.histogram(topk)
+    pl.close()
+
+
+def test_tiered_kernel_hands_back_a_rank_with_both_supply_and_demand():
+    """The tier-by-tier sums leave out the diagonal, which is right only while no rank has both supply and demand;
+    a problem that has such a rank must come back from that kernel and be solved by the general one."""
+    R, B = 256, 4
+    pl, C = _planner(B, R, 0.1, iters=60)
+    loads = W.sweep_rank_loads(B, R, seed=5, device="cuda")
+    ex, sp, s, d = pl.excess_spare(loads)
+    s = s.clone(); d = d.clone()
+    j = int(torch.nonzero(d[1] > 0)[0])
+    s[1, j] = 7.0                                        # problem 1: rank j now has both
+    out = pl.sinkhorn(s, d)
+    torch.cuda.synchronize()
+    plan, iters, err = cpu(out["plan"]), cpu(out["iters"]), cpu(out["row_err"])
+    assert (iters == 60).all()
+    for b in range(B):
+        check_sinkhorn_problem(cpu(s)[b], cpu(d)[b], C.numpy(), 0.1 * max(SWEEP_TIERS), plan[b], iters[b], err[b], 60, 0.0)
+    assert plan[1][j, j] > 0                             # the diagonal entry took part
     pl.close()
