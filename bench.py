@@ -201,10 +201,29 @@ def cpu_model():
     return "unknown"
 
 
+def tiered_sums(R, B, tiers, gpus_per_node, nodes_per_group):
+    """Does the library take the tier-by-tier Sinkhorn kernel for this shape?  (Its rule: a cost that depends only
+    on same node of 8 / same rail group of 32 / neither, 256, 512 or 1024 ranks, and at least 8 problems beyond 256
+    ranks.)  The generated costs have that structure when nodes hold 8 ranks and, if there is a group tier, groups
+    hold 4 nodes."""
+    if R not in (256, 512, 1024) or gpus_per_node != 8 or (R > 256 and B < 8):
+        return False
+    return len(tiers) == 3 or (len(tiers) == 4 and nodes_per_group == 4)
+
+
+def tiered_fma_per_iteration(R):
+    """FMAs the tier-by-tier kernel executes per problem and iteration: per half-step one product per rank, the node
+    and group factors, and three per rank for its own sum."""
+    return 2 * (4 * R + R // 4 + 1)
+
+
 def sinkhorn_work(out, cfg):
-    """FMA count the Sinkhorn kernel executed: 2 mat-vecs over the |hot| x |cold| block per iteration."""
+    """FMA count the Sinkhorn kernel executed: 2 mat-vecs over the |hot| x |cold| block per iteration, or the
+    tier-by-tier sums where the library takes those."""
     ex = out["excess"].cpu().numpy(); sp = out["spare"].cpu().numpy(); it = out["sinkhorn_iters"].cpu().numpy()
     hn = (ex > 0).sum(1).astype(np.int64); cn = (sp > 0).sum(1).astype(np.int64)
+    if tiered_sums(cfg.R, cfg.L, cfg.tiers, cfg.gpus_per_node, cfg.nodes_per_group):
+        return int((tiered_fma_per_iteration(cfg.R) * np.maximum(it - 1, 0)).sum()), it
     return int((2 * hn * cn * np.maximum(it - 1, 0)).sum()), it
 
 
@@ -233,7 +252,9 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count):
     if stage == "sinkhorn":
         fma, _ = sinkhorn_work(out, cfg)
         a = 2 * fma / (ms * 1e-3) / 1e12
-        return dict(kernel="sinkhorn_tile_kernel", bound="alu", achieved=a, peak=fp32_peak, unit="TFLOP/s",
+        tiered = tiered_sums(cfg.R, cfg.L, cfg.tiers, cfg.gpus_per_node, cfg.nodes_per_group)
+        return dict(kernel="sinkhorn_tiered_kernel" if tiered else "sinkhorn_tile_kernel", bound="alu", achieved=a,
+                    peak=fp32_peak, unit="TFLOP/s",
                     frac=a / fp32_peak, traffic=None,
                     peak_source=fp32_src, flops_per_launch=2 * fma,
                     note="one dependent chain of small mat-vecs per problem and only L problems per call: "
@@ -538,10 +559,14 @@ def run_sweep(args):
         reps = 3 if B * R * R < 5e8 else 1
         ms = timed_steps(lambda: pl.sinkhorn(s, d, out), reps + 1, None)[1:]
         hn = (ex > 0).sum(1).double(); cn = (sp > 0).sum(1).double()
-        fma = float((2 * hn * cn * (SWEEP_ITERS - 1)).sum())
+        dense_fma = float((2 * hn * cn * (SWEEP_ITERS - 1)).sum())        # a solver that holds the kernel matrix
+        tiered = tiered_sums(R, B, SWEEP_TIERS, 8, 4)
+        fma = float(B * tiered_fma_per_iteration(R) * (SWEEP_ITERS - 1)) if tiered else dense_fma
         t = float(np.median(ms)) * 1e-3
         cells.append(dict(B=B, R=R, eps_frac=eps_frac, ms=t * 1e3, plans_per_s=B / t,
+                          kernel="tiered sums" if tiered else "kernel matrix",
                           tflops=2 * fma / t / 1e12, frac_fp32_peak=2 * fma / t / 1e12 / fp32_peak,
+                          matrix_equiv_tflops=2 * dense_fma / t / 1e12,
                           hot_mean=float(hn.mean()), cold_mean=float(cn.mean()),
                           info_or=int(out["info"].max())))
         pl.close()
