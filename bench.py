@@ -201,14 +201,19 @@ def cpu_model():
     return "unknown"
 
 
-def tiered_sums(R, B, tiers, gpus_per_node, nodes_per_group):
-    """Does the library take the tier-by-tier Sinkhorn kernel for this shape?  (Its rule: a cost that depends only
-    on same node of 8 / same rail group of 32 / neither, 256, 512 or 1024 ranks, and at least 8 problems beyond 256
-    ranks.)  The generated costs have that structure when nodes hold 8 ranks and, if there is a group tier, groups
-    hold 4 nodes."""
-    if R not in (256, 512, 1024) or gpus_per_node != 8 or (R > 256 and B < 8):
+def tiered_sums(C, B):
+    """Does the library take the tier-by-tier Sinkhorn kernel for this cost matrix and batch?  Its rule, applied to
+    the matrix itself: 256, 512 or 1024 ranks, every off-diagonal cost equal to one of three values according to
+    same node of 8 ranks / same rail group of 32 / neither, and at least 8 problems beyond 256 ranks."""
+    R = C.shape[0]
+    if R not in (256, 512, 1024) or (R > 256 and B < 8):
         return False
-    return len(tiers) == 3 or (len(tiers) == 4 and nodes_per_group == 4)
+    i = torch.arange(R)
+    node = (i[:, None] // 8) == (i[None, :] // 8)
+    group = (i[:, None] // 32) == (i[None, :] // 32)
+    want = torch.where(node, C[0, 1], torch.where(group, C[0, 8], C[0, 32]))
+    off = i[:, None] != i[None, :]
+    return bool(torch.isfinite(want).all()) and bool((C[off] == want[off]).all())
 
 
 def tiered_fma_per_iteration(R):
@@ -222,7 +227,7 @@ def sinkhorn_work(out, cfg):
     tier-by-tier sums where the library takes those."""
     ex = out["excess"].cpu().numpy(); sp = out["spare"].cpu().numpy(); it = out["sinkhorn_iters"].cpu().numpy()
     hn = (ex > 0).sum(1).astype(np.int64); cn = (sp > 0).sum(1).astype(np.int64)
-    if tiered_sums(cfg.R, cfg.L, cfg.tiers, cfg.gpus_per_node, cfg.nodes_per_group):
+    if tiered_sums(W.cost_matrix(cfg.R, cfg.gpus_per_node, cfg.tiers, cfg.nodes_per_group), cfg.L):
         return int((tiered_fma_per_iteration(cfg.R) * np.maximum(it - 1, 0)).sum()), it
     return int((2 * hn * cn * np.maximum(it - 1, 0)).sum()), it
 
@@ -252,7 +257,7 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count):
     if stage == "sinkhorn":
         fma, _ = sinkhorn_work(out, cfg)
         a = 2 * fma / (ms * 1e-3) / 1e12
-        tiered = tiered_sums(cfg.R, cfg.L, cfg.tiers, cfg.gpus_per_node, cfg.nodes_per_group)
+        tiered = tiered_sums(W.cost_matrix(cfg.R, cfg.gpus_per_node, cfg.tiers, cfg.nodes_per_group), cfg.L)
         return dict(kernel="sinkhorn_tiered_kernel" if tiered else "sinkhorn_tile_kernel", bound="alu", achieved=a,
                     peak=fp32_peak, unit="TFLOP/s",
                     frac=a / fp32_peak, traffic=None,
@@ -560,7 +565,7 @@ def run_sweep(args):
         ms = timed_steps(lambda: pl.sinkhorn(s, d, out), reps + 1, None)[1:]
         hn = (ex > 0).sum(1).double(); cn = (sp > 0).sum(1).double()
         dense_fma = float((2 * hn * cn * (SWEEP_ITERS - 1)).sum())        # a solver that holds the kernel matrix
-        tiered = tiered_sums(R, B, SWEEP_TIERS, 8, 4)
+        tiered = tiered_sums(C, B)
         fma = float(B * tiered_fma_per_iteration(R) * (SWEEP_ITERS - 1)) if tiered else dense_fma
         t = float(np.median(ms)) * 1e-3
         cells.append(dict(B=B, R=R, eps_frac=eps_frac, ms=t * 1e3, plans_per_s=B / t,
