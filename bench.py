@@ -222,6 +222,25 @@ def tiered_fma_per_iteration(R):
     return 2 * (4 * R + R // 4 + 1)
 
 
+def sinkhorn_chain_floor(out, cfg, lat):
+    """Cycles of the dependent chain of ONE iteration of the kernel that solves this shape with few problems per
+    call, from the measured latencies: shuffle-reduction levels, the two scaling updates, and the multiply-add
+    chains in front of them.  None where no such model is kept (multi-warp tiles, clusters)."""
+    ex = out["excess"].cpu().numpy(); sp = out["spare"].cpu().numpy()
+    hn = int((ex > 0).sum(1).max()); cn = int((sp > 0).sum(1).max())
+    if tiered_sums(W.cost_matrix(cfg.R, cfg.gpus_per_node, cfg.tiers, cfg.nodes_per_group), cfg.L):
+        # per half-step: node sum (two chains of four adds), node and group factors, five shuffle levels, three
+        # multiply-adds of the rank's own sum, the scaling update
+        return 2 * (5 * lat["shuffle_level"] + 9 * lat["fma"] + lat["rcp_mul"]), "2 x (5 shuffle levels + 9 fma + rcp-mul)"
+    if cfg.R <= 64:
+        # 4 x 8 lane grid: row sums over 8 column lanes (3 levels), column sums over 4 row lanes (2 levels); the
+        # lane-local multiply-add chains are as long as the tile is deep (rows in steps of 4, columns in steps of 8)
+        nra = max(1, -(-hn // 4)); ncg = max(2, -(-cn // 8))
+        return (5 * lat["shuffle_level"] + (nra + ncg) * lat["fma"] + 2 * lat["rcp_mul"],
+                f"5 shuffle levels + {nra + ncg} fma + 2 rcp-mul")
+    return None, None
+
+
 def sinkhorn_work(out, cfg):
     """FMA count the Sinkhorn kernel executed: 2 mat-vecs over the |hot| x |cold| block per iteration, or the
     tier-by-tier sums where the library takes those."""
@@ -258,7 +277,19 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count):
         fma, _ = sinkhorn_work(out, cfg)
         a = 2 * fma / (ms * 1e-3) / 1e12
         tiered = tiered_sums(W.cost_matrix(cfg.R, cfg.gpus_per_node, cfg.tiers, cfg.nodes_per_group), cfg.L)
-        return dict(kernel="sinkhorn_tiered_kernel" if tiered else "sinkhorn_tile_kernel", bound="alu", achieved=a,
+        latency = None
+        if peaks.get("latency_cycles"):
+            cyc, model = sinkhorn_chain_floor(out, cfg, peaks["latency_cycles"])
+            if cyc:
+                its = int(out["sinkhorn_iters"].max().item())
+                floor_ns = cyc / (peaks["sm_max_mhz"] * 1e-3)
+                ach_ns = ms * 1e6 / max(its, 1)
+                latency = dict(bound="dependent chain of one iteration", floor_ns_per_iteration=floor_ns,
+                               achieved_ns_per_iteration=ach_ns, frac=floor_ns / ach_ns, iterations=its, model=model,
+                               cycles=peaks["latency_cycles"],
+                               note="achieved = stage time / iterations of the slowest problem (set-up and "
+                                    "write-out included); floor from taot_measure_latencies at the maximum SM clock")
+        d = dict(kernel="sinkhorn_tiered_kernel" if tiered else "sinkhorn_tile_kernel", bound="alu", achieved=a,
                     peak=fp32_peak, unit="TFLOP/s",
                     frac=a / fp32_peak, traffic=None,
                     peak_source=fp32_src, flops_per_launch=2 * fma,
@@ -266,6 +297,9 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count):
                          "latency-bound; DRAM traffic is ~0.1 MB per launch (ncu); the fp32-FMA fraction is "
                          "reported, not claimed as the binding limit (see profiles/sweep_config5.md for batches "
                          "that fill the GPU)")
+        if latency:
+            d["latency"] = latency
+        return d
     rounds = out["rounds"].cpu().numpy().astype(np.int64)
     ops = int((rounds[:, 0] * cfg.R * cfg.E + rounds[:, 1] * cfg.R * cfg.S).sum())
     a = ops / (ms * 1e-3) / 1e12
@@ -386,6 +420,7 @@ def run_ours(args):
     peaks = measured_peaks()
     import paper_2608_03676_b200 as P
     peaks.update(P.measure_alu_peaks())              # FP32-FMA and ex2 ceilings of this GPU, measured once, untimed
+    peaks["latency_cycles"] = P.measure_latencies() # dependent-operation latencies, for the chain floor of the Sinkhorn stage
     props = torch.cuda.get_device_properties(local)
     topk = W.routing_topk(cfg, device="cuda")
     pl = build_planner(cfg)

@@ -328,6 +328,17 @@ int taot_get_stage_ms(taot_handle_t h, float* h_ms /* [5] */);
  */
 int taot_measure_alu_peaks(float* h_fma_tflops, float* h_ex2_tops, void* d_sink, void* stream);
 
+/*
+ * Latencies of the current device, measured, in SM clock cycles per dependent operation: h_cycles[0] one level of
+ * a warp shuffle reduction (shfl.xor + add), [1] one FP32 fused multiply-add, [2] one scaling update (rcp.approx +
+ * multiply-add).  With few problems per call the Sinkhorn stage is one dependent chain per problem: the sum of
+ * these latencies along one iteration is the floor its iteration time is compared with.  (The paper has no
+ * counterpart: a measurement aid, not a step of the method.)  Launches one warp on `stream` and WAITS for it.
+ * d_sink: device memory of at least 16 bytes (overwritten).  h_cycles: host floats [3].
+ * Errors: TAOT_ERR_NULL, TAOT_ERR_CUDA.
+ */
+int taot_measure_latencies(float* h_cycles /* [3] */, void* d_sink, void* stream);
+
 /* Kernels launched by the last call on this handle (for launch accounting). */
 int taot_last_launch_count(taot_handle_t h, int32_t* count);
 

@@ -26,6 +26,7 @@ from .binding import (  # noqa: F401
     INFO_INTERNAL,
     ReportRow,
     measure_alu_peaks,
+    measure_latencies,
     PipelinedHostPlanner,
     StreamingHostPlanner,
     split_layers,

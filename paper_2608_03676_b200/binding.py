@@ -26,7 +26,7 @@ ABLATE_TOPOLOGY = 2
 _SYMBOLS = [
     "taot_create", "taot_destroy", "taot_workspace_bytes", "taot_host_workspace_bytes",
     "taot_histogram", "taot_histogram_static", "taot_excess_spare", "taot_sinkhorn", "taot_match", "taot_assign",
-    "taot_plan", "taot_plan_host", "taot_report", "taot_dispatch", "taot_measure_alu_peaks", "taot_set_profiling", "taot_get_stage_ms", "taot_last_launch_count",
+    "taot_plan", "taot_plan_host", "taot_report", "taot_dispatch", "taot_measure_alu_peaks", "taot_measure_latencies", "taot_set_profiling", "taot_get_stage_ms", "taot_last_launch_count",
     "taot_status_string",
 ]
 
@@ -148,6 +148,16 @@ def measure_alu_peaks() -> Dict[str, float]:
     _check(lib.taot_measure_alu_peaks(ctypes.byref(fma), ctypes.byref(ex2), _ptr(sink), _stream()),
            "taot_measure_alu_peaks")
     return dict(fma_tflops=float(fma.value), ex2_tops=float(ex2.value))
+
+
+def measure_latencies() -> Dict[str, float]:
+    """SM clock cycles per dependent operation on the current GPU (`taot_measure_latencies`): one shuffle-reduction
+    level, one FMA, one reciprocal-and-multiply."""
+    lib = load_library()
+    sink = torch.zeros(4, dtype=torch.float32, device="cuda")
+    cyc = (ctypes.c_float * 3)()
+    _check(lib.taot_measure_latencies(cyc, _ptr(sink), _stream()), "taot_measure_latencies")
+    return dict(shuffle_level=float(cyc[0]), fma=float(cyc[1]), rcp_mul=float(cyc[2]))
 
 
 @dataclass

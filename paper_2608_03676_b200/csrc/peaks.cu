@@ -55,7 +55,61 @@ ex2_peak_kernel(float* sink, int outer)
     if (s == 12345.678f) sink[blockIdx.x * kPeakThreads + threadIdx.x] = s;
 }
 
+// Latency of the dependent operations a one-warp Sinkhorn iteration is made of, in SM clock cycles per operation:
+// one level of a shuffle reduction (shfl.xor + add), one fused multiply-add, one scaling update (rcp.approx + mul).
+// One warp, one long dependent chain per measurement, timed with the SM's own cycle counter.
+__global__ void __launch_bounds__(32)
+latency_kernel(float* out, int n, float a, float b)
+{
+    const unsigned full = 0xffffffffu;
+    float x = 1.0f + (float)threadIdx.x * 1e-3f;
+    float res[3];
+    for (int which = 0; which < 3; ++which) {
+        float y = x;
+        for (int pass = 0; pass < 2; ++pass) {                   // the first pass warms the instruction cache
+            const long long t0 = clock64();
+            if (which == 0) {
+#pragma unroll 16
+                for (int i = 0; i < n; ++i) y = y * 0.5f + __shfl_xor_sync(full, y, 1 << (i & 3)) * 0.5f;
+            } else if (which == 1) {
+#pragma unroll 16
+                for (int i = 0; i < n; ++i) y = fmaf(y, a, b);
+            } else {
+#pragma unroll 16
+                for (int i = 0; i < n; ++i) {
+                    float r;
+                    asm volatile("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(y));
+                    y = a * r + 1.0f;
+                }
+            }
+            const long long t1 = clock64();
+            res[which] = (float)(t1 - t0) / (float)n;
+        }
+        x += y * 1e-30f;
+    }
+    // level 0 carries one multiply more than a plain reduction level (it keeps the value bounded): take it off
+    if (threadIdx.x == 0) {
+        out[0] = res[0] - res[1];
+        out[1] = res[1];
+        out[2] = res[2];
+        out[3] = x;
+    }
+}
+
 }  // namespace
+
+extern "C" int taot_measure_latencies(float* h_cycles, void* d_sink, void* stream)
+{
+    if (!h_cycles || !d_sink) return TAOT_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    latency_kernel<<<1, 32, 0, st>>>(static_cast<float*>(d_sink), 4096, 0.999f, 1e-3f);
+    TAOT_CUDA_OK(cudaGetLastError());
+    float h[4];
+    TAOT_CUDA_OK(cudaMemcpyAsync(h, d_sink, sizeof(h), cudaMemcpyDeviceToHost, st));
+    TAOT_CUDA_OK(cudaStreamSynchronize(st));
+    h_cycles[0] = h[0]; h_cycles[1] = h[1]; h_cycles[2] = h[2];
+    return TAOT_OK;
+}
 
 extern "C" int taot_measure_alu_peaks(float* h_fma_tflops, float* h_ex2_tops, void* d_sink, void* stream)
 {
