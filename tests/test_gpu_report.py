@@ -182,3 +182,16 @@ def test_measured_alu_peaks_are_plausible():
     assert 0.5 * fma_nominal < pk["fma_tflops"] < 1.1 * fma_nominal, pk
     assert 0.5 * ex2_nominal < pk["ex2_tops"] < 1.1 * ex2_nominal, pk
     print(pk, fma_nominal, ex2_nominal)
+
+
+def test_measured_latencies_are_plausible():
+    """Dependent-operation latencies used for the chain floor of a Sinkhorn iteration: a fused multiply-add takes a
+    few cycles, a shuffle-reduction level and a reciprocal-and-multiply a few tens; the same call twice agrees."""
+    import paper_2608_03676_b200 as P
+    a = P.measure_latencies()
+    b = P.measure_latencies()
+    assert 2.0 < a["fma"] < 12.0, a
+    assert 10.0 < a["shuffle_level"] < 80.0, a
+    assert 8.0 < a["rcp_mul"] < 80.0, a
+    for key in a:
+        assert abs(a[key] - b[key]) <= 0.15 * a[key] + 1.0, (a, b)
