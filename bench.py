@@ -203,10 +203,10 @@ def cpu_model():
 
 def tiered_sums(C, B):
     """Does the library take the tier-by-tier Sinkhorn kernel for this cost matrix and batch?  Its rule, applied to
-    the matrix itself: 256, 512 or 1024 ranks, every off-diagonal cost equal to one of three values according to
-    same node of 8 ranks / same rail group of 32 / neither, and at least 8 problems beyond 256 ranks."""
+    the matrix itself: 256, 512 or 1024 ranks and every off-diagonal cost equal to one of three values according to
+    same node of 8 ranks / same rail group of 32 / neither (any batch size)."""
     R = C.shape[0]
-    if R not in (256, 512, 1024) or (R > 256 and B < 8):
+    if R not in (256, 512, 1024):
         return False
     i = torch.arange(R)
     node = (i[:, None] // 8) == (i[None, :] // 8)

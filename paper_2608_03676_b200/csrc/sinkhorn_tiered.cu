@@ -15,8 +15,9 @@
 // inside the fp32 range: a term that underflows is smaller by e^-87 than another term of the same sum.  The two
 // differences lose nothing that matters: e1_i N_n >= e2_i f_n N_n * exp((c2 - c1)/eps) >= e2_i f_n N_n, so the
 // rounding error of G (relative to G) enters the row sum with a weight no larger than the row sum itself, and
-// likewise for T.  A lane owns R/32 consecutive ranks (a node at 256 ranks, a rail group at 1024); node sums are
-// lane-local, group and total sums are xor-shuffle all-reduces (5 levels per half-step whatever R is).
+// likewise for T.  A lane owns R/32 consecutive ranks (a node at 256 ranks, the size this kernel is launched for:
+// large batches; sinkhorn_tiered_mw.cu spreads a problem over four warps for small batches and larger R); node
+// sums are lane-local, group and total sums are xor-shuffle all-reduces (5 levels per half-step).
 //
 // The iteration, its stopping rule, the drift fold of u~, v~ into the fp64 potentials (which recomputes every
 // factor above), the first iteration in the log domain and the final plan follow the register-tile kernels;
@@ -417,21 +418,21 @@ int launch_rpl(const SinkArgs& a, const TierCosts& tc, int32_t B, cudaStream_t s
 
 }  // namespace
 
-// Launches the tiered-cost kernel if the handle's cost matrix has the node / rail-group structure and R is one
-// of the sizes a warp splits evenly (256, 512, 1024 ranks); returns the number of kernels launched (0: not
+// Launches a tiered-cost kernel if the handle's cost matrix has the node / rail-group structure (checked at
+// taot_create, which also requires 256, 512 or 1024 ranks); returns the number of kernels launched (0: not
 // applicable, the caller takes the general kernels).
+int taot_launch_sinkhorn_tiered_mw(const SinkArgs& a, const float* tier_cost3, int32_t B, cudaStream_t st);
+
 int taot_launch_sinkhorn_tiered(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st)
 {
     if (!h->tier_ok) return 0;
-    if (h->p.R > 256 && B < 8) return 0;          // a few large problems: the four-CTA clusters have the shorter iteration
+    // few problems per call: four warps per problem (a lone warp is bound by the instructions it issues); batches
+    // of 256-rank problems that fill the GPU several times over: one warp per problem (fewest instructions per
+    // problem).  Beyond 256 ranks the four-warp kernel wins at every batch size (8 ranks per lane fit the registers).
+    if (B < 4 * h->sm_count || h->p.R > 256) return taot_launch_sinkhorn_tiered_mw(a, h->tier_cost, B, st);
     TierCosts tc;
     tc.c1 = (double)h->tier_cost[0] * a.inv_eps;
     tc.c2 = (double)h->tier_cost[1] * a.inv_eps;
     tc.c3 = (double)h->tier_cost[2] * a.inv_eps;
-    switch (h->p.R) {
-        case 256: return launch_rpl<8>(a, tc, B, st);
-        case 512: return launch_rpl<16>(a, tc, B, st);
-        case 1024: return launch_rpl<32>(a, tc, B, st);
-        default: return 0;
-    }
+    return launch_rpl<8>(a, tc, B, st);
 }

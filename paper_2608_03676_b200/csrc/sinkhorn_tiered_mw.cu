@@ -1,0 +1,436 @@
+// Sinkhorn-Knopp (Appendix A.2) for a tiered cost matrix, four warps per problem: the tier-by-tier sums of
+// sinkhorn_tiered.cu (see there for the factorisation and its error argument) with the ranks spread over 128
+// lanes, for calls with few problems, where one warp per problem is bound by the instructions it has to issue.
+//
+// Lane gl = 32 * warp + lane owns RPL = R / 128 consecutive ranks (2 at 256 ranks, 4 at 512, 8 at 1024): a node of
+// 8 ranks is 8 / RPL adjacent lanes, a rail group 32 / RPL lanes, a warp holds RPL whole groups.  A half-step is
+// lane-local products, five xor-shuffle levels (node, group, groups of the warp), one shared-memory exchange of
+// the four warp totals (one block barrier), three multiply-adds and a reciprocal per rank.  Every decision
+// (stop, drift fold, hand-back) is taken from values that went through an exchange, so it is the same in all 128
+// threads and every barrier is reached by all of them: the error partials of iterate t ride the exchange of
+// half-step 2, the drift and range flags of an update ride the first exchange of the next iteration (a fold
+// then discards that half-step's sums and starts the iteration again with the new factors).
+#include "sinkhorn_common.cuh"
+
+using namespace taot_sk;
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+constexpr int kNode = 8;
+constexpr int kGroup = 32;
+constexpr int kWarps = 4;
+constexpr int kThreads = kWarps * 32;
+
+__device__ __forceinline__ float rcp_fast(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ float exp_or_zero(double x) { return x == -INFINITY ? 0.0f : exp_split(x); }
+
+struct TierCosts {
+    double c1, c2, c3;            // cost / eps of the three tiers off the diagonal
+};
+
+__device__ __forceinline__ double tier_cost(const TierCosts& tc, int i, int j)
+{
+    return (i / kNode == j / kNode) ? tc.c1 : ((i / kGroup == j / kGroup) ? tc.c2 : tc.c3);
+}
+
+template <int LO, int HI>
+__device__ __forceinline__ float xor_sum(float v)           // all-reduce over lane bits LO <= offset < HI
+{
+#pragma unroll
+    for (int o = LO; o < HI; o <<= 1) v += __shfl_xor_sync(kFull, v, o);
+    return v;
+}
+template <int LO, int HI>
+__device__ __forceinline__ double xor_max(double v)
+{
+#pragma unroll
+    for (int o = LO; o < HI; o <<= 1) v = fmax(v, __shfl_xor_sync(kFull, v, o));
+    return v;
+}
+
+struct Exchange {                 // what one warp hands to the others in one half-step
+    float total;                  // its share of the sum over all groups
+    float err;                    // half-step 2: its share of the row error of the iterate
+    int flags;                    // half-step 1: drift (1) / range (2) of the previous update; half-step 2: range of the row sums (2)
+    int pad;
+};
+
+template <int RPL, bool TOL>
+__global__ void __launch_bounds__(kThreads)
+sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
+{
+    constexpr int LPN = kNode / RPL;              // lanes per node
+    constexpr int LPG = kGroup / RPL;             // lanes per rail group
+    static_assert(RPL >= 1 && RPL <= kNode && kNode % RPL == 0, "a lane holds part of one node");
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int R = a.R, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t b = blockIdx.x;
+    if (b >= nprob) return;
+    double* alpha = reinterpret_cast<double*>(smem_raw);          // [R] potentials by rank (supply ranks; -inf elsewhere)
+    double* beta = alpha + R;                                      // [R] (demand ranks)
+    float* fgs = reinterpret_cast<float*>(beta + R);               // [R] column cap of the final plan, 0 off the demand ranks
+    int32_t* hot = reinterpret_cast<int32_t*>(fgs + R);            // [R] supply ranks, ascending
+    __shared__ Exchange xch[2][kWarps];
+    __shared__ double dred[2][kWarps];
+    __shared__ int ired[kWarps];
+
+    // block-wide reductions for the set-up and the folds (two barriers each; not used inside an iteration)
+    auto block_sum2 = [&](double& p, double& q) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            p += __shfl_xor_sync(kFull, p, o);
+            q += __shfl_xor_sync(kFull, q, o);
+        }
+        if (lane == 0) { dred[0][warp] = p; dred[1][warp] = q; }
+        __syncthreads();
+        p = 0.0; q = 0.0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) { p += dred[0][w]; q += dred[1][w]; }
+        __syncthreads();
+    };
+    auto block_max2 = [&](double& p, double& q) {               // p, q already reduced over the warp
+        if (lane == 0) { dred[0][warp] = p; dred[1][warp] = q; }
+        __syncthreads();
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) { p = fmax(p, dred[0][w]); q = fmax(q, dred[1][w]); }
+        __syncthreads();
+    };
+
+    // ---- supply scaling gamma = min(1, sum d / max(sum s, eps0)); masses of this lane's ranks
+    const int q0 = tid * RPL;                     // first rank of this lane
+    float x[RPL];
+    unsigned hotm = 0u, coldm = 0u;
+    int both = 0;
+    double ps = 0.0, pd = 0.0;
+#pragma unroll
+    for (int i = 0; i < RPL; ++i) {
+        const float sv = a.s[b * R + q0 + i], dv = a.d[b * R + q0 + i];
+        if (sv > 0.0f) { ps += (double)sv; hotm |= 1u << i; }
+        if (dv > 0.0f) { pd += (double)dv; coldm |= 1u << i; }
+        both |= (sv > 0.0f && dv > 0.0f) ? 1 : 0;
+        x[i] = sv > 0.0f ? sv : (dv > 0.0f ? dv : 0.0f);
+    }
+    block_sum2(ps, pd);
+    if (__syncthreads_or(both)) {                 // the diagonal would take part: not this kernel's case
+        if (tid == 0) a.iters[b] = kHandBack;
+        return;
+    }
+    const double sum_s = ps, sum_d = pd;
+    const double gamma = fmin(1.0, sum_d / fmax(sum_s, (double)a.eps0));
+#pragma unroll
+    for (int i = 0; i < RPL; ++i)
+        if ((hotm >> i) & 1u) x[i] = (float)(gamma * (double)x[i]);
+    int info = 0;
+    if (sum_s > sum_d) info |= TAOT_INFO_SUPPLY_SCALED;
+    float* out = a.plan + b * (int64_t)R * R;
+    // supply ranks in ascending order: prefix over the lanes of a warp, then over the warps
+    const int Hn_lane = __popc(hotm), Cn_lane = __popc(coldm);
+    int incl = Hn_lane, Cw = Cn_lane;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(kFull, incl, o);
+        if (lane >= o) incl += up;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) Cw += __shfl_xor_sync(kFull, Cw, o);
+    if (lane == 31) ired[warp] = incl;
+    if (lane == 0) dred[0][warp] = (double)Cw;
+    __syncthreads();
+    int Hn = 0, hbase = incl - Hn_lane, Cn = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        if (w < warp) hbase += ired[w];
+        Hn += ired[w];
+        Cn += (int)dred[0][w];
+    }
+    __syncthreads();
+    if (Hn == 0 || Cn == 0) {
+        for (int q = tid; q < R * R; q += kThreads) out[q] = 0.0f;
+        if (tid == 0) {
+            a.iters[b] = 0;
+            a.row_err[b] = 0.0f;
+            if (info) atomicOr(a.info + b, info);
+        }
+        return;
+    }
+    {
+        int k = hbase;
+#pragma unroll
+        for (int i = 0; i < RPL; ++i)
+            if ((hotm >> i) & 1u) hot[k++] = q0 + i;
+    }
+    double sum_st = 0.0, unused = 0.0;
+#pragma unroll
+    for (int i = 0; i < RPL; ++i)
+        if ((hotm >> i) & 1u) sum_st += (double)x[i];
+    block_sum2(sum_st, unused);
+    const double tol_abs = (double)a.tol * sum_st;
+    const float tol_abs_f = (float)tol_abs;
+
+    // ---- iteration 1 in the log domain (v = 1 on every rank): phi = log s~ - LSE_j(-C_ij/eps) over all j,
+    //      psi_j = log d_j - LSE_i(phi_i - C_ij/eps)
+#pragma unroll
+    for (int i = 0; i < RPL; ++i)
+        alpha[q0 + i] = ((hotm >> i) & 1u) ? log((double)x[i]) - a.rowlse0[q0 + i] : -INFINITY;
+    __syncthreads();
+#pragma unroll 1
+    for (int i = 0; i < RPL; ++i) {
+        const int q = q0 + i;
+        double bj = -INFINITY;
+        if ((coldm >> i) & 1u) {
+            double mx = -INFINITY;
+            for (int h = 0; h < Hn; ++h) {
+                const int r = hot[h];
+                const double v = alpha[r] - tier_cost(tc, r, q);
+                mx = v > mx ? v : mx;
+            }
+            double acc = 0.0;
+            for (int h = 0; h < Hn; ++h) {
+                const int r = hot[h];
+                acc += (double)exp_split(alpha[r] - tier_cost(tc, r, q) - mx);
+            }
+            bj = log((double)a.d[b * R + q]) - (mx + log(acc));
+        }
+        beta[q] = bj;
+    }
+    __syncthreads();
+
+    // ---- per-rank state: z = u~ or v~, w = weight inside the node sum, k1..k3 = tier coefficients of its own sum;
+    // node and group factors of both trees (b: demand side, feeds the row sums; a: supply side, feeds the column sums)
+    float z[RPL], w[RPL], k1[RPL], k2[RPL], k3[RPL];
+    float fb = 0.0f, fa = 0.0f, Fb = 0.0f, Fa = 0.0f;
+#pragma unroll
+    for (int i = 0; i < RPL; ++i) z[i] = 1.0f;
+
+    auto rebuild = [&]() {                         // block-uniform: holds barriers
+        double m1 = -INFINITY, p1 = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < RPL; ++i) {
+            if ((coldm >> i) & 1u) m1 = fmax(m1, beta[q0 + i]);
+            if ((hotm >> i) & 1u) p1 = fmax(p1, alpha[q0 + i]);
+        }
+        m1 = xor_max<1, LPN>(m1); p1 = xor_max<1, LPN>(p1);
+        const double m2 = xor_max<LPN, LPG>(m1), p2 = xor_max<LPN, LPG>(p1);
+        double m3 = xor_max<LPG, 32>(m2), p3 = xor_max<LPG, 32>(p2);
+        block_max2(m3, p3);
+        fb = exp_or_zero(m1 == -INFINITY ? -INFINITY : m1 - m2);
+        fa = exp_or_zero(p1 == -INFINITY ? -INFINITY : p1 - p2);
+        Fb = exp_or_zero(m2 == -INFINITY ? -INFINITY : m2 - m3);
+        Fa = exp_or_zero(p2 == -INFINITY ? -INFINITY : p2 - p3);
+#pragma unroll
+        for (int i = 0; i < RPL; ++i) {
+            const bool ish = (hotm >> i) & 1u, isc = (coldm >> i) & 1u;
+            float wv = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
+            if (ish) {
+                const double al = alpha[q0 + i];
+                wv = exp_or_zero(al - p1);
+                a1 = exp_or_zero(m1 == -INFINITY ? -INFINITY : al - tc.c1 + m1);
+                a2 = exp_or_zero(m2 == -INFINITY ? -INFINITY : al - tc.c2 + m2);
+                a3 = exp_or_zero(m3 == -INFINITY ? -INFINITY : al - tc.c3 + m3);
+            } else if (isc) {
+                const double be = beta[q0 + i];
+                wv = exp_or_zero(be - m1);
+                a1 = exp_or_zero(p1 == -INFINITY ? -INFINITY : be - tc.c1 + p1);
+                a2 = exp_or_zero(p2 == -INFINITY ? -INFINITY : be - tc.c2 + p2);
+                a3 = exp_or_zero(p3 == -INFINITY ? -INFINITY : be - tc.c3 + p3);
+            }
+            w[i] = wv; k1[i] = a1; k2[i] = a2; k3[i] = a3;
+        }
+    };
+    auto fold = [&]() {                            // u~, v~ into the fp64 potentials, then every factor anew
+#pragma unroll
+        for (int i = 0; i < RPL; ++i) {
+            if ((hotm >> i) & 1u) alpha[q0 + i] += log((double)z[i]);
+            if ((coldm >> i) & 1u) beta[q0 + i] += log((double)z[i]);
+            z[i] = 1.0f;
+        }
+        rebuild();
+    };
+    // first part of a half-step: this lane's node sum N, group sum G (times the group factor: FG) and the warp's
+    // share of the total
+    auto partial = [&](const bool rows, const float (&zsrc)[RPL], float& N, float& G, float& FG) {
+        const unsigned srcm = rows ? coldm : hotm;
+        float p = 0.0f;
+#pragma unroll
+        for (int i = 0; i < RPL; ++i) p += ((srcm >> i) & 1u) ? w[i] * zsrc[i] : 0.0f;
+        N = xor_sum<1, LPN>(p);
+        // every node appears LPN times among the lanes of its group: sum one copy per node
+        G = xor_sum<LPN, LPG>((rows ? fb : fa) * N);
+        FG = (rows ? Fb : Fa) * G;
+        return xor_sum<LPG, 32>(FG);               // every group appears once per LPG lanes
+    };
+    auto own_sums = [&](const bool rows, float N, float G, float FG, float T, float (&res)[RPL]) {
+        const float Gx = G - (rows ? fb : fa) * N, Tx = T - FG;
+#pragma unroll
+        for (int i = 0; i < RPL; ++i) res[i] = fmaf(k1[i], N, fmaf(k2[i], Gx, k3[i] * Tx));
+    };
+    rebuild();
+
+    int t = 1;
+    int until_check = a.check_every;
+    float err_out = 0.0f;
+    const uint32_t lo_bits = __float_as_uint(kDriftLo), span_bits = __float_as_uint(kDriftHi) - lo_bits;
+    const unsigned anym = hotm | coldm;
+    int prev_flags = 0;                            // drift (1) / range (2) of the update that produced the current z
+    int k = 0;                                     // exchanges so far (their parity picks the buffer)
+    for (;;) {
+        // ================= half-step 1: r = K~ v~ on the supply ranks; these row sums belong to iterate t
+        float N, G, FG;
+        float tw = partial(true, z, N, G, FG);
+        const int wf = (__any_sync(kFull, prev_flags & 1) ? 1 : 0) | (__any_sync(kFull, prev_flags & 2) ? 2 : 0);
+        if (lane == 0) { xch[k & 1][warp].total = tw; xch[k & 1][warp].flags = wf; }
+        __syncthreads();
+        float T = 0.0f;
+        int flags = 0;
+#pragma unroll
+        for (int wv = 0; wv < kWarps; ++wv) { T += xch[k & 1][wv].total; flags |= xch[k & 1][wv].flags; }
+        ++k;
+        if (flags & 2) {                           // a sum of the previous update left the safe range: hand back
+            if (tid == 0) a.iters[b] = kHandBack;
+            return;
+        }
+        if (flags & 1) {                           // u~, v~ drifted: fold them and take the half-step again
+            fold();
+            prev_flags = 0;
+            continue;
+        }
+        float r[RPL];
+        own_sums(true, N, G, FG, T, r);
+        const bool last = t >= a.max_iters;
+        bool check_now = false;
+        if (TOL) {
+            check_now = until_check == 1;
+            until_check = check_now ? a.check_every : until_check - 1;
+        }
+        const bool test = last || check_now;
+        float ew = 0.0f;
+        int badr = 0;
+        if (test) {
+            float e = 0.0f;
+#pragma unroll
+            for (int i = 0; i < RPL; ++i) {
+                const bool ish = (hotm >> i) & 1u;
+                e += ish ? fabsf(fmaf(z[i], r[i], -x[i])) : 0.0f;
+                badr |= (ish && !(r[i] > kSumLo && r[i] < kSumHi)) ? 2 : 0;
+            }
+            ew = xor_sum<1, 32>(e);
+            badr = __any_sync(kFull, badr) ? 2 : 0;
+        }
+        float zn[RPL];
+#pragma unroll
+        for (int i = 0; i < RPL; ++i) zn[i] = ((hotm >> i) & 1u) ? x[i] * rcp_fast(r[i]) : z[i];
+        // ================= half-step 2: c = K~^T u' on the demand ranks, v' = d / c
+        tw = partial(false, zn, N, G, FG);
+        if (lane == 0) { xch[k & 1][warp].total = tw; xch[k & 1][warp].err = ew; xch[k & 1][warp].flags = badr; }
+        __syncthreads();
+        T = 0.0f;
+        float err = 0.0f;
+        flags = 0;
+#pragma unroll
+        for (int wv = 0; wv < kWarps; ++wv) {
+            T += xch[k & 1][wv].total;
+            err += xch[k & 1][wv].err;
+            flags |= xch[k & 1][wv].flags;
+        }
+        ++k;
+        if (test && (last || err <= tol_abs_f)) {  // iterate t is the result; half-step 2 is dropped
+            if (flags & 2) { if (tid == 0) a.iters[b] = kHandBack; return; }
+            err_out = (float)((double)err / sum_st);
+            if (TOL && !(err <= tol_abs_f)) info |= TAOT_INFO_SINKHORN_CAP;
+            break;
+        }
+        float c[RPL];
+        own_sums(false, N, G, FG, T, c);
+        // a sum outside the safe range shows in its reciprocal (zero, infinite or not a number), so the drift test
+        // catches it too; both flags travel with the next exchange
+        int f = 0;
+#pragma unroll
+        for (int i = 0; i < RPL; ++i) {
+            const bool ish = (hotm >> i) & 1u, isc = (coldm >> i) & 1u;
+            zn[i] = isc ? x[i] * rcp_fast(c[i]) : zn[i];
+            f |= (((anym >> i) & 1u) && (__float_as_uint(zn[i]) - lo_bits) > span_bits) ? 1 : 0;
+            f |= ((ish && !(r[i] > kSumLo && r[i] < kSumHi)) || (isc && !(c[i] > kSumLo && c[i] < kSumHi))) ? 2 : 0;
+        }
+        prev_flags = f;
+#pragma unroll
+        for (int i = 0; i < RPL; ++i) z[i] = zn[i];
+        ++t;
+    }
+
+    // ---- T = diag(u) M diag(v) from the total potentials, then the column cap
+    fold();
+    {
+        float N, G, FG;
+        const float tw = partial(false, z, N, G, FG);          // column sums of K~ itself (u~ = 1)
+        if (lane == 0) xch[k & 1][warp].total = tw;
+        __syncthreads();
+        float T = 0.0f;
+#pragma unroll
+        for (int wv = 0; wv < kWarps; ++wv) T += xch[k & 1][wv].total;
+        float c[RPL];
+        own_sums(false, N, G, FG, T, c);
+#pragma unroll
+        for (int i = 0; i < RPL; ++i)
+            fgs[q0 + i] = ((coldm >> i) & 1u) ? (float)fmin(1.0, (double)x[i] / ((double)c[i] + (double)a.eps0)) : 0.0f;
+    }
+    __syncthreads();
+    int nonfinite = 0;
+    for (int row = warp; row < R; row += kWarps) {
+        const double al = alpha[row];
+        float* orow = out + (int64_t)row * R;
+        if (al == -INFINITY) {
+            for (int j = lane; j < R; j += 32) orow[j] = 0.0f;
+            continue;
+        }
+#pragma unroll 4
+        for (int j = lane; j < R; j += 32) {
+            const float fg = fgs[j];
+            float val = 0.0f;
+            if (fg > 0.0f) {
+                val = exp_split(al + beta[j] - tier_cost(tc, row, j)) * fg;
+                if (!isfinite(val)) nonfinite = 1;
+            }
+            orow[j] = val;
+        }
+    }
+    if (__syncthreads_or(nonfinite)) info |= TAOT_INFO_NONFINITE;
+    if (tid == 0) {
+        a.iters[b] = t;
+        a.row_err[b] = err_out;
+        if (info) atomicOr(a.info + b, info);
+    }
+}
+
+template <int RPL>
+int launch_mw(const SinkArgs& a, const TierCosts& tc, int32_t B, cudaStream_t st)
+{
+    const size_t smem = (size_t)a.R * (2 * sizeof(double) + sizeof(float) + sizeof(int32_t));
+    if (a.tol > 0.0f) sinkhorn_tiered_mw_kernel<RPL, true><<<B, kThreads, smem, st>>>(a, tc, (int64_t)B);
+    else sinkhorn_tiered_mw_kernel<RPL, false><<<B, kThreads, smem, st>>>(a, tc, (int64_t)B);
+    TAOT_CUDA_OK(cudaGetLastError());
+    return 1;
+}
+
+}  // namespace
+
+// Four warps per problem (256, 512 or 1024 ranks); the caller has checked that the cost is tiered.
+int taot_launch_sinkhorn_tiered_mw(const SinkArgs& a, const float* tier_cost3, int32_t B, cudaStream_t st)
+{
+    TierCosts tc;
+    tc.c1 = (double)tier_cost3[0] * a.inv_eps;
+    tc.c2 = (double)tier_cost3[1] * a.inv_eps;
+    tc.c3 = (double)tier_cost3[2] * a.inv_eps;
+    switch (a.R) {
+        case 256: return launch_mw<2>(a, tc, B, st);
+        case 512: return launch_mw<4>(a, tc, B, st);
+        case 1024: return launch_mw<8>(a, tc, B, st);
+        default: return 0;
+    }
+}

@@ -32,7 +32,7 @@ def _planner(B, R, eps_frac, iters=SWEEP_ITERS, tol=0.0, general=False):
     (8, 64, 64, False), (16, 64, 64, False), (64, 64, 16, False), (256, 64, 4, False), (1024, 3, 1, False),
     # batches of at least 4 x 148 problems take the batch builds of the kernels
     (16, 1024, 8, False), (64, 1024, 6, False), (256, 640, 3, False),
-    # 8 or more problems beyond 256 ranks: tier-by-tier sums with 16 and 32 ranks per lane
+    # beyond 256 ranks with the tiered cost: tier-by-tier sums, four warps per problem, 4 and 8 ranks per lane
     (512, 8, 2, False), (1024, 8, 1, False),
     # a cost that is not tiered: 16-warp register tile, 4-warp batch tile, clusters
     (256, 64, 3, True), (256, 640, 2, True), (1024, 3, 1, True)])
