@@ -254,7 +254,8 @@ sinkhorn_tiered_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
 
     // sums of the absorbed kernel matrix against the current scalings: ROWS: (K~ v~)_i on the supply ranks (sources
     // are the demand ranks), else (K~^T u~)_j on the demand ranks; zsrc = scalings of the sources
-    auto tier_sums = [&](const bool rows, const float (&zsrc)[RPL], float (&res)[RPL]) {
+    // `carry` (if with_carry): one more value summed over the warp in the same shuffle levels (the row-error partial)
+    auto tier_sums = [&](const bool rows, const bool with_carry, const float (&zsrc)[RPL], float (&res)[RPL], float& carry) {
         const unsigned srcm = rows ? coldm : hotm;
         float N[NPL];
 #pragma unroll
@@ -271,9 +272,20 @@ sinkhorn_tiered_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
         float g = 0.0f;
 #pragma unroll
         for (int n = 0; n < NPL; ++n) g = fmaf(rows ? fb[n] : fa[n], N[n], g);
-        const float G = group_sum<LPG>(g);
+#pragma unroll
+        for (int o = 1; o < LPG; o <<= 1) {
+            g += __shfl_xor_sync(kFull, g, o);
+            if (with_carry) carry += __shfl_xor_sync(kFull, carry, o);
+        }
+        const float G = g;
         const float FG = (rows ? Fb : Fa) * G;
-        const float Tx = across_groups_sum<LPG>(FG) - FG;
+        float tt = FG;
+#pragma unroll
+        for (int o = LPG; o < 32; o <<= 1) {
+            tt += __shfl_xor_sync(kFull, tt, o);
+            if (with_carry) carry += __shfl_xor_sync(kFull, carry, o);
+        }
+        const float Tx = tt - FG;
 #pragma unroll
         for (int i = 0; i < RPL; ++i) {
             const int n = i / kNode;
@@ -301,7 +313,8 @@ sinkhorn_tiered_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
     for (;;) {
         // ================= half-step 1: r = K~ v~ on the supply ranks; these row sums belong to iterate t
         float r[RPL];
-        tier_sums(true, z, r);
+        float nocarry = 0.0f;
+        tier_sums(true, false, z, r, nocarry);
         auto rows_bad = [&]() {
             bool bad = false;
 #pragma unroll
@@ -322,14 +335,15 @@ sinkhorn_tiered_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
             float e = 0.0f;
 #pragma unroll
             for (int i = 0; i < RPL; ++i) e += ((hotm >> i) & 1u) ? fabsf(fmaf(z[i], r[i], -x[i])) : 0.0f;
-            err = warp_sum(e);
+            err = e;                               // summed over the warp inside half-step 2's reduction
         }
         float zn[RPL];
 #pragma unroll
         for (int i = 0; i < RPL; ++i) zn[i] = ((hotm >> i) & 1u) ? x[i] * rcp_fast(r[i]) : z[i];
         // ================= half-step 2: c = K~^T u' on the demand ranks, v' = d / c
         float c[RPL];
-        tier_sums(false, zn, c);
+        if (test) tier_sums(false, true, zn, c, err);
+        else tier_sums(false, false, zn, c, nocarry);
         if (test && (last || err <= tol_abs_f)) {
             if (rows_bad()) { if (lane == 0) a.iters[b] = kHandBack; return; }
             err_out = (float)((double)err / sum_st);
@@ -364,7 +378,8 @@ sinkhorn_tiered_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
     fold();
     {
         float c[RPL];
-        tier_sums(false, z, c);                    // column sums of K~ itself (u~ = 1)
+        float nocarry = 0.0f;
+        tier_sums(false, false, z, c, nocarry);    // column sums of K~ itself (u~ = 1)
 #pragma unroll
         for (int i = 0; i < RPL; ++i) {
             const int q = lane * RPL + i;

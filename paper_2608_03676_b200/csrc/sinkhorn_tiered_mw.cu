@@ -255,16 +255,36 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
     };
     // first part of a half-step: this lane's node sum N, group sum G (times the group factor: FG) and the warp's
     // share of the total
-    auto partial = [&](const bool rows, const float (&zsrc)[RPL], float& N, float& G, float& FG) {
+    // `carry` (if with_carry): one more value summed over the whole warp in the same five shuffle levels, so that
+    // its reduction overlaps this one instead of following it (the row-error partial of the iterate)
+    auto partial = [&](const bool rows, const bool with_carry, const float (&zsrc)[RPL], float& N, float& G, float& FG,
+                       float& carry) {
         const unsigned srcm = rows ? coldm : hotm;
         float p = 0.0f;
 #pragma unroll
         for (int i = 0; i < RPL; ++i) p += ((srcm >> i) & 1u) ? w[i] * zsrc[i] : 0.0f;
-        N = xor_sum<1, LPN>(p);
+#pragma unroll
+        for (int o = 1; o < LPN; o <<= 1) {
+            p += __shfl_xor_sync(kFull, p, o);
+            if (with_carry) carry += __shfl_xor_sync(kFull, carry, o);
+        }
+        N = p;
         // every node appears LPN times among the lanes of its group: sum one copy per node
-        G = xor_sum<LPN, LPG>((rows ? fb : fa) * N);
+        float g = (rows ? fb : fa) * N;
+#pragma unroll
+        for (int o = LPN; o < LPG; o <<= 1) {
+            g += __shfl_xor_sync(kFull, g, o);
+            if (with_carry) carry += __shfl_xor_sync(kFull, carry, o);
+        }
+        G = g;
         FG = (rows ? Fb : Fa) * G;
-        return xor_sum<LPG, 32>(FG);               // every group appears once per LPG lanes
+        float tt = FG;                             // every group appears once per LPG lanes
+#pragma unroll
+        for (int o = LPG; o < 32; o <<= 1) {
+            tt += __shfl_xor_sync(kFull, tt, o);
+            if (with_carry) carry += __shfl_xor_sync(kFull, carry, o);
+        }
+        return tt;
     };
     auto own_sums = [&](const bool rows, float N, float G, float FG, float T, float (&res)[RPL]) {
         const float Gx = G - (rows ? fb : fa) * N, Tx = T - FG;
@@ -283,7 +303,8 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
     for (;;) {
         // ================= half-step 1: r = K~ v~ on the supply ranks; these row sums belong to iterate t
         float N, G, FG;
-        float tw = partial(true, z, N, G, FG);
+        float nocarry = 0.0f;
+        float tw = partial(true, false, z, N, G, FG, nocarry);
         const int wf = (__any_sync(kFull, prev_flags & 1) ? 1 : 0) | (__any_sync(kFull, prev_flags & 2) ? 2 : 0);
         if (lane == 0) { xch[k & 1][warp].total = tw; xch[k & 1][warp].flags = wf; }
         __syncthreads();
@@ -320,14 +341,14 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
                 e += ish ? fabsf(fmaf(z[i], r[i], -x[i])) : 0.0f;
                 badr |= (ish && !(r[i] > kSumLo && r[i] < kSumHi)) ? 2 : 0;
             }
-            ew = xor_sum<1, 32>(e);
+            ew = e;                                // summed over the warp inside half-step 2's reduction
             badr = __any_sync(kFull, badr) ? 2 : 0;
         }
         float zn[RPL];
 #pragma unroll
         for (int i = 0; i < RPL; ++i) zn[i] = ((hotm >> i) & 1u) ? x[i] * rcp_fast(r[i]) : z[i];
         // ================= half-step 2: c = K~^T u' on the demand ranks, v' = d / c
-        tw = partial(false, zn, N, G, FG);
+        tw = test ? partial(false, true, zn, N, G, FG, ew) : partial(false, false, zn, N, G, FG, nocarry);
         if (lane == 0) { xch[k & 1][warp].total = tw; xch[k & 1][warp].err = ew; xch[k & 1][warp].flags = badr; }
         __syncthreads();
         T = 0.0f;
@@ -368,7 +389,8 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
     fold();
     {
         float N, G, FG;
-        const float tw = partial(false, z, N, G, FG);          // column sums of K~ itself (u~ = 1)
+        float nocarry = 0.0f;
+        const float tw = partial(false, false, z, N, G, FG, nocarry);          // column sums of K~ itself (u~ = 1)
         if (lane == 0) xch[k & 1][warp].total = tw;
         __syncthreads();
         float T = 0.0f;

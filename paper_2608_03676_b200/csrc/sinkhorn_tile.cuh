@@ -408,10 +408,18 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
             for (int ra = 1; ra < NRA; ++ra) acc = fmaf(K[ra][cg], un[ra], acc);
             cp[cg] = acc;
         }
+        // tolerance mode: the error of iterate t (from the row sums just formed) is reduced over the row lanes in the
+        // same shuffle levels as the column sums, so that its two levels overlap theirs instead of following them
+        float e_tol = 0.0f;
+        if (TOL) {
+#pragma unroll
+            for (int ra = 0; ra < NRA; ++ra) e_tol += row_ok[ra] ? fabsf(fmaf(uo[ra], r[ra], -stl[ra])) : 0.0f;
+        }
 #pragma unroll
         for (int off = CL; off < 32; off <<= 1) {
 #pragma unroll
             for (int cg = 0; cg < NCG; ++cg) cp[cg] += __shfl_xor_sync(kFull, cp[cg], off);
+            if (TOL) e_tol += __shfl_xor_sync(kFull, e_tol, off);
         }
         // ---- the row sums belong to iterate t: is this where the solve stops?  The loop body is kept free of
         // branches (a lone warp pays dearly for each one) and the one branch it has never waits for this iteration's
@@ -434,7 +442,7 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
         float err_now = 0.0f;
         bool check_now = false;
         if (TOL) {
-            err_now = row_error();
+            err_now = e_tol;
             check_now = until_check == 1;
             until_check = check_now ? a.check_every : until_check - 1;
         }
