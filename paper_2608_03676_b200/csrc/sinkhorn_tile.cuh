@@ -362,8 +362,8 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
     const float tol_abs_f = (float)tol_abs;
     const uint32_t lo_bits = __float_as_uint(kDriftLo), span_bits = __float_as_uint(kDriftHi) - lo_bits;
     float usave[NRA], vsave[NCG];    // tolerance mode: the iterate whose error is still to be tested
-    bool pend = false;
-    float err_pend = 0.0f;
+    bool pend = false, near_pend = false;
+    float e_pend = 0.0f;
 #pragma unroll
     for (int ra = 0; ra < NRA; ++ra) usave[ra] = 1.0f;
 #pragma unroll
@@ -408,19 +408,30 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
             for (int ra = 1; ra < NRA; ++ra) acc = fmaf(K[ra][cg], un[ra], acc);
             cp[cg] = acc;
         }
-        // tolerance mode: the error of iterate t (from the row sums just formed) is reduced over the row lanes in the
-        // same shuffle levels as the column sums, so that its two levels overlap theirs instead of following them
-        float e_tol = 0.0f;
+        // tolerance mode: this lane's share of the error of iterate t (from the row sums just formed).  Up to 32
+        // ranks (VOTE) the shares are not summed here: as long as one of them alone exceeds the tolerance the sum does
+        // too (they are non-negative), and that is settled by one vote; the sum is formed only when no share does
+        // (see below).  Beyond 32 ranks the sum is formed in the shuffle levels of the column sums (measured: the
+        // vote costs the larger tiles more than it saves).
+        constexpr bool VOTE = CG == 1;
+        float e_loc = 0.0f;
+        bool near_now = true;
         if (TOL) {
 #pragma unroll
-            for (int ra = 0; ra < NRA; ++ra) e_tol += row_ok[ra] ? fabsf(fmaf(uo[ra], r[ra], -stl[ra])) : 0.0f;
+            for (int ra = 0; ra < NRA; ++ra) e_loc += row_ok[ra] ? fabsf(fmaf(uo[ra], r[ra], -stl[ra])) : 0.0f;
+            if (VOTE) near_now = !__any_sync(kFull, e_loc > tol_abs_f);
         }
 #pragma unroll
         for (int off = CL; off < 32; off <<= 1) {
 #pragma unroll
             for (int cg = 0; cg < NCG; ++cg) cp[cg] += __shfl_xor_sync(kFull, cp[cg], off);
-            if (TOL) e_tol += __shfl_xor_sync(kFull, e_tol, off);
+            if (TOL && !VOTE) e_loc += __shfl_xor_sync(kFull, e_loc, off);
         }
+        auto over_row_lanes = [&](float e) {
+#pragma unroll
+            for (int off = CL; off < 32; off <<= 1) e += __shfl_xor_sync(kFull, e, off);
+            return e;                                                    // the same bits in every lane
+        };
         // ---- the row sums belong to iterate t: is this where the solve stops?  The loop body is kept free of
         // branches (a lone warp pays dearly for each one) and the one branch it has never waits for this iteration's
         // error: in tolerance mode the error of iterate t is computed every iteration but TESTED one iteration later,
@@ -439,18 +450,19 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
             for (int ra = 0; ra < NRA; ++ra) bad_r |= row_ok[ra] && !(r[ra] > kSumLo && r[ra] < kSumHi);
             return __any_sync(kFull, bad_r) != 0;
         };
-        float err_now = 0.0f;
         bool check_now = false;
         if (TOL) {
-            err_now = e_tol;
             check_now = until_check == 1;
             until_check = check_now ? a.check_every : until_check - 1;
         }
 #pragma unroll
         for (int cg = 0; cg < NCG; ++cg) vnew[cg] = col_ok[cg] ? ddg[cg] * rcp_fast(cp[cg]) : 1.0f;
-        const bool stop_prev = TOL && pend && err_pend <= tol_abs_f;
+        // VOTE: no share of iterate t-1's error exceeded the tolerance; else: its error, already summed, met it
+        const bool stop_maybe = TOL && pend && (VOTE ? near_pend : e_pend <= tol_abs_f);
         const bool last = t >= a.max_iters;
-        if (stop_prev | last | odd) {
+        if (stop_maybe | last | odd) {
+            const bool stop_prev = stop_maybe && (VOTE ? over_row_lanes(e_pend) : e_pend) <= tol_abs_f;
+            const float err_now = TOL ? (VOTE ? over_row_lanes(e_loc) : e_loc) : 0.0f;
             if (stop_prev) {
                 // iterate t-1 met the tolerance: go back to it (its row sums are recomputed for the range check)
 #pragma unroll
@@ -472,6 +484,7 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
                 if (TOL && !(err <= tol_abs_f)) info |= TAOT_INFO_SINKHORN_CAP;
                 break;
             }
+            if (odd) {
             // rare: either u~, v~ merely drifted (fold them into the potentials) or a sum of this update left the
             // range in which fp32 products are trustworthy (hand the problem back)
             bool bad = false;
@@ -496,11 +509,14 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
             pend = false;                        // the test of iterate t was settled above
             ++t;
             continue;
+            }
+            // neither: the shares of iterate t-1 were all small but their sum was not; carry on
         }
         // ---- commit iteration t+1; iterate t stays behind until its error has been tested
         if (TOL) {
             pend = check_now;
-            err_pend = err_now;
+            near_pend = near_now;
+            e_pend = e_loc;
 #pragma unroll
             for (int ra = 0; ra < NRA; ++ra) usave[ra] = uo[ra];
 #pragma unroll
