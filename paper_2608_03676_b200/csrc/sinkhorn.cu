@@ -5,7 +5,7 @@
 // log v~  with (alpha, beta) in fp64 and (u~, v~) in fp32 near 1, and the kernel matrix held on
 // chip is  K~_ij = exp(alpha_i + beta_j - C_ij/eps)  rounded to fp32.  A half-step is then an
 // fp32 mat-vec over K~ followed by a divide, exactly the paper's GEMV form, but it cannot
-// under- or overflow for any C/eps: whenever u~ or v~ drifts outside [e^-20, e^20] the factors
+// under- or overflow for any C/eps: whenever u~ or v~ drifts outside [e^-40, e^40] the factors
 // are folded into (alpha, beta) and K~ is rebuilt (fp64 exp, a few times per solve).  Only rows
 // with supply and columns with demand carry flow, so K~ is compacted to |hot| x |cold|.
 // The first iteration (v = 1 on every rank) is done in the log domain in fp64; so is any

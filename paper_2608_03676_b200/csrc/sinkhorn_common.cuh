@@ -37,8 +37,8 @@ __device__ __forceinline__ float exp_split(double x)
     return expf(xh) * (1.0f + xl);
 }
 
-constexpr float kDriftLo = 2.0611536e-9f;   // e^-20
-constexpr float kDriftHi = 4.8516520e8f;    // e^+20
+constexpr float kDriftLo = 4.2483543e-18f;  // e^-40
+constexpr float kDriftHi = 2.3538527e17f;   // e^+40
 constexpr float kSumLo = 1e-30f;
 constexpr float kSumHi = 1e30f;
 constexpr int kHandBack = -1;               // iters[b] value meaning "not solved here"

@@ -67,7 +67,7 @@ struct TileSmem {
     float part[NW > 1 ? NW * RMAX : 1];
     float errw[32];
     int32_t hot[RMAX], cold[RMAX], hpos[RMAX], cpos[RMAX], wcnt[32];
-    int flags[4];                    // [parity]: some u~, v~ of this iteration left [e^-20, e^20]
+    int flags[4];                    // [parity]: some u~, v~ of this iteration left [e^-40, e^40]
     double sum[2];
 };
 
@@ -117,7 +117,7 @@ __device__ __forceinline__ bool tile_solve(const SinkArgs& a, TileSmem<NW, CG>& 
     int until_check = a.check_every; // iterations until the next tolerance test (tested when it reaches 1)
     float err_out = 0.0f;
     const float tol_abs_f = (float)tol_abs;
-    // u~ and v~ must stay inside [e^-20, e^20]; for positive floats that is one unsigned compare on the bits
+    // u~ and v~ must stay inside [e^-40, e^40]; for positive floats that is one unsigned compare on the bits
     // (negative, NaN and infinite values fall outside too)
     const uint32_t lo_bits = __float_as_uint(kDriftLo), span_bits = __float_as_uint(kDriftHi) - lo_bits;
 
@@ -372,7 +372,7 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
     for (;;) {
         // Drift test on the u~, v~ this iteration STARTS from; the vote is issued here and consumed at the end of
         // the iteration, so neither it nor the branch it feeds sits on the dependent chain.  Acting one update
-        // late is safe: a value that left [e^-20, e^20] is still far inside the fp32 range, and should an update
+        // late is safe: a value that left [e^-40, e^40] is still far inside the fp32 range, and should an update
         // jump past that range after all, its sums leave (kSumLo, kSumHi) and the problem is handed back.
         bool odd = false;
 #pragma unroll
