@@ -3,7 +3,8 @@
 
 int taot_launch_sinkhorn_tile_r64(const SinkArgs& a, int32_t B, int sm_count, cudaStream_t st)
 {
-    sinkhorn_tile_kernel<1, 2, 8, 16, 32, 1><<<B, 32, 0, st>>>(a, (int64_t)B);
+    if (a.tol > 0.0f) sinkhorn_tile_kernel<1, 2, 8, 16, 32, 1, true><<<B, 32, 0, st>>>(a, (int64_t)B);
+    else sinkhorn_tile_kernel<1, 2, 8, 16, 32, 1, false><<<B, 32, 0, st>>>(a, (int64_t)B);
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
 }
