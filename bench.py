@@ -53,7 +53,7 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-groups", type=int, default=4,
                     help="layer groups (streams) the end-to-end host call is pipelined over")
-    ap.add_argument("--e2e-depth", type=int, default=3,
+    ap.add_argument("--e2e-depth", type=int, default=4,
                     help="host calls in flight in the end-to-end measurement")
     ap.add_argument("--e2e-stream-groups", type=int, default=1,
                     help="layer groups per call when several calls are in flight")
@@ -490,6 +490,9 @@ def run_ours(args):
     hp.close(); del host_out
     sp = P.StreamingHostPlanner(L=cfg.L, depth=depth, groups=args.e2e_stream_groups, **kw)
     host_outs = sp.alloc_host_outputs(names)
+    packed = "_block" in host_outs[0]
+    if packed:                                       # one block (every output but the routing table) + the table
+        d2h = host_outs[0]["_block"].numel() + host_outs[0]["new_idx"].numel() * 4
 
     # (b) `depth` calls in flight: step i starts once step i - depth has delivered its outputs (and L2 has been
     # flushed after that), while the steps between them are still copying and computing
@@ -544,7 +547,7 @@ def run_ours(args):
         e2e=dict(value=e2e_value, unit="plans/s", h2d_bytes_per_step=topk_bytes, d2h_bytes_per_step=d2h,
                  ms_per_step=float(np.mean(e2e_ms)), in_flight=depth,
                  serial_value=serial_value, serial_ms_per_step=float(np.mean(serial_ms)),
-                 api=f"StreamingHostPlanner.submit: taot_plan_host, {depth} call(s) in flight, each on "
+                 api=f"StreamingHostPlanner.submit: {'taot_plan_host_block (outputs packed: two copies back)' if packed else 'taot_plan_host'}, {depth} call(s) in flight, each on "
                      f"{len(sp.lanes[0].planners)} group(s) of layers; serial_*: PipelinedHostPlanner.plan_host, one "
                      f"call at a time on {n_groups} groups of layers (one stream each)"),
         gpu_launches=launches,

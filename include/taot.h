@@ -249,6 +249,19 @@ int taot_plan_host(taot_handle_t h, const int32_t* h_topk, const taot_outputs* o
                    void* stream);
 
 /*
+ * taot_plan_host with the results packed: the rewritten routing table goes to h_new_idx [L,T,k] and EVERY other
+ * member of taot_outputs to one host block, in two device-to-host copies instead of one per output (a small copy
+ * costs the copy engine about as much as 0.5 MB does, which bounds throughput when several calls are in flight).
+ * taot_host_block_layout gives the block's size and, in the order of taot_outputs' members, the byte offset of every
+ * output inside it (multiples of 256; the entry of new_idx, member 12, is SIZE_MAX).  Bytes between outputs are
+ * overwritten.  Pinned host memory makes the copies asynchronous.  d_ws: taot_host_workspace_bytes bytes.
+ * Errors: TAOT_ERR_NULL, TAOT_ERR_ALIGN, and those of taot_plan.
+ */
+int taot_host_block_layout(taot_handle_t h, size_t* offsets /* [14] */, size_t* bytes);
+int taot_plan_host_block(taot_handle_t h, const int32_t* h_topk, int32_t* h_new_idx, void* h_block, void* d_ws,
+                         void* stream);
+
+/*
  * Dispatch metadata for the token all-to-all that follows the planner (Method: the rewritten routing is what the
  * dispatcher executes; the paper does not spell the bookkeeping out, so the layout below is this library's).
  * For each problem l and source rank r (the R contiguous segments of (T/R)*k entries of d_new_idx[l]):

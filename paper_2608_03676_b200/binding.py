@@ -26,7 +26,7 @@ ABLATE_TOPOLOGY = 2
 _SYMBOLS = [
     "taot_create", "taot_destroy", "taot_workspace_bytes", "taot_host_workspace_bytes",
     "taot_histogram", "taot_histogram_static", "taot_excess_spare", "taot_sinkhorn", "taot_match", "taot_assign",
-    "taot_plan", "taot_plan_host", "taot_report", "taot_dispatch", "taot_measure_alu_peaks", "taot_measure_latencies", "taot_set_profiling", "taot_get_stage_ms", "taot_last_launch_count",
+    "taot_plan", "taot_plan_host", "taot_host_block_layout", "taot_plan_host_block", "taot_report", "taot_dispatch", "taot_measure_alu_peaks", "taot_measure_latencies", "taot_set_profiling", "taot_get_stage_ms", "taot_last_launch_count",
     "taot_status_string",
 ]
 
@@ -370,6 +370,43 @@ class Planner:
                       info=((L,), torch.int32))
         return {nm: torch.empty(shapes[nm][0], dtype=shapes[nm][1]).pin_memory() for nm in names}
 
+    def alloc_host_block(self) -> Dict[str, torch.Tensor]:
+        """Pinned host buffers for `plan_host_block`: the rewritten routing table, one block for every other output,
+        and a view into the block per output (all 14 names of the outputs, plus "_block")."""
+        offs = (ctypes.c_size_t * 14)()
+        nbytes = ctypes.c_size_t()
+        _check(self.lib.taot_host_block_layout(self.handle, offs, ctypes.byref(nbytes)), "taot_host_block_layout")
+        L, R, E, K, S, T, k = self.L, self.R, self.E, self.K, self.S, self.T, self.k
+        shapes = dict(n=((L, R, E), torch.int32), expert_load=((L, E), torch.int32), rank_load=((L, R), torch.int32),
+                      excess=((L, R), torch.int32), spare=((L, R), torch.int32), plan=((L, R, R), torch.float32),
+                      sinkhorn_iters=((L,), torch.int32), row_err=((L,), torch.float32),
+                      slot_expert=((L, R, K), torch.int32), slot_tokens=((L, R, K), torch.int32),
+                      X=((L, R, S), torch.int32), rounds=((L, 2), torch.int32), info=((L,), torch.int32))
+        block = torch.empty(nbytes.value, dtype=torch.uint8).pin_memory()
+        out = {"_block": block, "new_idx": torch.empty((L, T, k), dtype=torch.int32).pin_memory()}
+        for i, (name, _) in enumerate(_Outputs._fields_):
+            if name == "new_idx":
+                continue
+            shape, dt = shapes[name]
+            count = 1
+            for d in shape:
+                count *= d
+            out[name] = block[offs[i]: offs[i] + 4 * count].view(dt).view(shape)
+        return out
+
+    def plan_host_block(self, topk_host: torch.Tensor, out_host: Dict[str, torch.Tensor]) -> Dict[str, torch.Tensor]:
+        """`plan_host` into buffers from `alloc_host_block`: two device-to-host copies for all outputs."""
+        if topk_host.is_cuda or topk_host.dtype != torch.int32 or not topk_host.is_contiguous():
+            raise TaotError("topk_host: expected a contiguous CPU int32 tensor")
+        if "_block" not in out_host:
+            raise TaotError("out_host: expected the buffers of alloc_host_block")
+        if self._host_ws is None:
+            self._host_ws = torch.empty(self.host_ws_bytes, dtype=torch.uint8, device=self.device)
+        _check(self.lib.taot_plan_host_block(self.handle, _ptr(topk_host), _ptr(out_host["new_idx"]),
+                                             _ptr(out_host["_block"]), _ptr(self._host_ws), _stream()),
+               "taot_plan_host_block")
+        return out_host
+
     def plan_host(self, topk_host: torch.Tensor, out_host: Dict[str, torch.Tensor]) -> Dict[str, torch.Tensor]:
         """Whole path from a HOST routing table to HOST results; copies ride the current stream."""
         if topk_host.is_cuda or topk_host.dtype != torch.int32 or not topk_host.is_contiguous():
@@ -407,6 +444,12 @@ class PipelinedHostPlanner:
         self.L = L
         self._key, self._calls, self._held = None, [], None
 
+    def alloc_host_block(self) -> Dict[str, torch.Tensor]:
+        """Packed host outputs (see `Planner.alloc_host_block`); only with a single group of layers."""
+        if len(self.planners) != 1:
+            raise TaotError("packed host outputs need a single group of layers")
+        return self.planners[0].alloc_host_block()
+
     def alloc_host_outputs(self, names=("plan", "slot_expert", "slot_tokens", "X", "new_idx", "info")):
         parts = [p.alloc_host_outputs(names) for p in self.planners]
         # one pinned tensor per output, of which every group sees its slice
@@ -419,6 +462,18 @@ class PipelinedHostPlanner:
     def plan_host(self, topk_host: torch.Tensor, out_host: Dict[str, torch.Tensor], join: bool = True) -> Dict[str, torch.Tensor]:
         if topk_host.is_cuda or topk_host.dtype != torch.int32 or not topk_host.is_contiguous():
             raise TaotError("topk_host: expected a contiguous CPU int32 tensor")
+        if "_block" in out_host:                      # packed outputs: a single group, one call
+            if len(self.planners) != 1:
+                raise TaotError("packed host outputs need a single group of layers")
+            cur = torch.cuda.current_stream()
+            st = self.streams[0]
+            st.wait_stream(cur)
+            with torch.cuda.stream(st):
+                self.planners[0].plan_host_block(topk_host, out_host)
+            self._held = (topk_host, out_host)
+            if join:
+                self.join()
+            return out_host
         # the per-group argument blocks depend only on the buffers' addresses: marshal them once per buffer set
         key = (topk_host.data_ptr(),) + tuple((k, v.data_ptr()) for k, v in sorted(out_host.items()))
         if key != self._key:
@@ -473,8 +528,14 @@ class StreamingHostPlanner:
         self._outs = [None] * depth
         self._n = 0
 
-    def alloc_host_outputs(self, names=("plan", "slot_expert", "slot_tokens", "X", "new_idx", "info")):
-        """One pinned output set per lane."""
+    def alloc_host_outputs(self, names=("plan", "slot_expert", "slot_tokens", "X", "new_idx", "info"), packed=None):
+        """One pinned output set per lane.  packed (default: whenever a call is one group of layers): every output
+        but the routing table lives in one block per lane and comes back in one copy (all outputs are then
+        present, whatever `names` says)."""
+        if packed is None:
+            packed = all(len(lane.planners) == 1 for lane in self.lanes)
+        if packed:
+            return [lane.alloc_host_block() for lane in self.lanes]
         return [lane.alloc_host_outputs(names) for lane in self.lanes]
 
     def submit(self, topk_host: torch.Tensor, out_host: Dict[str, torch.Tensor]) -> int:

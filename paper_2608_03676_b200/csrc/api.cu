@@ -505,6 +505,31 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, voi
     return TAOT_OK;
 }
 
+// H2D copy of the routing table, the whole path on device staging buffers; `d` receives the device pointers
+static int plan_on_staging(taot_handle_t h, const int32_t* h_topk, void* d_ws, void* stream, taot_outputs* d)
+{
+    const taot_params& p = h->p;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t NE = (size_t)p.L * p.T * p.k;
+    d->n = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_n));
+    d->expert_load = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_el));
+    d->rank_load = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_rl));
+    d->excess = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_ex));
+    d->spare = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_sp));
+    d->plan = reinterpret_cast<float*>(at(d_ws, h->hoff_plan));
+    d->sinkhorn_iters = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_it));
+    d->row_err = reinterpret_cast<float*>(at(d_ws, h->hoff_err));
+    d->slot_expert = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_se));
+    d->slot_tokens = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_st));
+    d->X = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_X));
+    d->rounds = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_rounds));
+    d->new_idx = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_new));
+    d->info = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_info));
+    int32_t* d_topk = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_topk));
+    TAOT_CUDA_OK(cudaMemcpyAsync(d_topk, h_topk, sizeof(int32_t) * NE, cudaMemcpyHostToDevice, st));
+    return taot_plan(h, d_topk, d, at(d_ws, h->hoff_ws), stream);
+}
+
 int taot_plan_host(taot_handle_t h, const int32_t* h_topk, const taot_outputs* o, void* d_ws, void* stream)
 {
     if (!h || !h_topk || !o || !d_ws) return TAOT_ERR_NULL;
@@ -513,23 +538,7 @@ int taot_plan_host(taot_handle_t h, const int32_t* h_topk, const taot_outputs* o
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t LR = (size_t)p.L * p.R, S = (size_t)p.R * p.K, NE = (size_t)p.L * p.T * p.k;
     taot_outputs d;
-    d.n = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_n));
-    d.expert_load = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_el));
-    d.rank_load = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_rl));
-    d.excess = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_ex));
-    d.spare = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_sp));
-    d.plan = reinterpret_cast<float*>(at(d_ws, h->hoff_plan));
-    d.sinkhorn_iters = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_it));
-    d.row_err = reinterpret_cast<float*>(at(d_ws, h->hoff_err));
-    d.slot_expert = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_se));
-    d.slot_tokens = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_st));
-    d.X = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_X));
-    d.rounds = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_rounds));
-    d.new_idx = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_new));
-    d.info = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_info));
-    int32_t* d_topk = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_topk));
-    TAOT_CUDA_OK(cudaMemcpyAsync(d_topk, h_topk, sizeof(int32_t) * NE, cudaMemcpyHostToDevice, st));
-    const int rc = taot_plan(h, d_topk, &d, at(d_ws, h->hoff_ws), stream);
+    const int rc = plan_on_staging(h, h_topk, d_ws, stream, &d);
     if (rc != TAOT_OK) return rc;
 #define TAOT_BACK(member, count, type)                                                                       \
     if (o->member)                                                                                           \
@@ -549,6 +558,34 @@ int taot_plan_host(taot_handle_t h, const int32_t* h_topk, const taot_outputs* o
     TAOT_BACK(new_idx, NE, int32_t);
     TAOT_BACK(info, (size_t)p.L, int32_t);
 #undef TAOT_BACK
+    return TAOT_OK;
+}
+
+int taot_host_block_layout(taot_handle_t h, size_t* offsets, size_t* bytes)
+{
+    if (!h || !offsets || !bytes) return TAOT_ERR_NULL;
+    const size_t base = h->hoff_n;
+    const size_t off[14] = {h->hoff_n, h->hoff_el, h->hoff_rl, h->hoff_ex, h->hoff_sp, h->hoff_plan, h->hoff_it,
+                            h->hoff_err, h->hoff_se, h->hoff_st, h->hoff_X, h->hoff_rounds, 0, h->hoff_info};
+    for (int i = 0; i < 14; ++i) offsets[i] = (i == 12) ? (size_t)-1 : off[i] - base;     // member 12 is new_idx
+    *bytes = h->hoff_ws - base;
+    return TAOT_OK;
+}
+
+int taot_plan_host_block(taot_handle_t h, const int32_t* h_topk, int32_t* h_new_idx, void* h_block, void* d_ws,
+                         void* stream)
+{
+    if (!h || !h_topk || !h_new_idx || !h_block || !d_ws) return TAOT_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(d_ws) & 255) return TAOT_ERR_ALIGN;
+    const taot_params& p = h->p;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t NE = (size_t)p.L * p.T * p.k;
+    taot_outputs d;
+    const int rc = plan_on_staging(h, h_topk, d_ws, stream, &d);
+    if (rc != TAOT_OK) return rc;
+    // the staging buffers of all outputs but the routing table are one contiguous range: one copy
+    TAOT_CUDA_OK(cudaMemcpyAsync(h_block, at(d_ws, h->hoff_n), h->hoff_ws - h->hoff_n, cudaMemcpyDeviceToHost, st));
+    TAOT_CUDA_OK(cudaMemcpyAsync(h_new_idx, d.new_idx, sizeof(int32_t) * NE, cudaMemcpyDeviceToHost, st));
     return TAOT_OK;
 }
 

@@ -252,8 +252,11 @@ def test_pipelined_host_planner_equals_the_single_call():
     hp.close(); pl.close()
 
 
-def test_streaming_host_planner_keeps_steps_apart():
-    """Two host calls in flight on alternating inputs: every step's outputs are those of a lone call on its input."""
+@pytest.mark.parametrize("groups", [1, 2])
+def test_streaming_host_planner_keeps_steps_apart(groups):
+    """Two host calls in flight on alternating inputs: every step's outputs are those of a lone call on its input.
+    With one group of layers per call the outputs are packed (one block and one copy for all but the routing
+    table); with two, every output has its own buffer and copy."""
     import paper_2608_03676_b200 as P
     cfg = W.get_config("cfg2").replace(L=5)
     e2r, C = topology(cfg)
@@ -262,9 +265,10 @@ def test_streaming_host_planner_keeps_steps_apart():
     names = ("n", "plan", "sinkhorn_iters", "slot_expert", "slot_tokens", "X", "new_idx", "info", "rounds")
     want = [{k: cpu(v).copy() for k, v in pl.plan(t).items()} for t in inputs]
     assert (want[0]["new_idx"] != want[1]["new_idx"]).any()
-    sp = P.StreamingHostPlanner(L=cfg.L, depth=2, groups=2, R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k, T=cfg.T, e2r=e2r,
+    sp = P.StreamingHostPlanner(L=cfg.L, depth=2, groups=groups, R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k, T=cfg.T, e2r=e2r,
                                 C=C, eps=cfg.eps, max_iters=cfg.max_iters, tol=cfg.tol)
     outs = sp.alloc_host_outputs(names)
+    assert ("_block" in outs[0]) == (groups == 1)
     host_in = [t.cpu().pin_memory() for t in inputs]
     tickets = []
     for step in range(7):
