@@ -145,3 +145,23 @@ def test_tiered_kernel_hands_back_a_rank_with_both_supply_and_demand():
         check_sinkhorn_problem(cpu(s)[b], cpu(d)[b], C.numpy(), 0.1 * max(SWEEP_TIERS), plan[b], iters[b], err[b], 60, 0.0)
     assert plan[1][j, j] > 0                             # the diagonal entry took part
     pl.close()
+
+
+def test_tiered_kernel_with_two_tiers_only():
+    """A node / cross-node cost without a rail-group tier is still a pure tier cost (the group and far tiers carry the
+    same value): it takes the tier-by-tier sums, four warps per problem, and the one-warp build for a large batch."""
+    import paper_2608_03676_b200 as P
+    R = 256
+    C = W.cost_matrix(R, 8, (0.0, 1.0, 12.0), None)
+    for B, check in ((6, 3), (600, 2)):
+        pl = P.Planner(L=B, R=R, E=R, K=1, k=1, T=R, e2r=torch.arange(R, dtype=torch.int32), C=C, eps=1.2,
+                       max_iters=80, tol=0.0)
+        loads = W.sweep_rank_loads(B, R, seed=91, device="cuda")
+        ex, sp, s, d = pl.excess_spare(loads)
+        out = pl.sinkhorn(s, d)
+        torch.cuda.synchronize()
+        plan, iters, err, info = cpu(out["plan"]), cpu(out["iters"]), cpu(out["row_err"]), cpu(out["info"])
+        assert (iters == 80).all() and (info == 0).all()
+        for b in range(check):
+            check_sinkhorn_problem(cpu(s)[b], cpu(d)[b], C.numpy(), 1.2, plan[b], iters[b], err[b], 80, 0.0)
+        pl.close()

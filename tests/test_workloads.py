@@ -70,3 +70,27 @@ def test_sweep_loads_sum_exactly():
     assert not torch.equal(l[0], l[1])
     ratio = float(srt[0, 0] / srt[0, 1])
     assert abs(ratio - 2 ** 1.2) < 0.01
+
+
+def test_bench_recognises_the_tiered_costs_of_the_workloads():
+    """bench.py decides from the cost matrix which Sinkhorn kernel the library takes (to count its work): the costs
+    of config 4 and of the sweep from 256 ranks up are pure tier costs, smaller ones and perturbed ones are not."""
+    import importlib.util
+    import os
+    import torch
+    import workloads as W
+    from workloads.configs import SWEEP_TIERS
+    spec = importlib.util.spec_from_file_location("bench_mod", os.path.join(os.path.dirname(__file__), "..", "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    for R in (256, 512, 1024):
+        assert bench.tiered_sums(W.cost_matrix(R, 8, SWEEP_TIERS, 4), 1)
+    assert not bench.tiered_sums(W.cost_matrix(64, 8, SWEEP_TIERS, 4), 64)
+    cfg = W.get_config("cfg4")
+    C = W.cost_matrix(cfg.R, cfg.gpus_per_node, cfg.tiers, cfg.nodes_per_group)
+    assert bench.tiered_sums(C, cfg.L)
+    C2 = C.clone(); C2[3, 77] += 1.0
+    assert not bench.tiered_sums(C2, cfg.L)
+    two_tier = W.cost_matrix(256, 8, (0.0, 1.0, 12.0), None)          # node / cross-node only: still a tier cost
+    assert bench.tiered_sums(two_tier, 8)
+    assert bench.tiered_fma_per_iteration(256) == 2 * (4 * 256 + 64 + 1)
