@@ -165,3 +165,22 @@ def test_tiered_kernel_with_two_tiers_only():
         for b in range(check):
             check_sinkhorn_problem(cpu(s)[b], cpu(d)[b], C.numpy(), 1.2, plan[b], iters[b], err[b], 80, 0.0)
         pl.close()
+
+
+@pytest.mark.parametrize("R", [512, 1024])
+def test_tiered_kernel_in_tolerance_mode_beyond_256_ranks(R):
+    """The stopping rule of the four-warp tier-by-tier kernel with 4 and 8 ranks per lane: first iterate whose row
+    error meets the tolerance, or the cap."""
+    B = 3
+    pl, C = _planner(B, R, 0.1, iters=400, tol=1e-6)
+    loads = W.sweep_rank_loads(B, R, seed=57, device="cuda")
+    ex, sp, s, d = pl.excess_spare(loads)
+    out = pl.sinkhorn(s, d)
+    torch.cuda.synchronize()
+    plan, iters, err, info = cpu(out["plan"]), cpu(out["iters"]), cpu(out["row_err"]), cpu(out["info"])
+    assert (iters >= 1).all() and (iters <= 400).all() and ((info & ~(2 | 16)) == 0).all()
+    for b in range(B):
+        check_sinkhorn_problem(cpu(s)[b], cpu(d)[b], C.numpy(), 0.1 * max(SWEEP_TIERS), plan[b], iters[b], err[b],
+                               400, 1e-6)
+    print(f"R={R}: iterations {iters.tolist()}")
+    pl.close()
