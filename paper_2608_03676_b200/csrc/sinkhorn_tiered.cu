@@ -16,7 +16,7 @@
 // differences lose nothing that matters: e1_i N_n >= e2_i f_n N_n * exp((c2 - c1)/eps) >= e2_i f_n N_n, so the
 // rounding error of G (relative to G) enters the row sum with a weight no larger than the row sum itself, and
 // likewise for T.  A lane owns R/32 consecutive ranks (a node at 256 ranks, the size this kernel is launched for:
-// large batches; sinkhorn_tiered_mw.cu spreads a problem over four warps for small batches and larger R); node
+// large batches; sinkhorn_tiered_mw.cu spreads a problem over eight warps for small batches and larger R); node
 // sums are lane-local, group and total sums are xor-shuffle all-reduces (5 levels per half-step).
 //
 // The iteration, its stopping rule, the drift fold of u~, v~ into the fp64 potentials (which recomputes every
@@ -441,9 +441,9 @@ int taot_launch_sinkhorn_tiered_mw(const SinkArgs& a, const float* tier_cost3, i
 int taot_launch_sinkhorn_tiered(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st)
 {
     if (!h->tier_ok) return 0;
-    // few problems per call: four warps per problem (a lone warp is bound by the instructions it issues); batches
+    // few problems per call: eight warps per problem (a lone warp is bound by the instructions it issues); batches
     // of 256-rank problems that fill the GPU several times over: one warp per problem (fewest instructions per
-    // problem).  Beyond 256 ranks the four-warp kernel wins at every batch size (8 ranks per lane fit the registers).
+    // problem).  Beyond 256 ranks the eight-warp kernel wins at every batch size (32 ranks per lane do not fit the registers).
     if (B < 4 * h->sm_count || h->p.R > 256) return taot_launch_sinkhorn_tiered_mw(a, h->tier_cost, B, st);
     TierCosts tc;
     tc.c1 = (double)h->tier_cost[0] * a.inv_eps;

@@ -1,12 +1,12 @@
-// Sinkhorn-Knopp (Appendix A.2) for a tiered cost matrix, four warps per problem: the tier-by-tier sums of
-// sinkhorn_tiered.cu (see there for the factorisation and its error argument) with the ranks spread over 128
+// Sinkhorn-Knopp (Appendix A.2) for a tiered cost matrix, eight warps per problem: the tier-by-tier sums of
+// sinkhorn_tiered.cu (see there for the factorisation and its error argument) with the ranks spread over 256
 // lanes, for calls with few problems, where one warp per problem is bound by the instructions it has to issue.
 //
-// Lane gl = 32 * warp + lane owns RPL = R / 128 consecutive ranks (2 at 256 ranks, 4 at 512, 8 at 1024): a node of
+// Lane gl = 32 * warp + lane owns RPL = R / 256 consecutive ranks (1 at 256 ranks, 2 at 512, 4 at 1024): a node of
 // 8 ranks is 8 / RPL adjacent lanes, a rail group 32 / RPL lanes, a warp holds RPL whole groups.  A half-step is
 // lane-local products, five xor-shuffle levels (node, group, groups of the warp), one shared-memory exchange of
-// the four warp totals (one block barrier), three multiply-adds and a reciprocal per rank.  Every decision
-// (stop, drift fold, hand-back) is taken from values that went through an exchange, so it is the same in all 128
+// the eight warp totals (one block barrier), three multiply-adds and a reciprocal per rank.  Every decision
+// (stop, drift fold, hand-back) is taken from values that went through an exchange, so it is the same in all 256
 // threads and every barrier is reached by all of them: the error partials of iterate t ride the exchange of
 // half-step 2, the drift and range flags of an update ride the first exchange of the next iteration (a fold
 // then discards that half-step's sums and starts the iteration again with the new factors).
@@ -19,7 +19,7 @@ namespace {
 constexpr unsigned kFull = 0xffffffffu;
 constexpr int kNode = 8;
 constexpr int kGroup = 32;
-constexpr int kWarps = 4;
+constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 
 __device__ __forceinline__ float rcp_fast(float x)
@@ -442,7 +442,7 @@ int launch_mw(const SinkArgs& a, const TierCosts& tc, int32_t B, cudaStream_t st
 
 }  // namespace
 
-// Four warps per problem (256, 512 or 1024 ranks); the caller has checked that the cost is tiered.
+// Eight warps per problem (256, 512 or 1024 ranks); the caller has checked that the cost is tiered.
 int taot_launch_sinkhorn_tiered_mw(const SinkArgs& a, const float* tier_cost3, int32_t B, cudaStream_t st)
 {
     TierCosts tc;
@@ -450,9 +450,9 @@ int taot_launch_sinkhorn_tiered_mw(const SinkArgs& a, const float* tier_cost3, i
     tc.c2 = (double)tier_cost3[1] * a.inv_eps;
     tc.c3 = (double)tier_cost3[2] * a.inv_eps;
     switch (a.R) {
-        case 256: return launch_mw<2>(a, tc, B, st);
-        case 512: return launch_mw<4>(a, tc, B, st);
-        case 1024: return launch_mw<8>(a, tc, B, st);
+        case 256: return launch_mw<1>(a, tc, B, st);
+        case 512: return launch_mw<2>(a, tc, B, st);
+        case 1024: return launch_mw<4>(a, tc, B, st);
         default: return 0;
     }
 }

@@ -32,7 +32,7 @@ def _planner(B, R, eps_frac, iters=SWEEP_ITERS, tol=0.0, general=False):
     (8, 64, 64, False), (16, 64, 64, False), (64, 64, 16, False), (256, 64, 4, False), (1024, 3, 1, False),
     # batches of at least 4 x 148 problems take the batch builds of the kernels
     (16, 1024, 8, False), (64, 1024, 6, False), (256, 640, 3, False),
-    # beyond 256 ranks with the tiered cost: tier-by-tier sums, four warps per problem, 4 and 8 ranks per lane
+    # beyond 256 ranks with the tiered cost: tier-by-tier sums, eight warps per problem, 2 and 4 ranks per lane
     (512, 8, 2, False), (1024, 8, 1, False),
     # a cost that is not tiered: 16-warp register tile, 4-warp batch tile, clusters
     (256, 64, 3, True), (256, 640, 2, True), (1024, 3, 1, True)])
@@ -149,7 +149,7 @@ def test_tiered_kernel_hands_back_a_rank_with_both_supply_and_demand():
 
 def test_tiered_kernel_with_two_tiers_only():
     """A node / cross-node cost without a rail-group tier is still a pure tier cost (the group and far tiers carry the
-    same value): it takes the tier-by-tier sums, four warps per problem, and the one-warp build for a large batch."""
+    same value): it takes the tier-by-tier sums, eight warps per problem, and the one-warp build for a large batch."""
     import paper_2608_03676_b200 as P
     R = 256
     C = W.cost_matrix(R, 8, (0.0, 1.0, 12.0), None)
@@ -169,7 +169,7 @@ def test_tiered_kernel_with_two_tiers_only():
 
 @pytest.mark.parametrize("R", [512, 1024])
 def test_tiered_kernel_in_tolerance_mode_beyond_256_ranks(R):
-    """The stopping rule of the four-warp tier-by-tier kernel with 4 and 8 ranks per lane: first iterate whose row
+    """The stopping rule of the eight-warp tier-by-tier kernel with 2 and 4 ranks per lane: first iterate whose row
     error meets the tolerance, or the cap."""
     B = 3
     pl, C = _planner(B, R, 0.1, iters=400, tol=1e-6)
