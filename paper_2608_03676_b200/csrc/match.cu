@@ -533,8 +533,10 @@ int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expe
     if (smem > 227 * 1024) return TAOT_ERR_UNSUPPORTED;
     TAOT_CUDA_OK(cudaFuncSetAttribute(match_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int need = p.R * p.K > p.R ? p.R * p.K : p.R;
-    int NT = ((need + 31) / 32) * 32;
-    NT = NT < 128 ? 128 : (NT > 1024 ? 1024 : NT);
+    // two threads per slot (or rank): Phase 2 splits each rank's scan over more lanes, and the extra warps cost the
+    // auction's barriers less than that saves (measured: 256 threads for 16 and 64 ranks, 512 for 256 ranks x 1 slot)
+    int NT = 2 * (((need + 31) / 32) * 32);
+    NT = NT < 256 ? 256 : (NT > 1024 ? 1024 : NT);
     match_kernel<<<p.L, NT, smem, st>>>(a);
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
