@@ -410,7 +410,8 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
         for (int ra = 0; ra < NRA; ++ra) odd |= (__float_as_uint(uo[ra]) - lo_bits) > span_bits;
 #pragma unroll
         for (int cg = 0; cg < NCG; ++cg) odd |= (__float_as_uint(vreg[cg]) - lo_bits) > span_bits;
-        odd = __any_sync(kFull, odd);
+        // (tolerance mode up to 32 ranks: this vote is taken further down, in one ballot with the error shares)
+        if (!(TOL && CG == 1)) odd = __any_sync(kFull, odd);
         // ================= half-step 1: r = K~ v~, u' = s~ / r
         float r[NRA], un[NRA];
         auto row_sums = [&]() {
@@ -450,7 +451,16 @@ __device__ __forceinline__ bool grid_solve(const SinkArgs& a, TileSmem<1, CG>& s
         if (TOL) {
 #pragma unroll
             for (int ra = 0; ra < NRA; ++ra) e_loc += row_ok[ra] ? fabsf(fmaf(uo[ra], r[ra], -stl[ra])) : 0.0f;
-            if (VOTE) near_now = !__any_sync(kFull, e_loc > tol_abs_f);
+            if (VOTE) {
+                // One ballot carries both votes: u~ is the same in the 8 column lanes of a row lane, v~ in the 4 row
+                // lanes of a column lane and the error share in the 8 column lanes, so the lanes with lr + lc even
+                // (every lr and every lc occurs among them) vote on the drift and the others on the error share.
+                constexpr unsigned kDriftLanes = 0xAA55AA55u;
+                const bool drift_lane = (kDriftLanes >> lane) & 1u;
+                const unsigned votes = __ballot_sync(kFull, drift_lane ? odd : (e_loc > tol_abs_f));
+                odd = (votes & kDriftLanes) != 0u;
+                near_now = (votes & ~kDriftLanes) == 0u;
+            }
         }
 #pragma unroll
         for (int off = CL; off < 32; off <<= 1) {
