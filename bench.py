@@ -5,11 +5,14 @@ One step = one pass of the whole path (histogram -> excess/spare -> Sinkhorn -> 
 auction -> token reassignment) over one batch of L synthetic routing problems, through
 `taot_plan`.  Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--impl ours|reference]
 
-N > 1 is launched with torch.distributed.run; every rank plans its own L problems (independent
-replicas, no data-path collective), the timed region is bracketed by barriers and the slowest
-rank's device time is reported.
+The default workload is the largest single-GPU configuration (config 4: 48 layers, 256 ranks, a
+1.6 GB routing table).  N > 1: one process per GPU.  Started under torch.distributed.run the ranks
+come from the environment; started as a plain `python bench.py --gpus N` the script launches the N
+ranks itself (torch.distributed.run, rendezvous on 127.0.0.1).  Every rank plans its own L problems
+(independent replicas, no data-path collective), the timed region is bracketed by barriers and the
+slowest rank's device time is reported.
 """
 from __future__ import annotations
 
@@ -33,9 +36,9 @@ import workloads as W  # noqa: E402
 L2_BYTES = 126 * 1024 * 1024
 FLUSH_BYTES = 256 * 1024 * 1024
 FP32_LANES_PER_SM = 128
-# DRAM bytes per algorithmic byte of the streaming kernels, from the ncu captures summarised under profiles/
-# (config 3 shape with 8 layers; traffic grows in proportion to the entries processed, so a full launch is
-# scaled by its own algorithmic bytes).  The reassignment figure is read + write once dirty L2 lines drain.
+# DRAM bytes per algorithmic byte of the streaming kernels, from one ncu capture each (config 3 shape with
+# 8 layers; traffic grows in proportion to the entries processed, so a full launch is scaled by its own
+# algorithmic bytes).  The reassignment figure is read + write once dirty L2 lines drain.
 HIST_TRAFFIC_RATIO = 1.045
 ASSIGN_TRAFFIC_RATIO = 1.01
 STAGES = ["histogram", "merge", "sinkhorn", "match_auction", "assign"]
@@ -47,14 +50,17 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", default="cfg2", choices=sorted(W.CONFIGS))
+    ap.add_argument("--workload", default="cfg4", choices=sorted(W.CONFIGS))
     ap.add_argument("--layers", type=int, default=0, help="override L (smaller batch, e.g. for a profiler capture)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-groups", type=int, default=4,
                     help="layer groups (streams) the end-to-end host call is pipelined over")
-    ap.add_argument("--e2e-depth", type=int, default=4,
-                    help="host calls in flight in the end-to-end measurement")
+    ap.add_argument("--e2e-depth", type=int, default=0,
+                    help="host calls in flight in the end-to-end measurement (0: 4 for tables up to 64 MB, else 2)")
+    ap.add_argument("--rendezvous-only", action="store_true",
+                    help="check the launch path only: every rank joins the process group (gloo when there is no "
+                         "GPU), the ranks reduce a per-rank time to the slowest one, rank 0 prints one JSON line")
     ap.add_argument("--e2e-stream-groups", type=int, default=1,
                     help="layer groups per call when several calls are in flight")
     ap.add_argument("--no-streams", action="store_true", help="skip the HBM-sized streaming report")
@@ -137,6 +143,15 @@ def measured_peaks():
 
 
 METRIC = "placement plans/s (whole planner path: histogram, excess/spare, Sinkhorn, matching+auction, token remap)"
+
+
+def config_dict(args, cfg):
+    """The `config` object of the JSON line; both arms print the same one for the same arguments."""
+    table = cfg.L * cfg.T * cfg.k * 4
+    return dict(workload=args.workload, L=cfg.L, R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k, T=cfg.T,
+                eps=cfg.eps, max_iters=cfg.max_iters, tol=cfg.tol, routing_table_bytes=table,
+                l2="inputs larger than L2" if 2 * table >= 4 * L2_BYTES else "flushed between steps (256 MiB write)",
+                parallelism=f"{max(1, args.gpus)} independent replica(s)")
 
 
 def build_planner(cfg):
@@ -338,29 +353,35 @@ def dispatch_timing(pl, out, table_bytes, peaks, steps, flush):
     return dict(dispatch_ms=ms, dispatch_gbs=gbs, dispatch_frac=gbs / peaks["hbm_gbs"])
 
 
-def stream_report(name, peaks, steps=5):
-    """Histogram and reassignment on an HBM-sized routing table (larger than L2): GB/s of each."""
+def stream_report(name, peaks, steps=5, flush=None):
+    """Per-stage times of another workload: GB/s of the histogram and the reassignment (an HBM figure where the
+    routing table is larger than L2; otherwise L2 is flushed between steps and the entry says so)."""
     cfg = W.get_config(name)
     topk = W.routing_topk(cfg, device="cuda")
     pl = build_planner(cfg)
     out = pl.alloc_outputs()
+    b = topk.numel() * 4
+    if 2 * b >= 4 * L2_BYTES:
+        flush = None
     for _ in range(3):
         pl.plan(topk, out)
     pl.set_profiling(True)
     acc = np.zeros(5)
     for _ in range(steps):
+        if flush is not None:
+            flush.zero_()
         pl.plan(topk, out)
         acc += np.array(pl.stage_ms())
     acc /= steps
-    b = topk.numel() * 4
-    rep = dict(workload=name, topk_bytes=b, stages_ms=dict(zip(STAGES, [float(x) for x in acc])),
+    rep = dict(workload=name, topk_bytes=b, table_larger_than_l2=2 * b >= 4 * L2_BYTES,
+               stages_ms=dict(zip(STAGES, [float(x) for x in acc])), ms_per_step=float(acc.sum()),
                histogram_gbs=b / (acc[0] * 1e-3) / 1e9, assign_gbs=2 * b / (acc[4] * 1e-3) / 1e9,
                peak_gbs=peaks["hbm_gbs"], peak_source=peaks["source"],
                remapped_tokens_per_s=cfg.L * cfg.T / (acc[4] * 1e-3),
                plans_per_s=cfg.L / (acc.sum() * 1e-3))
     rep["histogram_frac"] = rep["histogram_gbs"] / peaks["hbm_gbs"]
     rep["assign_frac"] = rep["assign_gbs"] / peaks["hbm_gbs"]
-    rep.update(dispatch_timing(pl, out, b, peaks, steps, None))
+    rep.update(dispatch_timing(pl, out, b, peaks, steps, flush))
     pl.close()
     del topk, out
     torch.cuda.empty_cache()
@@ -379,8 +400,13 @@ def run_reference(args):
     if args.layers > 0:
         cfg = cfg.replace(L=args.layers)
     dev = "cuda" if torch.cuda.is_available() else "cpu"
-    topk = W.routing_topk(cfg, device=dev).cpu().numpy()
     per_step = max(2.0, min(args.cpu_seconds, 60.0 / max(1, args.steps + args.warmup)))
+    # the sample never needs more layers than steps x (layers one step gets through); a quarter of the workload
+    # bounds the input generation when there is no GPU to draw it on
+    n_gen = cfg.L if dev == "cuda" else max(1, min(cfg.L, 12, args.steps + args.warmup))
+    topk = W.routing_topk(cfg, device=dev, layers=range(n_gen)).cpu().numpy()
+    full = cfg
+    cfg = cfg.replace(L=n_gen)
     layers, secs = 0, 0.0
     for i in range(args.warmup + args.steps):
         n, t = oracle_sample(cfg, topk, per_step)
@@ -389,11 +415,13 @@ def run_reference(args):
     value = layers / secs
     line = dict(metric=METRIC, value=value, unit="plans/s", n_gpus=args.gpus,
                 steps=args.steps, warmup=args.warmup, ms_per_step=1e3 * secs / max(1, args.steps),
+                layers_per_step=layers / max(1, args.steps),
                 higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
-                impl="reference", config=dict(workload=args.workload, L=cfg.L, R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k,
-                                              T=cfg.T),
+                impl="reference", config=config_dict(args, full),
                 cpu_baseline=dict(value=value, unit="plans/s", cores=1, kind="oracle",
-                                  sample=f"{layers // max(1, args.steps)} whole layer(s) per step of {cfg.L}"),
+                                  sample=f"{layers / max(1, args.steps):.1f} whole layer(s) per step of the "
+                                         f"{full.L}-layer workload (taken round-robin from its first {n_gen})",
+                                  cpu=cpu_model()),
                 e2e=dict(value=value, unit="plans/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(line))
 
@@ -473,10 +501,21 @@ def run_ours(args):
     host_in = topk.cpu().pin_memory()
     e2r_h = W.expert_to_rank(cfg.E, cfg.R, cfg.e2r_mode)
     C_h = W.cost_matrix(cfg.R, cfg.gpus_per_node, cfg.tiers, cfg.nodes_per_group)
-    depth = max(1, args.e2e_depth)
+    depth = args.e2e_depth if args.e2e_depth > 0 else (4 if topk_bytes <= (64 << 20) else 2)
     kw = dict(R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k, T=cfg.T, e2r=e2r_h, C=C_h, eps=cfg.eps, max_iters=cfg.max_iters,
               tol=cfg.tol)
     names = ("plan", "slot_expert", "slot_tokens", "X", "new_idx", "info")
+    # what the host link allows: one pinned copy of the routing table each way (the two directions of a step can
+    # overlap, so the slower direction bounds a step that moves the table in and the rewritten table out)
+    dev_buf = torch.empty_like(topk)
+    back = torch.empty_like(host_in).pin_memory()
+    link = {}
+    for nm, fn in (("h2d", lambda: dev_buf.copy_(host_in, non_blocking=True)),
+                   ("d2h", lambda: back.copy_(dev_buf, non_blocking=True))):
+        fn(); torch.cuda.synchronize()
+        link[nm] = topk_bytes / (min(timed_steps(fn, 3, None)) * 1e-3) / 1e9
+    del dev_buf, back
+    link_ms = topk_bytes / (min(link.values()) * 1e9) * 1e3
     # (a) one call at a time, pipelined over groups of layers inside the call: every step waits for the previous one
     hp = P.PipelinedHostPlanner(L=cfg.L, groups=args.e2e_groups, **kw)
     host_out = hp.alloc_host_outputs(names)
@@ -531,10 +570,7 @@ def run_ours(args):
         ms_per_step=float(np.mean(ms)), ms_per_step_median=float(np.median(ms)), ms_per_step_min=float(np.min(ms)),
         higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
         data="synthetic",
-        config=dict(workload=args.workload, L=cfg.L, R=cfg.R, E=cfg.E, K=cfg.K, k=cfg.k, T=cfg.T,
-                    eps=cfg.eps, max_iters=cfg.max_iters, tol=cfg.tol,
-                    l2="flushed between steps (256 MiB write)" if need_flush else "inputs larger than L2",
-                    parallelism=f"{world} independent replica(s)"),
+        config=config_dict(args, cfg),
         remapped_tokens_per_s=cfg.L * cfg.T / (float(stage_ms[4]) * 1e-3),
         histogram_tokens_per_s=cfg.L * cfg.T / (float(stage_ms[0]) * 1e-3),
         planned_tokens_per_s=world * cfg.L * cfg.T * args.steps / total_s,
@@ -546,6 +582,10 @@ def run_ours(args):
         roofline=roof, clocks=clocks,
         e2e=dict(value=e2e_value, unit="plans/s", h2d_bytes_per_step=topk_bytes, d2h_bytes_per_step=d2h,
                  ms_per_step=float(np.mean(e2e_ms)), in_flight=depth,
+                 host_link=dict(h2d_gbs=link["h2d"], d2h_gbs=link["d2h"], bound_ms_per_step=link_ms,
+                                bound_value=world * cfg.L / (link_ms * 1e-3),
+                                note="pinned copy of the routing table alone, each way; a step moves it in and the "
+                                     "rewritten table out, so the slower direction bounds the step"),
                  serial_value=serial_value, serial_ms_per_step=float(np.mean(serial_ms)),
                  api=f"StreamingHostPlanner.submit: {'taot_plan_host_block (outputs packed: two copies back)' if packed else 'taot_plan_host'}, {depth} call(s) in flight, each on "
                      f"{len(sp.lanes[0].planners)} group(s) of layers; serial_*: PipelinedHostPlanner.plan_host, one "
@@ -561,7 +601,12 @@ def run_ours(args):
                          for i, s in enumerate(STAGES)}
 
     if world == 1 and not args.no_streams:
+        del host_in, host_outs
+        sp.close()
+        torch.cuda.empty_cache()
+        fl = flush if flush is not None else torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda")
         line["hbm_streams"] = [stream_report(nm, peaks) for nm in ("cfg3", "cfg4") if nm != args.workload]
+        line["l2_resident_workloads"] = [stream_report(nm, peaks, flush=fl) for nm in ("cfg2",) if nm != args.workload]
     if world == 1 and not args.no_cpu_baseline:
         n_layers, secs = oracle_sample(cfg, topk.cpu().numpy(), args.cpu_seconds)
         line["cpu_baseline"] = dict(value=n_layers / secs, unit="plans/s", cores=1, kind="oracle",
@@ -622,8 +667,60 @@ def run_sweep(args):
                           cells=cells)))
 
 
+def free_port() -> int:
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def launch_ranks(args, argv) -> int:
+    """`python bench.py --gpus N` outside a launcher: start the N ranks (one process per GPU) under
+    torch.distributed.run on this node and hand back its exit code.  Rank 0's JSON line goes to this process's
+    stdout unchanged."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + list(argv)
+    env = dict(os.environ)
+    env.setdefault("OMP_NUM_THREADS", "1")
+    return subprocess.call(cmd, env=env)
+
+
+def run_rendezvous_only(args):
+    """The launch path without the planner: join the process group (nccl on GPUs, gloo without), reduce a per-rank
+    time to the slowest rank's as the timed arms do, and print what the ranks saw."""
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    gpu = torch.cuda.is_available()
+    if gpu:
+        torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl" if gpu else "gloo")
+    dev = "cuda" if gpu else "cpu"
+    cfg = rank_config(W.get_config(args.workload), rank)
+    slowest = max_over_ranks(10.0 * (rank + 1), world, dev)
+    seeds = [None] * world
+    if world > 1:
+        dist.all_gather_object(seeds, cfg.seed)
+        dist.barrier()
+    else:
+        seeds = [cfg.seed]
+    if rank == 0:
+        print(json.dumps(dict(rendezvous_only=True, n_gpus=world, gpus_requested=args.gpus,
+                              backend=("nccl" if gpu else "gloo") if world > 1 else None, slowest_ms=slowest,
+                              seeds=seeds, value=whole_job_rate(cfg.L, 1, world, slowest), unit="plans/s")))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     args = parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.sweep:
+        raise SystemExit(launch_ranks(args, sys.argv[1:]))
+    if args.rendezvous_only:
+        run_rendezvous_only(args)
+        return
     if args.sweep:
         run_sweep(args)
         return

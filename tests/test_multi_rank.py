@@ -51,3 +51,36 @@ def test_two_ranks_are_independent_replicas_timed_by_the_slowest():
         assert ret["slowest"] == 20.0
         assert ret["rate"] == world * 1 * 4 / 20e-3            # whole-job plans/s
         assert len(set(ret["seeds"])) == world and len(set(ret["digests"])) == world
+
+
+def test_bench_starts_its_own_ranks_when_asked_for_more_than_one_gpu():
+    """`python bench.py --gpus 2` with no launcher around it must itself start two processes (here on the CPU:
+    gloo, the launch path only) and report a two-rank job."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--rendezvous-only",
+                        "--workload", "cfg1"], capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads([ln for ln in r.stdout.splitlines() if ln.startswith("{")][-1])
+    assert line["n_gpus"] == 2 and line["gpus_requested"] == 2
+    assert line["slowest_ms"] == 20.0                      # the slower of the two ranks' times
+    assert len(set(line["seeds"])) == 2                    # every rank plans its own batch
+
+
+def test_both_arms_describe_the_workload_with_the_same_config_object():
+    import argparse
+    import bench
+    import workloads as W
+    args = argparse.Namespace(workload="cfg4", gpus=1)
+    cfg = W.get_config("cfg4")
+    a = bench.config_dict(args, cfg)
+    b = bench.config_dict(args, bench.rank_config(cfg, 0))
+    assert a == b and a["workload"] == "cfg4" and a["routing_table_bytes"] == 48 * 1048576 * 8 * 4
+    assert a["l2"] == "inputs larger than L2"
+    sys_argv = sys.argv
+    try:
+        sys.argv = ["bench.py"]
+        assert bench.parse_args().workload == "cfg4"       # the default is the largest single-GPU configuration
+    finally:
+        sys.argv = sys_argv
