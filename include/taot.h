@@ -60,7 +60,7 @@ typedef enum {
 enum {
     TAOT_INFO_BAD_INDEX = 1,        /* topk_idx held a value outside [0, E): skipped / copied through */
     TAOT_INFO_SINKHORN_CAP = 2,     /* tolerance mode reached max_iters above tol */
-    TAOT_INFO_NONFINITE = 4,        /* a non-finite value appeared in the Sinkhorn solve */
+    TAOT_INFO_NONFINITE = 4,        /* a non-finite value in the Sinkhorn solve, or in the s / d given to taot_sinkhorn */
     TAOT_INFO_AUCTION_RESIDUAL = 8, /* the auction stopped at auction_max_rounds with tokens unplaced */
     TAOT_INFO_SUPPLY_SCALED = 16,   /* sum(s) > sum(d): supply was scaled by gamma < 1 */
     TAOT_INFO_SINKHORN_SIZE = 32,   /* |hot| * |cold| exceeds the on-chip capacity: plan left at zero */
@@ -168,7 +168,8 @@ int taot_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_n, int32_t
  * TAOT_STATIC_SCRATCH_BYTES that is part of the library image.  Every GPU on which the library is
  * loaded holds that array until the process exits.
  *
- *   d_topk [L,T,k], d_e2r [E] (home rank of each expert, values in [0,R) -- not checked here),
+ *   d_topk [L,T,k], d_e2r [E] (home rank of each expert, values in [0,R); an entry outside that range is
+ *   caught on the device: the expert is left out of d_rank_load and TAOT_INFO_BAD_INDEX is set),
  *   d_n [L,R,E], d_expert_load [L,E], d_rank_load [L,R], d_info [L]: device memory of the caller,
  *   same meaning, layout and overwrite rules as taot_histogram; d_info is OR-ed into.
  *
@@ -207,7 +208,8 @@ int taot_excess_spare(taot_handle_t h, const int32_t* d_rank_load, int32_t B, in
  * `ws` is needed only for R > 256 (the kernel matrix then lives in workspace; batches larger than
  * the handle's L are solved in slices of L).  Problems with |{s>0}| * |{d>0}| beyond the capacity
  * (R*R/4 for R > 128, which disjoint supply/demand ranks never exceed) get TAOT_INFO_SINKHORN_SIZE
- * and a zero plan.
+ * and a zero plan.  A problem whose s or d holds a NaN or an infinity gets TAOT_INFO_NONFINITE, a zero
+ * plan and 0 iterations; the other problems of the batch are not affected.
  */
 int taot_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
                   int32_t* d_iters, float* d_row_err, int32_t* d_info, void* ws, void* stream);
@@ -226,7 +228,8 @@ int taot_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load
                void* stream);
 
 /*
- * Token reassignment ("token routing is adjusted accordingly", Problem Formulation).  Within each
+ * Token reassignment (Problem Formulation: the paper leaves the per-token rule open and fixes only
+ * the counts X; the rule here is earliest entries first, lowest slot first).  Within each
  * (source rank, expert) group, in flat order t*k + j, the slots holding that expert take, lowest
  * slot first, the first X[r][s] entries; an entry so taken is rewritten to E + s, the rest keep e.
  *   d_new_idx [L,T,k] must not alias d_topk.

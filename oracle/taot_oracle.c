@@ -202,7 +202,7 @@ done:
 
 /*
  * The same solve written exactly as the paper prints it: Gibbs kernel M and scaling vectors
- * (u, v) in fp64, a fixed number of iterations, no logarithms.  Valid only while exp(-W/eps)
+ * (u, v) in fp64, an iteration count given in advance, no logarithms.  Valid only while exp(-W/eps)
  * does not underflow; used to cross-check the log-domain routine above.
  */
 void oracle_sinkhorn_gibbs(const float* s32, const float* d32, int32_t R, const float* C32,
@@ -458,8 +458,8 @@ int64_t oracle_auction(int32_t R, int32_t E, int32_t K, const int32_t* n /*[R,E]
 }
 
 /* ------------------------------------------------------------------------------------------
- * Token reassignment given the schedule (the paper only says routing "is adjusted
- * accordingly"; the rule here is: earliest tokens move first, lowest slot fills first).
+ * Token reassignment given the schedule (Problem Formulation: the paper gives the counts X and
+ * no per-token rule; the rule here is: earliest tokens move first, lowest slot fills first).
  * Walk one layer's routing table in flat order q = t*k + j.  For source rank r = src(t) and
  * expert e = topk[q], let ord be the number of earlier entries of the same (r, e).  The slots
  * holding e, in ascending slot order s_1 < s_2 < ..., take the first X[r][s_1] such entries,

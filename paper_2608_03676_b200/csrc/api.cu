@@ -378,7 +378,10 @@ int taot_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B
                                  ws ? reinterpret_cast<float*>(at(ws, h->off_kt)) : nullptr,
                                  static_cast<cudaStream_t>(stream));
     if (a < 0) return a;
-    h->last_launches = a;
+    // s and d are the caller's here: problems with a NaN or an infinity in them are closed out after the solve
+    int g = taot_launch_sinkhorn_guard(h, d_s, d_d, B, d_plan, d_iters, d_row_err, d_info, static_cast<cudaStream_t>(stream));
+    if (g < 0) return g;
+    h->last_launches = a + g;
     return TAOT_OK;
 }
 
@@ -509,6 +512,7 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, voi
 static int plan_on_staging(taot_handle_t h, const int32_t* h_topk, void* d_ws, void* stream, taot_outputs* d)
 {
     const taot_params& p = h->p;
+    if (p.R > 256) return TAOT_ERR_UNSUPPORTED;      // what taot_plan would refuse is refused before the copy is queued
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t NE = (size_t)p.L * p.T * p.k;
     d->n = reinterpret_cast<int32_t*>(at(d_ws, h->hoff_n));

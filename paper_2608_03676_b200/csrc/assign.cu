@@ -1,7 +1,7 @@
 // Token reassignment: rewrite the routing table so that, within every (source rank, expert)
 // group, the earliest entries move to the guest slots holding that expert (lowest slot first,
-// X[r][s] entries each) and the rest stay.  ("Token routing is adjusted accordingly", Problem
-// Formulation; the paper fixes the counts X, this rule fixes which entries.)
+// X[r][s] entries each) and the rest stay.  (Problem Formulation: the paper fixes the counts X
+// and leaves the per-token rule open; this rule fixes which entries move.)
 //
 // Within a (rank, expert) group the slots take consecutive ordinal intervals [0,x1), [x1,x1+x2), ...
 // The chunk counts of the histogram pass say which ordinals of each expert fall into each chunk of
@@ -451,8 +451,11 @@ assign_chunk_kernel(AssignArgs a, int only_split)
     __syncthreads();                                     // table row in place; the barrier is initialised
     if (STAGE) {
         const bool ok = mbar_wait(&bar, 0);
-        if (__syncthreads_or(!ok)) {                     // the copy never landed: report and leave (bounded wait already spent)
-            if (tid == 0) atomicOr(a.info + (int32_t)((id / a.nc) / a.R), TAOT_INFO_INTERNAL);
+        if (__syncthreads_or(!ok)) {                     // the copy has not landed: report, and give the copies still in
+            if (tid == 0) {                              // flight one more bounded wait before the CTA's memory goes away
+                atomicOr(a.info + (int32_t)((id / a.nc) / a.R), TAOT_INFO_INTERNAL);
+                (void)mbar_wait(&bar, 0);
+            }
             return;
         }
     }

@@ -117,7 +117,7 @@ __device__ void excess_spare_row(const int32_t* s_rl, int32_t R, long long* s_to
 __global__ void __launch_bounds__(1024)
 merge_kernel(const int32_t* __restrict__ cc, const int32_t* __restrict__ e2r, int32_t* __restrict__ n,
              int32_t* __restrict__ expert_load, int32_t* __restrict__ rank_load, int32_t* excess,
-             int32_t* spare, float* fs, float* fd, int32_t R, int32_t E, int32_t nc)
+             int32_t* spare, float* fs, float* fd, int32_t R, int32_t E, int32_t nc, int32_t* info)
 {
     extern __shared__ int32_t sh[];                      // el[E], rl[R]
     __shared__ long long s_tot;
@@ -139,7 +139,14 @@ merge_kernel(const int32_t* __restrict__ cc, const int32_t* __restrict__ e2r, in
     for (int e = tid; e < E; e += blockDim.x) {
         const int32_t v = s_el[e];
         expert_load[(int64_t)l * E + e] = v;
-        if (v) atomicAdd(s_rl + e2r[e], v);
+        // a handle's map was validated on the host; a caller-supplied device map (the entry point without a handle)
+        // was not: an expert whose home rank is out of range is left out of the rank loads and flagged
+        const uint32_t home = (uint32_t)e2r[e];
+        if (home < (uint32_t)R) {
+            if (v) atomicAdd(s_rl + home, v);
+        } else if (info) {
+            atomicOr(info + l, TAOT_INFO_BAD_INDEX);
+        }
     }
     __syncthreads();
     for (int r = tid; r < R; r += blockDim.x) rank_load[(int64_t)l * R + r] = s_rl[r];
@@ -196,12 +203,12 @@ int taot_launch_chunk_counts(taot_handle_t h, const int32_t* d_idx, int32_t* d_c
 
 int taot_launch_merge(taot_handle_t h, const int32_t* d_cc, int32_t* d_n, int32_t* d_expert_load,
                       int32_t* d_rank_load, int32_t* d_excess, int32_t* d_spare, float* d_s, float* d_d,
-                      cudaStream_t st)
+                      cudaStream_t st, int32_t* d_info)
 {
     const taot_params& p = h->p;
     const size_t smem = sizeof(int32_t) * (p.E + p.R);
     merge_kernel<<<p.L, 1024, smem, st>>>(d_cc, h->d_e2r, d_n, d_expert_load, d_rank_load, d_excess, d_spare,
-                                          d_s, d_d, p.R, p.E, h->nc);
+                                          d_s, d_d, p.R, p.E, h->nc, d_info);
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
 }
@@ -278,7 +285,8 @@ extern "C" int taot_histogram_static(const int32_t* d_topk, int32_t L, int64_t T
     // with plain stores before the merge kernel reads them.
     int a = taot_launch_histogram(&view, d_topk, counts, d_info, st);
     if (a < 0) return a;
-    int b = taot_launch_merge(&view, counts, d_n, d_expert_load, d_rank_load, nullptr, nullptr, nullptr, nullptr, st);
+    int b = taot_launch_merge(&view, counts, d_n, d_expert_load, d_rank_load, nullptr, nullptr, nullptr, nullptr, st,
+                              d_info);
     if (b < 0) return b;
     return TAOT_OK;
 }

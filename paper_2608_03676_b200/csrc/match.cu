@@ -242,7 +242,7 @@ match_kernel(MatchArgs a)
                         const float t1 = t12[((int64_t)q * 2) * R + r];
                         const float t2 = t12[((int64_t)q * 2 + 1) * R + r];
                         const float sc = __fadd_rn(__fadd_rn((float)gain, t1), t2);
-                        const u64 k64 = ((u64)__float_as_uint(sc) << 32) | (u64)(0xFFFFFFFFu - (uint32_t)e);
+                        const u64 k64 = ((u64)ordered_bits(sc) << 32) | (u64)(0xFFFFFFFFu - (uint32_t)e);   // ordered: a negative preference may give a negative score
                         key = k64 > key ? k64 : key;
                     }
                 }

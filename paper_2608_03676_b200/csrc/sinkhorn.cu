@@ -337,6 +337,38 @@ int taot_launch_sinkhorn_tile(taot_handle_t h, const SinkArgs& a, int32_t B, cud
 int taot_launch_sinkhorn_cluster(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st);
 int taot_launch_sinkhorn_tiered(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st);
 
+// Caller-supplied supply / demand vectors (the stand-alone entry point; inside taot_plan they come from integer
+// loads and are always finite): a problem whose s or d holds a NaN or an infinity has no solution.  One warp per
+// problem rereads the inputs after the solve; for such a problem it clears the plan, reports 0 iterations and sets
+// TAOT_INFO_NONFINITE.  The solve kernels themselves never index with a value derived from s or d and all their
+// loops are bounded, so whatever they computed on that problem before is harmless and is overwritten here.
+__global__ void __launch_bounds__(128)
+sinkhorn_input_guard_kernel(const float* __restrict__ s, const float* __restrict__ d, int32_t B, int32_t R,
+                            float* plan, int32_t* iters, float* row_err, int32_t* info)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t b = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (b >= B) return;
+    bool bad = false;
+    for (int r = lane; r < R; r += 32) bad |= !isfinite(s[b * R + r]) || !isfinite(d[b * R + r]);
+    if (!__any_sync(0xffffffffu, bad)) return;
+    float* out = plan + b * (int64_t)R * R;
+    for (int64_t q = lane; q < (int64_t)R * R; q += 32) out[q] = 0.0f;
+    if (lane == 0) {
+        iters[b] = 0;
+        row_err[b] = 0.0f;
+        atomicOr(info + b, TAOT_INFO_NONFINITE);
+    }
+}
+
+int taot_launch_sinkhorn_guard(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
+                               int32_t* d_iters, float* d_row_err, int32_t* d_info, cudaStream_t st)
+{
+    sinkhorn_input_guard_kernel<<<(B + 3) / 4, 128, 0, st>>>(d_s, d_d, B, h->p.R, d_plan, d_iters, d_row_err, d_info);
+    TAOT_CUDA_OK(cudaGetLastError());
+    return 1;
+}
+
 int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
                          int32_t* d_iters, float* d_row_err, int32_t* d_info, float* d_kt, cudaStream_t st)
 {

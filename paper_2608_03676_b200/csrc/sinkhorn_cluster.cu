@@ -165,6 +165,9 @@ sinkhorn_cluster_kernel(SinkArgs a, int32_t kcap)
         }
         return;
     }
+    // every CTA of the cluster must be running before any of them writes into another's shared memory; the
+    // early return above is taken by all four or by none, so all four reach this barrier
+    cluster.sync();
 
     double sum_st = 0.0;
     for (int i = 0; i < Hn; ++i) sum_st += (double)m.st[i];              // same order in every thread

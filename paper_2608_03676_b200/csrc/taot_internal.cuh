@@ -58,11 +58,13 @@ static inline size_t taot_align_up(size_t x, size_t a) { return (x + a - 1) / a 
 int taot_launch_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_cc, int32_t* d_info, cudaStream_t st);
 int taot_launch_merge(taot_handle_t h, const int32_t* d_cc, int32_t* d_n, int32_t* d_expert_load,
                       int32_t* d_rank_load, int32_t* d_excess, int32_t* d_spare, float* d_s, float* d_d,
-                      cudaStream_t st);
+                      cudaStream_t st, int32_t* d_info = nullptr);
 int taot_launch_excess_spare(taot_handle_t h, const int32_t* d_rank_load, int32_t B, int32_t* d_excess,
                              int32_t* d_spare, float* d_s, float* d_d, cudaStream_t st);
 int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
                          int32_t* d_iters, float* d_row_err, int32_t* d_info, float* d_kt, cudaStream_t st);
+int taot_launch_sinkhorn_guard(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
+                               int32_t* d_iters, float* d_row_err, int32_t* d_info, cudaStream_t st);
 int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load,
                       const int32_t* d_rank_load, const float* d_plan, int32_t* d_slot_expert,
                       int32_t* d_slot_tokens, int32_t* d_X, int32_t* d_rounds, int32_t* d_info,

@@ -260,3 +260,77 @@ def test_smallest_table_and_everything_on_one_expert():
     out = _full_check(cfg, topk, pl)
     assert out["rank_load"][0].max() == cfg.T * cfg.k and (out["slot_expert"][0] >= 0).sum() > 0
     pl.close()
+
+
+@pytest.mark.parametrize("R,B", [(16, 6), (64, 5), (256, 4)])
+def test_non_finite_supply_or_demand_is_flagged_on_its_problem_only(R, B):
+    """taot_sinkhorn takes the caller's s and d: a NaN or an infinity in one entry of one problem must give that
+    problem TAOT_INFO_NONFINITE, a zero plan and 0 iterations, leave its neighbours within tolerance, and trap
+    nothing (the injection is on the host; the kernels only ever see bounded loops and data-independent indices)."""
+    import paper_2608_03676_b200 as P
+    from workloads.configs import SWEEP_TIERS
+    C = W.cost_matrix(R, 8, SWEEP_TIERS, 4)
+    eps = 0.1 * max(SWEEP_TIERS)
+    pl = P.Planner(L=B, R=R, E=R, K=1, k=1, T=R, e2r=torch.arange(R, dtype=torch.int32), C=C, eps=eps,
+                   max_iters=60, tol=0.0)
+    loads = W.sweep_rank_loads(B, R, seed=123, device="cuda")
+    ex, sp, s, d = pl.excess_spare(loads)
+    s = s.clone(); d = d.clone()
+    hot1 = int(torch.nonzero(s[1] > 0)[0]); cold2 = int(torch.nonzero(d[2] > 0)[-1])
+    s[1, hot1] = float("nan")                        # problem 1: NaN supply
+    d[2, cold2] = float("inf")                       # problem 2: infinite demand
+    s[3, int(torch.nonzero(s[3] > 0)[-1])] = float("inf")   # problem 3: infinite supply
+    out = pl.sinkhorn(s, d)
+    torch.cuda.synchronize()
+    plan, iters, err, info = cpu(out["plan"]), cpu(out["iters"]), cpu(out["row_err"]), cpu(out["info"])
+    for b in (1, 2, 3):
+        assert info[b] & P.INFO_NONFINITE and iters[b] == 0 and (plan[b] == 0).all(), b
+    for b in [0] + list(range(4, B)):
+        assert info[b] == 0 and iters[b] == 60
+        check_sinkhorn_problem(cpu(s)[b], cpu(d)[b], C.numpy(), eps, plan[b], iters[b], err[b], 60, 0.0)
+    # the context is alive and the handle still usable
+    again = pl.sinkhorn(s, d)
+    torch.cuda.synchronize()
+    assert torch.equal(again["plan"], out["plan"])
+    pl.close()
+
+
+def test_supports_beyond_the_on_chip_capacity_at_256_ranks_are_flagged_not_solved():
+    """At 256 ranks a problem whose |supply ranks| x |demand ranks| exceeds R*R/4 (possible only with overlapping
+    supports, which the planner's own excess / spare never produce) gets TAOT_INFO_SINKHORN_SIZE and a zero plan;
+    a problem at the limit and an ordinary one in the same batch are solved."""
+    import paper_2608_03676_b200 as P
+    R = 256
+    C = W.cost_matrix(R, 8, (0.0, 1.0, 6.0, 16.0), 4)
+    i = torch.arange(R)
+    C = C + 0.25 * (((i[:, None] * 5 + i[None, :] * 3) % 11 == 0) & (i[:, None] != i[None, :])).float()   # general cost
+    pl = P.Planner(L=3, R=R, E=R, K=1, k=1, T=R, e2r=torch.arange(R, dtype=torch.int32), C=C, eps=1.6,
+                   max_iters=30, tol=0.0)
+    g = torch.Generator().manual_seed(11)
+    s = torch.zeros((3, R)); d = torch.zeros((3, R))
+    s[0, :200] = torch.rand(200, generator=g) * 50 + 1; d[0, 56:] = torch.rand(200, generator=g) * 50 + 1   # 200 x 200 > 16384
+    s[1, :128] = torch.rand(128, generator=g) * 50 + 1; d[1, 128:] = torch.rand(128, generator=g) * 50 + 1  # 128 x 128: the limit
+    s[2, :20] = torch.rand(20, generator=g) * 50 + 1; d[2, 100:160] = torch.rand(60, generator=g) * 50 + 1
+    out = pl.sinkhorn(s.cuda(), d.cuda())
+    torch.cuda.synchronize()
+    plan, iters, err, info = cpu(out["plan"]), cpu(out["iters"]), cpu(out["row_err"]), cpu(out["info"])
+    assert info[0] & P.INFO_SINKHORN_SIZE and (plan[0] == 0).all()
+    for b in (1, 2):
+        assert (info[b] & P.INFO_SINKHORN_SIZE) == 0 and iters[b] == 30
+        check_sinkhorn_problem(s[b].numpy(), d[b].numpy(), C.numpy(), 1.6, plan[b], iters[b], err[b], 30, 0.0)
+    pl.close()
+
+
+def test_negative_preference_entries_order_scores_as_floats_do():
+    """A preference matrix with negative entries makes some Phase-2 scores negative; the integer key the kernel
+    takes its arg-max over must still order them as the floating-point comparison of the oracle does."""
+    cfg = W.get_config("cfg2").replace(L=4)
+    e2r, C = topology(cfg)
+    B = O.default_preference(C.numpy()).copy()
+    g = np.random.default_rng(5)
+    B[g.random(B.shape) < 0.3] *= -400.0             # alpha * B then outweighs any gain: negative scores compete
+    np.fill_diagonal(B, 0.0)
+    topk = W.routing_topk(cfg, device="cuda")
+    pl = make_planner(cfg, B=torch.from_numpy(B))
+    _full_check(cfg, topk, pl, B=B)
+    pl.close()

@@ -184,3 +184,32 @@ def test_tiered_kernel_in_tolerance_mode_beyond_256_ranks(R):
                                400, 1e-6)
     print(f"R={R}: iterations {iters.tolist()}")
     pl.close()
+
+
+@pytest.mark.parametrize("R", [16, 64])
+@pytest.mark.parametrize("B,check", [(1, 1), (4096, 6)])
+@pytest.mark.parametrize("tol", [0.0, 1e-6])
+def test_smallest_and_largest_batch_of_the_sweep(R, B, check, tol):
+    """The two ends of the sweep's batch axis (one problem; 4096 problems, the register-capped batch builds of the
+    one-warp kernels), with a fixed count and in tolerance mode, sampled problems against the oracle."""
+    iters_cap = 300
+    pl, C = _planner(B, R, 0.1, iters=iters_cap, tol=tol)
+    loads = W.sweep_rank_loads(B, R, seed=2000 + R + B, device="cuda")
+    ex, sp, s, d = pl.excess_spare(loads)
+    out = pl.sinkhorn(s, d)
+    torch.cuda.synchronize()
+    plan, iters, err, info = cpu(out["plan"]), cpu(out["iters"]), cpu(out["row_err"]), cpu(out["info"])
+    if tol > 0:
+        assert (iters >= 1).all() and (iters <= iters_cap).all() and ((info & ~2) == 0).all()
+    else:
+        assert (iters == iters_cap).all() and (info == 0).all()
+    sample = sorted(set([0, B - 1] + [int(x) for x in np.linspace(0, B - 1, check)]))
+    if tol > 0 and B > 1:
+        sample = sorted(set(sample + [int(iters.argmax()), int(iters.argmin())]))
+    for b in sample:
+        check_sinkhorn_problem(cpu(s)[b], cpu(d)[b], C.numpy(), 0.1 * max(SWEEP_TIERS), plan[b], iters[b], err[b],
+                               iters_cap, tol)
+    tot = s.double().sum(1)
+    col_viol = (out["plan"].double().sum(1) - d.double()).abs().sum(1)
+    assert bool((col_viol <= 1e-5 * tot).all()) and bool((out["plan"] >= 0).all())
+    pl.close()
