@@ -26,7 +26,7 @@ ABLATE_TOPOLOGY = 2
 _SYMBOLS = [
     "taot_create", "taot_destroy", "taot_workspace_bytes", "taot_host_workspace_bytes",
     "taot_histogram", "taot_histogram_static", "taot_excess_spare", "taot_sinkhorn", "taot_match", "taot_assign",
-    "taot_plan", "taot_plan_host", "taot_host_block_layout", "taot_plan_host_block", "taot_report", "taot_dispatch", "taot_measure_alu_peaks", "taot_measure_latencies", "taot_set_profiling", "taot_get_stage_ms", "taot_last_launch_count",
+    "taot_plan", "taot_plan_host", "taot_host_block_layout", "taot_plan_host_block", "taot_report", "taot_dispatch", "taot_measure_alu_peaks", "taot_measure_latencies", "taot_set_profiling", "taot_get_stage_ms", "taot_get_match_cycles", "taot_last_launch_count",
     "taot_status_string",
 ]
 
@@ -241,8 +241,9 @@ class Planner:
         _check(self.lib.taot_last_launch_count(self.handle, ctypes.byref(c)), "taot_last_launch_count")
         return c.value
 
-    def set_profiling(self, on: bool):
-        _check(self.lib.taot_set_profiling(self.handle, ctypes.c_int32(1 if on else 0)), "taot_set_profiling")
+    def set_profiling(self, on):
+        """False / 0: off.  True / 1: stage events.  2: stage events and the cycle counters of the matching kernel."""
+        _check(self.lib.taot_set_profiling(self.handle, ctypes.c_int32(int(on))), "taot_set_profiling")
 
     def stage_ms(self):
         """Durations (ms) of the five kernels of the last profiled plan call:
@@ -250,6 +251,13 @@ class Planner:
         ms = (ctypes.c_float * 5)()
         _check(self.lib.taot_get_stage_ms(self.handle, ms), "taot_get_stage_ms")
         return [float(x) for x in ms]
+
+    def match_cycles(self) -> torch.Tensor:
+        """SM cycles per part of the matching + auction kernel of the last profiled call, int64 [L, 8] on the host
+        (`taot_get_match_cycles`: set-up, Phase 2, Phase-3 set-up, Phase-3 bids, Phase-3 updates, whole kernel)."""
+        out = torch.zeros((self.L, 8), dtype=torch.int64)
+        _check(self.lib.taot_get_match_cycles(self.handle, _ptr(self.ws), _ptr(out)), "taot_get_match_cycles")
+        return out
 
     # ------------------------------------------------------------------ stages
     def histogram(self, topk: torch.Tensor, info: Optional[torch.Tensor] = None):

@@ -73,6 +73,7 @@ void layout(taot_handle_t h)
     h->off_t12 = take(path * sizeof(float) * (size_t)p.L * p.E * 2 * p.R);
     h->off_kt = take(sizeof(float) * (size_t)p.L * (size_t)h->kcap_global);
     h->off_dc = take(path * sizeof(int32_t) * LR * h->nc * ((size_t)p.E + (size_t)p.R * p.K + 1));
+    h->off_cyc = take(path * sizeof(long long) * (size_t)p.L * 8);
     h->ws_bytes = off;
 
     const size_t S = (size_t)p.R * p.K;
@@ -322,7 +323,7 @@ int taot_host_workspace_bytes(taot_handle_t h, size_t* bytes)
 int taot_set_profiling(taot_handle_t h, int32_t on)
 {
     if (!h) return TAOT_ERR_NULL;
-    h->profiling = on ? 1 : 0;
+    h->profiling = on < 0 ? 0 : (on > 2 ? 2 : on);
     return TAOT_OK;
 }
 
@@ -331,6 +332,15 @@ int taot_get_stage_ms(taot_handle_t h, float* h_ms)
     if (!h || !h_ms) return TAOT_ERR_NULL;
     TAOT_CUDA_OK(cudaEventSynchronize(h->ev[5]));
     for (int i = 0; i < 5; ++i) TAOT_CUDA_OK(cudaEventElapsedTime(h_ms + i, h->ev[i], h->ev[i + 1]));
+    return TAOT_OK;
+}
+
+int taot_get_match_cycles(taot_handle_t h, const void* ws, int64_t* h_cycles)
+{
+    if (!h || !ws || !h_cycles) return TAOT_ERR_NULL;
+    if (h->p.R > 256) return TAOT_ERR_UNSUPPORTED;
+    TAOT_CUDA_OK(cudaMemcpy(h_cycles, static_cast<const char*>(ws) + h->off_cyc, sizeof(int64_t) * (size_t)h->p.L * 8,
+                            cudaMemcpyDeviceToHost));
     return TAOT_OK;
 }
 
@@ -396,7 +406,8 @@ int taot_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load
     if (reinterpret_cast<uintptr_t>(ws) & 255) return TAOT_ERR_ALIGN;
     int a = taot_launch_match(h, d_n, d_expert_load, d_rank_load, d_plan, d_slot_expert, d_slot_tokens, d_X,
                               d_rounds, d_info, reinterpret_cast<int32_t*>(at(ws, h->off_nrem)),
-                              reinterpret_cast<float*>(at(ws, h->off_t12)), static_cast<cudaStream_t>(stream));
+                              reinterpret_cast<float*>(at(ws, h->off_t12)), static_cast<cudaStream_t>(stream),
+                              (h->profiling & 2) ? reinterpret_cast<long long*>(at(ws, h->off_cyc)) : nullptr);
     if (a < 0) return a;
     h->last_launches = a;
     return TAOT_OK;
@@ -496,7 +507,8 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, voi
     TAOT_MARK(3);
     if ((a = taot_launch_match(h, o->n, o->expert_load, o->rank_load, o->plan, o->slot_expert, o->slot_tokens,
                                o->X, o->rounds, o->info, reinterpret_cast<int32_t*>(at(ws, h->off_nrem)),
-                               reinterpret_cast<float*>(at(ws, h->off_t12)), st)) < 0)
+                               reinterpret_cast<float*>(at(ws, h->off_t12)), st,
+                               (h->profiling & 2) ? reinterpret_cast<long long*>(at(ws, h->off_cyc)) : nullptr)) < 0)
         return a;
     total += a;
     TAOT_MARK(4);

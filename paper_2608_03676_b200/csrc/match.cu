@@ -54,6 +54,10 @@ struct MatchArgs {
     int32_t nrem_in_smem;
     int32_t tm_in_smem;
     int32_t big_floats;          // 4-byte words of the shared block that holds the Phase-2 score rows, then nrem
+    long long* cyc;              // [L][8] SM cycles per part of the kernel as thread 0 sees them, or null (profiling aid):
+                                 // 0 set-up, 1 Phase 2, 2 Phase-3 set-up, 3 Phase-3 bids (to the first barrier of a round),
+                                 // 4 Phase-3 updates (to the second barrier), 5 whole kernel, 6 / 7 the busiest thread's own
+                                 // probe and arbitration time in Phase 3
 };
 
 __device__ __forceinline__ uint32_t ordered_bits(float f)
@@ -112,6 +116,7 @@ __device__ __forceinline__ void arbitrate(u64* arb, int target, u64 key)
     }
 }
 
+template <bool TIMED>
 __global__ void __launch_bounds__(1024)
 match_kernel(MatchArgs a)
 {
@@ -152,6 +157,9 @@ match_kernel(MatchArgs a)
     int32_t* nrem = a.nrem_in_smem ? nrem_s : a.nrem_g + l * (int64_t)a.dmax * R;
     float* t12 = a.t12 + l * (int64_t)E * 2 * R;      // global scratch; replaced by shared memory below if the rows fit
 
+    const bool timed = TIMED && tid == 0;
+    const long long c_start = timed ? clock64() : 0;
+    long long c_bid = 0, c_upd = 0, c_probe = 0, c_atom = 0;
     // ---- integer mean, excess, spare (Appendix A.1)
     if (tid == 0) { s_tot = 0; s_cnt = 0; }
     __syncthreads();
@@ -213,6 +221,7 @@ match_kernel(MatchArgs a)
     __syncthreads();
 
     // =========================================================== Phase 2
+    const long long c_p2 = timed ? clock64() : 0;
     int rounds2 = 0;
     int qsh = 0;                                  // lanes per rank in the scan: QS = 2^qsh, the largest power of two <= min(32, NT / R)
     while ((2 << qsh) <= 32 && (2 << qsh) * R <= NT) ++qsh;
@@ -281,6 +290,8 @@ match_kernel(MatchArgs a)
     }
 
     // =========================================================== Phase 3
+    const long long c_p3 = timed ? clock64() : 0;
+    long long c_p3loop = c_p3;
     // compact the experts that sit in some slot; keep their per-rank remaining counts transposed [col][r]
     for (int e = tid; e < E; e += NT) dcol[e] = -1;
     if (tid == 0) s_cnt = 0;
@@ -353,72 +364,118 @@ match_kernel(MatchArgs a)
                     if (mk) { ++nz; wd = w; val = mk; }
                 }
                 tw_word[t * S + s] = nz <= 1 ? wd : -1;
-                tw_mask[t * S + s] = nz <= 1 ? val : 0u;
+                tw_mask[t * S + s] = nz <= 1 ? val : tm[(t * W) * tms];      // several words: the mask of word 0
             }
         }
-        int cur = 0;                             // first list entry (start of a group of equal scores) that may still hit
-        int prev_r = -1;                         // rank whose arbiter entry this slot won last round
-        for (;;) {
-            if (a.auction_max_rounds > 0 && rounds3 >= a.auction_max_rounds) break;
-            if (rounds3 >= cap) break;
-            uint32_t* arb = reinterpret_cast<uint32_t*>(arb_r) + (rounds3 & 1) * R;       // [R] best bid per rank, ping-pong
-            uint32_t* arb_o = reinterpret_cast<uint32_t*>(arb_r) + ((rounds3 & 1) ^ 1) * R;
-            // Step 1: bid for the source rank with the best bonus minus price
+        // Per-slot state of the walk, all in registers: the cursor, and the entry under it decoded once per cursor
+        // position into exactly what a probe needs -- this slot's tier mask for the word it looks at, the addresses of
+        // that word in the expert's availability set and in the win-count set, and the arbitration key of the entry.
+        int cur = 0;                             // list entry (start of a group of equal scores) that may still hit
+        int pw = 0;                              // word the probe looks at
+        uint32_t e_pr = 0u;                      // the list word under the cursor
+        uint32_t e_mk = 0u;                      // tier mask for word pw; 0 for a group of tied entries (generic probe)
+        int e_wd = -1;                           // the tier's only word, or -1 if it spans several
+        const uint32_t* p_av = av;               // &avail[pw][col]
+        uint32_t* p_lv = lvl;                    // &lvl[pw][win count of the entry]
+        uint32_t keyb = 0u;                      // (list position, slot) packed for the arbiter
+        auto load_entry = [&]() {
+            if (cur >= a.nbid) { live = false; e_mk = 0u; return; }     // nothing left this slot could ever bid for
+            e_pr = bid_s[cur];
+            const int t = (int)(e_pr & 0xFFu), wl = (int)((e_pr >> 8) & 0xFFFFu);
+            e_wd = tw_word[t * S + s];
+            pw = e_wd >= 0 ? e_wd : 0;
+            e_mk = (e_pr & 0x80000000u) ? 0u : tw_mask[t * S + s];      // several words: the mask of word 0
+            p_av = av + pw * a.dmax;
+            p_lv = lvl + pw * LS + wl;
+            keyb = ((uint32_t)(a.nbid - cur) << 16) | (uint32_t)(0xFFFF - s);
+        };
+        if (live) load_entry();
+        uint32_t* const arb = reinterpret_cast<uint32_t*>(arb_r);     // [R] best bid per rank; the winner clears its entry
+        long long limit = cap;
+        if (a.auction_max_rounds > 0 && a.auction_max_rounds < limit) limit = a.auction_max_rounds;
+        const int round_limit = (int)(limit < 0x7fffffffLL ? limit : 0x7fffffffLL);
+        if (timed) c_p3loop = clock64();
+        while (rounds3 < round_limit) {
+            const long long c_r0 = TIMED ? clock64() : 0;
+            // Step 1: bid for the source rank with the best bonus minus price.
+            // An entry whose score no other entry shares: while the cursor rests on it its candidate set (tier for this
+            // host AND holding the expert AND this win count) can only shrink -- a rank enters this win count from the
+            // one below, and the entry of the same tier with that lower count comes earlier in the list, so it was found
+            // empty for good before the cursor got here.  Words found empty therefore stay empty: the probe is one word
+            // (the tier's only word, or the word of the last hit), two loads and two ANDs, the same for every lane.
+            uint32_t hit = 0u;
+            uint32_t* p_sel = p_lv;              // win-count word of the rank bid for (the tied groups set their own)
             int r_best = -1;
             if (live) {
-                while (cur < a.nbid) {
-                    int g = cur;
-                    uint32_t pr;
-                    do {
-                        pr = bid_s[g++];
-                        const int t = (int)(pr & 0xFFu), wl = (int)((pr >> 8) & 0xFFFFu);
-                        const int wd = tw_word[t * S + s];
-                        int r;
-                        if (wd >= 0) {
-                            const uint32_t hit = tw_mask[t * S + s] & av[wd * a.dmax] & lvl[wd * LS + wl];
-                            r = hit ? (wd << 5) + __ffs(hit) - 1 : -1;
+                for (;;) {
+                    hit = e_mk & *p_av & *p_lv;
+                    if (hit) { r_best = (pw << 5) + __ffs(hit) - 1; p_sel = p_lv; break; }
+                    if (!(e_pr & 0x80000000u)) { // an empty word: the tier's next word, or the next entry
+                        if (e_wd < 0 && pw + 1 < W) {
+                            ++pw;
+                            e_mk = tm[((int)(e_pr & 0xFFu) * W + pw) * tms];
+                            p_av += a.dmax;
+                            p_lv += LS;
                         } else {
-                            uint32_t cand[kMaxW];
-#pragma unroll
-                            for (int w = 0; w < kMaxW; ++w) cand[w] = (w < W) ? (tm[(t * W + w) * tms] & av[w * a.dmax]) : 0u;
-                            r = first_hit(cand, lvl + wl, LS, W);
+                            ++cur;
+                            load_entry();
                         }
-                        if (r >= 0 && (r_best < 0 || r < r_best)) r_best = r;
-                    } while (pr & 0x80000000u);
-                    if (r_best >= 0) break;
-                    cur = g;                     // the whole group is empty for good
+                    } else {
+                        // a group of entries with one and the same fp32 score: probe every entry, the lowest rank wins
+                        int g = cur;
+                        uint32_t pr;
+                        do {
+                            pr = bid_s[g++];
+                            const int t = (int)(pr & 0xFFu), wl = (int)((pr >> 8) & 0xFFFFu);
+                            const int wd = tw_word[t * S + s];
+                            int r;
+                            if (wd >= 0) {
+                                const uint32_t h1 = tw_mask[t * S + s] & av[wd * a.dmax] & lvl[wd * LS + wl];
+                                r = h1 ? (wd << 5) + __ffs(h1) - 1 : -1;
+                            } else {
+                                uint32_t cand[kMaxW];
+#pragma unroll
+                                for (int w = 0; w < kMaxW; ++w) cand[w] = (w < W) ? (tm[(t * W + w) * tms] & av[w * a.dmax]) : 0u;
+                                r = first_hit(cand, lvl + wl, LS, W);
+                            }
+                            if (r >= 0 && (r_best < 0 || r < r_best)) { r_best = r; p_sel = lvl + (r >> 5) * LS + wl; }
+                        } while (pr & 0x80000000u);
+                        if (r_best >= 0) break;
+                        cur = g;                 // the whole group is empty for good
+                        load_entry();
+                    }
+                    if (!live) break;
                 }
             }
             // Step 2: the rank keeps its best bidder (ties: lowest slot).  The position of a score in the list orders
             // scores exactly as their fp32 values do, so (list position, slot) packs into one 32-bit key and a single
             // native shared-memory atomicMax arbitrates: smaller position = higher score, then the lower slot.
             const bool bids = r_best >= 0;
-            const int rsel = r_best;
-            const uint32_t key = ((uint32_t)(a.nbid - cur) << 16) | (uint32_t)(0xFFFF - s);
-            if (bids) atomicMax(arb + rsel, key);
+            const long long c_rp = TIMED ? clock64() : 0;
+            if (bids) atomicMax(arb + r_best, keyb);
+            if (TIMED) { const long long c_ra = clock64(); c_probe += c_rp - c_r0; c_atom += c_ra - c_rp; }
             if (!__syncthreads_or(bids)) break;
-            if (prev_r >= 0) { arb_o[prev_r] = 0u; prev_r = -1; }     // last round's winner clears the entry it used
-            // Steps 3-4: the winning slot of each rank collects x = min(n, A); holdings, plan and price follow
-            if (bids && arb[rsel] == key) {
-                int32_t* cell = nrem + col * R + rsel;
+            const long long c_r1 = TIMED ? clock64() : 0;
+            // Steps 3-4: the winning slot of each rank collects x = min(n, A); holdings, plan and price follow.  The
+            // rank bid for holds tokens of the expert (its availability bit was set) and the slot still wants some, so
+            // x > 0 and the rank's win count goes from the entry's to the next: its bit moves one word up in lvl.
+            if (bids && arb[r_best] == keyb) {
+                const uint32_t bit = 1u << (r_best & 31);
+                atomicAnd(p_sel, ~bit);
+                atomicOr(p_sel + 1, bit);
+                arb[r_best] = 0u;                // losers of this round compare against their own key: 0 is nobody's
+                int32_t* cell = nrem + col * R + r_best;
                 const int32_t have = *cell;
                 const int32_t x = have < A ? have : A;
-                Xl[(int64_t)rsel * S + s] = x;             // a (rank, slot) pair is served at most once
+                Xl[(int64_t)r_best * S + s] = x;           // a (rank, slot) pair is served at most once
                 *cell = have - x;
                 A -= x;
-                const uint32_t bit = 1u << (rsel & 31);
-                if (have - x == 0) atomicAnd(avail + (rsel >> 5) * a.dmax + col, ~bit);
-                if (x > 0) {
-                    const int w0 = wins[rsel];
-                    wins[rsel] = w0 + 1;
-                    atomicAnd(lvl + (rsel >> 5) * LS + w0, ~bit);
-                    atomicOr(lvl + (rsel >> 5) * LS + w0 + 1, bit);
-                }
-                prev_r = rsel;
+                if (have - x == 0) atomicAnd(avail + (r_best >> 5) * a.dmax + col, ~bit);
                 if (A <= 0) live = false;
             }
             ++rounds3;
             __syncthreads();
+            if (TIMED && timed) { const long long c_r2 = clock64(); c_bid += c_r1 - c_r0; c_upd += c_r2 - c_r1; }
         }
         if (s < S) slot_a[s] = A;
         __syncthreads();
@@ -481,9 +538,23 @@ match_kernel(MatchArgs a)
         if (slot_e[s] >= 0 && slot_a[s] > 0) residual = 1;
     }
     residual = __syncthreads_or(residual);
+    if (TIMED) {                                  // the busiest thread's own probe and arbitration time
+        __shared__ unsigned long long s_mx[2];
+        if (tid == 0) { s_mx[0] = 0; s_mx[1] = 0; }
+        __syncthreads();
+        atomicMax(&s_mx[0], (unsigned long long)c_probe);
+        atomicMax(&s_mx[1], (unsigned long long)c_atom);
+        __syncthreads();
+        c_probe = (long long)s_mx[0]; c_atom = (long long)s_mx[1];
+    }
     if (tid == 0) {
         if (a.rounds) { a.rounds[l * 2] = rounds2; a.rounds[l * 2 + 1] = rounds3; }
         if (residual) atomicOr(a.info + l, TAOT_INFO_AUCTION_RESIDUAL);
+        if (timed) {
+            long long* c = a.cyc + l * 8;
+            c[0] = c_p2 - c_start; c[1] = c_p3 - c_p2; c[2] = c_p3loop - c_p3; c[3] = c_bid; c[4] = c_upd;
+            c[5] = clock64() - c_start; c[6] = c_probe; c[7] = c_atom;
+        }
     }
 }
 
@@ -499,10 +570,11 @@ size_t match_smem_fixed(int R, int E, int K, int dmax, int W, int ntiers)
 int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load,
                       const int32_t* d_rank_load, const float* d_plan, int32_t* d_slot_expert,
                       int32_t* d_slot_tokens, int32_t* d_X, int32_t* d_rounds, int32_t* d_info,
-                      int32_t* d_nrem, float* d_t12, cudaStream_t st)
+                      int32_t* d_nrem, float* d_t12, cudaStream_t st, long long* d_cyc)
 {
     const taot_params& p = h->p;
     MatchArgs a;
+    a.cyc = d_cyc;
     a.n = d_n; a.expert_load = d_expert_load; a.rank_load = d_rank_load; a.plan = d_plan;
     a.e2r = h->d_e2r; a.B = h->d_B; a.rank_off = h->d_rank_off; a.rank_list = h->d_rank_list;
     a.tiermask = h->d_tiermask; a.tierval = h->d_tierval; a.bidlist = h->d_bidlist;
@@ -531,13 +603,15 @@ int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expe
     a.big_floats = (int32_t)(big / 4);
     smem += big;
     if (smem > 227 * 1024) return TAOT_ERR_UNSUPPORTED;
-    TAOT_CUDA_OK(cudaFuncSetAttribute(match_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    TAOT_CUDA_OK(cudaFuncSetAttribute(match_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    if (d_cyc) TAOT_CUDA_OK(cudaFuncSetAttribute(match_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int need = p.R * p.K > p.R ? p.R * p.K : p.R;
     // two threads per slot (or rank): Phase 2 splits each rank's scan over more lanes, and the extra warps cost the
     // auction's barriers less than that saves (measured: 256 threads for 16 and 64 ranks, 512 for 256 ranks x 1 slot)
     int NT = 2 * (((need + 31) / 32) * 32);
     NT = NT < 256 ? 256 : (NT > 1024 ? 1024 : NT);
-    match_kernel<<<p.L, NT, smem, st>>>(a);
+    if (d_cyc) match_kernel<true><<<p.L, NT, smem, st>>>(a);
+    else match_kernel<false><<<p.L, NT, smem, st>>>(a);
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
 }

@@ -41,7 +41,7 @@ struct taot_handle_s {
     int32_t kcap;            // Sinkhorn kernel-matrix capacity in floats per problem (shared memory)
     int64_t kcap_global;     // same, global-memory scratch per problem (R > 256 only), else 0
     // workspace layout (byte offsets)
-    size_t off_cc, off_tabg, off_nbg, off_soff, off_work, off_splits, off_excess, off_spare, off_s, off_d, off_nrem, off_t12, off_kt, off_dc;
+    size_t off_cc, off_tabg, off_nbg, off_soff, off_work, off_splits, off_excess, off_spare, off_s, off_d, off_nrem, off_t12, off_kt, off_dc, off_cyc;
     size_t ws_bytes;
     // host-call staging layout (byte offsets into d_ws of taot_plan_host)
     size_t hoff_topk, hoff_new, hoff_n, hoff_el, hoff_rl, hoff_ex, hoff_sp, hoff_plan, hoff_it, hoff_err,
@@ -68,7 +68,7 @@ int taot_launch_sinkhorn_guard(taot_handle_t h, const float* d_s, const float* d
 int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load,
                       const int32_t* d_rank_load, const float* d_plan, int32_t* d_slot_expert,
                       int32_t* d_slot_tokens, int32_t* d_X, int32_t* d_rounds, int32_t* d_info,
-                      int32_t* d_nrem, float* d_t12, cudaStream_t st);
+                      int32_t* d_nrem, float* d_t12, cudaStream_t st, long long* d_cyc = nullptr);
 int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, void* ws, const int32_t* d_slot_expert,
                        const int32_t* d_X, int32_t* d_new_idx, int32_t* d_info, cudaStream_t st);
 
