@@ -340,13 +340,15 @@ int taot_get_stage_ms(taot_handle_t h, float* h_ms /* [5] */);
  * Where the matching + auction kernel spends its time (a measurement aid; the paper has no counterpart).
  * With profiling level 2 (taot_set_profiling), taot_match / taot_plan make the kernel count SM clock cycles, as thread 0 of each layer's
  * CTA sees them, into `ws`; this call copies them to the host (it synchronises the device).
- *   h_cycles [L][8]: 0 set-up (loads, spill, round-invariant score terms), 1 Phase 2 (Algorithm 2),
+ *   h_cycles [L][16]: 0 set-up (loads, spill, round-invariant score terms), 1 Phase 2 (Algorithm 2),
  *   2 set-up of Phase 3, 3 Phase-3 bids (round start to the barrier after arbitration, summed over rounds),
  *   4 Phase-3 updates (to the barrier that ends the round), 5 the whole kernel, 6 / 7 the probe and the
- *   arbitration time of the thread that spent most on each (its own time, no waiting at barriers).
+ *   arbitration time of the thread that spent most on each (its own time, no waiting at barriers),
+ *   8-11 Phase 2 split: rank scans + arbitration, winners, re-forming the served experts' keys, forming all keys
+ *   once per slot index; 12-15 zero.
  * `ws` is the workspace of the profiled call.  Errors: TAOT_ERR_NULL, TAOT_ERR_UNSUPPORTED (R > 256).
  */
-int taot_get_match_cycles(taot_handle_t h, const void* ws, int64_t* h_cycles /* [L][8] */);
+int taot_get_match_cycles(taot_handle_t h, const void* ws, int64_t* h_cycles /* [L][16] */);
 
 /*
  * Arithmetic ceilings of the current device, measured: FP32 fused multiply-add throughput (TFLOP/s, 2 flops per

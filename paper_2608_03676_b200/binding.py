@@ -253,9 +253,9 @@ class Planner:
         return [float(x) for x in ms]
 
     def match_cycles(self) -> torch.Tensor:
-        """SM cycles per part of the matching + auction kernel of the last profiled call, int64 [L, 8] on the host
+        """SM cycles per part of the matching + auction kernel of the last profiled call, int64 [L, 16] on the host
         (`taot_get_match_cycles`: set-up, Phase 2, Phase-3 set-up, Phase-3 bids, Phase-3 updates, whole kernel)."""
-        out = torch.zeros((self.L, 8), dtype=torch.int64)
+        out = torch.zeros((self.L, 16), dtype=torch.int64)
         _check(self.lib.taot_get_match_cycles(self.handle, _ptr(self.ws), _ptr(out)), "taot_get_match_cycles")
         return out
 

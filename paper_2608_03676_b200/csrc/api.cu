@@ -73,7 +73,7 @@ void layout(taot_handle_t h)
     h->off_t12 = take(path * sizeof(float) * (size_t)p.L * p.E * 2 * p.R);
     h->off_kt = take(sizeof(float) * (size_t)p.L * (size_t)h->kcap_global);
     h->off_dc = take(path * sizeof(int32_t) * LR * h->nc * ((size_t)p.E + (size_t)p.R * p.K + 1));
-    h->off_cyc = take(path * sizeof(long long) * (size_t)p.L * 8);
+    h->off_cyc = take(path * sizeof(long long) * (size_t)p.L * 16);
     h->ws_bytes = off;
 
     const size_t S = (size_t)p.R * p.K;
@@ -339,7 +339,7 @@ int taot_get_match_cycles(taot_handle_t h, const void* ws, int64_t* h_cycles)
 {
     if (!h || !ws || !h_cycles) return TAOT_ERR_NULL;
     if (h->p.R > 256) return TAOT_ERR_UNSUPPORTED;
-    TAOT_CUDA_OK(cudaMemcpy(h_cycles, static_cast<const char*>(ws) + h->off_cyc, sizeof(int64_t) * (size_t)h->p.L * 8,
+    TAOT_CUDA_OK(cudaMemcpy(h_cycles, static_cast<const char*>(ws) + h->off_cyc, sizeof(int64_t) * (size_t)h->p.L * 16,
                             cudaMemcpyDeviceToHost));
     return TAOT_OK;
 }

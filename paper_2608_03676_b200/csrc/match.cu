@@ -54,7 +54,7 @@ struct MatchArgs {
     int32_t nrem_in_smem;
     int32_t tm_in_smem;
     int32_t big_floats;          // 4-byte words of the shared block that holds the Phase-2 score rows, then nrem
-    long long* cyc;              // [L][8] SM cycles per part of the kernel as thread 0 sees them, or null (profiling aid):
+    long long* cyc;              // [L][16] SM cycles per part of the kernel as thread 0 sees them, or null (profiling aid):
                                  // 0 set-up, 1 Phase 2, 2 Phase-3 set-up, 3 Phase-3 bids (to the first barrier of a round),
                                  // 4 Phase-3 updates (to the second barrier), 5 whole kernel, 6 / 7 the busiest thread's own
                                  // probe and arbitration time in Phase 3
@@ -75,7 +75,26 @@ __device__ __forceinline__ u64 warp_max_u64(u64 k)
     return k;
 }
 
+// Barriers over the first `nthreads` threads of the CTA only (a multiple of 32), on hardware barrier 1: the auction's
+// rounds involve the warps that hold slots, the others wait at the CTA-wide barrier that follows the auction.
+__device__ __forceinline__ void bar_part(int nthreads)
+{
+    asm volatile("barrier.sync 1, %0;" ::"r"(nthreads) : "memory");
+}
+__device__ __forceinline__ bool bar_part_or(int nthreads, bool pred)
+{
+    int out;
+    asm volatile(
+        "{\n\t.reg .pred pin, pout;\n\tsetp.ne.s32 pin, %2, 0;\n\tbarrier.red.or.pred pout, 1, %1, pin;\n\t"
+        "selp.s32 %0, 1, 0, pout;\n\t}"
+        : "=r"(out)
+        : "r"(nthreads), "r"((int)pred)
+        : "memory");
+    return out != 0;
+}
+
 constexpr int kMaxW = 8;          // words of a rank bit set: R <= 256
+constexpr size_t kSmemBudget = 224 * 1024;   // dynamic shared memory the kernel plans with (227 KB per CTA less the static part)
 
 // Lowest set bit over kMaxW words (bit index = 32*w + bit), or -1: independent ANDs and a select tree
 // instead of a word-by-word scan, so that a lone warp is not held up by a long dependency chain.
@@ -101,6 +120,7 @@ __device__ __forceinline__ int first_hit(const uint32_t (&cand)[8], const uint32
 // shared-memory arbiter.  key = (score bits << 32) | inverted bidder index; valid bids have key != 0.
 __device__ __forceinline__ void arbitrate(u64* arb, int target, u64 key)
 {
+    // (a hardware match-any on the target was measured several times slower than this loop over distinct targets)
     unsigned todo = __ballot_sync(0xffffffffu, key != 0);
     const uint32_t hi = (uint32_t)(key >> 32), lo = (uint32_t)key;
     const int lane = threadIdx.x & 31;
@@ -148,7 +168,8 @@ match_kernel(MatchArgs a)
     uint32_t* tw_mask = reinterpret_cast<uint32_t*>(tw_word + (a.nbid ? a.ntiers * S : 0));   // [ntiers][S] that word's mask
     int32_t* nrem_s = reinterpret_cast<int32_t*>(tw_mask + (a.nbid ? a.ntiers * S : 0));      // [dmax*R] if it fits
     __shared__ long long s_tot;
-    __shared__ int s_cnt, s_any;
+    __shared__ int s_cnt, s_any, s_ns;
+    __shared__ int s_wcnt[32];
 
     const int32_t* n = a.n + l * (int64_t)R * E;
     const int32_t* el = a.expert_load + l * E;
@@ -159,7 +180,7 @@ match_kernel(MatchArgs a)
 
     const bool timed = TIMED && tid == 0;
     const long long c_start = timed ? clock64() : 0;
-    long long c_bid = 0, c_upd = 0, c_probe = 0, c_atom = 0;
+    long long c_bid = 0, c_upd = 0, c_probe = 0, c_atom = 0, c_scan = 0, c_win = 0, c_row = 0, c_build = 0;
     // ---- integer mean, excess, spare (Appendix A.1)
     if (tid == 0) { s_tot = 0; s_cnt = 0; }
     __syncthreads();
@@ -192,20 +213,39 @@ match_kernel(MatchArgs a)
         const int32_t sp = (int32_t)((hi > 0 ? hi : 0) - (lo > 0 ? lo : 0));
         spill[e] = sp;
         arb_e[e] = 0;
-        if (sp > 0) {
-            const int q = atomicAdd(&s_cnt, 1);
-            hot0[q] = e;
-            hot_home[q] = r;
-        }
     }
     for (int s = tid; s < S; s += NT) { slot_e[s] = -1; slot_a0[s] = 0; }
     __syncthreads();
-    const int nhot0 = s_cnt;
+    // the experts that spill, in ascending index order (position q in this list orders them as the index does, so
+    // "lowest expert on ties" is "lowest position on ties")
+    int nhot0 = 0;
+    for (int base = 0; base < E; base += NT) {
+        const int e = base + tid;
+        const bool hot = e < E && spill[e] > 0;
+        const unsigned bal = __ballot_sync(0xffffffffu, hot);
+        if (lane == 0) s_wcnt[warp] = __popc(bal);
+        __syncthreads();
+        int off = nhot0, tot = 0;
+        for (int w = 0; w < NW; ++w) { const int c = s_wcnt[w]; if (w < warp) off += c; tot += c; }
+        if (hot) {
+            const int q = off + __popc(bal & ((1u << lane) - 1u));
+            hot0[q] = e;
+            hot_home[q] = a.e2r[e];
+        }
+        nhot0 += tot;
+        __syncthreads();
+    }
 
     const float alpha = __fdiv_rn((float)(mean * (long long)R), (float)E);
     const float beta = __fmul_rn(0.1f, alpha);
-    // the rows are only read in Phase 2 and the remaining counts only exist in Phase 3: they share one block
-    if ((int64_t)nhot0 * 2 * R <= (int64_t)a.big_floats) t12 = reinterpret_cast<float*>(nrem_s);
+    // Phase 2 keeps the current score of every (rank, spilling expert) pair as an integer key, row stride odd so that
+    // neither a rank's scan nor an expert's update meets bank conflicts; the keys and the round-invariant rows below
+    // are only used in Phase 2 and the remaining counts only exist in Phase 3: they share one block
+    const int NHs = nhot0 | 1;
+    const bool keyed = nhot0 > 0 && (int64_t)NHs * R <= (int64_t)a.big_floats;
+    uint32_t* keyM = reinterpret_cast<uint32_t*>(nrem_s);                       // [R][NHs]
+    const int64_t key_words = keyed ? (int64_t)NHs * R : 0;
+    if (key_words + (int64_t)nhot0 * 2 * R <= (int64_t)a.big_floats) t12 = reinterpret_cast<float*>(nrem_s) + key_words;
 
     // ---- round-invariant score terms of the spilling experts: t1 = alpha*B, t2 = beta*T/max(excess, eps0)
 #pragma unroll 4
@@ -227,7 +267,99 @@ match_kernel(MatchArgs a)
     while ((2 << qsh) <= 32 && (2 << qsh) * R <= NT) ++qsh;
     const int QS = 1 << qsh;
     const int qs = tid & (QS - 1);
-    for (int kappa = 0; kappa < K; ++kappa) {
+    // score of expert position q on rank r as an ordered integer key, 0 if the pair is no candidate (Algorithm 2's mask:
+    // the expert still spills, r is not its home, it is not on r already); the rank-side conditions (unmatched, spare
+    // left) are tested by the rank's scan
+    auto pair_key = [&](int q, int r, int kappa) -> uint32_t {
+        const int e = hot0[q];
+        const int32_t se = spill[e];
+        bool ok = se > 0 && hot_home[q] != r;
+        for (int kk = 0; kk < kappa; ++kk) ok = ok && (slot_e[r * K + kk] != e);
+        const int32_t sp = spare[r];
+        const int32_t gain = se < sp ? se : sp;
+        const float sc = __fadd_rn(__fadd_rn((float)gain, t12[((int64_t)q * 2) * R + r]), t12[((int64_t)q * 2 + 1) * R + r]);
+        return ok ? ordered_bits(sc) : 0u;
+    };
+    int32_t* served = dcol;                       // [E] positions of the experts served in a round (dcol is Phase 3's)
+    for (int kappa = 0; keyed && kappa < K; ++kappa) {
+        // Between rounds a pair's score changes only when its expert was served (its spill shrank): a rank's spare
+        // changes only when it is matched, and then it is out for this slot index.  So all keys are formed once per
+        // slot index and a round re-forms the rows of the experts it served; a rank's arg-max is one load and one
+        // compare per spilling expert.
+        const long long c_b0 = timed ? clock64() : 0;
+        for (int r = tid; r < R; r += NT) matched[r] = 0;
+        for (int64_t idx = tid; idx < (int64_t)nhot0 * R; idx += NT) {
+            const int q = (int)(idx / R), r = (int)(idx - (int64_t)q * R);
+            keyM[r * NHs + q] = pair_key(q, r, kappa);
+        }
+        if (timed) c_build += clock64() - c_b0;
+        for (;;) {
+            if (tid == 0) { s_any = 0; s_ns = 0; }
+            __syncthreads();
+            const long long c_s0 = timed ? clock64() : 0;
+            // Steps 1-2: every unmatched cold rank takes its best candidate expert (ties: lowest position = lowest index)
+            for (int rb = 0; rb < R; rb += NT >> qsh) {
+                const int r = rb + (tid >> qsh);                  // whole warps stay in the loop for the warp-wide steps
+                u64 key = 0;
+                if (r < R && !matched[r] && spare[r] > 0) {
+                    const uint32_t* row = keyM + r * NHs;
+                    uint32_t bk = 0u;
+                    int bq = 0;
+#pragma unroll 4
+                    for (int q = qs; q < nhot0; q += QS) {      // ascending positions: a strict compare keeps the lowest
+                        const uint32_t k32 = row[q];
+                        if (k32 > bk) { bk = k32; bq = q; }
+                    }
+                    if (bk != 0u) key = ((u64)bk << 32) | (u64)(0xFFFFFFFFu - (uint32_t)bq);
+                }
+                for (int o = 1; o < QS; o <<= 1) {
+                    const u64 other = __shfl_xor_sync(0xffffffffu, key, o);
+                    key = other > key ? other : key;
+                }
+                const int best_q = key != 0 ? (int)(0xFFFFFFFFu - (uint32_t)key) : -1;
+                const bool lead = qs == 0 && r < R;
+                if (lead) {
+                    estar[r] = best_q;
+                    if (key != 0) s_any = 1;
+                }
+                // Step 3: arbitration, best rank per expert (ties: lowest rank)
+                arbitrate(arb_e, best_q >= 0 ? hot0[best_q] : -1,
+                          (key == 0 || !lead) ? 0ull : ((key & 0xFFFFFFFF00000000ull) | (u64)(0xFFFFFFFFu - (uint32_t)r)));
+            }
+            __syncthreads();
+            const long long c_s1 = timed ? clock64() : 0;
+            if (timed) c_scan += c_s1 - c_s0;
+            if (!s_any) break;
+            // Step 4: winners take min(spill, spare)
+            for (int r = tid; r < R; r += NT) {
+                const int q = estar[r];
+                if (q < 0) continue;
+                const int e = hot0[q];
+                if ((uint32_t)arb_e[e] == 0xFFFFFFFFu - (uint32_t)r) {
+                    const int32_t g = spill[e] < spare[r] ? spill[e] : spare[r];
+                    spill[e] -= g;
+                    spare[r] -= g;
+                    matched[r] = 1;
+                    slot_e[r * K + kappa] = e;
+                    slot_a0[r * K + kappa] = g;
+                    served[atomicAdd(&s_ns, 1)] = q;
+                }
+            }
+            __syncthreads();
+            const long long c_s2 = timed ? clock64() : 0;
+            const int ns = s_ns;
+            for (int i = tid; i < ns; i += NT) arb_e[hot0[served[i]]] = 0;
+            for (int idx = tid; idx < ns * R; idx += NT) {
+                const int i = idx / R, r = idx - i * R;
+                const int q = served[i];
+                keyM[r * NHs + q] = pair_key(q, r, kappa);
+            }
+            ++rounds2;
+            if (timed) { const long long c_s3 = clock64(); c_win += c_s2 - c_s1; c_row += c_s3 - c_s2; }
+        }
+        __syncthreads();
+    }
+    for (int kappa = 0; !keyed && kappa < K; ++kappa) {
         for (int r = tid; r < R; r += NT) matched[r] = 0;
         for (;;) {
             if (tid == 0) s_any = 0;
@@ -395,7 +527,8 @@ match_kernel(MatchArgs a)
         if (a.auction_max_rounds > 0 && a.auction_max_rounds < limit) limit = a.auction_max_rounds;
         const int round_limit = (int)(limit < 0x7fffffffLL ? limit : 0x7fffffffLL);
         if (timed) c_p3loop = clock64();
-        while (rounds3 < round_limit) {
+        const int NP = ((S + 31) >> 5) << 5;      // threads that take part in the rounds: the warps holding slots
+        while (tid < NP && rounds3 < round_limit) {
             const long long c_r0 = TIMED ? clock64() : 0;
             // Step 1: bid for the source rank with the best bonus minus price.
             // An entry whose score no other entry shares: while the cursor rests on it its candidate set (tier for this
@@ -454,7 +587,7 @@ match_kernel(MatchArgs a)
             const long long c_rp = TIMED ? clock64() : 0;
             if (bids) atomicMax(arb + r_best, keyb);
             if (TIMED) { const long long c_ra = clock64(); c_probe += c_rp - c_r0; c_atom += c_ra - c_rp; }
-            if (!__syncthreads_or(bids)) break;
+            if (!bar_part_or(NP, bids)) break;
             const long long c_r1 = TIMED ? clock64() : 0;
             // Steps 3-4: the winning slot of each rank collects x = min(n, A); holdings, plan and price follow.  The
             // rank bid for holds tokens of the expert (its availability bit was set) and the slot still wants some, so
@@ -474,7 +607,7 @@ match_kernel(MatchArgs a)
                 if (A <= 0) live = false;
             }
             ++rounds3;
-            __syncthreads();
+            bar_part(NP);
             if (TIMED && timed) { const long long c_r2 = clock64(); c_bid += c_r1 - c_r0; c_upd += c_r2 - c_r1; }
         }
         if (s < S) slot_a[s] = A;
@@ -551,9 +684,11 @@ match_kernel(MatchArgs a)
         if (a.rounds) { a.rounds[l * 2] = rounds2; a.rounds[l * 2 + 1] = rounds3; }
         if (residual) atomicOr(a.info + l, TAOT_INFO_AUCTION_RESIDUAL);
         if (timed) {
-            long long* c = a.cyc + l * 8;
+            long long* c = a.cyc + l * 16;
             c[0] = c_p2 - c_start; c[1] = c_p3 - c_p2; c[2] = c_p3loop - c_p3; c[3] = c_bid; c[4] = c_upd;
             c[5] = clock64() - c_start; c[6] = c_probe; c[7] = c_atom;
+            c[8] = c_scan; c[9] = c_win; c[10] = c_row; c[11] = c_build;
+            for (int i = 12; i < 16; ++i) c[i] = 0;
         }
     }
 }
@@ -593,12 +728,13 @@ int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expe
     const size_t tm_bytes = sizeof(uint32_t) * (size_t)a.ntiers * a.W * p.R * p.K;
     a.tm_in_smem = (a.ntiers > 0 && smem + tm_bytes <= 96 * 1024) ? 1 : 0;
     if (a.tm_in_smem) smem += tm_bytes;
-    a.nrem_in_smem = (smem + nrem_bytes <= 200 * 1024) ? 1 : 0;
-    // one block for the Phase-2 score rows (2 * R floats per spilling expert) and then the remaining counts: as large
-    // as the counts need if those live in shared memory, and at least 64 KB when there is room
+    a.nrem_in_smem = (smem + nrem_bytes <= kSmemBudget) ? 1 : 0;
+    // one block for Phase 2 (per spilling expert R keys and 2 * R floats of round-invariant score rows) and then the
+    // remaining counts: as large as the counts need if those live in shared memory, and as much of what Phase 2 could
+    // use as there is room for
     size_t big = a.nrem_in_smem ? nrem_bytes : 0;
-    const size_t want = sizeof(float) * 2 * (size_t)p.R * (size_t)p.E;
-    const size_t room = 200 * 1024 > smem ? 200 * 1024 - smem : 0;
+    const size_t want = sizeof(float) * ((size_t)p.R * ((size_t)p.E | 1) + 2 * (size_t)p.R * (size_t)p.E);
+    const size_t room = kSmemBudget > smem ? kSmemBudget - smem : 0;
     if (big < want) big = want < room ? want : (room > big ? room : big);
     a.big_floats = (int32_t)(big / 4);
     smem += big;
