@@ -26,7 +26,7 @@ ABLATE_TOPOLOGY = 2
 _SYMBOLS = [
     "taot_create", "taot_destroy", "taot_workspace_bytes", "taot_host_workspace_bytes",
     "taot_histogram", "taot_histogram_static", "taot_excess_spare", "taot_sinkhorn", "taot_match", "taot_assign",
-    "taot_plan", "taot_plan_host", "taot_host_block_layout", "taot_plan_host_block", "taot_report", "taot_dispatch", "taot_measure_alu_peaks", "taot_measure_latencies", "taot_set_profiling", "taot_get_stage_ms", "taot_get_match_cycles", "taot_last_launch_count",
+    "taot_plan", "taot_plan_host", "taot_host_block_layout", "taot_plan_host_block", "taot_report", "taot_dispatch", "taot_measure_alu_peaks", "taot_measure_latencies", "taot_set_profiling", "taot_get_stage_ms", "taot_get_match_cycles", "taot_get_group_trace", "taot_last_launch_count",
     "taot_status_string",
 ]
 
@@ -229,7 +229,9 @@ class Planner:
             info=torch.zeros((L,), dtype=i32, device=self.device))
 
     def plan_launches(self) -> int:
-        """Kernels one `plan` call of this handle enqueues (16-byte aligned routing table, E % 4 == 0)."""
+        """Kernels one `plan` call of this handle enqueues (16-byte aligned routing table, E % 4 == 0) when it plans all
+        layers as one group; a handle that splits a large table into layer groups enqueues them once per group
+        (`last_launch_count()` reports what the last call did)."""
         sms = torch.cuda.get_device_properties(self.device).multi_processor_count
         seg = self.T // self.R * self.k
         chunks = self.L * self.R * ((seg + 16383) // 16384)
@@ -251,6 +253,15 @@ class Planner:
         ms = (ctypes.c_float * 5)()
         _check(self.lib.taot_get_stage_ms(self.handle, ms), "taot_get_stage_ms")
         return [float(x) for x in ms]
+
+    def group_trace(self):
+        """Timeline (ms from the start of the call) of the layer groups of the last plan made with profiling level 3:
+        a list with one [start, histogram, merge, Sinkhorn, matching, reassignment] row per group; [] if the handle
+        plans all layers as one group."""
+        n = ctypes.c_int32(0)
+        ms = (ctypes.c_float * 24)()
+        _check(self.lib.taot_get_group_trace(self.handle, ctypes.byref(n), ms), "taot_get_group_trace")
+        return [[float(ms[g * 6 + i]) for i in range(6)] for g in range(n.value)]
 
     def match_cycles(self) -> torch.Tensor:
         """SM cycles per part of the matching + auction kernel of the last profiled call, int64 [L, 16] on the host

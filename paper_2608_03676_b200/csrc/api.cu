@@ -63,7 +63,7 @@ void layout(taot_handle_t h)
     h->off_tabg = take(path * sizeof(int32_t) * LR * h->nc * (p.E + 20));   // E targets + row tail (assign.cu: kRowTail)
     h->off_nbg = take(path * sizeof(int32_t) * LR * h->nc);
     h->off_soff = take(path * sizeof(int32_t) * LR * h->nc);
-    h->off_work = take(16);
+    h->off_work = take(16 * TAOT_MAX_GROUPS);     // one work counter per layer group
     h->off_splits = take(path * 16 * LR * (size_t)p.R * p.K);
     h->off_excess = take(sizeof(int32_t) * LR);
     h->off_spare = take(sizeof(int32_t) * LR);
@@ -98,6 +98,33 @@ void layout(taot_handle_t h)
 }
 
 inline char* at(void* base, size_t off) { return static_cast<char*>(base) + off; }
+
+// View of handle h on layers [l0, l0 + Lg): every per-layer array of the workspace starts at the group's first layer.
+taot_handle_s* make_view(const taot_handle_s* h, int g, int l0, int Lg)
+{
+    taot_handle_s* v = new taot_handle_s(*h);
+    const taot_params& p = h->p;
+    v->is_view = 1;
+    v->ngroups = 0;
+    v->p.L = Lg;
+    const size_t R = p.R, E = p.E, S = (size_t)p.R * p.K, nc = h->nc, l = (size_t)l0;
+    const size_t dmax = E < S ? E : S;
+    v->off_cc += 4 * l * R * nc * E;
+    v->off_tabg += 4 * l * R * nc * (E + 20);
+    v->off_nbg += 4 * l * R * nc;
+    v->off_soff += 4 * l * R * nc;
+    v->off_work += 16 * (size_t)g;
+    v->off_splits += 16 * l * R * S;
+    v->off_excess += 4 * l * R;
+    v->off_spare += 4 * l * R;
+    v->off_s += 4 * l * R;
+    v->off_d += 4 * l * R;
+    v->off_nrem += 4 * l * dmax * R;
+    v->off_t12 += 4 * l * E * 2 * R;
+    v->off_dc += 4 * l * R * nc * (E + S + 1);
+    v->off_cyc += 8 * l * 16;
+    return v;
+}
 
 }  // namespace
 
@@ -284,10 +311,55 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
     if (rc == TAOT_OK && h->nbid > 0) rc = upload(&h->d_bidlist, bidlist.data(), bidlist.size());
     for (int i = 0; i < 6 && rc == TAOT_OK; ++i)
         if (cudaEventCreate(&h->ev[i]) != cudaSuccess) rc = TAOT_ERR_CUDA;
+    // Layer groups for taot_plan: only where every group's routing table still keeps the memory system busy (more
+    // chunks than three waves of the per-chunk kernels), i.e. where there are bandwidth-bound stages to hide
+    if (rc == TAOT_OK && R <= 256) {
+        int G = TAOT_MAX_GROUPS;
+        if (const char* env = std::getenv("TAOT_PLAN_GROUPS")) {      // tuning knob: cap on the number of groups (1 = never split)
+            const int cap = std::atoi(env);
+            if (cap >= 1 && cap < G) G = cap;
+        }
+        const int64_t chunks_per_layer = (int64_t)R * h->nc;
+        while (G > 1 && (params->L < 2 * G || (params->L / G) * chunks_per_layer <= 3 * (int64_t)h->sm_count)) --G;
+        if (G > 1) {
+            if (cudaEventCreate(&h->ev_fork) != cudaSuccess) rc = TAOT_ERR_CUDA;      // timed: origin of the group trace
+            // Group sizes grow geometrically: a group's chain of latency-bound stages takes about as long whatever its
+            // size, so a group can only finish (and rewrite its part of the table) under the others' chains if it
+            // started earlier by about the time its reassignment takes; the stagger of the starts is the histogram
+            // of the group itself, roughly half as long as its reassignment, hence sizes that grow by about a factor 1.6 (2 : 3 : 5 : 8 measured best on configs 3 and 4).
+            const double wt[TAOT_MAX_GROUPS] = {2.0, 3.0, 5.0, 8.0};
+            double wsum = 0.0;
+            for (int g = 0; g < G; ++g) wsum += wt[g];
+            int l0 = 0;
+            double acc = 0.0;
+            for (int g = 0; g < G && rc == TAOT_OK; ++g) {
+                acc += wt[g];
+                int end = g + 1 == G ? params->L : (int)std::lround(params->L * acc / wsum);
+                if (end < l0 + 1) end = l0 + 1;
+                if (end > params->L - (G - 1 - g)) end = params->L - (G - 1 - g);
+                const int Lg = end - l0;
+                h->group_len[g] = Lg;
+                h->group_l0[g] = l0;
+                l0 += Lg;
+                if (g > 0 && cudaStreamCreateWithFlags(&h->gstream[g], cudaStreamNonBlocking) != cudaSuccess) rc = TAOT_ERR_CUDA;
+                if (rc == TAOT_OK && cudaEventCreateWithFlags(&h->ev_hist[g], cudaEventDisableTiming) != cudaSuccess) rc = TAOT_ERR_CUDA;
+                if (rc == TAOT_OK && cudaEventCreateWithFlags(&h->ev_join[g], cudaEventDisableTiming) != cudaSuccess) rc = TAOT_ERR_CUDA;
+                h->ngroups = g + 1;
+            }
+        }
+    }
     if (rc == TAOT_OK && cudaDeviceSynchronize() != cudaSuccess) rc = TAOT_ERR_CUDA;
     if (rc != TAOT_OK) {
         taot_destroy(h);
         return rc;
+    }
+    // the views copy the finished handle (every device pointer is in place by now)
+    for (int g = 0; g < h->ngroups; ++g) {
+        h->group[g] = make_view(h, g, h->group_l0[g], h->group_len[g]);
+        for (int i = 0; i < 6; ++i) {          // the group's own stage events (profiling level 3)
+            h->group[g]->ev[i] = nullptr;
+            if (cudaEventCreate(&h->group[g]->ev[i]) != cudaSuccess) { taot_destroy(h); return TAOT_ERR_CUDA; }
+        }
     }
     *out = h;
     return TAOT_OK;
@@ -297,6 +369,16 @@ int taot_destroy(taot_handle_t h)
 {
     if (!h) return TAOT_OK;
     cudaDeviceSynchronize();
+    for (int g = 0; g < TAOT_MAX_GROUPS; ++g) {
+        if (h->group[g])
+            for (int i = 0; i < 6; ++i)
+                if (h->group[g]->ev[i]) cudaEventDestroy(h->group[g]->ev[i]);
+        delete h->group[g];                    // a view owns nothing but its stage events
+        if (h->gstream[g]) cudaStreamDestroy(h->gstream[g]);
+        if (h->ev_hist[g]) cudaEventDestroy(h->ev_hist[g]);
+        if (h->ev_join[g]) cudaEventDestroy(h->ev_join[g]);
+    }
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     cudaFree(h->d_e2r); cudaFree(h->d_C); cudaFree(h->d_B); cudaFree(h->d_rowlse0);
     cudaFree(h->d_rank_off); cudaFree(h->d_rank_list); cudaFree(h->d_tierval); cudaFree(h->d_tiermask);
     cudaFree(h->d_tpos); cudaFree(h->d_torder); cudaFree(h->d_tdest); cudaFree(h->d_bidlist);
@@ -323,7 +405,7 @@ int taot_host_workspace_bytes(taot_handle_t h, size_t* bytes)
 int taot_set_profiling(taot_handle_t h, int32_t on)
 {
     if (!h) return TAOT_ERR_NULL;
-    h->profiling = on < 0 ? 0 : (on > 2 ? 2 : on);
+    h->profiling = on < 0 ? 0 : (on > 3 ? 3 : on);
     return TAOT_OK;
 }
 
@@ -341,6 +423,17 @@ int taot_get_match_cycles(taot_handle_t h, const void* ws, int64_t* h_cycles)
     if (h->p.R > 256) return TAOT_ERR_UNSUPPORTED;
     TAOT_CUDA_OK(cudaMemcpy(h_cycles, static_cast<const char*>(ws) + h->off_cyc, sizeof(int64_t) * (size_t)h->p.L * 16,
                             cudaMemcpyDeviceToHost));
+    return TAOT_OK;
+}
+
+int taot_get_group_trace(taot_handle_t h, int32_t* groups, float* h_ms)
+{
+    if (!h || !groups || !h_ms) return TAOT_ERR_NULL;
+    *groups = h->ngroups > 1 ? h->ngroups : 0;
+    for (int g = 0; g < *groups; ++g) {
+        TAOT_CUDA_OK(cudaEventSynchronize(h->group[g]->ev[5]));
+        for (int i = 0; i < 6; ++i) TAOT_CUDA_OK(cudaEventElapsedTime(h_ms + g * 6 + i, h->ev_fork, h->group[g]->ev[i]));
+    }
     return TAOT_OK;
 }
 
@@ -467,19 +560,17 @@ int taot_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_slot_ex
     return TAOT_OK;
 }
 
-int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, void* ws, void* stream)
+}  // extern "C"
+
+namespace {
+
+// The five stages for the layers of one handle (or of one view of it) on one stream.  `hist_after`, if set, is waited for
+// before the chunk histogram starts and `hist_done`, if set, is recorded after it: consecutive layer groups start
+// their bandwidth-bound first stage one after the other instead of sharing the memory system.
+int plan_stages(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, void* ws, cudaStream_t st, bool marks,
+                cudaEvent_t hist_after, cudaEvent_t hist_done, int* launches)
 {
-    if (h && h->p.R > 256) return TAOT_ERR_UNSUPPORTED;      // beyond 256 ranks only Phase 1 is built
-    if (!h || !d_topk || !o || !ws) return TAOT_ERR_NULL;
-    if (!o->n || !o->expert_load || !o->rank_load || !o->plan || !o->sinkhorn_iters || !o->row_err ||
-        !o->slot_expert || !o->slot_tokens || !o->X || !o->new_idx || !o->info)
-        return TAOT_ERR_NULL;
-    if ((reinterpret_cast<uintptr_t>(d_topk) & 3) || (reinterpret_cast<uintptr_t>(o->new_idx) & 3) ||
-        (reinterpret_cast<uintptr_t>(ws) & 255))
-        return TAOT_ERR_ALIGN;
-    if (d_topk == o->new_idx) return TAOT_ERR_PARAM;
     const taot_params& p = h->p;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     int32_t* cc = reinterpret_cast<int32_t*>(at(ws, h->off_cc));
     int32_t* excess = o->excess ? o->excess : reinterpret_cast<int32_t*>(at(ws, h->off_excess));
     int32_t* spare = o->spare ? o->spare : reinterpret_cast<int32_t*>(at(ws, h->off_spare));
@@ -487,10 +578,12 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, voi
     float* fd = reinterpret_cast<float*>(at(ws, h->off_d));
     TAOT_CUDA_OK(cudaMemsetAsync(o->info, 0, sizeof(int32_t) * p.L, st));
     int total = 0, a;
-#define TAOT_MARK(i) if (h->profiling) TAOT_CUDA_OK(cudaEventRecord(h->ev[i], st))
+#define TAOT_MARK(i) if (marks) TAOT_CUDA_OK(cudaEventRecord(h->ev[i], st))
     TAOT_MARK(0);
+    if (hist_after) TAOT_CUDA_OK(cudaStreamWaitEvent(st, hist_after, 0));
     if ((a = taot_launch_histogram(h, d_topk, cc, o->info, st)) < 0) return a;
     total += a;
+    if (hist_done) TAOT_CUDA_OK(cudaEventRecord(hist_done, st));
     TAOT_MARK(1);
     if ((a = taot_launch_merge(h, cc, o->n, o->expert_load, o->rank_load, excess, spare, fs, fd, st)) < 0) return a;
     total += a;
@@ -508,7 +601,7 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, voi
     if ((a = taot_launch_match(h, o->n, o->expert_load, o->rank_load, o->plan, o->slot_expert, o->slot_tokens,
                                o->X, o->rounds, o->info, reinterpret_cast<int32_t*>(at(ws, h->off_nrem)),
                                reinterpret_cast<float*>(at(ws, h->off_t12)), st,
-                               (h->profiling & 2) ? reinterpret_cast<long long*>(at(ws, h->off_cyc)) : nullptr)) < 0)
+                               (marks && (h->profiling & 2)) ? reinterpret_cast<long long*>(at(ws, h->off_cyc)) : nullptr)) < 0)
         return a;
     total += a;
     TAOT_MARK(4);
@@ -516,6 +609,66 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, voi
     total += a;
     TAOT_MARK(5);
 #undef TAOT_MARK
+    *launches += total;
+    return TAOT_OK;
+}
+
+// the outputs of layers [l0, ...) of a call
+taot_outputs outputs_from_layer(const taot_params& p, const taot_outputs* o, int l0)
+{
+    const size_t l = (size_t)l0, R = p.R, E = p.E, S = (size_t)p.R * p.K;
+    taot_outputs g = *o;
+    g.n += l * R * E; g.expert_load += l * E; g.rank_load += l * R;
+    if (g.excess) g.excess += l * R;
+    if (g.spare) g.spare += l * R;
+    g.plan += l * R * R; g.sinkhorn_iters += l; g.row_err += l;
+    g.slot_expert += l * S; g.slot_tokens += l * S; g.X += l * R * S;
+    if (g.rounds) g.rounds += l * 2;
+    g.new_idx += l * (size_t)p.T * p.k; g.info += l;
+    return g;
+}
+
+}  // namespace
+
+extern "C" {
+
+int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, void* ws, void* stream)
+{
+    if (h && h->p.R > 256) return TAOT_ERR_UNSUPPORTED;      // beyond 256 ranks only Phase 1 is built
+    if (!h || !d_topk || !o || !ws) return TAOT_ERR_NULL;
+    if (!o->n || !o->expert_load || !o->rank_load || !o->plan || !o->sinkhorn_iters || !o->row_err ||
+        !o->slot_expert || !o->slot_tokens || !o->X || !o->new_idx || !o->info)
+        return TAOT_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(d_topk) & 3) || (reinterpret_cast<uintptr_t>(o->new_idx) & 3) ||
+        (reinterpret_cast<uintptr_t>(ws) & 255))
+        return TAOT_ERR_ALIGN;
+    if (d_topk == o->new_idx) return TAOT_ERR_PARAM;
+    const taot_params& p = h->p;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int total = 0;
+    if (h->ngroups <= 1 || (h->profiling && h->profiling != 3)) {
+        // one group on the caller's stream (always when stage times are asked for: they are only defined here)
+        const int rc = plan_stages(h, d_topk, o, ws, st, h->profiling != 0, nullptr, nullptr, &total);
+        if (rc != TAOT_OK) return rc;
+        h->last_launches = total;
+        return TAOT_OK;
+    }
+    // Layer groups: group 0 on the caller's stream, the others on the handle's streams, forked from the caller's
+    // stream by an event and joined back into it by one event each; no allocation, no synchronisation, and the fork /
+    // join pattern is what stream capture expects.
+    TAOT_CUDA_OK(cudaEventRecord(h->ev_fork, st));
+    for (int g = 0; g < h->ngroups; ++g) {
+        taot_handle_s* v = h->group[g];
+        const int l0 = h->group_l0[g];
+        cudaStream_t gs = g == 0 ? st : h->gstream[g];
+        if (g > 0) TAOT_CUDA_OK(cudaStreamWaitEvent(gs, h->ev_fork, 0));
+        const taot_outputs go = outputs_from_layer(p, o, l0);
+        const int rc = plan_stages(v, d_topk + (size_t)l0 * p.T * p.k, &go, ws, gs, h->profiling == 3,
+                                   g > 0 ? h->ev_hist[g - 1] : nullptr, g + 1 < h->ngroups ? h->ev_hist[g] : nullptr, &total);
+        if (rc != TAOT_OK) return rc;
+        if (g > 0) TAOT_CUDA_OK(cudaEventRecord(h->ev_join[g], gs));
+    }
+    for (int g = 1; g < h->ngroups; ++g) TAOT_CUDA_OK(cudaStreamWaitEvent(st, h->ev_join[g], 0));
     h->last_launches = total;
     return TAOT_OK;
 }

@@ -430,12 +430,26 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
     }
 }
 
+constexpr size_t kExclusiveSmem = 200 * 1024;
+
 template <int RPL>
 int launch_mw(const SinkArgs& a, const TierCosts& tc, int32_t B, cudaStream_t st)
 {
-    const size_t smem = (size_t)a.R * (2 * sizeof(double) + sizeof(float) + sizeof(int32_t));
-    if (a.tol > 0.0f) sinkhorn_tiered_mw_kernel<RPL, true><<<B, kThreads, smem, st>>>(a, tc, (int64_t)B);
-    else sinkhorn_tiered_mw_kernel<RPL, false><<<B, kThreads, smem, st>>>(a, tc, (int64_t)B);
+    size_t smem = (size_t)a.R * (2 * sizeof(double) + sizeof(float) + sizeof(int32_t));
+    // A batch far smaller than the GPU is one dependent chain per problem: give each problem an SM to itself (a
+    // shared-memory request no two CTAs of any kernel can share an SM with), so that neither the problems of other
+    // launches in flight nor the bandwidth-bound kernels of other layer groups take issue slots from the chain.
+    int dev = 0, sms = 0;
+    TAOT_CUDA_OK(cudaGetDevice(&dev));
+    TAOT_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    if (2 * B <= sms && smem < kExclusiveSmem) smem = kExclusiveSmem;
+    if (a.tol > 0.0f) {
+        TAOT_CUDA_OK(cudaFuncSetAttribute(sinkhorn_tiered_mw_kernel<RPL, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        sinkhorn_tiered_mw_kernel<RPL, true><<<B, kThreads, smem, st>>>(a, tc, (int64_t)B);
+    } else {
+        TAOT_CUDA_OK(cudaFuncSetAttribute(sinkhorn_tiered_mw_kernel<RPL, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        sinkhorn_tiered_mw_kernel<RPL, false><<<B, kThreads, smem, st>>>(a, tc, (int64_t)B);
+    }
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
 }

@@ -13,6 +13,7 @@
 #define TAOT_CHUNK 16384
 #define TAOT_STREAM_THREADS 256            // threads of the streaming kernels: 64 elements each
 #define TAOT_MAX_TIERS 8                   // distinct bonus values the bit-set auction handles
+#define TAOT_MAX_GROUPS 4                  // layer groups taot_plan overlaps on internal streams
 
 struct taot_handle_s {
     taot_params p;
@@ -50,6 +51,17 @@ struct taot_handle_s {
     int32_t last_launches;
     int32_t profiling;
     cudaEvent_t ev[6];
+    // Layer groups of taot_plan (large routing tables only): group g is a view of this handle on layers
+    // [group_l0[g], group_l0[g] + group[g]->p.L) -- same topology pointers, workspace offsets moved to the group's
+    // first layer -- planned on a stream of its own so that the bandwidth-bound stages of one group run under the
+    // latency-bound stages of another.  ngroups <= 1: one group on the caller's stream.
+    int32_t is_view;                           // a view owns nothing
+    int32_t ngroups;
+    taot_handle_s* group[TAOT_MAX_GROUPS];
+    int32_t group_l0[TAOT_MAX_GROUPS];
+    int32_t group_len[TAOT_MAX_GROUPS];
+    cudaStream_t gstream[TAOT_MAX_GROUPS];     // [0] unused: group 0 runs on the caller's stream
+    cudaEvent_t ev_fork, ev_hist[TAOT_MAX_GROUPS], ev_join[TAOT_MAX_GROUPS];
 };
 
 static inline size_t taot_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

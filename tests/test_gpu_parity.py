@@ -228,6 +228,52 @@ def test_plan_is_capturable_in_a_cuda_graph():
     pl.close()
 
 
+def test_layer_groups_on_internal_streams_change_no_bit_and_can_be_captured(monkeypatch):
+    """A routing table large enough to be bandwidth-bound makes taot_plan split the layers into groups on streams of
+    its own (fork / join by events).  The split must change no output, it must be capturable in a CUDA graph, and the
+    group timeline must show every group passing through the five stages in order."""
+    cfg = W.get_config("cfg3").replace(L=9)              # 9 x 64 x 4 chunks: four groups of 1, 2, 2 and 4 layers
+    topk = _routing(cfg)
+    monkeypatch.setenv("TAOT_PLAN_GROUPS", "1")
+    single = make_planner(cfg)
+    monkeypatch.delenv("TAOT_PLAN_GROUPS")
+    pl = make_planner(cfg)
+    want = {k: cpu(v).copy() for k, v in single.plan(topk).items()}
+    out = pl.alloc_outputs()
+    pl.plan(topk, out)
+    torch.cuda.synchronize()
+    n1 = single.last_launch_count()
+    assert 4 * (n1 - 1) <= pl.last_launch_count() <= 4 * n1     # four groups, the same kernels each (a group of one
+                                                                # wave of chunks rewrites it with one kernel fewer)
+    for key, val in out.items():
+        assert (cpu(val) == want[key]).all(), key
+    pl.set_profiling(3)
+    pl.plan(topk, out)
+    trace = pl.group_trace()
+    pl.set_profiling(0)
+    assert len(trace) == 4 and single.group_trace() == []
+    for row in trace:
+        assert all(b >= a for a, b in zip(row, row[1:]))                     # stages in order
+    assert all(trace[g + 1][1] >= trace[g][1] for g in range(3))             # the histograms run one after the other
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        pl.plan(topk, out)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        pl.plan(topk, out)
+    for _ in range(2):
+        for v in out.values():
+            v.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        for key, val in out.items():
+            assert (cpu(val) == want[key]).all(), key
+    pl.close(); single.close()
+
+
 def test_pipelined_host_planner_equals_the_single_call():
     import paper_2608_03676_b200 as P
     cfg = W.get_config("cfg2").replace(L=7)            # 7 layers over 3 groups: uneven split
