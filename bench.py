@@ -266,7 +266,7 @@ def sinkhorn_work(out, cfg):
     return int((2 * hn * cn * np.maximum(it - 1, 0)).sum()), it
 
 
-def roofline_for(stage, ms, cfg, out, peaks, sm_count):
+def roofline_for(stage, ms, cfg, out, peaks, sm_count, match_cyc=None):
     topk_bytes = cfg.L * cfg.T * cfg.k * 4
     hbm = peaks["hbm_gbs"]
     if stage == "histogram":
@@ -318,11 +318,27 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count):
     rounds = out["rounds"].cpu().numpy().astype(np.int64)
     ops = int((rounds[:, 0] * cfg.R * cfg.E + rounds[:, 1] * cfg.R * cfg.S).sum())
     a = ops / (ms * 1e-3) / 1e12
-    return dict(kernel="match_kernel", bound="alu", achieved=a, peak=fp32_peak / 2, unit="Tscore/s",
-                frac=a / (fp32_peak / 2), traffic=None,
-                peak_source="half the FP32 FMA peak: one fp32 score evaluation per lane per clock",
-                note="dependent rounds of masked arg-max; dense score count of the paper's formulation "
-                     "(rounds x R x E and rounds x R x S), latency-bound by construction")
+    d = dict(kernel="match_kernel", bound="alu", achieved=a, peak=fp32_peak / 2, unit="Tscore/s",
+             frac=a / (fp32_peak / 2), traffic=None,
+             peak_source="half the FP32 FMA peak: one fp32 score evaluation per lane per clock",
+             note="dependent rounds of masked arg-max, one CTA per layer; the figure counts the dense scores of the "
+                  "paper's formulation (rounds x R x E and rounds x R x S) and no bandwidth or FLOP bound applies: "
+                  "the stage is as long as its slowest layer's chain of rounds, see `rounds`")
+    if match_cyc is not None:
+        # the layer that takes longest; cycles as thread 0 of its CTA counts them (the counting build of the kernel is
+        # ~10 % slower than the timed one, so the split is given in cycles and as shares, not as a time)
+        w = int(match_cyc[:, 5].argmax())
+        c = match_cyc[w]
+        r2, r3 = int(rounds[w, 0]), int(rounds[w, 1])
+        d["rounds"] = dict(
+            slowest_layer=w, phase2_rounds=r2, phase3_rounds=r3, kernel_cycles=c[5],
+            share=dict(setup=(c[0] + c[2]) / c[5], phase2=c[1] / c[5], phase3_bids=c[3] / c[5], phase3_updates=c[4] / c[5]),
+            phase2_cycles_per_round=c[1] / max(1, r2),
+            phase3_cycles_per_round=dict(bid_to_first_barrier=c[3] / max(1, r3), update_to_second_barrier=c[4] / max(1, r3),
+                                         busiest_thread_probe=c[6] / max(1, r3), busiest_thread_arbitration=c[7] / max(1, r3)),
+            phase2_split=dict(scan_and_arbitration=c[8], winners=c[9], served_rows=c[10], all_keys_per_slot_index=c[11]),
+            ns_per_phase3_round_at_max_clock=(c[3] + c[4]) / max(1, r3) / (peaks["sm_max_mhz"] * 1e-3))
+    return d
 
 
 def rank_config(cfg, rank: int):
@@ -474,9 +490,17 @@ def run_ours(args):
             flush.zero_()
         pl.plan(topk, out)
         stage_ms += np.array(pl.stage_ms())
-    pl.set_profiling(False)
     stage_ms /= args.steps
     clocks = sampler.stop() if rank == 0 else None
+    # where the matching kernel's time goes (cycle counters inside the kernel, one untimed call) and the timeline of
+    # the layer groups of an overlapped call (one untimed call with per-group events)
+    pl.set_profiling(2)
+    pl.plan(topk, out)
+    match_cyc = pl.match_cycles().numpy().astype(np.float64)
+    pl.set_profiling(3)
+    pl.plan(topk, out)
+    group_trace = pl.group_trace()
+    pl.set_profiling(False)
     dispatch = dispatch_timing(pl, out, topk_bytes, peaks, args.steps, flush) if world == 1 else None
 
     total_s = max_over_ranks(sum(ms), world, "cuda") * 1e-3
@@ -560,7 +584,7 @@ def run_ours(args):
         return
 
     dominant = int(np.argmax(stage_ms))
-    roof = roofline_for(STAGES[dominant], float(stage_ms[dominant]), cfg, out, peaks, props.multi_processor_count)
+    roof = roofline_for(STAGES[dominant], float(stage_ms[dominant]), cfg, out, peaks, props.multi_processor_count, match_cyc)
     fma, iters = sinkhorn_work(out, cfg)
     rounds = out["rounds"].cpu().numpy()
     info = out["info"].cpu().numpy()
@@ -597,8 +621,16 @@ def run_ours(args):
     if graph_ms is not None:
         line["cuda_graph"] = dict(ms_per_step=float(np.mean(graph_ms)), value=cfg.L / (float(np.mean(graph_ms)) * 1e-3),
                                   unit="plans/s", note="the same taot_plan call captured once and replayed")
-    line["rooflines"] = {s: roofline_for(s, float(stage_ms[i]), cfg, out, peaks, props.multi_processor_count)
+    line["rooflines"] = {s: roofline_for(s, float(stage_ms[i]), cfg, out, peaks, props.multi_processor_count, match_cyc)
                          for i, s in enumerate(STAGES)}
+    line["stages_note"] = ("stages_ms: the call planned as one group of layers on one stream (stage events); ms_per_step: "
+                           "the call as a user makes it, which for a table this large overlaps layer groups on internal "
+                           "streams, so it is shorter than the sum of the stages")
+    if group_trace:
+        line["layer_groups"] = dict(
+            groups=len(group_trace), columns=["start", "histogram", "merge", "sinkhorn", "match_auction", "assign"],
+            ms_from_call_start=group_trace,
+            note="one untimed call with per-group events: when each group of layers finished each stage")
 
     if world == 1 and not args.no_streams:
         del host_in, host_outs
