@@ -69,6 +69,10 @@ def parse_args():
     ap.add_argument("--sweep-batches", type=int, nargs="+", default=[1, 64, 1024, 4096], help="batch sizes of --sweep")
     ap.add_argument("--sweep-ranks", type=int, nargs="+", default=[8, 16, 64, 256, 1024], help="rank counts of --sweep")
     ap.add_argument("--sweep-eps", type=float, nargs="+", default=[0.1, 0.01], help="eps / max(C) values of --sweep")
+    ap.add_argument("--sweep-general-cost", action="store_true",
+                    help="--sweep with a cost that has no tier structure (a tenth of the entries raised by 0.25): the "
+                         "kernels that hold the kernel matrix, the clusters and the tensor-core products instead of the "
+                         "tier-by-tier sums")
     ap.add_argument("--sweep-max-elems", type=float, default=6e9,
                     help="skip sweep cells whose plan tensor would exceed this many floats")
     return ap.parse_args()
@@ -310,8 +314,8 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count, match_cyc=None):
                     peak_source=fp32_src, flops_per_launch=2 * fma,
                     note="one dependent chain of small mat-vecs per problem and only L problems per call: "
                          "latency-bound; DRAM traffic is ~0.1 MB per launch (ncu); the fp32-FMA fraction is "
-                         "reported, not claimed as the binding limit (see profiles/sweep_config5.md for batches "
-                         "that fill the GPU)")
+                         "reported, not claimed as the binding limit (`bench.py --sweep` times batches that fill "
+                         "the GPU)")
         if latency:
             d["latency"] = latency
         return d
@@ -663,6 +667,13 @@ def run_sweep(args):
     props = torch.cuda.get_device_properties(0)
     alu = P.measure_alu_peaks()
     fp32_peak = alu["fma_tflops"]                    # measured FMA-chain throughput of this GPU
+    # dense TF32 ceiling: the measured bf16 GEMM burst figure times the nominal TF32 : bf16 ratio (1.1 : 2.25 PFLOP/s)
+    try:
+        bf16 = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops"])
+        tf32_src = "measured bf16 GEMM burst x nominal ratio 1.1 / 2.25"
+    except Exception:
+        bf16, tf32_src = 1590.0, "fallback bf16 figure x nominal ratio 1.1 / 2.25"
+    tf32_peak = bf16 * 1.1 / 2.25
     cells = []
     cells_todo = W.sweep_cells(batches=tuple(args.sweep_batches), ranks=tuple(args.sweep_ranks),
                                eps_fracs=tuple(args.sweep_eps))
@@ -671,6 +682,9 @@ def run_sweep(args):
             cells.append(dict(B=B, R=R, eps_frac=eps_frac, skipped="plan tensor larger than --sweep-max-elems"))
             continue
         C = W.cost_matrix(R, 8, SWEEP_TIERS, 4)
+        if args.sweep_general_cost:
+            ii = torch.arange(R)
+            C = C + 0.25 * (((ii[:, None] * 5 + ii[None, :] * 3) % 11 == 0) & (ii[:, None] != ii[None, :])).to(C.dtype)
         pl = P.Planner(L=B, R=R, E=R, K=1, k=1, T=R, e2r=torch.arange(R, dtype=torch.int32), C=C,
                        eps=eps_frac * max(SWEEP_TIERS), max_iters=SWEEP_ITERS, tol=0.0)
         loads = W.sweep_rank_loads(B, R, seed=5000 + R, device="cuda")
@@ -683,6 +697,21 @@ def run_sweep(args):
         tiered = tiered_sums(C, B)
         fma = float(B * tiered_fma_per_iteration(R) * (SWEEP_ITERS - 1)) if tiered else dense_fma
         t = float(np.median(ms)) * 1e-3
+        # the library's rule for the dense products on the tensor cores, mirrored
+        tensor = (not tiered and R > 256 and R % 128 == 0 and B >= 256 and float(C.max()) / (eps_frac * max(SWEEP_TIERS)) <= 20.0
+                  and not os.environ.get("TAOT_NO_TENSOR_CORES"))
+        if tensor:
+            # executed: per iteration two products [R,R] x [R,B], each as three TF32 products
+            tc_flops = 2.0 * 3.0 * 2.0 * R * R * B * SWEEP_ITERS
+            cells.append(dict(B=B, R=R, eps_frac=eps_frac, ms=t * 1e3, plans_per_s=B / t, kernel="tensor-core products (3 x TF32)",
+                              tflops=tc_flops / t / 1e12, frac_tf32_peak=tc_flops / t / 1e12 / tf32_peak,
+                              tf32_peak_tflops=tf32_peak, useful_tflops=tc_flops / 3.0 / t / 1e12,
+                              matrix_equiv_tflops=2 * dense_fma / t / 1e12,
+                              hot_mean=float(hn.mean()), cold_mean=float(cn.mean()), info_or=int(out["info"].max())))
+            pl.close()
+            del out, loads, s, d, ex, sp
+            torch.cuda.empty_cache()
+            continue
         cells.append(dict(B=B, R=R, eps_frac=eps_frac, ms=t * 1e3, plans_per_s=B / t,
                           kernel="tiered sums" if tiered else "kernel matrix",
                           tflops=2 * fma / t / 1e12, frac_fp32_peak=2 * fma / t / 1e12 / fp32_peak,
@@ -694,7 +723,8 @@ def run_sweep(args):
         torch.cuda.empty_cache()
     print(json.dumps(dict(metric="Sinkhorn placement plans/s per (B, R, eps) cell, 500 fixed iterations",
                           unit="plans/s", fp32_peak_tflops=fp32_peak, ex2_peak_tops=alu["ex2_tops"],
-                          fp32_peak_source="measured: taot_measure_alu_peaks",
+                          fp32_peak_source="measured: taot_measure_alu_peaks", tf32_peak_tflops=tf32_peak,
+                          tf32_peak_source=tf32_src, general_cost=bool(args.sweep_general_cost),
                           fp32_peak_derived=props.multi_processor_count * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12,
                           cells=cells)))
 

@@ -208,7 +208,16 @@ int taot_excess_spare(taot_handle_t h, const int32_t* d_rank_load, int32_t B, in
  * `ws` is needed only for R > 256 (the kernel matrix then lives in workspace; batches larger than
  * the handle's L are solved in slices of L).  Problems with |{s>0}| * |{d>0}| beyond the capacity
  * (R*R/4 for R > 128, which disjoint supply/demand ranks never exceed) get TAOT_INFO_SINKHORN_SIZE
- * and a zero plan.  A problem whose s or d holds a NaN or an infinity gets TAOT_INFO_NONFINITE, a zero
+ * and a zero plan.
+ * Kernel choice (all give the same iterates up to fp32 rounding): a cost that depends only on the tier of a rank
+ * pair (same node of 8 / same rail group of 32 / neither) at 256, 512 or 1024 ranks is summed tier by tier; up to
+ * 256 ranks the kernel matrix of a problem lives in registers or shared memory; beyond 256 ranks a batch of at least
+ * 256 problems with a fixed iteration count (tol <= 0) and max(C)/eps <= 20 is solved as dense products
+ * [R,R] x [R,B] on the tensor cores (tcgen05, three TF32 products per term; the row error it reports is the true row
+ * violation of the returned plan, a few 1e-6 of the total mass from accumulator truncation), anything else beyond
+ * 256 ranks by four-CTA clusters.  Environment, read at taot_create / at the call: TAOT_NO_TENSOR_CORES (any value)
+ * keeps the dense path off, TAOT_TC_TILE_N = 64 | 128 | 256 forces its tile width.
+ * A problem whose s or d holds a NaN or an infinity gets TAOT_INFO_NONFINITE, a zero
  * plan and 0 iterations; the other problems of the batch are not affected.
  */
 int taot_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,

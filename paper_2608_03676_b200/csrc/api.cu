@@ -74,6 +74,7 @@ void layout(taot_handle_t h)
     h->off_kt = take(sizeof(float) * (size_t)p.L * (size_t)h->kcap_global);
     h->off_dc = take(path * sizeof(int32_t) * LR * h->nc * ((size_t)p.E + (size_t)p.R * p.K + 1));
     h->off_cyc = take(path * sizeof(long long) * (size_t)p.L * 16);
+    h->off_tc = take((p.R > 256 && p.R % 128 == 0) ? sizeof(float) * taot_sinkhorn_tc_ws_floats(p.R, p.L) : 0);
     h->ws_bytes = off;
 
     const size_t S = (size_t)p.R * p.K;
@@ -277,6 +278,37 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
         for (int j = 0; j < R; ++j) acc += std::exp(-(double)h_C[(size_t)i * R + j] / (double)params->eps - mx);
         lse0[i] = mx + std::log(acc);
     }
+    // Gibbs kernel for the tensor-core solve (more than 256 ranks, no tier structure, exp(-C/eps) well inside fp32):
+    // M and its transpose, each split into two TF32-exact parts (high: low 13 mantissa bits cleared; low: the rest,
+    // again with 13 bits cleared)
+    std::vector<float> gibbs;
+    if (R > 256 && R % 128 == 0 && !h->tier_ok && !std::getenv("TAOT_NO_TENSOR_CORES")) {
+        double worst = 0.0;
+        for (size_t q = 0; q < (size_t)R * R; ++q) worst = std::max(worst, (double)h_C[q] / (double)params->eps);
+        if (worst <= 20.0) {
+            gibbs.resize(4 * (size_t)R * R);
+            auto split = [](float x, float* hi, float* lo) {
+                uint32_t b;
+                std::memcpy(&b, &x, 4);
+                b &= 0xFFFFE000u;
+                std::memcpy(hi, &b, 4);
+                float l = x - *hi;
+                std::memcpy(&b, &l, 4);
+                b &= 0xFFFFE000u;
+                std::memcpy(lo, &b, 4);
+            };
+            for (int i = 0; i < R; ++i)
+                for (int j = 0; j < R; ++j) {
+                    const float m = (float)std::exp(-(double)h_C[(size_t)i * R + j] / (double)params->eps);
+                    float hi, lo;
+                    split(m, &hi, &lo);
+                    gibbs[(size_t)i * R + j] = hi;
+                    gibbs[(size_t)R * R + (size_t)i * R + j] = lo;
+                    gibbs[2 * (size_t)R * R + (size_t)j * R + i] = hi;
+                    gibbs[3 * (size_t)R * R + (size_t)j * R + i] = lo;
+                }
+        }
+    }
     // experts by home rank (CSR), ascending expert index inside a rank
     std::vector<int32_t> off(R + 1, 0), list(E);
     for (int e = 0; e < E; ++e) off[h_e2r[e] + 1]++;
@@ -290,6 +322,7 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
     if (rc == TAOT_OK) rc = upload(&h->d_C, h_C, (size_t)R * R);
     if (rc == TAOT_OK) rc = upload(&h->d_B, B.data(), (size_t)R * R);
     if (rc == TAOT_OK) rc = upload(&h->d_rowlse0, lse0.data(), (size_t)R);
+    if (rc == TAOT_OK && !gibbs.empty()) rc = upload(&h->d_gibbs, gibbs.data(), gibbs.size());
     if (rc == TAOT_OK) rc = upload(&h->d_rank_off, off.data(), (size_t)R + 1);
     if (rc == TAOT_OK) rc = upload(&h->d_rank_list, list.data(), (size_t)E);
     if (rc == TAOT_OK && h->ntiers > 0) rc = upload(&h->d_tierval, tierval.data(), tierval.size());
@@ -379,7 +412,7 @@ int taot_destroy(taot_handle_t h)
         if (h->ev_join[g]) cudaEventDestroy(h->ev_join[g]);
     }
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
-    cudaFree(h->d_e2r); cudaFree(h->d_C); cudaFree(h->d_B); cudaFree(h->d_rowlse0);
+    cudaFree(h->d_e2r); cudaFree(h->d_C); cudaFree(h->d_B); cudaFree(h->d_rowlse0); cudaFree(h->d_gibbs);
     cudaFree(h->d_rank_off); cudaFree(h->d_rank_list); cudaFree(h->d_tierval); cudaFree(h->d_tiermask);
     cudaFree(h->d_tpos); cudaFree(h->d_torder); cudaFree(h->d_tdest); cudaFree(h->d_bidlist);
     for (int i = 0; i < 6; ++i)
@@ -479,7 +512,8 @@ int taot_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B
     if (h->kcap_global > 0 && (!ws || (reinterpret_cast<uintptr_t>(ws) & 255))) return ws ? TAOT_ERR_ALIGN : TAOT_ERR_NULL;
     int a = taot_launch_sinkhorn(h, d_s, d_d, B, d_plan, d_iters, d_row_err, d_info,
                                  ws ? reinterpret_cast<float*>(at(ws, h->off_kt)) : nullptr,
-                                 static_cast<cudaStream_t>(stream));
+                                 static_cast<cudaStream_t>(stream),
+                                 ws ? reinterpret_cast<float*>(at(ws, h->off_tc)) : nullptr);
     if (a < 0) return a;
     // s and d are the caller's here: problems with a NaN or an infinity in them are closed out after the solve
     int g = taot_launch_sinkhorn_guard(h, d_s, d_d, B, d_plan, d_iters, d_row_err, d_info, static_cast<cudaStream_t>(stream));

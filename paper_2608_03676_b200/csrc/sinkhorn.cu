@@ -336,6 +336,7 @@ __global__ void __launch_bounds__(1024) sinkhorn_kernel(SinkArgs a)
 int taot_launch_sinkhorn_tile(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st);
 int taot_launch_sinkhorn_cluster(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st);
 int taot_launch_sinkhorn_tiered(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st);
+int taot_launch_sinkhorn_dense_tc(taot_handle_t h, const SinkArgs& a, int32_t B, float* ws_tc, cudaStream_t st);
 
 // Caller-supplied supply / demand vectors (the stand-alone entry point; inside taot_plan they come from integer
 // loads and are always finite): a problem whose s or d holds a NaN or an infinity has no solution.  One warp per
@@ -370,7 +371,7 @@ int taot_launch_sinkhorn_guard(taot_handle_t h, const float* d_s, const float* d
 }
 
 int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
-                         int32_t* d_iters, float* d_row_err, int32_t* d_info, float* d_kt, cudaStream_t st)
+                         int32_t* d_iters, float* d_row_err, int32_t* d_info, float* d_kt, cudaStream_t st, float* d_tc)
 {
     const taot_params& p = h->p;
     SinkArgs a;
@@ -407,7 +408,12 @@ int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, in
             if (n < 0) return n;
             launched += n;
         } else {
-            // beyond 256 ranks: four-CTA clusters hold the kernel matrix in distributed shared memory; what they hand
+            // beyond 256 ranks, a large batch with a fixed iteration count and a Gibbs kernel inside fp32: the whole
+            // batch as dense products on the tensor cores (complete: nothing is handed on)
+            const int ntc = taot_launch_sinkhorn_dense_tc(h, a, nb, d_tc, st);
+            if (ntc < 0) return ntc;
+            if (ntc > 0) { launched += ntc; continue; }
+            // otherwise four-CTA clusters hold the kernel matrix in distributed shared memory; what they hand
             // back (or everything, if no slice fits) goes to the kernel below with the matrix in workspace
             const int n = taot_launch_sinkhorn_cluster(h, a, nb, st);
             if (n < 0) return n;

@@ -24,6 +24,8 @@ struct taot_handle_s {
     float* d_C;              // [R,R]
     float* d_B;              // [R,R] topology preference (given or derived)
     double* d_rowlse0;       // [R]  LSE_j(-C_ij/eps) over all ranks j: the first u-update with v = 1
+    float* d_gibbs;          // [4][R,R] exp(-C/eps) and its transpose, each as TF32-exact high and low parts (tensor-core
+                             // solve: more than 256 ranks, no tier structure, max C/eps <= 20), else null
     int32_t* d_rank_off;     // [R+1] CSR of experts by home rank
     int32_t* d_rank_list;    // [E]
     uint32_t* d_tiermask;    // [ntiers][W][R hosts] bit r of word w set iff bonus(32w + r -> host) == tierval[t]; null if ntiers == 0
@@ -42,7 +44,7 @@ struct taot_handle_s {
     int32_t kcap;            // Sinkhorn kernel-matrix capacity in floats per problem (shared memory)
     int64_t kcap_global;     // same, global-memory scratch per problem (R > 256 only), else 0
     // workspace layout (byte offsets)
-    size_t off_cc, off_tabg, off_nbg, off_soff, off_work, off_splits, off_excess, off_spare, off_s, off_d, off_nrem, off_t12, off_kt, off_dc, off_cyc;
+    size_t off_cc, off_tabg, off_nbg, off_soff, off_work, off_splits, off_excess, off_spare, off_s, off_d, off_nrem, off_t12, off_kt, off_dc, off_cyc, off_tc;
     size_t ws_bytes;
     // host-call staging layout (byte offsets into d_ws of taot_plan_host)
     size_t hoff_topk, hoff_new, hoff_n, hoff_el, hoff_rl, hoff_ex, hoff_sp, hoff_plan, hoff_it, hoff_err,
@@ -74,7 +76,9 @@ int taot_launch_merge(taot_handle_t h, const int32_t* d_cc, int32_t* d_n, int32_
 int taot_launch_excess_spare(taot_handle_t h, const int32_t* d_rank_load, int32_t B, int32_t* d_excess,
                              int32_t* d_spare, float* d_s, float* d_d, cudaStream_t st);
 int taot_launch_sinkhorn(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
-                         int32_t* d_iters, float* d_row_err, int32_t* d_info, float* d_kt, cudaStream_t st);
+                         int32_t* d_iters, float* d_row_err, int32_t* d_info, float* d_kt, cudaStream_t st,
+                         float* d_tc = nullptr);
+size_t taot_sinkhorn_tc_ws_floats(int32_t R, int32_t B);
 int taot_launch_sinkhorn_guard(taot_handle_t h, const float* d_s, const float* d_d, int32_t B, float* d_plan,
                                int32_t* d_iters, float* d_row_err, int32_t* d_info, cudaStream_t st);
 int taot_launch_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load,

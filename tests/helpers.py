@@ -30,8 +30,9 @@ def make_planner(cfg, **over):
 
 
 def check_sinkhorn_problem(s, d, C, eps, gpu_plan, gpu_iters, gpu_err, max_iters, tol, check_every=1,
-                           eps0=1e-8):
-    """Replay the oracle for exactly the iteration count the GPU reports and compare."""
+                           eps0=1e-8, err_band=STOP_BAND):
+    """Replay the oracle for exactly the iteration count the GPU reports and compare.  err_band: how far the row
+    error the GPU reports may be from the oracle's (the plan's own marginals are always held to MASS_TOL)."""
     R = len(s)
     ref = O.sinkhorn(s, d, C, eps, max(int(gpu_iters), 1) if gpu_iters > 0 else 1, 0.0, 1, eps0,
                      history=(tol > 0 and gpu_iters > 0))
@@ -55,7 +56,7 @@ def check_sinkhorn_problem(s, d, C, eps, gpu_plan, gpu_iters, gpu_err, max_iters
     row_viol_gpu = np.abs(gp.sum(1) - st).sum()
     row_viol_ref = np.abs(T.sum(1) - st).sum()
     assert abs(row_viol_gpu - row_viol_ref) <= MASS_TOL * total
-    assert abs(float(gpu_err) - ref["row_err"]) <= max(STOP_BAND, 1e-3 * ref["row_err"])
+    assert abs(float(gpu_err) - ref["row_err"]) <= max(err_band, 1e-3 * ref["row_err"])
     if tol > 0:
         h = ref["err_hist"]
         n = int(gpu_iters)

@@ -213,3 +213,59 @@ def test_smallest_and_largest_batch_of_the_sweep(R, B, check, tol):
     col_viol = (out["plan"].double().sum(1) - d.double()).abs().sum(1)
     assert bool((col_viol <= 1e-5 * tot).all()) and bool((out["plan"] >= 0).all())
     pl.close()
+
+
+@pytest.mark.parametrize("R,B,iters,check", [(512, 300, 40, (0, 1, 299)), (1024, 256, 30, (0, 255)), (1024, 700, 12, (3, 699))])
+def test_large_batch_with_a_general_cost_takes_the_tensor_core_solve(R, B, iters, check):
+    """More than 256 ranks, a cost without tier structure, a fixed iteration count and a batch of 256 problems or more:
+    the batch is solved as dense products on the tensor cores (three TF32 products per term, four accumulators per
+    tile).  Sampled problems against the oracle, a ragged last tile (B not a multiple of the tile width), and the
+    marginals of every problem.  The tensor cores accumulate with truncation, so the row error this path reports -- the
+    true row violation of the plan it returns -- may sit a few 1e-6 above the oracle's; it is held to the 1e-5 of total
+    mass that bounds any marginal violation, the plan itself to the usual 1e-4 per entry."""
+    from helpers import MASS_TOL
+    pl, C = _planner(B, R, 0.1, iters=iters, general=True)
+    loads = W.sweep_rank_loads(B, R, seed=4000 + R + B, device="cuda")
+    ex, sp, s, d = pl.excess_spare(loads)
+    out = pl.sinkhorn(s, d)
+    torch.cuda.synchronize()
+    assert pl.last_launch_count() == 2 * iters + 4          # prepare, two products per iteration, plan, report, input guard
+    plan, it, err, info = cpu(out["plan"]), cpu(out["iters"]), cpu(out["row_err"]), cpu(out["info"])
+    assert (it == iters).all() and (info == 0).all()
+    for b in check:
+        r = check_sinkhorn_problem(cpu(s)[b], cpu(d)[b], C.numpy(), 0.1 * max(SWEEP_TIERS), plan[b], it[b], err[b], iters,
+                                   0.0, err_band=MASS_TOL)
+        print(f"R={R} problem {b}: max rel err {r['max_rel']:.2e}")
+    tot = s.double().sum(1)
+    col_viol = (out["plan"].double().sum(1) - d.double()).abs().sum(1)
+    assert bool((col_viol <= 1e-5 * tot).all()) and bool((out["plan"] >= 0).all())
+    # the reported row error is the plan's own row violation
+    row_viol = (out["plan"].double().sum(2) - s.double()).abs().sum(1) / tot
+    assert bool(((row_viol - out["row_err"].double()).abs() <= 1e-6 + 1e-4 * row_viol).all())
+    again = pl.sinkhorn(s, d)
+    torch.cuda.synchronize()
+    assert torch.equal(again["plan"], out["plan"]) and torch.equal(again["row_err"], out["row_err"])     # deterministic
+    pl.close()
+
+
+def test_tensor_core_solve_is_not_taken_where_it_does_not_apply():
+    """Tolerance mode, a small batch or a Gibbs kernel near the edge of fp32 stay on the other kernels (launch counts
+    tell which path ran); the results are checked by the cells above and by the sweep cells."""
+    R = 512
+    for kw, B in ((dict(iters=30, tol=1e-6), 300), (dict(iters=30), 8)):
+        pl, C = _planner(B, R, 0.1, general=True, **kw)
+        loads = W.sweep_rank_loads(B, R, seed=9, device="cuda")
+        ex, sp, s, d = pl.excess_spare(loads)
+        pl.sinkhorn(s, d)
+        torch.cuda.synchronize()
+        assert pl.last_launch_count() <= 4
+        pl.close()
+    pl, C = _planner(300, R, 0.01, iters=30, general=True)      # C / eps up to 100: beyond the range the dense form is built for
+    loads = W.sweep_rank_loads(300, R, seed=9, device="cuda")
+    ex, sp, s, d = pl.excess_spare(loads)
+    out = pl.sinkhorn(s, d)
+    torch.cuda.synchronize()
+    assert pl.last_launch_count() <= 4
+    check_sinkhorn_problem(cpu(s)[0], cpu(d)[0], C.numpy(), 0.01 * max(SWEEP_TIERS), cpu(out["plan"])[0], cpu(out["iters"])[0],
+                           cpu(out["row_err"])[0], 30, 0.0)
+    pl.close()
