@@ -221,16 +221,28 @@ def cpu_model():
 
 
 def tiered_sums(C, B):
-    """Does the library take the tier-by-tier Sinkhorn kernel for this cost matrix and batch?  Its rule, applied to
-    the matrix itself: 256, 512 or 1024 ranks and every off-diagonal cost equal to one of three values according to
-    same node of 8 ranks / same rail group of 32 / neither (any batch size)."""
+    """Does the library take the tier-by-tier Sinkhorn kernel for this cost matrix?  Its rule, applied to the matrix
+    itself: 256, 512 or 1024 ranks and every off-diagonal cost equal to one of three values according to same node /
+    same rail group / neither, with the block sizes read off the first row (ranks per node / per group 8 / 32, 4 / 16,
+    4 / 32 or 16 / 32; a two-valued cost has no group tier)."""
     R = C.shape[0]
     if R not in (256, 512, 1024):
         return False
+    row = C[0]
+    node = 1
+    while node < R and bool(row[node] == row[1]):
+        node += 1
+    group = node
+    while group < R and bool(row[group] == row[min(node, R - 1)]):
+        group += 1
+    if group >= R:
+        group = max(32, 2 * node)
+    if (node, group) not in ((8, 32), (4, 16), (4, 32), (16, 32)) or R % group:
+        return False
     i = torch.arange(R)
-    node = (i[:, None] // 8) == (i[None, :] // 8)
-    group = (i[:, None] // 32) == (i[None, :] // 32)
-    want = torch.where(node, C[0, 1], torch.where(group, C[0, 8], C[0, 32]))
+    same_node = (i[:, None] // node) == (i[None, :] // node)
+    same_group = (i[:, None] // group) == (i[None, :] // group)
+    want = torch.where(same_node, row[1], torch.where(same_group, row[node], row[min(group, R - 1)]))
     off = i[:, None] != i[None, :]
     return bool(torch.isfinite(want).all()) and bool((C[off] == want[off]).all())
 

@@ -210,7 +210,7 @@ int taot_excess_spare(taot_handle_t h, const int32_t* d_rank_load, int32_t B, in
  * (R*R/4 for R > 128, which disjoint supply/demand ranks never exceed) get TAOT_INFO_SINKHORN_SIZE
  * and a zero plan.
  * Kernel choice (all give the same iterates up to fp32 rounding): a cost that depends only on the tier of a rank
- * pair (same node of 8 / same rail group of 32 / neither) at 256, 512 or 1024 ranks is summed tier by tier; up to
+ * pair (same node / same rail group / neither; see taot_tier_structure) at 256, 512 or 1024 ranks is summed tier by tier; up to
  * 256 ranks the kernel matrix of a problem lives in registers or shared memory; beyond 256 ranks a batch of at least
  * 256 problems with a fixed iteration count (tol <= 0) and max(C)/eps <= 20 is solved as dense products
  * [R,R] x [R,B] on the tensor cores (tcgen05, three TF32 products per term; the row error it reports is the true row
@@ -357,6 +357,14 @@ int taot_get_stage_ms(taot_handle_t h, float* h_ms /* [5] */);
  * The environment variable TAOT_PLAN_GROUPS (read by taot_create) caps the number of groups; 1 disables the split.
  */
 int taot_get_group_trace(taot_handle_t h, int32_t* groups, float* h_ms /* [4][6] */);
+
+/*
+ * The hierarchy taot_create found in the cost matrix (Appendix A.1 builds W from node membership): if C depends
+ * only on whether two ranks share a node, share a rail group of nodes, or neither, with block sizes the tier-by-tier
+ * Sinkhorn kernels are built for (ranks per node / per group: 8 / 32, 4 / 16, 4 / 32, 16 / 32; 256, 512 or 1024
+ * ranks), *node and *group receive those sizes; otherwise both are 0 and the kernels that hold the kernel matrix run.
+ */
+int taot_tier_structure(taot_handle_t h, int32_t* node, int32_t* group);
 
 /*
  * Where the matching + auction kernel spends its time (a measurement aid; the paper has no counterpart).

@@ -26,7 +26,7 @@ ABLATE_TOPOLOGY = 2
 _SYMBOLS = [
     "taot_create", "taot_destroy", "taot_workspace_bytes", "taot_host_workspace_bytes",
     "taot_histogram", "taot_histogram_static", "taot_excess_spare", "taot_sinkhorn", "taot_match", "taot_assign",
-    "taot_plan", "taot_plan_host", "taot_host_block_layout", "taot_plan_host_block", "taot_report", "taot_dispatch", "taot_measure_alu_peaks", "taot_measure_latencies", "taot_set_profiling", "taot_get_stage_ms", "taot_get_match_cycles", "taot_get_group_trace", "taot_last_launch_count",
+    "taot_plan", "taot_plan_host", "taot_host_block_layout", "taot_plan_host_block", "taot_report", "taot_dispatch", "taot_measure_alu_peaks", "taot_measure_latencies", "taot_set_profiling", "taot_get_stage_ms", "taot_get_match_cycles", "taot_get_group_trace", "taot_tier_structure", "taot_last_launch_count",
     "taot_status_string",
 ]
 
@@ -253,6 +253,13 @@ class Planner:
         ms = (ctypes.c_float * 5)()
         _check(self.lib.taot_get_stage_ms(self.handle, ms), "taot_get_stage_ms")
         return [float(x) for x in ms]
+
+    def tier_structure(self):
+        """(ranks per node, ranks per rail group) of the hierarchy found in the cost matrix, or (0, 0) if the
+        tier-by-tier Sinkhorn kernels do not apply to it."""
+        n = ctypes.c_int32(0); g = ctypes.c_int32(0)
+        _check(self.lib.taot_tier_structure(self.handle, ctypes.byref(n), ctypes.byref(g)), "taot_tier_structure")
+        return n.value, g.value
 
     def group_trace(self):
         """Timeline (ms from the start of the call) of the layer groups of the last plan made with profiling level 3:

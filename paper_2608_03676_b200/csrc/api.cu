@@ -9,6 +9,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "taot_internal.cuh"
 
 namespace {
@@ -253,17 +255,30 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
     // sums be taken tier by tier (sinkhorn_tiered.cu)
     h->tier_ok = 0;
     if (R == 256 || R == 512 || R == 1024) {
-        const float c1 = h_C[1], c2 = h_C[8], c3 = h_C[32];
-        bool ok = std::isfinite(c1) && std::isfinite(c2) && std::isfinite(c3);
-        for (int i = 0; i < R && ok; ++i)
-            for (int j = 0; j < R && ok; ++j) {
-                if (i == j) continue;
-                const float want = (i / 8 == j / 8) ? c1 : ((i / 32 == j / 32) ? c2 : c3);
-                ok = h_C[(size_t)i * R + j] == want;
+        // The block sizes are read off the first row: a node is the run of ranks at rank 0's cheapest off-diagonal
+        // cost, a rail group the run up to the next change (a cost with two values only has no group tier: any group
+        // size then gives the same sums, 32 is taken).  The whole matrix is then checked against that structure.
+        const int shapes[4][2] = {{8, 32}, {4, 16}, {4, 32}, {16, 32}};
+        int node = 1;
+        while (node < R && h_C[node] == h_C[1]) ++node;
+        int group = node;
+        while (group < R && h_C[group] == h_C[node < R ? node : R - 1]) ++group;
+        if (group >= R) group = 32 > node ? 32 : 2 * node;             // two tiers only
+        for (int k = 0; k < 4 && !h->tier_ok; ++k) {
+            if (shapes[k][0] != node || shapes[k][1] != group || R % group != 0) continue;
+            const float c1 = h_C[1], c2 = h_C[node], c3 = h_C[group < R ? group : R - 1];
+            bool ok = std::isfinite(c1) && std::isfinite(c2) && std::isfinite(c3);
+            for (int i = 0; i < R && ok; ++i)
+                for (int j = 0; j < R && ok; ++j) {
+                    if (i == j) continue;
+                    const float want = (i / node == j / node) ? c1 : ((i / group == j / group) ? c2 : c3);
+                    ok = h_C[(size_t)i * R + j] == want;
+                }
+            if (ok) {
+                h->tier_ok = 1;
+                h->tier_node = node; h->tier_group = group;
+                h->tier_cost[0] = c1; h->tier_cost[1] = c2; h->tier_cost[2] = c3;
             }
-        if (ok) {
-            h->tier_ok = 1;
-            h->tier_cost[0] = c1; h->tier_cost[1] = c2; h->tier_cost[2] = c3;
         }
     }
     // first Sinkhorn row update with v = 1 on every rank: log-sum-exp of -C_ij/eps over all j
@@ -470,6 +485,14 @@ int taot_get_group_trace(taot_handle_t h, int32_t* groups, float* h_ms)
     return TAOT_OK;
 }
 
+int taot_tier_structure(taot_handle_t h, int32_t* node, int32_t* group)
+{
+    if (!h || !node || !group) return TAOT_ERR_NULL;
+    *node = h->tier_ok ? h->tier_node : 0;
+    *group = h->tier_ok ? h->tier_group : 0;
+    return TAOT_OK;
+}
+
 int taot_last_launch_count(taot_handle_t h, int32_t* count)
 {
     if (!h || !count) return TAOT_ERR_NULL;
@@ -613,33 +636,55 @@ int plan_stages(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, v
     TAOT_CUDA_OK(cudaMemsetAsync(o->info, 0, sizeof(int32_t) * p.L, st));
     int total = 0, a;
 #define TAOT_MARK(i) if (marks) TAOT_CUDA_OK(cudaEventRecord(h->ev[i], st))
+    // NVTX ranges around the enqueue of each stage (header-only NVTX: free unless a profiler is attached)
+    struct Range {
+        explicit Range(const char* name) { nvtxRangePushA(name); }
+        ~Range() { nvtxRangePop(); }
+    };
     TAOT_MARK(0);
     if (hist_after) TAOT_CUDA_OK(cudaStreamWaitEvent(st, hist_after, 0));
-    if ((a = taot_launch_histogram(h, d_topk, cc, o->info, st)) < 0) return a;
+    {
+        Range r("taot:histogram");
+        if ((a = taot_launch_histogram(h, d_topk, cc, o->info, st)) < 0) return a;
+    }
     total += a;
     if (hist_done) TAOT_CUDA_OK(cudaEventRecord(hist_done, st));
     TAOT_MARK(1);
-    if ((a = taot_launch_merge(h, cc, o->n, o->expert_load, o->rank_load, excess, spare, fs, fd, st)) < 0) return a;
+    {
+        Range r("taot:merge+excess_spare");
+        if ((a = taot_launch_merge(h, cc, o->n, o->expert_load, o->rank_load, excess, spare, fs, fd, st)) < 0) return a;
+    }
     total += a;
     TAOT_MARK(2);
+    nvtxRangePushA("taot:sinkhorn");
     if (p.ablation & TAOT_ABLATE_HINT) {       // Phase 1 switched off: no solve, a zero hint
         TAOT_CUDA_OK(cudaMemsetAsync(o->plan, 0, sizeof(float) * (size_t)p.L * p.R * p.R, st));
         TAOT_CUDA_OK(cudaMemsetAsync(o->sinkhorn_iters, 0, sizeof(int32_t) * p.L, st));
         TAOT_CUDA_OK(cudaMemsetAsync(o->row_err, 0, sizeof(float) * p.L, st));
         a = 0;
     } else if ((a = taot_launch_sinkhorn(h, fs, fd, p.L, o->plan, o->sinkhorn_iters, o->row_err, o->info,
-                                         reinterpret_cast<float*>(at(ws, h->off_kt)), st)) < 0)
+                                         reinterpret_cast<float*>(at(ws, h->off_kt)), st)) < 0) {
+        nvtxRangePop();
         return a;
+    }
+    nvtxRangePop();
     total += a;
     TAOT_MARK(3);
+    nvtxRangePushA("taot:match+auction");
     if ((a = taot_launch_match(h, o->n, o->expert_load, o->rank_load, o->plan, o->slot_expert, o->slot_tokens,
                                o->X, o->rounds, o->info, reinterpret_cast<int32_t*>(at(ws, h->off_nrem)),
                                reinterpret_cast<float*>(at(ws, h->off_t12)), st,
-                               (marks && (h->profiling & 2)) ? reinterpret_cast<long long*>(at(ws, h->off_cyc)) : nullptr)) < 0)
+                               (marks && (h->profiling & 2)) ? reinterpret_cast<long long*>(at(ws, h->off_cyc)) : nullptr)) < 0) {
+        nvtxRangePop();
         return a;
+    }
+    nvtxRangePop();
     total += a;
     TAOT_MARK(4);
-    if ((a = taot_launch_assign(h, d_topk, ws, o->slot_expert, o->X, o->new_idx, o->info, st)) < 0) return a;
+    {
+        Range r("taot:reassignment");
+        if ((a = taot_launch_assign(h, d_topk, ws, o->slot_expert, o->X, o->new_idx, o->info, st)) < 0) return a;
+    }
     total += a;
     TAOT_MARK(5);
 #undef TAOT_MARK

@@ -436,7 +436,7 @@ int launch_rpl(const SinkArgs& a, const TierCosts& tc, int32_t B, cudaStream_t s
 // Launches a tiered-cost kernel if the handle's cost matrix has the node / rail-group structure (checked at
 // taot_create, which also requires 256, 512 or 1024 ranks); returns the number of kernels launched (0: not
 // applicable, the caller takes the general kernels).
-int taot_launch_sinkhorn_tiered_mw(const SinkArgs& a, const float* tier_cost3, int32_t B, cudaStream_t st);
+int taot_launch_sinkhorn_tiered_mw(const SinkArgs& a, const float* tier_cost3, int node, int group, int32_t B, cudaStream_t st);
 
 int taot_launch_sinkhorn_tiered(taot_handle_t h, const SinkArgs& a, int32_t B, cudaStream_t st)
 {
@@ -444,7 +444,9 @@ int taot_launch_sinkhorn_tiered(taot_handle_t h, const SinkArgs& a, int32_t B, c
     // few problems per call: eight warps per problem (a lone warp is bound by the instructions it issues); batches
     // of 256-rank problems that fill the GPU several times over: one warp per problem (fewest instructions per
     // problem).  Beyond 256 ranks the eight-warp kernel wins at every batch size (32 ranks per lane do not fit the registers).
-    if (B < 4 * h->sm_count || h->p.R > 256) return taot_launch_sinkhorn_tiered_mw(a, h->tier_cost, B, st);
+    // (the one-warp kernel is built for nodes of 8 and rail groups of 32 ranks: a lane is a node)
+    if (B < 4 * h->sm_count || h->p.R > 256 || h->tier_node != 8 || h->tier_group != 32)
+        return taot_launch_sinkhorn_tiered_mw(a, h->tier_cost, h->tier_node, h->tier_group, B, st);
     TierCosts tc;
     tc.c1 = (double)h->tier_cost[0] * a.inv_eps;
     tc.c2 = (double)h->tier_cost[1] * a.inv_eps;

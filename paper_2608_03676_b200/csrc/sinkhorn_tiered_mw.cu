@@ -17,8 +17,6 @@ using namespace taot_sk;
 namespace {
 
 constexpr unsigned kFull = 0xffffffffu;
-constexpr int kNode = 8;
-constexpr int kGroup = 32;
 constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 
@@ -35,6 +33,7 @@ struct TierCosts {
     double c1, c2, c3;            // cost / eps of the three tiers off the diagonal
 };
 
+template <int kNode, int kGroup>
 __device__ __forceinline__ double tier_cost(const TierCosts& tc, int i, int j)
 {
     return (i / kNode == j / kNode) ? tc.c1 : ((i / kGroup == j / kGroup) ? tc.c2 : tc.c3);
@@ -62,10 +61,12 @@ struct Exchange {                 // what one warp hands to the others in one ha
     int pad;
 };
 
-template <int RPL, bool TOL>
+// kNode ranks per node, kGroup ranks per rail group (powers of two, kNode < kGroup, a group inside one warp)
+template <int kNode, int kGroup, int RPL, bool TOL>
 __global__ void __launch_bounds__(kThreads)
 sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
 {
+    static_assert(kGroup / RPL <= 32 && kGroup > kNode && kGroup % kNode == 0, "a rail group is held by the lanes of one warp");
     constexpr int LPN = kNode / RPL;              // lanes per node
     constexpr int LPG = kGroup / RPL;             // lanes per rail group
     static_assert(RPL >= 1 && RPL <= kNode && kNode % RPL == 0, "a lane holds part of one node");
@@ -188,13 +189,13 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
             double mx = -INFINITY;
             for (int h = 0; h < Hn; ++h) {
                 const int r = hot[h];
-                const double v = alpha[r] - tier_cost(tc, r, q);
+                const double v = alpha[r] - tier_cost<kNode, kGroup>(tc, r, q);
                 mx = v > mx ? v : mx;
             }
             double acc = 0.0;
             for (int h = 0; h < Hn; ++h) {
                 const int r = hot[h];
-                acc += (double)exp_split(alpha[r] - tier_cost(tc, r, q) - mx);
+                acc += (double)exp_split(alpha[r] - tier_cost<kNode, kGroup>(tc, r, q) - mx);
             }
             bj = log((double)a.d[b * R + q]) - (mx + log(acc));
         }
@@ -416,7 +417,7 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
             const float fg = fgs[j];
             float val = 0.0f;
             if (fg > 0.0f) {
-                val = exp_split(al + beta[j] - tier_cost(tc, row, j)) * fg;
+                val = exp_split(al + beta[j] - tier_cost<kNode, kGroup>(tc, row, j)) * fg;
                 if (!isfinite(val)) nonfinite = 1;
             }
             orow[j] = val;
@@ -432,7 +433,7 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
 
 constexpr size_t kExclusiveSmem = 200 * 1024;
 
-template <int RPL>
+template <int kNode, int kGroup, int RPL>
 int launch_mw(const SinkArgs& a, const TierCosts& tc, int32_t B, cudaStream_t st)
 {
     size_t smem = (size_t)a.R * (2 * sizeof(double) + sizeof(float) + sizeof(int32_t));
@@ -444,29 +445,40 @@ int launch_mw(const SinkArgs& a, const TierCosts& tc, int32_t B, cudaStream_t st
     TAOT_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     if (2 * B <= sms && smem < kExclusiveSmem) smem = kExclusiveSmem;
     if (a.tol > 0.0f) {
-        TAOT_CUDA_OK(cudaFuncSetAttribute(sinkhorn_tiered_mw_kernel<RPL, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        sinkhorn_tiered_mw_kernel<RPL, true><<<B, kThreads, smem, st>>>(a, tc, (int64_t)B);
+        TAOT_CUDA_OK(cudaFuncSetAttribute(sinkhorn_tiered_mw_kernel<kNode, kGroup, RPL, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        sinkhorn_tiered_mw_kernel<kNode, kGroup, RPL, true><<<B, kThreads, smem, st>>>(a, tc, (int64_t)B);
     } else {
-        TAOT_CUDA_OK(cudaFuncSetAttribute(sinkhorn_tiered_mw_kernel<RPL, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        sinkhorn_tiered_mw_kernel<RPL, false><<<B, kThreads, smem, st>>>(a, tc, (int64_t)B);
+        TAOT_CUDA_OK(cudaFuncSetAttribute(sinkhorn_tiered_mw_kernel<kNode, kGroup, RPL, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        sinkhorn_tiered_mw_kernel<kNode, kGroup, RPL, false><<<B, kThreads, smem, st>>>(a, tc, (int64_t)B);
     }
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
 }
 
+template <int kNode, int kGroup>
+int launch_mw_ranks(const SinkArgs& a, const TierCosts& tc, int32_t B, cudaStream_t st)
+{
+    switch (a.R) {
+        case 256: return launch_mw<kNode, kGroup, 1>(a, tc, B, st);
+        case 512: if constexpr (kNode >= 2) return launch_mw<kNode, kGroup, 2>(a, tc, B, st); else return 0;
+        case 1024: if constexpr (kNode >= 4) return launch_mw<kNode, kGroup, 4>(a, tc, B, st); else return 0;
+        default: return 0;
+    }
+}
+
 }  // namespace
 
-// Eight warps per problem (256, 512 or 1024 ranks); the caller has checked that the cost is tiered.
-int taot_launch_sinkhorn_tiered_mw(const SinkArgs& a, const float* tier_cost3, int32_t B, cudaStream_t st)
+// Eight warps per problem (256, 512 or 1024 ranks); the caller has checked that the cost is tiered with `node` ranks
+// per node and `group` ranks per rail group.  0 if that shape is not built.
+int taot_launch_sinkhorn_tiered_mw(const SinkArgs& a, const float* tier_cost3, int node, int group, int32_t B, cudaStream_t st)
 {
     TierCosts tc;
     tc.c1 = (double)tier_cost3[0] * a.inv_eps;
     tc.c2 = (double)tier_cost3[1] * a.inv_eps;
     tc.c3 = (double)tier_cost3[2] * a.inv_eps;
-    switch (a.R) {
-        case 256: return launch_mw<1>(a, tc, B, st);
-        case 512: return launch_mw<2>(a, tc, B, st);
-        case 1024: return launch_mw<4>(a, tc, B, st);
-        default: return 0;
-    }
+    if (node == 8 && group == 32) return launch_mw_ranks<8, 32>(a, tc, B, st);
+    if (node == 4 && group == 16) return launch_mw_ranks<4, 16>(a, tc, B, st);
+    if (node == 4 && group == 32) return launch_mw_ranks<4, 32>(a, tc, B, st);
+    if (node == 16 && group == 32) return launch_mw_ranks<16, 32>(a, tc, B, st);
+    return 0;
 }

@@ -36,7 +36,8 @@ struct taot_handle_s {
     int32_t ntiers;          // 0: too many distinct values, the auction scans densely
     uint32_t* d_bidlist;     // [nbid] every (tier, win count) pair, best score first: w << 8 | t, bit 31 = next has the same score
     int32_t nbid;            // 0: no list (no tiers, or price step <= 0): the auction scans densely
-    int32_t tier_ok;         // 1: C has the node (8 ranks) / rail-group (32 ranks) structure and R is 256, 512 or 1024
+    int32_t tier_ok;         // 1: C has a node / rail-group structure one of the tier-by-tier kernels is built for and R is 256, 512 or 1024
+    int32_t tier_node, tier_group;   // ranks per node and per rail group of that structure (8 / 32, 4 / 16, 4 / 32 or 16 / 32)
     float tier_cost[3];      // its three costs off the diagonal: same node, same rail group, otherwise
     // derived sizes
     int64_t seg;             // elements per (layer, rank) segment

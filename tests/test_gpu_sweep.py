@@ -269,3 +269,32 @@ def test_tensor_core_solve_is_not_taken_where_it_does_not_apply():
     check_sinkhorn_problem(cpu(s)[0], cpu(d)[0], C.numpy(), 0.01 * max(SWEEP_TIERS), cpu(out["plan"])[0], cpu(out["iters"])[0],
                            cpu(out["row_err"])[0], 30, 0.0)
     pl.close()
+
+
+@pytest.mark.parametrize("gpus_per_node,nodes_per_group,want", [(4, 4, (4, 16)), (4, 8, (4, 32)), (16, 2, (16, 32)), (8, 4, (8, 32)),
+                                                                (2, 4, (0, 0))])
+def test_hierarchies_other_than_8_gpus_per_node_are_found_in_the_cost_matrix(gpus_per_node, nodes_per_group, want):
+    """The tier-by-tier kernels are chosen from the cost matrix itself: 4- and 16-GPU nodes at 256 ranks take them too
+    (a shape that is not built, 2-GPU nodes here, takes the general kernels); every case against the oracle, few and many
+    problems per call, and a two-tier cost."""
+    import paper_2608_03676_b200 as P
+    R = 256
+    for tiers, npg in ((SWEEP_TIERS, nodes_per_group), ((0.0, 1.0, 9.0), None)):
+        C = W.cost_matrix(R, gpus_per_node, tiers, npg)
+        for B, check in ((5, 2), (600, 2)):
+            pl = P.Planner(L=B, R=R, E=R, K=1, k=1, T=R, e2r=torch.arange(R, dtype=torch.int32), C=C, eps=0.1 * max(tiers),
+                           max_iters=60, tol=0.0)
+            found = pl.tier_structure()
+            if npg is not None:
+                assert found == want
+            else:
+                assert found == ((gpus_per_node, 32) if gpus_per_node in (4, 8, 16) else (0, 0))
+            loads = W.sweep_rank_loads(B, R, seed=300 + gpus_per_node, device="cuda")
+            ex, sp, s, d = pl.excess_spare(loads)
+            out = pl.sinkhorn(s, d)
+            torch.cuda.synchronize()
+            plan, iters, err, info = cpu(out["plan"]), cpu(out["iters"]), cpu(out["row_err"]), cpu(out["info"])
+            assert (iters == 60).all() and (info == 0).all()
+            for b in range(check):
+                check_sinkhorn_problem(cpu(s)[b], cpu(d)[b], C.numpy(), 0.1 * max(tiers), plan[b], iters[b], err[b], 60, 0.0)
+            pl.close()
