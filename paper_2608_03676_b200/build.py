@@ -35,7 +35,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(OBJ, exist_ok=True)
     headers = [os.path.join(CSRC, "taot_internal.cuh"), os.path.join(CSRC, "sinkhorn_common.cuh"),
                os.path.join(CSRC, "sinkhorn_tile.cuh"),
-               os.path.join(ROOT, "include", "taot.h")]
+               os.path.join(ROOT, "include", "taot.h"), os.path.join(ROOT, "include", "taot_measure.h")]
     nvcc = _nvcc()
 
     def compile_one(src: str):

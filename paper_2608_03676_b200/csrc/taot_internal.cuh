@@ -6,6 +6,7 @@
 #include <stddef.h>
 
 #include "taot.h"
+#include "taot_measure.h"
 
 // Elements of topk_idx one CTA of the histogram / reassignment kernels owns.  A chunk never
 // crosses a (layer, source rank) segment, so a segment of SEG = (T/R)*k elements has

@@ -1,4 +1,5 @@
-"""The C-ABI library loads without a GPU and exports every function include/taot.h declares."""
+"""The C-ABI library loads without a GPU and exports every function the headers under include/ declare
+(taot.h: the planner; taot_measure.h: measurement aids)."""
 import ctypes
 import os
 import re
@@ -7,7 +8,8 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _declared():
-    text = open(os.path.join(ROOT, "include", "taot.h")).read()
+    text = "".join(open(os.path.join(ROOT, "include", f)).read() for f in sorted(os.listdir(os.path.join(ROOT, "include")))
+                   if f.endswith(".h"))
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(taot_[a-z_0-9]+)\s*\(", text)))
 
