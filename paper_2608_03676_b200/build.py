@@ -34,7 +34,7 @@ def _stale(target: str, deps) -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(OBJ, exist_ok=True)
     headers = [os.path.join(CSRC, "taot_internal.cuh"), os.path.join(CSRC, "sinkhorn_common.cuh"),
-               os.path.join(CSRC, "sinkhorn_tile.cuh"),
+               os.path.join(CSRC, "sinkhorn_tile.cuh"), os.path.join(CSRC, "sinkhorn_tiered_common.cuh"),
                os.path.join(ROOT, "include", "taot.h"), os.path.join(ROOT, "include", "taot_measure.h")]
     nvcc = _nvcc()
 

@@ -23,34 +23,14 @@
 // factor above), the first iteration in the log domain and the final plan follow the register-tile kernels;
 // problems this kernel cannot take (a rank with both supply and demand, sums outside the safe fp32 range) are
 // handed back (iters = -1) to the general kernel.
-#include "sinkhorn_common.cuh"
+#include "sinkhorn_tiered_common.cuh"
 
 using namespace taot_sk;
 
 namespace {
 
-constexpr unsigned kFull = 0xffffffffu;
 constexpr int kNode = 8;          // ranks per node
 constexpr int kGroup = 32;        // ranks per rail group
-
-__device__ __forceinline__ float rcp_fast(float x)
-{
-    float y;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-__device__ __forceinline__ float exp_or_zero(double x) { return x == -INFINITY ? 0.0f : exp_split(x); }
-
-struct TierCosts {
-    double c1, c2, c3;            // cost / eps of the three tiers off the diagonal
-};
-
-// C_ij / eps for i != j, from the indices alone
-__device__ __forceinline__ double tier_cost(const TierCosts& tc, int i, int j)
-{
-    return (i / kNode == j / kNode) ? tc.c1 : ((i / kGroup == j / kGroup) ? tc.c2 : tc.c3);
-}
 
 // all-reduce over the lanes of one rail group (LPG lanes), and over the groups (one value per group, held by all
 // of its lanes)
@@ -182,20 +162,7 @@ sinkhorn_tiered_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
     for (int i = 0; i < RPL; ++i) {
         const int q = lane * RPL + i;
         double bj = -INFINITY;
-        if ((coldm >> i) & 1u) {
-            double mx = -INFINITY;
-            for (int h = 0; h < Hn; ++h) {
-                const int r = hot[h];
-                const double v = alpha[r] - tier_cost(tc, r, q);
-                mx = v > mx ? v : mx;
-            }
-            double acc = 0.0;
-            for (int h = 0; h < Hn; ++h) {
-                const int r = hot[h];
-                acc += (double)exp_split(alpha[r] - tier_cost(tc, r, q) - mx);
-            }
-            bj = log((double)a.d[b * R + q]) - (mx + log(acc));
-        }
+        if ((coldm >> i) & 1u) bj = first_column_potential<kNode, kGroup>(tc, alpha, hot, Hn, q, a.d[b * R + q]);
         beta[q] = bj;
     }
     __syncwarp();
@@ -387,25 +354,7 @@ sinkhorn_tiered_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
         }
     }
     __syncwarp();
-    int nonfinite = 0;
-    for (int row = 0; row < R; ++row) {
-        const double al = alpha[row];
-        float* orow = out + (int64_t)row * R;
-        if (al == -INFINITY) {
-            for (int j = lane; j < R; j += 32) orow[j] = 0.0f;
-            continue;
-        }
-#pragma unroll 4
-        for (int j = lane; j < R; j += 32) {
-            const float fg = fgs[j];
-            float val = 0.0f;
-            if (fg > 0.0f) {
-                val = exp_split(al + beta[j] - tier_cost(tc, row, j)) * fg;
-                if (!isfinite(val)) nonfinite = 1;
-            }
-            orow[j] = val;
-        }
-    }
+    const int nonfinite = write_plan_rows<kNode, kGroup>(tc, alpha, beta, fgs, R, 0, 1, lane, out);
     if (__any_sync(kFull, nonfinite != 0)) info |= TAOT_INFO_NONFINITE;
     if (lane == 0) {
         a.iters[b] = t;

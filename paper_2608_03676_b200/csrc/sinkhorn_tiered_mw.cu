@@ -10,34 +10,14 @@
 // threads and every barrier is reached by all of them: the error partials of iterate t ride the exchange of
 // half-step 2, the drift and range flags of an update ride the first exchange of the next iteration (a fold
 // then discards that half-step's sums and starts the iteration again with the new factors).
-#include "sinkhorn_common.cuh"
+#include "sinkhorn_tiered_common.cuh"
 
 using namespace taot_sk;
 
 namespace {
 
-constexpr unsigned kFull = 0xffffffffu;
 constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
-
-__device__ __forceinline__ float rcp_fast(float x)
-{
-    float y;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-__device__ __forceinline__ float exp_or_zero(double x) { return x == -INFINITY ? 0.0f : exp_split(x); }
-
-struct TierCosts {
-    double c1, c2, c3;            // cost / eps of the three tiers off the diagonal
-};
-
-template <int kNode, int kGroup>
-__device__ __forceinline__ double tier_cost(const TierCosts& tc, int i, int j)
-{
-    return (i / kNode == j / kNode) ? tc.c1 : ((i / kGroup == j / kGroup) ? tc.c2 : tc.c3);
-}
 
 template <int LO, int HI>
 __device__ __forceinline__ float xor_sum(float v)           // all-reduce over lane bits LO <= offset < HI
@@ -185,20 +165,7 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
     for (int i = 0; i < RPL; ++i) {
         const int q = q0 + i;
         double bj = -INFINITY;
-        if ((coldm >> i) & 1u) {
-            double mx = -INFINITY;
-            for (int h = 0; h < Hn; ++h) {
-                const int r = hot[h];
-                const double v = alpha[r] - tier_cost<kNode, kGroup>(tc, r, q);
-                mx = v > mx ? v : mx;
-            }
-            double acc = 0.0;
-            for (int h = 0; h < Hn; ++h) {
-                const int r = hot[h];
-                acc += (double)exp_split(alpha[r] - tier_cost<kNode, kGroup>(tc, r, q) - mx);
-            }
-            bj = log((double)a.d[b * R + q]) - (mx + log(acc));
-        }
+        if ((coldm >> i) & 1u) bj = first_column_potential<kNode, kGroup>(tc, alpha, hot, Hn, q, a.d[b * R + q]);
         beta[q] = bj;
     }
     __syncthreads();
@@ -404,25 +371,7 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
             fgs[q0 + i] = ((coldm >> i) & 1u) ? (float)fmin(1.0, (double)x[i] / ((double)c[i] + (double)a.eps0)) : 0.0f;
     }
     __syncthreads();
-    int nonfinite = 0;
-    for (int row = warp; row < R; row += kWarps) {
-        const double al = alpha[row];
-        float* orow = out + (int64_t)row * R;
-        if (al == -INFINITY) {
-            for (int j = lane; j < R; j += 32) orow[j] = 0.0f;
-            continue;
-        }
-#pragma unroll 4
-        for (int j = lane; j < R; j += 32) {
-            const float fg = fgs[j];
-            float val = 0.0f;
-            if (fg > 0.0f) {
-                val = exp_split(al + beta[j] - tier_cost<kNode, kGroup>(tc, row, j)) * fg;
-                if (!isfinite(val)) nonfinite = 1;
-            }
-            orow[j] = val;
-        }
-    }
+    const int nonfinite = write_plan_rows<kNode, kGroup>(tc, alpha, beta, fgs, R, warp, kWarps, lane, out);
     if (__syncthreads_or(nonfinite)) info |= TAOT_INFO_NONFINITE;
     if (tid == 0) {
         a.iters[b] = t;
