@@ -126,13 +126,18 @@ merge_kernel(const int32_t* __restrict__ cc, const int32_t* __restrict__ e2r, in
     const int l = blockIdx.x, tid = threadIdx.x;
     for (int i = tid; i < E + R; i += blockDim.x) sh[i] = 0;
     __syncthreads();
-    const int64_t RE = (int64_t)R * E;
-    for (int64_t idx = tid; idx < RE; idx += blockDim.x) {
-        const int32_t r = (int32_t)(idx / E), e = (int32_t)(idx % E);
-        const int32_t* p = cc + (((int64_t)l * R + r) * nc) * E + e;
+    const int32_t RE = R * E;                            // at most 256 x 1024
+    const int32_t* ccl = cc + (int64_t)l * RE * nc;
+    int32_t* nl = n + (int64_t)l * RE;
+    // (32-bit index arithmetic and several independent loads in flight per thread: the kernel sits in the chain of
+    // latency-bound stages, one CTA per layer)
+#pragma unroll 4
+    for (int32_t idx = tid; idx < RE; idx += blockDim.x) {
+        const int32_t r = idx / E, e = idx - r * E;
+        const int32_t* p = ccl + r * nc * E + e;
         int32_t v = 0;
-        for (int c = 0; c < nc; ++c) v += p[(int64_t)c * E];
-        n[(int64_t)l * RE + idx] = v;
+        for (int c = 0; c < nc; ++c) v += __ldg(p + c * E);
+        nl[idx] = v;
         if (v) atomicAdd(s_el + e, v);
     }
     __syncthreads();

@@ -116,9 +116,9 @@ struct TcArgs {
 };
 
 // The tensor cores add into their fp32 accumulator with truncation, so a long sum of positive terms comes out low by
-// an amount that grows with its length (measured: plan error up to 1e-4 at 1024 ranks with one accumulator).  The K
-// range is therefore cut into kAcc contiguous parts with an accumulator each (all 512 columns of tensor memory are
-// used) and the epilogue adds the parts in fp32 with rounding.
+// an amount that grows with its length (measured: plan error up to 1e-4 at 1024 ranks with one accumulator).  The
+// terms are therefore dealt round-robin to kAcc accumulators (k-step j to accumulator j mod kAcc; all 512 columns of
+// tensor memory are used) and the epilogue adds the accumulators in fp32 with rounding.
 template <int N>
 struct TcAcc {
     static constexpr int kAcc = 512 / N < 4 ? 512 / N : 4;
@@ -209,16 +209,26 @@ sinkhorn_tc_halfstep_kernel(const __grid_constant__ CUtensorMap map_a_hi, const 
                 const uint32_t st = smem_addr(tiles + (size_t)s * SM::kStageBytes);
                 const uint32_t a_hi = st, a_lo = st + kTileM * kBlockK * 4;
                 const uint32_t b_hi = st + 2 * kTileM * kBlockK * 4, b_lo = b_hi + N * kBlockK * 4;
-                // this k-block's part of the K range and whether it opens that part's accumulator
-                const int part = (int)(((int64_t)kb * TcAcc<N>::kAcc) / nk);
-                const bool opens = kb == 0 || (int)(((int64_t)(kb - 1) * TcAcc<N>::kAcc) / nk) != part;
-                const uint32_t tmem_acc = tmem_d + (uint32_t)(part * N);
+                // The four k-steps of a block go to different accumulators (k-step j of the whole sum to accumulator
+                // j mod kAcc), and the three products of a term are issued k-step by k-step: consecutive MMAs then never
+                // add into the same accumulator, which they would otherwise do one full MMA latency apart.
+                constexpr int kAcc = TcAcc<N>::kAcc;
+                const uint32_t fresh = kb == 0 ? 0u : 1u;
 #pragma unroll
                 for (int k = 0; k < kBlockK / kUmmaK; ++k) {
                     const uint32_t off = (uint32_t)k * kUmmaK * 4;        // 32 bytes along the swizzled row
-                    umma_tf32(tmem_acc, umma_desc_sw128(a_hi + off), umma_desc_sw128(b_hi + off), idesc, (opens && k == 0) ? 0u : 1u);
-                    umma_tf32(tmem_acc, umma_desc_sw128(a_hi + off), umma_desc_sw128(b_lo + off), idesc, 1u);
-                    umma_tf32(tmem_acc, umma_desc_sw128(a_lo + off), umma_desc_sw128(b_hi + off), idesc, 1u);
+                    umma_tf32(tmem_d + (uint32_t)((k % kAcc) * N), umma_desc_sw128(a_hi + off), umma_desc_sw128(b_hi + off), idesc,
+                              k < kAcc ? fresh : 1u);
+                }
+#pragma unroll
+                for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+                    const uint32_t off = (uint32_t)k * kUmmaK * 4;
+                    umma_tf32(tmem_d + (uint32_t)((k % kAcc) * N), umma_desc_sw128(a_hi + off), umma_desc_sw128(b_lo + off), idesc, 1u);
+                }
+#pragma unroll
+                for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+                    const uint32_t off = (uint32_t)k * kUmmaK * 4;
+                    umma_tf32(tmem_d + (uint32_t)((k % kAcc) * N), umma_desc_sw128(a_lo + off), umma_desc_sw128(b_hi + off), idesc, 1u);
                 }
                 umma_commit(&empty[s]);                   // the stage is free once these MMAs have read it
             }
