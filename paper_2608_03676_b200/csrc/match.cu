@@ -287,19 +287,31 @@ match_kernel(MatchArgs a)
         // slot index and a round re-forms the rows of the experts it served; a rank's arg-max is one load and one
         // compare per spilling expert.
         const long long c_b0 = timed ? clock64() : 0;
-        for (int r = tid; r < R; r += NT) matched[r] = 0;
+        // arbitration state per expert: best score among this round's bidders, then the lowest rank that has it
+        uint32_t* arb_hi = reinterpret_cast<uint32_t*>(arb_e);
+        uint32_t* arb_lo = arb_hi + E;
+        int smax = 0;                              // largest spare of this slot index: a row changes only below it
+        for (int r = tid; r < R; r += NT) { matched[r] = 0; smax = spare[r] > smax ? spare[r] : smax; }
+        for (int e = tid; e < E; e += NT) { arb_hi[e] = 0u; arb_lo[e] = 0xFFFFFFFFu; }
+        smax = __reduce_max_sync(0xffffffffu, smax);
+        if (tid == 0) s_cnt = 0;
+        __syncthreads();
+        if (lane == 0) atomicMax(&s_cnt, smax);
         for (int64_t idx = tid; idx < (int64_t)nhot0 * R; idx += NT) {
             const int q = (int)(idx / R), r = (int)(idx - (int64_t)q * R);
             keyM[r * NHs + q] = pair_key(q, r, kappa);
         }
+        __syncthreads();
+        const int32_t spare_cap = s_cnt;
         if (timed) c_build += clock64() - c_b0;
         for (;;) {
-            if (tid == 0) { s_any = 0; s_ns = 0; }
-            __syncthreads();
             const long long c_s0 = timed ? clock64() : 0;
             // Steps 1-2: every unmatched cold rank takes its best candidate expert (ties: lowest position = lowest index)
-            for (int rb = 0; rb < R; rb += NT >> qsh) {
-                const int r = rb + (tid >> qsh);                  // whole warps stay in the loop for the warp-wide steps
+            // (QS lanes per rank with QS * R <= NT: one pass covers every rank)
+            const int r = tid >> qsh;
+            uint32_t my_bk = 0u;                   // this thread's bid, if it is the lead lane of a bidding rank
+            int my_q = -1;
+            {
                 u64 key = 0;
                 if (r < R && !matched[r] && spare[r] > 0) {
                     const uint32_t* row = keyM + r * NHs;
@@ -316,43 +328,46 @@ match_kernel(MatchArgs a)
                     const u64 other = __shfl_xor_sync(0xffffffffu, key, o);
                     key = other > key ? other : key;
                 }
-                const int best_q = key != 0 ? (int)(0xFFFFFFFFu - (uint32_t)key) : -1;
-                const bool lead = qs == 0 && r < R;
-                if (lead) {
-                    estar[r] = best_q;
-                    if (key != 0) s_any = 1;
+                if (qs == 0 && r < R && key != 0) {
+                    my_bk = (uint32_t)(key >> 32);
+                    my_q = (int)(0xFFFFFFFFu - (uint32_t)key);
                 }
-                // Step 3: arbitration, best rank per expert (ties: lowest rank)
-                arbitrate(arb_e, best_q >= 0 ? hot0[best_q] : -1,
-                          (key == 0 || !lead) ? 0ull : ((key & 0xFFFFFFFF00000000ull) | (u64)(0xFFFFFFFFu - (uint32_t)r)));
             }
+            const int my_e = my_q >= 0 ? hot0[my_q] : 0;
+            // Step 3, first half: the best score any rank offers the expert (native 32-bit shared-memory atomics; agreeing
+            // inside the warp first on the expert most lanes want was measured and cost more than the conflicts it saves)
+            if (my_q >= 0) atomicMax(&arb_hi[my_e], my_bk);
+            if (!__syncthreads_or(my_q >= 0)) break;
+            if (tid == 0) s_ns = 0;
+            // Step 3, second half: among the ranks that offer it, the lowest
+            if (my_q >= 0 && arb_hi[my_e] == my_bk) atomicMin(&arb_lo[my_e], (uint32_t)r);
             __syncthreads();
             const long long c_s1 = timed ? clock64() : 0;
             if (timed) c_scan += c_s1 - c_s0;
-            if (!s_any) break;
-            // Step 4: winners take min(spill, spare)
-            for (int r = tid; r < R; r += NT) {
-                const int q = estar[r];
-                if (q < 0) continue;
-                const int e = hot0[q];
-                if ((uint32_t)arb_e[e] == 0xFFFFFFFFu - (uint32_t)r) {
-                    const int32_t g = spill[e] < spare[r] ? spill[e] : spare[r];
-                    spill[e] -= g;
-                    spare[r] -= g;
-                    matched[r] = 1;
-                    slot_e[r * K + kappa] = e;
-                    slot_a0[r * K + kappa] = g;
-                    served[atomicAdd(&s_ns, 1)] = q;
-                }
+            // Step 4: winners take min(spill, spare), and put the arbitration entries back.  A row of keys changes only
+            // where min(spill, spare_r) does, i.e. for ranks with more spare than the expert now spills: rows whose
+            // expert still spills at least the largest spare of this slot index are left as they are.
+            if (my_q >= 0 && arb_lo[my_e] == (uint32_t)r) {
+                const int32_t g = spill[my_e] < spare[r] ? spill[my_e] : spare[r];
+                spill[my_e] -= g;
+                spare[r] -= g;
+                matched[r] = 1;
+                slot_e[r * K + kappa] = my_e;
+                slot_a0[r * K + kappa] = g;
+                arb_hi[my_e] = 0u;                 // (a loser compares arb_lo with its own rank: the reset value is nobody's)
+                arb_lo[my_e] = 0xFFFFFFFFu;
+                if (spill[my_e] < spare_cap) served[atomicAdd(&s_ns, 1)] = my_q;
             }
             __syncthreads();
             const long long c_s2 = timed ? clock64() : 0;
             const int ns = s_ns;
-            for (int i = tid; i < ns; i += NT) arb_e[hot0[served[i]]] = 0;
-            for (int idx = tid; idx < ns * R; idx += NT) {
-                const int i = idx / R, r = idx - i * R;
-                const int q = served[i];
-                keyM[r * NHs + q] = pair_key(q, r, kappa);
+            if (ns > 0) {                          // uniform over the CTA
+                for (int idx = tid; idx < ns * R; idx += NT) {
+                    const int i = idx / R, r = idx - i * R;
+                    const int q = served[i];
+                    keyM[r * NHs + q] = pair_key(q, r, kappa);
+                }
+                __syncthreads();
             }
             ++rounds2;
             if (timed) { const long long c_s3 = clock64(); c_win += c_s2 - c_s1; c_row += c_s3 - c_s2; }
