@@ -5,11 +5,15 @@
 // Lane gl = 32 * warp + lane owns RPL = R / 256 consecutive ranks (1 at 256 ranks, 2 at 512, 4 at 1024): a node of
 // 8 ranks is 8 / RPL adjacent lanes, a rail group 32 / RPL lanes, a warp holds RPL whole groups.  A half-step is
 // lane-local products, five xor-shuffle levels (node, group, groups of the warp), one shared-memory exchange of
-// the eight warp totals (one block barrier), three multiply-adds and a reciprocal per rank.  Every decision
-// (stop, drift fold, hand-back) is taken from values that went through an exchange, so it is the same in all 256
-// threads and every barrier is reached by all of them: the error partials of iterate t ride the exchange of
-// half-step 2, the drift and range flags of an update ride the first exchange of the next iteration (a fold
-// then discards that half-step's sums and starts the iteration again with the new factors).
+// the eight warp totals (one named barrier), one multiply-add and a reciprocal per rank.  The iteration is one
+// dependent chain on a nearly empty SM, so everything that is not on the chain is kept out of the loop:
+//   * the loop body holds no rare case: a thread that sees its u~ or v~ drift out of range stores the number of the
+//     next exchange in a flag word, every thread reads that word (and the stop word) after the exchange's barrier,
+//     and any event -- drift, stop, last iteration -- leaves the loop for code that all threads run together;
+//   * with a tolerance, the row error of an iterate is not reduced by the eight warps at all: each lane stores
+//     its term, and a ninth warp, which otherwise only takes part in the barriers, sums the 256 terms after
+//     half-step 2's barrier and posts the iteration number in the stop word if the error is within the tolerance.
+//     The others see the word after the next barrier, half a step into iteration t + 1, and put iterate t back.
 #include "sinkhorn_tiered_common.cuh"
 
 using namespace taot_sk;
@@ -34,33 +38,38 @@ __device__ __forceinline__ double xor_max(double v)
     return v;
 }
 
-struct Exchange {                 // what one warp hands to the others in one half-step
-    float total;                  // its share of the sum over all groups
-    float err;                    // half-step 2: its share of the row error of the iterate
-    int flags;                    // half-step 1: drift (1) / range (2) of the previous update; half-step 2: range of the row sums (2)
-    int pad;
-};
+// one of the two barriers of an iteration: every thread of the block, whatever code it is in
+__device__ __forceinline__ void bar_loop(const int nthreads)
+{
+    asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
+}
 
 // kNode ranks per node, kGroup ranks per rail group (powers of two, kNode < kGroup, a group inside one warp)
 template <int kNode, int kGroup, int RPL, bool TOL>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads + 32)
 sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
 {
     static_assert(kGroup / RPL <= 32 && kGroup > kNode && kGroup % kNode == 0, "a rail group is held by the lanes of one warp");
     constexpr int LPN = kNode / RPL;              // lanes per node
     constexpr int LPG = kGroup / RPL;             // lanes per rail group
     static_assert(RPL >= 1 && RPL <= kNode && kNode % RPL == 0, "a lane holds part of one node");
+    constexpr int NW = kWarps + (TOL ? 1 : 0);    // warps of the block: with a tolerance, one more that sums the error
+    constexpr int NT = NW * 32;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int R = a.R, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool mainw = warp < kWarps;             // this warp owns ranks
     const int64_t b = blockIdx.x;
     if (b >= nprob) return;
     double* alpha = reinterpret_cast<double*>(smem_raw);          // [R] potentials by rank (supply ranks; -inf elsewhere)
     double* beta = alpha + R;                                      // [R] (demand ranks)
     float* fgs = reinterpret_cast<float*>(beta + R);               // [R] column cap of the final plan, 0 off the demand ranks
     int32_t* hot = reinterpret_cast<int32_t*>(fgs + R);            // [R] supply ranks, ascending
-    __shared__ Exchange xch[2][kWarps];
-    __shared__ double dred[2][kWarps];
-    __shared__ int ired[kWarps];
+    __shared__ __align__(16) float xtot[2][kWarps + 4];  // what a warp hands to the others in one half-step: its share of the total
+    __shared__ __align__(16) float xe[kThreads];         // each lane's term of the row error of the iterate
+    __shared__ __align__(8) int xword[2];                // [0] number of the exchange before which some u~ or v~ drifted out of
+                                                         // range; [1] iteration whose iterate met the tolerance
+    __shared__ double dred[2][NW];
+    __shared__ int ired[NW];
 
     // block-wide reductions for the set-up and the folds (two barriers each; not used inside an iteration)
     auto block_sum2 = [&](double& p, double& q) {
@@ -73,14 +82,14 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
         __syncthreads();
         p = 0.0; q = 0.0;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) { p += dred[0][w]; q += dred[1][w]; }
+        for (int w = 0; w < NW; ++w) { p += dred[0][w]; q += dred[1][w]; }
         __syncthreads();
     };
     auto block_max2 = [&](double& p, double& q) {               // p, q already reduced over the warp
         if (lane == 0) { dred[0][warp] = p; dred[1][warp] = q; }
         __syncthreads();
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) { p = fmax(p, dred[0][w]); q = fmax(q, dred[1][w]); }
+        for (int w = 0; w < NW; ++w) { p = fmax(p, dred[0][w]); q = fmax(q, dred[1][w]); }
         __syncthreads();
     };
 
@@ -92,7 +101,7 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
     double ps = 0.0, pd = 0.0;
 #pragma unroll
     for (int i = 0; i < RPL; ++i) {
-        const float sv = a.s[b * R + q0 + i], dv = a.d[b * R + q0 + i];
+        const float sv = mainw ? a.s[b * R + q0 + i] : 0.0f, dv = mainw ? a.d[b * R + q0 + i] : 0.0f;
         if (sv > 0.0f) { ps += (double)sv; hotm |= 1u << i; }
         if (dv > 0.0f) { pd += (double)dv; coldm |= 1u << i; }
         both |= (sv > 0.0f && dv > 0.0f) ? 1 : 0;
@@ -126,14 +135,14 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
     __syncthreads();
     int Hn = 0, hbase = incl - Hn_lane, Cn = 0;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
+    for (int w = 0; w < NW; ++w) {
         if (w < warp) hbase += ired[w];
         Hn += ired[w];
         Cn += (int)dred[0][w];
     }
     __syncthreads();
     if (Hn == 0 || Cn == 0) {
-        for (int q = tid; q < R * R; q += kThreads) out[q] = 0.0f;
+        for (int q = tid; q < R * R; q += NT) out[q] = 0.0f;
         if (tid == 0) {
             a.iters[b] = 0;
             a.row_err[b] = 0.0f;
@@ -157,22 +166,26 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
 
     // ---- iteration 1 in the log domain (v = 1 on every rank): phi = log s~ - LSE_j(-C_ij/eps) over all j,
     //      psi_j = log d_j - LSE_i(phi_i - C_ij/eps)
+    if (mainw) {
 #pragma unroll
-    for (int i = 0; i < RPL; ++i)
-        alpha[q0 + i] = ((hotm >> i) & 1u) ? log((double)x[i]) - a.rowlse0[q0 + i] : -INFINITY;
-    __syncthreads();
-#pragma unroll 1
-    for (int i = 0; i < RPL; ++i) {
-        const int q = q0 + i;
-        double bj = -INFINITY;
-        if ((coldm >> i) & 1u) bj = first_column_potential<kNode, kGroup>(tc, alpha, hot, Hn, q, a.d[b * R + q]);
-        beta[q] = bj;
+        for (int i = 0; i < RPL; ++i)
+            alpha[q0 + i] = ((hotm >> i) & 1u) ? log((double)x[i]) - a.rowlse0[q0 + i] : -INFINITY;
     }
     __syncthreads();
-
-    // ---- per-rank state: z = u~ or v~, w = weight inside the node sum, k1..k3 = tier coefficients of its own sum;
-    // node and group factors of both trees (b: demand side, feeds the row sums; a: supply side, feeds the column sums)
-    float z[RPL], w[RPL], k1[RPL], k2[RPL], k3[RPL];
+    if (mainw) {
+#pragma unroll 1
+        for (int i = 0; i < RPL; ++i) {
+            const int q = q0 + i;
+            double bj = -INFINITY;
+            if ((coldm >> i) & 1u) bj = first_column_potential<kNode, kGroup>(tc, alpha, hot, Hn, q, a.d[b * R + q]);
+            beta[q] = bj;
+        }
+    }
+    __syncthreads();
+    // ---- per-rank state: z = u~ or v~, wr / wc = weight inside the node sum that feeds the row / column sums (zero
+    // unless the rank is a demand / supply rank), k1..k3 = tier coefficients of its own sum; node and group factors
+    // of both trees (b: demand side, feeds the row sums; a: supply side, feeds the column sums)
+    float z[RPL], wr[RPL], wc[RPL], k1[RPL], k2[RPL], k3[RPL];
     float fb = 0.0f, fa = 0.0f, Fb = 0.0f, Fa = 0.0f;
 #pragma unroll
     for (int i = 0; i < RPL; ++i) z[i] = 1.0f;
@@ -195,21 +208,21 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
 #pragma unroll
         for (int i = 0; i < RPL; ++i) {
             const bool ish = (hotm >> i) & 1u, isc = (coldm >> i) & 1u;
-            float wv = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
+            float wrow = 0.0f, wcol = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
             if (ish) {
                 const double al = alpha[q0 + i];
-                wv = exp_or_zero(al - p1);
+                wcol = exp_or_zero(al - p1);
                 a1 = exp_or_zero(m1 == -INFINITY ? -INFINITY : al - tc.c1 + m1);
                 a2 = exp_or_zero(m2 == -INFINITY ? -INFINITY : al - tc.c2 + m2);
                 a3 = exp_or_zero(m3 == -INFINITY ? -INFINITY : al - tc.c3 + m3);
             } else if (isc) {
                 const double be = beta[q0 + i];
-                wv = exp_or_zero(be - m1);
+                wrow = exp_or_zero(be - m1);
                 a1 = exp_or_zero(p1 == -INFINITY ? -INFINITY : be - tc.c1 + p1);
                 a2 = exp_or_zero(p2 == -INFINITY ? -INFINITY : be - tc.c2 + p2);
                 a3 = exp_or_zero(p3 == -INFINITY ? -INFINITY : be - tc.c3 + p3);
             }
-            w[i] = wv; k1[i] = a1; k2[i] = a2; k3[i] = a3;
+            wr[i] = wrow; wc[i] = wcol; k1[i] = a1; k2[i] = a2; k3[i] = a3;
         }
     };
     auto fold = [&]() {                            // u~, v~ into the fp64 potentials, then every factor anew
@@ -221,157 +234,196 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
         }
         rebuild();
     };
-    // first part of a half-step: this lane's node sum N, group sum G (times the group factor: FG) and the warp's
-    // share of the total
-    // `carry` (if with_carry): one more value summed over the whole warp in the same five shuffle levels, so that
-    // its reduction overlaps this one instead of following it (the row-error partial of the iterate)
-    auto partial = [&](const bool rows, const bool with_carry, const float (&zsrc)[RPL], float& N, float& G, float& FG,
-                       float& carry) {
-        const unsigned srcm = rows ? coldm : hotm;
+    // First part of a half-step, everything that does not need the other warps: the lane's node sum and group sum by
+    // five xor-shuffle levels, the warp's share `tw` of the total, and `base[i]`, each rank's own sum without the
+    // total's term: own sum = k1 N + k2 (G - f N) + k3 (T - F G) = base + k3 T.
+    auto partial = [&](const bool rows, const float (&wsrc)[RPL], const float (&zsrc)[RPL], float (&base)[RPL]) {
         float p = 0.0f;
 #pragma unroll
-        for (int i = 0; i < RPL; ++i) p += ((srcm >> i) & 1u) ? w[i] * zsrc[i] : 0.0f;
+        for (int i = 0; i < RPL; ++i) p = fmaf(wsrc[i], zsrc[i], p);
 #pragma unroll
-        for (int o = 1; o < LPN; o <<= 1) {
-            p += __shfl_xor_sync(kFull, p, o);
-            if (with_carry) carry += __shfl_xor_sync(kFull, carry, o);
-        }
-        N = p;
+        for (int o = 1; o < LPN; o <<= 1) p += __shfl_xor_sync(kFull, p, o);
+        const float N = p;
         // every node appears LPN times among the lanes of its group: sum one copy per node
-        float g = (rows ? fb : fa) * N;
+        const float f = rows ? fb : fa;
+        float g = f * N;
 #pragma unroll
-        for (int o = LPN; o < LPG; o <<= 1) {
-            g += __shfl_xor_sync(kFull, g, o);
-            if (with_carry) carry += __shfl_xor_sync(kFull, carry, o);
-        }
-        G = g;
-        FG = (rows ? Fb : Fa) * G;
+        for (int o = LPN; o < LPG; o <<= 1) g += __shfl_xor_sync(kFull, g, o);
+        const float G = g;
+        const float FG = (rows ? Fb : Fa) * G;
         float tt = FG;                             // every group appears once per LPG lanes
 #pragma unroll
-        for (int o = LPG; o < 32; o <<= 1) {
-            tt += __shfl_xor_sync(kFull, tt, o);
-            if (with_carry) carry += __shfl_xor_sync(kFull, carry, o);
-        }
+        for (int o = LPG; o < 32; o <<= 1) tt += __shfl_xor_sync(kFull, tt, o);
+        const float Gx = fmaf(-f, N, G);
+#pragma unroll
+        for (int i = 0; i < RPL; ++i) base[i] = fmaf(k1[i], N, fmaf(k2[i], Gx, -(k3[i] * FG)));
         return tt;
     };
-    auto own_sums = [&](const bool rows, float N, float G, float FG, float T, float (&res)[RPL]) {
-        const float Gx = G - (rows ? fb : fa) * N, Tx = T - FG;
+    // second part: the eight warp totals, summed pairwise (the same in every thread)
+    auto total_of = [&](const int buf) {
+        const float4 lo = *reinterpret_cast<const float4*>(&xtot[buf][0]);
+        const float4 hi = *reinterpret_cast<const float4*>(&xtot[buf][4]);
+        return ((lo.x + lo.y) + (lo.z + lo.w)) + ((hi.x + hi.y) + (hi.z + hi.w));
+    };
+    // exact row error of the iterate (u~, v~) = z whose row sums are r, and whether a row sum left the safe range:
+    // block-wide, for the iterate that is the result
+    auto exact_error = [&](const float (&r)[RPL], double& err, int& bad) {
+        double e = 0.0, unused = 0.0;
+        int b2 = 0;
 #pragma unroll
-        for (int i = 0; i < RPL; ++i) res[i] = fmaf(k1[i], N, fmaf(k2[i], Gx, k3[i] * Tx));
+        for (int i = 0; i < RPL; ++i) {
+            const bool ish = (hotm >> i) & 1u;
+            e += ish ? (double)fabsf(fmaf(z[i], r[i], -x[i])) : 0.0;
+            b2 |= (ish && !(r[i] > kSumLo && r[i] < kSumHi)) ? 1 : 0;
+        }
+        block_sum2(e, unused);
+        err = e;
+        bad = __syncthreads_or(b2);
     };
     rebuild();
 
+
+
+    // ---- the iterations.  t = iteration in progress; k = exchanges so far (their parity picks the buffer).
     int t = 1;
     int until_check = a.check_every;
     float err_out = 0.0f;
     const uint32_t lo_bits = __float_as_uint(kDriftLo), span_bits = __float_as_uint(kDriftHi) - lo_bits;
-    const unsigned anym = hotm | coldm;
-    int prev_flags = 0;                            // drift (1) / range (2) of the update that produced the current z
-    int k = 0;                                     // exchanges so far (their parity picks the buffer)
+    int k = 0;
+    float r[RPL], zkeep[RPL], base[RPL];
+#pragma unroll
+    for (int i = 0; i < RPL; ++i) { r[i] = 1.0f; zkeep[i] = 1.0f; base[i] = 0.0f; }
+    if (tid == 0) { xword[0] = -1; xword[1] = -1; }
+    __syncthreads();
+    enum { kEvStop = 1, kEvDrift = 2, kEvLast = 3 };
     for (;;) {
-        // ================= half-step 1: r = K~ v~ on the supply ranks; these row sums belong to iterate t
-        float N, G, FG;
-        float nocarry = 0.0f;
-        float tw = partial(true, false, z, N, G, FG, nocarry);
-        const int wf = (__any_sync(kFull, prev_flags & 1) ? 1 : 0) | (__any_sync(kFull, prev_flags & 2) ? 2 : 0);
-        if (lane == 0) { xch[k & 1][warp].total = tw; xch[k & 1][warp].flags = wf; }
-        __syncthreads();
+        int event = 0;
         float T = 0.0f;
-        int flags = 0;
+        if (mainw) {
+            for (;;) {
+                // ================= half-step 1: r = K~ v~ on the supply ranks; these row sums belong to iterate t
+                float tw = partial(true, wr, z, base);
+                if (lane == 0) xtot[k & 1][warp] = tw;
+                bar_loop(NT);
+                T = total_of(k & 1);
+                const int2 xw = *reinterpret_cast<const int2*>(xword);
+                event = (TOL && xw.y == t - 1) ? kEvStop : (xw.x == k ? kEvDrift : (t >= a.max_iters ? kEvLast : 0));
+                ++k;
+                if (event) break;
 #pragma unroll
-        for (int wv = 0; wv < kWarps; ++wv) { T += xch[k & 1][wv].total; flags |= xch[k & 1][wv].flags; }
-        ++k;
-        if (flags & 2) {                           // a sum of the previous update left the safe range: hand back
-            if (tid == 0) a.iters[b] = kHandBack;
-            return;
-        }
-        if (flags & 1) {                           // u~, v~ drifted: fold them and take the half-step again
-            fold();
-            prev_flags = 0;
-            continue;
-        }
-        float r[RPL];
-        own_sums(true, N, G, FG, T, r);
-        const bool last = t >= a.max_iters;
-        bool check_now = false;
-        if (TOL) {
-            check_now = until_check == 1;
-            until_check = check_now ? a.check_every : until_check - 1;
-        }
-        const bool test = last || check_now;
-        float ew = 0.0f;
-        int badr = 0;
-        if (test) {
-            float e = 0.0f;
+                for (int i = 0; i < RPL; ++i) r[i] = fmaf(k3[i], T, base[i]);
+                if (TOL) {
+                    const bool check_now = until_check == 1;
+                    until_check = check_now ? a.check_every : until_check - 1;
+                    if (check_now) {               // this lane's term of the row error, for the ninth warp
+                        float e = 0.0f;
 #pragma unroll
-            for (int i = 0; i < RPL; ++i) {
-                const bool ish = (hotm >> i) & 1u;
-                e += ish ? fabsf(fmaf(z[i], r[i], -x[i])) : 0.0f;
-                badr |= (ish && !(r[i] > kSumLo && r[i] < kSumHi)) ? 2 : 0;
+                        for (int i = 0; i < RPL; ++i) {
+                            const bool ok = r[i] > kSumLo && r[i] < kSumHi;
+                            e += ((hotm >> i) & 1u) ? (ok ? fabsf(fmaf(z[i], r[i], -x[i])) : INFINITY) : 0.0f;
+                            zkeep[i] = z[i];
+                        }
+                        xe[tid] = e;
+                    }
+                }
+                float zn[RPL];
+#pragma unroll
+                for (int i = 0; i < RPL; ++i) zn[i] = ((hotm >> i) & 1u) ? x[i] * rcp_fast(r[i]) : z[i];
+                // ================= half-step 2: c = K~^T u' on the demand ranks, v' = d / c
+                tw = partial(false, wc, zn, base);
+                if (lane == 0) xtot[k & 1][warp] = tw;
+                bar_loop(NT);
+                T = total_of(k & 1);
+                ++k;
+                // a sum outside the safe range shows in its reciprocal (zero, infinite or not a number), so the
+                // drift test catches it too; a rank that takes no part keeps z = 1
+                bool drift = false;
+#pragma unroll
+                for (int i = 0; i < RPL; ++i) {
+                    const float c = fmaf(k3[i], T, base[i]);
+                    z[i] = ((coldm >> i) & 1u) ? x[i] * rcp_fast(c) : zn[i];
+                    drift |= (__float_as_uint(z[i]) - lo_bits) > span_bits;
+                }
+                if (drift) xword[0] = k;           // read after the next exchange's barrier; every writer stores the same k
+                ++t;
             }
-            ew = e;                                // summed over the warp inside half-step 2's reduction
-            badr = __any_sync(kFull, badr) ? 2 : 0;
-        }
-        float zn[RPL];
+        } else {
+            // the ninth warp: the same barriers, the same events; between half-step 2's barrier and the next one it
+            // sums the 256 terms of the row error (eight per lane, then five shuffle levels: one fixed order)
+            for (;;) {
+                bar_loop(NT);
+                const int2 xw = *reinterpret_cast<const int2*>(xword);
+                event = (TOL && xw.y == t - 1) ? kEvStop : (xw.x == k ? kEvDrift : (t >= a.max_iters ? kEvLast : 0));
+                ++k;
+                if (event) break;
+                const bool check_now = until_check == 1;
+                until_check = check_now ? a.check_every : until_check - 1;
+                bar_loop(NT);
+                ++k;
+                if (check_now) {
+                    const float4 lo = *reinterpret_cast<const float4*>(&xe[lane * 8]);
+                    const float4 hi = *reinterpret_cast<const float4*>(&xe[lane * 8 + 4]);
+                    float e = ((lo.x + lo.y) + (lo.z + lo.w)) + ((hi.x + hi.y) + (hi.z + hi.w));
 #pragma unroll
-        for (int i = 0; i < RPL; ++i) zn[i] = ((hotm >> i) & 1u) ? x[i] * rcp_fast(r[i]) : z[i];
-        // ================= half-step 2: c = K~^T u' on the demand ranks, v' = d / c
-        tw = test ? partial(false, true, zn, N, G, FG, ew) : partial(false, false, zn, N, G, FG, nocarry);
-        if (lane == 0) { xch[k & 1][warp].total = tw; xch[k & 1][warp].err = ew; xch[k & 1][warp].flags = badr; }
-        __syncthreads();
-        T = 0.0f;
-        float err = 0.0f;
-        flags = 0;
-#pragma unroll
-        for (int wv = 0; wv < kWarps; ++wv) {
-            T += xch[k & 1][wv].total;
-            err += xch[k & 1][wv].err;
-            flags |= xch[k & 1][wv].flags;
+                    for (int o = 1; o < 32; o <<= 1) e += __shfl_xor_sync(kFull, e, o);
+                    if (lane == 0 && e <= tol_abs_f) xword[1] = t;
+                }
+                ++t;
+            }
         }
-        ++k;
-        if (test && (last || err <= tol_abs_f)) {  // iterate t is the result; half-step 2 is dropped
-            if (flags & 2) { if (tid == 0) a.iters[b] = kHandBack; return; }
-            err_out = (float)((double)err / sum_st);
-            if (TOL && !(err <= tol_abs_f)) info |= TAOT_INFO_SINKHORN_CAP;
+        // ---- an event: every thread of the block is here, after the barrier of half-step 1 of iteration t
+        if (event == kEvStop) {                    // iterate t - 1 met the tolerance: it is the result
+            --t;
+#pragma unroll
+            for (int i = 0; i < RPL; ++i) z[i] = zkeep[i];
+            double err;
+            int bad;
+            exact_error(r, err, bad);              // no row sum is out of range here: its term would have been infinite
+            err_out = (float)(err / sum_st);
             break;
         }
-        float c[RPL];
-        own_sums(false, N, G, FG, T, c);
-        // a sum outside the safe range shows in its reciprocal (zero, infinite or not a number), so the drift test
-        // catches it too; both flags travel with the next exchange
-        int f = 0;
+        if (event == kEvDrift) {
+            // Some u~ or v~ of the previous update left [e^-40, e^40].  Either a sum left the safe range -- its
+            // reciprocal is then zero, infinite, not a number or far outside any drift -- and the problem is handed
+            // back, or the factors drifted: fold them into the potentials and take the half-step again.
+            int range = 0;
 #pragma unroll
-        for (int i = 0; i < RPL; ++i) {
-            const bool ish = (hotm >> i) & 1u, isc = (coldm >> i) & 1u;
-            zn[i] = isc ? x[i] * rcp_fast(c[i]) : zn[i];
-            f |= (((anym >> i) & 1u) && (__float_as_uint(zn[i]) - lo_bits) > span_bits) ? 1 : 0;
-            f |= ((ish && !(r[i] > kSumLo && r[i] < kSumHi)) || (isc && !(c[i] > kSumLo && c[i] < kSumHi))) ? 2 : 0;
+            for (int i = 0; i < RPL; ++i)
+                range |= (!(z[i] > x[i] * kSumLo && z[i] < x[i] * kSumHi) && ((hotm | coldm) >> i & 1u)) ? 1 : 0;
+            if (__syncthreads_or(range)) {
+                if (tid == 0) a.iters[b] = kHandBack;
+                return;
+            }
+            fold();
+            continue;
         }
-        prev_flags = f;
+        // kEvLast: iterate t is the result whatever its error
 #pragma unroll
-        for (int i = 0; i < RPL; ++i) z[i] = zn[i];
-        ++t;
+        for (int i = 0; i < RPL; ++i) r[i] = fmaf(k3[i], T, base[i]);
+        double err;
+        int bad;
+        exact_error(r, err, bad);
+        if (bad) { if (tid == 0) a.iters[b] = kHandBack; return; }
+        err_out = (float)(err / sum_st);
+        if (TOL && !((float)err <= tol_abs_f)) info |= TAOT_INFO_SINKHORN_CAP;
+        break;
     }
 
     // ---- T = diag(u) M diag(v) from the total potentials, then the column cap
     fold();
     {
-        float N, G, FG;
-        float nocarry = 0.0f;
-        const float tw = partial(false, false, z, N, G, FG, nocarry);          // column sums of K~ itself (u~ = 1)
-        if (lane == 0) xch[k & 1][warp].total = tw;
+        const float tw = partial(false, wc, z, base);                           // column sums of K~ itself (u~ = 1)
+        if (lane == 0) xtot[k & 1][warp] = tw;
         __syncthreads();
-        float T = 0.0f;
+        const float T = total_of(k & 1);
 #pragma unroll
-        for (int wv = 0; wv < kWarps; ++wv) T += xch[k & 1][wv].total;
-        float c[RPL];
-        own_sums(false, N, G, FG, T, c);
-#pragma unroll
-        for (int i = 0; i < RPL; ++i)
-            fgs[q0 + i] = ((coldm >> i) & 1u) ? (float)fmin(1.0, (double)x[i] / ((double)c[i] + (double)a.eps0)) : 0.0f;
+        for (int i = 0; i < RPL; ++i) {
+            const float c = fmaf(k3[i], T, base[i]);
+            if (mainw) fgs[q0 + i] = ((coldm >> i) & 1u) ? (float)fmin(1.0, (double)x[i] / ((double)c + (double)a.eps0)) : 0.0f;
+        }
     }
     __syncthreads();
-    const int nonfinite = write_plan_rows<kNode, kGroup>(tc, alpha, beta, fgs, R, warp, kWarps, lane, out);
+    const int nonfinite = write_plan_rows<kNode, kGroup>(tc, alpha, beta, fgs, R, warp, NW, lane, out);
     if (__syncthreads_or(nonfinite)) info |= TAOT_INFO_NONFINITE;
     if (tid == 0) {
         a.iters[b] = t;
@@ -395,7 +447,7 @@ int launch_mw(const SinkArgs& a, const TierCosts& tc, int32_t B, cudaStream_t st
     if (2 * B <= sms && smem < kExclusiveSmem) smem = kExclusiveSmem;
     if (a.tol > 0.0f) {
         TAOT_CUDA_OK(cudaFuncSetAttribute(sinkhorn_tiered_mw_kernel<kNode, kGroup, RPL, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        sinkhorn_tiered_mw_kernel<kNode, kGroup, RPL, true><<<B, kThreads, smem, st>>>(a, tc, (int64_t)B);
+        sinkhorn_tiered_mw_kernel<kNode, kGroup, RPL, true><<<B, kThreads + 32, smem, st>>>(a, tc, (int64_t)B);
     } else {
         TAOT_CUDA_OK(cudaFuncSetAttribute(sinkhorn_tiered_mw_kernel<kNode, kGroup, RPL, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         sinkhorn_tiered_mw_kernel<kNode, kGroup, RPL, false><<<B, kThreads, smem, st>>>(a, tc, (int64_t)B);
