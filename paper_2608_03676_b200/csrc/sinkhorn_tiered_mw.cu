@@ -38,6 +38,22 @@ __device__ __forceinline__ double xor_max(double v)
     return v;
 }
 
+// ((a0 + a2) + (a4 + a6)) + ((a1 + a3) + (a5 + a7)) with packed fp32 additions: four instructions, three levels
+__device__ __forceinline__ float sum8(const float4 lo, const float4 hi)
+{
+    unsigned long long p0, p1, p2, p3;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(p0) : "f"(lo.x), "f"(lo.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(p1) : "f"(lo.z), "f"(lo.w));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(p2) : "f"(hi.x), "f"(hi.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(p3) : "f"(hi.z), "f"(hi.w));
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(p0) : "l"(p0), "l"(p1));
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(p2) : "l"(p2), "l"(p3));
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(p0) : "l"(p0), "l"(p2));
+    float x, y;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(x), "=f"(y) : "l"(p0));
+    return x + y;
+}
+
 // one of the two barriers of an iteration: every thread of the block, whatever code it is in
 __device__ __forceinline__ void bar_loop(const int nthreads)
 {
@@ -66,8 +82,7 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
     int32_t* hot = reinterpret_cast<int32_t*>(fgs + R);            // [R] supply ranks, ascending
     __shared__ __align__(16) float xtot[2][kWarps + 4];  // what a warp hands to the others in one half-step: its share of the total
     __shared__ __align__(16) float xe[kThreads];         // each lane's term of the row error of the iterate
-    __shared__ __align__(8) int xword[2];                // [0] number of the exchange before which some u~ or v~ drifted out of
-                                                         // range; [1] iteration whose iterate met the tolerance
+    __shared__ int xev[4];                               // events of the iteration loop (see there)
     __shared__ double dred[2][NW];
     __shared__ int ired[NW];
 
@@ -182,15 +197,20 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
         }
     }
     __syncthreads();
-    // ---- per-rank state: z = u~ or v~, wr / wc = weight inside the node sum that feeds the row / column sums (zero
-    // unless the rank is a demand / supply rank), k1..k3 = tier coefficients of its own sum; node and group factors
-    // of both trees (b: demand side, feeds the row sums; a: supply side, feeds the column sums)
-    float z[RPL], wr[RPL], wc[RPL], k1[RPL], k2[RPL], k3[RPL];
+    // ---- per-rank state: z = u~ or v~; pr / pc = this rank's term of its node sum for the next row / column sums
+    // (weight times scaling: zero unless the rank is a demand / supply rank); wrx / wcx = that weight times the rank's
+    // mass, so that the term follows from the reciprocal of a sum in one multiplication; kA, kB, k3 = coefficients of
+    // its own sum on the node sum, the group sum and the total:
+    //   own sum = k1 N + k2 (G - f N) + k3 (T - F G) = (k1 - k2 f) N + (k2 - k3 F) G + k3 T,
+    // with f, F the node and group factors of the tree the sum is taken over (b: demand side, feeds the row sums; a:
+    // supply side, feeds the column sums).  k1 >= k2 f exp((c2 - c1)/eps) and k2 >= k3 F exp((c3 - c2)/eps), so the two
+    // differences are formed without cancellation that matters.
+    float z[RPL], pr[RPL], pc[RPL], wrx[RPL], wcx[RPL], wc[RPL], kA[RPL], kB[RPL], k3[RPL];
     float fb = 0.0f, fa = 0.0f, Fb = 0.0f, Fa = 0.0f;
 #pragma unroll
     for (int i = 0; i < RPL; ++i) z[i] = 1.0f;
 
-    auto rebuild = [&]() {                         // block-uniform: holds barriers
+    auto rebuild = [&]() {                         // block-uniform: holds barriers; expects z = 1
         double m1 = -INFINITY, p1 = -INFINITY;
 #pragma unroll
         for (int i = 0; i < RPL; ++i) {
@@ -222,7 +242,13 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
                 a2 = exp_or_zero(p2 == -INFINITY ? -INFINITY : be - tc.c2 + p2);
                 a3 = exp_or_zero(p3 == -INFINITY ? -INFINITY : be - tc.c3 + p3);
             }
-            wr[i] = wrow; wc[i] = wcol; k1[i] = a1; k2[i] = a2; k3[i] = a3;
+            // a supply rank's own sum is a row sum (demand-side tree), a demand rank's a column sum
+            kA[i] = fmaf(-a2, ish ? fb : fa, a1);
+            kB[i] = fmaf(-a3, ish ? Fb : Fa, a2);
+            k3[i] = a3;
+            wc[i] = wcol;
+            wrx[i] = wrow * x[i]; wcx[i] = wcol * x[i];
+            pr[i] = wrow; pc[i] = wcol;            // z = 1
         }
     };
     auto fold = [&]() {                            // u~, v~ into the fp64 potentials, then every factor anew
@@ -235,35 +261,32 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
         rebuild();
     };
     // First part of a half-step, everything that does not need the other warps: the lane's node sum and group sum by
-    // five xor-shuffle levels, the warp's share `tw` of the total, and `base[i]`, each rank's own sum without the
-    // total's term: own sum = k1 N + k2 (G - f N) + k3 (T - F G) = base + k3 T.
-    auto partial = [&](const bool rows, const float (&wsrc)[RPL], const float (&zsrc)[RPL], float (&base)[RPL]) {
-        float p = 0.0f;
+    // five xor-shuffle levels, the warp's share of the total (the same value in all of its lanes when a warp is one
+    // rail group) and `base[i]`, each rank's own sum without the total's term.
+    auto partial = [&](const bool rows, const float (&term)[RPL], float (&base)[RPL]) {
+        float p = term[0];
 #pragma unroll
-        for (int i = 0; i < RPL; ++i) p = fmaf(wsrc[i], zsrc[i], p);
+        for (int i = 1; i < RPL; ++i) p += term[i];
 #pragma unroll
         for (int o = 1; o < LPN; o <<= 1) p += __shfl_xor_sync(kFull, p, o);
         const float N = p;
         // every node appears LPN times among the lanes of its group: sum one copy per node
-        const float f = rows ? fb : fa;
-        float g = f * N;
+        float g = (rows ? fb : fa) * N;
 #pragma unroll
         for (int o = LPN; o < LPG; o <<= 1) g += __shfl_xor_sync(kFull, g, o);
         const float G = g;
-        const float FG = (rows ? Fb : Fa) * G;
-        float tt = FG;                             // every group appears once per LPG lanes
+        float tt = (rows ? Fb : Fa) * G;           // every group appears once per LPG lanes
 #pragma unroll
         for (int o = LPG; o < 32; o <<= 1) tt += __shfl_xor_sync(kFull, tt, o);
-        const float Gx = fmaf(-f, N, G);
 #pragma unroll
-        for (int i = 0; i < RPL; ++i) base[i] = fmaf(k1[i], N, fmaf(k2[i], Gx, -(k3[i] * FG)));
+        for (int i = 0; i < RPL; ++i) base[i] = fmaf(kA[i], N, kB[i] * G);
         return tt;
     };
     // second part: the eight warp totals, summed pairwise (the same in every thread)
     auto total_of = [&](const int buf) {
         const float4 lo = *reinterpret_cast<const float4*>(&xtot[buf][0]);
         const float4 hi = *reinterpret_cast<const float4*>(&xtot[buf][4]);
-        return ((lo.x + lo.y) + (lo.z + lo.w)) + ((hi.x + hi.y) + (hi.z + hi.w));
+        return sum8(lo, hi);
     };
     // exact row error of the iterate (u~, v~) = z whose row sums are r, and whether a row sum left the safe range:
     // block-wide, for the iterate that is the result
@@ -282,45 +305,48 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
     };
     rebuild();
 
-
-
-    // ---- the iterations.  t = iteration in progress; k = exchanges so far (their parity picks the buffer).
+    // ---- the iterations; t = iteration in progress.  xev[0] = the iteration whose half-step 1 ends with an event: the
+    // last one unless a thread that saw its u~ or v~ drift (xev[2]) or the ninth warp that found the previous iterate
+    // within the tolerance (xev[1]) put the next iteration there.
     int t = 1;
     int until_check = a.check_every;
+    const bool every = a.check_every <= 1;
     float err_out = 0.0f;
     const uint32_t lo_bits = __float_as_uint(kDriftLo), span_bits = __float_as_uint(kDriftHi) - lo_bits;
-    int k = 0;
     float r[RPL], zkeep[RPL], base[RPL];
 #pragma unroll
     for (int i = 0; i < RPL; ++i) { r[i] = 1.0f; zkeep[i] = 1.0f; base[i] = 0.0f; }
-    if (tid == 0) { xword[0] = -1; xword[1] = -1; }
+    if (tid == 0) { xev[0] = a.max_iters; xev[1] = -1; xev[2] = -1; }
     __syncthreads();
-    enum { kEvStop = 1, kEvDrift = 2, kEvLast = 3 };
     for (;;) {
-        int event = 0;
         float T = 0.0f;
         if (mainw) {
             for (;;) {
                 // ================= half-step 1: r = K~ v~ on the supply ranks; these row sums belong to iterate t
-                float tw = partial(true, wr, z, base);
-                if (lane == 0) xtot[k & 1][warp] = tw;
+                xtot[0][warp] = partial(true, pr, base);
                 bar_loop(NT);
-                T = total_of(k & 1);
-                const int2 xw = *reinterpret_cast<const int2*>(xword);
-                event = (TOL && xw.y == t - 1) ? kEvStop : (xw.x == k ? kEvDrift : (t >= a.max_iters ? kEvLast : 0));
-                ++k;
-                if (event) break;
+                T = total_of(0);
+                if (xev[0] <= t) break;
+                float rr[RPL];
 #pragma unroll
-                for (int i = 0; i < RPL; ++i) r[i] = fmaf(k3[i], T, base[i]);
+                for (int i = 0; i < RPL; ++i) {
+                    r[i] = fmaf(k3[i], T, base[i]);
+                    rr[i] = rcp_fast(r[i]);
+                    pc[i] = ((hotm >> i) & 1u) ? wcx[i] * rr[i] : 0.0f;
+                }
+                // ================= half-step 2: c = K~^T u' on the demand ranks, v' = d / c
+                xtot[1][warp] = partial(false, pc, base);
                 if (TOL) {
-                    const bool check_now = until_check == 1;
-                    until_check = check_now ? a.check_every : until_check - 1;
+                    bool check_now = true;
+                    if (!every) {
+                        check_now = until_check == 1;
+                        until_check = check_now ? a.check_every : until_check - 1;
+                    }
                     if (check_now) {               // this lane's term of the row error, for the ninth warp
                         float e = 0.0f;
 #pragma unroll
                         for (int i = 0; i < RPL; ++i) {
-                            const bool ok = r[i] > kSumLo && r[i] < kSumHi;
-                            e += ((hotm >> i) & 1u) ? (ok ? fabsf(fmaf(z[i], r[i], -x[i])) : INFINITY) : 0.0f;
+                            e += ((hotm >> i) & 1u) ? fabsf(fmaf(z[i], r[i], -x[i])) : 0.0f;
                             zkeep[i] = z[i];
                         }
                         xe[tid] = e;
@@ -328,61 +354,61 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
                 }
                 float zn[RPL];
 #pragma unroll
-                for (int i = 0; i < RPL; ++i) zn[i] = ((hotm >> i) & 1u) ? x[i] * rcp_fast(r[i]) : z[i];
-                // ================= half-step 2: c = K~^T u' on the demand ranks, v' = d / c
-                tw = partial(false, wc, zn, base);
-                if (lane == 0) xtot[k & 1][warp] = tw;
+                for (int i = 0; i < RPL; ++i) zn[i] = ((hotm >> i) & 1u) ? x[i] * rr[i] : z[i];
                 bar_loop(NT);
-                T = total_of(k & 1);
-                ++k;
+                T = total_of(1);
                 // a sum outside the safe range shows in its reciprocal (zero, infinite or not a number), so the
                 // drift test catches it too; a rank that takes no part keeps z = 1
+                ++t;
                 bool drift = false;
 #pragma unroll
                 for (int i = 0; i < RPL; ++i) {
                     const float c = fmaf(k3[i], T, base[i]);
-                    z[i] = ((coldm >> i) & 1u) ? x[i] * rcp_fast(c) : zn[i];
+                    const float rc = rcp_fast(c);
+                    pr[i] = ((coldm >> i) & 1u) ? wrx[i] * rc : 0.0f;
+                    z[i] = ((coldm >> i) & 1u) ? x[i] * rc : zn[i];
                     drift |= (__float_as_uint(z[i]) - lo_bits) > span_bits;
                 }
-                if (drift) xword[0] = k;           // read after the next exchange's barrier; every writer stores the same k
-                ++t;
+                if (drift) { xev[2] = t; xev[0] = t; }     // read after the next barrier; every writer stores the same t
             }
         } else {
             // the ninth warp: the same barriers, the same events; between half-step 2's barrier and the next one it
             // sums the 256 terms of the row error (eight per lane, then five shuffle levels: one fixed order)
             for (;;) {
                 bar_loop(NT);
-                const int2 xw = *reinterpret_cast<const int2*>(xword);
-                event = (TOL && xw.y == t - 1) ? kEvStop : (xw.x == k ? kEvDrift : (t >= a.max_iters ? kEvLast : 0));
-                ++k;
-                if (event) break;
-                const bool check_now = until_check == 1;
-                until_check = check_now ? a.check_every : until_check - 1;
+                if (xev[0] <= t) break;
+                bool check_now = true;
+                if (!every) {
+                    check_now = until_check == 1;
+                    until_check = check_now ? a.check_every : until_check - 1;
+                }
                 bar_loop(NT);
-                ++k;
+                ++t;
                 if (check_now) {
                     const float4 lo = *reinterpret_cast<const float4*>(&xe[lane * 8]);
                     const float4 hi = *reinterpret_cast<const float4*>(&xe[lane * 8 + 4]);
                     float e = ((lo.x + lo.y) + (lo.z + lo.w)) + ((hi.x + hi.y) + (hi.z + hi.w));
 #pragma unroll
                     for (int o = 1; o < 32; o <<= 1) e += __shfl_xor_sync(kFull, e, o);
-                    if (lane == 0 && e <= tol_abs_f) xword[1] = t;
+                    if (lane == 0 && e <= tol_abs_f) { xev[1] = t; xev[0] = t; }
                 }
-                ++t;
             }
         }
         // ---- an event: every thread of the block is here, after the barrier of half-step 1 of iteration t
-        if (event == kEvStop) {                    // iterate t - 1 met the tolerance: it is the result
+        const int ev_stop = xev[1], ev_drift = xev[2];
+        __syncthreads();
+        if (TOL && ev_stop == t) {                 // iterate t - 1 met the tolerance: it is the result
             --t;
 #pragma unroll
             for (int i = 0; i < RPL; ++i) z[i] = zkeep[i];
             double err;
             int bad;
-            exact_error(r, err, bad);              // no row sum is out of range here: its term would have been infinite
+            exact_error(r, err, bad);
+            if (bad) { if (tid == 0) a.iters[b] = kHandBack; return; }
             err_out = (float)(err / sum_st);
             break;
         }
-        if (event == kEvDrift) {
+        if (ev_drift == t) {
             // Some u~ or v~ of the previous update left [e^-40, e^40].  Either a sum left the safe range -- its
             // reciprocal is then zero, infinite, not a number or far outside any drift -- and the problem is handed
             // back, or the factors drifted: fold them into the potentials and take the half-step again.
@@ -394,10 +420,11 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
                 if (tid == 0) a.iters[b] = kHandBack;
                 return;
             }
+            if (tid == 0) { xev[0] = a.max_iters; xev[2] = -1; }
             fold();
             continue;
         }
-        // kEvLast: iterate t is the result whatever its error
+        // the last iteration: iterate t is the result whatever its error
 #pragma unroll
         for (int i = 0; i < RPL; ++i) r[i] = fmaf(k3[i], T, base[i]);
         double err;
@@ -412,10 +439,9 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
     // ---- T = diag(u) M diag(v) from the total potentials, then the column cap
     fold();
     {
-        const float tw = partial(false, wc, z, base);                           // column sums of K~ itself (u~ = 1)
-        if (lane == 0) xtot[k & 1][warp] = tw;
+        xtot[0][warp] = partial(false, wc, base);                               // column sums of K~ itself (u~ = 1)
         __syncthreads();
-        const float T = total_of(k & 1);
+        const float T = total_of(0);
 #pragma unroll
         for (int i = 0; i < RPL; ++i) {
             const float c = fmaf(k3[i], T, base[i]);
