@@ -348,12 +348,14 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count, match_cyc=None):
         r2, r3 = int(rounds[w, 0]), int(rounds[w, 1])
         d["rounds"] = dict(
             slowest_layer=w, phase2_rounds=r2, phase3_rounds=r3, kernel_cycles=c[5],
-            share=dict(setup=(c[0] + c[2]) / c[5], phase2=c[1] / c[5], phase3_bids=c[3] / c[5], phase3_updates=c[4] / c[5]),
+            share=dict(setup=(c[0] + c[2]) / c[5], phase2=c[1] / c[5], phase3_rounds=c[12] / c[5]),
             phase2_cycles_per_round=c[1] / max(1, r2),
-            phase3_cycles_per_round=dict(bid_to_first_barrier=c[3] / max(1, r3), update_to_second_barrier=c[4] / max(1, r3),
+            phase3_cycles_per_round=dict(whole_round=c[12] / max(1, r3), bid_to_first_barrier=c[3] / max(1, r3), update_to_second_barrier=c[4] / max(1, r3),
                                          busiest_thread_probe=c[6] / max(1, r3), busiest_thread_arbitration=c[7] / max(1, r3)),
             phase2_split=dict(scan_and_arbitration=c[8], winners=c[9], served_rows=c[10], all_keys_per_slot_index=c[11]),
-            ns_per_phase3_round_at_max_clock=(c[3] + c[4]) / max(1, r3) / (peaks["sm_max_mhz"] * 1e-3))
+            ns_per_phase3_round_at_max_clock=c[12] / max(1, r3) / (peaks["sm_max_mhz"] * 1e-3),
+            note="cycle counts of the counting build of the kernel (every thread reads the clock three times a round): "
+                 "an upper bound on the timed build, whose stage time is `stages_ms.match_auction`")
     return d
 
 

@@ -49,7 +49,9 @@ int taot_get_group_trace(taot_handle_t h, int32_t* groups, float* h_ms /* [4][6]
  *   4 Phase-3 updates (to the barrier that ends the round), 5 the whole kernel, 6 / 7 the probe and the
  *   arbitration time of the thread that spent most on each (its own time, no waiting at barriers),
  *   8-11 Phase 2 split: rank scans + arbitration, winners, re-forming the served experts' keys, forming all keys
- *   once per slot index; 12-15 zero.
+ *   once per slot index; 12 the Phase-3 loop as a whole (3 and 4 are what thread 0 sees between its own clock reads:
+ *   loads of the next round that the compiler starts before the round's first clock read fall outside them, and the
+ *   counting build itself is slower than the timed one, so 12 / rounds is an upper bound per round); 13-15 zero.
  * `ws` is the workspace of the profiled call.  Errors: TAOT_ERR_NULL, TAOT_ERR_UNSUPPORTED (R > 256).
  */
 int taot_get_match_cycles(taot_handle_t h, const void* ws, int64_t* h_cycles /* [L][16] */);

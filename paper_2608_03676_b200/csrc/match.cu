@@ -57,7 +57,7 @@ struct MatchArgs {
     long long* cyc;              // [L][16] SM cycles per part of the kernel as thread 0 sees them, or null (profiling aid):
                                  // 0 set-up, 1 Phase 2, 2 Phase-3 set-up, 3 Phase-3 bids (to the first barrier of a round),
                                  // 4 Phase-3 updates (to the second barrier), 5 whole kernel, 6 / 7 the busiest thread's own
-                                 // probe and arbitration time in Phase 3
+                                 // probe and arbitration time in Phase 3, 8-11 Phase-2 split, 12 the Phase-3 loop as a whole
 };
 
 __device__ __forceinline__ uint32_t ordered_bits(float f)
@@ -438,7 +438,7 @@ match_kernel(MatchArgs a)
 
     // =========================================================== Phase 3
     const long long c_p3 = timed ? clock64() : 0;
-    long long c_p3loop = c_p3;
+    long long c_p3loop = c_p3, c_p3end = c_p3;
     // compact the experts that sit in some slot; keep their per-rank remaining counts transposed [col][r]
     for (int e = tid; e < E; e += NT) dcol[e] = -1;
     if (tid == 0) s_cnt = 0;
@@ -625,6 +625,7 @@ match_kernel(MatchArgs a)
             bar_part(NP);
             if (TIMED && timed) { const long long c_r2 = clock64(); c_bid += c_r1 - c_r0; c_upd += c_r2 - c_r1; }
         }
+        if (timed) c_p3end = clock64();
         if (s < S) slot_a[s] = A;
         __syncthreads();
     } else {
@@ -690,8 +691,13 @@ match_kernel(MatchArgs a)
         __shared__ unsigned long long s_mx[2];
         if (tid == 0) { s_mx[0] = 0; s_mx[1] = 0; }
         __syncthreads();
-        atomicMax(&s_mx[0], (unsigned long long)c_probe);
-        atomicMax(&s_mx[1], (unsigned long long)c_atom);
+        unsigned long long mp = (unsigned long long)c_probe, ma = (unsigned long long)c_atom;
+        for (int o = 16; o > 0; o >>= 1) {        // one atomic per warp: 64-bit shared-memory atomics from every thread
+            const unsigned long long op = __shfl_xor_sync(0xffffffffu, mp, o), oa = __shfl_xor_sync(0xffffffffu, ma, o);
+            mp = op > mp ? op : mp;               // would cost more than the rounds they report on
+            ma = oa > ma ? oa : ma;
+        }
+        if ((tid & 31) == 0) { atomicMax(&s_mx[0], mp); atomicMax(&s_mx[1], ma); }
         __syncthreads();
         c_probe = (long long)s_mx[0]; c_atom = (long long)s_mx[1];
     }
@@ -703,7 +709,8 @@ match_kernel(MatchArgs a)
             c[0] = c_p2 - c_start; c[1] = c_p3 - c_p2; c[2] = c_p3loop - c_p3; c[3] = c_bid; c[4] = c_upd;
             c[5] = clock64() - c_start; c[6] = c_probe; c[7] = c_atom;
             c[8] = c_scan; c[9] = c_win; c[10] = c_row; c[11] = c_build;
-            for (int i = 12; i < 16; ++i) c[i] = 0;
+            c[12] = c_p3end - c_p3loop;
+            for (int i = 13; i < 16; ++i) c[i] = 0;
         }
     }
 }
