@@ -58,6 +58,12 @@ __device__ __forceinline__ void st_stream(int4* p, const int4& v)
     asm volatile("st.global.cs.v4.s32 [%0], {%1,%2,%3,%4};" :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
+__device__ __forceinline__ void st_once(int4* p, const int4& v, uint64_t pol)
+{
+    asm volatile("st.global.L1::no_allocate.L2::cache_hint.v4.s32 [%0], {%1,%2,%3,%4}, %5;"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "l"(pol) : "memory");
+}
+
 __device__ __forceinline__ void chunk_geometry(const AssignArgs& a, int64_t id, int64_t& goff, int32_t& len)
 {
     const int32_t c = (int32_t)(id % a.nc);
@@ -400,6 +406,18 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
+// the same with an L2 policy for data that is read once: first in line for eviction
+__device__ __forceinline__ uint64_t policy_evict_first()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void bulk_load_once(void* dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t pol)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol) : "memory");
+}
 // Poll until the phase with the given parity completes; false if the spin bound ran out.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
 {
@@ -440,9 +458,10 @@ assign_chunk_kernel(AssignArgs a, int only_split)
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
             const uint32_t bytes = (uint32_t)len * 4u;
             mbar_expect_tx(&bar, bytes);
+            const uint64_t once = policy_evict_first();
             for (uint32_t o = 0; o < bytes; o += kBulkPiece)
-                bulk_load(reinterpret_cast<unsigned char*>(stage) + o, reinterpret_cast<const unsigned char*>(buf) + o,
-                          (bytes - o) < kBulkPiece ? (bytes - o) : kBulkPiece, &bar);
+                bulk_load_once(reinterpret_cast<unsigned char*>(stage) + o, reinterpret_cast<const unsigned char*>(buf) + o,
+                               (bytes - o) < kBulkPiece ? (bytes - o) : kBulkPiece, &bar, once);
         }
         buf = stage;
     }
@@ -512,6 +531,7 @@ assign_stream_kernel(AssignArgs a, int stages, uint32_t off_tab, int64_t nchunks
     if (warp == 0) {
         if (lane == 0) {
             long long armed_mask = 0;                    // stages whose copies may still be in flight
+            const uint64_t once = policy_evict_first();
             for (int64_t use = 0;; ++use) {
                 const int st = (int)(use % stages);
                 if (use >= stages) {                     // wait until the consumers have left this stage
@@ -539,7 +559,7 @@ assign_stream_kernel(AssignArgs a, int stages, uint32_t off_tab, int64_t nchunks
                 unsigned char* dstb = smem + (size_t)st * TAOT_CHUNK * 4;
                 const unsigned char* srcb = reinterpret_cast<const unsigned char*>(a.topk + goff);
                 for (uint32_t o = 0; o < bytes; o += kBulkPiece)
-                    bulk_load(dstb + o, srcb + o, (bytes - o) < kBulkPiece ? (bytes - o) : kBulkPiece, &full[st]);
+                    bulk_load_once(dstb + o, srcb + o, (bytes - o) < kBulkPiece ? (bytes - o) : kBulkPiece, &full[st], once);
                 bulk_load(smem + off_tab + (size_t)st * E * 4, a.tabg + id * (int64_t)(E + kRowTail), (uint32_t)E * 4u, &full[st]);
                 armed_mask |= 1ll << st;
             }
@@ -547,6 +567,7 @@ assign_stream_kernel(AssignArgs a, int stages, uint32_t off_tab, int64_t nchunks
         }
     } else {
         const int c = tid - 32;
+        const uint64_t wpol = policy_evict_first();
         for (int64_t use = 0;; ++use) {
             const int st = (int)(use % stages);
             if (!mbar_wait(&full[st], (uint32_t)((use / stages) & 1))) {
@@ -578,7 +599,7 @@ assign_stream_kernel(AssignArgs a, int stages, uint32_t off_tab, int64_t nchunks
                         o.y = (unsigned)o.y < (unsigned)E ? tab[o.y] : o.y;
                         o.z = (unsigned)o.z < (unsigned)E ? tab[o.z] : o.z;
                         o.w = (unsigned)o.w < (unsigned)E ? tab[o.w] : o.w;
-                        st_stream(dst + i, o);
+                        st_once(dst + i, o, wpol);
                     }
                 }
             }
