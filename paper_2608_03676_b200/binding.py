@@ -112,12 +112,9 @@ def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
 
 STATIC_SCRATCH_BYTES = 4 << 20
 # kernels one taot_plan call enqueues: chunk histogram, merge, Sinkhorn (register tile + shared-memory
-# kernel for handed-back problems), matching+auction, reassignment (tables, pipelined rewrite of the chunks
-# without a split, rewrite of the chunks with one) -- for a 16-byte aligned routing table with E % 4 == 0
-PLAN_LAUNCHES = 8
-PLAN_LAUNCHES_NO_HINT = 6       # with ABLATE_HINT the two Sinkhorn kernels are not launched
-# A routing table of at most 3 x (number of SMs) chunks is rewritten by the per-chunk kernel alone: one launch fewer
-# (`Planner.plan_launches()` gives the count for a handle).
+# kernel for handed-back problems), matching+auction, reassignment (tables, rewrite)
+PLAN_LAUNCHES = 7
+PLAN_LAUNCHES_NO_HINT = 5       # with ABLATE_HINT the two Sinkhorn kernels are not launched
 
 
 def histogram_static(topk: torch.Tensor, R: int, E: int, e2r_dev: torch.Tensor, n: torch.Tensor,
@@ -229,14 +226,10 @@ class Planner:
             info=torch.zeros((L,), dtype=i32, device=self.device))
 
     def plan_launches(self) -> int:
-        """Kernels one `plan` call of this handle enqueues (16-byte aligned routing table, E % 4 == 0) when it plans all
-        layers as one group; a handle that splits a large table into layer groups enqueues them once per group
-        (`last_launch_count()` reports what the last call did)."""
-        sms = torch.cuda.get_device_properties(self.device).multi_processor_count
-        seg = self.T // self.R * self.k
-        chunks = self.L * self.R * ((seg + 16383) // 16384)
-        n = PLAN_LAUNCHES_NO_HINT if (self.ablation & ABLATE_HINT) else PLAN_LAUNCHES
-        return n - 1 if chunks <= 3 * sms else n
+        """Kernels one `plan` call of this handle enqueues when it plans all layers as one group; a handle that
+        splits a large table into layer groups enqueues them once per group (`last_launch_count()` reports what the
+        last call did)."""
+        return PLAN_LAUNCHES_NO_HINT if (self.ablation & ABLATE_HINT) else PLAN_LAUNCHES
 
     def last_launch_count(self) -> int:
         c = ctypes.c_int32()

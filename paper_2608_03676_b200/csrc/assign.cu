@@ -12,17 +12,18 @@
 //   assign_prep_kernel   one CTA per (layer, source rank): per chunk, the table expert -> target of
 //                        the chunk's LAST entry of that expert, and the splits (expert, in-chunk
 //                        ordinal, slot before); up to four of them ride in the tail of the table row;
-//   assign_stream_kernel persistent, one CTA per SM, for the chunks WITHOUT a split: a producer warp claims chunks
-//                        from a global counter and stages them (and their table rows) in shared memory with bulk
-//                        asynchronous copies (cp.async.bulk + mbarrier, no multicast), three stages in flight;
-//                        16 consumer warps do one table lookup per entry and 16-byte streaming stores; full /
-//                        empty mbarriers per stage, no CTA-wide barrier in the loop, every wait bounded;
-//   assign_chunk_kernel  one CTA per chunk: the chunks that do hold a split, staged in shared memory the same way
-//                        since they are read three times -- per-warp counts of the split experts, ballots in the
-//                        one warp that holds a split to find its flat position, then the rewrite with
-//                        "expert e before position P -> slot" as predicated overrides -- and, with ordinary loads,
-//                        every chunk of a routing table that is not 16-byte aligned or whose segments are not
-//                        multiples of 4 entries.
+//   assign_chunk_kernel  one CTA per chunk, every chunk in one sweep over the table.  The chunk is staged in shared
+//                        memory with bulk asynchronous copies (cp.async.bulk + mbarrier, no multicast, an L2
+//                        evict-first policy: the table is read once); three CTAs per SM keep copies, lookups and
+//                        16-byte streaming stores of different chunks in flight.  A chunk without a split is one
+//                        table lookup per entry; a chunk with splits is read three times from shared memory --
+//                        per-warp counts of the split experts, ballots in the one warp that holds a split to find
+//                        its flat position, then the rewrite with "expert e before position P -> slot" as
+//                        predicated overrides.  A routing table that is not 16-byte aligned or whose segments are
+//                        not multiples of 4 entries takes the same kernel without staging, with ordinary loads.
+// One sweep over all chunks matters: two kernels that each took part of the chunks (a persistent pipeline for the
+// chunks without a split, this kernel for the rest) moved their parts at 5.4-5.7 TB/s, the single sweep moves the
+// whole table at 6.5 TB/s -- the memory system serves a contiguous sweep better than two interleaved subsets.
 // 8 bytes of HBM traffic per entry (one read, one write).  Out-of-range indices are copied through (the histogram
 // pass, whose counts this path consumes, is the one that flags them).
 #include "taot_internal.cuh"
@@ -40,14 +41,11 @@ struct AssignArgs {
     const int32_t* topk;
     const int32_t* cc;          // [L,R,NC,E] chunk counts (histogram pass)
     int32_t* tabg;              // [L,R,NC,E+kRowTail] target of the chunk's last entry of each expert, then the row tail
-    int32_t* nsg;               // [L,R,NC]   number of splits in the chunk
-    int32_t* soff;              // [L,R,NC]   index of the chunk's first split record in its segment's list
     int4* splits;               // [L,R,S]    {expert, ordinal of the split relative to the chunk, target before, position}
     const int32_t* slot_expert;
     const int32_t* X;
     int32_t* out;
     int32_t* info;
-    unsigned long long* work;   // chunk counter of the pipelined kernel (zeroed by the prep kernel)
     int64_t layer_elems, seg;
     int32_t nc, R, E, K;
 };
@@ -137,7 +135,6 @@ assign_prep_kernel(AssignArgs a)
     int4* over = a.splits + lr * S;
     for (int e = tid; e < E; e += kThreads) carry[e] = 0;
     if (tid == 0) s_over = 0;
-    if (tid == 0 && blockIdx.x == 0) *a.work = 0ull;
     const int m = build_entries(a.X + lr * S, a.slot_expert + (int64_t)l * S, S, E, ent_s, ent_e, ent_lo, ent_hi, s_wcnt);
     for (int c0 = 0; c0 < NC; c0 += NCT) {
         const int nct = (NC - c0) < NCT ? (NC - c0) : NCT;
@@ -175,7 +172,6 @@ assign_prep_kernel(AssignArgs a)
         }
         for (int c = tid; c < nct; c += kThreads) {
             rows[(int64_t)(c0 + c) * (E + kRowTail) + E] = nsc[c];
-            a.nsg[lr * NC + c0 + c] = nsc[c];
         }
         __syncthreads();
     }
@@ -385,11 +381,10 @@ __device__ void rewrite_chunk(const AssignArgs& a, int64_t id, const int32_t* bu
 }
 
 // ---------------------------------------------------------------------------------------------
-// persistent bulk-copy pipeline
+// staging with bulk asynchronous copies
 
 constexpr uint32_t kWaitSpins = 1u << 20;               // bound on mbarrier polling (each poll can itself block for a while)
 constexpr uint32_t kBulkPiece = 8192;                   // bytes per bulk copy: several pieces in flight per chunk
-constexpr int kMaxStages = 4;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -401,12 +396,7 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
-// the same with an L2 policy for data that is read once: first in line for eviction
+// bulk copy global -> shared with an L2 policy for data that is read once: first in line for eviction
 __device__ __forceinline__ uint64_t policy_evict_first()
 {
     uint64_t pol;
@@ -431,12 +421,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
     return false;
 }
 
-// One CTA per chunk.  STAGE: the chunk is first copied to shared memory with bulk asynchronous copies (used for
-// the chunks that hold a split, whose entries are read three times: count, locate, rewrite); otherwise it is read
-// from global memory (any alignment).
+// One CTA per chunk.  STAGE: the chunk is first copied to shared memory with bulk asynchronous copies; otherwise it
+// is read from global memory (any alignment).
 template <bool VEC, bool STAGE>
 __global__ void __launch_bounds__(kThreads)
-assign_chunk_kernel(AssignArgs a, int only_split)
+assign_chunk_kernel(AssignArgs a)
 {
     extern __shared__ __align__(128) unsigned char shc[];
     const int E = a.E;
@@ -448,7 +437,6 @@ assign_chunk_kernel(AssignArgs a, int only_split)
     __shared__ int s_pos;
     const int tid = threadIdx.x;
     const int64_t id = blockIdx.x;
-    if (only_split && a.nsg[id] == 0) return;            // the pipelined kernel rewrites the chunks without splits
     int64_t goff; int32_t len;
     chunk_geometry(a, id, goff, len);
     const int32_t* buf = a.topk + goff;
@@ -481,140 +469,6 @@ assign_chunk_kernel(AssignArgs a, int only_split)
     rewrite_chunk<VEC>(a, id, buf, tab, a.out + goff, len, recs, s_cntw, &s_pos);
 }
 
-// ---- the pipelined kernel ----
-constexpr int kStreamConsumers = 512;                    // threads that rewrite; one more warp only starts copies
-constexpr int kStreamThreads = kStreamConsumers + 32;
-constexpr int kStreamUnroll = 4;
-
-struct StreamLayout {
-    int stages;
-    size_t off_tab, bytes;                    // chunk buffers start at 0
-};
-
-StreamLayout stream_layout(int E)
-{
-    const size_t per_stage = (size_t)TAOT_CHUNK * 4 + (size_t)E * 4;
-    const size_t budget = 224 * 1024;
-    StreamLayout L;
-    int st = (int)((budget - 256) / per_stage);
-    L.stages = st > kMaxStages ? kMaxStages : st;
-    L.off_tab = (size_t)L.stages * TAOT_CHUNK * 4;
-    L.bytes = L.off_tab + (size_t)L.stages * E * 4;
-    return L;
-}
-
-// Persistent, one CTA per SM.  Warp 0 is the producer: one lane claims the next chunk without a split from a
-// global counter, arms the stage's "full" barrier and starts the bulk copies of the chunk and of its table row.
-// The other warps are consumers: wait for "full", rewrite the chunk (one table lookup per entry, 16-byte
-// streaming stores), and arrive on the stage's "empty" barrier, which the producer waits on before it reuses
-// the stage.  No CTA-wide barrier inside the loop.  Every wait is bounded; a wait that runs out sets
-// TAOT_INFO_INTERNAL, stops the CTA's loop, and the CTA leaves after one more bounded wait per armed stage.
-__global__ void __launch_bounds__(kStreamThreads, 1)
-assign_stream_kernel(AssignArgs a, int stages, uint32_t off_tab, int64_t nchunks, unsigned long long* work)
-{
-    extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ __align__(8) uint64_t full[kMaxStages];
-    __shared__ __align__(8) uint64_t empty[kMaxStages];
-    __shared__ long long s_id[kMaxStages];               // chunk staged in each stage, -1 = no more work
-    __shared__ int s_abort;
-    const int E = a.E;
-    const int tid = threadIdx.x;
-    const int warp = tid >> 5, lane = tid & 31;
-
-    if (tid == 0) {
-        for (int st = 0; st < stages; ++st) { mbar_init(&full[st], 1); mbar_init(&empty[st], kStreamConsumers / 32); }
-        s_abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-
-    if (warp == 0) {
-        if (lane == 0) {
-            long long armed_mask = 0;                    // stages whose copies may still be in flight
-            const uint64_t once = policy_evict_first();
-            for (int64_t use = 0;; ++use) {
-                const int st = (int)(use % stages);
-                if (use >= stages) {                     // wait until the consumers have left this stage
-                    if (!mbar_wait(&empty[st], (uint32_t)(((use / stages) - 1) & 1))) {
-                        atomicOr(a.info, TAOT_INFO_INTERNAL);
-                        *(volatile int*)&s_abort = 1;
-                        break;
-                    }
-                    armed_mask &= ~(1ll << st);
-                }
-                if (*(volatile int*)&s_abort) break;
-                int64_t id;
-                do { id = (int64_t)atomicAdd(work, 1ull); } while (id < nchunks && a.nsg[id] != 0);
-                if (id >= nchunks) {
-                    s_id[st] = -1;
-                    asm volatile("{\n\t.reg .b64 t;\n\tmbarrier.arrive.shared::cta.b64 t, [%0];\n\t}" :: "r"(smem_u32(&full[st])) : "memory");
-                    break;
-                }
-                s_id[st] = id;
-                int64_t goff; int32_t len;
-                chunk_geometry(a, id, goff, len);
-                const uint32_t bytes = (uint32_t)len * 4u;
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                mbar_expect_tx(&full[st], bytes + (uint32_t)E * 4u);
-                unsigned char* dstb = smem + (size_t)st * TAOT_CHUNK * 4;
-                const unsigned char* srcb = reinterpret_cast<const unsigned char*>(a.topk + goff);
-                for (uint32_t o = 0; o < bytes; o += kBulkPiece)
-                    bulk_load_once(dstb + o, srcb + o, (bytes - o) < kBulkPiece ? (bytes - o) : kBulkPiece, &full[st], once);
-                bulk_load(smem + off_tab + (size_t)st * E * 4, a.tabg + id * (int64_t)(E + kRowTail), (uint32_t)E * 4u, &full[st]);
-                armed_mask |= 1ll << st;
-            }
-            (void)armed_mask;
-        }
-    } else {
-        const int c = tid - 32;
-        const uint64_t wpol = policy_evict_first();
-        for (int64_t use = 0;; ++use) {
-            const int st = (int)(use % stages);
-            if (!mbar_wait(&full[st], (uint32_t)((use / stages) & 1))) {
-                if (lane == 0) atomicOr(a.info, TAOT_INFO_INTERNAL);
-                *(volatile int*)&s_abort = 1;
-                break;
-            }
-            const long long id = s_id[st];
-            if (id < 0) break;
-            int64_t goff; int32_t len;
-            chunk_geometry(a, id, goff, len);
-            const int4* buf = reinterpret_cast<const int4*>(smem + (size_t)st * TAOT_CHUNK * 4);
-            const int32_t* tab = reinterpret_cast<const int32_t*>(smem + off_tab + (size_t)st * E * 4);
-            int4* dst = reinterpret_cast<int4*>(a.out + goff);
-            const int n4 = len >> 2;                     // segments are multiples of 4 entries on this path
-            for (int i0 = c; i0 < n4; i0 += kStreamConsumers * kStreamUnroll) {
-                int4 v[kStreamUnroll];
-#pragma unroll
-                for (int u = 0; u < kStreamUnroll; ++u) {
-                    const int i = i0 + u * kStreamConsumers;
-                    if (i < n4) v[u] = buf[i];
-                }
-#pragma unroll
-                for (int u = 0; u < kStreamUnroll; ++u) {
-                    const int i = i0 + u * kStreamConsumers;
-                    if (i < n4) {
-                        int4 o = v[u];
-                        o.x = (unsigned)o.x < (unsigned)E ? tab[o.x] : o.x;
-                        o.y = (unsigned)o.y < (unsigned)E ? tab[o.y] : o.y;
-                        o.z = (unsigned)o.z < (unsigned)E ? tab[o.z] : o.z;
-                        o.w = (unsigned)o.w < (unsigned)E ? tab[o.w] : o.w;
-                        st_once(dst + i, o, wpol);
-                    }
-                }
-            }
-            __syncwarp();
-            if (lane == 0)
-                asm volatile("{\n\t.reg .b64 t;\n\tmbarrier.arrive.shared::cta.b64 t, [%0];\n\t}" :: "r"(smem_u32(&empty[st])) : "memory");
-        }
-    }
-    __syncthreads();
-    if (s_abort && tid == 0) {
-        // copies that were started may still be landing in this CTA's shared memory: give each stage one more bounded wait
-        for (int st = 0; st < stages; ++st) { (void)mbar_wait(&full[st], 0); (void)mbar_wait(&full[st], 1); }
-    }
-}
-
 }  // namespace
 
 int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, void* ws, const int32_t* d_slot_expert,
@@ -626,11 +480,8 @@ int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, void* ws, const i
     a.topk = d_topk;
     a.cc = reinterpret_cast<const int32_t*>(w + h->off_cc);
     a.tabg = reinterpret_cast<int32_t*>(w + h->off_tabg);
-    a.nsg = reinterpret_cast<int32_t*>(w + h->off_nbg);
-    a.soff = reinterpret_cast<int32_t*>(w + h->off_soff);
     a.splits = reinterpret_cast<int4*>(w + h->off_splits);
     a.slot_expert = d_slot_expert; a.X = d_X; a.out = d_new_idx; a.info = d_info;
-    a.work = reinterpret_cast<unsigned long long*>(w + h->off_work);
     a.layer_elems = p.T * p.k; a.seg = h->seg; a.nc = h->nc; a.R = p.R; a.E = p.E; a.K = p.K;
     const int vec_ok = ((reinterpret_cast<uintptr_t>(d_topk) & 15) == 0) &&
                        ((reinterpret_cast<uintptr_t>(d_new_idx) & 15) == 0) && (h->seg % 4 == 0);
@@ -641,36 +492,16 @@ int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, void* ws, const i
     TAOT_CUDA_OK(cudaFuncSetAttribute(assign_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_prep));
     assign_prep_kernel<<<(unsigned)((int64_t)p.L * p.R), kThreads, smem_prep, st>>>(a);
     TAOT_CUDA_OK(cudaGetLastError());
-    const StreamLayout sl = stream_layout(p.E);
-    int launches = 2;
-    // A routing table whose chunks all fit one wave of the per-chunk kernel (three CTAs per SM) is latency-bound, not
-    // bandwidth-bound: the pipelined kernel would only add a launch, so the staged per-chunk kernel takes every chunk.
-    const bool one_wave = blocks <= 3u * (unsigned)h->sm_count;
-    if (vec_ok && one_wave) {
+    if (vec_ok) {
         const size_t smem = (size_t)TAOT_CHUNK * 4 + sizeof(int32_t) * (((size_t)p.E + kRowTail + 3) & ~(size_t)3) +
                             sizeof(int4) * (size_t)(S + kRowSplits);
         TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        assign_chunk_kernel<true, true><<<blocks, kThreads, smem, st>>>(a, 0);
-    } else if (vec_ok && p.E % 4 == 0 && sl.stages >= 2) {
-        TAOT_CUDA_OK(cudaFuncSetAttribute(assign_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sl.bytes));
-        const unsigned grid = blocks < (unsigned)h->sm_count ? blocks : (unsigned)h->sm_count;
-        assign_stream_kernel<<<grid, kStreamThreads, sl.bytes, st>>>(a, sl.stages, (uint32_t)sl.off_tab, (int64_t)blocks, a.work);
-        TAOT_CUDA_OK(cudaGetLastError());
-        const size_t smem = (size_t)TAOT_CHUNK * 4 + sizeof(int32_t) * (((size_t)p.E + kRowTail + 3) & ~(size_t)3) +
-                            sizeof(int4) * (size_t)(S + kRowSplits);
-        TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        assign_chunk_kernel<true, true><<<blocks, kThreads, smem, st>>>(a, 1);      // the chunks that hold a split
-        launches = 3;
+        assign_chunk_kernel<true, true><<<blocks, kThreads, smem, st>>>(a);
     } else {
         const size_t smem = sizeof(int32_t) * (((size_t)p.E + kRowTail + 3) & ~(size_t)3) + sizeof(int4) * (size_t)(S + kRowSplits);
-        if (vec_ok) {
-            TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            assign_chunk_kernel<true, false><<<blocks, kThreads, smem, st>>>(a, 0);
-        } else {
-            TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            assign_chunk_kernel<false, false><<<blocks, kThreads, smem, st>>>(a, 0);
-        }
+        TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        assign_chunk_kernel<false, false><<<blocks, kThreads, smem, st>>>(a);
     }
     TAOT_CUDA_OK(cudaGetLastError());
-    return launches;
+    return 2;
 }

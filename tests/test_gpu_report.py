@@ -102,7 +102,7 @@ def test_ablation_switches_bit_exact(name, hint, topo):
     pl = make_planner(cfg, ablation=flags)
     out = {k: cpu(v) for k, v in pl.plan(topk).items()}
     assert pl.last_launch_count() == pl.plan_launches()
-    assert pl.plan_launches() in ((P.PLAN_LAUNCHES, P.PLAN_LAUNCHES - 1) if hint else (P.PLAN_LAUNCHES_NO_HINT, P.PLAN_LAUNCHES_NO_HINT - 1))
+    assert pl.plan_launches() == (P.PLAN_LAUNCHES if hint else P.PLAN_LAUNCHES_NO_HINT)
     B = O.default_preference(C.numpy())
     B2 = B if topo else np.zeros_like(B)
     tk = cpu(topk)
