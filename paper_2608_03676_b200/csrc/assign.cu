@@ -34,6 +34,7 @@ constexpr int kThreads = TAOT_STREAM_THREADS;
 constexpr int kWarps = kThreads / 32;
 constexpr int kWarpSpan = TAOT_CHUNK / kWarps;           // entries one warp owns, contiguous: 2048
 constexpr int kIters = kWarpSpan / 128;                  // 16-byte accesses per lane: 16
+constexpr int kPrepThreads = 64;                         // the table build is a chain of short dependent steps per (layer, rank): many small CTAs
 constexpr int kRowSplits = 4;                            // split records that ride in the tail of a table row
 constexpr int kRowTail = 4 + 4 * kRowSplits;             // {ns, soff, 0, 0} + records {expert, rel / -, target before, position}
 
@@ -54,12 +55,6 @@ struct AssignArgs {
 __device__ __forceinline__ void st_stream(int4* p, const int4& v)
 {
     asm volatile("st.global.cs.v4.s32 [%0], {%1,%2,%3,%4};" :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-
-__device__ __forceinline__ void st_once(int4* p, const int4& v, uint64_t pol)
-{
-    asm volatile("st.global.L1::no_allocate.L2::cache_hint.v4.s32 [%0], {%1,%2,%3,%4}, %5;"
-                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "l"(pol) : "memory");
 }
 
 __device__ __forceinline__ void chunk_geometry(const AssignArgs& a, int64_t id, int64_t& goff, int32_t& len)
@@ -111,7 +106,7 @@ __device__ int build_entries(const int32_t* Xrow, const int32_t* se, int S, int 
 // chunks of a segment handled per pass of the prep kernel (bounds its shared memory)
 __host__ __device__ inline int prep_tile(int E) { const int t = 6144 / E; return t < 1 ? 1 : (t > 32 ? 32 : t); }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kPrepThreads)
 assign_prep_kernel(AssignArgs a)
 {
     extern __shared__ int32_t sh[];
@@ -133,21 +128,21 @@ assign_prep_kernel(AssignArgs a)
     const int32_t* ccseg = a.cc + lr * NC * (int64_t)E;
     int32_t* rows = a.tabg + lr * NC * (int64_t)(E + kRowTail);
     int4* over = a.splits + lr * S;
-    for (int e = tid; e < E; e += kThreads) carry[e] = 0;
+    for (int e = tid; e < E; e += kPrepThreads) carry[e] = 0;
     if (tid == 0) s_over = 0;
     const int m = build_entries(a.X + lr * S, a.slot_expert + (int64_t)l * S, S, E, ent_s, ent_e, ent_lo, ent_hi, s_wcnt);
     for (int c0 = 0; c0 < NC; c0 += NCT) {
         const int nct = (NC - c0) < NCT ? (NC - c0) : NCT;
-        for (int i = tid; i < nct * E; i += kThreads) { cnts[i] = ccseg[(int64_t)c0 * E + i]; tab[i] = i % E; }
-        for (int c = tid; c < nct; c += kThreads) nsc[c] = 0;
+        for (int i = tid; i < nct * E; i += kPrepThreads) { cnts[i] = ccseg[(int64_t)c0 * E + i]; tab[i] = i % E; }
+        for (int c = tid; c < nct; c += kPrepThreads) nsc[c] = 0;
         __syncthreads();
-        for (int e = tid; e < E; e += kThreads) {
+        for (int e = tid; e < E; e += kPrepThreads) {
             int32_t b = carry[e];
             for (int c = 0; c < nct; ++c) { base[c * E + e] = b; b += cnts[c * E + e]; }
             carry[e] = b;
         }
         __syncthreads();
-        for (int i = tid; i < nct * m; i += kThreads) {
+        for (int i = tid; i < nct * m; i += kPrepThreads) {
             const int c = i / m, q = i - c * m;
             const int e = ent_e[q];
             const int32_t cnt = cnts[c * E + e];
@@ -166,17 +161,17 @@ assign_prep_kernel(AssignArgs a)
             }
         }
         __syncthreads();
-        for (int i = tid; i < nct * E; i += kThreads) {
+        for (int i = tid; i < nct * E; i += kPrepThreads) {
             const int c = i / E, e = i - c * E;
             rows[(int64_t)(c0 + c) * (E + kRowTail) + e] = tab[i];
         }
-        for (int c = tid; c < nct; c += kThreads) {
+        for (int c = tid; c < nct; c += kPrepThreads) {
             rows[(int64_t)(c0 + c) * (E + kRowTail) + E] = nsc[c];
         }
         __syncthreads();
     }
     // the overflow count is final only now: every row of the segment gets it
-    for (int c = tid; c < NC; c += kThreads) {
+    for (int c = tid; c < NC; c += kPrepThreads) {
         int32_t* tail = rows + (int64_t)c * (E + kRowTail) + E;
         tail[1] = s_over; tail[2] = 0; tail[3] = 0;
     }
@@ -490,7 +485,7 @@ int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, void* ws, const i
     const int nct = prep_tile(p.E) < h->nc ? prep_tile(p.E) : h->nc;
     const size_t smem_prep = sizeof(int32_t) * (4 * (size_t)S + (size_t)p.E + 3 * (size_t)nct * p.E + nct);
     TAOT_CUDA_OK(cudaFuncSetAttribute(assign_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_prep));
-    assign_prep_kernel<<<(unsigned)((int64_t)p.L * p.R), kThreads, smem_prep, st>>>(a);
+    assign_prep_kernel<<<(unsigned)((int64_t)p.L * p.R), kPrepThreads, smem_prep, st>>>(a);
     TAOT_CUDA_OK(cudaGetLastError());
     if (vec_ok) {
         const size_t smem = (size_t)TAOT_CHUNK * 4 + sizeof(int32_t) * (((size_t)p.E + kRowTail + 3) & ~(size_t)3) +
