@@ -112,9 +112,9 @@ def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
 
 STATIC_SCRATCH_BYTES = 4 << 20
 # kernels one taot_plan call enqueues: chunk histogram, merge, Sinkhorn (register tile + shared-memory
-# kernel for handed-back problems), matching+auction, reassignment (tables, rewrite)
-PLAN_LAUNCHES = 7
-PLAN_LAUNCHES_NO_HINT = 5       # with ABLATE_HINT the two Sinkhorn kernels are not launched
+# kernel for handed-back problems), matching+auction, reassignment
+PLAN_LAUNCHES = 6
+PLAN_LAUNCHES_NO_HINT = 4       # with ABLATE_HINT the two Sinkhorn kernels are not launched
 
 
 def histogram_static(topk: torch.Tensor, R: int, E: int, e2r_dev: torch.Tensor, n: torch.Tensor,

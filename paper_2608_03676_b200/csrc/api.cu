@@ -62,8 +62,6 @@ void layout(taot_handle_t h)
     auto take = [&](size_t bytes) { const size_t o = off; off = taot_align_up(off + bytes, 256); return o; };
     const size_t path = p.R <= 256 ? 1 : 0;       // beyond 256 ranks only Phase 1 runs: no schedule buffers
     h->off_cc = take(path * sizeof(int32_t) * LR * h->nc * p.E);
-    h->off_tabg = take(path * sizeof(int32_t) * LR * h->nc * (p.E + 20));   // E targets + row tail (assign.cu: kRowTail)
-    h->off_splits = take(path * 16 * LR * (size_t)p.R * p.K);
     h->off_excess = take(sizeof(int32_t) * LR);
     h->off_spare = take(sizeof(int32_t) * LR);
     h->off_s = take(sizeof(float) * LR);
@@ -110,8 +108,6 @@ taot_handle_s* make_view(const taot_handle_s* h, int g, int l0, int Lg)
     const size_t R = p.R, E = p.E, S = (size_t)p.R * p.K, nc = h->nc, l = (size_t)l0;
     const size_t dmax = E < S ? E : S;
     v->off_cc += 4 * l * R * nc * E;
-    v->off_tabg += 4 * l * R * nc * (E + 20);
-    v->off_splits += 16 * l * R * S;
     v->off_excess += 4 * l * R;
     v->off_spare += 4 * l * R;
     v->off_s += 4 * l * R;

@@ -9,13 +9,13 @@
 // the rewrite is a table lookup.  Where an interval ends strictly inside a chunk's ordinal range
 // (a "split": at most one per slot this rank feeds, about one chunk in five has one), the entries
 // before the split position go to that slot and the later ones follow the next interval.  Kernels:
-//   assign_prep_kernel   one CTA per (layer, source rank): per chunk, the table expert -> target of
-//                        the chunk's LAST entry of that expert, and the splits (expert, in-chunk
-//                        ordinal, slot before); up to four of them ride in the tail of the table row;
 //   assign_chunk_kernel  one CTA per chunk, every chunk in one sweep over the table.  The chunk is staged in shared
 //                        memory with bulk asynchronous copies (cp.async.bulk + mbarrier, no multicast, an L2
-//                        evict-first policy: the table is read once); three CTAs per SM keep copies, lookups and
-//                        16-byte streaming stores of different chunks in flight.  A chunk without a split is one
+//                        evict-first policy: the table is read once); while they are in flight the CTA builds the
+//                        chunk's table expert -> target (of the chunk's LAST entry of that expert) and its split
+//                        records (expert, in-chunk ordinal, slot before) from X, the slots' experts and the chunk
+//                        counts; three CTAs per SM keep copies, lookups and 16-byte streaming stores of different
+//                        chunks in flight.  A chunk without a split is one
 //                        table lookup per entry; a chunk with splits is read three times from shared memory --
 //                        per-warp counts of the split experts, ballots in the one warp that holds a split to find
 //                        its flat position, then the rewrite with "expert e before position P -> slot" as
@@ -34,15 +34,11 @@ constexpr int kThreads = TAOT_STREAM_THREADS;
 constexpr int kWarps = kThreads / 32;
 constexpr int kWarpSpan = TAOT_CHUNK / kWarps;           // entries one warp owns, contiguous: 2048
 constexpr int kIters = kWarpSpan / 128;                  // 16-byte accesses per lane: 16
-constexpr int kPrepThreads = 64;                         // the table build is a chain of short dependent steps per (layer, rank): many small CTAs
-constexpr int kRowSplits = 4;                            // split records that ride in the tail of a table row
-constexpr int kRowTail = 4 + 4 * kRowSplits;             // {ns, soff, 0, 0} + records {expert, rel / -, target before, position}
+constexpr int kFewSplits = 4;                            // splits of a chunk that are applied as predicated overrides from registers
 
 struct AssignArgs {
     const int32_t* topk;
     const int32_t* cc;          // [L,R,NC,E] chunk counts (histogram pass)
-    int32_t* tabg;              // [L,R,NC,E+kRowTail] target of the chunk's last entry of each expert, then the row tail
-    int4* splits;               // [L,R,S]    {expert, ordinal of the split relative to the chunk, target before, position}
     const int32_t* slot_expert;
     const int32_t* X;
     int32_t* out;
@@ -103,80 +99,6 @@ __device__ int build_entries(const int32_t* Xrow, const int32_t* se, int S, int 
     return m;
 }
 
-// chunks of a segment handled per pass of the prep kernel (bounds its shared memory)
-__host__ __device__ inline int prep_tile(int E) { const int t = 6144 / E; return t < 1 ? 1 : (t > 32 ? 32 : t); }
-
-__global__ void __launch_bounds__(kPrepThreads)
-assign_prep_kernel(AssignArgs a)
-{
-    extern __shared__ int32_t sh[];
-    const int E = a.E, S = a.R * a.K, NC = a.nc, NCT = prep_tile(E) < NC ? prep_tile(E) : NC;
-    int32_t* ent_s = sh;                // [S]
-    int32_t* ent_e = ent_s + S;
-    int32_t* ent_lo = ent_e + S;
-    int32_t* ent_hi = ent_lo + S;
-    int32_t* carry = ent_hi + S;        // [E] ordinal at the start of the current tile of chunks
-    int32_t* cnts = carry + E;          // [NCT][E] counts of the tile's chunks
-    int32_t* base = cnts + NCT * E;     // [NCT][E] ordinal at the start of each chunk
-    int32_t* tab = base + NCT * E;      // [NCT][E] targets
-    int32_t* nsc = tab + NCT * E;       // [NCT] splits per chunk
-    __shared__ int s_wcnt[32];
-    __shared__ int s_over;
-    const int tid = threadIdx.x;
-    const int64_t lr = blockIdx.x;
-    const int32_t l = (int32_t)(lr / a.R);
-    const int32_t* ccseg = a.cc + lr * NC * (int64_t)E;
-    int32_t* rows = a.tabg + lr * NC * (int64_t)(E + kRowTail);
-    int4* over = a.splits + lr * S;
-    for (int e = tid; e < E; e += kPrepThreads) carry[e] = 0;
-    if (tid == 0) s_over = 0;
-    const int m = build_entries(a.X + lr * S, a.slot_expert + (int64_t)l * S, S, E, ent_s, ent_e, ent_lo, ent_hi, s_wcnt);
-    for (int c0 = 0; c0 < NC; c0 += NCT) {
-        const int nct = (NC - c0) < NCT ? (NC - c0) : NCT;
-        for (int i = tid; i < nct * E; i += kPrepThreads) { cnts[i] = ccseg[(int64_t)c0 * E + i]; tab[i] = i % E; }
-        for (int c = tid; c < nct; c += kPrepThreads) nsc[c] = 0;
-        __syncthreads();
-        for (int e = tid; e < E; e += kPrepThreads) {
-            int32_t b = carry[e];
-            for (int c = 0; c < nct; ++c) { base[c * E + e] = b; b += cnts[c * E + e]; }
-            carry[e] = b;
-        }
-        __syncthreads();
-        for (int i = tid; i < nct * m; i += kPrepThreads) {
-            const int c = i / m, q = i - c * m;
-            const int e = ent_e[q];
-            const int32_t cnt = cnts[c * E + e];
-            if (cnt == 0) continue;
-            const int32_t b = base[c * E + e], lo = ent_lo[q], hi = ent_hi[q];
-            const int32_t last = b + cnt - 1;
-            if (lo <= last && last < hi) tab[c * E + e] = E + ent_s[q];    // the slot that takes the chunk's last entry of e
-            if (hi > b && hi < b + cnt) {                                  // this slot's quota ends inside the chunk
-                const int k = atomicAdd(&nsc[c], 1);
-                if (k < kRowSplits) {
-                    int32_t* tail = rows + (int64_t)(c0 + c) * (E + kRowTail) + E + 4 + 4 * k;
-                    tail[0] = e; tail[1] = hi - b; tail[2] = E + ent_s[q]; tail[3] = -1;
-                } else {
-                    over[atomicAdd(&s_over, 1)] = make_int4(e, hi - b, E + ent_s[q], c0 + c);   // the segment's overflow list
-                }
-            }
-        }
-        __syncthreads();
-        for (int i = tid; i < nct * E; i += kPrepThreads) {
-            const int c = i / E, e = i - c * E;
-            rows[(int64_t)(c0 + c) * (E + kRowTail) + e] = tab[i];
-        }
-        for (int c = tid; c < nct; c += kPrepThreads) {
-            rows[(int64_t)(c0 + c) * (E + kRowTail) + E] = nsc[c];
-        }
-        __syncthreads();
-    }
-    // the overflow count is final only now: every row of the segment gets it
-    for (int c = tid; c < NC; c += kPrepThreads) {
-        int32_t* tail = rows + (int64_t)c * (E + kRowTail) + E;
-        tail[1] = s_over; tail[2] = 0; tail[3] = 0;
-    }
-}
-
 // Flat position, inside the chunk held at `buf`, of the entry of expert eb whose in-chunk ordinal is rel
 // (entries of eb before it belong to the slot whose quota ends there).  Block-wide: warp w owns entries
 // [w*2048, (w+1)*2048); per-warp counts, then ballots in the one warp that holds the entry.
@@ -233,16 +155,15 @@ __device__ int32_t locate_split(const int32_t* buf, int32_t len, int eb, int rel
     return *s_pos;
 }
 
-// Rewrite one chunk: `buf` holds its entries (shared memory in the pipelined kernel, global memory in the
-// plain one), `tab` its table row with tail in shared memory, `recs` is scratch for S records.  Block-wide.
+// Rewrite one chunk: `buf` holds its entries (shared memory if staged, else global memory), `tab` its table and
+// `recs` its `ns` split records {expert, in-chunk ordinal of the split, target before, -} in shared memory.  Block-wide.
 template <bool VEC>
-__device__ void rewrite_chunk(const AssignArgs& a, int64_t id, const int32_t* buf, int32_t* tab, int32_t* dst,
-                              int32_t len, int4* recs, int* s_cntw, int* s_pos)
+__device__ void rewrite_chunk(const AssignArgs& a, const int32_t* buf, int32_t* tab, int32_t* dst,
+                              int32_t len, const int ns, int4* recs, int* s_cntw, int* s_pos)
 {
     const int E = a.E;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int32_t wbase = warp * kWarpSpan + lane * 4;
-    const int ns = tab[E];
     auto emit = [&](int32_t pos, const int4& v) {
         if (VEC) st_stream(reinterpret_cast<int4*>(dst + pos), v);
         else {
@@ -279,20 +200,21 @@ __device__ void rewrite_chunk(const AssignArgs& a, int64_t id, const int32_t* bu
         }
         return;
     }
-    if (ns <= kRowSplits) {
+    if (ns <= kFewSplits) {
         // ---- a few splits: locate each, then apply them latest position first as predicated overrides
-        int32_t re[kRowSplits], rp[kRowSplits], rt[kRowSplits];
+        int32_t re[kFewSplits], rp[kFewSplits], rt[kFewSplits];
 #pragma unroll
-        for (int k = 0; k < kRowSplits; ++k) {
+        for (int k = 0; k < kFewSplits; ++k) {
             re[k] = -1; rp[k] = -1; rt[k] = 0;            // -1 never equals a valid expert
             if (k < ns) {                                  // uniform over the block
-                re[k] = tab[E + 4 + 4 * k];
-                rt[k] = tab[E + 4 + 4 * k + 2];
-                rp[k] = locate_split<VEC>(buf, len, re[k], tab[E + 4 + 4 * k + 1], s_cntw, s_pos);
+                const int4 rec = recs[k];
+                re[k] = rec.x;
+                rt[k] = rec.z;
+                rp[k] = locate_split<VEC>(buf, len, rec.x, rec.y, s_cntw, s_pos);
             }
         }
 #pragma unroll
-        for (int x = 1; x < kRowSplits; ++x)               // sort by position, descending (unused records sink)
+        for (int x = 1; x < kFewSplits; ++x)               // sort by position, descending (unused records sink)
 #pragma unroll
             for (int y = x; y > 0; --y)
                 if (rp[y] > rp[y - 1]) {
@@ -313,7 +235,7 @@ __device__ void rewrite_chunk(const AssignArgs& a, int64_t id, const int32_t* bu
                     if ((uint32_t)e < (uint32_t)E) {
                         int32_t t = tab[e];
 #pragma unroll
-                        for (int k = 0; k < kRowSplits; ++k)
+                        for (int k = 0; k < kFewSplits; ++k)
                             if (e == re[k] && pos + j < rp[k]) t = rt[k];
                         xv[j] = t;
                     }
@@ -323,21 +245,8 @@ __device__ void rewrite_chunk(const AssignArgs& a, int64_t id, const int32_t* bu
         }
         return;
     }
-    // ---- many splits in one chunk (rare): all records into shared memory, located one by one, then a list walk
-    const int c = (int)(id % a.nc);
-    const int4* over = a.splits + (id / a.nc) * (int64_t)(a.R * a.K);
-    const int nover = tab[E + 1];
-    __shared__ int s_n;
-    if (tid == 0) s_n = 0;
-    __syncthreads();
-    for (int k = tid; k < kRowSplits; k += blockDim.x)
-        recs[atomicAdd(&s_n, 1)] = make_int4(tab[E + 4 + 4 * k], tab[E + 4 + 4 * k + 1], tab[E + 4 + 4 * k + 2], -1);
-    for (int q = tid; q < nover; q += blockDim.x) {
-        const int4 r = over[q];
-        if (r.w == c) recs[atomicAdd(&s_n, 1)] = make_int4(r.x, r.y, r.z, -1);
-    }
-    __syncthreads();
-    const int nrec = s_n;
+    // ---- many splits in one chunk (rare): located one by one, then a list walk
+    const int nrec = ns;
     for (int k = 0; k < nrec; ++k) {
         const int32_t P = locate_split<VEC>(buf, len, recs[k].x, recs[k].y, s_cntw, s_pos);
         if (tid == 0) recs[k].w = P;
@@ -416,22 +325,44 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
     return false;
 }
 
+// shared memory of one CTA after the staged chunk: table, this chunk's counts and starting ordinals per expert, the
+// entries of the source rank (slot, expert, ordinal interval), the split records
+__host__ __device__ inline size_t chunk_smem_words(int E, int S)
+{
+    const size_t Ep = ((size_t)E + 3) & ~(size_t)3, Sp = ((size_t)S + 3) & ~(size_t)3;
+    return 3 * Ep + 4 * Sp + 4 * Sp;
+}
+
 // One CTA per chunk.  STAGE: the chunk is first copied to shared memory with bulk asynchronous copies; otherwise it
-// is read from global memory (any alignment).
+// is read from global memory (any alignment).  While the copies are in flight the CTA builds what the rewrite needs:
+// the slots its source rank feeds with their ordinal intervals (X, slot experts), the ordinal each expert has reached
+// at the start of the chunk (sum of the counts of the segment's earlier chunks), the table expert -> target of the
+// chunk's last entry of that expert, and one split record per quota interval that ends inside the chunk.
 template <bool VEC, bool STAGE>
 __global__ void __launch_bounds__(kThreads)
 assign_chunk_kernel(AssignArgs a)
 {
     extern __shared__ __align__(128) unsigned char shc[];
-    const int E = a.E;
+    const int E = a.E, S = a.R * a.K;
+    const int Ep = (E + 3) & ~3, Sp = (S + 3) & ~3;
     int32_t* stage = reinterpret_cast<int32_t*>(shc);                      // [TAOT_CHUNK] if STAGE
-    int32_t* tab = reinterpret_cast<int32_t*>(shc + (STAGE ? (size_t)TAOT_CHUNK * 4 : 0));   // [E + kRowTail]
-    int4* recs = reinterpret_cast<int4*>(tab + ((E + kRowTail + 3) & ~3));
+    int32_t* tab = reinterpret_cast<int32_t*>(shc + (STAGE ? (size_t)TAOT_CHUNK * 4 : 0));   // [E] targets
+    int32_t* cnt = tab + Ep;                             // [E] entries of each expert in this chunk
+    int32_t* base = cnt + Ep;                            // [E] ordinal of each expert at the start of this chunk
+    int32_t* ent_s = base + Ep;                          // [S] slots this rank feeds, ascending ...
+    int32_t* ent_e = ent_s + Sp;                         //     ... their experts ...
+    int32_t* ent_lo = ent_e + Sp;                        //     ... and the ordinals [lo, hi) they take
+    int32_t* ent_hi = ent_lo + Sp;
+    int4* recs = reinterpret_cast<int4*>(ent_hi + Sp);   // [S] split records of this chunk
     __shared__ __align__(8) uint64_t bar;
     __shared__ int s_cntw[kWarps];
+    __shared__ int s_wcnt[32];
     __shared__ int s_pos;
+    __shared__ int s_ns;
     const int tid = threadIdx.x;
     const int64_t id = blockIdx.x;
+    const int64_t lr = id / a.nc;
+    const int c = (int)(id % a.nc);
     int64_t goff; int32_t len;
     chunk_geometry(a, id, goff, len);
     const int32_t* buf = a.topk + goff;
@@ -448,20 +379,39 @@ assign_chunk_kernel(AssignArgs a)
         }
         buf = stage;
     }
-    const int32_t* trow = a.tabg + id * (int64_t)(E + kRowTail);
-    for (int e = tid; e < E + kRowTail; e += kThreads) tab[e] = trow[e];
-    __syncthreads();                                     // table row in place; the barrier is initialised
+    // ---- the chunk's table and split records
+    if (tid == 0) s_ns = 0;
+    const int32_t* ccseg = a.cc + lr * a.nc * (int64_t)E;
+    for (int e = tid; e < E; e += kThreads) {
+        int32_t b = 0;
+        for (int cb = 0; cb < c; ++cb) b += ccseg[(int64_t)cb * E + e];
+        base[e] = b;
+        cnt[e] = ccseg[(int64_t)c * E + e];
+        tab[e] = e;
+    }
+    const int m = build_entries(a.X + lr * S, a.slot_expert + (lr / a.R) * S, S, E, ent_s, ent_e, ent_lo, ent_hi, s_wcnt);
+    for (int q = tid; q < m; q += kThreads) {
+        const int e = ent_e[q];
+        const int32_t n = cnt[e];
+        if (n == 0) continue;
+        const int32_t b = base[e], lo = ent_lo[q], hi = ent_hi[q];
+        const int32_t last = b + n - 1;
+        if (lo <= last && last < hi) tab[e] = E + ent_s[q];               // the slot that takes the chunk's last entry of e
+        if (hi > b && hi < b + n)                                         // this slot's quota ends inside the chunk
+            recs[atomicAdd(&s_ns, 1)] = make_int4(e, hi - b, E + ent_s[q], -1);
+    }
+    __syncthreads();                                     // table and records in place; the barrier is initialised
     if (STAGE) {
         const bool ok = mbar_wait(&bar, 0);
         if (__syncthreads_or(!ok)) {                     // the copy has not landed: report, and give the copies still in
             if (tid == 0) {                              // flight one more bounded wait before the CTA's memory goes away
-                atomicOr(a.info + (int32_t)((id / a.nc) / a.R), TAOT_INFO_INTERNAL);
+                atomicOr(a.info + (int32_t)(lr / a.R), TAOT_INFO_INTERNAL);
                 (void)mbar_wait(&bar, 0);
             }
             return;
         }
     }
-    rewrite_chunk<VEC>(a, id, buf, tab, a.out + goff, len, recs, s_cntw, &s_pos);
+    rewrite_chunk<VEC>(a, buf, tab, a.out + goff, len, s_ns, recs, s_cntw, &s_pos);
 }
 
 }  // namespace
@@ -474,29 +424,22 @@ int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, void* ws, const i
     AssignArgs a;
     a.topk = d_topk;
     a.cc = reinterpret_cast<const int32_t*>(w + h->off_cc);
-    a.tabg = reinterpret_cast<int32_t*>(w + h->off_tabg);
-    a.splits = reinterpret_cast<int4*>(w + h->off_splits);
     a.slot_expert = d_slot_expert; a.X = d_X; a.out = d_new_idx; a.info = d_info;
     a.layer_elems = p.T * p.k; a.seg = h->seg; a.nc = h->nc; a.R = p.R; a.E = p.E; a.K = p.K;
     const int vec_ok = ((reinterpret_cast<uintptr_t>(d_topk) & 15) == 0) &&
                        ((reinterpret_cast<uintptr_t>(d_new_idx) & 15) == 0) && (h->seg % 4 == 0);
     const int S = p.R * p.K;
     const unsigned blocks = (unsigned)((int64_t)p.L * p.R * h->nc);
-    const int nct = prep_tile(p.E) < h->nc ? prep_tile(p.E) : h->nc;
-    const size_t smem_prep = sizeof(int32_t) * (4 * (size_t)S + (size_t)p.E + 3 * (size_t)nct * p.E + nct);
-    TAOT_CUDA_OK(cudaFuncSetAttribute(assign_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_prep));
-    assign_prep_kernel<<<(unsigned)((int64_t)p.L * p.R), kPrepThreads, smem_prep, st>>>(a);
-    TAOT_CUDA_OK(cudaGetLastError());
+    const size_t words = chunk_smem_words(p.E, S);
     if (vec_ok) {
-        const size_t smem = (size_t)TAOT_CHUNK * 4 + sizeof(int32_t) * (((size_t)p.E + kRowTail + 3) & ~(size_t)3) +
-                            sizeof(int4) * (size_t)(S + kRowSplits);
+        const size_t smem = (size_t)TAOT_CHUNK * 4 + sizeof(int32_t) * words;
         TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         assign_chunk_kernel<true, true><<<blocks, kThreads, smem, st>>>(a);
     } else {
-        const size_t smem = sizeof(int32_t) * (((size_t)p.E + kRowTail + 3) & ~(size_t)3) + sizeof(int4) * (size_t)(S + kRowSplits);
+        const size_t smem = sizeof(int32_t) * words;
         TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         assign_chunk_kernel<false, false><<<blocks, kThreads, smem, st>>>(a);
     }
     TAOT_CUDA_OK(cudaGetLastError());
-    return 2;
+    return 1;
 }

@@ -46,7 +46,7 @@ struct taot_handle_s {
     int32_t kcap;            // Sinkhorn kernel-matrix capacity in floats per problem (shared memory)
     int64_t kcap_global;     // same, global-memory scratch per problem (R > 256 only), else 0
     // workspace layout (byte offsets)
-    size_t off_cc, off_tabg, off_splits, off_excess, off_spare, off_s, off_d, off_nrem, off_t12, off_kt, off_dc, off_cyc, off_tc;
+    size_t off_cc, off_excess, off_spare, off_s, off_d, off_nrem, off_t12, off_kt, off_dc, off_cyc, off_tc;
     size_t ws_bytes;
     // host-call staging layout (byte offsets into d_ws of taot_plan_host)
     size_t hoff_topk, hoff_new, hoff_n, hoff_el, hoff_rl, hoff_ex, hoff_sp, hoff_plan, hoff_it, hoff_err,
