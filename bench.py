@@ -222,11 +222,11 @@ def cpu_model():
 
 def tiered_sums(C, B):
     """Does the library take the tier-by-tier Sinkhorn kernel for this cost matrix?  Its rule, applied to the matrix
-    itself: 64, 128, 256, 512 or 1024 ranks and every off-diagonal cost equal to one of three values according to same node /
+    itself: 256, 512 or 1024 ranks and every off-diagonal cost equal to one of three values according to same node /
     same rail group / neither, with the block sizes read off the first row (ranks per node / per group 8 / 32, 4 / 16,
     4 / 32 or 16 / 32; a two-valued cost has no group tier)."""
     R = C.shape[0]
-    if R not in (64, 128, 256, 512, 1024):
+    if R not in (256, 512, 1024):
         return False
     row = C[0]
     node = 1

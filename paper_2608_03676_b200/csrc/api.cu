@@ -244,7 +244,7 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
     // a cost that depends only on "same node of 8 ranks / same rail group of 32 ranks / neither" lets the Sinkhorn
     // sums be taken tier by tier (sinkhorn_tiered.cu)
     h->tier_ok = 0;
-    if (R == 64 || R == 128 || R == 256 || R == 512 || R == 1024) {
+    if (R == 256 || R == 512 || R == 1024) {
         // The block sizes are read off the first row: a node is the run of ranks at rank 0's cheapest off-diagonal
         // cost, a rail group the run up to the next change (a cost with two values only has no group tier: any group
         // size then gives the same sums, 32 is taken).  The whole matrix is then checked against that structure.

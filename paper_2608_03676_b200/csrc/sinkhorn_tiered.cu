@@ -394,7 +394,7 @@ int taot_launch_sinkhorn_tiered(taot_handle_t h, const SinkArgs& a, int32_t B, c
     // of 256-rank problems that fill the GPU several times over: one warp per problem (fewest instructions per
     // problem).  Beyond 256 ranks the eight-warp kernel wins at every batch size (32 ranks per lane do not fit the registers).
     // (the one-warp kernel is built for nodes of 8 and rail groups of 32 ranks: a lane is a node)
-    if (B < 4 * h->sm_count || h->p.R != 256 || h->tier_node != 8 || h->tier_group != 32)
+    if (B < 4 * h->sm_count || h->p.R > 256 || h->tier_node != 8 || h->tier_group != 32)
         return taot_launch_sinkhorn_tiered_mw(a, h->tier_cost, h->tier_node, h->tier_group, B, st);
     TierCosts tc;
     tc.c1 = (double)h->tier_cost[0] * a.inv_eps;

@@ -1,18 +1,17 @@
-// Sinkhorn-Knopp (Appendix A.2) for a tiered cost matrix, several warps per problem: the tier-by-tier sums of
-// sinkhorn_tiered.cu (see there for the factorisation and its error argument) with the ranks spread over the lanes
-// of KW warps (2 at 64 ranks, 4 at 128, 8 from 256 on), for calls with few problems, where one warp per problem is
-// bound by the instructions it has to issue.
+// Sinkhorn-Knopp (Appendix A.2) for a tiered cost matrix, eight warps per problem: the tier-by-tier sums of
+// sinkhorn_tiered.cu (see there for the factorisation and its error argument) with the ranks spread over 256
+// lanes, for calls with few problems, where one warp per problem is bound by the instructions it has to issue.
 //
-// Lane gl = 32 * warp + lane owns RPL = R / (32 KW) consecutive ranks (1 up to 256 ranks, 2 at 512, 4 at 1024): a node
-// of 8 ranks is 8 / RPL adjacent lanes, a rail group 32 / RPL lanes, a warp holds RPL whole groups.  A half-step is
+// Lane gl = 32 * warp + lane owns RPL = R / 256 consecutive ranks (1 at 256 ranks, 2 at 512, 4 at 1024): a node of
+// 8 ranks is 8 / RPL adjacent lanes, a rail group 32 / RPL lanes, a warp holds RPL whole groups.  A half-step is
 // lane-local products, five xor-shuffle levels (node, group, groups of the warp), one shared-memory exchange of
-// the KW warp totals (one named barrier), one multiply-add and a reciprocal per rank.  The iteration is one
+// the eight warp totals (one named barrier), one multiply-add and a reciprocal per rank.  The iteration is one
 // dependent chain on a nearly empty SM, so everything that is not on the chain is kept out of the loop:
 //   * the loop body holds no rare case: a thread that sees its u~ or v~ drift out of range stores the number of the
 //     next exchange in a flag word, every thread reads that word (and the stop word) after the exchange's barrier,
 //     and any event -- drift, stop, last iteration -- leaves the loop for code that all threads run together;
-//   * with a tolerance, the row error of an iterate is not reduced by these warps at all: each lane stores
-//     its term, and one more warp, which otherwise only takes part in the barriers, sums the terms after
+//   * with a tolerance, the row error of an iterate is not reduced by the eight warps at all: each lane stores
+//     its term, and a ninth warp, which otherwise only takes part in the barriers, sums the 256 terms after
 //     half-step 2's barrier and posts the iteration number in the stop word if the error is within the tolerance.
 //     The others see the word after the next barrier, half a step into iteration t + 1, and put iterate t back.
 #include "sinkhorn_tiered_common.cuh"
@@ -21,6 +20,8 @@ using namespace taot_sk;
 
 namespace {
 
+constexpr int kWarps = 8;
+constexpr int kThreads = kWarps * 32;
 
 template <int LO, int HI>
 __device__ __forceinline__ float xor_sum(float v)           // all-reduce over lane bits LO <= offset < HI
@@ -60,12 +61,10 @@ __device__ __forceinline__ void bar_loop(const int nthreads)
 }
 
 // kNode ranks per node, kGroup ranks per rail group (powers of two, kNode < kGroup, a group inside one warp)
-template <int kNode, int kGroup, int KW, int RPL, bool TOL>
-__global__ void __launch_bounds__(KW * 32 + 32)
+template <int kNode, int kGroup, int RPL, bool TOL>
+__global__ void __launch_bounds__(kThreads + 32)
 sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
 {
-    constexpr int kWarps = KW, kThreads = KW * 32;
-    static_assert(KW == 2 || KW == 4 || KW == 8, "the warp totals are exchanged as one or two 16-byte words");
     static_assert(kGroup / RPL <= 32 && kGroup > kNode && kGroup % kNode == 0, "a rail group is held by the lanes of one warp");
     constexpr int LPN = kNode / RPL;              // lanes per node
     constexpr int LPG = kGroup / RPL;             // lanes per rail group
@@ -285,17 +284,9 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
     };
     // second part: the eight warp totals, summed pairwise (the same in every thread)
     auto total_of = [&](const int buf) {
-        if constexpr (KW == 8) {
-            const float4 lo = *reinterpret_cast<const float4*>(&xtot[buf][0]);
-            const float4 hi = *reinterpret_cast<const float4*>(&xtot[buf][4]);
-            return sum8(lo, hi);
-        } else if constexpr (KW == 4) {
-            const float4 v = *reinterpret_cast<const float4*>(&xtot[buf][0]);
-            return (v.x + v.y) + (v.z + v.w);
-        } else {
-            const float2 v = *reinterpret_cast<const float2*>(&xtot[buf][0]);
-            return v.x + v.y;
-        }
+        const float4 lo = *reinterpret_cast<const float4*>(&xtot[buf][0]);
+        const float4 hi = *reinterpret_cast<const float4*>(&xtot[buf][4]);
+        return sum8(lo, hi);
     };
     // exact row error of the iterate (u~, v~) = z whose row sums are r, and whether a row sum left the safe range:
     // block-wide, for the iterate that is the result
@@ -382,7 +373,7 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
             }
         } else {
             // the ninth warp: the same barriers, the same events; between half-step 2's barrier and the next one it
-            // sums the terms of the row error (KW per lane, then five shuffle levels: one fixed order)
+            // sums the 256 terms of the row error (eight per lane, then five shuffle levels: one fixed order)
             for (;;) {
                 bar_loop(NT);
                 if (xev[0] <= t) break;
@@ -394,18 +385,9 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
                 bar_loop(NT);
                 ++t;
                 if (check_now) {
-                    float e;
-                    if constexpr (KW == 8) {
-                        const float4 lo = *reinterpret_cast<const float4*>(&xe[lane * 8]);
-                        const float4 hi = *reinterpret_cast<const float4*>(&xe[lane * 8 + 4]);
-                        e = ((lo.x + lo.y) + (lo.z + lo.w)) + ((hi.x + hi.y) + (hi.z + hi.w));
-                    } else if constexpr (KW == 4) {
-                        const float4 v = *reinterpret_cast<const float4*>(&xe[lane * 4]);
-                        e = (v.x + v.y) + (v.z + v.w);
-                    } else {
-                        const float2 v = *reinterpret_cast<const float2*>(&xe[lane * 2]);
-                        e = v.x + v.y;
-                    }
+                    const float4 lo = *reinterpret_cast<const float4*>(&xe[lane * 8]);
+                    const float4 hi = *reinterpret_cast<const float4*>(&xe[lane * 8 + 4]);
+                    float e = ((lo.x + lo.y) + (lo.z + lo.w)) + ((hi.x + hi.y) + (hi.z + hi.w));
 #pragma unroll
                     for (int o = 1; o < 32; o <<= 1) e += __shfl_xor_sync(kFull, e, o);
                     if (lane == 0 && e <= tol_abs_f) { xev[1] = t; xev[0] = t; }
@@ -478,10 +460,9 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
 
 constexpr size_t kExclusiveSmem = 200 * 1024;
 
-template <int kNode, int kGroup, int KW, int RPL>
+template <int kNode, int kGroup, int RPL>
 int launch_mw(const SinkArgs& a, const TierCosts& tc, int32_t B, cudaStream_t st)
 {
-    constexpr int kThreads = KW * 32;
     size_t smem = (size_t)a.R * (2 * sizeof(double) + sizeof(float) + sizeof(int32_t));
     // A batch far smaller than the GPU is one dependent chain per problem: give each problem an SM to itself (a
     // shared-memory request no two CTAs of any kernel can share an SM with), so that neither the problems of other
@@ -491,11 +472,11 @@ int launch_mw(const SinkArgs& a, const TierCosts& tc, int32_t B, cudaStream_t st
     TAOT_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     if (2 * B <= sms && smem < kExclusiveSmem) smem = kExclusiveSmem;
     if (a.tol > 0.0f) {
-        TAOT_CUDA_OK(cudaFuncSetAttribute(sinkhorn_tiered_mw_kernel<kNode, kGroup, KW, RPL, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        sinkhorn_tiered_mw_kernel<kNode, kGroup, KW, RPL, true><<<B, kThreads + 32, smem, st>>>(a, tc, (int64_t)B);
+        TAOT_CUDA_OK(cudaFuncSetAttribute(sinkhorn_tiered_mw_kernel<kNode, kGroup, RPL, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        sinkhorn_tiered_mw_kernel<kNode, kGroup, RPL, true><<<B, kThreads + 32, smem, st>>>(a, tc, (int64_t)B);
     } else {
-        TAOT_CUDA_OK(cudaFuncSetAttribute(sinkhorn_tiered_mw_kernel<kNode, kGroup, KW, RPL, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        sinkhorn_tiered_mw_kernel<kNode, kGroup, KW, RPL, false><<<B, kThreads, smem, st>>>(a, tc, (int64_t)B);
+        TAOT_CUDA_OK(cudaFuncSetAttribute(sinkhorn_tiered_mw_kernel<kNode, kGroup, RPL, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        sinkhorn_tiered_mw_kernel<kNode, kGroup, RPL, false><<<B, kThreads, smem, st>>>(a, tc, (int64_t)B);
     }
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
@@ -505,18 +486,16 @@ template <int kNode, int kGroup>
 int launch_mw_ranks(const SinkArgs& a, const TierCosts& tc, int32_t B, cudaStream_t st)
 {
     switch (a.R) {
-        case 64: return launch_mw<kNode, kGroup, 2, 1>(a, tc, B, st);
-        case 128: return launch_mw<kNode, kGroup, 4, 1>(a, tc, B, st);
-        case 256: return launch_mw<kNode, kGroup, 8, 1>(a, tc, B, st);
-        case 512: if constexpr (kNode >= 2) return launch_mw<kNode, kGroup, 8, 2>(a, tc, B, st); else return 0;
-        case 1024: if constexpr (kNode >= 4) return launch_mw<kNode, kGroup, 8, 4>(a, tc, B, st); else return 0;
+        case 256: return launch_mw<kNode, kGroup, 1>(a, tc, B, st);
+        case 512: if constexpr (kNode >= 2) return launch_mw<kNode, kGroup, 2>(a, tc, B, st); else return 0;
+        case 1024: if constexpr (kNode >= 4) return launch_mw<kNode, kGroup, 4>(a, tc, B, st); else return 0;
         default: return 0;
     }
 }
 
 }  // namespace
 
-// Two to eight warps per problem (64, 128, 256, 512 or 1024 ranks); the caller has checked that the cost is tiered with `node` ranks
+// Eight warps per problem (256, 512 or 1024 ranks); the caller has checked that the cost is tiered with `node` ranks
 // per node and `group` ranks per rail group.  0 if that shape is not built.
 int taot_launch_sinkhorn_tiered_mw(const SinkArgs& a, const float* tier_cost3, int node, int group, int32_t B, cudaStream_t st)
 {
