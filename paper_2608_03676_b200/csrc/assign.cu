@@ -7,23 +7,23 @@
 // The chunk counts of the histogram pass say which ordinals of each expert fall into each chunk of
 // at most TAOT_CHUNK entries, so for most (chunk, expert) pairs every entry has the same target and
 // the rewrite is a table lookup.  Where an interval ends strictly inside a chunk's ordinal range
-// (a "split": at most one per slot this rank feeds, about one chunk in five has one), the entries
-// before the split position go to that slot and the later ones follow the next interval.  Kernels:
+// (a "split": at most one per slot this rank feeds; one chunk in five to two in five has one), the entries
+// before the split position go to that slot and the later ones follow the next interval.  One kernel:
 //   assign_chunk_kernel  one CTA per chunk, every chunk in one sweep over the table.  The chunk is staged in shared
 //                        memory with bulk asynchronous copies (cp.async.bulk + mbarrier, no multicast, an L2
 //                        evict-first policy: the table is read once); while they are in flight the CTA builds the
 //                        chunk's table expert -> target (of the chunk's LAST entry of that expert) and its split
 //                        records (expert, in-chunk ordinal, slot before) from X, the slots' experts and the chunk
 //                        counts; three CTAs per SM keep copies, lookups and 16-byte streaming stores of different
-//                        chunks in flight.  A chunk without a split is one
-//                        table lookup per entry; a chunk with splits is read three times from shared memory --
+//                        chunks in flight.  A chunk without a split is one table lookup per entry; a chunk with
+//                        splits is read three times from shared memory --
 //                        per-warp counts of the split experts, ballots in the one warp that holds a split to find
 //                        its flat position, then the rewrite with "expert e before position P -> slot" as
 //                        predicated overrides.  A routing table that is not 16-byte aligned or whose segments are
 //                        not multiples of 4 entries takes the same kernel without staging, with ordinary loads.
 // One sweep over all chunks matters: two kernels that each took part of the chunks (a persistent pipeline for the
-// chunks without a split, this kernel for the rest) moved their parts at 5.4-5.7 TB/s, the single sweep moves the
-// whole table at 6.5 TB/s -- the memory system serves a contiguous sweep better than two interleaved subsets.
+// chunks without a split, a per-chunk kernel for the rest) were measured at 5.4-5.7 TB/s on their parts, a single
+// sweep at 6.3-6.5 TB/s -- the memory system serves a contiguous sweep better than two interleaved subsets.
 // 8 bytes of HBM traffic per entry (one read, one write).  Out-of-range indices are copied through (the histogram
 // pass, whose counts this path consumes, is the one that flags them).
 #include "taot_internal.cuh"
@@ -46,7 +46,6 @@ struct AssignArgs {
     int64_t layer_elems, seg;
     int32_t nc, R, E, K;
 };
-
 
 __device__ __forceinline__ void st_stream(int4* p, const int4& v)
 {
