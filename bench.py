@@ -291,7 +291,7 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count, match_cyc=None):
                     traffic=HIST_TRAFFIC_RATIO * topk_bytes, peak_source=peaks["source"], bytes_per_launch=topk_bytes)
     if stage == "assign":
         a = 2 * topk_bytes / (ms * 1e-3) / 1e9
-        return dict(kernel="assign_chunk_kernel (+ assign_prep_kernel)", bound="hbm", achieved=a, peak=hbm, unit="GB/s",
+        return dict(kernel="assign_chunk_kernel", bound="hbm", achieved=a, peak=hbm, unit="GB/s",
                     frac=a / hbm, traffic=ASSIGN_TRAFFIC_RATIO * 2 * topk_bytes, peak_source=peaks["source"],
                     bytes_per_launch=2 * topk_bytes)
     if stage == "merge":
