@@ -253,7 +253,7 @@ int taot_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_slot_ex
  * The whole path (Algorithm 1: Phase 1, Phase 2, Phase 3, then the rewrite), asynchronous on `stream`; `out` holds
  * DEVICE pointers.  No allocation, no synchronisation: the call can be captured in a CUDA graph.
  * A routing table large enough to be bandwidth-bound (more than three waves of chunks per part) is planned in up to
- * four groups of consecutive layers: group 0 on `stream`, the others on streams the handle created, forked from
+ * six groups of consecutive layers: group 0 on `stream`, the others on streams the handle created, forked from
  * `stream` by an event and joined back into it by events before the call returns control to `stream`'s order; the
  * results are those of an unsplit call, bit for bit.  (The histogram and reassignment of one group then run under
  * the Sinkhorn and auction rounds of another.)  TAOT_PLAN_GROUPS (environment, read by taot_create) caps the number

@@ -30,14 +30,14 @@ int taot_get_stage_ms(taot_handle_t h, float* h_ms /* [5] */);
 /*
  * Timeline of the layer groups of the last taot_plan call made with profiling level 3 (a measurement aid; the
  * paper has no counterpart).  For a routing table large enough to be bandwidth-bound, taot_plan splits the L
- * problems into up to 4 groups of consecutive layers and plans each on a stream of its own, so that the
+ * problems into up to 6 groups of consecutive layers and plans each on a stream of its own, so that the
  * histogram and reassignment of one group run under the Sinkhorn and auction rounds of another; results are
  * those of an unsplit call.  *groups receives the number of groups (0: the handle does not split), h_ms
  * [groups][6] the time in ms, from the start of the call, at which each group reached: start, end of chunk
  * histogram, merge, Sinkhorn, matching + auction, reassignment.  Waits for the call to finish.
  * The environment variable TAOT_PLAN_GROUPS (read by taot_create) caps the number of groups; 1 disables the split.
  */
-int taot_get_group_trace(taot_handle_t h, int32_t* groups, float* h_ms /* [4][6] */);
+int taot_get_group_trace(taot_handle_t h, int32_t* groups, float* h_ms /* [6][6] */);
 
 
 /*

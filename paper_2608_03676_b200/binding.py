@@ -259,7 +259,7 @@ class Planner:
         a list with one [start, histogram, merge, Sinkhorn, matching, reassignment] row per group; [] if the handle
         plans all layers as one group."""
         n = ctypes.c_int32(0)
-        ms = (ctypes.c_float * 24)()
+        ms = (ctypes.c_float * 36)()
         _check(self.lib.taot_get_group_trace(self.handle, ctypes.byref(n), ms), "taot_get_group_trace")
         return [[float(ms[g * 6 + i]) for i in range(6)] for g in range(n.value)]
 

@@ -361,11 +361,15 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
         while (G > 1 && (params->L < 2 * G || (params->L / G) * chunks_per_layer <= 3 * (int64_t)h->sm_count)) --G;
         if (G > 1) {
             if (cudaEventCreate(&h->ev_fork) != cudaSuccess) rc = TAOT_ERR_CUDA;      // timed: origin of the group trace
-            // Group sizes grow geometrically: a group's chain of latency-bound stages takes about as long whatever its
-            // size, so a group can only finish (and rewrite its part of the table) under the others' chains if it
-            // started earlier by about the time its reassignment takes; the stagger of the starts is the histogram
-            // of the group itself, roughly half as long as its reassignment, hence sizes that grow by about a factor 1.6 (2 : 3 : 5 : 8 measured best on configs 3 and 4).
-            const double wt[TAOT_MAX_GROUPS] = {2.0, 3.0, 5.0, 8.0};
+            // Group sizes grow: a group's chain of latency-bound stages takes about as long whatever its size, so a
+            // group can only finish (and rewrite its part of the table) under the others' chains if it started
+            // earlier by about the time its reassignment takes; the stagger of the starts is the histogram of the
+            // group itself, roughly half as long as its reassignment.  Measured on configs 3 and 4: 2 : 3 : 5 : 8 best
+            // with four groups, 2 : 3 : 4 : 6 : 9 with five, 3 : 4 : 5 : 6 : 8 : 10 with six (and six about 2 % faster
+            // than four where the table is large enough for six).
+            static const double kWeights[3][TAOT_MAX_GROUPS] = {
+                {2.0, 3.0, 5.0, 8.0, 0.0, 0.0}, {2.0, 3.0, 4.0, 6.0, 9.0, 0.0}, {3.0, 4.0, 5.0, 6.0, 8.0, 10.0}};
+            const double* wt = kWeights[G <= 4 ? 0 : G - 4];
             double wsum = 0.0;
             for (int g = 0; g < G; ++g) wsum += wt[g];
             int l0 = 0;

@@ -14,7 +14,7 @@
 #define TAOT_CHUNK 16384
 #define TAOT_STREAM_THREADS 256            // threads of the streaming kernels: 64 elements each
 #define TAOT_MAX_TIERS 8                   // distinct bonus values the bit-set auction handles
-#define TAOT_MAX_GROUPS 4                  // layer groups taot_plan overlaps on internal streams
+#define TAOT_MAX_GROUPS 6                  // layer groups taot_plan overlaps on internal streams
 
 struct taot_handle_s {
     taot_params p;
