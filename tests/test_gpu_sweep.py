@@ -186,6 +186,31 @@ def test_tiered_kernel_in_tolerance_mode_beyond_256_ranks(R):
     pl.close()
 
 
+@pytest.mark.parametrize("R,check_every", [(256, 1), (256, 5), (512, 3)])
+def test_tiered_kernel_stops_at_the_first_checked_iterate_within_the_tolerance(R, check_every):
+    """The eight-warp kernel learns that an iterate met the tolerance half a step late (a ninth warp sums the row
+    error beside the iteration) and puts that iterate back: iteration count, plan and reported error must be those
+    of the first CHECKED iterate within the tolerance, also when only every few iterates are checked.  eps is large
+    enough for the problems to converge well before the cap."""
+    import paper_2608_03676_b200 as P
+    B = 6
+    C = W.cost_matrix(R, 8, SWEEP_TIERS, 4)
+    eps = 0.12 * max(SWEEP_TIERS)
+    pl = P.Planner(L=B, R=R, E=R, K=1, k=1, T=R, e2r=torch.arange(R, dtype=torch.int32), C=C, eps=eps,
+                   max_iters=2000, tol=1e-6, check_every=check_every)
+    loads = W.sweep_rank_loads(B, R, seed=91 + R, device="cuda")
+    ex, sp, s, d = pl.excess_spare(loads)
+    out = pl.sinkhorn(s, d)
+    torch.cuda.synchronize()
+    plan, iters, err, info = cpu(out["plan"]), cpu(out["iters"]), cpu(out["row_err"]), cpu(out["info"])
+    assert ((info & ~16) == 0).all(), info                       # nobody ran into the cap
+    assert (iters < 2000).all() and (iters % check_every == 0).all(), iters
+    for b in range(B):
+        check_sinkhorn_problem(cpu(s)[b], cpu(d)[b], C.numpy(), eps, plan[b], iters[b], err[b], 2000, 1e-6, check_every)
+    print(f"R={R} check_every={check_every}: iterations {iters.tolist()}")
+    pl.close()
+
+
 @pytest.mark.parametrize("R", [16, 64])
 @pytest.mark.parametrize("B,check", [(1, 1), (4096, 6)])
 @pytest.mark.parametrize("tol", [0.0, 1e-6])
