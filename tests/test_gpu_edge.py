@@ -99,9 +99,11 @@ def test_total_load_not_divisible_by_ranks_scales_the_supply():
     pl.close()
 
 
-@pytest.mark.parametrize("k,tpr,R,E", [(3, 1001, 4, 12), (5, 3333, 8, 16), (1, 40000, 2, 6), (8, 2049, 4, 8)])
+@pytest.mark.parametrize("k,tpr,R,E", [(3, 1001, 4, 12), (5, 3333, 8, 16), (1, 40000, 2, 6), (8, 2049, 4, 8), (2, 70001, 2, 6),
+                                       (4, 35000, 2, 6)])
 def test_unaligned_and_ragged_segments(k, tpr, R, E):
-    # SEG = tpr*k: not a multiple of 4 (scalar load path) and/or several chunks with a short last one
+    # SEG = tpr*k: not a multiple of 4 (scalar load path) and/or several chunks with a short last one (the last two
+    # cases: nine chunks per segment, so a chunk's starting ordinals are sums over up to eight earlier chunks)
     cfg = W.get_config("cfg1").replace(L=2, R=R, E=E, K=2, k=k, T=R * tpr, gpus_per_node=2, zipf=(1.3, 1.3))
     topk = W.routing_topk(cfg, device="cuda")
     pl = make_planner(cfg, max_iters=200, tol=1e-6)
