@@ -210,7 +210,10 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
 #pragma unroll
     for (int i = 0; i < RPL; ++i) z[i] = 1.0f;
 
-    auto rebuild = [&]() {                         // block-uniform: holds barriers; expects z = 1
+    // (keep: also store what the final plan is written from -- a supply rank's three tier coefficients, a demand
+    // rank's weight and that weight times its node factor and times node and group factor)
+    float pf1[RPL], pf2[RPL], pf3[RPL];
+    auto rebuild = [&](const bool keep) {          // block-uniform: holds barriers; expects z = 1
         double m1 = -INFINITY, p1 = -INFINITY;
 #pragma unroll
         for (int i = 0; i < RPL; ++i) {
@@ -249,16 +252,21 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
             wc[i] = wcol;
             wrx[i] = wrow * x[i]; wcx[i] = wcol * x[i];
             pr[i] = wrow; pc[i] = wcol;            // z = 1
+            if (keep) {
+                pf1[i] = ish ? a1 : wrow;
+                pf2[i] = ish ? a2 : fb * wrow;
+                pf3[i] = ish ? a3 : Fb * (fb * wrow);
+            }
         }
     };
-    auto fold = [&]() {                            // u~, v~ into the fp64 potentials, then every factor anew
+    auto fold = [&](const bool keep) {             // u~, v~ into the fp64 potentials, then every factor anew
 #pragma unroll
         for (int i = 0; i < RPL; ++i) {
             if ((hotm >> i) & 1u) alpha[q0 + i] += log((double)z[i]);
             if ((coldm >> i) & 1u) beta[q0 + i] += log((double)z[i]);
             z[i] = 1.0f;
         }
-        rebuild();
+        rebuild(keep);
     };
     // First part of a half-step, everything that does not need the other warps: the lane's node sum and group sum by
     // five xor-shuffle levels, the warp's share of the total (the same value in all of its lanes when a warp is one
@@ -303,7 +311,7 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
         err = e;
         bad = __syncthreads_or(b2);
     };
-    rebuild();
+    rebuild(false);
 
     // ---- the iterations; t = iteration in progress.  xev[0] = the iteration whose half-step 1 ends with an event: the
     // last one unless a thread that saw its u~ or v~ drift (xev[2]) or the ninth warp that found the previous iterate
@@ -421,7 +429,7 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
                 return;
             }
             if (tid == 0) { xev[0] = a.max_iters; xev[2] = -1; }
-            fold();
+            fold(false);
             continue;
         }
         // the last iteration: iterate t is the result whatever its error
@@ -436,20 +444,54 @@ sinkhorn_tiered_mw_kernel(SinkArgs a, TierCosts tc, int64_t nprob)
         break;
     }
 
-    // ---- T = diag(u) M diag(v) from the total potentials, then the column cap
-    fold();
+    // ---- T = diag(u) M diag(v) from the total potentials, then the column cap.  With the shifts of the tier sums an
+    // entry is a product of fp32 factors that are all in range: T_ij = a1_i w_j (same node), a2_i f_n(j) w_j (same rail
+    // group), a3_i F_g(j) f_n(j) w_j (neither), times the cap of column j; a factor that underflows belongs to an
+    // entry e^-87 below the largest of its row.  The factors go to shared memory (over the potentials, which are no
+    // longer needed) and a row costs one multiplication per entry.
+    fold(true);
+    float cap[RPL];
     {
         xtot[0][warp] = partial(false, wc, base);                               // column sums of K~ itself (u~ = 1)
-        __syncthreads();
+        __syncthreads();                                                        // (also: every potential has been read)
         const float T = total_of(0);
 #pragma unroll
         for (int i = 0; i < RPL; ++i) {
             const float c = fmaf(k3[i], T, base[i]);
-            if (mainw) fgs[q0 + i] = ((coldm >> i) & 1u) ? (float)fmin(1.0, (double)x[i] / ((double)c + (double)a.eps0)) : 0.0f;
+            cap[i] = ((coldm >> i) & 1u) ? (float)fmin(1.0, (double)x[i] / ((double)c + (double)a.eps0)) : 0.0f;
+        }
+    }
+    float* rowf = reinterpret_cast<float*>(smem_raw);     // [3][R] tier coefficients of a supply rank's row; [0] < 0: no row
+    float* colf = rowf + 3 * R;                            // [3][R] column factors by tier, zero off the demand ranks
+    if (mainw) {
+#pragma unroll
+        for (int i = 0; i < RPL; ++i) {
+            const bool ish = (hotm >> i) & 1u, isc = (coldm >> i) & 1u;
+            const int q = q0 + i;
+            rowf[q] = ish ? pf1[i] : -1.0f; rowf[R + q] = ish ? pf2[i] : 0.0f; rowf[2 * R + q] = ish ? pf3[i] : 0.0f;
+            colf[q] = isc ? pf1[i] * cap[i] : 0.0f; colf[R + q] = isc ? pf2[i] * cap[i] : 0.0f;
+            colf[2 * R + q] = isc ? pf3[i] * cap[i] : 0.0f;
         }
     }
     __syncthreads();
-    const int nonfinite = write_plan_rows<kNode, kGroup>(tc, alpha, beta, fgs, R, warp, NW, lane, out);
+    int nonfinite = 0;
+    for (int row = warp; row < R; row += NW) {
+        float* orow = out + (int64_t)row * R;
+        const float a1 = rowf[row];
+        if (a1 < 0.0f) {
+            for (int j = lane; j < R; j += 32) orow[j] = 0.0f;
+            continue;
+        }
+        const float a2 = rowf[R + row], a3 = rowf[2 * R + row];
+        const int node = row / kNode, group = row / kGroup;
+#pragma unroll 4
+        for (int j = lane; j < R; j += 32) {
+            const bool sn = j / kNode == node, sg = j / kGroup == group;
+            const float v = sn ? a1 * colf[j] : (sg ? a2 * colf[R + j] : a3 * colf[2 * R + j]);
+            if (!isfinite(v)) nonfinite = 1;
+            orow[j] = v;
+        }
+    }
     if (__syncthreads_or(nonfinite)) info |= TAOT_INFO_NONFINITE;
     if (tid == 0) {
         a.iters[b] = t;
