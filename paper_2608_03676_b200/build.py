@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libtaot.so")
 OBJ = os.path.join(PKG, "csrc", "build")
-SOURCES = ["api.cu", "histogram.cu", "sinkhorn.cu", "sinkhorn_cluster.cu", "sinkhorn_dense_tc.cu", "sinkhorn_tiered.cu", "sinkhorn_tiered_mw.cu", "sinkhorn_tile.cu", "sinkhorn_tile_r32.cu", "sinkhorn_tile_r32_batch.cu", "sinkhorn_tile_r64.cu", "sinkhorn_tile_r64_batch.cu", "sinkhorn_tile_r256_batch.cu", "match.cu", "assign.cu", "report.cu", "peaks.cu", "dispatch.cu"]
+SOURCES = ["api.cu", "histogram.cu", "sinkhorn.cu", "sinkhorn_cluster.cu", "sinkhorn_dense_tc.cu", "sinkhorn_tiered.cu", "sinkhorn_tile.cu", "sinkhorn_tile_r32.cu", "sinkhorn_tile_r32_batch.cu", "sinkhorn_tile_r64.cu", "sinkhorn_tile_r64_batch.cu", "sinkhorn_tile_r256_batch.cu", "match.cu", "assign.cu", "report.cu", "peaks.cu", "dispatch.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v",
               "-I", os.path.join(ROOT, "include"), "-I", CSRC] + os.environ.get("TAOT_EXTRA_NVCC_FLAGS", "").split()
@@ -34,7 +34,7 @@ def _stale(target: str, deps) -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(OBJ, exist_ok=True)
     headers = [os.path.join(CSRC, "taot_internal.cuh"), os.path.join(CSRC, "sinkhorn_common.cuh"),
-               os.path.join(CSRC, "sinkhorn_tile.cuh"), os.path.join(CSRC, "sinkhorn_tiered_common.cuh"),
+               os.path.join(CSRC, "sinkhorn_tile.cuh"),
                os.path.join(ROOT, "include", "taot.h"), os.path.join(ROOT, "include", "taot_measure.h")]
     nvcc = _nvcc()
 
