@@ -320,7 +320,7 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count, match_cyc=None):
                                cycles=peaks["latency_cycles"],
                                note="achieved = stage time / iterations of the slowest problem (set-up and "
                                     "write-out included); floor from taot_measure_latencies at the maximum SM clock")
-        d = dict(kernel="sinkhorn_tiered_kernel" if tiered else "sinkhorn_tile_kernel", bound="alu", achieved=a,
+        d = dict(kernel="sinkhorn_tiered_mw_kernel" if tiered else "sinkhorn_tile_kernel", bound="alu", achieved=a,
                     peak=fp32_peak, unit="TFLOP/s",
                     frac=a / fp32_peak, traffic=None,
                     peak_source=fp32_src, flops_per_launch=2 * fma,
