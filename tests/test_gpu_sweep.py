@@ -149,7 +149,7 @@ def test_tiered_kernel_hands_back_a_rank_with_both_supply_and_demand():
 
 def test_tiered_kernel_with_two_tiers_only():
     """A node / cross-node cost without a rail-group tier is still a pure tier cost (the group and far tiers carry the
-    same value): it takes the tier-by-tier sums, eight warps per problem, and the one-warp build for a large batch."""
+    same value): it takes the tier-by-tier sums, eight warps per problem, and the four-warp build for a large batch."""
     import paper_2608_03676_b200 as P
     R = 256
     C = W.cost_matrix(R, 8, (0.0, 1.0, 12.0), None)
@@ -183,6 +183,38 @@ def test_tiered_kernel_in_tolerance_mode_beyond_256_ranks(R):
         check_sinkhorn_problem(cpu(s)[b], cpu(d)[b], C.numpy(), 0.1 * max(SWEEP_TIERS), plan[b], iters[b], err[b],
                                400, 1e-6)
     print(f"R={R}: iterations {iters.tolist()}")
+    pl.close()
+
+
+@pytest.mark.parametrize("R,B", [(256, 40), (256, 300), (256, 2400), (512, 300), (1024, 80)])
+@pytest.mark.parametrize("tol", [0.0, 1e-6])
+def test_tiered_kernel_builds_by_batch_size(R, B, tol):
+    """The tier-by-tier kernel spreads a problem over eight, four or two warps depending on the batch (a problem
+    alone on an SM; a batch that fills the GPU; the largest batches at 256 ranks) and on the rank count (1 to 8 ranks
+    per lane): every build, with a fixed count and with the tolerance, sampled problems against the oracle."""
+    import paper_2608_03676_b200 as P
+    C = W.cost_matrix(R, 8, SWEEP_TIERS, 4)
+    eps = 0.12 * max(SWEEP_TIERS)
+    iters_cap = 60 if tol == 0.0 else 400
+    pl = P.Planner(L=B, R=R, E=R, K=1, k=1, T=R, e2r=torch.arange(R, dtype=torch.int32), C=C, eps=eps,
+                   max_iters=iters_cap, tol=tol)
+    loads = W.sweep_rank_loads(B, R, seed=7 + R + B, device="cuda")
+    ex, sp, s, d = pl.excess_spare(loads)
+    out = pl.sinkhorn(s, d)
+    torch.cuda.synchronize()
+    iters, info = cpu(out["iters"]), cpu(out["info"])
+    assert ((info & ~16) == 0).all(), info[info != 0]
+    if tol == 0.0:
+        assert (iters == iters_cap).all()
+    else:
+        assert (iters >= 1).all() and (iters < iters_cap).all(), (iters.min(), iters.max())
+    s_h, d_h, err = cpu(s), cpu(d), cpu(out["row_err"])
+    for b in sorted({0, B // 2, B - 1, int(iters.argmax()), int(iters.argmin())}):
+        check_sinkhorn_problem(s_h[b], d_h[b], C.numpy(), eps, cpu(out["plan"][b]), iters[b], err[b], iters_cap, tol)
+    # properties that hold for every problem, checked on the GPU
+    tot = s.double().sum(1)
+    col_viol = (out["plan"].double().sum(1) - d.double()).abs().sum(1)
+    assert bool((col_viol <= 1e-5 * tot).all()) and bool((out["plan"] >= 0).all())
     pl.close()
 
 
