@@ -186,8 +186,8 @@ def test_handle_validation_and_null_arguments_return_status_codes():
 
 def test_many_quota_boundaries_inside_one_chunk():
     """A hand-made schedule in which ten guest slots hold the same expert and every source rank feeds each of
-    them a few tokens: ten quota intervals end inside the single chunk of a segment, more than the four split
-    records a table row carries, so the rewrite walks the overflow list.  Checked through taot_assign alone."""
+    them a few tokens: ten quota intervals end inside the single chunk of a segment, more than the four splits the
+    rewrite applies from registers, so it walks the list of split records.  Checked through taot_assign alone."""
     cfg = W.get_config("cfg1").replace(L=2, R=8, E=8, K=4, k=2, T=8 * 4096)
     e2r, _ = topology(cfg)
     topk = W.routing_topk(cfg, device="cuda")
