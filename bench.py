@@ -298,7 +298,9 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count, match_cyc=None):
         b = cfg.L * cfg.R * cfg.E * 4 * (2 + max(1, (cfg.T // cfg.R * cfg.k + 16383) // 16384))
         a = b / (ms * 1e-3) / 1e9
         return dict(kernel="merge_kernel", bound="hbm", achieved=a, peak=hbm, unit="GB/s", frac=a / hbm,
-                    traffic=None, peak_source=peaks["source"], bytes_per_launch=b)
+                    traffic=None, peak_source=peaks["source"], bytes_per_launch=b,
+                    note="one CTA per layer over a few tens of MB of chunk counts: a short kernel in the chain of "
+                         "latency-bound stages, far from any bandwidth bound by construction")
     derived = sm_count * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
     fp32_peak = peaks.get("fma_tflops") or derived
     fp32_src = (f"measured: taot_measure_alu_peaks (FMA chain kernel; ex2 {peaks.get('ex2_tops', 0):.2f} T/s); "
