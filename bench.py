@@ -41,6 +41,9 @@ FP32_LANES_PER_SM = 128
 # algorithmic bytes).  The reassignment figure is read + write once dirty L2 lines drain.
 HIST_TRAFFIC_RATIO = 1.045
 ASSIGN_TRAFFIC_RATIO = 1.01
+# the matching kernel reads its layer's counts, plan and lists once and keeps every round in shared memory: DRAM bytes per
+# layer from one ncu capture at the config-4 shape (606 KB read, nothing written back by the end, for 2 layers)
+MATCH_DRAM_BYTES_PER_LAYER = 303_000
 STAGES = ["histogram", "merge", "sinkhorn", "match_auction", "assign"]
 
 
@@ -337,7 +340,7 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count, match_cyc=None):
     ops = int((rounds[:, 0] * cfg.R * cfg.E + rounds[:, 1] * cfg.R * cfg.S).sum())
     a = ops / (ms * 1e-3) / 1e12
     d = dict(kernel="match_kernel", bound="alu", achieved=a, peak=fp32_peak / 2, unit="Tscore/s",
-             frac=a / (fp32_peak / 2), traffic=None,
+             frac=a / (fp32_peak / 2), traffic=MATCH_DRAM_BYTES_PER_LAYER * cfg.L,
              peak_source="half the FP32 FMA peak: one fp32 score evaluation per lane per clock",
              note="dependent rounds of masked arg-max, one CTA per layer; the figure counts the dense scores of the "
                   "paper's formulation (rounds x R x E and rounds x R x S) and no bandwidth or FLOP bound applies: "
