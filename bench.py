@@ -360,7 +360,27 @@ def roofline_for(stage, ms, cfg, out, peaks, sm_count, match_cyc=None):
             phase2_split=dict(scan_and_arbitration=c[8], winners=c[9], served_rows=c[10], all_keys_per_slot_index=c[11]),
             ns_per_phase3_round_at_max_clock=c[12] / max(1, r3) / (peaks["sm_max_mhz"] * 1e-3),
             note="cycle counts of the counting build of the kernel (every thread reads the clock three times a round): "
-                 "an upper bound on the timed build, whose stage time is `stages_ms.match_auction`")
+                 "an upper bound on the timed build, whose stage time is `stages_ms.match_auction`; a barrier holds a "
+                 "warp up at its next shared-memory access, so the wait at the first barrier of a round (for the warps "
+                 "whose cursors move) is counted under update_to_second_barrier and the wait at the second under "
+                 "bid_to_first_barrier of the next round")
+        rl = peaks.get("round_latency_cycles")
+        if rl and r3 > 0:
+            # One auction round as a dependent chain: the probe (two independent shared-memory loads, AND, find-first-set,
+            # rank index), the arbitration (atomicMax, barrier, read-back: measured as a unit), the winner's update
+            # (load of its holding, subtract, store) and the closing barrier; six dependent integer operations at the
+            # latency of a multiply-add stand for the ALU steps in between.
+            fma = (peaks.get("latency_cycles") or {}).get("fma", 4.0)
+            floor_cyc = 2 * rl["shared_load"] + rl["arbitration"] + rl["barrier"] + 6 * fma
+            share3 = c[12] / c[5]
+            ach_ns = ms * 1e6 * share3 / r3
+            floor_ns = floor_cyc / (peaks["sm_max_mhz"] * 1e-3)
+            d["latency"] = dict(bound="dependent chain of one auction round", floor_ns_per_round=floor_ns,
+                                achieved_ns_per_round=ach_ns, frac=floor_ns / ach_ns, rounds=r3, cycles=rl,
+                                model="2 shared loads + (atomicMax, barrier, read-back) + barrier + 6 integer operations",
+                                note="achieved = stage time x the Phase-3 share of the slowest layer's cycles / its "
+                                     "rounds; floor from taot_measure_round_latencies (eight warps, one CTA per SM) at "
+                                     "the maximum SM clock")
     return d
 
 
@@ -490,6 +510,7 @@ def run_ours(args):
     import paper_2608_03676_b200 as P
     peaks.update(P.measure_alu_peaks())              # FP32-FMA and ex2 ceilings of this GPU, measured once, untimed
     peaks["latency_cycles"] = P.measure_latencies() # dependent-operation latencies, for the chain floor of the Sinkhorn stage
+    peaks["round_latency_cycles"] = P.measure_round_latencies()   # the operations an auction round is a chain of
     props = torch.cuda.get_device_properties(local)
     topk = W.routing_topk(cfg, device="cuda")
     pl = build_planner(cfg)

@@ -77,6 +77,18 @@ int taot_measure_alu_peaks(float* h_fma_tflops, float* h_ex2_tops, void* d_sink,
  */
 int taot_measure_latencies(float* h_cycles /* [3] */, void* d_sink, void* stream);
 
+/*
+ * Latencies of the operations a round of the Phase-3 auction (Algorithm 3) is a chain of, measured on the current
+ * device in SM clock cycles, the way the matching kernel uses them (one CTA of eight warps): h_cycles[0] a dependent
+ * shared-memory load, [1] a shared-memory atomicMax whose result is waited for, [2] a named barrier over the eight
+ * warps, [3] the arbitration triple as a unit (atomicMax into a word, barrier, read-back of the word).  A round is
+ * probe (load), arbitration (triple), update (atomic, load) and the closing barrier: their sum is the floor the
+ * measured time per round is compared with.  (The paper has no counterpart: a measurement aid, not a step of the
+ * method.)  Launches one CTA on `stream` and WAITS for it.  d_sink: device memory of at least 32 bytes (overwritten).
+ * h_cycles: host floats [4].  Errors: TAOT_ERR_NULL, TAOT_ERR_CUDA.
+ */
+int taot_measure_round_latencies(float* h_cycles /* [4] */, void* d_sink, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -27,6 +27,7 @@ from .binding import (  # noqa: F401
     ReportRow,
     measure_alu_peaks,
     measure_latencies,
+    measure_round_latencies,
     PipelinedHostPlanner,
     StreamingHostPlanner,
     split_layers,

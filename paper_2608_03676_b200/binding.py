@@ -26,7 +26,7 @@ ABLATE_TOPOLOGY = 2
 _SYMBOLS = [
     "taot_create", "taot_destroy", "taot_workspace_bytes", "taot_host_workspace_bytes",
     "taot_histogram", "taot_histogram_static", "taot_excess_spare", "taot_sinkhorn", "taot_match", "taot_assign",
-    "taot_plan", "taot_plan_host", "taot_host_block_layout", "taot_plan_host_block", "taot_report", "taot_dispatch", "taot_measure_alu_peaks", "taot_measure_latencies", "taot_set_profiling", "taot_get_stage_ms", "taot_get_match_cycles", "taot_get_group_trace", "taot_tier_structure", "taot_last_launch_count",
+    "taot_plan", "taot_plan_host", "taot_host_block_layout", "taot_plan_host_block", "taot_report", "taot_dispatch", "taot_measure_alu_peaks", "taot_measure_latencies", "taot_measure_round_latencies", "taot_set_profiling", "taot_get_stage_ms", "taot_get_match_cycles", "taot_get_group_trace", "taot_tier_structure", "taot_last_launch_count",
     "taot_status_string",
 ]
 
@@ -155,6 +155,17 @@ def measure_latencies() -> Dict[str, float]:
     cyc = (ctypes.c_float * 3)()
     _check(lib.taot_measure_latencies(cyc, _ptr(sink), _stream()), "taot_measure_latencies")
     return dict(shuffle_level=float(cyc[0]), fma=float(cyc[1]), rcp_mul=float(cyc[2]))
+
+
+def measure_round_latencies() -> Dict[str, float]:
+    """SM clock cycles of the operations an auction round is a chain of (`taot_measure_round_latencies`): a dependent
+    shared-memory load, a shared-memory atomicMax waited for, a named barrier over eight warps, and the arbitration
+    triple (atomicMax, barrier, read-back) as a unit."""
+    lib = load_library()
+    sink = torch.zeros(8, dtype=torch.float32, device="cuda")
+    cyc = (ctypes.c_float * 4)()
+    _check(lib.taot_measure_round_latencies(cyc, _ptr(sink), _stream()), "taot_measure_round_latencies")
+    return dict(shared_load=float(cyc[0]), shared_atomic=float(cyc[1]), barrier=float(cyc[2]), arbitration=float(cyc[3]))
 
 
 @dataclass

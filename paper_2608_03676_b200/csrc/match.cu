@@ -22,6 +22,11 @@
 // what orders the list, so win counts or tiers whose scores round to the same float compete on the
 // rank index alone, as in a dense scan.  A bonus matrix with more than kMaxTiers distinct values (or
 // a price step that is not positive) takes the dense scan instead.
+// A round of the bit-set auction is a chain of a few dozen dependent instructions between two plain barriers, so its
+// cost is the instructions on that chain: every lane, whatever its slot's state, runs the same straight code (a slot
+// that is done has an empty mask and sends its key to a word nobody reads), shared memory is addressed by 32-bit
+// shared addresses, the end of the auction is read from a counter of live slots instead of a reducing barrier, and
+// only the two rare events -- a cursor that has to move, a win -- branch off.
 #include "taot_internal.cuh"
 
 namespace {
@@ -57,7 +62,9 @@ struct MatchArgs {
     long long* cyc;              // [L][16] SM cycles per part of the kernel as thread 0 sees them, or null (profiling aid):
                                  // 0 set-up, 1 Phase 2, 2 Phase-3 set-up, 3 Phase-3 bids (to the first barrier of a round),
                                  // 4 Phase-3 updates (to the second barrier), 5 whole kernel, 6 / 7 the busiest thread's own
-                                 // probe and arbitration time in Phase 3, 8-11 Phase-2 split, 12 the Phase-3 loop as a whole
+                                 // probe and arbitration time in Phase 3, 8-11 Phase-2 split, 12 the Phase-3 loop as a whole.
+                                 // A barrier does not hold a warp up until its next shared-memory access, so the wait at
+                                 // the first barrier is counted under 4 and the wait at the second under 3 of the next round.
 };
 
 __device__ __forceinline__ uint32_t ordered_bits(float f)
@@ -92,6 +99,21 @@ __device__ __forceinline__ bool bar_part_or(int nthreads, bool pred)
         : "memory");
     return out != 0;
 }
+
+// Shared-memory accesses of the auction's rounds by 32-bit shared address: one instruction each, no 64-bit address
+// arithmetic and no address-space conversion on the chain of a round.
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory"); }
+__device__ __forceinline__ void red_max_u32(uint32_t addr, uint32_t v) { asm volatile("red.shared.max.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory"); }
+__device__ __forceinline__ void red_and_u32(uint32_t addr, uint32_t v) { asm volatile("red.shared.and.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory"); }
+__device__ __forceinline__ void red_add_u32(uint32_t addr, uint32_t v) { asm volatile("red.shared.add.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory"); }
+__device__ __forceinline__ void red_or_u32(uint32_t addr, uint32_t v) { asm volatile("red.shared.or.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory"); }
 
 constexpr int kMaxW = 8;          // words of a rank bit set: R <= 256
 constexpr size_t kSmemBudget = 224 * 1024;   // dynamic shared memory the kernel plans with (227 KB per CTA less the static part)
@@ -169,6 +191,7 @@ match_kernel(MatchArgs a)
     int32_t* nrem_s = reinterpret_cast<int32_t*>(tw_mask + (a.nbid ? a.ntiers * S : 0));      // [dmax*R] if it fits
     __shared__ long long s_tot;
     __shared__ int s_cnt, s_any, s_ns;
+    __shared__ uint32_t s_live3, s_lastwin;      // Phase 3: slots that can still bid; 1 + the last round somebody won
     __shared__ int s_wcnt[32];
 
     const int32_t* n = a.n + l * (int64_t)R * E;
@@ -537,12 +560,32 @@ match_kernel(MatchArgs a)
             keyb = ((uint32_t)(a.nbid - cur) << 16) | (uint32_t)(0xFFFF - s);
         };
         if (live) load_entry();
+        // The rounds end when no slot can bid any more.  A count of the slots that still can, kept in shared memory,
+        // tells: it is only ever changed between the two barriers of a round and only read between the second barrier
+        // of one round and the first of the next, so every thread sees the same value and no round needs a barrier that
+        // also reduces a predicate (about 150 cycles more than a plain one after a shared-memory atomic).
+        if (tid == 0) { s_live3 = 0u; s_lastwin = 0u; }
+        __syncthreads();
+        if (live) atomicAdd(&s_live3, 1u);
+        __syncthreads();
         uint32_t* const arb = reinterpret_cast<uint32_t*>(arb_r);     // [R] best bid per rank; the winner clears its entry
         long long limit = cap;
         if (a.auction_max_rounds > 0 && a.auction_max_rounds < limit) limit = a.auction_max_rounds;
         const int round_limit = (int)(limit < 0x7fffffffLL ? limit : 0x7fffffffLL);
         if (timed) c_p3loop = clock64();
         const int NP = ((S + 31) >> 5) << 5;      // threads that take part in the rounds: the warps holding slots
+        const uint32_t a_arb = smem_u32(arb), a_avc = smem_u32(av);
+        const uint32_t a_live = smem_u32(&s_live3), a_lastwin = smem_u32(&s_lastwin);
+        // a slot that does not bid sends its key to a word of its own behind the R arbiters (the block holds 4R words):
+        // the bid is one instruction for every lane, whatever the slot's state
+        const uint32_t a_idle = a_arb + 4u * (uint32_t)(R + tid % (3 * R));
+        const uint32_t dmax4 = (uint32_t)a.dmax * 4u;
+        uint32_t a_av = smem_u32(p_av), a_lv = smem_u32(p_lv);       // the two words a probe reads
+        const bool nrem_smem = a.nrem_in_smem != 0;
+        int32_t* const nrem_col = nrem + col * R;                    // this slot's expert: what each rank still holds
+        const uint32_t a_cell0 = nrem_smem ? smem_u32(nrem_col) : 0u;
+        int32_t* const Xs = Xl + s;                                   // column s of the plan
+        bool dying = false;                       // the cursor ran off the list: leave the count after the next barrier
         while (tid < NP && rounds3 < round_limit) {
             const long long c_r0 = TIMED ? clock64() : 0;
             // Step 1: bid for the source rank with the best bonus minus price.
@@ -550,11 +593,16 @@ match_kernel(MatchArgs a)
             // host AND holding the expert AND this win count) can only shrink -- a rank enters this win count from the
             // one below, and the entry of the same tier with that lower count comes earlier in the list, so it was found
             // empty for good before the cursor got here.  Words found empty therefore stay empty: the probe is one word
-            // (the tier's only word, or the word of the last hit), two loads and two ANDs, the same for every lane.
-            uint32_t hit = 0u;
-            uint32_t* p_sel = p_lv;              // win-count word of the rank bid for (the tied groups set their own)
-            int r_best = -1;
-            if (live) {
+            // (the tier's only word, or the word of the last hit), two loads and two ANDs, the same for every lane; a
+            // slot that is done keeps a zero mask.  Only a probe that comes back empty leaves this path.
+            const uint32_t nlive = lds_u32(a_live);
+            uint32_t hit = e_mk & lds_u32(a_av) & lds_u32(a_lv);
+            uint32_t a_sel = a_lv;               // win-count word of the rank bid for (the tied groups set their own)
+            int r_best = (pw << 5) + __ffs(hit) - 1;
+            bool bids = hit != 0u;
+            if (hit == 0u && live) {
+                uint32_t* p_sel = p_lv;
+                r_best = -1;
                 for (;;) {
                     hit = e_mk & *p_av & *p_lv;
                     if (hit) { r_best = (pw << 5) + __ffs(hit) - 1; p_sel = p_lv; break; }
@@ -594,40 +642,52 @@ match_kernel(MatchArgs a)
                     }
                     if (!live) break;
                 }
+                a_av = smem_u32(p_av);
+                a_lv = smem_u32(p_lv);
+                a_sel = smem_u32(p_sel);
+                bids = r_best >= 0;
+                dying = !live;
             }
             // Step 2: the rank keeps its best bidder (ties: lowest slot).  The position of a score in the list orders
             // scores exactly as their fp32 values do, so (list position, slot) packs into one 32-bit key and a single
-            // native shared-memory atomicMax arbitrates: smaller position = higher score, then the lower slot.
-            const bool bids = r_best >= 0;
+            // native shared-memory max arbitrates: smaller position = higher score, then the lower slot.
+            const uint32_t a_mine = bids ? a_arb + ((uint32_t)r_best << 2) : a_idle;
             const long long c_rp = TIMED ? clock64() : 0;
-            if (bids) atomicMax(arb + r_best, keyb);
+            red_max_u32(a_mine, keyb);
             if (TIMED) { const long long c_ra = clock64(); c_probe += c_rp - c_r0; c_atom += c_ra - c_rp; }
-            if (!bar_part_or(NP, bids)) break;
+            bar_part(NP);
             const long long c_r1 = TIMED ? clock64() : 0;
             // Steps 3-4: the winning slot of each rank collects x = min(n, A); holdings, plan and price follow.  The
             // rank bid for holds tokens of the expert (its availability bit was set) and the slot still wants some, so
             // x > 0 and the rank's win count goes from the entry's to the next: its bit moves one word up in lvl.
-            if (bids && arb[r_best] == keyb) {
+            const bool won = (lds_u32(a_mine) == keyb) & bids;
+            if (dying) { red_add_u32(a_live, 0xFFFFFFFFu); dying = false; }
+            if (won) {
                 const uint32_t bit = 1u << (r_best & 31);
-                atomicAnd(p_sel, ~bit);
-                atomicOr(p_sel + 1, bit);
-                arb[r_best] = 0u;                // losers of this round compare against their own key: 0 is nobody's
-                int32_t* cell = nrem + col * R + r_best;
-                const int32_t have = *cell;
+                red_and_u32(a_sel, ~bit);
+                red_or_u32(a_sel + 4u, bit);
+                sts_u32(a_mine, 0u);             // losers of this round compare against their own key: 0 is nobody's
+                sts_u32(a_lastwin, (uint32_t)rounds3 + 1u);
+                int32_t have;
+                if (nrem_smem) have = (int32_t)lds_u32(a_cell0 + ((uint32_t)r_best << 2));
+                else have = nrem_col[r_best];
                 const int32_t x = have < A ? have : A;
-                Xl[(int64_t)r_best * S + s] = x;           // a (rank, slot) pair is served at most once
-                *cell = have - x;
+                if (nrem_smem) sts_u32(a_cell0 + ((uint32_t)r_best << 2), (uint32_t)(have - x));
+                else nrem_col[r_best] = have - x;
                 A -= x;
-                if (have - x == 0) atomicAnd(avail + (r_best >> 5) * a.dmax + col, ~bit);
-                if (A <= 0) live = false;
+                if (have == x) red_and_u32(a_avc + (uint32_t)(r_best >> 5) * dmax4, ~bit);
+                if (A <= 0) { live = false; e_mk = 0u; red_add_u32(a_live, 0xFFFFFFFFu); }
+                Xs[(int64_t)r_best * S] = x;     // a (rank, slot) pair is served at most once
             }
-            ++rounds3;
+            // nobody was left before this round (the same answer in every thread): one more round, empty, ends the loop
+            rounds3 = nlive ? rounds3 + 1 : round_limit;
             bar_part(NP);
             if (TIMED && timed) { const long long c_r2 = clock64(); c_bid += c_r1 - c_r0; c_upd += c_r2 - c_r1; }
         }
         if (timed) c_p3end = clock64();
         if (s < S) slot_a[s] = A;
         __syncthreads();
+        rounds3 = (int)s_lastwin;                 // rounds in which somebody bid
     } else {
         for (;;) {
             if (a.auction_max_rounds > 0 && rounds3 >= a.auction_max_rounds) break;

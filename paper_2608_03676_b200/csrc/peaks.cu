@@ -96,6 +96,55 @@ latency_kernel(float* out, int n, float a, float b)
     }
 }
 
+
+// Latencies of the operations an auction round is a chain of, in SM clock cycles, measured the way the matching kernel
+// uses them: one CTA of eight warps on an SM of its own.  [0] a dependent shared-memory load (pointer chase);
+// [1] a shared-memory atomicMax whose result the next one depends on; [2] a named barrier over the eight warps, back to
+// back; [3] the arbitration triple as a unit: atomicMax into a word, barrier, read-back of the word.
+__global__ void __launch_bounds__(256)
+round_latency_kernel(float* out, int n)
+{
+    __shared__ int chase[256];
+    __shared__ unsigned arb[256];
+    const int tid = threadIdx.x;
+    chase[tid] = (tid * 37 + 11) & 255;                      // a permutation of 0..255 (37 is odd)
+    arb[tid] = 0u;
+    __syncthreads();
+    float res[4];
+    int p = tid;
+    unsigned v = (unsigned)tid + 1u;
+    for (int pass = 0; pass < 2; ++pass) {                   // the first pass warms the instruction cache
+        long long t0 = clock64();
+#pragma unroll 16
+        for (int i = 0; i < n; ++i) p = chase[p];
+        long long t1 = clock64();
+        res[0] = (float)(t1 - t0) / (float)n;
+        t0 = clock64();
+#pragma unroll 16
+        for (int i = 0; i < n; ++i) v = atomicMax(&arb[(tid + v) & 255], v + (unsigned)i) + 1u;
+        t1 = clock64();
+        res[1] = (float)(t1 - t0) / (float)n;
+        t0 = clock64();
+#pragma unroll 16
+        for (int i = 0; i < n; ++i) asm volatile("bar.sync 1, 256;" ::: "memory");
+        t1 = clock64();
+        res[2] = (float)(t1 - t0) / (float)n;
+        t0 = clock64();
+#pragma unroll 4
+        for (int i = 0; i < n; ++i) {
+            atomicMax(&arb[(p + i) & 255], v + (unsigned)i);
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            v += arb[(p + i) & 255] & 1u;
+        }
+        t1 = clock64();
+        res[3] = (float)(t1 - t0) / (float)n;
+    }
+    if (tid == 0) {
+        out[0] = res[0]; out[1] = res[1]; out[2] = res[2]; out[3] = res[3];
+        out[4] = (float)(p + (int)v) * 1e-30f;
+    }
+}
+
 }  // namespace
 
 extern "C" int taot_measure_latencies(float* h_cycles, void* d_sink, void* stream)
@@ -151,5 +200,18 @@ extern "C" int taot_measure_alu_peaks(float* h_fma_tflops, float* h_ex2_tops, vo
     cudaEventDestroy(e1);
     *h_fma_tflops = best_fma;
     *h_ex2_tops = best_ex2;
+    return TAOT_OK;
+}
+
+extern "C" int taot_measure_round_latencies(float* h_cycles, void* d_sink, void* stream)
+{
+    if (!h_cycles || !d_sink) return TAOT_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    round_latency_kernel<<<1, 256, 0, st>>>(static_cast<float*>(d_sink), 2048);
+    TAOT_CUDA_OK(cudaGetLastError());
+    float h[5];
+    TAOT_CUDA_OK(cudaMemcpyAsync(h, d_sink, sizeof(h), cudaMemcpyDeviceToHost, st));
+    TAOT_CUDA_OK(cudaStreamSynchronize(st));
+    for (int i = 0; i < 4; ++i) h_cycles[i] = h[i];
     return TAOT_OK;
 }

@@ -195,3 +195,19 @@ def test_measured_latencies_are_plausible():
     assert 8.0 < a["rcp_mul"] < 80.0, a
     for key in a:
         assert abs(a[key] - b[key]) <= 0.15 * a[key] + 1.0, (a, b)
+
+
+def test_measured_round_latencies_are_plausible():
+    """Latencies of the operations an auction round chains: a shared-memory load and a barrier over eight warps take a
+    few tens of cycles, an atomic with its result waited for somewhat more, and the arbitration triple (atomic,
+    barrier, read-back) at least as long as a barrier plus a load less the overlap; the same call twice agrees."""
+    import paper_2608_03676_b200 as P
+    a = P.measure_round_latencies()
+    b = P.measure_round_latencies()
+    assert 10.0 < a["shared_load"] < 80.0, a
+    assert 10.0 < a["shared_atomic"] < 300.0, a
+    assert 10.0 < a["barrier"] < 300.0, a
+    assert a["arbitration"] > max(a["barrier"], a["shared_load"]), a
+    assert a["arbitration"] < a["shared_atomic"] + a["barrier"] + 2 * a["shared_load"] + 50.0, a
+    for key in a:
+        assert abs(a[key] - b[key]) <= 0.15 * a[key] + 2.0, (a, b)
