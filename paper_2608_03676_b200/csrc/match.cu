@@ -82,22 +82,13 @@ __device__ __forceinline__ u64 warp_max_u64(u64 k)
     return k;
 }
 
-// Barriers over the first `nthreads` threads of the CTA only (a multiple of 32), on hardware barrier 1: the auction's
-// rounds involve the warps that hold slots, the others wait at the CTA-wide barrier that follows the auction.
+// Barrier over the first `nthreads` threads of the CTA only (a multiple of 32), on hardware barrier 1: the auction's
+// rounds involve the warps that hold slots, the others wait at the CTA-wide barrier that follows the auction.  The
+// aligned form: every lane of a warp that takes part reaches it together (the loop's conditions are the same for all
+// lanes of a warp and the branches inside a round close before it).
 __device__ __forceinline__ void bar_part(int nthreads)
 {
-    asm volatile("barrier.sync 1, %0;" ::"r"(nthreads) : "memory");
-}
-__device__ __forceinline__ bool bar_part_or(int nthreads, bool pred)
-{
-    int out;
-    asm volatile(
-        "{\n\t.reg .pred pin, pout;\n\tsetp.ne.s32 pin, %2, 0;\n\tbarrier.red.or.pred pout, 1, %1, pin;\n\t"
-        "selp.s32 %0, 1, 0, pout;\n\t}"
-        : "=r"(out)
-        : "r"(nthreads), "r"((int)pred)
-        : "memory");
-    return out != 0;
+    asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
 }
 
 // Shared-memory accesses of the auction's rounds by 32-bit shared address: one instruction each, no 64-bit address
