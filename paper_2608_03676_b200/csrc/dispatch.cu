@@ -10,7 +10,9 @@
 //   dispatch_scatter_kernel  one CTA per chunk: per-warp histograms of the warp's contiguous span, bases per
 //                            warp, then each warp walks its span in order, 32 entries at a time; the lanes with
 //                            the same target inside a step are found by OR-ing lane bits into a shared-memory
-//                            word per target and ranked by lane, so the order stays stable
+//                            word per target and ranked by lane, so the order stays stable; the lowest lane of
+//                            a group hands the group's running position to the others by a shuffle (one warp
+//                            barrier per step; the mask words of consecutive steps sit in alternating rows)
 // 12 bytes of HBM traffic per entry (two reads of the table, one write of the positions).
 #include "taot_internal.cuh"
 
@@ -104,14 +106,14 @@ __global__ void __launch_bounds__(kThreads)
 dispatch_scatter_kernel(DispatchArgs a)
 {
     extern __shared__ int32_t wh[];            // [kWarps][NB]: counts of the warp's span, then running positions;
-                                               // then [kWarps][NB] lane masks of the step being ranked
+                                               // then 2 x [kWarps][NB] lane masks of the steps being ranked
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, NB = a.NB;
     const int64_t id = blockIdx.x;
     int64_t goff; int32_t len;
     chunk_span(a, id, goff, len);
     const int32_t* src = a.idx + goff;
     int32_t* dst = a.perm + goff;
-    for (int q = tid; q < 2 * kWarps * NB; q += kThreads) wh[q] = 0;
+    for (int q = tid; q < 3 * kWarps * NB; q += kThreads) wh[q] = 0;
     __syncthreads();
     const int s0 = warp * kWarpSpan, s1 = min(len, s0 + kWarpSpan);
     int32_t* mine = wh + warp * NB;
@@ -132,6 +134,7 @@ dispatch_scatter_kernel(DispatchArgs a)
     __syncthreads();
     const unsigned lt = (1u << lane) - 1u;
     constexpr int U = 4;
+    unsigned* mask2 = mask + kWarps * NB;      // the second set of mask rows: steps alternate between the two
     for (int i0 = s0; i0 < s1; i0 += 32 * U) {
         int32_t v[U];
 #pragma unroll
@@ -144,17 +147,24 @@ dispatch_scatter_kernel(DispatchArgs a)
             const int i = i0 + u * 32 + lane;
             const bool ok = i < s1;
             const int b = ok ? bin_of(v[u], NB) : 0;
+            unsigned* mrow = (u & 1) ? mask2 : mask;
             // the lanes of this step that share my target: every lane ORs its bit into the target's word of the
             // warp's mask row (a set, so the result does not depend on the order of the atomics)
-            if (ok) atomicOr(&mask[b], 1u << lane);
+            if (ok) atomicOr(&mrow[b], 1u << lane);
             __syncwarp();
-            unsigned peers = 0;
-            int32_t pos = 0;
-            if (ok) { peers = mask[b]; pos = mine[b] + __popc(peers & lt); }
-            __syncwarp();
-            if (ok && (peers & lt) == 0) { mask[b] = 0; mine[b] += __popc(peers); }   // lowest lane of the group
-            __syncwarp();
-            if (ok) dst[i] = pos;
+            const unsigned peers = ok ? mrow[b] : (1u << lane);
+            // the lowest lane of a group reads the group's running position and hands it to the others by a shuffle,
+            // which every lane reaches with its copy of the word read; only then does that lane move the position on
+            // and clear the word.  The word is next written two steps later (the rows alternate) and the running
+            // position is next read after the next step's barrier.
+            const bool lead = ok && (peers & lt) == 0;
+            int32_t first = lead ? mine[b] : 0;
+            first = __shfl_sync(0xffffffffu, first, __ffs(peers) - 1);
+            if (lead) {
+                mine[b] = first + __popc(peers);
+                mrow[b] = 0u;
+            }
+            if (ok) dst[i] = first + __popc(peers & lt);
         }
     }
 }
@@ -175,7 +185,7 @@ int taot_launch_dispatch(taot_handle_t h, const int32_t* d_new_idx, int32_t* d_s
     a.nbits = 1;
     while ((1 << a.nbits) < a.NB) ++a.nbits;
     const size_t sm2 = sizeof(int32_t) * (2 * (size_t)a.NB + p.R + 1);
-    const size_t sm3 = sizeof(int32_t) * 2 * (size_t)kWarps * a.NB;
+    const size_t sm3 = sizeof(int32_t) * 3 * (size_t)kWarps * a.NB;
     TAOT_CUDA_OK(cudaFuncSetAttribute(dispatch_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3));
     const int rc = taot_launch_chunk_counts(h, d_new_idx, a.dc, d_info, a.NB - 1, st);
     if (rc < 0) return rc;
