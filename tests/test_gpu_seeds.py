@@ -12,6 +12,7 @@ pytestmark = pytest.mark.gpu
 SHAPES = {
     "cfg4_two_chunks_ragged": ("cfg4", dict(L=2, T=256 * 2304)),      # 256 ranks: tiered Sinkhorn, bit-set auction
     "cfg4_two_slots_per_rank": ("cfg4", dict(L=2, T=256 * 4096, K=2)),
+    "cfg4_four_slots_per_rank": ("cfg4", dict(L=1, T=256 * 2048, K=4)),  # 1024 slots: every thread of the CTA holds one
     "cfg3_ragged": ("cfg3", dict(L=3, T=64 * 2560)),
     "cfg3_four_chunks": ("cfg3", dict(L=2, T=64 * 8192)),
     "cfg2": ("cfg2", dict(L=4)),
