@@ -102,18 +102,21 @@ dispatch_offsets_kernel(DispatchArgs a)
     if (tid == 0 && sc[R] != 0) atomicOr(a.info + (int32_t)(lr / R), TAOT_INFO_BAD_INDEX);
 }
 
+// ALT: the mask words of consecutive ranking steps sit in alternating rows (one warp barrier per step); otherwise one
+// row and a second barrier per step, for target counts whose three rows would not fit in shared memory.
+template <bool ALT>
 __global__ void __launch_bounds__(kThreads)
 dispatch_scatter_kernel(DispatchArgs a)
 {
     extern __shared__ int32_t wh[];            // [kWarps][NB]: counts of the warp's span, then running positions;
-                                               // then 2 x [kWarps][NB] lane masks of the steps being ranked
+                                               // then (ALT: 2 x) [kWarps][NB] lane masks of the steps being ranked
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, NB = a.NB;
     const int64_t id = blockIdx.x;
     int64_t goff; int32_t len;
     chunk_span(a, id, goff, len);
     const int32_t* src = a.idx + goff;
     int32_t* dst = a.perm + goff;
-    for (int q = tid; q < 3 * kWarps * NB; q += kThreads) wh[q] = 0;
+    for (int q = tid; q < (ALT ? 3 : 2) * kWarps * NB; q += kThreads) wh[q] = 0;
     __syncthreads();
     const int s0 = warp * kWarpSpan, s1 = min(len, s0 + kWarpSpan);
     int32_t* mine = wh + warp * NB;
@@ -134,7 +137,7 @@ dispatch_scatter_kernel(DispatchArgs a)
     __syncthreads();
     const unsigned lt = (1u << lane) - 1u;
     constexpr int U = 4;
-    unsigned* mask2 = mask + kWarps * NB;      // the second set of mask rows: steps alternate between the two
+    unsigned* mask2 = ALT ? mask + kWarps * NB : mask;      // the second set of mask rows: steps alternate between the two
     for (int i0 = s0; i0 < s1; i0 += 32 * U) {
         int32_t v[U];
 #pragma unroll
@@ -165,6 +168,7 @@ dispatch_scatter_kernel(DispatchArgs a)
                 mrow[b] = 0u;
             }
             if (ok) dst[i] = first + __popc(peers & lt);
+            if (!ALT) __syncwarp();              // the cleared word is written again in the very next step
         }
     }
 }
@@ -185,13 +189,16 @@ int taot_launch_dispatch(taot_handle_t h, const int32_t* d_new_idx, int32_t* d_s
     a.nbits = 1;
     while ((1 << a.nbits) < a.NB) ++a.nbits;
     const size_t sm2 = sizeof(int32_t) * (2 * (size_t)a.NB + p.R + 1);
-    const size_t sm3 = sizeof(int32_t) * 3 * (size_t)kWarps * a.NB;
-    TAOT_CUDA_OK(cudaFuncSetAttribute(dispatch_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3));
+    const bool alt = sizeof(int32_t) * 3 * (size_t)kWarps * a.NB <= 64 * 1024;
+    const size_t sm3 = sizeof(int32_t) * (alt ? 3 : 2) * (size_t)kWarps * a.NB;
+    if (alt) TAOT_CUDA_OK(cudaFuncSetAttribute(dispatch_scatter_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3));
+    else TAOT_CUDA_OK(cudaFuncSetAttribute(dispatch_scatter_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3));
     const int rc = taot_launch_chunk_counts(h, d_new_idx, a.dc, d_info, a.NB - 1, st);
     if (rc < 0) return rc;
     dispatch_offsets_kernel<<<(unsigned)((int64_t)p.L * p.R), kThreads, sm2, st>>>(a);
     TAOT_CUDA_OK(cudaGetLastError());
-    dispatch_scatter_kernel<<<chunks, kThreads, sm3, st>>>(a);
+    if (alt) dispatch_scatter_kernel<true><<<chunks, kThreads, sm3, st>>>(a);
+    else dispatch_scatter_kernel<false><<<chunks, kThreads, sm3, st>>>(a);
     TAOT_CUDA_OK(cudaGetLastError());
     return 3;
 }
