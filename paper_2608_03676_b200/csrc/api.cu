@@ -116,6 +116,8 @@ taot_handle_s* make_view(const taot_handle_s* h, int g, int l0, int Lg)
     v->off_t12 += 4 * l * E * 2 * R;
     v->off_dc += 4 * l * R * nc * (E + S + 1);
     v->off_cyc += 8 * l * 16;
+    if (v->d_merge_part) v->d_merge_part += l * TAOT_MERGE_PARTS * E;
+    if (v->d_merge_cnt) v->d_merge_cnt += l;
     return v;
 }
 
@@ -347,6 +349,15 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
     }
     if (rc == TAOT_OK && h->ntiers > 0) rc = upload(&h->d_tiermask, tiermask.data(), tiermask.size());
     if (rc == TAOT_OK && h->nbid > 0) rc = upload(&h->d_bidlist, bidlist.data(), bidlist.size());
+    // the merge of a layer's chunk counts is shared by several CTAs where a layer has enough of them (the kernel sits in
+    // the chain of latency-bound stages): their partial expert loads and a counter of finished parts per layer
+    if (rc == TAOT_OK && R % (32 * TAOT_MERGE_PARTS) == 0) {
+        const size_t parts = (size_t)params->L * TAOT_MERGE_PARTS * E;
+        if (cudaMalloc(reinterpret_cast<void**>(&h->d_merge_part), sizeof(int32_t) * parts) != cudaSuccess ||
+            cudaMalloc(reinterpret_cast<void**>(&h->d_merge_cnt), sizeof(int32_t) * params->L) != cudaSuccess ||
+            cudaMemset(h->d_merge_cnt, 0, sizeof(int32_t) * params->L) != cudaSuccess)
+            rc = TAOT_ERR_CUDA;
+    }
     for (int i = 0; i < 6 && rc == TAOT_OK; ++i)
         if (cudaEventCreate(&h->ev[i]) != cudaSuccess) rc = TAOT_ERR_CUDA;
     // Layer groups for taot_plan: only where every group's routing table still keeps the memory system busy (more
@@ -424,6 +435,7 @@ int taot_destroy(taot_handle_t h)
     cudaFree(h->d_e2r); cudaFree(h->d_C); cudaFree(h->d_B); cudaFree(h->d_rowlse0); cudaFree(h->d_gibbs);
     cudaFree(h->d_rank_off); cudaFree(h->d_rank_list); cudaFree(h->d_tierval); cudaFree(h->d_tiermask);
     cudaFree(h->d_tpos); cudaFree(h->d_torder); cudaFree(h->d_tdest); cudaFree(h->d_bidlist);
+    cudaFree(h->d_merge_part); cudaFree(h->d_merge_cnt);
     for (int i = 0; i < 6; ++i)
         if (h->ev[i]) cudaEventDestroy(h->ev[i]);
     delete h;

@@ -113,26 +113,31 @@ __device__ void excess_spare_row(const int32_t* s_rl, int32_t R, long long* s_to
     }
 }
 
-// one CTA per layer: n = sum over chunks, expert_load = sum over ranks, rank_load by home rank
+// n = sum over chunks, expert_load = sum over ranks, rank_load by home rank.  `parts` CTAs share a layer, each taking a
+// block of source ranks; a part leaves its expert loads in part_el and counts itself done, and the part that finds
+// itself last adds them up and finishes the layer (no CTA waits for another).  parts == 1: one CTA per layer, no
+// exchange.  The kernel sits in the chain of latency-bound stages, so what counts is how long one layer takes.
 __global__ void __launch_bounds__(1024)
 merge_kernel(const int32_t* __restrict__ cc, const int32_t* __restrict__ e2r, int32_t* __restrict__ n,
              int32_t* __restrict__ expert_load, int32_t* __restrict__ rank_load, int32_t* excess,
-             int32_t* spare, float* fs, float* fd, int32_t R, int32_t E, int32_t nc, int32_t* info)
+             int32_t* spare, float* fs, float* fd, int32_t R, int32_t E, int32_t nc, int32_t* info,
+             int32_t parts, int32_t* part_el, int32_t* part_cnt)
 {
     extern __shared__ int32_t sh[];                      // el[E], rl[R]
     __shared__ long long s_tot;
+    __shared__ int s_last;
     int32_t* s_el = sh;
     int32_t* s_rl = sh + E;
-    const int l = blockIdx.x, tid = threadIdx.x;
+    const int l = blockIdx.x / parts, part = blockIdx.x - l * parts, tid = threadIdx.x;
     for (int i = tid; i < E + R; i += blockDim.x) sh[i] = 0;
     __syncthreads();
     const int32_t RE = R * E;                            // at most 256 x 1024
     const int32_t* ccl = cc + (int64_t)l * RE * nc;
     int32_t* nl = n + (int64_t)l * RE;
-    // (32-bit index arithmetic and several independent loads in flight per thread: the kernel sits in the chain of
-    // latency-bound stages, one CTA per layer)
+    // (32-bit index arithmetic and several independent loads in flight per thread)
+    const int32_t i0 = (int32_t)((int64_t)RE * part / parts), i1 = (int32_t)((int64_t)RE * (part + 1) / parts);
 #pragma unroll 4
-    for (int32_t idx = tid; idx < RE; idx += blockDim.x) {
+    for (int32_t idx = i0 + tid; idx < i1; idx += blockDim.x) {
         const int32_t r = idx / E, e = idx - r * E;
         const int32_t* p = ccl + r * nc * E + e;
         int32_t v = 0;
@@ -141,6 +146,24 @@ merge_kernel(const int32_t* __restrict__ cc, const int32_t* __restrict__ e2r, in
         if (v) atomicAdd(s_el + e, v);
     }
     __syncthreads();
+    if (parts > 1) {
+        int32_t* mine = part_el + ((int64_t)l * parts + part) * E;
+        for (int e = tid; e < E; e += blockDim.x) mine[e] = s_el[e];
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) s_last = atomicAdd(part_cnt + l, 1) == parts - 1;
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
+        const int32_t* all = part_el + (int64_t)l * parts * E;
+        for (int e = tid; e < E; e += blockDim.x) {
+            int32_t v = 0;
+            for (int q = 0; q < parts; ++q) v += __ldcg(all + (int64_t)q * E + e);   // written by other CTAs: not through L1
+            s_el[e] = v;
+        }
+        if (tid == 0) part_cnt[l] = 0;                   // as the next call expects it
+        __syncthreads();
+    }
     for (int e = tid; e < E; e += blockDim.x) {
         const int32_t v = s_el[e];
         expert_load[(int64_t)l * E + e] = v;
@@ -212,8 +235,10 @@ int taot_launch_merge(taot_handle_t h, const int32_t* d_cc, int32_t* d_n, int32_
 {
     const taot_params& p = h->p;
     const size_t smem = sizeof(int32_t) * (p.E + p.R);
-    merge_kernel<<<p.L, 1024, smem, st>>>(d_cc, h->d_e2r, d_n, d_expert_load, d_rank_load, d_excess, d_spare,
-                                          d_s, d_d, p.R, p.E, h->nc, d_info);
+    const int parts = (h->d_merge_part && h->d_merge_cnt) ? TAOT_MERGE_PARTS : 1;
+    merge_kernel<<<p.L * parts, 1024, smem, st>>>(d_cc, h->d_e2r, d_n, d_expert_load, d_rank_load, d_excess, d_spare,
+                                                  d_s, d_d, p.R, p.E, h->nc, d_info, parts, h->d_merge_part,
+                                                  h->d_merge_cnt);
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
 }

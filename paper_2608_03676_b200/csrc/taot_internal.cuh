@@ -14,6 +14,7 @@
 #define TAOT_CHUNK 16384
 #define TAOT_STREAM_THREADS 256            // threads of the streaming kernels: 64 elements each
 #define TAOT_MAX_TIERS 8                   // distinct bonus values the bit-set auction handles
+#define TAOT_MERGE_PARTS 8                 // CTAs that share the merge of one layer's chunk counts (256-rank tables)
 #define TAOT_MAX_GROUPS 6                  // layer groups taot_plan overlaps on internal streams
 
 struct taot_handle_s {
@@ -37,6 +38,8 @@ struct taot_handle_s {
     int32_t ntiers;          // 0: too many distinct values, the auction scans densely
     uint32_t* d_bidlist;     // [nbid] every (tier, win count) pair, best score first: w << 8 | t, bit 31 = next has the same score
     int32_t nbid;            // 0: no list (no tiers, or price step <= 0): the auction scans densely
+    int32_t* d_merge_part;   // [L][TAOT_MERGE_PARTS][E] expert loads of the parts of a layer's merge, or null (one CTA per layer)
+    int32_t* d_merge_cnt;    // [L] parts of a layer's merge that are done; zero between calls
     int32_t tier_ok;         // 1: C has a node / rail-group structure one of the tier-by-tier kernels is built for and R is 256, 512 or 1024
     int32_t tier_node, tier_group;   // ranks per node and per rail group of that structure (8 / 32, 4 / 16, 4 / 32 or 16 / 32)
     float tier_cost[3];      // its three costs off the diagonal: same node, same rail group, otherwise
