@@ -72,6 +72,9 @@ void layout(taot_handle_t h)
     h->off_dc = take(path * sizeof(int32_t) * LR * h->nc * ((size_t)p.E + (size_t)p.R * p.K + 1));
     h->off_cyc = take(path * sizeof(long long) * (size_t)p.L * 16);
     h->off_tc = take((p.R > 256 && p.R % 128 == 0) ? sizeof(float) * taot_sinkhorn_tc_ws_floats(p.R, p.L) : 0);
+    h->tb_ok = (path && p.E <= 256 && h->seg % 16 == 0) ? 1 : 0;
+    h->off_tb = take(h->tb_ok ? (size_t)p.L * (size_t)p.T * p.k : 0);
+    h->off_tbflag = take(h->tb_ok ? sizeof(int32_t) * LR * h->nc : 0);
     h->ws_bytes = off;
 
     const size_t S = (size_t)p.R * p.K;
@@ -116,6 +119,8 @@ taot_handle_s* make_view(const taot_handle_s* h, int g, int l0, int Lg)
     v->off_t12 += 4 * l * E * 2 * R;
     v->off_dc += 4 * l * R * nc * (E + S + 1);
     v->off_cyc += 8 * l * 16;
+    v->off_tb += l * (size_t)p.T * p.k;
+    v->off_tbflag += 4 * l * R * nc;
     if (v->d_merge_part) v->d_merge_part += l * TAOT_MERGE_PARTS * E;
     if (v->d_merge_cnt) v->d_merge_cnt += l;
     return v;
@@ -514,7 +519,7 @@ int taot_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_n, int32_t
     if ((reinterpret_cast<uintptr_t>(d_topk) & 3) || (reinterpret_cast<uintptr_t>(ws) & 255)) return TAOT_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int32_t* cc = reinterpret_cast<int32_t*>(at(ws, h->off_cc));
-    int a = taot_launch_histogram(h, d_topk, cc, d_info, st);
+    int a = taot_launch_histogram(h, d_topk, cc, d_info, st, ws);
     if (a < 0) return a;
     int b = taot_launch_merge(h, cc, d_n, d_expert_load, d_rank_load, nullptr, nullptr, nullptr, nullptr, st);
     if (b < 0) return b;
@@ -613,7 +618,7 @@ int taot_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_slot_ex
     int32_t* cc = reinterpret_cast<int32_t*>(at(ws, h->off_cc));
     int launches = 0;
     if (!reuse_counts) {
-        int a = taot_launch_histogram(h, d_topk, cc, d_info, st);
+        int a = taot_launch_histogram(h, d_topk, cc, d_info, st, ws);
         if (a < 0) return a;
         launches += a;
     }
@@ -651,7 +656,7 @@ int plan_stages(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, v
     if (hist_after) TAOT_CUDA_OK(cudaStreamWaitEvent(st, hist_after, 0));
     {
         Range r("taot:histogram");
-        if ((a = taot_launch_histogram(h, d_topk, cc, o->info, st)) < 0) return a;
+        if ((a = taot_launch_histogram(h, d_topk, cc, o->info, st, ws)) < 0) return a;
     }
     total += a;
     if (hist_done) TAOT_CUDA_OK(cudaEventRecord(hist_done, st));

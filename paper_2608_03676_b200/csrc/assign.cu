@@ -26,6 +26,7 @@
 // sweep at 6.3-6.5 TB/s -- the memory system serves a contiguous sweep better than two interleaved subsets.
 // 8 bytes of HBM traffic per entry (one read, one write).  Out-of-range indices are copied through (the histogram
 // pass, whose counts this path consumes, is the one that flags them).
+#include <type_traits>
 #include "taot_internal.cuh"
 
 namespace {
@@ -43,6 +44,8 @@ struct AssignArgs {
     const int32_t* X;
     int32_t* out;
     int32_t* info;
+    const uint8_t* tb;          // the table as one byte per entry (histogram pass), or null
+    const int32_t* tbflag;      // [L,R,NC] nonzero: the chunk holds a value that is no expert (its bytes are not used)
     int64_t layer_elems, seg;
     int32_t nc, R, E, K;
 };
@@ -101,15 +104,24 @@ __device__ int build_entries(const int32_t* Xrow, const int32_t* se, int S, int 
 // Flat position, inside the chunk held at `buf`, of the entry of expert eb whose in-chunk ordinal is rel
 // (entries of eb before it belong to the slot whose quota ends there).  Block-wide: warp w owns entries
 // [w*2048, (w+1)*2048); per-warp counts, then ballots in the one warp that holds the entry.
-template <bool VEC>
-__device__ int32_t locate_split(const int32_t* buf, int32_t len, int eb, int rel, int* s_cntw, int* s_pos)
+// four entries at pos (a multiple of 4) of a chunk held as one byte per entry
+__device__ __forceinline__ int4 unpack_bytes(const void* buf, int32_t pos)
 {
+    const uint32_t w = *reinterpret_cast<const uint32_t*>(static_cast<const uint8_t*>(buf) + pos);
+    return make_int4((int)(w & 255u), (int)((w >> 8) & 255u), (int)((w >> 16) & 255u), (int)(w >> 24));
+}
+
+template <bool VEC, bool BYTES>
+__device__ int32_t locate_split(const void* bufv, int32_t len, int eb, int rel, int* s_cntw, int* s_pos)
+{
+    const int32_t* buf = static_cast<const int32_t*>(bufv);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int32_t wbase = warp * kWarpSpan + lane * 4;
     const unsigned lt = (1u << lane) - 1u;
     auto load4 = [&](int32_t pos) {
         int4 v = make_int4(-1, -1, -1, -1);
-        if (VEC && pos + 3 < len) v = *reinterpret_cast<const int4*>(buf + pos);
+        if (BYTES) { if (pos < len) v = unpack_bytes(bufv, pos); }
+        else if (VEC && pos + 3 < len) v = *reinterpret_cast<const int4*>(buf + pos);
         else {
             if (pos < len) v.x = buf[pos];
             if (pos + 1 < len) v.y = buf[pos + 1];
@@ -156,10 +168,11 @@ __device__ int32_t locate_split(const int32_t* buf, int32_t len, int eb, int rel
 
 // Rewrite one chunk: `buf` holds its entries (shared memory if staged, else global memory), `tab` its table and
 // `recs` its `ns` split records {expert, in-chunk ordinal of the split, target before, -} in shared memory.  Block-wide.
-template <bool VEC>
-__device__ void rewrite_chunk(const AssignArgs& a, const int32_t* buf, int32_t* tab, int32_t* dst,
+template <bool VEC, bool BYTES>
+__device__ void rewrite_chunk(const AssignArgs& a, const void* bufv, int32_t* tab, int32_t* dst,
                               int32_t len, const int ns, int4* recs, int* s_cntw, int* s_pos)
 {
+    const int32_t* buf = static_cast<const int32_t*>(bufv);
     const int E = a.E;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int32_t wbase = warp * kWarpSpan + lane * 4;
@@ -174,7 +187,8 @@ __device__ void rewrite_chunk(const AssignArgs& a, const int32_t* buf, int32_t* 
     };
     auto fetch = [&](int32_t pos) {
         int4 v = make_int4(-1, -1, -1, -1);
-        if (VEC) v = *reinterpret_cast<const int4*>(buf + pos);
+        if (BYTES) v = unpack_bytes(bufv, pos);
+        else if (VEC) v = *reinterpret_cast<const int4*>(buf + pos);
         else {
             if (pos < len) v.x = buf[pos];
             if (pos + 1 < len) v.y = buf[pos + 1];
@@ -190,10 +204,10 @@ __device__ void rewrite_chunk(const AssignArgs& a, const int32_t* buf, int32_t* 
             const int32_t pos = wbase + it * 128;
             if (pos < len) {
                 int4 v = fetch(pos);
-                if ((uint32_t)v.x < (uint32_t)E) v.x = tab[v.x];
-                if ((uint32_t)v.y < (uint32_t)E) v.y = tab[v.y];
-                if ((uint32_t)v.z < (uint32_t)E) v.z = tab[v.z];
-                if ((uint32_t)v.w < (uint32_t)E) v.w = tab[v.w];
+                if (BYTES || (uint32_t)v.x < (uint32_t)E) v.x = tab[v.x];  // a staged byte is an expert
+                if (BYTES || (uint32_t)v.y < (uint32_t)E) v.y = tab[v.y];
+                if (BYTES || (uint32_t)v.z < (uint32_t)E) v.z = tab[v.z];
+                if (BYTES || (uint32_t)v.w < (uint32_t)E) v.w = tab[v.w];
                 emit(pos, v);
             }
         }
@@ -209,7 +223,7 @@ __device__ void rewrite_chunk(const AssignArgs& a, const int32_t* buf, int32_t* 
                 const int4 rec = recs[k];
                 re[k] = rec.x;
                 rt[k] = rec.z;
-                rp[k] = locate_split<VEC>(buf, len, rec.x, rec.y, s_cntw, s_pos);
+                rp[k] = locate_split<VEC, BYTES>(bufv, len, rec.x, rec.y, s_cntw, s_pos);
             }
         }
 #pragma unroll
@@ -222,32 +236,40 @@ __device__ void rewrite_chunk(const AssignArgs& a, const int32_t* buf, int32_t* 
                     t = re[y]; re[y] = re[y - 1]; re[y - 1] = t;
                     t = rt[y]; rt[y] = rt[y - 1]; rt[y - 1] = t;
                 }
+        // the loop over the entries, with as many overrides per entry as the chunk has splits (the same for the block)
+        auto sweep = [&](auto nsc) {
+            constexpr int NS = decltype(nsc)::value;
 #pragma unroll 2
-        for (int it = 0; it < kIters; ++it) {
-            const int32_t pos = wbase + it * 128;
-            if (pos < len) {
-                int4 v = fetch(pos);
-                int32_t* xv = reinterpret_cast<int32_t*>(&v);
+            for (int it = 0; it < kIters; ++it) {
+                const int32_t pos = wbase + it * 128;
+                if (pos < len) {
+                    int4 v = fetch(pos);
+                    int32_t* xv = reinterpret_cast<int32_t*>(&v);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int32_t e = xv[j];
-                    if ((uint32_t)e < (uint32_t)E) {
-                        int32_t t = tab[e];
+                    for (int j = 0; j < 4; ++j) {
+                        const int32_t e = xv[j];
+                        if (BYTES || (uint32_t)e < (uint32_t)E) {          // a staged byte is an expert
+                            int32_t t = tab[e];
 #pragma unroll
-                        for (int k = 0; k < kFewSplits; ++k)
-                            if (e == re[k] && pos + j < rp[k]) t = rt[k];
-                        xv[j] = t;
+                            for (int k = 0; k < NS; ++k)
+                                if (e == re[k] && pos + j < rp[k]) t = rt[k];
+                            xv[j] = t;
+                        }
                     }
+                    emit(pos, v);
                 }
-                emit(pos, v);
             }
-        }
+        };
+        if (ns == 1) sweep(std::integral_constant<int, 1>{});
+        else if (ns == 2) sweep(std::integral_constant<int, 2>{});
+        else if (ns == 3) sweep(std::integral_constant<int, 3>{});
+        else sweep(std::integral_constant<int, kFewSplits>{});
         return;
     }
     // ---- many splits in one chunk (rare): located one by one, then a list walk
     const int nrec = ns;
     for (int k = 0; k < nrec; ++k) {
-        const int32_t P = locate_split<VEC>(buf, len, recs[k].x, recs[k].y, s_cntw, s_pos);
+        const int32_t P = locate_split<VEC, BYTES>(bufv, len, recs[k].x, recs[k].y, s_cntw, s_pos);
         if (tid == 0) recs[k].w = P;
     }
     __syncthreads();
@@ -337,7 +359,9 @@ __host__ __device__ inline size_t chunk_smem_words(int E, int S)
 // the slots its source rank feeds with their ordinal intervals (X, slot experts), the ordinal each expert has reached
 // at the start of the chunk (sum of the counts of the segment's earlier chunks), the table expert -> target of the
 // chunk's last entry of that expert, and one split record per quota interval that ends inside the chunk.
-template <bool VEC, bool STAGE>
+// BYTES (with STAGE): what is staged is the chunk as one byte per entry, left by the histogram pass -- a quarter of the
+// bytes; a chunk whose flag says it holds a value that is no expert is read from the table itself, without staging.
+template <bool VEC, bool STAGE, bool BYTES>
 __global__ void __launch_bounds__(kThreads)
 assign_chunk_kernel(AssignArgs a)
 {
@@ -345,7 +369,7 @@ assign_chunk_kernel(AssignArgs a)
     const int E = a.E, S = a.R * a.K;
     const int Ep = (E + 3) & ~3, Sp = (S + 3) & ~3;
     int32_t* stage = reinterpret_cast<int32_t*>(shc);                      // [TAOT_CHUNK] if STAGE
-    int32_t* tab = reinterpret_cast<int32_t*>(shc + (STAGE ? (size_t)TAOT_CHUNK * 4 : 0));   // [E] targets
+    int32_t* tab = reinterpret_cast<int32_t*>(shc + (STAGE ? (size_t)TAOT_CHUNK * (BYTES ? 1 : 4) : 0));   // [E] targets
     int32_t* cnt = tab + Ep;                             // [E] entries of each expert in this chunk
     int32_t* base = cnt + Ep;                            // [E] ordinal of each expert at the start of this chunk
     int32_t* ent_s = base + Ep;                          // [S] slots this rank feeds, ascending ...
@@ -364,20 +388,22 @@ assign_chunk_kernel(AssignArgs a)
     const int c = (int)(id % a.nc);
     int64_t goff; int32_t len;
     chunk_geometry(a, id, goff, len);
-    const int32_t* buf = a.topk + goff;
+    const void* buf = a.topk + goff;
     if (STAGE) {
         if (tid == 0) {
             mbar_init(&bar, 1);
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-            const uint32_t bytes = (uint32_t)len * 4u;
+            const uint32_t bytes = (uint32_t)len * (BYTES ? 1u : 4u);
+            const unsigned char* from = BYTES ? a.tb + goff : reinterpret_cast<const unsigned char*>(a.topk + goff);
             mbar_expect_tx(&bar, bytes);
             const uint64_t once = policy_evict_first();
             for (uint32_t o = 0; o < bytes; o += kBulkPiece)
-                bulk_load_once(reinterpret_cast<unsigned char*>(stage) + o, reinterpret_cast<const unsigned char*>(buf) + o,
+                bulk_load_once(reinterpret_cast<unsigned char*>(stage) + o, from + o,
                                (bytes - o) < kBulkPiece ? (bytes - o) : kBulkPiece, &bar, once);
         }
         buf = stage;
     }
+    const int32_t flagged = BYTES ? a.tbflag[id] : 0;    // the staged bytes are of no use: read the table itself
     // ---- the chunk's table and split records
     if (tid == 0) s_ns = 0;
     const int32_t* ccseg = a.cc + lr * a.nc * (int64_t)E;
@@ -410,7 +436,8 @@ assign_chunk_kernel(AssignArgs a)
             return;
         }
     }
-    rewrite_chunk<VEC>(a, buf, tab, a.out + goff, len, s_ns, recs, s_cntw, &s_pos);
+    if (BYTES && flagged) rewrite_chunk<VEC, false>(a, a.topk + goff, tab, a.out + goff, len, s_ns, recs, s_cntw, &s_pos);
+    else rewrite_chunk<VEC, BYTES>(a, buf, tab, a.out + goff, len, s_ns, recs, s_cntw, &s_pos);
 }
 
 }  // namespace
@@ -430,14 +457,22 @@ int taot_launch_assign(taot_handle_t h, const int32_t* d_topk, void* ws, const i
     const int S = p.R * p.K;
     const unsigned blocks = (unsigned)((int64_t)p.L * p.R * h->nc);
     const size_t words = chunk_smem_words(p.E, S);
-    if (vec_ok) {
+    a.tb = nullptr; a.tbflag = nullptr;
+    if (vec_ok && h->tb_ok) {
+        // the histogram pass that left the chunk counts also left the table as one byte per entry
+        a.tb = reinterpret_cast<const uint8_t*>(w + h->off_tb);
+        a.tbflag = reinterpret_cast<const int32_t*>(w + h->off_tbflag);
+        const size_t smem = (size_t)TAOT_CHUNK + sizeof(int32_t) * words;
+        TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        assign_chunk_kernel<true, true, true><<<blocks, kThreads, smem, st>>>(a);
+    } else if (vec_ok) {
         const size_t smem = (size_t)TAOT_CHUNK * 4 + sizeof(int32_t) * words;
-        TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        assign_chunk_kernel<true, true><<<blocks, kThreads, smem, st>>>(a);
+        TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<true, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        assign_chunk_kernel<true, true, false><<<blocks, kThreads, smem, st>>>(a);
     } else {
         const size_t smem = sizeof(int32_t) * words;
-        TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        assign_chunk_kernel<false, false><<<blocks, kThreads, smem, st>>>(a);
+        TAOT_CUDA_OK(cudaFuncSetAttribute(assign_chunk_kernel<false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        assign_chunk_kernel<false, false, false><<<blocks, kThreads, smem, st>>>(a);
     }
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;

@@ -33,10 +33,20 @@ __device__ __forceinline__ void count_one(int32_t* hist, int32_t e, int32_t E, i
     else { bad = 1; if (EXTRA) atomicAdd(hist + E, 1); }
 }
 
+// four entries as four bytes (E <= 256; a value that is no expert leaves a byte nobody reads: its chunk is flagged)
+__device__ __forceinline__ uint32_t pack_bytes(const int4& x)
+{
+    return ((uint32_t)x.x & 255u) | (((uint32_t)x.y & 255u) << 8) | (((uint32_t)x.z & 255u) << 16) | ((uint32_t)x.w << 24);
+}
+
+// tb (may be null; only with vec_ok): the table again as one byte per entry, written beside the counts, and tbflag:
+// one word per chunk, nonzero if the chunk holds a value that is no expert.  The reassignment reads these 1-byte
+// entries instead of the table (a quarter of the bytes) wherever the chunk's flag is zero.
 template <bool EXTRA>
 __global__ void __launch_bounds__(kThreads)
 hist_chunk_kernel(const int32_t* __restrict__ topk, int32_t* __restrict__ cc, int32_t* __restrict__ info,
-                  int64_t layer_elems, int64_t seg, int32_t nc, int32_t R, int32_t E, int vec_ok)
+                  int64_t layer_elems, int64_t seg, int32_t nc, int32_t R, int32_t E, int vec_ok,
+                  uint8_t* __restrict__ tb, int32_t* __restrict__ tbflag)
 {
     const int32_t nb = EXTRA ? E + 1 : E;
     extern __shared__ int32_t sh_hist[];                 // [kWarps][nb]
@@ -49,6 +59,7 @@ hist_chunk_kernel(const int32_t* __restrict__ topk, int32_t* __restrict__ cc, in
     const int64_t start = (int64_t)c * TAOT_CHUNK;
     const int32_t len = (int32_t)((seg - start) < (int64_t)TAOT_CHUNK ? (seg - start) : (int64_t)TAOT_CHUNK);
     const int32_t* src = topk + (int64_t)l * layer_elems + (int64_t)r * seg + start;
+    uint32_t* tb4 = (!EXTRA && tb) ? reinterpret_cast<uint32_t*>(tb + (int64_t)l * layer_elems + (int64_t)r * seg + start) : nullptr;
 
     for (int i = tid; i < kWarps * nb; i += kThreads) sh_hist[i] = 0;
     __syncthreads();
@@ -64,6 +75,10 @@ hist_chunk_kernel(const int32_t* __restrict__ topk, int32_t* __restrict__ cc, in
             int4 x[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) x[u] = ld_stream(src4 + v + u * kThreads);
+            if (!EXTRA && tb4) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) tb4[v + u * kThreads] = pack_bytes(x[u]);
+            }
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 count_one<EXTRA>(hist, x[u].x, E, bad); count_one<EXTRA>(hist, x[u].y, E, bad);
@@ -72,6 +87,7 @@ hist_chunk_kernel(const int32_t* __restrict__ topk, int32_t* __restrict__ cc, in
         }
         for (; v < nvec; v += kThreads) {
             const int4 x = ld_stream(src4 + v);
+            if (!EXTRA && tb4) tb4[v] = pack_bytes(x);
             count_one<EXTRA>(hist, x.x, E, bad); count_one<EXTRA>(hist, x.y, E, bad);
             count_one<EXTRA>(hist, x.z, E, bad); count_one<EXTRA>(hist, x.w, E, bad);
         }
@@ -88,6 +104,7 @@ hist_chunk_kernel(const int32_t* __restrict__ topk, int32_t* __restrict__ cc, in
         out[e] = tot;
     }
     if (any_bad && tid == 0) atomicOr(info + l, TAOT_INFO_BAD_INDEX);
+    if (!EXTRA && tbflag && tid == 0) tbflag[id] = any_bad;
 }
 
 // excess / spare of one row of rank loads held in shared memory (Appendix A.1, integer mean)
@@ -198,15 +215,20 @@ excess_spare_kernel(const int32_t* __restrict__ rank_load, int32_t* excess, int3
 
 }  // namespace
 
-int taot_launch_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_cc, int32_t* d_info, cudaStream_t st)
+int taot_launch_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_cc, int32_t* d_info, cudaStream_t st,
+                          void* ws)
 {
     const taot_params& p = h->p;
     const int64_t layer_elems = p.T * p.k;
     const int64_t blocks = (int64_t)p.L * p.R * h->nc;
     const int vec_ok = ((reinterpret_cast<uintptr_t>(d_topk) & 15) == 0) && (h->seg % 4 == 0);
     const size_t smem = sizeof(int32_t) * kWarps * p.E;
+    // with a workspace (and 16-byte accesses) the pass also leaves the table as one byte per entry for the reassignment
+    const bool bytes = ws && h->tb_ok && vec_ok;
+    uint8_t* tb = bytes ? reinterpret_cast<uint8_t*>(static_cast<char*>(ws) + h->off_tb) : nullptr;
+    int32_t* tbflag = bytes ? reinterpret_cast<int32_t*>(static_cast<char*>(ws) + h->off_tbflag) : nullptr;
     hist_chunk_kernel<false><<<(unsigned)blocks, kThreads, smem, st>>>(d_topk, d_cc, d_info, layer_elems, h->seg,
-                                                                        h->nc, p.R, p.E, vec_ok);
+                                                                        h->nc, p.R, p.E, vec_ok, tb, tbflag);
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
 }
@@ -224,7 +246,7 @@ int taot_launch_chunk_counts(taot_handle_t h, const int32_t* d_idx, int32_t* d_c
     if (smem > 48 * 1024)
         TAOT_CUDA_OK(cudaFuncSetAttribute(hist_chunk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     hist_chunk_kernel<true><<<(unsigned)blocks, kThreads, smem, st>>>(d_idx, d_counts, d_info, p.T * p.k, h->seg, h->nc,
-                                                                       p.R, bins, vec_ok);
+                                                                       p.R, bins, vec_ok, nullptr, nullptr);
     TAOT_CUDA_OK(cudaGetLastError());
     return 1;
 }

@@ -50,6 +50,9 @@ struct taot_handle_s {
     int64_t kcap_global;     // same, global-memory scratch per problem (R > 256 only), else 0
     // workspace layout (byte offsets)
     size_t off_cc, off_excess, off_spare, off_s, off_d, off_nrem, off_t12, off_kt, off_dc, off_cyc, off_tc;
+    size_t off_tb, off_tbflag;   // one-byte copy of the routing table and one flag per chunk (see tb_ok)
+    int32_t tb_ok;               // 1: the histogram pass also leaves the table as one byte per entry (E <= 256 experts,
+                                 // segments of a multiple of 16 entries) for the reassignment to read instead of the table
     size_t ws_bytes;
     // host-call staging layout (byte offsets into d_ws of taot_plan_host)
     size_t hoff_topk, hoff_new, hoff_n, hoff_el, hoff_rl, hoff_ex, hoff_sp, hoff_plan, hoff_it, hoff_err,
@@ -74,7 +77,8 @@ struct taot_handle_s {
 static inline size_t taot_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // kernel launchers (each returns the number of kernels it enqueued, or a negative taot_status)
-int taot_launch_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_cc, int32_t* d_info, cudaStream_t st);
+int taot_launch_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_cc, int32_t* d_info, cudaStream_t st,
+                          void* ws = nullptr);
 int taot_launch_merge(taot_handle_t h, const int32_t* d_cc, int32_t* d_n, int32_t* d_expert_load,
                       int32_t* d_rank_load, int32_t* d_excess, int32_t* d_spare, float* d_s, float* d_d,
                       cudaStream_t st, int32_t* d_info = nullptr);
