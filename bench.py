@@ -40,7 +40,24 @@ FP32_LANES_PER_SM = 128
 # 8 layers; traffic grows in proportion to the entries processed, so a full launch is scaled by its own
 # algorithmic bytes).  The reassignment figure is read + write once dirty L2 lines drain.
 HIST_TRAFFIC_RATIO = 1.045
+HIST_TRAFFIC_RATIO_BYTES = 1.01      # with the one-byte copy of the table written beside the counts (config 4 shape, 8 layers)
 ASSIGN_TRAFFIC_RATIO = 1.01
+
+
+def byte_table(cfg) -> bool:
+    """The library's rule for leaving the routing table as one byte per entry in the histogram pass (which the
+    reassignment then reads instead of the table): at most 256 experts, rank segments of a multiple of 16 entries."""
+    return cfg.R <= 256 and cfg.E <= 256 and (cfg.T // cfg.R * cfg.k) % 16 == 0
+
+
+def stream_bytes(cfg):
+    """Algorithmic HBM bytes of the histogram and of the reassignment for one call: 4 B per entry read and 4 B per entry
+    written in any case; with the byte table the histogram also writes 1 B per entry and the reassignment reads that byte
+    instead of the entry (10 B per entry for the two kernels together instead of 12)."""
+    entries = cfg.L * cfg.T * cfg.k
+    if byte_table(cfg):
+        return 5 * entries, 5 * entries
+    return 4 * entries, 8 * entries
 # the matching kernel reads its layer's counts, plan and lists once and keeps every round in shared memory: DRAM bytes per
 # layer from one ncu capture at the config-4 shape (606 KB read, nothing written back by the end, for 2 layers)
 MATCH_DRAM_BYTES_PER_LAYER = 303_000
@@ -288,15 +305,18 @@ def sinkhorn_work(out, cfg):
 def roofline_for(stage, ms, cfg, out, peaks, sm_count, match_cyc=None):
     topk_bytes = cfg.L * cfg.T * cfg.k * 4
     hbm = peaks["hbm_gbs"]
+    hist_bytes, assign_bytes = stream_bytes(cfg)
     if stage == "histogram":
-        a = topk_bytes / (ms * 1e-3) / 1e9
+        a = hist_bytes / (ms * 1e-3) / 1e9
         return dict(kernel="hist_chunk_kernel", bound="hbm", achieved=a, peak=hbm, unit="GB/s", frac=a / hbm,
-                    traffic=HIST_TRAFFIC_RATIO * topk_bytes, peak_source=peaks["source"], bytes_per_launch=topk_bytes)
+                    traffic=(HIST_TRAFFIC_RATIO_BYTES if byte_table(cfg) else HIST_TRAFFIC_RATIO) * hist_bytes,
+                    peak_source=peaks["source"], bytes_per_launch=hist_bytes,
+                    byte_table=byte_table(cfg))
     if stage == "assign":
-        a = 2 * topk_bytes / (ms * 1e-3) / 1e9
+        a = assign_bytes / (ms * 1e-3) / 1e9
         return dict(kernel="assign_chunk_kernel", bound="hbm", achieved=a, peak=hbm, unit="GB/s",
-                    frac=a / hbm, traffic=ASSIGN_TRAFFIC_RATIO * 2 * topk_bytes, peak_source=peaks["source"],
-                    bytes_per_launch=2 * topk_bytes)
+                    frac=a / hbm, traffic=ASSIGN_TRAFFIC_RATIO * assign_bytes, peak_source=peaks["source"],
+                    bytes_per_launch=assign_bytes, byte_table=byte_table(cfg))
     if stage == "merge":
         b = cfg.L * cfg.R * cfg.E * 4 * (2 + max(1, (cfg.T // cfg.R * cfg.k + 16383) // 16384))
         a = b / (ms * 1e-3) / 1e9
@@ -436,7 +456,8 @@ def stream_report(name, peaks, steps=5, flush=None):
     pl.set_profiling(False)
     rep = dict(workload=name, topk_bytes=b, table_larger_than_l2=2 * b >= 4 * L2_BYTES,
                stages_ms=dict(zip(STAGES, [float(x) for x in acc])), stages_sum_ms=float(acc.sum()), ms_per_step=call_ms,
-               histogram_gbs=b / (acc[0] * 1e-3) / 1e9, assign_gbs=2 * b / (acc[4] * 1e-3) / 1e9,
+               histogram_gbs=stream_bytes(cfg)[0] / (acc[0] * 1e-3) / 1e9, assign_gbs=stream_bytes(cfg)[1] / (acc[4] * 1e-3) / 1e9,
+               byte_table=byte_table(cfg),
                peak_gbs=peaks["hbm_gbs"], peak_source=peaks["source"],
                remapped_tokens_per_s=cfg.L * cfg.T / (acc[4] * 1e-3),
                plans_per_s=cfg.L / (call_ms * 1e-3))

@@ -139,7 +139,8 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
 /* Frees the handle's device copies.  Synchronises the device.  NULL is accepted. */
 int taot_destroy(taot_handle_t h);
 
-/* Scratch bytes taot_* calls need in `ws` for this handle (device memory, 256-byte aligned). */
+/* Scratch bytes taot_* calls need in `ws` for this handle (device memory, 256-byte aligned).  With at most 256
+ * experts this includes L*T*k bytes for a one-byte copy of the routing table (see taot_assign). */
 int taot_workspace_bytes(taot_handle_t h, size_t* bytes);
 
 /* Device scratch bytes taot_plan_host needs (staging of inputs/outputs plus the workspace). */
@@ -242,8 +243,10 @@ int taot_match(taot_handle_t h, const int32_t* d_n, const int32_t* d_expert_load
  * (source rank, expert) group, in flat order t*k + j, the slots holding that expert take, lowest
  * slot first, the first X[r][s] entries; an entry so taken is rewritten to E + s, the rest keep e.
  *   d_new_idx [L,T,k] must not alias d_topk.
- *   reuse_counts != 0: trust the per-chunk counts left in `ws` by taot_histogram on the same
- *   d_topk; 0: recount (one more read of d_topk).
+ *   reuse_counts != 0: trust what taot_histogram left in `ws` for the same d_topk -- the per-chunk counts and, with at
+ *   most 256 experts, 16-byte aligned tables and rank segments of a multiple of 16 entries, a copy of the table as one
+ *   byte per entry with one flag per chunk, which the rewrite then reads instead of d_topk (chunks holding a value that
+ *   is no expert are read from d_topk itself); 0: recount (one more read of d_topk).
  */
 int taot_assign(taot_handle_t h, const int32_t* d_topk, const int32_t* d_slot_expert,
                 const int32_t* d_X, int32_t* d_new_idx, int32_t* d_info, void* ws,

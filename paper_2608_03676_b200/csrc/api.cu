@@ -380,12 +380,17 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
             // Group sizes grow: a group's chain of latency-bound stages takes about as long whatever its size, so a
             // group can only finish (and rewrite its part of the table) under the others' chains if it started
             // earlier by about the time its reassignment takes; the stagger of the starts is the histogram of the
-            // group itself, roughly half as long as its reassignment.  Measured on configs 3 and 4: 2 : 3 : 5 : 8 best
-            // with four groups, 2 : 3 : 4 : 6 : 9 with five, 3 : 4 : 5 : 6 : 8 : 10 with six (and six about 2 % faster
-            // than four where the table is large enough for six).
-            static const double kWeights[3][TAOT_MAX_GROUPS] = {
-                {2.0, 3.0, 5.0, 8.0, 0.0, 0.0}, {2.0, 3.0, 4.0, 6.0, 9.0, 0.0}, {3.0, 4.0, 5.0, 6.0, 8.0, 10.0}};
-            const double* wt = kWeights[G <= 4 ? 0 : G - 4];
+            // group itself.  Measured on configs 3 and 4: 2 : 3 : 5 : 8 best with four groups, 2 : 3 : 4 : 6 : 9 with
+            // five, 3 : 4 : 5 : 6 : 8 : 10 with six (and six about 2 % faster than four where the table is large enough
+            // for six).  At 256 ranks the chain (a thousand Sinkhorn iterations, two thousand auction rounds) is several
+            // times as long as all bandwidth-bound work together, and since the reassignment reads one byte per entry
+            // it is short enough to fit behind the other groups' chains whatever the order: equal sizes, which keep
+            // the last chain's own reassignment small, measured 1.88 ms against 1.95 ms with growing sizes at config 4
+            // (config 3, 64 ranks: 0.82 ms growing, 0.84 ms equal).
+            static const double kWeights[4][TAOT_MAX_GROUPS] = {
+                {2.0, 3.0, 5.0, 8.0, 0.0, 0.0}, {2.0, 3.0, 4.0, 6.0, 9.0, 0.0}, {3.0, 4.0, 5.0, 6.0, 8.0, 10.0},
+                {1.0, 1.0, 1.0, 1.0, 1.0, 1.0}};
+            const double* wt = kWeights[G <= 4 ? 0 : ((G == 6 && R >= 256) ? 3 : G - 4)];
             double wsum = 0.0;
             for (int g = 0; g < G; ++g) wsum += wt[g];
             int l0 = 0;

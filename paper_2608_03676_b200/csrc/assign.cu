@@ -24,8 +24,11 @@
 // One sweep over all chunks matters: two kernels that each took part of the chunks (a persistent pipeline for the
 // chunks without a split, a per-chunk kernel for the rest) were measured at 5.4-5.7 TB/s on their parts, a single
 // sweep at 6.3-6.5 TB/s -- the memory system serves a contiguous sweep better than two interleaved subsets.
-// 8 bytes of HBM traffic per entry (one read, one write).  Out-of-range indices are copied through (the histogram
-// pass, whose counts this path consumes, is the one that flags them).
+// 8 bytes of HBM traffic per entry (one read, one write) -- or 5 where the histogram pass has left the table as one byte
+// per entry beside its counts (at most 256 experts, 16-byte aligned tables, segments of a multiple of 16 entries): the
+// rewrite only needs to know each entry's expert, so it stages those 16 KB per chunk instead of 64 KB of the table; a chunk
+// that holds a value which is no expert (flagged by the histogram pass) is read from the table itself.  Out-of-range
+// indices are copied through (the histogram pass, whose counts this path consumes, is the one that flags them).
 #include <type_traits>
 #include "taot_internal.cuh"
 

@@ -6,7 +6,10 @@
 // chunk of at most TAOT_CHUNK elements of one segment: it streams the chunk with 16-byte loads,
 // counts into per-warp private shared-memory histograms, and stores its E counts with plain
 // stores -- no global atomics, no zero-fill of the outputs.  The per-chunk counts are kept: the
-// reassignment kernel turns them into each chunk's starting ordinals.
+// reassignment kernel turns them into each chunk's starting ordinals.  Where the table has at most
+// 256 experts the pass also leaves every entry as one byte in the workspace (plus one flag per
+// chunk for values that are no expert): the reassignment, which runs last and alone on the memory
+// system, then reads a quarter of the bytes, for one more byte per entry written here.
 #include <cstring>
 #include <mutex>
 
