@@ -112,7 +112,8 @@ def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
 
 STATIC_SCRATCH_BYTES = 4 << 20
 # kernels one taot_plan call enqueues: chunk histogram, merge, Sinkhorn (register tile + shared-memory
-# kernel for handed-back problems), matching+auction, reassignment
+# kernel for handed-back problems), matching+auction, reassignment (a handle that splits a 256-rank table into layer
+# groups adds one launch per group: the one-byte copy of the group's table)
 PLAN_LAUNCHES = 6
 PLAN_LAUNCHES_NO_HINT = 4       # with ABLATE_HINT the two Sinkhorn kernels are not launched
 

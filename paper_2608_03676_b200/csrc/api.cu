@@ -377,6 +377,8 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
         while (G > 1 && (params->L < 2 * G || (params->L / G) * chunks_per_layer <= 3 * (int64_t)h->sm_count)) --G;
         if (G > 1) {
             if (cudaEventCreate(&h->ev_fork) != cudaSuccess) rc = TAOT_ERR_CUDA;      // timed: origin of the group trace
+            // (only where a group's chain of latency-bound stages outlasts the copy of the whole table: 256 ranks)
+            if (rc == TAOT_OK && h->tb_ok && R >= 256 && cudaStreamCreateWithFlags(&h->bstream, cudaStreamNonBlocking) != cudaSuccess) rc = TAOT_ERR_CUDA;
             // Group sizes grow: a group's chain of latency-bound stages takes about as long whatever its size, so a
             // group can only finish (and rewrite its part of the table) under the others' chains if it started
             // earlier by about the time its reassignment takes; the stagger of the starts is the histogram of the
@@ -407,6 +409,7 @@ int taot_create(taot_handle_t* out, const taot_params* params, const int32_t* h_
                 if (g > 0 && cudaStreamCreateWithFlags(&h->gstream[g], cudaStreamNonBlocking) != cudaSuccess) rc = TAOT_ERR_CUDA;
                 if (rc == TAOT_OK && cudaEventCreateWithFlags(&h->ev_hist[g], cudaEventDisableTiming) != cudaSuccess) rc = TAOT_ERR_CUDA;
                 if (rc == TAOT_OK && cudaEventCreateWithFlags(&h->ev_join[g], cudaEventDisableTiming) != cudaSuccess) rc = TAOT_ERR_CUDA;
+                if (rc == TAOT_OK && cudaEventCreateWithFlags(&h->ev_bytes[g], cudaEventDisableTiming) != cudaSuccess) rc = TAOT_ERR_CUDA;
                 h->ngroups = g + 1;
             }
         }
@@ -440,8 +443,10 @@ int taot_destroy(taot_handle_t h)
         if (h->gstream[g]) cudaStreamDestroy(h->gstream[g]);
         if (h->ev_hist[g]) cudaEventDestroy(h->ev_hist[g]);
         if (h->ev_join[g]) cudaEventDestroy(h->ev_join[g]);
+        if (h->ev_bytes[g]) cudaEventDestroy(h->ev_bytes[g]);
     }
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->bstream) cudaStreamDestroy(h->bstream);
     cudaFree(h->d_e2r); cudaFree(h->d_C); cudaFree(h->d_B); cudaFree(h->d_rowlse0); cudaFree(h->d_gibbs);
     cudaFree(h->d_rank_off); cudaFree(h->d_rank_list); cudaFree(h->d_tierval); cudaFree(h->d_tiermask);
     cudaFree(h->d_tpos); cudaFree(h->d_torder); cudaFree(h->d_tdest); cudaFree(h->d_bidlist);
@@ -640,8 +645,10 @@ namespace {
 // The five stages for the layers of one handle (or of one view of it) on one stream.  `hist_after`, if set, is waited for
 // before the chunk histogram starts and `hist_done`, if set, is recorded after it: consecutive layer groups start
 // their bandwidth-bound first stage one after the other instead of sharing the memory system.
+// `bytes_later`: the one-byte copy of the table is not made by the histogram pass and the reassignment is left out --
+// the caller makes the copy elsewhere and then calls assign_stage.
 int plan_stages(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, void* ws, cudaStream_t st, bool marks,
-                cudaEvent_t hist_after, cudaEvent_t hist_done, int* launches)
+                cudaEvent_t hist_after, cudaEvent_t hist_done, int* launches, bool bytes_later = false)
 {
     const taot_params& p = h->p;
     int32_t* cc = reinterpret_cast<int32_t*>(at(ws, h->off_cc));
@@ -661,7 +668,7 @@ int plan_stages(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, v
     if (hist_after) TAOT_CUDA_OK(cudaStreamWaitEvent(st, hist_after, 0));
     {
         Range r("taot:histogram");
-        if ((a = taot_launch_histogram(h, d_topk, cc, o->info, st, ws)) < 0) return a;
+        if ((a = taot_launch_histogram(h, d_topk, cc, o->info, st, ws, !bytes_later)) < 0) return a;
     }
     total += a;
     if (hist_done) TAOT_CUDA_OK(cudaEventRecord(hist_done, st));
@@ -697,14 +704,27 @@ int plan_stages(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, v
     nvtxRangePop();
     total += a;
     TAOT_MARK(4);
-    {
+    if (!bytes_later) {
         Range r("taot:reassignment");
         if ((a = taot_launch_assign(h, d_topk, ws, o->slot_expert, o->X, o->new_idx, o->info, st)) < 0) return a;
+        total += a;
+        TAOT_MARK(5);
     }
-    total += a;
-    TAOT_MARK(5);
 #undef TAOT_MARK
     *launches += total;
+    return TAOT_OK;
+}
+
+// The last stage on its own, for a call whose plan_stages left it out.
+int assign_stage(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, void* ws, cudaStream_t st, bool marks,
+                 int* launches)
+{
+    nvtxRangePushA("taot:reassignment");
+    const int a = taot_launch_assign(h, d_topk, ws, o->slot_expert, o->X, o->new_idx, o->info, st);
+    nvtxRangePop();
+    if (a < 0) return a;
+    if (marks) TAOT_CUDA_OK(cudaEventRecord(h->ev[5], st));
+    *launches += a;
     return TAOT_OK;
 }
 
@@ -752,6 +772,8 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, voi
     // stream by an event and joined back into it by one event each; no allocation, no synchronisation, and the fork /
     // join pattern is what stream capture expects.
     TAOT_CUDA_OK(cudaEventRecord(h->ev_fork, st));
+    const bool side_bytes = h->bstream != nullptr && h->tb_ok && (reinterpret_cast<uintptr_t>(d_topk) & 15) == 0 &&
+                            (reinterpret_cast<uintptr_t>(o->new_idx) & 15) == 0;
     for (int g = 0; g < h->ngroups; ++g) {
         taot_handle_s* v = h->group[g];
         const int l0 = h->group_l0[g];
@@ -759,9 +781,31 @@ int taot_plan(taot_handle_t h, const int32_t* d_topk, const taot_outputs* o, voi
         if (g > 0) TAOT_CUDA_OK(cudaStreamWaitEvent(gs, h->ev_fork, 0));
         const taot_outputs go = outputs_from_layer(p, o, l0);
         const int rc = plan_stages(v, d_topk + (size_t)l0 * p.T * p.k, &go, ws, gs, h->profiling == 3,
-                                   g > 0 ? h->ev_hist[g - 1] : nullptr, g + 1 < h->ngroups ? h->ev_hist[g] : nullptr, &total);
+                                   g > 0 ? h->ev_hist[g - 1] : nullptr,
+                                   (g + 1 < h->ngroups || side_bytes) ? h->ev_hist[g] : nullptr, &total, side_bytes);
         if (rc != TAOT_OK) return rc;
-        if (g > 0) TAOT_CUDA_OK(cudaEventRecord(h->ev_join[g], gs));
+        if (g > 0 && !side_bytes) TAOT_CUDA_OK(cudaEventRecord(h->ev_join[g], gs));
+    }
+    if (side_bytes) {
+        // The one-byte copies the reassignment reads are made on a stream of their own once every histogram is done (the
+        // memory system is idle from then until the first matching ends), by a grid too small to get in the way of the
+        // chains; each group's reassignment waits for its copy.
+        TAOT_CUDA_OK(cudaStreamWaitEvent(h->bstream, h->ev_hist[h->ngroups - 1], 0));
+        for (int g = 0; g < h->ngroups; ++g) {
+            const int a = taot_launch_table_bytes(h->group[g], d_topk + (size_t)h->group_l0[g] * p.T * p.k, ws, h->bstream);
+            if (a < 0) return a;
+            total += a;
+            TAOT_CUDA_OK(cudaEventRecord(h->ev_bytes[g], h->bstream));
+        }
+        for (int g = 0; g < h->ngroups; ++g) {
+            cudaStream_t gs = g == 0 ? st : h->gstream[g];
+            const taot_outputs go = outputs_from_layer(p, o, h->group_l0[g]);
+            TAOT_CUDA_OK(cudaStreamWaitEvent(gs, h->ev_bytes[g], 0));
+            const int rc = assign_stage(h->group[g], d_topk + (size_t)h->group_l0[g] * p.T * p.k, &go, ws, gs,
+                                        h->profiling == 3, &total);
+            if (rc != TAOT_OK) return rc;
+            if (g > 0) TAOT_CUDA_OK(cudaEventRecord(h->ev_join[g], gs));
+        }
     }
     for (int g = 1; g < h->ngroups; ++g) TAOT_CUDA_OK(cudaStreamWaitEvent(st, h->ev_join[g], 0));
     h->last_launches = total;

@@ -218,8 +218,46 @@ excess_spare_kernel(const int32_t* __restrict__ rank_load, int32_t* excess, int3
 
 }  // namespace
 
+namespace {
+
+// The table as one byte per entry, as a pass of its own: a grid of a few CTAs that walks the whole table, for use while
+// other streams run latency-bound kernels that want SMs to themselves (its dynamic shared memory is only there to keep
+// such CTAs off the SMs it sits on, and it off theirs).
+constexpr int kBytesCtas = 48;
+constexpr int kBytesSmem = 100 * 1024;
+
+__global__ void __launch_bounds__(1024)
+table_bytes_kernel(const int4* __restrict__ src, uint32_t* __restrict__ dst, int64_t nvec)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; v + 3 * stride < nvec; v += 4 * stride) {
+        int4 x[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) x[u] = ld_stream(src + v + u * stride);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) dst[v + u * stride] = pack_bytes(x[u]);
+    }
+    for (; v < nvec; v += stride) dst[v] = pack_bytes(ld_stream(src + v));
+}
+
+}  // namespace
+
+int taot_launch_table_bytes(taot_handle_t h, const int32_t* d_topk, void* ws, cudaStream_t st)
+{
+    const taot_params& p = h->p;
+    const int vec_ok = ((reinterpret_cast<uintptr_t>(d_topk) & 15) == 0) && (h->seg % 4 == 0);
+    if (!ws || !h->tb_ok || !vec_ok) return 0;
+    const int64_t nvec = (int64_t)p.L * p.T * p.k / 4;
+    TAOT_CUDA_OK(cudaFuncSetAttribute(table_bytes_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBytesSmem));
+    table_bytes_kernel<<<kBytesCtas, 1024, kBytesSmem, st>>>(reinterpret_cast<const int4*>(d_topk),
+                                                              reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + h->off_tb), nvec);
+    TAOT_CUDA_OK(cudaGetLastError());
+    return 1;
+}
+
 int taot_launch_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_cc, int32_t* d_info, cudaStream_t st,
-                          void* ws)
+                          void* ws, bool write_bytes)
 {
     const taot_params& p = h->p;
     const int64_t layer_elems = p.T * p.k;
@@ -228,7 +266,7 @@ int taot_launch_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_cc,
     const size_t smem = sizeof(int32_t) * kWarps * p.E;
     // with a workspace (and 16-byte accesses) the pass also leaves the table as one byte per entry for the reassignment
     const bool bytes = ws && h->tb_ok && vec_ok;
-    uint8_t* tb = bytes ? reinterpret_cast<uint8_t*>(static_cast<char*>(ws) + h->off_tb) : nullptr;
+    uint8_t* tb = (bytes && write_bytes) ? reinterpret_cast<uint8_t*>(static_cast<char*>(ws) + h->off_tb) : nullptr;
     int32_t* tbflag = bytes ? reinterpret_cast<int32_t*>(static_cast<char*>(ws) + h->off_tbflag) : nullptr;
     hist_chunk_kernel<false><<<(unsigned)blocks, kThreads, smem, st>>>(d_topk, d_cc, d_info, layer_elems, h->seg,
                                                                         h->nc, p.R, p.E, vec_ok, tb, tbflag);

@@ -72,13 +72,17 @@ struct taot_handle_s {
     int32_t group_len[TAOT_MAX_GROUPS];
     cudaStream_t gstream[TAOT_MAX_GROUPS];     // [0] unused: group 0 runs on the caller's stream
     cudaEvent_t ev_fork, ev_hist[TAOT_MAX_GROUPS], ev_join[TAOT_MAX_GROUPS];
+    cudaStream_t bstream;                      // the one-byte copies of the groups' tables are made here, after all histograms
+    cudaEvent_t ev_bytes[TAOT_MAX_GROUPS];     // group g's copy is there
 };
 
 static inline size_t taot_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // kernel launchers (each returns the number of kernels it enqueued, or a negative taot_status)
 int taot_launch_histogram(taot_handle_t h, const int32_t* d_topk, int32_t* d_cc, int32_t* d_info, cudaStream_t st,
-                          void* ws = nullptr);
+                          void* ws = nullptr, bool write_bytes = true);
+// the table as one byte per entry, by a few CTAs that leave the other SMs alone (returns 0 if this handle keeps no such copy)
+int taot_launch_table_bytes(taot_handle_t h, const int32_t* d_topk, void* ws, cudaStream_t st);
 int taot_launch_merge(taot_handle_t h, const int32_t* d_cc, int32_t* d_n, int32_t* d_expert_load,
                       int32_t* d_rank_load, int32_t* d_excess, int32_t* d_spare, float* d_s, float* d_d,
                       cudaStream_t st, int32_t* d_info = nullptr);

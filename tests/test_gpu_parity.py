@@ -228,12 +228,13 @@ def test_plan_is_capturable_in_a_cuda_graph():
     pl.close()
 
 
-@pytest.mark.parametrize("L,G", [(9, 4), (13, 6)])
-def test_layer_groups_on_internal_streams_change_no_bit_and_can_be_captured(monkeypatch, L, G):
+@pytest.mark.parametrize("base,over,L,G", [("cfg3", {}, 9, 4), ("cfg3", {}, 13, 6), ("cfg4", dict(T=256 * 2048), 12, 6)])
+def test_layer_groups_on_internal_streams_change_no_bit_and_can_be_captured(monkeypatch, base, over, L, G):
     """A routing table large enough to be bandwidth-bound makes taot_plan split the layers into groups on streams of
     its own (fork / join by events).  The split must change no output, it must be capturable in a CUDA graph, and the
-    group timeline must show every group passing through the five stages in order."""
-    cfg = W.get_config("cfg3").replace(L=L)              # L x 64 x 4 chunks: 9 layers make four groups, 13 make six
+    group timeline must show every group passing through the five stages in order.  At 256 ranks the one-byte copies of
+    the groups' tables are made on one more stream after the histograms, and the reassignments wait for them."""
+    cfg = W.get_config(base).replace(L=L, **over)        # L x 64 x 4 chunks: 9 layers make four groups, 13 make six
     topk = _routing(cfg)
     monkeypatch.setenv("TAOT_PLAN_GROUPS", "1")
     single = make_planner(cfg)
@@ -244,7 +245,8 @@ def test_layer_groups_on_internal_streams_change_no_bit_and_can_be_captured(monk
     pl.plan(topk, out)
     torch.cuda.synchronize()
     n1 = single.last_launch_count()
-    assert pl.last_launch_count() == G * n1                     # G groups, the same kernels each
+    # G groups, the same kernels each; at 256 ranks the one-byte copy of each group's table is a launch of its own
+    assert pl.last_launch_count() in (G * n1, G * (n1 + 1))
     for key, val in out.items():
         assert (cpu(val) == want[key]).all(), key
     pl.set_profiling(3)
